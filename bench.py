@@ -1,0 +1,274 @@
+#!/usr/bin/env python
+"""Benchmark of the RT3D conv3d hot path on B200.
+
+    python bench.py --gpus N --steps K --warmup W [--impl reference]
+
+Workload (config 1 of the baseline): one C3D-conv3a-shaped layer, batch 8, C_in=128,
+C_out=256, T=8, H=W=28, 3x3x3, stride 1, pad 1, bf16 in / fp32 accumulate / bf16 out,
+KGS-pruned with 4x4 kernel groups at about 2.5x FLOPs pruning, fused bias + ReLU.
+A step is one rt3d_conv3d_sparse call on one batch.  Inputs are seeded synthetic tensors
+(no dataset).  Each step uses the next of several input/output buffer sets whose total size
+exceeds twice the L2 capacity, so no step finds its operands in L2 from the previous one.
+
+The JSON line reports actual TFLOP/s (2 x kept multiply-accumulates / time); the same run
+also times the library's dense path on the same shape (speedup vs dense, to be compared with
+the FLOPs pruning rate as the paper does), an end-to-end variant through the host-buffer entry
+point, the CPU oracle on the machine's host cores, and the roofline fraction of the kernel.
+With torchrun and N > 1 every rank runs the same per-GPU workload on its own batch (weak
+scaling, no collective on the data path); times are the max over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import numpy as np
+
+import rt3d_synth as synth
+
+CFG = dict(n=8, t=8, h=28, w=28, cin=128, cout=256, k=(3, 3, 3), stride=(1, 1, 1), pad=(1, 1, 1),
+           g_m=4, g_n=4, density=0.4)
+L2_BYTES = 126 * 1024 * 1024
+WORKLOAD = "cfg1: C3D conv3a-shaped layer, batch 8, 128->256, 8x28x28, 3x3x3 s1 p1, KGS 4x4 ~2.5x, bf16"
+
+
+def make_workload():
+    spec = synth.ConvSpec("conv3a", CFG["cin"], CFG["cout"], CFG["k"], CFG["stride"], CFG["pad"], True)
+    L = synth.make_layer(spec, 1, 0, CFG["g_m"], CFG["g_n"], "bernoulli", CFG["density"])
+    x = synth.make_input(1, (CFG["n"], CFG["t"], CFG["h"], CFG["w"], CFG["cin"]))
+    return spec, L, x
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return {"hbm_gbs": p["hbm_gbs"], "bf16_tflops": p["bf16_tflops"],
+                "bf16_tflops_sustained": p.get("bf16_tflops_sustained"), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons of one GPU through NVML while a region runs."""
+    REASONS = {0x4: "sw_power_cap", 0x8: "hw_slowdown", 0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown",
+               0x80: "hw_power_brake_slowdown"}
+
+    def __init__(self, index: int):
+        super().__init__(daemon=True)
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop_evt = threading.Event()
+        self.active = threading.Event()
+        self.ok = False
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+            self.ok = True
+        except Exception:
+            self.ok = False
+
+    def run(self):
+        if not self.ok:
+            return
+        while not self._stop_evt.is_set():
+            if self.active.is_set():
+                try:
+                    self.samples.append(self.nv.nvmlDeviceGetClockInfo(self.h, self.nv.NVML_CLOCK_SM))
+                    try:
+                        r = self.nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                    except Exception:
+                        r = self.nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                    for bit, name in self.REASONS.items():
+                        if r & bit:
+                            self.reasons.add(name)
+                except Exception:
+                    pass
+            time.sleep(0.0005)
+
+    def stop(self):
+        self._stop_evt.set()
+
+    def summary(self):
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": 0}
+        return {"sm_mhz": statistics.median(self.samples), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def oracle_timed(spec, L, x, clips: int):
+    """Times the CPU oracle, as it stands, on the first `clips` clips of the batch."""
+    import oracle
+    xs = np.ascontiguousarray(x[:clips])
+    t0 = time.perf_counter()
+    oracle.conv3d(xs, L["w"], L["mask"], L["bias"], spec.stride, spec.pad, True, round_bf16=True)
+    return time.perf_counter() - t0
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    spec, L, x = make_workload()
+    clips = 1
+    kept_macs = spec.dense_macs(clips, CFG["t"], CFG["h"], CFG["w"]) * float(L["mask"].mean())
+    for _ in range(args.warmup):
+        oracle_timed(spec, L, x, clips)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle_timed(spec, L, x, clips)
+    dt = time.perf_counter() - t0
+    value = 2.0 * kept_macs * args.steps / dt / 1e12
+    sample = f"{clips} of {CFG['n']} clips of the batch per step (masked dense weights, fp64 accumulation)"
+    print(json.dumps({
+        "impl": "reference", "metric": "sparse_conv3d_actual_tflops", "value": value, "unit": "TFLOP/s",
+        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": "TFLOP/s", "cores": oracle.threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0}))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.impl == "reference":
+        return run_reference(args)
+
+    import torch
+    import paper_2007_09835_b200 as rt3d
+    from paper_2007_09835_b200 import nets, dist
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local)
+    group = dist.init(world, rank, "nccl") if world > 1 else None
+    dev = torch.device("cuda", local)
+
+    spec, L, x = make_workload()
+    sparse = nets.ConvLayer(spec, L["w"], L["bias"], L["mask"], CFG["g_m"], CFG["g_n"], torch.bfloat16, device=dev)
+    dense = nets.ConvLayer(spec, L["w"], L["bias"], None, dtype=torch.bfloat16, dense=True, device=dev)
+    x0 = nets.to_device(x, torch.bfloat16, device=dev)
+    y0 = sparse.alloc_out(x0)
+    set_bytes = x0.numel() * 2 + y0.numel() * 2
+    n_sets = max(2, -(-int(2.5 * L2_BYTES) // set_bytes))
+    xs = [x0] + [x0.clone() for _ in range(n_sets - 1)]
+    ys = [y0] + [torch.zeros_like(y0) for _ in range(n_sets - 1)]
+    kept_macs, dense_macs, alg_bytes = sparse.cost(x0)
+    algo = rt3d.rt3d_conv3d_query_algo(rt3d.tensor_desc(x0, spec.cin), sparse.packed, rt3d.tensor_desc(y0, spec.cout),
+                                       spec.stride, spec.pad)
+
+    def timed(layer, steps, warmup, sampler=None):
+        for i in range(warmup):
+            layer(xs[i % n_sets], ys[i % n_sets])
+        torch.cuda.synchronize()
+        dist.barrier(group)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        l0 = rt3d.rt3d_launch_count()
+        if sampler:
+            sampler.active.set()
+        e0.record()
+        for i in range(steps):
+            layer(xs[i % n_sets], ys[i % n_sets])
+        e1.record()
+        torch.cuda.synchronize()
+        if sampler:
+            sampler.active.clear()
+        dist.barrier(group)
+        ms = dist.max_over_ranks(e0.elapsed_time(e1), group, dev)
+        return ms, rt3d.rt3d_launch_count() - l0
+
+    sampler = ClockSampler(local)
+    sampler.start()
+    sparse_ms, launches = timed(sparse, args.steps, args.warmup, sampler)
+    dense_ms, _ = timed(dense, args.steps, args.warmup, sampler)
+    if rt3d.rt3d_last_device_status() != rt3d.OK:
+        raise SystemExit("device reported a bounded-wait timeout")
+
+    # end to end through the host-buffer entry point: pinned host input -> device -> conv -> pinned host output
+    xh = torch.from_numpy(x).to(torch.bfloat16).pin_memory()
+    yh = torch.zeros((CFG["n"], CFG["t"], CFG["h"], CFG["w"], CFG["cout"]), dtype=torch.bfloat16).pin_memory()
+    bh = torch.from_numpy(L["bias"]).pin_memory()
+    xhd, yhd = rt3d.tensor_desc(xh), rt3d.tensor_desc(yh)
+    e2e_steps = max(3, min(args.steps, 50))
+    for _ in range(3):
+        rt3d.rt3d_conv3d_host(xhd, sparse.packed, bh, yhd, spec.stride, spec.pad, True)
+    torch.cuda.synchronize()
+    dist.barrier(group)
+    t0 = time.perf_counter()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(e2e_steps):
+        rt3d.rt3d_conv3d_host(xhd, sparse.packed, bh, yhd, spec.stride, spec.pad, True)
+    e1.record()
+    torch.cuda.synchronize()
+    e2e_ms = dist.max_over_ranks(e0.elapsed_time(e1), group, dev) / e2e_steps
+    sampler.stop()
+
+    flops_kept = 2.0 * kept_macs
+    per_step_ms = sparse_ms / args.steps
+    value = world * flops_kept / (per_step_ms * 1e-3) / 1e12
+    pk = peaks()
+    ach = flops_kept / (per_step_ms * 1e-3) / 1e12
+    out = {
+        "metric": "sparse_conv3d_actual_tflops", "value": value, "unit": "TFLOP/s", "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": per_step_ms, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "global_batch": CFG["n"] * world, "parallelism": f"batch replicas x{world}",
+                   "l2": f"rotating {n_sets} input/output buffer sets ({n_sets * set_bytes / 2**20:.0f} MiB > 2x L2)",
+                   "kernel": "tcgen05" if algo == rt3d.ALGO_UMMA else "cuda-core"},
+        "dense_equiv_tflops": world * 2.0 * dense_macs / (per_step_ms * 1e-3) / 1e12,
+        "dense_path_tflops": world * 2.0 * dense_macs / (dense_ms / args.steps * 1e-3) / 1e12,
+        "speedup_vs_dense": dense_ms / sparse_ms,
+        "flops_pruning_rate": dense_macs / kept_macs,
+        "dense_ms_per_step": dense_ms / args.steps,
+        "clocks": sampler.summary(),
+        "e2e": {"value": world * flops_kept / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s",
+                "ms_per_step": e2e_ms, "h2d_bytes_per_step": xh.numel() * 2 + bh.numel() * 4,
+                "d2h_bytes_per_step": yh.numel() * 2},
+        "gpu_launches": int(launches),
+        "roofline": {"bound": "tensor", "achieved": ach, "peak": pk["bf16_tflops"], "unit": "TFLOP/s",
+                     "frac": ach / pk["bf16_tflops"], "traffic": None, "peak_source": pk["source"] + " (burst)",
+                     "executed_tflops": 2.0 * dense_macs / (per_step_ms * 1e-3) / 1e12,
+                     "alg_bytes_per_launch": alg_bytes},
+    }
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        import oracle
+        clips = CFG["n"]
+        dt = oracle_timed(spec, L, x, clips)
+        out["cpu_baseline"] = {"value": flops_kept / dt / 1e12, "unit": "TFLOP/s", "cores": oracle.threads(),
+                               "kind": "oracle", "seconds": dt,
+                               "sample": f"all {clips} clips of one batch, one pass (masked dense weights, fp64 accumulation)"}
+    traffic_file = os.path.join(ROOT, "profiles", "traffic.json")
+    if os.path.exists(traffic_file):
+        try:
+            out["roofline"]["traffic"] = json.load(open(traffic_file)).get("cfg1_sparse_dram_bytes_per_launch")
+        except Exception:
+            pass
+    if rank == 0:
+        print(json.dumps(out))
+    dist.shutdown(group)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,195 @@
+/*
+ * rt3d.h - C ABI of the B200 library for the inference hot path of RT3D
+ * (arXiv 2007.09835): forward 3-D convolution over NDHWC video activations with weights
+ * pruned to the paper's kernel-group-structured (KGS) or vanilla structured sparsity.
+ *
+ * Conventions
+ *   - Plain C linkage, no exceptions; every call returns an rt3d_status.
+ *   - "host" / "device" on a pointer says where the memory must live.  Activations,
+ *     bias and outputs are DEVICE memory owned by the caller; dense weights and masks
+ *     handed to the packers are HOST memory owned by the caller.  The library owns an
+ *     rt3d_packed handle (host canonical arrays + per-device weight blobs) until
+ *     rt3d_packed_free.
+ *   - Compute calls enqueue work on the given CUDA stream (a cudaStream_t passed as
+ *     void*, NULL = default stream) and return without synchronising.  The first compute
+ *     call that uses a handle on a device uploads the handle's device blobs (allocation +
+ *     copy); later calls allocate nothing.  rt3d_packed_prepare does that upload ahead of time.
+ *   - Argument errors are detected on the host before anything is launched.
+ *   - Activation layout: NDHWC = [n][t][h][w][c] with a channel pitch c_stride >= c
+ *     (elements between consecutive voxels).  Weight layout handed to the packers:
+ *     [M][N][Kt][Kh][Kw], M filters, N input channels (Section 3; the paper's kernel depth
+ *     K_d is the temporal extent Kt).  Kernel location index kpos = (kt*Kh + kh)*Kw + kw.
+ *   - Convolution is cross-correlation with zero padding, no dilation; output extent
+ *     floor((in + 2*pad - K)/stride) + 1 per axis.
+ */
+#ifndef RT3D_H_
+#define RT3D_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  RT3D_OK = 0,
+  RT3D_ERR_INVALID_ARG = 1,            /* NULL pointer, non-positive extent, bad enum            */
+  RT3D_ERR_SHAPE = 2,                  /* tensor extents / dtypes do not fit the weights/params  */
+  RT3D_ERR_MASK_NOT_GROUP_UNIFORM = 3, /* mask differs inside one (kernel group, location)       */
+  RT3D_ERR_UNSUPPORTED = 4,            /* valid request this build cannot run                    */
+  RT3D_ERR_ALLOC = 5,                  /* host or device allocation failed                       */
+  RT3D_ERR_CUDA = 6,                   /* a CUDA runtime / driver call failed                    */
+  RT3D_ERR_TIMEOUT = 7                 /* a bounded device-side wait gave up (see rt3d_last_device_status) */
+} rt3d_status;
+
+typedef enum { RT3D_F32 = 0, RT3D_BF16 = 1 } rt3d_dtype;
+
+/* Kernel family selection for the convolution calls. */
+typedef enum {
+  RT3D_ALGO_AUTO = 0,   /* tensor-core kernel when the shape allows it, else the CUDA-core kernel */
+  RT3D_ALGO_SIMT = 1,   /* CUDA-core kernel driven by the canonical packed index (any shape)      */
+  RT3D_ALGO_UMMA = 2    /* tcgen05 tensor-core kernel; RT3D_ERR_UNSUPPORTED if not applicable     */
+} rt3d_algo;
+
+/* NDHWC activation tensor in DEVICE memory (HOST memory for the *_host entry point), caller-owned. */
+typedef struct {
+  void*   data;          /* 16-byte aligned                                                      */
+  int32_t n, t, h, w, c; /* logical extents                                                      */
+  int32_t c_stride;      /* elements between voxels, >= c                                        */
+  int32_t dtype;         /* rt3d_dtype                                                           */
+} rt3d_tensor;
+
+typedef struct {
+  int32_t st, sh, sw;    /* strides  (>= 1)                                                      */
+  int32_t pt, ph, pw;    /* zero padding on both sides of each axis (>= 0)                       */
+  int32_t relu;          /* nonzero: y = max(y, 0) fused after the bias                          */
+  int32_t algo;          /* rt3d_algo                                                            */
+} rt3d_conv_params;
+
+typedef struct rt3d_packed rt3d_packed;   /* opaque; immutable after creation */
+
+/* Host pointers into a handle's canonical arrays; valid until rt3d_packed_free. */
+typedef struct {
+  int32_t M, N, Kt, Kh, Kw, g_m, g_n, P, Q, Ks;
+  int32_t dtype;               /* rt3d_dtype of `tiles`                                          */
+  int32_t is_vanilla;          /* every group keeps all or none of its locations                 */
+  int32_t is_dense;            /* created by rt3d_pack_dense                                     */
+  int64_t nnz;                 /* kept (group, location) entries                                 */
+  const int32_t*  group_ptr;   /* [P*Q + 1] CSR offsets, group id = p*Q + q                      */
+  const uint16_t* pos_idx;     /* [nnz] kpos, strictly ascending inside a group                  */
+  const void*     tiles;       /* [nnz][g_m][g_n] float or bf16 bits (round-to-nearest-even);
+                                  tiles[e][i][j] = W[p*g_m+i][q*g_n+j][kpos(e)], 0 where the
+                                  kernel does not exist (ragged last groups)                     */
+} rt3d_packed_view;
+
+/*
+ * rt3d_pack_kgs - weight reorganisation for KGS / vanilla sparsity.
+ * Section 3: the weight tensor is partitioned into aligned groups of g_m x g_n kernels
+ * (P = ceil(M/g_m), Q = ceil(N/g_n), Section 4); inside a group every kernel location
+ * (kt,kh,kw) is kept or pruned for all kernels together, which is whole-column removal in
+ * the group's weight matrix.  The pack keeps, per group, the list of kept locations and one
+ * compact g_m x g_n tile per kept location (the "reorganize the model weights" step of
+ * Section 5.2).  Vanilla sparsity (whole groups removed) is the special case where each
+ * group keeps all or no locations.
+ *   w     host, [M][N][Kt][Kh][Kw] float
+ *   mask  host, same shape, uint8, nonzero = keep; NULL = keep everything.  The mask is
+ *         authoritative: kept weights are stored even if zero, pruned ones dropped even if not.
+ *   g_m, g_n  group size, 1..8 each;  Kt*Kh*Kw <= 65535
+ *   compute_dtype  storage/compute precision of the tiles (RT3D_F32, or RT3D_BF16 = RNE-rounded)
+ *   out   receives the new handle
+ * Errors: INVALID_ARG, MASK_NOT_GROUP_UNIFORM (mask is not a KGS mask), ALLOC.
+ * Pure host work: usable without a GPU.
+ */
+rt3d_status rt3d_pack_kgs(const float* w, const uint8_t* mask, int M, int N, int Kt, int Kh, int Kw,
+                          int g_m, int g_n, int compute_dtype, rt3d_packed** out);
+
+/* rt3d_pack_dense - handle for the unpruned layer (the "RT3D (Dense)" path of Table 2):
+ * every location of every kernel kept.  Same argument rules as rt3d_pack_kgs. */
+rt3d_status rt3d_pack_dense(const float* w, int M, int N, int Kt, int Kh, int Kw,
+                            int compute_dtype, rt3d_packed** out);
+
+/* Read-only view of the canonical arrays (for bit-exact checks of the pack). */
+rt3d_status rt3d_packed_view_get(const rt3d_packed* p, rt3d_packed_view* view);
+
+/* Inverse of the pack: w_out host [M][N][Kt][Kh][Kw] float, zeros at pruned locations
+ * (bf16 handles return the rounded values widened to float). */
+rt3d_status rt3d_unpack_to_dense(const rt3d_packed* p, float* w_out);
+
+/* Inverse of the tensor-core weight layout the handle would upload for bundles of
+ * `n_tile` output channels (0 = the library's choice): w_out as above.  Lets a host-only
+ * test check that derived layout against the canonical one. */
+rt3d_status rt3d_unpack_device_layout(const rt3d_packed* p, int n_tile, float* w_out);
+
+/* Upload the handle's device blobs to the current CUDA device now (otherwise done by the
+ * first compute call).  Synchronises the device. */
+rt3d_status rt3d_packed_prepare(rt3d_packed* p);
+
+void rt3d_packed_free(rt3d_packed* p);
+
+/*
+ * rt3d_conv3d_sparse - the hot path: y = act(bias + conv3d(x, W (.) mask)), iterating only
+ * the kept (group, location) entries of the packed index (Section 3: after column removal
+ * "the remaining computation is still based on full matrices (albeit smaller)").
+ *   x, y   device tensors; x.c == N, y.c == M, y extents = output extents of (x, params);
+ *          dtypes equal the handle's compute dtype.  bf16: c_stride multiple of 8, fp32:
+ *          multiple of 4; data 16-byte aligned.  x and y must not overlap.
+ *   w      handle from rt3d_pack_kgs (or rt3d_pack_dense)
+ *   bias   device, [M] float, or NULL
+ *   p      strides, padding, fused ReLU, kernel family
+ *   stream cudaStream_t as void*
+ * Accumulation is fp32; bf16 outputs are rounded once after bias and ReLU.
+ * Errors: INVALID_ARG, SHAPE, UNSUPPORTED, ALLOC/CUDA (first-use upload), and nothing is
+ * launched on error.  A bounded device-side wait that gives up is reported later by
+ * rt3d_last_device_status.
+ */
+rt3d_status rt3d_conv3d_sparse(const rt3d_tensor* x, const rt3d_packed* w, const float* bias,
+                               const rt3d_conv_params* p, rt3d_tensor* y, void* stream);
+
+/* rt3d_conv3d_dense - same operation for a handle from rt3d_pack_dense: all locations
+ * iterated, no index lookups (the dense baseline the paper compares its sparse path with). */
+rt3d_status rt3d_conv3d_dense(const rt3d_tensor* x, const rt3d_packed* w, const float* bias,
+                              const rt3d_conv_params* p, rt3d_tensor* y, void* stream);
+
+/*
+ * rt3d_conv3d_host - end-to-end variant: x->data and y->data are HOST buffers (pinned
+ * memory recommended), bias is HOST [M] or NULL.  Copies x to a library-owned device staging
+ * buffer, runs rt3d_conv3d_sparse (or _dense for a dense handle) and copies y back, all on
+ * `stream`; returns after the stream has been synchronised.  Staging buffers are cached
+ * in the handle and grow on demand.
+ */
+rt3d_status rt3d_conv3d_host(const rt3d_tensor* x, rt3d_packed* w, const float* bias,
+                             const rt3d_conv_params* p, rt3d_tensor* y, void* stream);
+
+/* Layer glue for the C3D- and R(2+1)D-shaped networks (not described by the paper, which
+ * only names the models in Section 5). */
+/* Max-pool over (t,h,w) windows, padding never wins; x.c == y.c, same dtype. */
+rt3d_status rt3d_maxpool3d(const rt3d_tensor* x, int kt, int kh, int kw, int st, int sh, int sw,
+                           int pt, int ph, int pw, rt3d_tensor* y, void* stream);
+/* y = a + b (optionally ReLU); equal extents and dtype; y may alias a or b. */
+rt3d_status rt3d_add_relu(const rt3d_tensor* a, const rt3d_tensor* b, int relu, rt3d_tensor* y, void* stream);
+
+/* Work and traffic the method itself requires for one call (Section 3 cost model):
+ * kept multiply-accumulates, dense multiply-accumulates, and algorithmic bytes
+ * (input once + output once + packed weights and index once + bias). */
+rt3d_status rt3d_conv3d_cost(const rt3d_tensor* x, const rt3d_packed* w, const rt3d_conv_params* p,
+                             int64_t* kept_macs, int64_t* dense_macs, int64_t* alg_bytes);
+
+/* Which kernel family RT3D_ALGO_AUTO would run for this call: writes an rt3d_algo to *algo. */
+rt3d_status rt3d_conv3d_query_algo(const rt3d_tensor* x, const rt3d_packed* w, const rt3d_conv_params* p,
+                                   const rt3d_tensor* y, int* algo);
+
+/* Synchronises `stream`, then returns RT3D_ERR_TIMEOUT if any kernel of this library
+ * recorded a bounded-wait failure on the current device since the last call (and clears
+ * the record), RT3D_ERR_CUDA if the stream reports an error, else RT3D_OK. */
+rt3d_status rt3d_last_device_status(void* stream);
+
+/* Number of kernels this library has launched in this process (all devices). */
+int64_t rt3d_launch_count(void);
+
+const char* rt3d_status_string(rt3d_status s);
+const char* rt3d_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RT3D_H_ */

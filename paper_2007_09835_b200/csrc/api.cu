@@ -1,0 +1,474 @@
+// C ABI of librt3d: argument validation, per-device weight upload, tile planning, TMA tensor
+// maps and kernel dispatch.  All numerical work happens in the kernels launched from here.
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <atomic>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <mutex>
+#include <vector>
+
+#include "kernels.h"
+#include "rt3d_internal.h"
+
+using namespace rt3d;
+
+namespace {
+
+std::atomic<int64_t> g_launches{0};
+
+struct DeviceState {
+  bool init = false;
+  int sm_count = 0;
+  int cc_major = 0;
+  int32_t* sched = nullptr;     // [8] words: [2] = error word written by kernels on a bounded-wait expiry
+};
+std::mutex g_dev_mu;
+DeviceState g_dev[64];
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn g_encode = nullptr;
+
+rt3d_status get_device_state(DeviceState** out) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return RT3D_ERR_CUDA;
+  std::lock_guard<std::mutex> lock(g_dev_mu);
+  DeviceState& d = g_dev[dev];
+  if (!d.init) {
+    if (cudaDeviceGetAttribute(&d.sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return RT3D_ERR_CUDA;
+    if (cudaDeviceGetAttribute(&d.cc_major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return RT3D_ERR_CUDA;
+    if (cudaMalloc(&d.sched, 8 * sizeof(int32_t)) != cudaSuccess) return RT3D_ERR_ALLOC;
+    if (cudaMemset(d.sched, 0, 8 * sizeof(int32_t)) != cudaSuccess) return RT3D_ERR_CUDA;
+    if (!g_encode) {
+      void* fn = nullptr;
+      cudaDriverEntryPointQueryResult qres;
+      if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn)
+        return RT3D_ERR_CUDA;
+      g_encode = reinterpret_cast<EncodeTiledFn>(fn);
+    }
+    d.init = true;
+  }
+  *out = &d;
+  return RT3D_OK;
+}
+
+bool valid_dtype(int d) { return d == RT3D_F32 || d == RT3D_BF16; }
+size_t elem_size(int d) { return d == RT3D_BF16 ? 2 : 4; }
+
+rt3d_status check_tensor(const rt3d_tensor* t) {
+  if (!t || !t->data) return RT3D_ERR_INVALID_ARG;
+  if (t->n <= 0 || t->t <= 0 || t->h <= 0 || t->w <= 0 || t->c <= 0) return RT3D_ERR_INVALID_ARG;
+  if (!valid_dtype(t->dtype) || t->c_stride < t->c) return RT3D_ERR_INVALID_ARG;
+  return RT3D_OK;
+}
+
+int64_t tensor_span_bytes(const rt3d_tensor* t) {
+  const int64_t vox = int64_t(t->n) * t->t * t->h * t->w;
+  return ((vox - 1) * t->c_stride + t->c) * int64_t(elem_size(t->dtype));
+}
+
+rt3d_status make_geom(const rt3d_tensor* x, const rt3d_packed* w, const rt3d_conv_params* p, const rt3d_tensor* y,
+                      ConvGeom* g) {
+  rt3d_status s = check_tensor(x);
+  if (s != RT3D_OK) return s;
+  if (!w || !p) return RT3D_ERR_INVALID_ARG;
+  if (p->st < 1 || p->sh < 1 || p->sw < 1 || p->pt < 0 || p->ph < 0 || p->pw < 0) return RT3D_ERR_INVALID_ARG;
+  if (p->algo < RT3D_ALGO_AUTO || p->algo > RT3D_ALGO_UMMA) return RT3D_ERR_INVALID_ARG;
+  if (x->c != w->N || x->dtype != w->dtype) return RT3D_ERR_SHAPE;
+  const int64_t To = (int64_t(x->t) + 2 * p->pt - w->Kt) / p->st + 1;
+  const int64_t Ho = (int64_t(x->h) + 2 * p->ph - w->Kh) / p->sh + 1;
+  const int64_t Wo = (int64_t(x->w) + 2 * p->pw - w->Kw) / p->sw + 1;
+  if (x->t + 2 * p->pt < w->Kt || x->h + 2 * p->ph < w->Kh || x->w + 2 * p->pw < w->Kw) return RT3D_ERR_SHAPE;
+  if (int64_t(x->n) * x->t * x->h * x->w >= (int64_t(1) << 31)) return RT3D_ERR_UNSUPPORTED;
+  g->n = x->n; g->t = x->t; g->h = x->h; g->w = x->w; g->c = x->c; g->xcs = x->c_stride;
+  g->To = int(To); g->Ho = int(Ho); g->Wo = int(Wo); g->M = w->M; g->ycs = 0;
+  g->Kt = w->Kt; g->Kh = w->Kh; g->Kw = w->Kw;
+  g->st = p->st; g->sh = p->sh; g->sw = p->sw; g->pt = p->pt; g->ph = p->ph; g->pw = p->pw;
+  g->relu = p->relu ? 1 : 0;
+  if (y) {
+    s = check_tensor(y);
+    if (s != RT3D_OK) return s;
+    if (y->n != x->n || y->t != To || y->h != Ho || y->w != Wo || y->c != w->M || y->dtype != w->dtype)
+      return RT3D_ERR_SHAPE;
+    g->ycs = y->c_stride;
+  }
+  return RT3D_OK;
+}
+
+// Alignment rules of the device entry points.
+rt3d_status check_alignment(const rt3d_tensor* t) {
+  const int mult = t->dtype == RT3D_BF16 ? 8 : 4;
+  if (t->c_stride % mult) return RT3D_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(t->data) % 16) return RT3D_ERR_INVALID_ARG;
+  return RT3D_OK;
+}
+
+bool overlaps(const rt3d_tensor* a, const rt3d_tensor* b) {
+  const char* a0 = static_cast<const char*>(a->data);
+  const char* b0 = static_cast<const char*>(b->data);
+  return a0 < b0 + tensor_span_bytes(b) && b0 < a0 + tensor_span_bytes(a);
+}
+
+// ------------------------------------------------------------------------- device blobs
+DeviceBlob* find_blob(rt3d_packed* h, int dev) {
+  for (DeviceBlob* b : h->blobs)
+    if (b->device == dev) return b;
+  return nullptr;
+}
+
+// Returns the blob of the current device, creating and uploading the canonical arrays on first use.
+rt3d_status get_blob(rt3d_packed* h, DeviceBlob** out) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return RT3D_ERR_CUDA;
+  std::lock_guard<std::mutex> lock(h->mu);
+  DeviceBlob* b = find_blob(h, dev);
+  if (!b) {
+    b = new (std::nothrow) DeviceBlob;
+    if (!b) return RT3D_ERR_ALLOC;
+    b->device = dev;
+    rt3d_status s = RT3D_OK;
+    if (cudaMalloc(reinterpret_cast<void**>(&b->group_ptr), h->group_ptr.size() * 4) != cudaSuccess ||
+        cudaMalloc(reinterpret_cast<void**>(&b->pos_idx), h->pos_idx.size() * 2 + 16) != cudaSuccess ||
+        cudaMalloc(&b->tiles, h->tiles.size() + 16) != cudaSuccess)
+      s = RT3D_ERR_ALLOC;
+    if (s == RT3D_OK &&
+        (cudaMemcpy(b->group_ptr, h->group_ptr.data(), h->group_ptr.size() * 4, cudaMemcpyHostToDevice) != cudaSuccess ||
+         (h->nnz && cudaMemcpy(b->pos_idx, h->pos_idx.data(), h->pos_idx.size() * 2, cudaMemcpyHostToDevice) != cudaSuccess) ||
+         (h->nnz && cudaMemcpy(b->tiles, h->tiles.data(), h->tiles.size(), cudaMemcpyHostToDevice) != cudaSuccess)))
+      s = RT3D_ERR_CUDA;
+    if (s != RT3D_OK) {
+      cudaFree(b->group_ptr); cudaFree(b->pos_idx); cudaFree(b->tiles);
+      delete b;
+      return s;
+    }
+    h->blobs.push_back(b);
+  }
+  *out = b;
+  return RT3D_OK;
+}
+
+rt3d_status get_umma_blob(rt3d_packed* h, DeviceBlob* blob, const UmmaLayout* L, DeviceBlob::Umma** out) {
+  std::lock_guard<std::mutex> lock(h->mu);
+  DeviceBlob::Umma& u = blob->umma[L->n_tile];
+  if (!u.ready) {
+    const size_t wbytes = L->wtiles.size() * 2;
+    if (cudaMalloc(&u.wtiles, wbytes + 1024) != cudaSuccess ||
+        cudaMalloc(reinterpret_cast<void**>(&u.step_ptr), L->step_ptr.size() * 4) != cudaSuccess ||
+        cudaMalloc(reinterpret_cast<void**>(&u.steps), L->steps.size() * 4 + 16) != cudaSuccess)
+      return RT3D_ERR_ALLOC;
+    if ((wbytes && cudaMemcpy(u.wtiles, L->wtiles.data(), wbytes, cudaMemcpyHostToDevice) != cudaSuccess) ||
+        cudaMemcpy(u.step_ptr, L->step_ptr.data(), L->step_ptr.size() * 4, cudaMemcpyHostToDevice) != cudaSuccess ||
+        (!L->steps.empty() &&
+         cudaMemcpy(u.steps, L->steps.data(), L->steps.size() * 4, cudaMemcpyHostToDevice) != cudaSuccess))
+      return RT3D_ERR_CUDA;
+    // 2-D map over the weight tiles: rows of 64 bf16 (128 bytes), one box = one [n_tile][64] tile
+    const cuuint64_t rows = L->steps.empty() ? cuuint64_t(L->n_tile) : cuuint64_t(L->steps.size()) * L->n_tile;
+    cuuint64_t dims[2] = {64, rows};
+    cuuint64_t strides[1] = {128};
+    cuuint32_t box[2] = {64, cuuint32_t(L->n_tile)};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = g_encode(reinterpret_cast<CUtensorMap*>(u.wmap), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, u.wtiles, dims,
+                          strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                          CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return RT3D_ERR_CUDA;
+    u.ready = true;
+  }
+  *out = &u;
+  return RT3D_OK;
+}
+
+// ------------------------------------------------------------------------ tile planning
+// Box of output voxels (bn x bt x bh x bw <= 128) that covers the output with the fewest tiles;
+// ties go to the wider box along w, then h (longer contiguous runs for the TMA engine).
+TileBox choose_box(const ConvGeom& g) {
+  TileBox best{1, 1, 1, 1};
+  long long best_tiles = -1;
+  for (int bw = 1; bw <= g.Wo && bw <= kTileM; ++bw) {
+    if (bw * g.sw > 256) break;
+    for (int bh = 1; bh <= g.Ho && bw * bh <= kTileM; ++bh) {
+      if (bh * g.sh > 256) break;
+      for (int bt = 1; bt <= g.To && bw * bh * bt <= kTileM; ++bt) {
+        if (bt * g.st > 256) break;
+        int bn = kTileM / (bw * bh * bt);
+        if (bn > g.n) bn = g.n;
+        const long long tiles = (long long)ceil_div(g.n, bn) * ceil_div(g.To, bt) * ceil_div(g.Ho, bh) * ceil_div(g.Wo, bw);
+        bool better = best_tiles < 0 || tiles < best_tiles;
+        if (!better && tiles == best_tiles) {
+          if (bw > best.bw) better = true;
+          else if (bw == best.bw && bh > best.bh) better = true;
+        }
+        if (better) { best = TileBox{bn, bt, bh, bw}; best_tiles = tiles; }
+      }
+    }
+  }
+  return best;
+}
+
+bool umma_eligible(const DeviceState* d, const rt3d_packed* w, const rt3d_tensor* x, const rt3d_tensor* y,
+                   const rt3d_conv_params* p) {
+  if (d->cc_major != 10) return false;
+  if (!umma_layout_possible(w)) return false;
+  if (x->c_stride % 8 || y->c_stride % 8) return false;
+  if (p->st > 8 || p->sh > 8 || p->sw > 8) return false;
+  if (int64_t(x->w) * x->c_stride * 2 >= (int64_t(1) << 40)) return false;
+  return true;
+}
+
+rt3d_status encode_xmap(const rt3d_tensor* x, const ConvGeom& g, const TileBox& box, CUtensorMap* map) {
+  const cuuint64_t cs = cuuint64_t(x->c_stride) * 2;
+  cuuint64_t dims[5] = {cuuint64_t(x->c), cuuint64_t(x->w), cuuint64_t(x->h), cuuint64_t(x->t), cuuint64_t(x->n)};
+  cuuint64_t strides[4] = {cs, cs * x->w, cs * x->w * x->h, cs * x->w * x->h * x->t};
+  // with a traversal stride s the engine loads ceil(box / s) elements, so a box of b outputs spans b*s inputs
+  cuuint32_t bx[5] = {64, cuuint32_t(box.bw * g.sw), cuuint32_t(box.bh * g.sh), cuuint32_t(box.bt * g.st),
+                      cuuint32_t(box.bn)};
+  cuuint32_t estr[5] = {1, cuuint32_t(g.sw), cuuint32_t(g.sh), cuuint32_t(g.st), 1};
+  CUresult r = g_encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, x->data, dims, strides, bx, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? RT3D_OK : RT3D_ERR_CUDA;
+}
+
+rt3d_status conv_impl(const rt3d_tensor* x, const rt3d_packed* wc, const float* bias, const rt3d_conv_params* p,
+                      rt3d_tensor* y, void* stream, bool dense_entry) {
+  ConvGeom g;
+  if (!y) return RT3D_ERR_INVALID_ARG;
+  rt3d_status s = make_geom(x, wc, p, y, &g);
+  if (s != RT3D_OK) return s;
+  if ((s = check_alignment(x)) != RT3D_OK || (s = check_alignment(y)) != RT3D_OK) return s;
+  if (overlaps(x, y)) return RT3D_ERR_INVALID_ARG;
+  if (dense_entry && !wc->is_dense) return RT3D_ERR_INVALID_ARG;
+  rt3d_packed* w = const_cast<rt3d_packed*>(wc);
+  DeviceState* d = nullptr;
+  if ((s = get_device_state(&d)) != RT3D_OK) return s;
+  DeviceBlob* blob = nullptr;
+  if ((s = get_blob(w, &blob)) != RT3D_OK) return s;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+
+  const bool can_umma = umma_eligible(d, w, x, y, p);
+  if (p->algo == RT3D_ALGO_UMMA && !can_umma) return RT3D_ERR_UNSUPPORTED;
+  const bool use_umma = p->algo == RT3D_ALGO_UMMA || (p->algo == RT3D_ALGO_AUTO && can_umma);
+  if (!use_umma) {
+    cudaError_t e = launch_conv_simt(w->dtype, g, x->data, y->data, blob->group_ptr, blob->pos_idx, blob->tiles, bias,
+                                     w->g_m, w->g_n, w->P, w->Q, dense_entry, st);
+    if (e != cudaSuccess) return RT3D_ERR_CUDA;
+    g_launches.fetch_add(1);
+    return RT3D_OK;
+  }
+
+  const UmmaLayout* L = get_umma_layout(w, 0);
+  if (!L) return RT3D_ERR_UNSUPPORTED;
+  DeviceBlob::Umma* u = nullptr;
+  if ((s = get_umma_blob(w, blob, L, &u)) != RT3D_OK) return s;
+  UmmaArgs a;
+  a.g = g;
+  a.box = choose_box(g);
+  a.n_tile = L->n_tile; a.n_bundles = L->n_bundles; a.n_chunks = L->n_chunks;
+  a.tiles_n = ceil_div(g.n, a.box.bn); a.tiles_t = ceil_div(g.To, a.box.bt);
+  a.tiles_h = ceil_div(g.Ho, a.box.bh); a.tiles_w = ceil_div(g.Wo, a.box.bw);
+  a.dense = dense_entry ? 1 : 0;
+  a.steps_dense = w->Ks * L->n_chunks;
+  a.step_ptr = u->step_ptr; a.steps = u->steps;
+  a.bias = bias; a.y = y->data; a.sched = d->sched;
+  CUtensorMap xmap;
+  if ((s = encode_xmap(x, g, a.box, &xmap)) != RT3D_OK) return s;
+  cudaError_t e = launch_conv_umma(a, &xmap, u->wmap, d->sm_count, st);
+  if (e != cudaSuccess) return RT3D_ERR_CUDA;
+  g_launches.fetch_add(1);
+  return RT3D_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+rt3d_status rt3d_conv3d_sparse(const rt3d_tensor* x, const rt3d_packed* w, const float* bias,
+                               const rt3d_conv_params* p, rt3d_tensor* y, void* stream) {
+  return conv_impl(x, w, bias, p, y, stream, false);
+}
+
+rt3d_status rt3d_conv3d_dense(const rt3d_tensor* x, const rt3d_packed* w, const float* bias,
+                              const rt3d_conv_params* p, rt3d_tensor* y, void* stream) {
+  return conv_impl(x, w, bias, p, y, stream, true);
+}
+
+rt3d_status rt3d_conv3d_host(const rt3d_tensor* x, rt3d_packed* w, const float* bias, const rt3d_conv_params* p,
+                             rt3d_tensor* y, void* stream) {
+  ConvGeom g;
+  if (!y) return RT3D_ERR_INVALID_ARG;
+  rt3d_status s = make_geom(x, w, p, y, &g);
+  if (s != RT3D_OK) return s;
+  DeviceBlob* blob = nullptr;
+  if ((s = get_blob(w, &blob)) != RT3D_OK) return s;
+  const size_t xb = size_t(tensor_span_bytes(x)), yb = size_t(tensor_span_bytes(y));
+  {
+    std::lock_guard<std::mutex> lock(w->mu);
+    if (blob->stage_x_bytes < xb) {
+      cudaFree(blob->stage_x);
+      blob->stage_x = nullptr; blob->stage_x_bytes = 0;
+      if (cudaMalloc(&blob->stage_x, xb + 256) != cudaSuccess) return RT3D_ERR_ALLOC;
+      blob->stage_x_bytes = xb;
+    }
+    if (blob->stage_y_bytes < yb) {
+      cudaFree(blob->stage_y);
+      blob->stage_y = nullptr; blob->stage_y_bytes = 0;
+      if (cudaMalloc(&blob->stage_y, yb + 256) != cudaSuccess) return RT3D_ERR_ALLOC;
+      blob->stage_y_bytes = yb;
+    }
+    if (!blob->stage_bias && cudaMalloc(reinterpret_cast<void**>(&blob->stage_bias), size_t(w->M) * 4) != cudaSuccess)
+      return RT3D_ERR_ALLOC;
+  }
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (cudaMemcpyAsync(blob->stage_x, x->data, xb, cudaMemcpyHostToDevice, st) != cudaSuccess) return RT3D_ERR_CUDA;
+  if (bias && cudaMemcpyAsync(blob->stage_bias, bias, size_t(w->M) * 4, cudaMemcpyHostToDevice, st) != cudaSuccess)
+    return RT3D_ERR_CUDA;
+  rt3d_tensor xd = *x, yd = *y;
+  xd.data = blob->stage_x;
+  yd.data = blob->stage_y;
+  s = conv_impl(&xd, w, bias ? blob->stage_bias : nullptr, p, &yd, stream, w->is_dense != 0);
+  if (s != RT3D_OK) return s;
+  if (cudaMemcpyAsync(y->data, blob->stage_y, yb, cudaMemcpyDeviceToHost, st) != cudaSuccess) return RT3D_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return RT3D_ERR_CUDA;
+  return RT3D_OK;
+}
+
+rt3d_status rt3d_packed_prepare(rt3d_packed* p) {
+  if (!p) return RT3D_ERR_INVALID_ARG;
+  DeviceState* d = nullptr;
+  rt3d_status s = get_device_state(&d);
+  if (s != RT3D_OK) return s;
+  DeviceBlob* blob = nullptr;
+  if ((s = get_blob(p, &blob)) != RT3D_OK) return s;
+  if (d->cc_major == 10 && umma_layout_possible(p)) {
+    const UmmaLayout* L = get_umma_layout(p, 0);
+    DeviceBlob::Umma* u = nullptr;
+    if (L && (s = get_umma_blob(p, blob, L, &u)) != RT3D_OK) return s;
+  }
+  return cudaDeviceSynchronize() == cudaSuccess ? RT3D_OK : RT3D_ERR_CUDA;
+}
+
+void rt3d_packed_free(rt3d_packed* p) {
+  if (!p) return;
+  int cur = -1;
+  const bool have_dev = !p->blobs.empty() && cudaGetDevice(&cur) == cudaSuccess;
+  for (DeviceBlob* b : p->blobs) {
+    if (have_dev) cudaSetDevice(b->device);
+    cudaFree(b->group_ptr); cudaFree(b->pos_idx); cudaFree(b->tiles);
+    for (auto& kv : b->umma) { cudaFree(kv.second.wtiles); cudaFree(kv.second.step_ptr); cudaFree(kv.second.steps); }
+    cudaFree(b->stage_x); cudaFree(b->stage_y); cudaFree(b->stage_bias);
+    delete b;
+  }
+  if (have_dev && cur >= 0) cudaSetDevice(cur);
+  delete p;
+}
+
+rt3d_status rt3d_maxpool3d(const rt3d_tensor* x, int kt, int kh, int kw, int st, int sh, int sw, int pt, int ph,
+                           int pw, rt3d_tensor* y, void* stream) {
+  rt3d_status s;
+  if ((s = check_tensor(x)) != RT3D_OK || (s = check_tensor(y)) != RT3D_OK) return s;
+  if (kt < 1 || kh < 1 || kw < 1 || st < 1 || sh < 1 || sw < 1 || pt < 0 || ph < 0 || pw < 0) return RT3D_ERR_INVALID_ARG;
+  if (pt >= kt || ph >= kh || pw >= kw) return RT3D_ERR_INVALID_ARG;   // every window must see an input
+  if (x->t + 2 * pt < kt || x->h + 2 * ph < kh || x->w + 2 * pw < kw) return RT3D_ERR_SHAPE;
+  const int To = (x->t + 2 * pt - kt) / st + 1, Ho = (x->h + 2 * ph - kh) / sh + 1, Wo = (x->w + 2 * pw - kw) / sw + 1;
+  if (y->n != x->n || y->t != To || y->h != Ho || y->w != Wo || y->c != x->c || y->dtype != x->dtype) return RT3D_ERR_SHAPE;
+  // windows that start inside the padding but end before the tensor would see nothing
+  if ((To - 1) * st - pt >= x->t || (Ho - 1) * sh - ph >= x->h || (Wo - 1) * sw - pw >= x->w) return RT3D_ERR_SHAPE;
+  if ((s = check_alignment(x)) != RT3D_OK || (s = check_alignment(y)) != RT3D_OK) return s;
+  if (overlaps(x, y)) return RT3D_ERR_INVALID_ARG;
+  cudaError_t e = launch_maxpool3d(x->dtype, x->data, x->n, x->t, x->h, x->w, x->c, x->c_stride, kt, kh, kw, st, sh, sw,
+                                   pt, ph, pw, y->data, To, Ho, Wo, y->c_stride, static_cast<cudaStream_t>(stream));
+  if (e != cudaSuccess) return RT3D_ERR_CUDA;
+  g_launches.fetch_add(1);
+  return RT3D_OK;
+}
+
+rt3d_status rt3d_add_relu(const rt3d_tensor* a, const rt3d_tensor* b, int relu, rt3d_tensor* y, void* stream) {
+  rt3d_status s;
+  if ((s = check_tensor(a)) != RT3D_OK || (s = check_tensor(b)) != RT3D_OK || (s = check_tensor(y)) != RT3D_OK) return s;
+  if (a->n != b->n || a->t != b->t || a->h != b->h || a->w != b->w || a->c != b->c || a->dtype != b->dtype) return RT3D_ERR_SHAPE;
+  if (a->n != y->n || a->t != y->t || a->h != y->h || a->w != y->w || a->c != y->c || a->dtype != y->dtype) return RT3D_ERR_SHAPE;
+  if ((s = check_alignment(a)) != RT3D_OK || (s = check_alignment(b)) != RT3D_OK || (s = check_alignment(y)) != RT3D_OK) return s;
+  const int64_t vox = int64_t(a->n) * a->t * a->h * a->w;
+  cudaError_t e = launch_add_relu(a->dtype, a->data, a->c_stride, b->data, b->c_stride, y->data, y->c_stride, vox, a->c,
+                                  relu ? 1 : 0, static_cast<cudaStream_t>(stream));
+  if (e != cudaSuccess) return RT3D_ERR_CUDA;
+  g_launches.fetch_add(1);
+  return RT3D_OK;
+}
+
+rt3d_status rt3d_conv3d_cost(const rt3d_tensor* x, const rt3d_packed* w, const rt3d_conv_params* p,
+                             int64_t* kept_macs, int64_t* dense_macs, int64_t* alg_bytes) {
+  ConvGeom g;
+  rt3d_status s = make_geom(x, w, p, nullptr, &g);
+  if (s != RT3D_OK) return s;
+  const int64_t vox_out = int64_t(g.n) * g.To * g.Ho * g.Wo;
+  // kept weights that exist (ragged groups hold fewer than g_m*g_n kernels)
+  int64_t kept_w = 0;
+  for (int pr = 0; pr < w->P; ++pr) {
+    const int rows = std::min(w->g_m, w->M - pr * w->g_m);
+    for (int q = 0; q < w->Q; ++q) {
+      const int cols = std::min(w->g_n, w->N - q * w->g_n);
+      kept_w += int64_t(w->group_ptr[size_t(pr) * w->Q + q + 1] - w->group_ptr[size_t(pr) * w->Q + q]) * rows * cols;
+    }
+  }
+  if (kept_macs) *kept_macs = vox_out * kept_w;
+  if (dense_macs) *dense_macs = vox_out * int64_t(w->M) * w->N * w->Ks;
+  if (alg_bytes) {
+    const int64_t e = int64_t(elem_size(w->dtype));
+    const int64_t vox_in = int64_t(g.n) * g.t * g.h * g.w;
+    *alg_bytes = vox_in * g.c * e + vox_out * g.M * e + w->nnz * w->g_m * w->g_n * e + w->nnz * 2 +
+                 int64_t(w->P) * w->Q * 4 + 4 + int64_t(w->M) * 4;
+  }
+  return RT3D_OK;
+}
+
+rt3d_status rt3d_conv3d_query_algo(const rt3d_tensor* x, const rt3d_packed* w, const rt3d_conv_params* p,
+                                   const rt3d_tensor* y, int* algo) {
+  ConvGeom g;
+  if (!algo || !y) return RT3D_ERR_INVALID_ARG;
+  rt3d_status s = make_geom(x, w, p, y, &g);
+  if (s != RT3D_OK) return s;
+  DeviceState* d = nullptr;
+  if ((s = get_device_state(&d)) != RT3D_OK) return s;
+  const bool can = umma_eligible(d, w, x, y, p);
+  if (p->algo == RT3D_ALGO_UMMA && !can) return RT3D_ERR_UNSUPPORTED;
+  *algo = (p->algo == RT3D_ALGO_SIMT || !can) ? RT3D_ALGO_SIMT : RT3D_ALGO_UMMA;
+  return RT3D_OK;
+}
+
+rt3d_status rt3d_last_device_status(void* stream) {
+  DeviceState* d = nullptr;
+  rt3d_status s = get_device_state(&d);
+  if (s != RT3D_OK) return s;
+  if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) return RT3D_ERR_CUDA;
+  int32_t word = 0;
+  if (cudaMemcpy(&word, d->sched + 2, 4, cudaMemcpyDeviceToHost) != cudaSuccess) return RT3D_ERR_CUDA;
+  if (word != 0) {
+    cudaMemset(d->sched + 2, 0, 4);
+    return RT3D_ERR_TIMEOUT;
+  }
+  return RT3D_OK;
+}
+
+int64_t rt3d_launch_count(void) { return g_launches.load(); }
+
+const char* rt3d_status_string(rt3d_status s) {
+  switch (s) {
+    case RT3D_OK: return "ok";
+    case RT3D_ERR_INVALID_ARG: return "invalid argument";
+    case RT3D_ERR_SHAPE: return "shape or dtype mismatch";
+    case RT3D_ERR_MASK_NOT_GROUP_UNIFORM: return "mask is not uniform inside a kernel group";
+    case RT3D_ERR_UNSUPPORTED: return "unsupported";
+    case RT3D_ERR_ALLOC: return "allocation failed";
+    case RT3D_ERR_CUDA: return "CUDA error";
+    case RT3D_ERR_TIMEOUT: return "device-side wait timed out";
+  }
+  return "unknown status";
+}
+
+const char* rt3d_version(void) { return "rt3d-b200 0.1 (sm_100a)"; }
+
+}  // extern "C"

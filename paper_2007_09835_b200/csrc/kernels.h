@@ -1,0 +1,56 @@
+// Launch interfaces of the CUDA kernels (device work), called from api.cu.
+#pragma once
+
+#include <cstdint>
+#include <cuda_runtime.h>
+
+namespace rt3d {
+
+// Geometry of one convolution call (all extents already validated on the host).
+struct ConvGeom {
+  int n, t, h, w, c, xcs;          // input extents and channel pitch
+  int To, Ho, Wo, M, ycs;          // output extents and channel pitch
+  int Kt, Kh, Kw;
+  int st, sh, sw, pt, ph, pw;
+  int relu;
+};
+
+// CUDA-core kernel driven by the canonical packed arrays.  dtype: 0 fp32, 1 bf16.
+cudaError_t launch_conv_simt(int dtype, const ConvGeom& g, const void* x, void* y,
+                             const int32_t* group_ptr, const uint16_t* pos_idx, const void* tiles,
+                             const float* bias, int g_m, int g_n, int P, int Q, bool dense,
+                             cudaStream_t stream);
+
+cudaError_t launch_maxpool3d(int dtype, const void* x, int n, int t, int h, int w, int c, int xcs,
+                             int kt, int kh, int kw, int st, int sh, int sw, int pt, int ph, int pw,
+                             void* y, int To, int Ho, int Wo, int ycs, cudaStream_t stream);
+
+cudaError_t launch_add_relu(int dtype, const void* a, int acs, const void* b, int bcs, void* y, int ycs,
+                            int64_t voxels, int c, int relu, cudaStream_t stream);
+
+// Output-voxel box of one tensor-core tile: bn*bt*bh*bw <= 128 voxels.
+struct TileBox { int bn, bt, bh, bw; };
+
+// Everything the tcgen05 kernel needs besides the two tensor maps.
+struct UmmaArgs {
+  ConvGeom g;
+  TileBox box;
+  int n_tile, n_bundles, n_chunks;
+  int tiles_n, tiles_t, tiles_h, tiles_w;   // number of boxes along each axis
+  int dense;                                // 1: steps are computed, not read
+  int steps_dense;                          // Ks * n_chunks (dense only)
+  const int32_t* step_ptr;                  // device, [n_bundles + 1]   (sparse)
+  const int32_t* steps;                     // device                     (sparse)
+  const float* bias;                        // device or nullptr
+  void* y;
+  int32_t* sched;                           // device [8]: [0] tile counter, [1] finished CTAs, [2] error word
+};
+
+// xmap / wmap point to 128-byte CUtensorMap objects in host memory.
+cudaError_t launch_conv_umma(const UmmaArgs& a, const void* xmap, const void* wmap, int sm_count,
+                             cudaStream_t stream);
+
+// Shared memory the tcgen05 kernel needs for a bundle width (for the host-side eligibility check).
+size_t umma_smem_bytes(int n_tile);
+
+}  // namespace rt3d

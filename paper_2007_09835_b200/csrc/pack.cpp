@@ -1,0 +1,235 @@
+// Host-side weight reorganisation: the KGS pack (Section 3 / Section 5.2 of the paper), its
+// inverse, and the derivation of the tensor-core weight layout from the canonical arrays.
+// Pure host code: no CUDA calls, usable without a GPU.
+#include <cstring>
+#include <new>
+
+#include "rt3d_internal.h"
+
+namespace rt3d {
+
+uint16_t f32_to_bf16_bits(float f) {
+  uint32_t u;
+  std::memcpy(&u, &f, 4);
+  if ((u & 0x7F800000u) == 0x7F800000u && (u & 0x007FFFFFu)) return uint16_t((u >> 16) | 0x40u);
+  u += 0x7FFFu + ((u >> 16) & 1u);   // ties to even
+  return uint16_t(u >> 16);
+}
+
+float bf16_bits_to_f32(uint16_t b) {
+  uint32_t u = uint32_t(b) << 16;
+  float f;
+  std::memcpy(&f, &u, 4);
+  return f;
+}
+
+int default_n_tile(int M) {
+  const int bundles = ceil_div(round_up(M, 16), 256);
+  return round_up(ceil_div(M, bundles), 16);
+}
+
+bool umma_layout_possible(const rt3d_packed* p) {
+  return p->dtype == RT3D_BF16 && p->Kt <= 63 && p->Kh <= 63 && p->Kw <= 63 && ceil_div(p->N, kChunk) <= 4095;
+}
+
+static float tile_value(const rt3d_packed* p, int64_t e, int i, int j) {
+  const int64_t o = (e * p->g_m + i) * p->g_n + j;
+  if (p->dtype == RT3D_BF16) return bf16_bits_to_f32(reinterpret_cast<const uint16_t*>(p->tiles.data())[o]);
+  return reinterpret_cast<const float*>(p->tiles.data())[o];
+}
+
+// For each bundle of n_tile output channels, list the (kernel location, 64-channel chunk)
+// steps in which at least one kernel group of the bundle keeps that location, and build the
+// matching [n_tile][64] weight tiles (zeros where a group prunes the location).  Steps are
+// ordered by location, then chunk.
+const UmmaLayout* get_umma_layout(rt3d_packed* p, int n_tile) {
+  if (!umma_layout_possible(p)) return nullptr;
+  if (n_tile <= 0) n_tile = default_n_tile(p->M);
+  if (n_tile % 16 || n_tile > 256) return nullptr;
+  std::lock_guard<std::mutex> lock(p->mu);
+  auto it = p->umma_layouts.find(n_tile);
+  if (it != p->umma_layouts.end()) return &it->second;
+
+  UmmaLayout L;
+  L.n_tile = n_tile;
+  L.n_bundles = ceil_div(p->M, n_tile);
+  L.n_chunks = ceil_div(p->N, kChunk);
+  L.step_ptr.assign(L.n_bundles + 1, 0);
+  const int Ks = p->Ks;
+  std::vector<int32_t> slot(size_t(Ks) * L.n_chunks);
+  for (int b = 0; b < L.n_bundles; ++b) {
+    const int m_lo = b * n_tile, m_hi = std::min(p->M, m_lo + n_tile);
+    const int p_lo = m_lo / p->g_m, p_hi = ceil_div(m_hi, p->g_m);
+    // pass 1: which steps are non-empty
+    std::fill(slot.begin(), slot.end(), -1);
+    for (int pr = p_lo; pr < p_hi; ++pr)
+      for (int q = 0; q < p->Q; ++q) {
+        const int c_lo = q * p->g_n, c_hi = std::min(p->N, c_lo + p->g_n);
+        for (int32_t e = p->group_ptr[pr * p->Q + q]; e < p->group_ptr[pr * p->Q + q + 1]; ++e)
+          for (int ch = c_lo / kChunk; ch <= (c_hi - 1) / kChunk; ++ch)
+            slot[size_t(p->pos_idx[e]) * L.n_chunks + ch] = 0;
+      }
+    const int32_t base = L.step_ptr[b];
+    int32_t cnt = 0;
+    for (int kpos = 0; kpos < Ks; ++kpos)
+      for (int ch = 0; ch < L.n_chunks; ++ch)
+        if (slot[size_t(kpos) * L.n_chunks + ch] == 0) {
+          slot[size_t(kpos) * L.n_chunks + ch] = base + cnt++;
+          const int kw = kpos % p->Kw, kh = (kpos / p->Kw) % p->Kh, kt = kpos / (p->Kw * p->Kh);
+          L.steps.push_back(encode_step(kt, kh, kw, ch));
+        }
+    L.step_ptr[b + 1] = base + cnt;
+    L.max_steps = std::max(L.max_steps, int(cnt));
+    L.wtiles.resize(size_t(base + cnt) * n_tile * kChunk, 0);
+    // pass 2: scatter the kept tiles
+    for (int pr = p_lo; pr < p_hi; ++pr)
+      for (int q = 0; q < p->Q; ++q)
+        for (int32_t e = p->group_ptr[pr * p->Q + q]; e < p->group_ptr[pr * p->Q + q + 1]; ++e)
+          for (int i = 0; i < p->g_m; ++i) {
+            const int m = pr * p->g_m + i;
+            if (m < m_lo || m >= m_hi) continue;
+            for (int j = 0; j < p->g_n; ++j) {
+              const int c = q * p->g_n + j;
+              if (c >= p->N) continue;
+              const int32_t s = slot[size_t(p->pos_idx[e]) * L.n_chunks + c / kChunk];
+              L.wtiles[(size_t(s) * n_tile + (m - m_lo)) * kChunk + c % kChunk] =
+                  reinterpret_cast<const uint16_t*>(p->tiles.data())[(int64_t(e) * p->g_m + i) * p->g_n + j];
+            }
+          }
+  }
+  auto res = p->umma_layouts.emplace(n_tile, std::move(L));
+  return &res.first->second;
+}
+
+static rt3d_status pack_impl(const float* w, const uint8_t* mask, int M, int N, int Kt, int Kh, int Kw,
+                             int g_m, int g_n, int dtype, int is_dense, rt3d_packed** out) {
+  if (!w || !out) return RT3D_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (M <= 0 || N <= 0 || Kt <= 0 || Kh <= 0 || Kw <= 0) return RT3D_ERR_INVALID_ARG;
+  if (g_m < 1 || g_n < 1 || g_m > kMaxGroup || g_n > kMaxGroup) return RT3D_ERR_INVALID_ARG;
+  if (dtype != RT3D_F32 && dtype != RT3D_BF16) return RT3D_ERR_INVALID_ARG;
+  const int64_t Ks64 = int64_t(Kt) * Kh * Kw;
+  if (Ks64 > 65535) return RT3D_ERR_INVALID_ARG;
+  rt3d_packed* h = new (std::nothrow) rt3d_packed;
+  if (!h) return RT3D_ERR_ALLOC;
+  try {
+    h->M = M; h->N = N; h->Kt = Kt; h->Kh = Kh; h->Kw = Kw; h->g_m = g_m; h->g_n = g_n;
+    h->P = ceil_div(M, g_m); h->Q = ceil_div(N, g_n); h->Ks = int(Ks64);
+    h->dtype = dtype; h->is_dense = is_dense;
+    const int Ks = h->Ks;
+    const size_t esz = dtype == RT3D_BF16 ? 2 : 4;
+    h->group_ptr.resize(size_t(h->P) * h->Q + 1);
+    // pass 1: group-level decisions with the uniformity check of the KGS definition
+    std::vector<uint8_t> keep(size_t(h->P) * h->Q * Ks);
+    int64_t nnz = 0;
+    bool vanilla = true;
+    for (int pr = 0; pr < h->P; ++pr)
+      for (int q = 0; q < h->Q; ++q) {
+        int kept_here = 0;
+        for (int k = 0; k < Ks; ++k) {
+          int decided = -1;
+          if (!mask) decided = 1;
+          else
+            for (int i = 0; i < g_m && pr * g_m + i < M; ++i)
+              for (int j = 0; j < g_n && q * g_n + j < N; ++j) {
+                const int bit = mask[(int64_t(pr * g_m + i) * N + (q * g_n + j)) * Ks + k] ? 1 : 0;
+                if (decided < 0) decided = bit;
+                else if (decided != bit) { delete h; return RT3D_ERR_MASK_NOT_GROUP_UNIFORM; }
+              }
+          keep[(size_t(pr) * h->Q + q) * Ks + k] = uint8_t(decided > 0);
+          kept_here += decided > 0;
+        }
+        if (kept_here != 0 && kept_here != Ks) vanilla = false;
+        nnz += kept_here;
+      }
+    if (nnz > 0x7FFFFFFF) { delete h; return RT3D_ERR_UNSUPPORTED; }
+    h->nnz = nnz;
+    h->is_vanilla = vanilla;
+    h->pos_idx.resize(size_t(nnz));
+    h->tiles.assign(size_t(nnz) * g_m * g_n * esz, 0);
+    // pass 2: emit index and tiles
+    int64_t e = 0;
+    for (int pr = 0; pr < h->P; ++pr)
+      for (int q = 0; q < h->Q; ++q) {
+        h->group_ptr[size_t(pr) * h->Q + q] = int32_t(e);
+        for (int k = 0; k < Ks; ++k) {
+          if (!keep[(size_t(pr) * h->Q + q) * Ks + k]) continue;
+          h->pos_idx[size_t(e)] = uint16_t(k);
+          for (int i = 0; i < g_m && pr * g_m + i < M; ++i)
+            for (int j = 0; j < g_n && q * g_n + j < N; ++j) {
+              const float v = w[(int64_t(pr * g_m + i) * N + (q * g_n + j)) * Ks + k];
+              const size_t o = (size_t(e) * g_m + i) * g_n + j;
+              if (dtype == RT3D_BF16) reinterpret_cast<uint16_t*>(h->tiles.data())[o] = f32_to_bf16_bits(v);
+              else reinterpret_cast<float*>(h->tiles.data())[o] = v;
+            }
+          ++e;
+        }
+      }
+    h->group_ptr[size_t(h->P) * h->Q] = int32_t(e);
+  } catch (const std::bad_alloc&) {
+    delete h;
+    return RT3D_ERR_ALLOC;
+  }
+  *out = h;
+  return RT3D_OK;
+}
+
+}  // namespace rt3d
+
+using namespace rt3d;
+
+extern "C" {
+
+rt3d_status rt3d_pack_kgs(const float* w, const uint8_t* mask, int M, int N, int Kt, int Kh, int Kw,
+                          int g_m, int g_n, int compute_dtype, rt3d_packed** out) {
+  return pack_impl(w, mask, M, N, Kt, Kh, Kw, g_m, g_n, compute_dtype, 0, out);
+}
+
+rt3d_status rt3d_pack_dense(const float* w, int M, int N, int Kt, int Kh, int Kw, int compute_dtype,
+                            rt3d_packed** out) {
+  return pack_impl(w, nullptr, M, N, Kt, Kh, Kw, 4, 4, compute_dtype, 1, out);
+}
+
+rt3d_status rt3d_packed_view_get(const rt3d_packed* p, rt3d_packed_view* v) {
+  if (!p || !v) return RT3D_ERR_INVALID_ARG;
+  v->M = p->M; v->N = p->N; v->Kt = p->Kt; v->Kh = p->Kh; v->Kw = p->Kw;
+  v->g_m = p->g_m; v->g_n = p->g_n; v->P = p->P; v->Q = p->Q; v->Ks = p->Ks;
+  v->dtype = p->dtype; v->is_vanilla = p->is_vanilla; v->is_dense = p->is_dense; v->nnz = p->nnz;
+  v->group_ptr = p->group_ptr.data();
+  v->pos_idx = p->pos_idx.data();
+  v->tiles = p->tiles.data();
+  return RT3D_OK;
+}
+
+rt3d_status rt3d_unpack_to_dense(const rt3d_packed* p, float* w_out) {
+  if (!p || !w_out) return RT3D_ERR_INVALID_ARG;
+  std::memset(w_out, 0, sizeof(float) * size_t(p->M) * p->N * p->Ks);
+  for (int pr = 0; pr < p->P; ++pr)
+    for (int q = 0; q < p->Q; ++q)
+      for (int32_t e = p->group_ptr[size_t(pr) * p->Q + q]; e < p->group_ptr[size_t(pr) * p->Q + q + 1]; ++e)
+        for (int i = 0; i < p->g_m && pr * p->g_m + i < p->M; ++i)
+          for (int j = 0; j < p->g_n && q * p->g_n + j < p->N; ++j)
+            w_out[(int64_t(pr * p->g_m + i) * p->N + (q * p->g_n + j)) * p->Ks + p->pos_idx[e]] =
+                tile_value(p, e, i, j);
+  return RT3D_OK;
+}
+
+rt3d_status rt3d_unpack_device_layout(const rt3d_packed* p, int n_tile, float* w_out) {
+  if (!p || !w_out) return RT3D_ERR_INVALID_ARG;
+  const UmmaLayout* L = get_umma_layout(const_cast<rt3d_packed*>(p), n_tile);
+  if (!L) return RT3D_ERR_UNSUPPORTED;
+  std::memset(w_out, 0, sizeof(float) * size_t(p->M) * p->N * p->Ks);
+  for (int b = 0; b < L->n_bundles; ++b)
+    for (int32_t s = L->step_ptr[b]; s < L->step_ptr[b + 1]; ++s) {
+      int kt, kh, kw, ch;
+      decode_step(L->steps[s], kt, kh, kw, ch);
+      const int kpos = (kt * p->Kh + kh) * p->Kw + kw;
+      for (int r = 0; r < L->n_tile && b * L->n_tile + r < p->M; ++r)
+        for (int j = 0; j < kChunk && ch * kChunk + j < p->N; ++j)
+          w_out[(int64_t(b * L->n_tile + r) * p->N + (ch * kChunk + j)) * p->Ks + kpos] =
+              bf16_bits_to_f32(L->wtiles[(size_t(s) * L->n_tile + r) * kChunk + j]);
+    }
+  return RT3D_OK;
+}
+
+}  // extern "C"

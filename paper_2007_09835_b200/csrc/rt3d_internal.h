@@ -1,0 +1,88 @@
+// Internal declarations shared by the translation units of librt3d (host side).
+#pragma once
+
+#include <cstdint>
+#include <cstddef>
+#include <map>
+#include <mutex>
+#include <vector>
+
+#include "rt3d.h"
+
+namespace rt3d {
+
+constexpr int kMaxGroup = 8;        // g_m, g_n <= 8
+constexpr int kChunk = 64;          // input channels per tensor-core K step (one 128-byte swizzle row of bf16)
+constexpr int kTileM = 128;         // output voxels per tensor-core tile (TMEM lanes)
+
+inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
+inline int64_t ceil_div64(int64_t a, int64_t b) { return (a + b - 1) / b; }
+inline int round_up(int a, int b) { return ceil_div(a, b) * b; }
+
+// Round-to-nearest-even float -> bfloat16 bits (NaN kept quiet), and back.
+uint16_t f32_to_bf16_bits(float f);
+float bf16_bits_to_f32(uint16_t b);
+
+// Encoded K step of the tensor-core path: which kernel location and which 64-channel chunk.
+inline int32_t encode_step(int kt, int kh, int kw, int chunk) {
+  return (kt << 24) | (kh << 18) | (kw << 12) | chunk;
+}
+inline void decode_step(int32_t s, int& kt, int& kh, int& kw, int& chunk) {
+  kt = (s >> 24) & 63; kh = (s >> 18) & 63; kw = (s >> 12) & 63; chunk = s & 4095;
+}
+
+// Weight layout consumed by the tcgen05 kernel, derived from the canonical arrays for one
+// bundle width n_tile (output channels per accumulator tile).
+struct UmmaLayout {
+  int n_tile = 0;                    // multiple of 16, <= 256
+  int n_bundles = 0;                 // ceil(M / n_tile)
+  int n_chunks = 0;                  // ceil(N / 64)
+  std::vector<int32_t> step_ptr;     // [n_bundles + 1] offsets into steps / weight tiles
+  std::vector<int32_t> steps;        // encoded (kt,kh,kw,chunk), only non-empty steps of each bundle
+  std::vector<uint16_t> wtiles;      // [steps.size()][n_tile][64] bf16 bits, zero where pruned / absent
+  int max_steps = 0;                 // longest bundle list
+};
+
+// Per-device copies of a handle's arrays.
+struct DeviceBlob {
+  int device = -1;
+  int32_t* group_ptr = nullptr;      // canonical arrays (CUDA-core kernel)
+  uint16_t* pos_idx = nullptr;
+  void* tiles = nullptr;
+  struct Umma {
+    void* wtiles = nullptr;
+    int32_t* step_ptr = nullptr;
+    int32_t* steps = nullptr;
+    alignas(64) unsigned char wmap[128];   // CUtensorMap of wtiles
+    bool ready = false;
+  };
+  std::map<int, Umma> umma;          // keyed by n_tile
+  int32_t* sched = nullptr;          // [8] tile counter, finished-CTA counter (zero between launches)
+  void* stage_x = nullptr; size_t stage_x_bytes = 0;   // staging for rt3d_conv3d_host
+  void* stage_y = nullptr; size_t stage_y_bytes = 0;
+  float* stage_bias = nullptr;
+};
+
+}  // namespace rt3d
+
+struct rt3d_packed {
+  int M = 0, N = 0, Kt = 0, Kh = 0, Kw = 0, g_m = 0, g_n = 0, P = 0, Q = 0, Ks = 0;
+  int dtype = 0, is_vanilla = 0, is_dense = 0;
+  int64_t nnz = 0;
+  std::vector<int32_t> group_ptr;
+  std::vector<uint16_t> pos_idx;
+  std::vector<unsigned char> tiles;  // nnz * g_m * g_n elements of float or bf16 bits
+  std::mutex mu;                     // guards the lazily built members below
+  std::map<int, rt3d::UmmaLayout> umma_layouts;   // keyed by n_tile
+  std::vector<rt3d::DeviceBlob*> blobs;
+};
+
+namespace rt3d {
+
+// Default bundle width for M output channels: as few bundles as possible with n_tile <= 256.
+int default_n_tile(int M);
+// Builds (or returns the cached) tensor-core layout; nullptr if the handle cannot use it.
+const UmmaLayout* get_umma_layout(rt3d_packed* p, int n_tile);
+bool umma_layout_possible(const rt3d_packed* p);
+
+}  // namespace rt3d

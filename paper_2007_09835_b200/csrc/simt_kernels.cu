@@ -1,0 +1,274 @@
+// CUDA-core kernels: the index-driven KGS convolution (any shape, fp32 or bf16 storage, fp32
+// accumulation), 3-D max-pool and add(+ReLU) over NDHWC tensors.
+//
+// The convolution follows the group view of Section 3 of the paper directly: one thread owns
+// one output voxel and one row of kernel groups (g_m output channels); for every kernel
+// group of that row it walks the kept kernel locations of the packed index and applies the
+// group's g_m x g_n weight tile to the g_n input channels at the shifted voxel.  Pruned
+// locations are never visited.  It is the cross-check for the tensor-core kernel and the
+// production path for shapes that kernel does not take.
+#include <cuda_bf16.h>
+
+#include "kernels.h"
+
+namespace rt3d {
+namespace {
+
+constexpr int kThreads = 128;
+
+template <typename T> __device__ __forceinline__ float to_f32(T v);
+template <> __device__ __forceinline__ float to_f32<float>(float v) { return v; }
+template <> __device__ __forceinline__ float to_f32<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
+template <typename T> __device__ __forceinline__ T from_f32(float v);
+template <> __device__ __forceinline__ float from_f32<float>(float v) { return v; }
+template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
+
+// GM/GN > 0: compile-time group size; 0: run-time size (<= 8).
+template <typename T, int GM, int GN, bool DENSE>
+__global__ void __launch_bounds__(kThreads)
+conv3d_kgs_simt_kernel(ConvGeom g, const T* __restrict__ x, T* __restrict__ y,
+                       const int32_t* __restrict__ group_ptr, const uint16_t* __restrict__ pos_idx,
+                       const T* __restrict__ tiles, const float* __restrict__ bias,
+                       int g_m_rt, int g_n_rt, int Q, long long total_voxels) {
+  constexpr int MAXM = GM ? GM : 8;
+  constexpr int MAXN = GN ? GN : 8;
+  const int g_m = GM ? GM : g_m_rt;
+  const int g_n = GN ? GN : g_n_rt;
+  const int p = blockIdx.y;
+  const long long v = (long long)blockIdx.x * kThreads + threadIdx.x;
+  const bool valid = v < total_voxels;
+  int wo = 0, ho = 0, to = 0, nn = 0;
+  if (valid) {
+    long long r = v;
+    wo = int(r % g.Wo); r /= g.Wo;
+    ho = int(r % g.Ho); r /= g.Ho;
+    to = int(r % g.To); nn = int(r / g.To);
+  }
+  const int t0 = to * g.st - g.pt, h0 = ho * g.sh - g.ph, w0 = wo * g.sw - g.pw;
+  float acc[MAXM];
+#pragma unroll
+  for (int i = 0; i < MAXM; ++i) acc[i] = 0.f;
+
+  const int tile_elems = g_m * g_n;
+  for (int q = 0; q < Q; ++q) {
+    const int e0 = group_ptr[p * Q + q], e1 = group_ptr[p * Q + q + 1];
+    const int c0 = q * g_n;
+    for (int e = e0; e < e1; ++e) {
+      const int kpos = DENSE ? (e - e0) : int(pos_idx[e]);
+      const int kw = kpos % g.Kw;
+      const int kh = (kpos / g.Kw) % g.Kh;
+      const int kt = kpos / (g.Kw * g.Kh);
+      const int ti = t0 + kt, hi = h0 + kh, wi = w0 + kw;
+      if (!valid || ti < 0 || ti >= g.t || hi < 0 || hi >= g.h || wi < 0 || wi >= g.w) continue;
+      const T* xp = x + ((((long long)nn * g.t + ti) * g.h + hi) * g.w + wi) * g.xcs + c0;
+      float xv[MAXN];
+#pragma unroll
+      for (int j = 0; j < MAXN; ++j) xv[j] = (j < g_n && c0 + j < g.c) ? to_f32<T>(xp[j]) : 0.f;
+      const T* tp = tiles + (long long)e * tile_elems;
+#pragma unroll
+      for (int i = 0; i < MAXM; ++i) {
+        if (i < g_m) {
+#pragma unroll
+          for (int j = 0; j < MAXN; ++j)
+            if (j < g_n) acc[i] = fmaf(xv[j], to_f32<T>(tp[i * g_n + j]), acc[i]);
+        }
+      }
+    }
+  }
+  if (!valid) return;
+  T* yp = y + v * g.ycs + p * g_m;
+#pragma unroll
+  for (int i = 0; i < MAXM; ++i) {
+    const int m = p * g_m + i;
+    if (i < g_m && m < g.M) {
+      float r = acc[i] + (bias ? bias[m] : 0.f);
+      if (g.relu) r = fmaxf(r, 0.f);
+      yp[i] = from_f32<T>(r);
+    }
+  }
+}
+
+template <typename T, bool DENSE>
+cudaError_t launch_conv_t(const ConvGeom& g, const void* x, void* y, const int32_t* group_ptr,
+                          const uint16_t* pos_idx, const void* tiles, const float* bias, int g_m, int g_n,
+                          int P, int Q, cudaStream_t stream) {
+  const long long total = (long long)g.n * g.To * g.Ho * g.Wo;
+  if (total == 0) return cudaSuccess;
+  dim3 grid((unsigned)((total + kThreads - 1) / kThreads), (unsigned)P);
+  const T* xt = static_cast<const T*>(x);
+  T* yt = static_cast<T*>(y);
+  const T* tt = static_cast<const T*>(tiles);
+#define RT3D_LAUNCH(GM_, GN_) \
+  conv3d_kgs_simt_kernel<T, GM_, GN_, DENSE><<<grid, kThreads, 0, stream>>>(g, xt, yt, group_ptr, pos_idx, tt, bias, g_m, g_n, Q, total)
+  if (g_m == 4 && g_n == 4) RT3D_LAUNCH(4, 4);
+  else if (g_m == 8 && g_n == 4) RT3D_LAUNCH(8, 4);
+  else if (g_m == 8 && g_n == 8) RT3D_LAUNCH(8, 8);
+  else RT3D_LAUNCH(0, 0);
+#undef RT3D_LAUNCH
+  return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------- max-pool
+template <typename T>
+__global__ void maxpool3d_kernel(const T* __restrict__ x, int t, int h, int w, int c, int xcs,
+                                 int kt, int kh, int kw, int st, int sh, int sw, int pt, int ph, int pw,
+                                 T* __restrict__ y, int To, int Ho, int Wo, int ycs, long long total) {
+  const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= total) return;
+  const int cc = int(idx % c);
+  long long r = idx / c;
+  const int wo = int(r % Wo); r /= Wo;
+  const int ho = int(r % Ho); r /= Ho;
+  const int to = int(r % To);
+  const int nn = int(r / To);
+  float best = -INFINITY;
+  for (int a = 0; a < kt; ++a) {
+    const int ti = to * st - pt + a;
+    if (ti < 0 || ti >= t) continue;
+    for (int b = 0; b < kh; ++b) {
+      const int hi = ho * sh - ph + b;
+      if (hi < 0 || hi >= h) continue;
+      for (int d = 0; d < kw; ++d) {
+        const int wi = wo * sw - pw + d;
+        if (wi < 0 || wi >= w) continue;
+        best = fmaxf(best, to_f32<T>(x[((((long long)nn * t + ti) * h + hi) * w + wi) * xcs + cc]));
+      }
+    }
+  }
+  y[((((long long)nn * To + to) * Ho + ho) * Wo + wo) * ycs + cc] = from_f32<T>(best);
+}
+
+// bf16, 8 channels (16 bytes) per thread; needs c % 8 == 0 and 8-element pitches.
+__global__ void maxpool3d_bf16x8_kernel(const uint4* __restrict__ x, int t, int h, int w, int c8, int xcs8,
+                                        int kt, int kh, int kw, int st, int sh, int sw, int pt, int ph, int pw,
+                                        uint4* __restrict__ y, int To, int Ho, int Wo, int ycs8, long long total) {
+  const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= total) return;
+  const int cc = int(idx % c8);
+  long long r = idx / c8;
+  const int wo = int(r % Wo); r /= Wo;
+  const int ho = int(r % Ho); r /= Ho;
+  const int to = int(r % To);
+  const int nn = int(r / To);
+  const __nv_bfloat162 ninf = __float2bfloat162_rn(-INFINITY);
+  __nv_bfloat162 best[4] = {ninf, ninf, ninf, ninf};
+  for (int a = 0; a < kt; ++a) {
+    const int ti = to * st - pt + a;
+    if (ti < 0 || ti >= t) continue;
+    for (int b = 0; b < kh; ++b) {
+      const int hi = ho * sh - ph + b;
+      if (hi < 0 || hi >= h) continue;
+      for (int d = 0; d < kw; ++d) {
+        const int wi = wo * sw - pw + d;
+        if (wi < 0 || wi >= w) continue;
+        const uint4 v = __ldg(x + ((((long long)nn * t + ti) * h + hi) * w + wi) * xcs8 + cc);
+        const __nv_bfloat162* pv = reinterpret_cast<const __nv_bfloat162*>(&v);
+#pragma unroll
+        for (int k = 0; k < 4; ++k) best[k] = __hmax2(best[k], pv[k]);
+      }
+    }
+  }
+  uint4 out;
+  __nv_bfloat162* po = reinterpret_cast<__nv_bfloat162*>(&out);
+#pragma unroll
+  for (int k = 0; k < 4; ++k) po[k] = best[k];
+  y[((((long long)nn * To + to) * Ho + ho) * Wo + wo) * ycs8 + cc] = out;
+}
+
+// ----------------------------------------------------------------------------- add + relu
+template <typename T>
+__global__ void add_relu_kernel(const T* __restrict__ a, int acs, const T* __restrict__ b, int bcs,
+                                T* __restrict__ y, int ycs, int c, int relu, long long total) {
+  const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= total) return;
+  const int cc = int(idx % c);
+  const long long v = idx / c;
+  float r = to_f32<T>(a[v * acs + cc]) + to_f32<T>(b[v * bcs + cc]);
+  if (relu) r = fmaxf(r, 0.f);
+  y[v * ycs + cc] = from_f32<T>(r);
+}
+
+__global__ void add_relu_bf16x8_kernel(const uint4* __restrict__ a, int acs8, const uint4* __restrict__ b,
+                                       int bcs8, uint4* __restrict__ y, int ycs8, int c8, int relu,
+                                       long long total) {
+  const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= total) return;
+  const int cc = int(idx % c8);
+  const long long v = idx / c8;
+  const uint4 va = a[v * acs8 + cc], vb = b[v * bcs8 + cc];
+  const __nv_bfloat162* pa = reinterpret_cast<const __nv_bfloat162*>(&va);
+  const __nv_bfloat162* pb = reinterpret_cast<const __nv_bfloat162*>(&vb);
+  uint4 out;
+  __nv_bfloat162* po = reinterpret_cast<__nv_bfloat162*>(&out);
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    float2 fa = __bfloat1622float2(pa[k]), fb = __bfloat1622float2(pb[k]);
+    float2 r = make_float2(fa.x + fb.x, fa.y + fb.y);
+    if (relu) { r.x = fmaxf(r.x, 0.f); r.y = fmaxf(r.y, 0.f); }
+    po[k] = __float22bfloat162_rn(r);
+  }
+  y[v * ycs8 + cc] = out;
+}
+
+}  // namespace
+
+cudaError_t launch_conv_simt(int dtype, const ConvGeom& g, const void* x, void* y, const int32_t* group_ptr,
+                             const uint16_t* pos_idx, const void* tiles, const float* bias, int g_m, int g_n,
+                             int P, int Q, bool dense, cudaStream_t stream) {
+  if (dtype == 0)
+    return dense ? launch_conv_t<float, true>(g, x, y, group_ptr, pos_idx, tiles, bias, g_m, g_n, P, Q, stream)
+                 : launch_conv_t<float, false>(g, x, y, group_ptr, pos_idx, tiles, bias, g_m, g_n, P, Q, stream);
+  return dense ? launch_conv_t<__nv_bfloat16, true>(g, x, y, group_ptr, pos_idx, tiles, bias, g_m, g_n, P, Q, stream)
+               : launch_conv_t<__nv_bfloat16, false>(g, x, y, group_ptr, pos_idx, tiles, bias, g_m, g_n, P, Q, stream);
+}
+
+cudaError_t launch_maxpool3d(int dtype, const void* x, int n, int t, int h, int w, int c, int xcs,
+                             int kt, int kh, int kw, int st, int sh, int sw, int pt, int ph, int pw,
+                             void* y, int To, int Ho, int Wo, int ycs, cudaStream_t stream) {
+  const long long vox = (long long)n * To * Ho * Wo;
+  if (vox == 0) return cudaSuccess;
+  const int threads = 256;
+  if (dtype == 1 && c % 8 == 0 && xcs % 8 == 0 && ycs % 8 == 0) {
+    const long long total = vox * (c / 8);
+    maxpool3d_bf16x8_kernel<<<(unsigned)((total + threads - 1) / threads), threads, 0, stream>>>(
+        static_cast<const uint4*>(x), t, h, w, c / 8, xcs / 8, kt, kh, kw, st, sh, sw, pt, ph, pw,
+        static_cast<uint4*>(y), To, Ho, Wo, ycs / 8, total);
+  } else {
+    const long long total = vox * c;
+    const unsigned blocks = (unsigned)((total + threads - 1) / threads);
+    if (dtype == 0)
+      maxpool3d_kernel<float><<<blocks, threads, 0, stream>>>(static_cast<const float*>(x), t, h, w, c, xcs, kt, kh, kw,
+                                                             st, sh, sw, pt, ph, pw, static_cast<float*>(y), To, Ho, Wo,
+                                                             ycs, total);
+    else
+      maxpool3d_kernel<__nv_bfloat16><<<blocks, threads, 0, stream>>>(
+          static_cast<const __nv_bfloat16*>(x), t, h, w, c, xcs, kt, kh, kw, st, sh, sw, pt, ph, pw,
+          static_cast<__nv_bfloat16*>(y), To, Ho, Wo, ycs, total);
+  }
+  return cudaGetLastError();
+}
+
+cudaError_t launch_add_relu(int dtype, const void* a, int acs, const void* b, int bcs, void* y, int ycs,
+                            int64_t voxels, int c, int relu, cudaStream_t stream) {
+  if (voxels == 0) return cudaSuccess;
+  const int threads = 256;
+  if (dtype == 1 && c % 8 == 0 && acs % 8 == 0 && bcs % 8 == 0 && ycs % 8 == 0) {
+    const long long total = voxels * (c / 8);
+    add_relu_bf16x8_kernel<<<(unsigned)((total + threads - 1) / threads), threads, 0, stream>>>(
+        static_cast<const uint4*>(a), acs / 8, static_cast<const uint4*>(b), bcs / 8, static_cast<uint4*>(y),
+        ycs / 8, c / 8, relu, total);
+  } else {
+    const long long total = voxels * c;
+    const unsigned blocks = (unsigned)((total + threads - 1) / threads);
+    if (dtype == 0)
+      add_relu_kernel<float><<<blocks, threads, 0, stream>>>(static_cast<const float*>(a), acs, static_cast<const float*>(b),
+                                                            bcs, static_cast<float*>(y), ycs, c, relu, total);
+    else
+      add_relu_kernel<__nv_bfloat16><<<blocks, threads, 0, stream>>>(
+          static_cast<const __nv_bfloat16*>(a), acs, static_cast<const __nv_bfloat16*>(b), bcs,
+          static_cast<__nv_bfloat16*>(y), ycs, c, relu, total);
+  }
+  return cudaGetLastError();
+}
+
+}  // namespace rt3d

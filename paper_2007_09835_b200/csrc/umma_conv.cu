@@ -1,0 +1,372 @@
+// Tensor-core KGS convolution for sm_100a: implicit GEMM on tcgen05 with TMA-staged operands
+// and fp32 accumulators in tensor memory.
+//
+// Mapping of the paper's group-matrix view (Section 3) onto the hardware:
+//   D[128 output voxels x n_tile output channels] += A[128 x 64] * B[n_tile x 64]^T
+// once per K step, where a K step is one kernel location (kt,kh,kw) and one chunk of 64 input
+// channels.  A is the input tile shifted by the kernel location (a 5-D TMA box over NDHWC whose
+// out-of-range part is zero-filled = the convolution's zero padding); B is the bundle's weight
+// tile for that step, pre-arranged at pack time.  For a KGS-pruned layer the producer walks the
+// bundle's packed step list, so a (location, chunk) that no kernel group of the bundle keeps
+// costs no loads and no MMAs; the dense kernel computes the steps arithmetically.
+//
+// One persistent CTA per SM, 6 warps: warp 0 = TMA producer, warp 1 = MMA issuer (and TMEM
+// owner), warps 2..5 = epilogue (TMEM -> registers -> +bias, ReLU, bf16 -> NDHWC stores).  Two
+// accumulator buffers in TMEM let the epilogue of one tile overlap the MMAs of the next.
+// Every wait on an mbarrier is bounded: on expiry the CTA records an error word in global
+// memory, all roles fall through, TMEM is released and the kernel returns.
+#include <cuda.h>
+#include <cuda_bf16.h>
+
+#include "kernels.h"
+
+namespace rt3d {
+namespace {
+
+constexpr int kThreadsUmma = 192;
+constexpr int kMaxStages = 8;
+constexpr int kABytes = 128 * 128;                  // 128 voxel rows x 64 bf16
+constexpr long long kWaitCycles = 1ll << 31;        // about one second of SM clocks
+constexpr size_t kSmemBudget = 200 * 1024;
+
+struct __align__(8) Barriers {
+  unsigned long long full[kMaxStages];
+  unsigned long long empty[kMaxStages];
+  unsigned long long tmem_full[2];
+  unsigned long long tmem_empty[2];
+  unsigned int tmem_base;
+  volatile int abort_flag;
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+      "selp.u32 %0, 1, 0, p;\n"
+      "}\n"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+
+// Bounded wait.  Returns false (and raises the CTA's abort flag + the global error word) when the
+// phase did not complete within kWaitCycles, or when another role already aborted.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, Barriers* bars, int32_t* err, int code) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long start = clock64();
+  for (;;) {
+#pragma unroll 1
+    for (int i = 0; i < 128; ++i)
+      if (mbar_try_wait(bar, parity)) return true;
+    if (bars->abort_flag) return false;
+    if (clock64() - start > kWaitCycles) {
+      bars->abort_flag = 1;
+      atomicCAS(err, 0, code);
+      return false;
+    }
+  }
+}
+
+__device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2,
+                                            int c3, int c4) {
+  asm volatile(
+      "cp.async.bulk.tensor.5d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4)
+      : "memory");
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1)
+      : "memory");
+}
+
+// Shared-memory matrix descriptor: K-major tile of 128-byte rows, 128-byte swizzle, 8-row groups
+// 1024 bytes apart; descriptor version 1 (sm_100).
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
+  uint64_t d = 0;
+  d |= uint64_t((addr & 0x3FFFFu) >> 4);
+  d |= uint64_t(1) << 16;                 // leading byte offset (unused for swizzled K-major)
+  d |= uint64_t(1024 >> 4) << 32;         // stride byte offset between 8-row groups
+  d |= uint64_t(1) << 46;                 // version
+  d |= uint64_t(2) << 61;                 // SWIZZLE_128B
+  return d;
+}
+
+// Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128, N = n.
+__device__ __forceinline__ uint32_t instr_desc_bf16(int n) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | (uint32_t(n >> 3) << 17) | (uint32_t(128 >> 4) << 24);
+}
+
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      "setp.ne.b32 p, %4, 0;\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n"
+      "}\n"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc)
+      : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr));
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+struct ItemCoord {
+  int bundle, n0, t0, h0, w0;     // bundle index and first output voxel of the box
+};
+
+__device__ __forceinline__ ItemCoord decode_item(const UmmaArgs& a, int item, int n_mtiles) {
+  ItemCoord c;
+  c.bundle = item / n_mtiles;
+  int mt = item - c.bundle * n_mtiles;
+  const int iw = mt % a.tiles_w; mt /= a.tiles_w;
+  const int ih = mt % a.tiles_h; mt /= a.tiles_h;
+  const int it = mt % a.tiles_t; mt /= a.tiles_t;
+  c.w0 = iw * a.box.bw; c.h0 = ih * a.box.bh; c.t0 = it * a.box.bt; c.n0 = mt * a.box.bn;
+  return c;
+}
+
+template <bool kDense>
+__global__ void __launch_bounds__(kThreadsUmma, 1)
+conv3d_umma_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CUtensorMap wmap,
+                   const UmmaArgs a, const int stages, const int tmem_cols) {
+  extern __shared__ unsigned char smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t tiles_base = (raw + 1023u) & ~1023u;            // operand tiles need 1024-byte alignment
+  const uint32_t b_bytes = uint32_t(a.n_tile) * 128u;
+  const uint32_t stage_bytes = kABytes + b_bytes;
+  Barriers* bars = reinterpret_cast<Barriers*>(smem_raw + (tiles_base - raw) + size_t(stages) * stage_bytes);
+  int32_t* err = a.sched + 2;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int n_mtiles = a.tiles_n * a.tiles_t * a.tiles_h * a.tiles_w;
+  const int n_items = n_mtiles * a.n_bundles;
+  const int box_rows = a.box.bn * a.box.bt * a.box.bh * a.box.bw;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < stages; ++s) {
+      mbar_init(smem_u32(&bars->full[s]), 1);
+      mbar_init(smem_u32(&bars->empty[s]), 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(smem_u32(&bars->tmem_full[b]), 1);
+      mbar_init(smem_u32(&bars->tmem_empty[b]), 4);
+    }
+    bars->abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                 ::"r"(smem_u32(&bars->tmem_base)), "r"(uint32_t(tmem_cols)) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = bars->tmem_base;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      uint32_t k = 0;
+      bool ok = true;
+      for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
+        const ItemCoord c = decode_item(a, item, n_mtiles);
+        const int s_begin = kDense ? c.bundle * a.steps_dense : a.step_ptr[c.bundle];
+        const int nsteps = kDense ? a.steps_dense : a.step_ptr[c.bundle + 1] - s_begin;
+        const int wq = c.w0 * a.g.sw - a.g.pw, hq = c.h0 * a.g.sh - a.g.ph, tq = c.t0 * a.g.st - a.g.pt;
+        for (int i = 0; i < nsteps; ++i, ++k) {
+          const int stage = k % stages;
+          const uint32_t round = k / stages;
+          if (!mbar_wait(smem_u32(&bars->empty[stage]), (round & 1u) ^ 1u, bars, err, 1)) { ok = false; break; }
+          int kt, kh, kw, ch;
+          if (kDense) {
+            ch = i % a.n_chunks;
+            const int pos = i / a.n_chunks;
+            kw = pos % a.g.Kw; kh = (pos / a.g.Kw) % a.g.Kh; kt = pos / (a.g.Kw * a.g.Kh);
+          } else {
+            const int enc = a.steps[s_begin + i];
+            kt = (enc >> 24) & 63; kh = (enc >> 18) & 63; kw = (enc >> 12) & 63; ch = enc & 4095;
+          }
+          const uint32_t full = smem_u32(&bars->full[stage]);
+          const uint32_t a_dst = tiles_base + stage * stage_bytes;
+          mbar_expect_tx(full, uint32_t(box_rows) * 128u + b_bytes);
+          tma_load_5d(a_dst, &xmap, full, ch * 64, wq + kw, hq + kh, tq + kt, c.n0);
+          tma_load_2d(a_dst + kABytes, &wmap, full, 0, (s_begin + i) * a.n_tile);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      const uint32_t idesc = instr_desc_bf16(a.n_tile);
+      uint32_t k = 0, j = 0;
+      bool ok = true;
+      for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++j) {
+        const int bundle = item / n_mtiles;
+        const int nsteps = kDense ? a.steps_dense : a.step_ptr[bundle + 1] - a.step_ptr[bundle];
+        const uint32_t buf = j & 1u;
+        if (!mbar_wait(smem_u32(&bars->tmem_empty[buf]), ((j >> 1) & 1u) ^ 1u, bars, err, 2)) break;
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + buf * uint32_t(a.n_tile);
+        for (int i = 0; i < nsteps; ++i, ++k) {
+          const int stage = k % stages;
+          if (!mbar_wait(smem_u32(&bars->full[stage]), (k / stages) & 1u, bars, err, 3)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t a_addr = tiles_base + stage * stage_bytes;
+          const uint64_t adesc = smem_desc_sw128(a_addr);
+          const uint64_t bdesc = smem_desc_sw128(a_addr + kABytes);
+#pragma unroll
+          for (int kk = 0; kk < 4; ++kk)      // 4 x K=16 per 64-channel chunk: +32 bytes = +2 in descriptor units
+            umma_bf16(d_tmem, adesc + 2 * kk, bdesc + 2 * kk, idesc, (i | kk) ? 1u : 0u);
+          umma_commit(smem_u32(&bars->empty[stage]));
+        }
+        if (!ok) break;
+        if (nsteps > 0) umma_commit(smem_u32(&bars->tmem_full[buf]));
+        else mbar_arrive(smem_u32(&bars->tmem_full[buf]));
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue (warps 2..5)
+    const int quad = warp & 3;                 // TMEM lane quadrant this warp may read
+    const int row = quad * 32 + lane;          // voxel row inside the box
+    int r = row;
+    const int bw_i = r % a.box.bw; r /= a.box.bw;
+    const int bh_i = r % a.box.bh; r /= a.box.bh;
+    const int bt_i = r % a.box.bt; r /= a.box.bt;
+    const int bn_i = r;
+    __nv_bfloat16* yb = static_cast<__nv_bfloat16*>(a.y);
+    uint32_t j = 0;
+    for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++j) {
+      const ItemCoord c = decode_item(a, item, n_mtiles);
+      const int nsteps = kDense ? a.steps_dense : a.step_ptr[c.bundle + 1] - a.step_ptr[c.bundle];
+      const uint32_t buf = j & 1u;
+      if (!mbar_wait(smem_u32(&bars->tmem_full[buf]), (j >> 1) & 1u, bars, err, 4)) break;
+      tc_fence_after();
+      const int nn = c.n0 + bn_i, to = c.t0 + bt_i, ho = c.h0 + bh_i, wo = c.w0 + bw_i;
+      const bool in_range = row < box_rows && nn < a.g.n && to < a.g.To && ho < a.g.Ho && wo < a.g.Wo;
+      const long long vox = (((long long)nn * a.g.To + to) * a.g.Ho + ho) * a.g.Wo + wo;
+      const int m_base = c.bundle * a.n_tile;
+      const uint32_t taddr = tmem_base + (uint32_t(quad * 32) << 16) + buf * uint32_t(a.n_tile);
+      for (int col = 0; col < a.n_tile; col += 16) {
+        const int m0 = m_base + col;
+        if (m0 >= a.g.M) break;                      // warp-uniform
+        uint32_t v[16];
+        if (nsteps > 0) tmem_ld16(taddr + col, v);   // warp-uniform: .sync.aligned
+        else {
+#pragma unroll
+          for (int q = 0; q < 16; ++q) v[q] = 0u;
+        }
+        if (!in_range) continue;
+        float f[16];
+#pragma unroll
+        for (int q = 0; q < 16; ++q) {
+          f[q] = __uint_as_float(v[q]);
+          if (a.bias != nullptr && m0 + q < a.g.M) f[q] += __ldg(a.bias + m0 + q);
+          if (a.g.relu) f[q] = fmaxf(f[q], 0.f);
+        }
+        __nv_bfloat16* dst = yb + vox * a.g.ycs + m0;
+        if (m0 + 16 <= a.g.M) {
+          uint4 o[2];
+          __nv_bfloat162* po = reinterpret_cast<__nv_bfloat162*>(o);
+#pragma unroll
+          for (int q = 0; q < 8; ++q) po[q] = __floats2bfloat162_rn(f[2 * q], f[2 * q + 1]);
+          reinterpret_cast<uint4*>(dst)[0] = o[0];
+          reinterpret_cast<uint4*>(dst)[1] = o[1];
+        } else {
+          for (int q = 0; q < 16 && m0 + q < a.g.M; ++q) dst[q] = __float2bfloat16_rn(f[q]);
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&bars->tmem_empty[buf]));
+    }
+  }
+
+  // ---------------------------------------------------------------------- teardown
+  if (bars->abort_flag) {
+    // error path: give asynchronous copies / MMAs still in flight time to land before TMEM goes away
+    const long long t0 = clock64();
+    while (clock64() - t0 < 2000000ll) { }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(uint32_t(tmem_cols)) : "memory");
+  }
+}
+
+int pick_stages(int n_tile) {
+  const size_t stage = kABytes + size_t(n_tile) * 128;
+  int s = int(kSmemBudget / stage);
+  return s > kMaxStages ? kMaxStages : s;
+}
+
+}  // namespace
+
+size_t umma_smem_bytes(int n_tile) {
+  return size_t(pick_stages(n_tile)) * (kABytes + size_t(n_tile) * 128) + 1024 + sizeof(Barriers);
+}
+
+cudaError_t launch_conv_umma(const UmmaArgs& a, const void* xmap, const void* wmap, int sm_count,
+                             cudaStream_t stream) {
+  const int stages = pick_stages(a.n_tile);
+  if (stages < 2) return cudaErrorInvalidValue;
+  const size_t smem = umma_smem_bytes(a.n_tile);
+  int cols = 32;
+  while (cols < 2 * a.n_tile) cols *= 2;
+  if (cols > 512) return cudaErrorInvalidValue;
+  const long long n_items = (long long)a.tiles_n * a.tiles_t * a.tiles_h * a.tiles_w * a.n_bundles;
+  if (n_items <= 0) return cudaSuccess;
+  const int grid = int(n_items < sm_count ? n_items : sm_count);
+  CUtensorMap xm, wm;
+  memcpy(&xm, xmap, sizeof(CUtensorMap));
+  memcpy(&wm, wmap, sizeof(CUtensorMap));
+  cudaError_t e;
+  if (a.dense) {
+    static bool attr_done_d = false;
+    if (!attr_done_d) {
+      e = cudaFuncSetAttribute(conv3d_umma_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+      if (e != cudaSuccess) return e;
+      attr_done_d = true;
+    }
+    conv3d_umma_kernel<true><<<grid, kThreadsUmma, smem, stream>>>(xm, wm, a, stages, cols);
+  } else {
+    static bool attr_done_s = false;
+    if (!attr_done_s) {
+      e = cudaFuncSetAttribute(conv3d_umma_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+      if (e != cudaSuccess) return e;
+      attr_done_s = true;
+    }
+    conv3d_umma_kernel<false><<<grid, kThreadsUmma, smem, stream>>>(xm, wm, a, stages, cols);
+  }
+  return cudaGetLastError();
+}
+
+}  // namespace rt3d

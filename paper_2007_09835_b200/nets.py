@@ -1,0 +1,162 @@
+"""Layer and network runners on top of the C-ABI binding (orchestration only).
+
+A layer owns a packed weight handle and a device bias; a network is the list of calls the
+C3D-shaped and R(2+1)D-shaped forward passes make (Section 5 of the paper names the
+models; pooling / residual structure follows the cited architectures).  Every numerical
+step is a call into librt3d; torch provides device memory and streams.
+"""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+from . import binding as B
+
+
+def pitch_for(c: int, dtype) -> int:
+    """Channel pitch that satisfies the library's alignment rule (16 bytes per voxel row start)."""
+    mult = 8 if dtype == torch.bfloat16 else 4
+    return -(-c // mult) * mult
+
+
+def to_device(x_np: np.ndarray, dtype=torch.bfloat16, c_stride: int | None = None, device="cuda"):
+    """float32 numpy NDHWC -> device tensor [n,t,h,w,c_stride] (extra channels zero)."""
+    c = x_np.shape[-1]
+    cs = pitch_for(c, dtype) if c_stride is None else c_stride
+    t = torch.zeros(x_np.shape[:-1] + (cs,), dtype=dtype, device=device)
+    t[..., :c] = torch.from_numpy(np.ascontiguousarray(x_np)).to(dtype).to(device)
+    return t
+
+
+def to_numpy(t: torch.Tensor, c: int) -> np.ndarray:
+    return t[..., :c].float().cpu().numpy()
+
+
+class ConvLayer:
+    """One convolution layer: packed weights (KGS mask or dense) + bias on the device."""
+
+    def __init__(self, spec, w, bias, mask, g_m=4, g_n=4, dtype=torch.bfloat16, dense=False, device="cuda"):
+        self.spec = spec
+        self.dtype = dtype
+        cd = B.RT3D_BF16 if dtype == torch.bfloat16 else B.RT3D_F32
+        self.dense = dense
+        self.packed = B.rt3d_pack_dense(w, cd) if dense else B.rt3d_pack_kgs(w, mask, g_m, g_n, cd)
+        self.bias = None if bias is None else torch.from_numpy(np.ascontiguousarray(bias, np.float32)).to(device)
+        self.device = device
+
+    def out_shape(self, x: torch.Tensor):
+        n, t, h, w, _ = x.shape
+        to, ho, wo = self.spec.out_extent(t, h, w)
+        return (n, to, ho, wo, pitch_for(self.spec.cout, self.dtype))
+
+    def alloc_out(self, x: torch.Tensor) -> torch.Tensor:
+        return torch.zeros(self.out_shape(x), dtype=self.dtype, device=x.device)
+
+    def __call__(self, x: torch.Tensor, y: torch.Tensor | None = None, algo=B.ALGO_AUTO, relu=None, stream=None):
+        if y is None:
+            y = self.alloc_out(x)
+        xd = B.tensor_desc(x, self.spec.cin)
+        yd = B.tensor_desc(y, self.spec.cout)
+        fn = B.rt3d_conv3d_dense if self.dense else B.rt3d_conv3d_sparse
+        fn(xd, self.packed, self.bias, yd, self.spec.stride, self.spec.pad,
+           self.spec.relu if relu is None else relu, algo, stream)
+        return y
+
+    def cost(self, x: torch.Tensor):
+        return B.rt3d_conv3d_cost(B.tensor_desc(x, self.spec.cin), self.packed, self.spec.stride, self.spec.pad)
+
+
+def maxpool(x: torch.Tensor, c: int, pool, y: torch.Tensor | None = None, stream=None) -> torch.Tensor:
+    n, t, h, w, cs = x.shape
+    ext = [(d + 2 * p - k) // s + 1 for d, p, k, s in zip((t, h, w), pool.pad, pool.k, pool.stride)]
+    if y is None:
+        y = torch.zeros((n, ext[0], ext[1], ext[2], cs), dtype=x.dtype, device=x.device)
+    B.rt3d_maxpool3d(B.tensor_desc(x, c), pool.k, pool.stride, pool.pad, B.tensor_desc(y, c), stream)
+    return y
+
+
+def add_relu(a: torch.Tensor, b: torch.Tensor, c: int, relu=True, y: torch.Tensor | None = None, stream=None):
+    if y is None:
+        y = torch.zeros_like(a)
+    B.rt3d_add_relu(B.tensor_desc(a, c), B.tensor_desc(b, c), relu, B.tensor_desc(y, c), stream)
+    return y
+
+
+class Workspace:
+    """Activation buffers keyed by (name, shape): allocated on first use, reused afterwards so a
+    steady-state forward pass allocates nothing."""
+
+    def __init__(self):
+        self.bufs = {}
+
+    def get(self, name, shape, dtype, device):
+        key = (name, tuple(shape), dtype)
+        if key not in self.bufs:
+            self.bufs[key] = torch.zeros(shape, dtype=dtype, device=device)
+        return self.bufs[key]
+
+
+class C3DNet:
+    """C3D-shaped forward: 8 convs (3x3x3, ReLU) and 5 max-pools.  `layers` maps conv name -> ConvLayer."""
+
+    def __init__(self, plan, layers):
+        self.plan = plan
+        self.layers = layers
+        self.ws = Workspace()
+
+    def forward(self, x: torch.Tensor, algo=B.ALGO_AUTO, keep=None, stream=None) -> torch.Tensor:
+        c = self.plan[0].cin
+        for op in self.plan:
+            if hasattr(op, "cout"):
+                layer = self.layers[op.name]
+                y = self.ws.get(op.name, layer.out_shape(x), x.dtype, x.device)
+                x = layer(x, y, algo=algo, stream=stream)
+                c = op.cout
+            else:
+                n, t, h, w, cs = x.shape
+                ext = [(d + 2 * p - k) // s + 1 for d, p, k, s in zip((t, h, w), op.pad, op.k, op.stride)]
+                y = self.ws.get(op.name, (n, ext[0], ext[1], ext[2], cs), x.dtype, x.device)
+                x = maxpool(x, c, op, y, stream=stream)
+            if keep is not None:
+                keep[op.name] = x
+        return x
+
+    def n_launches(self) -> int:
+        return len(self.plan)
+
+
+class R2Plus1DNet:
+    """R(2+1)D-18-shaped forward: stem, then residual blocks of two factorised convs each
+    (spatial 1x3x3 then temporal 3x1x1), optional 1x1x1 strided projection, add + ReLU."""
+
+    def __init__(self, stem, blocks, layers):
+        self.stem, self.blocks, self.layers = stem, blocks, layers
+        self.ws = Workspace()
+
+    def _conv(self, spec, x, algo, stream):
+        layer = self.layers[spec.name]
+        y = self.ws.get(spec.name, layer.out_shape(x), x.dtype, x.device)
+        return layer(x, y, algo=algo, stream=stream)
+
+    def forward(self, x: torch.Tensor, algo=B.ALGO_AUTO, keep=None, stream=None) -> torch.Tensor:
+        for spec in self.stem:
+            x = self._conv(spec, x, algo, stream)
+            if keep is not None:
+                keep[spec.name] = x
+        for blk in self.blocks:
+            inp = x
+            for spec in blk.convs:
+                x = self._conv(spec, x, algo, stream)
+                if keep is not None:
+                    keep[spec.name] = x
+            sc = inp if blk.shortcut is None else self._conv(blk.shortcut, inp, algo, stream)
+            if keep is not None and blk.shortcut is not None:
+                keep[blk.shortcut.name] = sc
+            y = self.ws.get(blk.name + ".out", x.shape, x.dtype, x.device)
+            x = add_relu(x, sc, blk.convs[-1].cout, True, y, stream=stream)
+            if keep is not None:
+                keep[blk.name + ".out"] = x
+        return x
+
+    def n_launches(self) -> int:
+        return len(self.stem) + sum(5 + (blk.shortcut is not None) for blk in self.blocks)

@@ -1,0 +1,224 @@
+"""GPU parity: the CUDA library (through its C ABI) against the CPU oracle on the same seeded inputs.
+
+Tolerances (global max norm over the whole output, both sides):
+  fp32:  max|err| <= 1e-3 * max|ref|
+  bf16 inputs, fp32 accumulation, bf16 outputs:  max|err| <= 2e-2 * max|ref|
+A comparison is void unless at least 10 % of the reference outputs are non-zero.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import rt3d_synth as synth
+import paper_2007_09835_b200 as rt3d
+from paper_2007_09835_b200 import nets
+
+pytestmark = pytest.mark.gpu
+
+TOL = {torch.float32: 1e-3, torch.bfloat16: 2e-2}
+
+
+def check(y, ref, dtype, what=""):
+    assert y.shape == ref.shape, (y.shape, ref.shape)
+    assert np.isfinite(y).all(), f"{what}: non-finite output"
+    scale = np.abs(ref).max()
+    assert (ref != 0).mean() >= 0.10, f"{what}: reference is mostly zero, comparison void"
+    err = np.abs(y - ref).max()
+    assert err <= TOL[dtype] * scale, f"{what}: max|err| {err:.4g} > {TOL[dtype]} * {scale:.4g}"
+    return err / scale
+
+
+def run_case(spec, n, t, h, w, g_m, g_n, mask_kind, mask_arg, dtype, algo, cfg=7, layer=0, dense=False,
+             x_pitch=None, bias=True):
+    L = synth.make_layer(spec, cfg, layer, g_m, g_n, mask_kind, mask_arg)
+    x = synth.make_input(cfg * 100 + layer, (n, t, h, w, spec.cin))
+    b = L["bias"] if bias else None
+    ref = oracle.conv3d(x, L["w"], None if dense else L["mask"], b, spec.stride, spec.pad, spec.relu,
+                        round_bf16=(dtype == torch.bfloat16))
+    lay = nets.ConvLayer(spec, L["w"], b, L["mask"], g_m, g_n, dtype, dense=dense)
+    xd = nets.to_device(x, dtype, x_pitch)
+    y = lay(xd, algo=algo)
+    assert rt3d.rt3d_last_device_status() == rt3d.OK
+    return nets.to_numpy(y, spec.cout), ref, lay, xd, y
+
+
+# ----------------------------------------------------------------------- cfg0 (fp32)
+@pytest.mark.parametrize("relu", [True, False])
+def test_cfg0_fp32_kgs_14_of_27(relu):
+    spec = synth.ConvSpec("cfg0", 16, 32, (3, 3, 3), (1, 1, 1), (1, 1, 1), relu)
+    y, ref, *_ = run_case(spec, 1, 8, 28, 28, 4, 4, "exact_per_group", 14, torch.float32, rt3d.ALGO_AUTO, cfg=0)
+    check(y, ref, torch.float32, "cfg0")
+
+
+def test_cfg0_dense_path_fp32():
+    spec = synth.ConvSpec("cfg0", 16, 32, (3, 3, 3), (1, 1, 1), (1, 1, 1), True)
+    y, ref, *_ = run_case(spec, 1, 8, 28, 28, 4, 4, "none", None, torch.float32, rt3d.ALGO_AUTO, cfg=0, dense=True)
+    check(y, ref, torch.float32, "cfg0 dense")
+
+
+# ------------------------------------------------------------- CUDA-core kernel, odd shapes
+SIMT_CASES = [
+    # cin, cout, k, stride, pad, (n,t,h,w), g_m, g_n, density
+    (5, 6, (3, 3, 3), (1, 1, 1), (1, 1, 1), (2, 4, 5, 6), 4, 4, 0.5),
+    (3, 45, (1, 7, 7), (1, 2, 2), (0, 3, 3), (1, 3, 20, 22), 4, 4, 0.4),
+    (45, 64, (3, 1, 1), (1, 1, 1), (1, 0, 0), (1, 5, 6, 7), 4, 4, 0.4),
+    (24, 40, (3, 3, 3), (2, 2, 2), (1, 1, 1), (1, 6, 9, 9), 8, 4, 0.3),
+    (16, 16, (1, 1, 1), (2, 2, 2), (0, 0, 0), (2, 4, 6, 6), 8, 8, 0.6),
+    (7, 9, (2, 2, 1), (1, 1, 1), (0, 1, 0), (1, 4, 4, 4), 3, 2, 0.5),
+]
+
+
+@pytest.mark.parametrize("case", SIMT_CASES)
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_simt_kernel_against_oracle(case, dtype):
+    cin, cout, k, stride, pad, (n, t, h, w), g_m, g_n, d = case
+    spec = synth.ConvSpec("s", cin, cout, k, stride, pad, True)
+    y, ref, *_ = run_case(spec, n, t, h, w, g_m, g_n, "bernoulli", d, dtype, rt3d.ALGO_SIMT)
+    check(y, ref, dtype, f"simt {case}")
+
+
+# ------------------------------------------------------------- tensor-core kernel, small shapes
+UMMA_CASES = [
+    # cin, cout, k, stride, pad, (n,t,h,w), g_m, g_n, density
+    (64, 64, (3, 3, 3), (1, 1, 1), (1, 1, 1), (2, 4, 8, 8), 4, 4, 0.4),      # 4 full tiles
+    (64, 64, (3, 3, 3), (1, 1, 1), (1, 1, 1), (1, 3, 7, 9), 4, 4, 0.4),      # ragged boxes
+    (128, 256, (3, 3, 3), (1, 1, 1), (1, 1, 1), (1, 4, 12, 12), 4, 4, 0.4),  # 2 chunks, n_tile 256
+    (96, 80, (3, 3, 3), (1, 1, 1), (1, 1, 1), (1, 2, 8, 8), 8, 4, 0.5),      # partial chunk, n_tile 80
+    (144, 45, (3, 1, 1), (1, 1, 1), (1, 0, 0), (1, 6, 6, 6), 4, 4, 0.4),     # ragged M, 3x1x1
+    (64, 512, (1, 1, 1), (1, 1, 1), (0, 0, 0), (2, 2, 9, 9), 8, 8, 0.5),     # two bundles, Ks = 1
+    (3, 64, (3, 3, 3), (1, 1, 1), (1, 1, 1), (1, 4, 10, 10), 4, 4, 0.3),     # C_in = 3 (pitch 8)
+    (64, 64, (1, 3, 3), (1, 1, 1), (0, 1, 1), (3, 5, 6, 6), 4, 4, 0.4),
+]
+
+
+@pytest.mark.parametrize("case", UMMA_CASES)
+def test_umma_kernel_against_oracle(case):
+    cin, cout, k, stride, pad, (n, t, h, w), g_m, g_n, d = case
+    spec = synth.ConvSpec("u", cin, cout, k, stride, pad, True)
+    y, ref, *_ = run_case(spec, n, t, h, w, g_m, g_n, "bernoulli", d, torch.bfloat16, rt3d.ALGO_UMMA)
+    check(y, ref, torch.bfloat16, f"umma {case}")
+
+
+UMMA_STRIDED = [
+    (64, 64, (3, 3, 3), (2, 2, 2), (1, 1, 1), (1, 6, 11, 12), 4, 4, 0.4),
+    (64, 230, (1, 3, 3), (1, 2, 2), (0, 1, 1), (1, 4, 14, 14), 4, 4, 0.4),
+    (230, 128, (3, 1, 1), (2, 1, 1), (1, 0, 0), (1, 8, 7, 7), 4, 4, 0.4),
+    (64, 128, (1, 1, 1), (2, 2, 2), (0, 0, 0), (2, 4, 10, 10), 4, 4, 1.0),
+    (3, 45, (1, 7, 7), (1, 2, 2), (0, 3, 3), (1, 2, 28, 28), 4, 4, 0.4),
+]
+
+
+@pytest.mark.parametrize("case", UMMA_STRIDED)
+def test_umma_kernel_strided(case):
+    cin, cout, k, stride, pad, (n, t, h, w), g_m, g_n, d = case
+    spec = synth.ConvSpec("u", cin, cout, k, stride, pad, False)
+    y, ref, *_ = run_case(spec, n, t, h, w, g_m, g_n, "bernoulli", d, torch.bfloat16, rt3d.ALGO_UMMA)
+    check(y, ref, torch.bfloat16, f"umma strided {case}")
+
+
+def test_umma_dense_entry_point():
+    spec = synth.ConvSpec("u", 128, 128, (3, 3, 3), (1, 1, 1), (1, 1, 1), True)
+    y, ref, *_ = run_case(spec, 2, 4, 8, 8, 4, 4, "none", None, torch.bfloat16, rt3d.ALGO_UMMA, dense=True)
+    check(y, ref, torch.bfloat16, "umma dense")
+
+
+def test_umma_bundle_with_every_group_pruned_outputs_bias():
+    spec = synth.ConvSpec("u", 64, 512, (3, 3, 3), (1, 1, 1), (1, 1, 1), True)
+    L = synth.make_layer(spec, 7, 3, 4, 4, "bernoulli", 0.4)
+    L["mask"][256:] = 0                                   # second bundle of 256 channels: nothing kept
+    x = synth.make_input(703, (1, 2, 8, 8, 64))
+    ref = oracle.conv3d(x, L["w"], L["mask"], L["bias"], spec.stride, spec.pad, True, round_bf16=True)
+    lay = nets.ConvLayer(spec, L["w"], L["bias"], L["mask"], 4, 4, torch.bfloat16)
+    y = nets.to_numpy(lay(nets.to_device(x), algo=rt3d.ALGO_UMMA), 512)
+    check(y, ref, torch.bfloat16, "empty bundle")
+    np.testing.assert_allclose(y[..., 256:], np.broadcast_to(np.maximum(L["bias"][256:], 0), y[..., 256:].shape),
+                               rtol=1e-2, atol=1e-4)
+
+
+def test_umma_and_simt_agree_and_are_deterministic():
+    spec = synth.ConvSpec("u", 128, 64, (3, 3, 3), (1, 1, 1), (1, 1, 1), True)
+    y1, ref, lay, xd, yt = run_case(spec, 1, 4, 10, 10, 4, 4, "bernoulli", 0.4, torch.bfloat16, rt3d.ALGO_UMMA)
+    first = yt.clone()
+    lay(xd, yt, algo=rt3d.ALGO_UMMA)
+    torch.cuda.synchronize()
+    assert torch.equal(first, yt)                          # no atomics, no split-K: bitwise repeatable
+    ys = nets.to_numpy(lay(xd, algo=rt3d.ALGO_SIMT), 64)
+    check(ys, ref, torch.bfloat16, "simt")
+    assert np.abs(ys - y1).max() <= 2e-2 * np.abs(ref).max()
+
+
+def test_output_pitch_guard_band_untouched():
+    spec = synth.ConvSpec("u", 64, 40, (3, 3, 3), (1, 1, 1), (1, 1, 1), False)
+    L = synth.make_layer(spec, 7, 5, 4, 4, "bernoulli", 0.5)
+    x = synth.make_input(705, (1, 2, 6, 6, 64))
+    lay = nets.ConvLayer(spec, L["w"], L["bias"], L["mask"], 4, 4, torch.bfloat16)
+    for algo in (rt3d.ALGO_UMMA, rt3d.ALGO_SIMT):
+        y = torch.full((1, 2, 6, 6, 48), 777.0, dtype=torch.bfloat16, device="cuda")   # pitch 48 > 40 channels
+        lay(nets.to_device(x), y, algo=algo)
+        torch.cuda.synchronize()
+        assert (y[..., 40:] == 777.0).all()
+        ref = oracle.conv3d(x, L["w"], L["mask"], L["bias"], spec.stride, spec.pad, False, round_bf16=True)
+        check(nets.to_numpy(y, 40), ref, torch.bfloat16, "pitch")
+
+
+# ------------------------------------------------------------------------- cfg1, full size
+@pytest.mark.parametrize("mode", ["kgs", "dense", "vanilla"])
+def test_cfg1_c3d_conv3a_full_size(mode):
+    spec = synth.ConvSpec("conv3a", 128, 256, (3, 3, 3), (1, 1, 1), (1, 1, 1), True)
+    if mode == "kgs":
+        args = ("bernoulli", 0.4)
+    elif mode == "vanilla":
+        args = ("vanilla_total", round(64 * 32 * 0.4))
+    else:
+        args = ("none", None)
+    y, ref, *_ = run_case(spec, 8, 8, 28, 28, 4, 4, *args, torch.bfloat16, rt3d.ALGO_AUTO, cfg=1,
+                          dense=(mode == "dense"))
+    rel = check(y, ref, torch.bfloat16, f"cfg1 {mode}")
+    assert rel < 1e-2
+
+
+# ------------------------------------------------------------------ host entry point, glue
+def test_conv3d_host_entry_point_matches_device_call():
+    spec = synth.ConvSpec("h", 64, 64, (3, 3, 3), (1, 1, 1), (1, 1, 1), True)
+    L = synth.make_layer(spec, 7, 9, 4, 4, "bernoulli", 0.4)
+    x = synth.make_input(709, (2, 4, 8, 8, 64))
+    lay = nets.ConvLayer(spec, L["w"], L["bias"], L["mask"], 4, 4, torch.bfloat16)
+    yd = lay(nets.to_device(x))
+    xh = torch.from_numpy(x).to(torch.bfloat16).pin_memory()
+    yh = torch.zeros((2, 4, 8, 8, 64), dtype=torch.bfloat16).pin_memory()
+    bh = torch.from_numpy(L["bias"]).pin_memory()
+    rt3d.rt3d_conv3d_host(rt3d.tensor_desc(xh), lay.packed, bh, rt3d.tensor_desc(yh), spec.stride, spec.pad, True)
+    assert torch.equal(yh, yd.cpu())
+
+
+def test_maxpool_and_add_relu_against_oracle():
+    for dtype in (torch.bfloat16, torch.float32):
+        for c, shape, pool in ((64, (2, 4, 8, 8), synth.PoolSpec("p", (2, 2, 2), (2, 2, 2), (0, 0, 0))),
+                               (64, (1, 3, 14, 14), synth.PoolSpec("p", (1, 2, 2), (1, 2, 2), (0, 0, 0))),
+                               (16, (1, 2, 7, 7), synth.PoolSpec("p", (2, 2, 2), (2, 2, 2), (0, 1, 1))),
+                               (5, (1, 2, 6, 6), synth.PoolSpec("p", (2, 2, 2), (2, 2, 2), (0, 0, 0)))):
+            x = synth.make_input(800 + c, shape + (c,))
+            xr = oracle.bf16_round(x) if dtype == torch.bfloat16 else x
+            y = nets.to_numpy(nets.maxpool(nets.to_device(x, dtype), c, pool), c)
+            np.testing.assert_array_equal(y, oracle.maxpool3d(xr, pool.k, pool.stride, pool.pad))
+        a = synth.make_input(901, (2, 3, 5, 5, 24))
+        b = synth.make_input(902, (2, 3, 5, 5, 24))
+        ar, br = (oracle.bf16_round(a), oracle.bf16_round(b)) if dtype == torch.bfloat16 else (a, b)
+        for relu in (True, False):
+            y = nets.to_numpy(nets.add_relu(nets.to_device(a, dtype), nets.to_device(b, dtype), 24, relu), 24)
+            ref = oracle.add_relu(ar, br, relu)
+            if dtype == torch.bfloat16:
+                ref = oracle.bf16_round(ref)
+            np.testing.assert_array_equal(y, ref)
+
+
+def test_cost_model_counts_kept_macs():
+    spec = synth.ConvSpec("c", 16, 32, (3, 3, 3), (1, 1, 1), (1, 1, 1), True)
+    L = synth.make_layer(spec, 0, 0, 4, 4, "exact_per_group", 14)
+    lay = nets.ConvLayer(spec, L["w"], L["bias"], L["mask"], 4, 4, torch.float32)
+    x = nets.to_device(synth.make_input(0, (1, 8, 28, 28, 16)), torch.float32)
+    kept, dense, nbytes = lay.cost(x)
+    assert dense == spec.dense_macs(1, 8, 28, 28)
+    assert kept * 27 == dense * 14
+    assert nbytes == (6272 * 16 + 6272 * 32) * 4 + 448 * 16 * 4 + 448 * 2 + 33 * 4 + 32 * 4
