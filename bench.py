@@ -147,6 +147,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--l2-warm", action="store_true", help="reuse one buffer set (operands stay in L2); default rotates sets")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":
@@ -171,7 +172,7 @@ def main():
     x0 = nets.to_device(x, torch.bfloat16, device=dev)
     y0 = sparse.alloc_out(x0)
     set_bytes = x0.numel() * 2 + y0.numel() * 2
-    n_sets = max(2, -(-int(2.5 * L2_BYTES) // set_bytes))
+    n_sets = 1 if args.l2_warm else max(2, -(-int(2.5 * L2_BYTES) // set_bytes))
     xs = [x0] + [x0.clone() for _ in range(n_sets - 1)]
     ys = [y0] + [torch.zeros_like(y0) for _ in range(n_sets - 1)]
     kept_macs, dense_macs, alg_bytes = sparse.cost(x0)
@@ -235,7 +236,8 @@ def main():
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": per_step_ms, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": WORKLOAD, "global_batch": CFG["n"] * world, "parallelism": f"batch replicas x{world}",
-                   "l2": f"rotating {n_sets} input/output buffer sets ({n_sets * set_bytes / 2**20:.0f} MiB > 2x L2)",
+                   "l2": ("warm: one buffer set reused every step" if args.l2_warm else
+                          f"rotating {n_sets} input/output buffer sets ({n_sets * set_bytes / 2**20:.0f} MiB > 2x L2)"),
                    "kernel": "tcgen05" if algo == rt3d.ALGO_UMMA else "cuda-core"},
         "dense_equiv_tflops": world * 2.0 * dense_macs / (per_step_ms * 1e-3) / 1e12,
         "dense_path_tflops": world * 2.0 * dense_macs / (dense_ms / args.steps * 1e-3) / 1e12,

@@ -13,7 +13,7 @@ import os
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "librt3d.so")
+LIB_PATH = os.environ.get("RT3D_LIB") or os.path.join(_HERE, "librt3d.so")   # RT3D_LIB: alternative build of the same library
 
 RT3D_F32, RT3D_BF16 = 0, 1
 ALGO_AUTO, ALGO_SIMT, ALGO_UMMA = 0, 1, 2

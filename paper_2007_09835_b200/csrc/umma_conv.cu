@@ -193,31 +193,50 @@ conv3d_umma_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_consta
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
-      uint32_t k = 0;
+      int stage = 0;
+      uint32_t phase = 0;
       bool ok = true;
+      const uint32_t tx_bytes = uint32_t(box_rows) * 128u + b_bytes;
       for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
         const ItemCoord c = decode_item(a, item, n_mtiles);
         const int s_begin = kDense ? c.bundle * a.steps_dense : a.step_ptr[c.bundle];
         const int nsteps = kDense ? a.steps_dense : a.step_ptr[c.bundle + 1] - s_begin;
         const int wq = c.w0 * a.g.sw - a.g.pw, hq = c.h0 * a.g.sh - a.g.ph, tq = c.t0 * a.g.st - a.g.pt;
-        for (int i = 0; i < nsteps; ++i, ++k) {
-          const int stage = k % stages;
-          const uint32_t round = k / stages;
-          if (!mbar_wait(smem_u32(&bars->empty[stage]), (round & 1u) ^ 1u, bars, err, 1)) { ok = false; break; }
-          int kt, kh, kw, ch;
+        // Everything a step needs is computed (dense) or fetched one step ahead (indexed) before the
+        // wait on the stage, so a freed stage is re-armed without further latency.
+        int kt = 0, kh = 0, kw = 0, ch = 0;
+        int enc_next = (!kDense && nsteps > 0) ? __ldg(a.steps + s_begin) : 0;
+        int wrow = s_begin * a.n_tile;
+        for (int i = 0; i < nsteps; ++i, wrow += a.n_tile) {
+          int c_ch, c_w, c_h, c_t;
           if (kDense) {
-            ch = i % a.n_chunks;
-            const int pos = i / a.n_chunks;
-            kw = pos % a.g.Kw; kh = (pos / a.g.Kw) % a.g.Kh; kt = pos / (a.g.Kw * a.g.Kh);
+            c_ch = ch * 64; c_w = wq + kw; c_h = hq + kh; c_t = tq + kt;
+            if (++ch == a.n_chunks) { ch = 0; if (++kw == a.g.Kw) { kw = 0; if (++kh == a.g.Kh) { kh = 0; ++kt; } } }
           } else {
-            const int enc = a.steps[s_begin + i];
-            kt = (enc >> 24) & 63; kh = (enc >> 18) & 63; kw = (enc >> 12) & 63; ch = enc & 4095;
+            const int enc = enc_next;
+            if (i + 1 < nsteps) enc_next = __ldg(a.steps + s_begin + i + 1);
+            c_t = tq + ((enc >> 24) & 63); c_h = hq + ((enc >> 18) & 63); c_w = wq + ((enc >> 12) & 63);
+            c_ch = (enc & 4095) * 64;
           }
           const uint32_t full = smem_u32(&bars->full[stage]);
           const uint32_t a_dst = tiles_base + stage * stage_bytes;
-          mbar_expect_tx(full, uint32_t(box_rows) * 128u + b_bytes);
-          tma_load_5d(a_dst, &xmap, full, ch * 64, wq + kw, hq + kh, tq + kt, c.n0);
-          tma_load_2d(a_dst + kABytes, &wmap, full, 0, (s_begin + i) * a.n_tile);
+          if (!mbar_wait(smem_u32(&bars->empty[stage]), phase ^ 1u, bars, err, 1)) { ok = false; break; }
+#if defined(RT3D_EXPERIMENT) && RT3D_EXPERIMENT == 1      /* timing ablation: A tile loaded once per item */
+          mbar_expect_tx(full, i == 0 ? tx_bytes : b_bytes);
+          if (i == 0) tma_load_5d(a_dst, &xmap, full, c_ch, c_w, c_h, c_t, c.n0);
+          tma_load_2d(a_dst + kABytes, &wmap, full, 0, wrow);
+#elif defined(RT3D_EXPERIMENT) && RT3D_EXPERIMENT == 2    /* timing ablation: B tile loaded once per item */
+          mbar_expect_tx(full, i == 0 ? tx_bytes : tx_bytes - b_bytes);
+          tma_load_5d(a_dst, &xmap, full, c_ch, c_w, c_h, c_t, c.n0);
+          if (i == 0) tma_load_2d(a_dst + kABytes, &wmap, full, 0, wrow);
+#elif defined(RT3D_EXPERIMENT) && RT3D_EXPERIMENT == 4    /* timing ablation: no loads at all */
+          mbar_arrive(full);
+#else
+          mbar_expect_tx(full, tx_bytes);
+          tma_load_5d(a_dst, &xmap, full, c_ch, c_w, c_h, c_t, c.n0);
+          tma_load_2d(a_dst + kABytes, &wmap, full, 0, wrow);
+#endif
+          if (++stage == stages) { stage = 0; phase ^= 1u; }
         }
       }
     }
@@ -225,7 +244,8 @@ conv3d_umma_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_consta
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
       const uint32_t idesc = instr_desc_bf16(a.n_tile);
-      uint32_t k = 0, j = 0;
+      uint32_t j = 0, phase = 0;
+      int stage = 0;
       bool ok = true;
       for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++j) {
         const int bundle = item / n_mtiles;
@@ -234,17 +254,20 @@ conv3d_umma_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_consta
         if (!mbar_wait(smem_u32(&bars->tmem_empty[buf]), ((j >> 1) & 1u) ^ 1u, bars, err, 2)) break;
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + buf * uint32_t(a.n_tile);
-        for (int i = 0; i < nsteps; ++i, ++k) {
-          const int stage = k % stages;
-          if (!mbar_wait(smem_u32(&bars->full[stage]), (k / stages) & 1u, bars, err, 3)) { ok = false; break; }
+        for (int i = 0; i < nsteps; ++i) {
+          if (!mbar_wait(smem_u32(&bars->full[stage]), phase, bars, err, 3)) { ok = false; break; }
           tc_fence_after();
           const uint32_t a_addr = tiles_base + stage * stage_bytes;
           const uint64_t adesc = smem_desc_sw128(a_addr);
           const uint64_t bdesc = smem_desc_sw128(a_addr + kABytes);
 #pragma unroll
           for (int kk = 0; kk < 4; ++kk)      // 4 x K=16 per 64-channel chunk: +32 bytes = +2 in descriptor units
+#if defined(RT3D_EXPERIMENT) && RT3D_EXPERIMENT == 3      /* timing ablation: one MMA per step instead of four */
+            if (kk == 0)
+#endif
             umma_bf16(d_tmem, adesc + 2 * kk, bdesc + 2 * kk, idesc, (i | kk) ? 1u : 0u);
           umma_commit(smem_u32(&bars->empty[stage]));
+          if (++stage == stages) { stage = 0; phase ^= 1u; }
         }
         if (!ok) break;
         if (nsteps > 0) umma_commit(smem_u32(&bars->tmem_full[buf]));

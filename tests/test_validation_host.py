@@ -1,0 +1,64 @@
+"""Host-side argument validation of the compute entry points (no GPU, nothing is launched):
+every shape / dtype / alignment error is reported before any CUDA call is made."""
+import ctypes
+
+import numpy as np
+import pytest
+
+import rt3d_synth as synth
+import paper_2007_09835_b200 as rt3d
+from paper_2007_09835_b200 import binding as B
+
+FAKE = 0x10000     # a 16-byte aligned, never dereferenced address
+
+
+def tensor(n, t, h, w, c, cs=None, dtype=B.RT3D_BF16, data=FAKE):
+    return B.Tensor(data, n, t, h, w, c, c if cs is None else cs, dtype)
+
+
+@pytest.fixture(scope="module")
+def packed():
+    spec = synth.ConvSpec("v", 16, 32, (3, 3, 3), (1, 1, 1), (1, 1, 1))
+    L = synth.make_layer(spec, 5, 0, 4, 4, "bernoulli", 0.5)
+    return B.rt3d_pack_kgs(L["w"], L["mask"], 4, 4, B.RT3D_BF16)
+
+
+def call(packed, x, y, stride=(1, 1, 1), pad=(1, 1, 1), algo=0, fn="rt3d_conv3d_sparse"):
+    p = B.ConvParams(*stride, *pad, 1, algo)
+    return getattr(B.lib(), fn)(ctypes.byref(x), packed.handle, None, ctypes.byref(p), ctypes.byref(y), None)
+
+
+def test_conv_argument_errors(packed):
+    good_x, good_y = tensor(1, 4, 8, 8, 16), tensor(1, 4, 8, 8, 32)
+    assert call(packed, tensor(1, 4, 8, 8, 24), good_y) == B.ERR_SHAPE                 # channels != N
+    assert call(packed, good_x, tensor(1, 4, 8, 8, 16)) == B.ERR_SHAPE                 # channels != M
+    assert call(packed, good_x, tensor(1, 4, 8, 7, 32)) == B.ERR_SHAPE                 # wrong output extent
+    assert call(packed, tensor(1, 4, 8, 8, 16, dtype=B.RT3D_F32), good_y) == B.ERR_SHAPE   # dtype != handle's
+    assert call(packed, good_x, good_y, stride=(0, 1, 1)) == B.ERR_INVALID_ARG
+    assert call(packed, good_x, good_y, pad=(-1, 1, 1)) == B.ERR_INVALID_ARG
+    assert call(packed, good_x, good_y, algo=9) == B.ERR_INVALID_ARG
+    assert call(packed, tensor(1, 4, 8, 8, 16, data=0), good_y) == B.ERR_INVALID_ARG   # NULL data
+    assert call(packed, tensor(1, 4, 8, 8, 16, cs=12), good_y) == B.ERR_INVALID_ARG    # pitch < channels
+    assert call(packed, tensor(1, 4, 8, 8, 16, cs=20), good_y) == B.ERR_INVALID_ARG    # pitch not a multiple of 8
+    assert call(packed, tensor(1, 4, 8, 8, 16, data=FAKE + 2), good_y) == B.ERR_INVALID_ARG   # misaligned
+    assert call(packed, good_x, good_y) == B.ERR_INVALID_ARG                           # x and y overlap
+    assert call(packed, tensor(1, 1, 1, 1, 16), tensor(1, 1, 1, 1, 32), pad=(0, 0, 0)) == B.ERR_SHAPE   # smaller than kernel
+    far_y = tensor(1, 4, 8, 8, 32, data=FAKE + (1 << 24))
+    assert call(packed, good_x, far_y, fn="rt3d_conv3d_dense") == B.ERR_INVALID_ARG    # dense entry needs a dense handle
+
+
+def test_cost_needs_no_device(packed):
+    k, d, b = B.rt3d_conv3d_cost(tensor(2, 4, 8, 8, 16), packed, (1, 1, 1), (1, 1, 1))
+    assert d == 2 * 4 * 8 * 8 * 32 * 16 * 27 and 0 < k < d and b > 0
+
+
+def test_pool_and_add_argument_errors():
+    x = tensor(1, 4, 8, 8, 16)
+    y = tensor(1, 2, 4, 4, 16, data=FAKE + (1 << 24))
+    lib = B.lib()
+    bad = tensor(1, 2, 4, 5, 16, data=FAKE + (1 << 24))
+    assert lib.rt3d_maxpool3d(ctypes.byref(x), 2, 2, 2, 2, 2, 2, 0, 0, 0, ctypes.byref(bad), None) == B.ERR_SHAPE
+    assert lib.rt3d_maxpool3d(ctypes.byref(x), 2, 2, 2, 2, 2, 2, 2, 0, 0, ctypes.byref(y), None) == B.ERR_INVALID_ARG
+    assert lib.rt3d_maxpool3d(ctypes.byref(x), 0, 2, 2, 2, 2, 2, 0, 0, 0, ctypes.byref(y), None) == B.ERR_INVALID_ARG
+    a, b = tensor(1, 2, 4, 4, 16), tensor(1, 2, 4, 4, 24)
+    assert lib.rt3d_add_relu(ctypes.byref(a), ctypes.byref(b), 1, ctypes.byref(a), None) == B.ERR_SHAPE
