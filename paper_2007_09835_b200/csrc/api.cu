@@ -232,6 +232,72 @@ rt3d_status encode_xmap(const rt3d_tensor* x, const ConvGeom& g, const TileBox& 
   return r == CUDA_SUCCESS ? RT3D_OK : RT3D_ERR_CUDA;
 }
 
+// Small-C_in kernel: bf16, C_in <= 8 stored at pitch 8, stride 1, M <= 256.
+bool smallc_eligible(const DeviceState* d, rt3d_packed* w, const rt3d_tensor* x, const rt3d_tensor* y,
+                     const rt3d_conv_params* p, const SmallCLayout** out) {
+  if (d->cc_major != 10 || w->dtype != RT3D_BF16) return false;
+  if (x->c > 8 || x->c_stride != 8 || y->c_stride % 8) return false;
+  if (p->st != 1 || p->sh != 1 || p->sw != 1) return false;
+  if (w->Kt > 16 || w->Kh > 32 || w->Kw > 32) return false;
+  const SmallCLayout* L = get_smallc_layout(w);
+  if (!L) return false;
+  if (smallc_smem_bytes(L->n_pairs, L->n_pad, L->halo_w * L->halo_h * L->halo_t * 16) > 227 * 1024) return false;
+  *out = L;
+  return true;
+}
+
+rt3d_status launch_smallc(rt3d_packed* w, DeviceBlob* blob, const DeviceState* d, const SmallCLayout* L,
+                          const rt3d_tensor* x, const ConvGeom& g, const float* bias, rt3d_tensor* y, cudaStream_t st) {
+  {
+    std::lock_guard<std::mutex> lock(w->mu);
+    if (!blob->smallc_wimg) {
+      void* wi = nullptr;
+      int32_t* po = nullptr;
+      if (cudaMalloc(&wi, L->wimg.size() * 2 + 16) != cudaSuccess ||
+          cudaMalloc(reinterpret_cast<void**>(&po), L->pair_off.size() * 4 + 16) != cudaSuccess)
+        return RT3D_ERR_ALLOC;
+      if ((!L->wimg.empty() && cudaMemcpy(wi, L->wimg.data(), L->wimg.size() * 2, cudaMemcpyHostToDevice) != cudaSuccess) ||
+          (!L->pair_off.empty() &&
+           cudaMemcpy(po, L->pair_off.data(), L->pair_off.size() * 4, cudaMemcpyHostToDevice) != cudaSuccess))
+        return RT3D_ERR_CUDA;
+      blob->smallc_pairs = po;
+      blob->smallc_wimg = wi;
+    }
+  }
+  SmallCArgs a;
+  a.g = g;
+  a.n_pad = L->n_pad; a.n_pairs = L->n_pairs;
+  a.halo_w = L->halo_w; a.halo_h = L->halo_h; a.halo_t = L->halo_t;
+  a.halo_bytes = L->halo_w * L->halo_h * L->halo_t * 16;
+  a.tiles_h = ceil_div(g.Ho, kSmallCTileH); a.tiles_w = ceil_div(g.Wo, kSmallCTileW);
+  a.tmem_cols = 0;
+  a.wimg = blob->smallc_wimg; a.pair_off = blob->smallc_pairs;
+  a.bias = bias; a.y = y->data; a.sched = d->sched;
+  // input as [n][t][h][w][8]: box = the halo of one 1 x 16 x 8 output tile, no swizzle
+  CUtensorMap xmap;
+  const cuuint64_t cs = 16;
+  cuuint64_t dims[5] = {cuuint64_t(x->c), cuuint64_t(x->w), cuuint64_t(x->h), cuuint64_t(x->t), cuuint64_t(x->n)};
+  cuuint64_t strides[4] = {cs, cs * x->w, cs * x->w * x->h, cs * x->w * x->h * x->t};
+  cuuint32_t bx[5] = {8, cuuint32_t(L->halo_w), cuuint32_t(L->halo_h), cuuint32_t(L->halo_t), 1};
+  cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+#if defined(RT3D_EXPERIMENT) && RT3D_EXPERIMENT == 5
+  cuuint64_t dims4[4] = {cuuint64_t(x->w) * 8, cuuint64_t(x->h), cuuint64_t(x->t), cuuint64_t(x->n)};
+  cuuint64_t strides4[3] = {cs * x->w, cs * x->w * x->h, cs * x->w * x->h * x->t};
+  cuuint32_t bx4[4] = {cuuint32_t(L->halo_w) * 8, cuuint32_t(L->halo_h), cuuint32_t(L->halo_t), 1};
+  (void)dims; (void)strides; (void)bx;
+  if (g_encode(&xmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, x->data, dims4, strides4, bx4, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+               CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+    return RT3D_ERR_CUDA;
+#else
+  if (g_encode(&xmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, x->data, dims, strides, bx, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+               CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+    return RT3D_ERR_CUDA;
+#endif
+  if (launch_conv_umma_smallc(a, &xmap, d->sm_count, st) != cudaSuccess) return RT3D_ERR_CUDA;
+  g_launches.fetch_add(1);
+  return RT3D_OK;
+}
+
 rt3d_status conv_impl(const rt3d_tensor* x, const rt3d_packed* wc, const float* bias, const rt3d_conv_params* p,
                       rt3d_tensor* y, void* stream, bool dense_entry) {
   ConvGeom g;
@@ -258,6 +324,9 @@ rt3d_status conv_impl(const rt3d_tensor* x, const rt3d_packed* wc, const float* 
     g_launches.fetch_add(1);
     return RT3D_OK;
   }
+
+  const SmallCLayout* SL = nullptr;
+  if (smallc_eligible(d, w, x, y, p, &SL)) return launch_smallc(w, blob, d, SL, x, g, bias, y, st);
 
   const UmmaLayout* L = get_umma_layout(w, 0);
   if (!L) return RT3D_ERR_UNSUPPORTED;
@@ -359,6 +428,7 @@ void rt3d_packed_free(rt3d_packed* p) {
     cudaFree(b->group_ptr); cudaFree(b->pos_idx); cudaFree(b->tiles);
     for (auto& kv : b->umma) { cudaFree(kv.second.wtiles); cudaFree(kv.second.step_ptr); cudaFree(kv.second.steps); }
     cudaFree(b->stage_x); cudaFree(b->stage_y); cudaFree(b->stage_bias);
+    cudaFree(b->smallc_wimg); cudaFree(b->smallc_pairs);
     delete b;
   }
   if (have_dev && cur >= 0) cudaSetDevice(cur);

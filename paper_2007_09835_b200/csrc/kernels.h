@@ -4,6 +4,8 @@
 #include <cstdint>
 #include <cuda_runtime.h>
 
+#include "tile_consts.h"
+
 namespace rt3d {
 
 // Geometry of one convolution call (all extents already validated on the host).
@@ -50,7 +52,23 @@ struct UmmaArgs {
 cudaError_t launch_conv_umma(const UmmaArgs& a, const void* xmap, const void* wmap, int sm_count,
                              cudaStream_t stream);
 
+// Arguments of the small-C_in tensor-core kernel (C_in <= 8 at channel pitch 8, stride 1).
+struct SmallCArgs {
+  ConvGeom g;
+  int n_pad, n_pairs;                 // padded output channels; pairs of kept kernel locations
+  int halo_w, halo_h, halo_t, halo_bytes;
+  int tiles_h, tiles_w;               // 16 x 8 output tiles per frame
+  int tmem_cols;                      // filled in by the launcher
+  const void* wimg;                   // device: [n_pairs][2][n_pad/8][8][8] bf16
+  const int32_t* pair_off;            // device: [n_pairs][2] byte offsets inside the staged halo
+  const float* bias;
+  void* y;
+  int32_t* sched;
+};
+cudaError_t launch_conv_umma_smallc(const SmallCArgs& a, const void* xmap, int sm_count, cudaStream_t stream);
+size_t smallc_smem_bytes(int n_pairs, int n_pad, int halo_bytes);
+
 // Shared memory the tcgen05 kernel needs for a bundle width (for the host-side eligibility check).
-size_t umma_smem_bytes(int n_tile);
+size_t umma_smem_bytes(int n_tile, int n_bundles);
 
 }  // namespace rt3d

@@ -101,6 +101,50 @@ const UmmaLayout* get_umma_layout(rt3d_packed* p, int n_tile) {
   return &res.first->second;
 }
 
+// Small-C_in layout: kernel locations kept by at least one group are listed in ascending order and
+// paired; each pair is one K=16 MMA whose two K halves are the 8 (padded) channels at the two
+// locations.  Operands use the no-swizzle core-matrix layout (8 rows x 16 bytes).
+const SmallCLayout* get_smallc_layout(rt3d_packed* p) {
+  if (p->dtype != RT3D_BF16 || p->N > 8 || p->M > 256) return nullptr;
+  std::lock_guard<std::mutex> lock(p->mu);
+  if (p->smallc_built) return &p->smallc;
+  SmallCLayout& L = p->smallc;
+  L.n_pad = round_up(p->M, 16);
+  L.halo_w = kSmallCTileW + p->Kw - 1;
+  L.halo_h = kSmallCTileH + p->Kh - 1;
+  L.halo_t = p->Kt;
+  std::vector<uint8_t> used(size_t(p->Ks), 0);
+  for (int64_t e = 0; e < p->nnz; ++e) used[p->pos_idx[size_t(e)]] = 1;
+  std::vector<int> pos;
+  for (int k = 0; k < p->Ks; ++k)
+    if (used[size_t(k)]) pos.push_back(k);
+  L.n_pairs = ceil_div(int(pos.size()), 2);
+  L.pair_off.assign(size_t(L.n_pairs) * 2, 0);
+  L.wimg.assign(size_t(L.n_pairs) * 2 * L.n_pad * 8, 0);
+  std::vector<int> slot(size_t(p->Ks), -1);       // location -> pair*2 + half
+  for (size_t i = 0; i < pos.size(); ++i) {
+    const int k = pos[i];
+    const int kw = k % p->Kw, kh = (k / p->Kw) % p->Kh, kt = k / (p->Kw * p->Kh);
+    L.pair_off[i] = ((kt * L.halo_h + kh) * L.halo_w + kw) * 16;
+    slot[size_t(k)] = int(i);
+  }
+  if (pos.size() % 2) L.pair_off[pos.size()] = L.pair_off[pos.size() - 1] + 16;   // unused half: zero weights
+  const uint16_t* tiles = reinterpret_cast<const uint16_t*>(p->tiles.data());
+  for (int pr = 0; pr < p->P; ++pr)
+    for (int q = 0; q < p->Q; ++q)
+      for (int32_t e = p->group_ptr[size_t(pr) * p->Q + q]; e < p->group_ptr[size_t(pr) * p->Q + q + 1]; ++e) {
+        const int s = slot[p->pos_idx[size_t(e)]];
+        for (int i = 0; i < p->g_m && pr * p->g_m + i < p->M; ++i)
+          for (int j = 0; j < p->g_n && q * p->g_n + j < p->N; ++j) {
+            const int m = pr * p->g_m + i, c = q * p->g_n + j;
+            L.wimg[((size_t(s) * (L.n_pad / 8) + m / 8) * 8 + m % 8) * 8 + c] =
+                tiles[(size_t(e) * p->g_m + i) * p->g_n + j];
+          }
+      }
+  p->smallc_built = true;
+  return &L;
+}
+
 static rt3d_status pack_impl(const float* w, const uint8_t* mask, int M, int N, int Kt, int Kh, int Kw,
                              int g_m, int g_n, int dtype, int is_dense, rt3d_packed** out) {
   if (!w || !out) return RT3D_ERR_INVALID_ARG;

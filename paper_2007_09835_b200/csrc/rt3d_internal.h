@@ -8,6 +8,7 @@
 #include <vector>
 
 #include "rt3d.h"
+#include "tile_consts.h"
 
 namespace rt3d {
 
@@ -43,6 +44,16 @@ struct UmmaLayout {
   int max_steps = 0;                 // longest bundle list
 };
 
+// Layout for the small-C_in tensor-core kernel (C_in <= 8, channel pitch 8): the K dimension is
+// walked in pairs of kernel locations (8 padded channels each), one K=16 MMA per pair.
+struct SmallCLayout {
+  int n_pad = 0;                     // output channels rounded up to 16 (<= 256)
+  int n_pairs = 0;
+  int halo_w = 0, halo_h = 0, halo_t = 0;   // input voxels staged per 1x16x8 output tile
+  std::vector<int32_t> pair_off;     // [n_pairs][2] byte offset of each location inside the staged halo
+  std::vector<uint16_t> wimg;        // [n_pairs][2][n_pad/8][8][8] bf16 bits, zero where pruned / absent
+};
+
 // Per-device copies of a handle's arrays.
 struct DeviceBlob {
   int device = -1;
@@ -57,6 +68,8 @@ struct DeviceBlob {
     bool ready = false;
   };
   std::map<int, Umma> umma;          // keyed by n_tile
+  void* smallc_wimg = nullptr;       // small-C_in kernel: weight image and location-pair offsets
+  int32_t* smallc_pairs = nullptr;
   int32_t* sched = nullptr;          // [8] tile counter, finished-CTA counter (zero between launches)
   void* stage_x = nullptr; size_t stage_x_bytes = 0;   // staging for rt3d_conv3d_host
   void* stage_y = nullptr; size_t stage_y_bytes = 0;
@@ -74,6 +87,8 @@ struct rt3d_packed {
   std::vector<unsigned char> tiles;  // nnz * g_m * g_n elements of float or bf16 bits
   std::mutex mu;                     // guards the lazily built members below
   std::map<int, rt3d::UmmaLayout> umma_layouts;   // keyed by n_tile
+  rt3d::SmallCLayout smallc;         // built on first use
+  bool smallc_built = false;
   std::vector<rt3d::DeviceBlob*> blobs;
 };
 
@@ -84,5 +99,7 @@ int default_n_tile(int M);
 // Builds (or returns the cached) tensor-core layout; nullptr if the handle cannot use it.
 const UmmaLayout* get_umma_layout(rt3d_packed* p, int n_tile);
 bool umma_layout_possible(const rt3d_packed* p);
+// Small-C_in layout (nullptr if the handle does not qualify: needs bf16, N <= 8, M <= 256).
+const SmallCLayout* get_smallc_layout(rt3d_packed* p);
 
 }  // namespace rt3d

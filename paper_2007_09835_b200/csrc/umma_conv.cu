@@ -15,125 +15,11 @@
 // accumulator buffers in TMEM let the epilogue of one tile overlap the MMAs of the next.
 // Every wait on an mbarrier is bounded: on expiry the CTA records an error word in global
 // memory, all roles fall through, TMEM is released and the kernel returns.
-#include <cuda.h>
-#include <cuda_bf16.h>
-
 #include "kernels.h"
+#include "umma_common.cuh"
 
 namespace rt3d {
 namespace {
-
-constexpr int kThreadsUmma = 192;
-constexpr int kMaxStages = 8;
-constexpr int kABytes = 128 * 128;                  // 128 voxel rows x 64 bf16
-constexpr long long kWaitCycles = 1ll << 31;        // about one second of SM clocks
-constexpr size_t kSmemBudget = 200 * 1024;
-
-struct __align__(8) Barriers {
-  unsigned long long full[kMaxStages];
-  unsigned long long empty[kMaxStages];
-  unsigned long long tmem_full[2];
-  unsigned long long tmem_empty[2];
-  unsigned int tmem_base;
-  volatile int abort_flag;
-};
-
-__device__ __forceinline__ uint32_t smem_u32(const void* p) {
-  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
-}
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n"
-      ".reg .pred p;\n"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
-      "selp.u32 %0, 1, 0, p;\n"
-      "}\n"
-      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-  return ok != 0;
-}
-
-// Bounded wait.  Returns false (and raises the CTA's abort flag + the global error word) when the
-// phase did not complete within kWaitCycles, or when another role already aborted.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, Barriers* bars, int32_t* err, int code) {
-  if (mbar_try_wait(bar, parity)) return true;
-  const long long start = clock64();
-  for (;;) {
-#pragma unroll 1
-    for (int i = 0; i < 128; ++i)
-      if (mbar_try_wait(bar, parity)) return true;
-    if (bars->abort_flag) return false;
-    if (clock64() - start > kWaitCycles) {
-      bars->abort_flag = 1;
-      atomicCAS(err, 0, code);
-      return false;
-    }
-  }
-}
-
-__device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2,
-                                            int c3, int c4) {
-  asm volatile(
-      "cp.async.bulk.tensor.5d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
-      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4)
-      : "memory");
-}
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1)
-      : "memory");
-}
-
-// Shared-memory matrix descriptor: K-major tile of 128-byte rows, 128-byte swizzle, 8-row groups
-// 1024 bytes apart; descriptor version 1 (sm_100).
-__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
-  uint64_t d = 0;
-  d |= uint64_t((addr & 0x3FFFFu) >> 4);
-  d |= uint64_t(1) << 16;                 // leading byte offset (unused for swizzled K-major)
-  d |= uint64_t(1024 >> 4) << 32;         // stride byte offset between 8-row groups
-  d |= uint64_t(1) << 46;                 // version
-  d |= uint64_t(2) << 61;                 // SWIZZLE_128B
-  return d;
-}
-
-// Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128, N = n.
-__device__ __forceinline__ uint32_t instr_desc_bf16(int n) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | (uint32_t(n >> 3) << 17) | (uint32_t(128 >> 4) << 24);
-}
-
-__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
-  asm volatile(
-      "{\n"
-      ".reg .pred p;\n"
-      "setp.ne.b32 p, %4, 0;\n"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n"
-      "}\n"
-      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc)
-      : "memory");
-}
-__device__ __forceinline__ void umma_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
-      : "r"(taddr));
-  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
 struct ItemCoord {
   int bundle, n0, t0, h0, w0;     // bundle index and first output voxel of the box
@@ -160,7 +46,10 @@ conv3d_umma_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_consta
   const uint32_t b_bytes = uint32_t(a.n_tile) * 128u;
   const uint32_t stage_bytes = kABytes + b_bytes;
   Barriers* bars = reinterpret_cast<Barriers*>(smem_raw + (tiles_base - raw) + size_t(stages) * stage_bytes);
+  float* bias_s = reinterpret_cast<float*>(bars + 1);              // bias of all bundles (zeros if none), padded
   int32_t* err = a.sched + 2;
+  for (int i = threadIdx.x; i < a.n_bundles * a.n_tile; i += blockDim.x)
+    bias_s[i] = (a.bias != nullptr && i < a.g.M) ? __ldg(a.bias + i) : 0.f;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n_mtiles = a.tiles_n * a.tiles_t * a.tiles_h * a.tiles_w;
@@ -296,35 +185,8 @@ conv3d_umma_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_consta
       const long long vox = (((long long)nn * a.g.To + to) * a.g.Ho + ho) * a.g.Wo + wo;
       const int m_base = c.bundle * a.n_tile;
       const uint32_t taddr = tmem_base + (uint32_t(quad * 32) << 16) + buf * uint32_t(a.n_tile);
-      for (int col = 0; col < a.n_tile; col += 16) {
-        const int m0 = m_base + col;
-        if (m0 >= a.g.M) break;                      // warp-uniform
-        uint32_t v[16];
-        if (nsteps > 0) tmem_ld16(taddr + col, v);   // warp-uniform: .sync.aligned
-        else {
-#pragma unroll
-          for (int q = 0; q < 16; ++q) v[q] = 0u;
-        }
-        if (!in_range) continue;
-        float f[16];
-#pragma unroll
-        for (int q = 0; q < 16; ++q) {
-          f[q] = __uint_as_float(v[q]);
-          if (a.bias != nullptr && m0 + q < a.g.M) f[q] += __ldg(a.bias + m0 + q);
-          if (a.g.relu) f[q] = fmaxf(f[q], 0.f);
-        }
-        __nv_bfloat16* dst = yb + vox * a.g.ycs + m0;
-        if (m0 + 16 <= a.g.M) {
-          uint4 o[2];
-          __nv_bfloat162* po = reinterpret_cast<__nv_bfloat162*>(o);
-#pragma unroll
-          for (int q = 0; q < 8; ++q) po[q] = __floats2bfloat162_rn(f[2 * q], f[2 * q + 1]);
-          reinterpret_cast<uint4*>(dst)[0] = o[0];
-          reinterpret_cast<uint4*>(dst)[1] = o[1];
-        } else {
-          for (int q = 0; q < 16 && m0 + q < a.g.M; ++q) dst[q] = __float2bfloat16_rn(f[q]);
-        }
-      }
+      epilogue_row(taddr, a.n_tile, nsteps > 0, in_range, bias_s, a.g.relu,
+                   yb + vox * a.g.ycs + m_base, m_base, a.g.M);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&bars->tmem_empty[buf]));
@@ -353,15 +215,17 @@ int pick_stages(int n_tile) {
 
 }  // namespace
 
-size_t umma_smem_bytes(int n_tile) {
-  return size_t(pick_stages(n_tile)) * (kABytes + size_t(n_tile) * 128) + 1024 + sizeof(Barriers);
+size_t umma_smem_bytes(int n_tile, int n_bundles) {
+  return size_t(pick_stages(n_tile)) * (kABytes + size_t(n_tile) * 128) + 1024 + sizeof(Barriers) +
+         size_t(n_tile) * n_bundles * 4;
 }
 
 cudaError_t launch_conv_umma(const UmmaArgs& a, const void* xmap, const void* wmap, int sm_count,
                              cudaStream_t stream) {
   const int stages = pick_stages(a.n_tile);
   if (stages < 2) return cudaErrorInvalidValue;
-  const size_t smem = umma_smem_bytes(a.n_tile);
+  const size_t smem = umma_smem_bytes(a.n_tile, a.n_bundles);
+  if (smem > 227 * 1024) return cudaErrorInvalidValue;
   int cols = 32;
   while (cols < 2 * a.n_tile) cols *= 2;
   if (cols > 512) return cudaErrorInvalidValue;

@@ -1,0 +1,202 @@
+// Tensor-core convolution for layers with very few input channels (C_in <= 8 stored at a channel
+// pitch of 8, e.g. the RGB first layer of the C3D-shaped network), stride 1.
+//
+// With 16 bytes per voxel the input halo of an output tile of 1 x 16 x 8 voxels can be staged in
+// shared memory exactly as it lies in global memory, [t][h][w][8 channels], by one TMA box whose
+// out-of-range part is zero-filled (= the zero padding; channels >= C_in are zero-filled too).
+// In the no-swizzle operand layout a core matrix is 8 rows of 16 bytes, i.e. 8 consecutive voxels
+// along w with their 8 channels: every shifted window of the halo is a valid A operand whose
+// 8-row groups are one halo row apart, and the two K halves of a K=16 MMA can be two different
+// kernel locations (leading byte offset = distance between the two shifted windows).  So each pair
+// of kept kernel locations is one MMA, the input is read from L2 once per tile, and the layer is
+// bound by writing its output.  Kernel locations that no group keeps are not in the pair list.
+//
+// Roles as in the main kernel: warp 0 TMA producer, warp 1 MMA issuer / TMEM owner, warps 2..5
+// epilogue; bounded mbarrier waits.
+#include "kernels.h"
+#include "umma_common.cuh"
+
+namespace rt3d {
+namespace {
+
+constexpr int kSmallCStages = 3;
+
+template <int kDummy>
+__global__ void __launch_bounds__(kThreadsUmma, 1)
+conv3d_umma_smallc_kernel(const __grid_constant__ CUtensorMap xmap, const SmallCArgs a) {
+  extern __shared__ unsigned char smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 127u) & ~127u;
+  const uint32_t w_bytes = uint32_t(a.n_pairs) * 2u * uint32_t(a.n_pad) * 16u;
+  const uint32_t w_smem = base;                                         // weight image, whole layer
+  const uint32_t halo_smem = base + ((w_bytes + 127u) & ~127u);         // ring of staged halos
+  const uint32_t halo_stride = (uint32_t(a.halo_bytes) + 127u) & ~127u;
+  unsigned char* gen = smem_raw + (base - raw);
+  int32_t* pair_smem = reinterpret_cast<int32_t*>(gen + (halo_smem - base) + kSmallCStages * halo_stride);
+  Barriers* bars = reinterpret_cast<Barriers*>(reinterpret_cast<unsigned char*>(pair_smem) +
+                                               ((size_t(a.n_pairs) * 8 + 15) & ~size_t(15)));
+  float* bias_s = reinterpret_cast<float*>(bars + 1);
+  int32_t* err = a.sched + 2;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  for (int i = threadIdx.x; i < a.n_pad; i += blockDim.x)
+    bias_s[i] = (a.bias != nullptr && i < a.g.M) ? __ldg(a.bias + i) : 0.f;
+  const int tiles_per_frame = a.tiles_h * a.tiles_w;
+  const int n_items = a.g.n * a.g.To * tiles_per_frame;
+
+  // weight image and pair offsets: plain cooperative copy, once per CTA
+  {
+    const uint4* src = reinterpret_cast<const uint4*>(a.wimg);
+    uint4* dst = reinterpret_cast<uint4*>(gen);
+    for (uint32_t i = threadIdx.x; i < w_bytes / 16; i += blockDim.x) dst[i] = __ldg(src + i);
+    for (int i = threadIdx.x; i < a.n_pairs * 2; i += blockDim.x) pair_smem[i] = __ldg(a.pair_off + i);
+  }
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kSmallCStages; ++s) {
+      mbar_init(smem_u32(&bars->full[s]), 1);
+      mbar_init(smem_u32(&bars->empty[s]), 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(smem_u32(&bars->tmem_full[b]), 1);
+      mbar_init(smem_u32(&bars->tmem_empty[b]), 4);
+    }
+    bars->abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  // generic-proxy writes of the weight image must be visible to the tensor core (async proxy)
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                 ::"r"(smem_u32(&bars->tmem_base)), "r"(uint32_t(a.tmem_cols)) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = bars->tmem_base;
+
+  if (warp == 0) {
+    if (lane == 0 && a.n_pairs > 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
+        int r = item;
+        const int iw = r % a.tiles_w; r /= a.tiles_w;
+        const int ih = r % a.tiles_h; r /= a.tiles_h;
+        const int to = r % a.g.To;
+        const int nn = r / a.g.To;
+        if (!mbar_wait(smem_u32(&bars->empty[stage]), phase ^ 1u, bars, err, 11)) break;
+        const uint32_t full = smem_u32(&bars->full[stage]);
+        mbar_expect_tx(full, uint32_t(a.halo_bytes));
+#if defined(RT3D_EXPERIMENT) && RT3D_EXPERIMENT == 5
+        tma_load_4d(halo_smem + stage * halo_stride, &xmap, full, (iw * kSmallCTileW - a.g.pw) * 8,
+                    ih * kSmallCTileH - a.g.ph, to - a.g.pt, nn);
+#else
+        tma_load_5d(halo_smem + stage * halo_stride, &xmap, full, 0, iw * kSmallCTileW - a.g.pw,
+                    ih * kSmallCTileH - a.g.ph, to - a.g.pt, nn);
+#endif
+        if (++stage == kSmallCStages) { stage = 0; phase ^= 1u; }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      const uint32_t idesc = instr_desc_bf16(a.n_pad);
+      const uint32_t sbo_a = uint32_t(a.halo_w) * 16u;            // next 8-voxel group = next halo row
+      const uint32_t lbo_b = uint32_t(a.n_pad) * 16u;             // second K half of the weight image
+      int stage = 0;
+      uint32_t phase = 0, j = 0;
+      for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++j) {
+        const uint32_t buf = j & 1u;
+        if (!mbar_wait(smem_u32(&bars->tmem_empty[buf]), ((j >> 1) & 1u) ^ 1u, bars, err, 12)) break;
+        if (a.n_pairs == 0) { mbar_arrive(smem_u32(&bars->tmem_full[buf])); continue; }
+        if (!mbar_wait(smem_u32(&bars->full[stage]), phase, bars, err, 13)) break;
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + buf * uint32_t(a.n_pad);
+        const uint32_t halo = halo_smem + stage * halo_stride;
+        for (int p = 0; p < a.n_pairs; ++p) {
+          const uint32_t o0 = uint32_t(pair_smem[2 * p]), o1 = uint32_t(pair_smem[2 * p + 1]);
+          const uint64_t adesc = smem_desc_noswizzle(halo + o0, o1 - o0, sbo_a);
+          const uint64_t bdesc = smem_desc_noswizzle(w_smem + uint32_t(p) * 2u * lbo_b, lbo_b, 128u);
+          umma_bf16(d_tmem, adesc, bdesc, idesc, p ? 1u : 0u);
+        }
+        umma_commit(smem_u32(&bars->empty[stage]));
+        umma_commit(smem_u32(&bars->tmem_full[buf]));
+        if (++stage == kSmallCStages) { stage = 0; phase ^= 1u; }
+      }
+    }
+  } else {
+    const int quad = warp & 3;
+    const int row = quad * 32 + lane;
+    const int bh_i = row / kSmallCTileW, bw_i = row % kSmallCTileW;
+    __nv_bfloat16* yb = static_cast<__nv_bfloat16*>(a.y);
+    uint32_t j = 0;
+    for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++j) {
+      int r = item;
+      const int iw = r % a.tiles_w; r /= a.tiles_w;
+      const int ih = r % a.tiles_h; r /= a.tiles_h;
+      const int to = r % a.g.To;
+      const int nn = r / a.g.To;
+      const uint32_t buf = j & 1u;
+      if (!mbar_wait(smem_u32(&bars->tmem_full[buf]), (j >> 1) & 1u, bars, err, 14)) break;
+      tc_fence_after();
+      const int ho = ih * kSmallCTileH + bh_i, wo = iw * kSmallCTileW + bw_i;
+      const bool in_range = ho < a.g.Ho && wo < a.g.Wo;
+      const long long vox = (((long long)nn * a.g.To + to) * a.g.Ho + ho) * a.g.Wo + wo;
+      const uint32_t taddr = tmem_base + (uint32_t(quad * 32) << 16) + buf * uint32_t(a.n_pad);
+      epilogue_row(taddr, a.n_pad, a.n_pairs > 0, in_range, bias_s, a.g.relu, yb + vox * a.g.ycs, 0, a.g.M);
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&bars->tmem_empty[buf]));
+    }
+  }
+
+  if (bars->abort_flag) {
+    const long long t0 = clock64();
+    while (clock64() - t0 < 2000000ll) { }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(uint32_t(a.tmem_cols)) : "memory");
+  }
+}
+
+}  // namespace
+
+size_t smallc_smem_bytes(int n_pairs, int n_pad, int halo_bytes) {
+  const size_t w = (size_t(n_pairs) * 2 * n_pad * 16 + 127) & ~size_t(127);
+  const size_t halo = (size_t(halo_bytes) + 127) & ~size_t(127);
+  return 128 + w + kSmallCStages * halo + ((size_t(n_pairs) * 8 + 15) & ~size_t(15)) + sizeof(Barriers) + size_t(n_pad) * 4;
+}
+
+cudaError_t launch_conv_umma_smallc(const SmallCArgs& a_in, const void* xmap, int sm_count, cudaStream_t stream) {
+  SmallCArgs a = a_in;
+  int cols = 32;
+  while (cols < 2 * a.n_pad) cols *= 2;
+  if (cols > 512) return cudaErrorInvalidValue;
+  a.tmem_cols = cols;
+  const size_t smem = smallc_smem_bytes(a.n_pairs, a.n_pad, a.halo_bytes);
+  if (smem > 227 * 1024) return cudaErrorInvalidValue;
+  const long long n_items = (long long)a.g.n * a.g.To * a.tiles_h * a.tiles_w;
+  if (n_items <= 0) return cudaSuccess;
+  // several CTAs per SM (the layer is bound by its epilogue / output stores): limited by shared
+  // memory, by the 512 TMEM columns of an SM, and kept at four.
+  int per_sm = int((220 * 1024) / (smem + 1024));
+  if (per_sm > 512 / cols) per_sm = 512 / cols;
+  if (per_sm > 4) per_sm = 4;
+  if (per_sm < 1) per_sm = 1;
+  const long long want = (long long)sm_count * per_sm;
+  const int grid = int(n_items < want ? n_items : want);
+  CUtensorMap xm;
+  memcpy(&xm, xmap, sizeof(CUtensorMap));
+  static bool attr_done = false;
+  if (!attr_done) {
+    cudaError_t e = cudaFuncSetAttribute(conv3d_umma_smallc_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    if (e != cudaSuccess) return e;
+    attr_done = true;
+  }
+  conv3d_umma_smallc_kernel<0><<<grid, kThreadsUmma, smem, stream>>>(xm, a);
+  return cudaGetLastError();
+}
+
+}  // namespace rt3d

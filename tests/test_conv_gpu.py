@@ -100,6 +100,37 @@ def test_umma_kernel_against_oracle(case):
     check(y, ref, torch.bfloat16, f"umma {case}")
 
 
+SMALLC_CASES = [
+    # C_in <= 8 at pitch 8, stride 1: the staged-halo kernel with location-pair MMAs
+    (3, 64, (3, 3, 3), (1, 1, 1), (1, 1, 1), (2, 5, 33, 19), 4, 4, 0.3),     # ragged 16x8 tiles, several frames
+    (3, 64, (3, 3, 3), (1, 1, 1), (1, 1, 1), (1, 3, 32, 16), 4, 4, 1.0),     # all 27 locations (odd count)
+    (8, 45, (1, 7, 7), (1, 1, 1), (0, 3, 3), (1, 2, 20, 20), 4, 4, 0.5),     # 49 locations, ragged C_out
+    (1, 16, (3, 1, 1), (1, 1, 1), (1, 0, 0), (1, 6, 9, 9), 4, 4, 0.7),
+    (5, 256, (2, 2, 2), (1, 1, 1), (0, 0, 0), (1, 4, 18, 10), 8, 4, 0.5),    # no padding, even kernel
+    (3, 32, (3, 3, 3), (1, 1, 1), (0, 1, 2), (1, 5, 17, 9), 4, 4, 0.05),     # very sparse: few pairs
+]
+
+
+@pytest.mark.parametrize("case", SMALLC_CASES)
+def test_small_cin_kernel_against_oracle(case):
+    cin, cout, k, stride, pad, (n, t, h, w), g_m, g_n, d = case
+    spec = synth.ConvSpec("c", cin, cout, k, stride, pad, True)
+    y, ref, lay, xd, yt = run_case(spec, n, t, h, w, g_m, g_n, "bernoulli", d, torch.bfloat16, rt3d.ALGO_UMMA)
+    check(y, ref, torch.bfloat16, f"small-cin {case}")
+    ys = nets.to_numpy(lay(xd, algo=rt3d.ALGO_SIMT), cout)
+    check(ys, ref, torch.bfloat16, f"small-cin simt {case}")
+
+
+def test_small_cin_all_pruned_outputs_bias():
+    spec = synth.ConvSpec("c", 3, 32, (3, 3, 3), (1, 1, 1), (1, 1, 1), False)
+    L = synth.make_layer(spec, 7, 4, 4, 4, "bernoulli", 0.5)
+    L["mask"][:] = 0
+    lay = nets.ConvLayer(spec, L["w"], L["bias"], L["mask"], 4, 4, torch.bfloat16)
+    y = nets.to_numpy(lay(nets.to_device(synth.make_input(704, (1, 2, 16, 8, 3))), algo=rt3d.ALGO_UMMA), 32)
+    assert rt3d.rt3d_last_device_status() == rt3d.OK
+    np.testing.assert_array_equal(y, np.broadcast_to(oracle.bf16_round(L["bias"]), y.shape))
+
+
 UMMA_STRIDED = [
     (64, 64, (3, 3, 3), (2, 2, 2), (1, 1, 1), (1, 6, 11, 12), 4, 4, 0.4),
     (64, 230, (1, 3, 3), (1, 2, 2), (0, 1, 1), (1, 4, 14, 14), 4, 4, 0.4),
