@@ -208,6 +208,37 @@ TileBox choose_box(const ConvGeom& g) {
   return best;
 }
 
+// Bundle width and number of K splits for a call.  Model (fitted to timings on B200): a K step costs
+// the issuing thread about 175 ns of barrier hand-shake plus 4 MMA issues, or the tensor time of the
+// step if that is longer; a layer with few output tiles runs as many serial steps per CTA as its
+// step list is long, so it is split along K (at the price of writing and re-reading fp32 partial
+// tiles) until the SMs are occupied; narrower bundles are the fallback when K is short.
+struct UmmaPlan { int n_tile, n_splits; };
+
+UmmaPlan pick_plan(int M, long long m_tiles, int steps, int sm_count) {
+  const int widest = default_n_tile(M);
+  UmmaPlan best{widest, 1};
+  double best_ns = -1.0;
+  static const int kSplits[] = {1, 2, 3, 4, 6, 8};
+  for (int n = widest; n >= 32; n = (n > 128 ? 128 : n / 2)) {
+    if (n % 16) break;
+    const long long items = m_tiles * ceil_div(M, n);
+    const double issue = 175.0 + 4.0 * (25.0 + 0.06 * n), tensor = 1.02 * n;
+    const double step_ns = issue > tensor ? issue : tensor;
+    for (int S : kSplits) {
+      if (S > 1 && (steps / S < 8 || items >= 2LL * sm_count)) continue;
+      const double waves = double(ceil_div64(items * S, sm_count));
+      double ns = waves * ceil_div(steps, S) * step_ns;
+      // partial tile out (every split) and S partial tiles back in (the CTA that arrives last), plus the
+      // traffic of all partials (written once, read once) at about 2.5 TB/s
+      if (S > 1) ns += 3000.0 + (1.0 + S) * n * 4.0 + double(items) * S * (kTileM * n * 4.0 * 2.0) / 2500.0;
+      if (best_ns < 0 || ns < best_ns * 0.97) { best = UmmaPlan{n, S}; best_ns = ns; }
+    }
+    if (n == 32) break;
+  }
+  return best;
+}
+
 bool umma_eligible(const DeviceState* d, const rt3d_packed* w, const rt3d_tensor* x, const rt3d_tensor* y,
                    const rt3d_conv_params* p) {
   if (d->cc_major != 10) return false;
@@ -328,20 +359,44 @@ rt3d_status conv_impl(const rt3d_tensor* x, const rt3d_packed* wc, const float* 
   const SmallCLayout* SL = nullptr;
   if (smallc_eligible(d, w, x, y, p, &SL)) return launch_smallc(w, blob, d, SL, x, g, bias, y, st);
 
-  const UmmaLayout* L = get_umma_layout(w, 0);
-  if (!L) return RT3D_ERR_UNSUPPORTED;
-  DeviceBlob::Umma* u = nullptr;
-  if ((s = get_umma_blob(w, blob, L, &u)) != RT3D_OK) return s;
   UmmaArgs a;
   a.g = g;
   a.box = choose_box(g);
-  a.n_tile = L->n_tile; a.n_bundles = L->n_bundles; a.n_chunks = L->n_chunks;
   a.tiles_n = ceil_div(g.n, a.box.bn); a.tiles_t = ceil_div(g.To, a.box.bt);
   a.tiles_h = ceil_div(g.Ho, a.box.bh); a.tiles_w = ceil_div(g.Wo, a.box.bw);
+  const long long m_tiles = (long long)a.tiles_n * a.tiles_t * a.tiles_h * a.tiles_w;
+  const UmmaPlan plan = pick_plan(w->M, m_tiles, w->Ks * ceil_div(w->N, kChunk), d->sm_count);
+  const UmmaLayout* L = get_umma_layout(w, plan.n_tile);
+  if (!L) return RT3D_ERR_UNSUPPORTED;
+  DeviceBlob::Umma* u = nullptr;
+  if ((s = get_umma_blob(w, blob, L, &u)) != RT3D_OK) return s;
+  a.n_tile = L->n_tile; a.n_bundles = L->n_bundles; a.n_chunks = L->n_chunks;
   a.dense = dense_entry ? 1 : 0;
   a.steps_dense = w->Ks * L->n_chunks;
   a.step_ptr = u->step_ptr; a.steps = u->steps;
   a.bias = bias; a.y = y->data; a.sched = d->sched;
+  a.n_splits = plan.n_splits; a.scratch = nullptr; a.counters = nullptr;
+  if (a.n_splits > 1) {
+    // split-K workspace of this handle on this device: partial tiles + per-warp arrival counters
+    const long long tiles = m_tiles * L->n_bundles;
+    const size_t need = size_t(tiles) * a.n_splits * kTileM * L->n_tile * sizeof(float);
+    const size_t need_cnt = size_t(tiles) * 4 * sizeof(int32_t);
+    std::lock_guard<std::mutex> lock(w->mu);
+    if (blob->splitk_bytes < need) {
+      cudaFree(blob->splitk);
+      blob->splitk = nullptr; blob->splitk_bytes = 0;
+      if (cudaMalloc(reinterpret_cast<void**>(&blob->splitk), need) != cudaSuccess) return RT3D_ERR_ALLOC;
+      blob->splitk_bytes = need;
+    }
+    if (blob->splitk_cnt_bytes < need_cnt) {
+      cudaFree(blob->splitk_cnt);
+      blob->splitk_cnt = nullptr; blob->splitk_cnt_bytes = 0;
+      if (cudaMalloc(reinterpret_cast<void**>(&blob->splitk_cnt), need_cnt) != cudaSuccess) return RT3D_ERR_ALLOC;
+      if (cudaMemset(blob->splitk_cnt, 0, need_cnt) != cudaSuccess) return RT3D_ERR_CUDA;
+      blob->splitk_cnt_bytes = need_cnt;
+    }
+    a.scratch = blob->splitk; a.counters = blob->splitk_cnt;
+  }
   CUtensorMap xmap;
   if ((s = encode_xmap(x, g, a.box, &xmap)) != RT3D_OK) return s;
   cudaError_t e = launch_conv_umma(a, &xmap, u->wmap, d->sm_count, st);
@@ -429,6 +484,7 @@ void rt3d_packed_free(rt3d_packed* p) {
     for (auto& kv : b->umma) { cudaFree(kv.second.wtiles); cudaFree(kv.second.step_ptr); cudaFree(kv.second.steps); }
     cudaFree(b->stage_x); cudaFree(b->stage_y); cudaFree(b->stage_bias);
     cudaFree(b->smallc_wimg); cudaFree(b->smallc_pairs);
+    cudaFree(b->splitk); cudaFree(b->splitk_cnt);
     delete b;
   }
   if (have_dev && cur >= 0) cudaSetDevice(cur);

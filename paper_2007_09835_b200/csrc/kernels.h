@@ -45,7 +45,10 @@ struct UmmaArgs {
   const int32_t* steps;                     // device                     (sparse)
   const float* bias;                        // device or nullptr
   void* y;
-  int32_t* sched;                           // device [8]: [0] tile counter, [1] finished CTAs, [2] error word
+  int32_t* sched;                           // device [8]: [2] = error word set by a bounded wait that gave up
+  int n_splits;                             // K splits per output tile (1 = none)
+  float* scratch;                           // device, split-K partial tiles [tile][split][128][n_tile] (n_splits > 1)
+  int32_t* counters;                        // device, [tiles * 4] arrival counters, zero between launches
 };
 
 // xmap / wmap point to 128-byte CUtensorMap objects in host memory.

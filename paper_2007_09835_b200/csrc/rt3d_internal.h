@@ -70,7 +70,8 @@ struct DeviceBlob {
   std::map<int, Umma> umma;          // keyed by n_tile
   void* smallc_wimg = nullptr;       // small-C_in kernel: weight image and location-pair offsets
   int32_t* smallc_pairs = nullptr;
-  int32_t* sched = nullptr;          // [8] tile counter, finished-CTA counter (zero between launches)
+  float* splitk = nullptr; size_t splitk_bytes = 0;            // split-K partial tiles (grown on demand)
+  int32_t* splitk_cnt = nullptr; size_t splitk_cnt_bytes = 0;  // split-K arrival counters, zero between launches
   void* stage_x = nullptr; size_t stage_x_bytes = 0;   // staging for rt3d_conv3d_host
   void* stage_y = nullptr; size_t stage_y_bytes = 0;
   float* stage_bias = nullptr;

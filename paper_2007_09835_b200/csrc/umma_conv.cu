@@ -13,6 +13,12 @@
 // One persistent CTA per SM, 6 warps: warp 0 = TMA producer, warp 1 = MMA issuer (and TMEM
 // owner), warps 2..5 = epilogue (TMEM -> registers -> +bias, ReLU, bf16 -> NDHWC stores).  Two
 // accumulator buffers in TMEM let the epilogue of one tile overlap the MMAs of the next.
+//
+// Layers with few output tiles are split along K: each of `n_splits` CTAs accumulates a slice of
+// the step list and writes its fp32 partial tile to a scratch buffer; the CTA that arrives last
+// (a counter per output tile and warp) adds the partials in split order, so the result does not depend
+// on which CTA that is, applies the epilogue and resets the counter for the next launch.
+//
 // Every wait on an mbarrier is bounded: on expiry the CTA records an error word in global
 // memory, all roles fall through, TMEM is released and the kernel returns.
 #include "kernels.h"
@@ -22,18 +28,95 @@ namespace rt3d {
 namespace {
 
 struct ItemCoord {
-  int bundle, n0, t0, h0, w0;     // bundle index and first output voxel of the box
+  int bundle, split, tile_id;     // tile_id = bundle * n_mtiles + m-tile
+  int n0, t0, h0, w0;             // first output voxel of the box
 };
 
 __device__ __forceinline__ ItemCoord decode_item(const UmmaArgs& a, int item, int n_mtiles) {
   ItemCoord c;
-  c.bundle = item / n_mtiles;
-  int mt = item - c.bundle * n_mtiles;
+  c.split = item % a.n_splits;
+  c.tile_id = item / a.n_splits;
+  c.bundle = c.tile_id / n_mtiles;
+  int mt = c.tile_id - c.bundle * n_mtiles;
   const int iw = mt % a.tiles_w; mt /= a.tiles_w;
   const int ih = mt % a.tiles_h; mt /= a.tiles_h;
   const int it = mt % a.tiles_t; mt /= a.tiles_t;
   c.w0 = iw * a.box.bw; c.h0 = ih * a.box.bh; c.t0 = it * a.box.bt; c.n0 = mt * a.box.bn;
   return c;
+}
+
+// Slice of the bundle's step list owned by this item: global index of its first step, number of
+// steps, and the index of the first step inside the bundle's list.
+template <bool kDense>
+__device__ __forceinline__ void item_steps(const UmmaArgs& a, const ItemCoord& c, int& s_begin, int& nsteps, int& local0) {
+  const int base = kDense ? c.bundle * a.steps_dense : a.step_ptr[c.bundle];
+  const int total = kDense ? a.steps_dense : a.step_ptr[c.bundle + 1] - base;
+  local0 = int((long long)total * c.split / a.n_splits);
+  const int hi = int((long long)total * (c.split + 1) / a.n_splits);
+  s_begin = base + local0;
+  nsteps = hi - local0;
+}
+
+// Split-K partial tiles are stored column-major, [column][128 rows] floats, so that the 32 lanes of a
+// warp (32 consecutive rows) always touch 128 contiguous bytes.
+// Raw fp32 accumulator row -> scratch; `dst` already points at this thread's row of column 0.
+__device__ __forceinline__ void store_partial_row(uint32_t taddr, int n_cols, bool has_acc, float* dst) {
+  for (int col = 0; col < n_cols; col += 32) {
+    uint32_t v[32];
+    const bool wide = col + 32 <= n_cols;
+    if (has_acc) {
+      if (wide) tmem_ld32(taddr + col, v);
+      else tmem_ld16(taddr + col, *reinterpret_cast<uint32_t(*)[16]>(v));
+    } else {
+#pragma unroll
+      for (int q = 0; q < 32; ++q) v[q] = 0u;
+    }
+#pragma unroll
+    for (int q = 0; q < 32; ++q)
+      if (wide || q < 16) dst[size_t(col + q) * 128] = __uint_as_float(v[q]);
+  }
+}
+
+// Sum of the partials of all splits (in split order, two splits' loads in flight at a time) + epilogue
+// for one output voxel; `part0` points at this thread's row of column 0 of split 0.
+template <int NC>
+__device__ __forceinline__ void reduce_partial_cols(const float* part0, size_t split_stride, int n_splits,
+                                                    const float* bias_s, int relu, __nv_bfloat16* dst, int valid) {
+  float acc[NC];
+#pragma unroll
+  for (int q = 0; q < NC; ++q) acc[q] = 0.f;
+  int s = 0;
+  for (; s + 1 < n_splits; s += 2) {
+    float t0[NC], t1[NC];
+    const float* p0 = part0 + size_t(s) * split_stride;
+    const float* p1 = p0 + split_stride;
+#pragma unroll
+    for (int q = 0; q < NC; ++q) { t0[q] = __ldcg(p0 + size_t(q) * 128); t1[q] = __ldcg(p1 + size_t(q) * 128); }
+#pragma unroll
+    for (int q = 0; q < NC; ++q) acc[q] = (acc[q] + t0[q]) + t1[q];
+  }
+  if (s < n_splits) {
+    const float* p0 = part0 + size_t(s) * split_stride;
+#pragma unroll
+    for (int q = 0; q < NC; ++q) acc[q] += __ldcg(p0 + size_t(q) * 128);
+  }
+  uint32_t v[NC];
+#pragma unroll
+  for (int q = 0; q < NC; ++q) v[q] = __float_as_uint(acc[q]);
+  epilogue_cols<NC>(v, bias_s, relu, dst, valid);
+}
+
+__device__ __forceinline__ void reduce_partial_row(const float* part0, size_t split_stride, int n_splits, int n_cols,
+                                                   bool in_range, const float* bias_s, int relu, __nv_bfloat16* dst,
+                                                   int m_base, int M) {
+  if (!in_range) return;
+  for (int col = 0; col < n_cols; col += 32) {
+    const int m0 = m_base + col;
+    if (m0 >= M) break;
+    const float* p = part0 + size_t(col) * 128;
+    if (col + 32 <= n_cols) reduce_partial_cols<32>(p, split_stride, n_splits, bias_s + m0, relu, dst + col, M - m0);
+    else reduce_partial_cols<16>(p, split_stride, n_splits, bias_s + m0, relu, dst + col, M - m0);
+  }
 }
 
 template <bool kDense>
@@ -53,7 +136,7 @@ conv3d_umma_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_consta
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n_mtiles = a.tiles_n * a.tiles_t * a.tiles_h * a.tiles_w;
-  const int n_items = n_mtiles * a.n_bundles;
+  const int n_items = n_mtiles * a.n_bundles * a.n_splits;
   const int box_rows = a.box.bn * a.box.bt * a.box.bh * a.box.bw;
 
   if (threadIdx.x == 0) {
@@ -88,12 +171,17 @@ conv3d_umma_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_consta
       const uint32_t tx_bytes = uint32_t(box_rows) * 128u + b_bytes;
       for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
         const ItemCoord c = decode_item(a, item, n_mtiles);
-        const int s_begin = kDense ? c.bundle * a.steps_dense : a.step_ptr[c.bundle];
-        const int nsteps = kDense ? a.steps_dense : a.step_ptr[c.bundle + 1] - s_begin;
+        int s_begin, nsteps, local0;
+        item_steps<kDense>(a, c, s_begin, nsteps, local0);
         const int wq = c.w0 * a.g.sw - a.g.pw, hq = c.h0 * a.g.sh - a.g.ph, tq = c.t0 * a.g.st - a.g.pt;
         // Everything a step needs is computed (dense) or fetched one step ahead (indexed) before the
         // wait on the stage, so a freed stage is re-armed without further latency.
         int kt = 0, kh = 0, kw = 0, ch = 0;
+        if (kDense) {
+          ch = local0 % a.n_chunks;
+          const int pos = local0 / a.n_chunks;
+          kw = pos % a.g.Kw; kh = (pos / a.g.Kw) % a.g.Kh; kt = pos / (a.g.Kw * a.g.Kh);
+        }
         int enc_next = (!kDense && nsteps > 0) ? __ldg(a.steps + s_begin) : 0;
         int wrow = s_begin * a.n_tile;
         for (int i = 0; i < nsteps; ++i, wrow += a.n_tile) {
@@ -110,21 +198,9 @@ conv3d_umma_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_consta
           const uint32_t full = smem_u32(&bars->full[stage]);
           const uint32_t a_dst = tiles_base + stage * stage_bytes;
           if (!mbar_wait(smem_u32(&bars->empty[stage]), phase ^ 1u, bars, err, 1)) { ok = false; break; }
-#if defined(RT3D_EXPERIMENT) && RT3D_EXPERIMENT == 1      /* timing ablation: A tile loaded once per item */
-          mbar_expect_tx(full, i == 0 ? tx_bytes : b_bytes);
-          if (i == 0) tma_load_5d(a_dst, &xmap, full, c_ch, c_w, c_h, c_t, c.n0);
-          tma_load_2d(a_dst + kABytes, &wmap, full, 0, wrow);
-#elif defined(RT3D_EXPERIMENT) && RT3D_EXPERIMENT == 2    /* timing ablation: B tile loaded once per item */
-          mbar_expect_tx(full, i == 0 ? tx_bytes : tx_bytes - b_bytes);
-          tma_load_5d(a_dst, &xmap, full, c_ch, c_w, c_h, c_t, c.n0);
-          if (i == 0) tma_load_2d(a_dst + kABytes, &wmap, full, 0, wrow);
-#elif defined(RT3D_EXPERIMENT) && RT3D_EXPERIMENT == 4    /* timing ablation: no loads at all */
-          mbar_arrive(full);
-#else
           mbar_expect_tx(full, tx_bytes);
           tma_load_5d(a_dst, &xmap, full, c_ch, c_w, c_h, c_t, c.n0);
           tma_load_2d(a_dst + kABytes, &wmap, full, 0, wrow);
-#endif
           if (++stage == stages) { stage = 0; phase ^= 1u; }
         }
       }
@@ -137,8 +213,9 @@ conv3d_umma_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_consta
       int stage = 0;
       bool ok = true;
       for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++j) {
-        const int bundle = item / n_mtiles;
-        const int nsteps = kDense ? a.steps_dense : a.step_ptr[bundle + 1] - a.step_ptr[bundle];
+        const ItemCoord c = decode_item(a, item, n_mtiles);
+        int s_begin, nsteps, local0;
+        item_steps<kDense>(a, c, s_begin, nsteps, local0);
         const uint32_t buf = j & 1u;
         if (!mbar_wait(smem_u32(&bars->tmem_empty[buf]), ((j >> 1) & 1u) ^ 1u, bars, err, 2)) break;
         tc_fence_after();
@@ -151,9 +228,6 @@ conv3d_umma_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_consta
           const uint64_t bdesc = smem_desc_sw128(a_addr + kABytes);
 #pragma unroll
           for (int kk = 0; kk < 4; ++kk)      // 4 x K=16 per 64-channel chunk: +32 bytes = +2 in descriptor units
-#if defined(RT3D_EXPERIMENT) && RT3D_EXPERIMENT == 3      /* timing ablation: one MMA per step instead of four */
-            if (kk == 0)
-#endif
             umma_bf16(d_tmem, adesc + 2 * kk, bdesc + 2 * kk, idesc, (i | kk) ? 1u : 0u);
           umma_commit(smem_u32(&bars->empty[stage]));
           if (++stage == stages) { stage = 0; phase ^= 1u; }
@@ -173,10 +247,12 @@ conv3d_umma_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_consta
     const int bt_i = r % a.box.bt; r /= a.box.bt;
     const int bn_i = r;
     __nv_bfloat16* yb = static_cast<__nv_bfloat16*>(a.y);
+    const size_t part_tile = size_t(128) * a.n_tile;       // floats per partial tile
     uint32_t j = 0;
     for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++j) {
       const ItemCoord c = decode_item(a, item, n_mtiles);
-      const int nsteps = kDense ? a.steps_dense : a.step_ptr[c.bundle + 1] - a.step_ptr[c.bundle];
+      int s_begin, nsteps, local0;
+      item_steps<kDense>(a, c, s_begin, nsteps, local0);
       const uint32_t buf = j & 1u;
       if (!mbar_wait(smem_u32(&bars->tmem_full[buf]), (j >> 1) & 1u, bars, err, 4)) break;
       tc_fence_after();
@@ -185,11 +261,33 @@ conv3d_umma_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_consta
       const long long vox = (((long long)nn * a.g.To + to) * a.g.Ho + ho) * a.g.Wo + wo;
       const int m_base = c.bundle * a.n_tile;
       const uint32_t taddr = tmem_base + (uint32_t(quad * 32) << 16) + buf * uint32_t(a.n_tile);
-      epilogue_row(taddr, a.n_tile, nsteps > 0, in_range, bias_s, a.g.relu,
-                   yb + vox * a.g.ycs + m_base, m_base, a.g.M);
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(smem_u32(&bars->tmem_empty[buf]));
+      __nv_bfloat16* dst = yb + vox * a.g.ycs + m_base;
+      if (a.n_splits == 1) {
+        epilogue_row(taddr, a.n_tile, nsteps > 0, in_range, bias_s, a.g.relu, dst, m_base, a.g.M);
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&bars->tmem_empty[buf]));
+      } else {
+        float* tile_part = a.scratch + size_t(c.tile_id) * a.n_splits * part_tile;
+        store_partial_row(taddr, a.n_tile, nsteps > 0, tile_part + size_t(c.split) * part_tile + row);
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&bars->tmem_empty[buf]));    // accumulator consumed: MMAs may go on
+        // Each warp owns 32 rows of the tile in every split, so the hand-over is per warp: fence the
+        // partial, count this warp in, and the warp that counts last reduces those 32 rows.
+        __threadfence();
+        __syncwarp();
+        int last = 0;
+        if (lane == 0) last = atomicAdd(a.counters + c.tile_id * 4 + quad, 1) == a.n_splits - 1;
+        last = __shfl_sync(0xffffffffu, last, 0);
+        if (last) {
+          __threadfence();
+          reduce_partial_row(tile_part + row, part_tile, a.n_splits, a.n_tile, in_range, bias_s,
+                             a.g.relu, dst, m_base, a.g.M);
+          __syncwarp();
+          if (lane == 0) a.counters[c.tile_id * 4 + quad] = 0;              // ready for the next launch
+        }
+      }
     }
   }
 
@@ -209,7 +307,7 @@ conv3d_umma_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_consta
 
 int pick_stages(int n_tile) {
   const size_t stage = kABytes + size_t(n_tile) * 128;
-  int s = int(kSmemBudget / stage);
+  const int s = int(kSmemBudget / stage);
   return s > kMaxStages ? kMaxStages : s;
 }
 
@@ -229,7 +327,8 @@ cudaError_t launch_conv_umma(const UmmaArgs& a, const void* xmap, const void* wm
   int cols = 32;
   while (cols < 2 * a.n_tile) cols *= 2;
   if (cols > 512) return cudaErrorInvalidValue;
-  const long long n_items = (long long)a.tiles_n * a.tiles_t * a.tiles_h * a.tiles_w * a.n_bundles;
+  if (a.n_splits < 1 || (a.n_splits > 1 && (a.scratch == nullptr || a.counters == nullptr))) return cudaErrorInvalidValue;
+  const long long n_items = (long long)a.tiles_n * a.tiles_t * a.tiles_h * a.tiles_w * a.n_bundles * a.n_splits;
   if (n_items <= 0) return cudaSuccess;
   const int grid = int(n_items < sm_count ? n_items : sm_count);
   CUtensorMap xm, wm;

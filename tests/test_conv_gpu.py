@@ -148,6 +148,31 @@ def test_umma_kernel_strided(case):
     check(y, ref, torch.bfloat16, f"umma strided {case}")
 
 
+SPLITK_CASES = [
+    # few output tiles, long K: the tensor-core kernel splits K across CTAs and reduces fp32 partials
+    (256, 256, (3, 3, 3), (1, 1, 1), (1, 1, 1), (1, 2, 7, 7), 4, 4, 0.4),
+    (512, 512, (3, 3, 3), (1, 1, 1), (1, 1, 1), (2, 2, 7, 7), 4, 4, 0.3),
+    (192, 230, (3, 3, 3), (1, 1, 1), (1, 1, 1), (1, 4, 9, 9), 8, 4, 0.4),      # ragged C_out, 3 m-tiles
+    (576, 96, (3, 1, 1), (1, 1, 1), (1, 0, 0), (1, 4, 7, 7), 4, 4, 0.4),
+]
+
+
+@pytest.mark.parametrize("case", SPLITK_CASES)
+@pytest.mark.parametrize("dense", [False, True])
+def test_umma_split_k_against_oracle(case, dense):
+    cin, cout, k, stride, pad, (n, t, h, w), g_m, g_n, d = case
+    spec = synth.ConvSpec("k", cin, cout, k, stride, pad, True)
+    y, ref, lay, xd, yt = run_case(spec, n, t, h, w, g_m, g_n, "none" if dense else "bernoulli", d, torch.bfloat16,
+                                   rt3d.ALGO_UMMA, dense=dense)
+    check(y, ref, torch.bfloat16, f"split-k {case}")
+    first = yt.clone()
+    for _ in range(3):                       # arrival counters reset themselves; the sum order is fixed
+        lay(xd, yt, algo=rt3d.ALGO_UMMA)
+        torch.cuda.synchronize()
+        assert torch.equal(first, yt)
+    assert rt3d.rt3d_last_device_status() == rt3d.OK
+
+
 def test_umma_dense_entry_point():
     spec = synth.ConvSpec("u", 128, 128, (3, 3, 3), (1, 1, 1), (1, 1, 1), True)
     y, ref, *_ = run_case(spec, 2, 4, 8, 8, 4, 4, "none", None, torch.bfloat16, rt3d.ALGO_UMMA, dense=True)
