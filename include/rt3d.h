@@ -39,7 +39,9 @@ typedef enum {
   RT3D_ERR_UNSUPPORTED = 4,            /* valid request this build cannot run                    */
   RT3D_ERR_ALLOC = 5,                  /* host or device allocation failed                       */
   RT3D_ERR_CUDA = 6,                   /* a CUDA runtime / driver call failed                    */
-  RT3D_ERR_TIMEOUT = 7                 /* a bounded device-side wait gave up (see rt3d_last_device_status) */
+  RT3D_ERR_TIMEOUT = 7,                /* a bounded device-side wait gave up (see rt3d_last_device_status) */
+  RT3D_ERR_WORKSPACE = 8,              /* rt3d_conv3d_sparse_noalloc: the call needs more than the fixed workspace */
+  RT3D_ERR_NOT_PREPARED = 9            /* rt3d_conv3d_sparse_noalloc: handle was not prepared on this device */
 } rt3d_status;
 
 typedef enum { RT3D_F32 = 0, RT3D_BF16 = 1 } rt3d_dtype;
@@ -149,6 +151,36 @@ rt3d_status rt3d_conv3d_sparse(const rt3d_tensor* x, const rt3d_packed* w, const
  * iterated, no index lookups (the dense baseline the paper compares its sparse path with). */
 rt3d_status rt3d_conv3d_dense(const rt3d_tensor* x, const rt3d_packed* w, const float* bias,
                               const rt3d_conv_params* p, rt3d_tensor* y, void* stream);
+
+/*
+ * rt3d_conv3d_sparse_noalloc - rt3d_conv3d_sparse for callers that must not allocate.
+ * (No counterpart in the paper: this is a deployment variant of the tensor-core kernel.)
+ * Some callers cannot call cudaMalloc at the point where they run a layer: code inside a
+ * real-time or latency-critical loop, code that runs while another component owns the device's
+ * memory budget, or a host thread that must never block on the allocator's device-wide
+ * synchronisation.  For them this entry point runs the same tensor-core convolution, including its
+ * K-split variant whose fp32 partial tiles need scratch memory, without any allocation: the scratch
+ * is a fixed array inside the library (16 MiB of partial tiles plus 2 KiB of counters, resident on
+ * every GPU that loads the library until the process exits).
+ *   - Same arguments, layouts and alignment rules as rt3d_conv3d_sparse (device x, y, bias); bf16 only.
+ *   - Everything that does need an allocation must exist already: call rt3d_packed_prepare(w) on this
+ *     device beforehand, else RT3D_ERR_NOT_PREPARED.  Shapes the tensor-core kernel does not take
+ *     (fp32, channel pitch not a multiple of 8, p->algo == RT3D_ALGO_SIMT) give RT3D_ERR_UNSUPPORTED.
+ *   - K is split S ways, S = min(8, SMs / output tiles, K steps / 8), at least 1, where an output
+ *     tile is 128 voxels x up to 256 channels and a K step is one kernel location x 64 input
+ *     channels.  If S > 1 and (output tiles x S) partial tiles of 128 x n_tile floats exceed
+ *     16 MiB, or there are more than 128 output tiles, the call is rejected with
+ *     RT3D_ERR_WORKSPACE and nothing is launched (rt3d_conv3d_sparse has no such limit).
+ *   - The first call on a device looks up the device address of the workspace; make that first
+ *     call before any stream capture begins.  No call allocates or frees device or pinned memory.
+ *   - All calls on a device share the one workspace, which keeps the previous call's contents; the
+ *     entry point clears the counters it needs on `stream` before the kernel.  Two calls whose
+ *     kernels may overlap on the GPU (different streams) race on it: serialise them.
+ *   - Results agree with rt3d_conv3d_sparse within the library's tolerance (the split count, and so
+ *     the fp32 summation order, may differ); repeated calls give identical bits.
+ */
+rt3d_status rt3d_conv3d_sparse_noalloc(const rt3d_tensor* x, const rt3d_packed* w, const float* bias,
+                                       const rt3d_conv_params* p, rt3d_tensor* y, void* stream);
 
 /*
  * rt3d_conv3d_host - end-to-end variant: x->data and y->data are HOST buffers (pinned

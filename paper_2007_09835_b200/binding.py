@@ -18,6 +18,7 @@ LIB_PATH = os.environ.get("RT3D_LIB") or os.path.join(_HERE, "librt3d.so")   # R
 RT3D_F32, RT3D_BF16 = 0, 1
 ALGO_AUTO, ALGO_SIMT, ALGO_UMMA = 0, 1, 2
 OK, ERR_INVALID_ARG, ERR_SHAPE, ERR_MASK_NOT_GROUP_UNIFORM, ERR_UNSUPPORTED, ERR_ALLOC, ERR_CUDA, ERR_TIMEOUT = range(8)
+ERR_WORKSPACE, ERR_NOT_PREPARED = 8, 9
 
 
 class Rt3dError(RuntimeError):
@@ -60,7 +61,7 @@ def _load():
     lib.rt3d_packed_prepare.argtypes = [vp]
     lib.rt3d_packed_free.argtypes = [vp]
     lib.rt3d_packed_free.restype = None
-    for name in ("rt3d_conv3d_sparse", "rt3d_conv3d_dense", "rt3d_conv3d_host"):
+    for name in ("rt3d_conv3d_sparse", "rt3d_conv3d_dense", "rt3d_conv3d_host", "rt3d_conv3d_sparse_noalloc"):
         getattr(lib, name).argtypes = [TP, vp, vp, CP, TP, vp]
     lib.rt3d_maxpool3d.argtypes = [TP] + [i] * 9 + [TP, vp]
     lib.rt3d_add_relu.argtypes = [TP, TP, i, TP, vp]
@@ -206,6 +207,17 @@ def rt3d_conv3d_sparse(x: Tensor, w: Packed, bias, y: Tensor, stride=(1, 1, 1), 
     _check(_lib.rt3d_conv3d_sparse(ctypes.byref(x), w.handle, _bias_ptr(bias),
                                    ctypes.byref(_params(stride, pad, relu, algo)), ctypes.byref(y),
                                    _stream_ptr(stream)), "rt3d_conv3d_sparse")
+
+
+def rt3d_conv3d_sparse_noalloc(x: Tensor, w: Packed, bias, y: Tensor, stride=(1, 1, 1), pad=(0, 0, 0), relu=False,
+                               algo=ALGO_AUTO, stream=None):
+    """rt3d_conv3d_sparse for callers that must not allocate device memory at call time (a real-time
+    loop, a thread that may not block on the allocator): the handle must have been prepared on this
+    device (`w.prepare()`), the K-split scratch is a fixed 16 MiB array inside the library, and a call
+    that would need more raises Rt3dError with status ERR_WORKSPACE."""
+    _check(_lib.rt3d_conv3d_sparse_noalloc(ctypes.byref(x), w.handle, _bias_ptr(bias),
+                                           ctypes.byref(_params(stride, pad, relu, algo)), ctypes.byref(y),
+                                           _stream_ptr(stream)), "rt3d_conv3d_sparse_noalloc")
 
 
 def rt3d_conv3d_dense(x: Tensor, w: Packed, bias, y: Tensor, stride=(1, 1, 1), pad=(0, 0, 0), relu=False,

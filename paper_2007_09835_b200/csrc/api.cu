@@ -579,6 +579,110 @@ rt3d_status rt3d_last_device_status(void* stream) {
   return RT3D_OK;
 }
 
+// ------------------------------------------------------------------ entry point without allocation
+// Fixed workspace for rt3d_conv3d_sparse_noalloc: split-K partial tiles followed by the per-warp
+// arrival counters.  It lives in every GPU context that loads this library, for the life of the
+// process.  In host code `g_noalloc_ws` is only a handle for the runtime, never a device address:
+// the address is looked up per device with cudaGetSymbolAddress below.
+#define RT3D_NOALLOC_PARTIAL_TILES 128                                   /* 128 x 256 fp32 each */
+#define RT3D_NOALLOC_PARTIAL_BYTES (RT3D_NOALLOC_PARTIAL_TILES * 128 * 256 * 4)   /* 16 MiB */
+#define RT3D_NOALLOC_COUNTER_BYTES (RT3D_NOALLOC_PARTIAL_TILES * 4 * 4)  /* 4 counters per output tile */
+static __device__ __align__(256) unsigned char g_noalloc_ws[RT3D_NOALLOC_PARTIAL_BYTES + RT3D_NOALLOC_COUNTER_BYTES];
+
+namespace {
+struct NoAllocState { bool ready = false; unsigned char* ws = nullptr; };
+NoAllocState g_noalloc[64];
+std::mutex g_noalloc_mu;
+
+// Once per device, with that device current: resolve the device address of the workspace.
+rt3d_status noalloc_workspace(int dev, unsigned char** ws) {
+  std::lock_guard<std::mutex> lock(g_noalloc_mu);
+  NoAllocState& st = g_noalloc[dev];
+  if (!st.ready) {
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_noalloc_ws) != cudaSuccess || p == nullptr) return RT3D_ERR_CUDA;
+    st.ws = static_cast<unsigned char*>(p);
+    st.ready = true;
+  }
+  *ws = st.ws;
+  return RT3D_OK;
+}
+}  // namespace
+
+rt3d_status rt3d_conv3d_sparse_noalloc(const rt3d_tensor* x, const rt3d_packed* wc, const float* bias,
+                                       const rt3d_conv_params* p, rt3d_tensor* y, void* stream) {
+  ConvGeom g;
+  if (!y) return RT3D_ERR_INVALID_ARG;
+  rt3d_status s = make_geom(x, wc, p, y, &g);
+  if (s != RT3D_OK) return s;
+  if ((s = check_alignment(x)) != RT3D_OK || (s = check_alignment(y)) != RT3D_OK) return s;
+  if (overlaps(x, y)) return RT3D_ERR_INVALID_ARG;
+  if (p->algo == RT3D_ALGO_SIMT) return RT3D_ERR_UNSUPPORTED;
+  rt3d_packed* w = const_cast<rt3d_packed*>(wc);
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return RT3D_ERR_CUDA;
+  // everything that needs an allocation must already exist: device state, weight blobs (rt3d_packed_prepare)
+  DeviceState* d = nullptr;
+  {
+    std::lock_guard<std::mutex> lock(g_dev_mu);
+    if (g_dev[dev].init) d = &g_dev[dev];
+  }
+  if (!d) return RT3D_ERR_NOT_PREPARED;
+  if (!umma_eligible(d, w, x, y, p)) return RT3D_ERR_UNSUPPORTED;
+  const int n_tile = default_n_tile(w->M);
+  DeviceBlob* blob = nullptr;
+  DeviceBlob::Umma* u = nullptr;
+  const UmmaLayout* L = nullptr;
+  {
+    std::lock_guard<std::mutex> lock(w->mu);
+    blob = find_blob(w, dev);
+    if (blob) {
+      auto it = blob->umma.find(n_tile);
+      if (it != blob->umma.end() && it->second.ready) u = &it->second;
+    }
+    auto li = w->umma_layouts.find(n_tile);
+    if (li != w->umma_layouts.end()) L = &li->second;
+  }
+  if (!blob || !u || !L) return RT3D_ERR_NOT_PREPARED;
+  unsigned char* ws = nullptr;
+  if ((s = noalloc_workspace(dev, &ws)) != RT3D_OK) return s;
+
+  UmmaArgs a;
+  a.g = g;
+  a.box = choose_box(g);
+  a.tiles_n = ceil_div(g.n, a.box.bn); a.tiles_t = ceil_div(g.To, a.box.bt);
+  a.tiles_h = ceil_div(g.Ho, a.box.bh); a.tiles_w = ceil_div(g.Wo, a.box.bw);
+  a.n_tile = L->n_tile; a.n_bundles = L->n_bundles; a.n_chunks = L->n_chunks;
+  a.dense = 0;
+  a.steps_dense = w->Ks * L->n_chunks;
+  a.step_ptr = u->step_ptr; a.steps = u->steps;
+  a.bias = bias; a.y = y->data; a.sched = d->sched;
+  // Split rule of this entry point: as many K splits (at most 8) as keep every SM busy, each with at
+  // least 8 of the layer's K steps.
+  const long long tiles = (long long)a.tiles_n * a.tiles_t * a.tiles_h * a.tiles_w * L->n_bundles;
+  long long splits = tiles > 0 ? d->sm_count / tiles : 1;
+  if (splits > 8) splits = 8;
+  if (splits > a.steps_dense / 8) splits = a.steps_dense / 8;
+  if (splits < 1) splits = 1;
+  a.n_splits = int(splits);
+  a.scratch = nullptr; a.counters = nullptr;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (a.n_splits > 1) {
+    const long long partial_bytes = tiles * a.n_splits * kTileM * L->n_tile * 4LL;
+    if (partial_bytes > RT3D_NOALLOC_PARTIAL_BYTES || tiles * 16 > RT3D_NOALLOC_COUNTER_BYTES)
+      return RT3D_ERR_WORKSPACE;
+    a.scratch = reinterpret_cast<float*>(ws);
+    a.counters = reinterpret_cast<int32_t*>(ws + RT3D_NOALLOC_PARTIAL_BYTES);
+    // the counters must start at zero; the workspace keeps whatever the last call left behind
+    if (cudaMemsetAsync(a.counters, 0, size_t(tiles) * 16, st) != cudaSuccess) return RT3D_ERR_CUDA;
+  }
+  CUtensorMap xmap;
+  if ((s = encode_xmap(x, g, a.box, &xmap)) != RT3D_OK) return s;
+  if (launch_conv_umma(a, &xmap, u->wmap, d->sm_count, st) != cudaSuccess) return RT3D_ERR_CUDA;
+  g_launches.fetch_add(1);
+  return RT3D_OK;
+}
+
 int64_t rt3d_launch_count(void) { return g_launches.load(); }
 
 const char* rt3d_status_string(rt3d_status s) {
@@ -591,6 +695,8 @@ const char* rt3d_status_string(rt3d_status s) {
     case RT3D_ERR_ALLOC: return "allocation failed";
     case RT3D_ERR_CUDA: return "CUDA error";
     case RT3D_ERR_TIMEOUT: return "device-side wait timed out";
+    case RT3D_ERR_WORKSPACE: return "request needs more than the library's fixed workspace";
+    case RT3D_ERR_NOT_PREPARED: return "handle not prepared on this device (call rt3d_packed_prepare first)";
   }
   return "unknown status";
 }
