@@ -114,6 +114,69 @@ def oracle_timed(spec, L, x, clips: int):
     return time.perf_counter() - t0
 
 
+def time_networks(torch, rt3d, nets, dev, iters=20):
+    """Forward passes of the C3D-shaped (cfg2: batch 1 and 16, KGS ~3.6x and dense) and R(2+1)D-18-shaped
+    (cfg3: batch 8, KGS ~2.5x) networks, each captured in a CUDA graph; clips per second."""
+    out = {}
+
+    def timed(fwd):
+        for _ in range(3):
+            fwd()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(iters):
+            fwd()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / iters
+
+    plan = synth.c3d_plan()
+    specs = [(i, op) for i, op in enumerate(plan) if isinstance(op, synth.ConvSpec)]
+    raw = {op.name: synth.make_layer(op, 2, i, 4, 4, "bernoulli", 1 / 3.6) for i, op in specs}
+    for mode in ("kgs", "dense"):
+        layers = {op.name: nets.ConvLayer(op, raw[op.name]["w"], raw[op.name]["bias"],
+                                          None if mode == "dense" else raw[op.name]["mask"], 4, 4, torch.bfloat16,
+                                          dense=(mode == "dense"), device=dev) for _, op in specs}
+        net = nets.C3DNet(plan, layers)
+        for batch in (1, 16):
+            x = nets.to_device(synth.make_input(2, (batch, 16, 112, 112, 3)), torch.bfloat16, device=dev)
+            ms = timed(nets.GraphedForward(net, x))
+            out[f"c3d_{mode}_b{batch}_clips_per_s"] = batch / ms * 1e3
+            out[f"c3d_{mode}_b{batch}_ms"] = ms
+        if mode == "kgs":
+            kept = dense = 0
+            t, h, w = 16, 112, 112
+            for op in plan:
+                if isinstance(op, synth.ConvSpec):
+                    k, d, _ = layers[op.name].cost(torch.empty((1, t, h, w, nets.pitch_for(op.cin, torch.bfloat16)),
+                                                               dtype=torch.bfloat16, device=dev))
+                    kept += k; dense += d
+                    t, h, w = op.out_extent(t, h, w)
+                else:
+                    t, h, w = [(dd + 2 * p - kk) // s + 1 for dd, p, kk, s in zip((t, h, w), op.pad, op.k, op.stride)]
+            out["c3d_flops_pruning_rate"] = dense / kept
+            out["c3d_dense_gmac_per_clip"] = dense / 1e9
+        del net, layers
+    out["c3d_b16_speedup_vs_dense"] = out["c3d_dense_b16_ms"] / out["c3d_kgs_b16_ms"]
+    del raw
+
+    stem, blocks = synth.r2plus1d18_plan()
+    rspecs = list(stem)
+    for blk in blocks:
+        rspecs += list(blk.convs) + ([blk.shortcut] if blk.shortcut is not None else [])
+    rlayers = {}
+    for i, sp in enumerate(rspecs):
+        L = synth.make_layer(sp, 3, i, 4, 4, "bernoulli", 0.4)
+        rlayers[sp.name] = nets.ConvLayer(sp, L["w"], L["bias"], L["mask"], 4, 4, torch.bfloat16, device=dev)
+    rnet = nets.R2Plus1DNet(stem, blocks, rlayers)
+    x = nets.to_device(synth.make_input(3, (8, 16, 112, 112, 3)), torch.bfloat16, device=dev)
+    ms = timed(nets.GraphedForward(rnet, x))
+    out["r2plus1d_kgs_b8_clips_per_s"] = 8 / ms * 1e3
+    out["r2plus1d_kgs_b8_ms"] = ms
+    return out
+
+
 def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
@@ -148,6 +211,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--l2-warm", action="store_true", help="reuse one buffer set (operands stay in L2); default rotates sets")
+    ap.add_argument("--no-networks", action="store_true", help="skip the C3D / R(2+1)D-shaped forward passes")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":
@@ -226,6 +290,10 @@ def main():
     e2e_ms = dist.max_over_ranks(e0.elapsed_time(e1), group, dev) / e2e_steps
     sampler.stop()
 
+    networks = None
+    if not args.no_networks:
+        networks = time_networks(torch, rt3d, nets, dev)
+
     flops_kept = 2.0 * kept_macs
     per_step_ms = sparse_ms / args.steps
     value = world * flops_kept / (per_step_ms * 1e-3) / 1e12
@@ -254,6 +322,8 @@ def main():
                      "executed_tflops": 2.0 * dense_macs / (per_step_ms * 1e-3) / 1e12,
                      "alg_bytes_per_launch": alg_bytes},
     }
+    if networks is not None:
+        out["networks"] = networks
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         import oracle
         clips = CFG["n"]
