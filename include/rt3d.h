@@ -50,7 +50,9 @@ typedef enum { RT3D_F32 = 0, RT3D_BF16 = 1 } rt3d_dtype;
 typedef enum {
   RT3D_ALGO_AUTO = 0,   /* tensor-core kernel when the shape allows it, else the CUDA-core kernel */
   RT3D_ALGO_SIMT = 1,   /* CUDA-core kernel driven by the canonical packed index (any shape)      */
-  RT3D_ALGO_UMMA = 2    /* tcgen05 tensor-core kernel; RT3D_ERR_UNSUPPORTED if not applicable     */
+  RT3D_ALGO_UMMA = 2,   /* tcgen05 tensor-core kernel, one CTA per tile; RT3D_ERR_UNSUPPORTED if not applicable */
+  RT3D_ALGO_UMMA_PAIR = 3 /* tcgen05 kernel on CTA pairs (two tiles per MMA, weight tile shared by the
+                             pair); RT3D_ERR_UNSUPPORTED if not applicable                        */
 } rt3d_algo;
 
 /* NDHWC activation tensor in DEVICE memory (HOST memory for the *_host entry point), caller-owned. */

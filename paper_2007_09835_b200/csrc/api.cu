@@ -77,7 +77,7 @@ rt3d_status make_geom(const rt3d_tensor* x, const rt3d_packed* w, const rt3d_con
   if (s != RT3D_OK) return s;
   if (!w || !p) return RT3D_ERR_INVALID_ARG;
   if (p->st < 1 || p->sh < 1 || p->sw < 1 || p->pt < 0 || p->ph < 0 || p->pw < 0) return RT3D_ERR_INVALID_ARG;
-  if (p->algo < RT3D_ALGO_AUTO || p->algo > RT3D_ALGO_UMMA) return RT3D_ERR_INVALID_ARG;
+  if (p->algo < RT3D_ALGO_AUTO || p->algo > RT3D_ALGO_UMMA_PAIR) return RT3D_ERR_INVALID_ARG;
   if (x->c != w->N || x->dtype != w->dtype) return RT3D_ERR_SHAPE;
   const int64_t To = (int64_t(x->t) + 2 * p->pt - w->Kt) / p->st + 1;
   const int64_t Ho = (int64_t(x->h) + 2 * p->ph - w->Kh) / p->sh + 1;
@@ -175,6 +175,13 @@ rt3d_status get_umma_blob(rt3d_packed* h, DeviceBlob* blob, const UmmaLayout* L,
                           strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                           CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return RT3D_ERR_CUDA;
+    if (L->n_tile % 32 == 0) {
+      cuuint32_t box_half[2] = {64, cuuint32_t(L->n_tile / 2)};
+      r = g_encode(reinterpret_cast<CUtensorMap*>(u.wmap_half), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, u.wtiles, dims,
+                   strides, box_half, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                   CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+      if (r != CUDA_SUCCESS) return RT3D_ERR_CUDA;
+    }
     u.ready = true;
   }
   *out = &u;
@@ -346,8 +353,9 @@ rt3d_status conv_impl(const rt3d_tensor* x, const rt3d_packed* wc, const float* 
   cudaStream_t st = static_cast<cudaStream_t>(stream);
 
   const bool can_umma = umma_eligible(d, w, x, y, p);
-  if (p->algo == RT3D_ALGO_UMMA && !can_umma) return RT3D_ERR_UNSUPPORTED;
-  const bool use_umma = p->algo == RT3D_ALGO_UMMA || (p->algo == RT3D_ALGO_AUTO && can_umma);
+  if ((p->algo == RT3D_ALGO_UMMA || p->algo == RT3D_ALGO_UMMA_PAIR) && !can_umma) return RT3D_ERR_UNSUPPORTED;
+  const bool use_umma = p->algo == RT3D_ALGO_UMMA || p->algo == RT3D_ALGO_UMMA_PAIR ||
+                        (p->algo == RT3D_ALGO_AUTO && can_umma);
   if (!use_umma) {
     cudaError_t e = launch_conv_simt(w->dtype, g, x->data, y->data, blob->group_ptr, blob->pos_idx, blob->tiles, bias,
                                      w->g_m, w->g_n, w->P, w->Q, dense_entry, st);
@@ -357,7 +365,8 @@ rt3d_status conv_impl(const rt3d_tensor* x, const rt3d_packed* wc, const float* 
   }
 
   const SmallCLayout* SL = nullptr;
-  if (smallc_eligible(d, w, x, y, p, &SL)) return launch_smallc(w, blob, d, SL, x, g, bias, y, st);
+  if (p->algo != RT3D_ALGO_UMMA_PAIR && smallc_eligible(d, w, x, y, p, &SL))
+    return launch_smallc(w, blob, d, SL, x, g, bias, y, st);
 
   UmmaArgs a;
   a.g = g;
@@ -365,7 +374,18 @@ rt3d_status conv_impl(const rt3d_tensor* x, const rt3d_packed* wc, const float* 
   a.tiles_n = ceil_div(g.n, a.box.bn); a.tiles_t = ceil_div(g.To, a.box.bt);
   a.tiles_h = ceil_div(g.Ho, a.box.bh); a.tiles_w = ceil_div(g.Wo, a.box.bw);
   const long long m_tiles = (long long)a.tiles_n * a.tiles_t * a.tiles_h * a.tiles_w;
-  const UmmaPlan plan = pick_plan(w->M, m_tiles, w->Ks * ceil_div(w->N, kChunk), d->sm_count);
+  UmmaPlan plan = pick_plan(w->M, m_tiles, w->Ks * ceil_div(w->N, kChunk), d->sm_count);
+  // CTA pairs: two tiles per MMA.  Worth it when every pair has work; forced by RT3D_ALGO_UMMA_PAIR.
+  bool use_pair = false;
+  if (p->algo == RT3D_ALGO_UMMA_PAIR) {
+    plan = UmmaPlan{default_n_tile(w->M), 1};
+    if (!umma_pair_supported(plan.n_tile, ceil_div(w->M, plan.n_tile))) return RT3D_ERR_UNSUPPORTED;
+    use_pair = true;
+  } else if (p->algo == RT3D_ALGO_AUTO && plan.n_splits == 1 &&
+             umma_pair_supported(plan.n_tile, ceil_div(w->M, plan.n_tile)) &&
+             m_tiles * ceil_div(w->M, plan.n_tile) >= d->sm_count) {
+    use_pair = true;
+  }
   const UmmaLayout* L = get_umma_layout(w, plan.n_tile);
   if (!L) return RT3D_ERR_UNSUPPORTED;
   DeviceBlob::Umma* u = nullptr;
@@ -399,7 +419,8 @@ rt3d_status conv_impl(const rt3d_tensor* x, const rt3d_packed* wc, const float* 
   }
   CUtensorMap xmap;
   if ((s = encode_xmap(x, g, a.box, &xmap)) != RT3D_OK) return s;
-  cudaError_t e = launch_conv_umma(a, &xmap, u->wmap, d->sm_count, st);
+  cudaError_t e = use_pair ? launch_conv_umma_pair(a, &xmap, u->wmap_half, d->sm_count, st)
+                           : launch_conv_umma(a, &xmap, u->wmap, d->sm_count, st);
   if (e != cudaSuccess) return RT3D_ERR_CUDA;
   g_launches.fetch_add(1);
   return RT3D_OK;

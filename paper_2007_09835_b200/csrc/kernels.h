@@ -55,6 +55,12 @@ struct UmmaArgs {
 cudaError_t launch_conv_umma(const UmmaArgs& a, const void* xmap, const void* wmap, int sm_count,
                              cudaStream_t stream);
 
+// CTA-pair variant (cta_group::2): wmap_half is a tensor map over the same weight tiles whose box is
+// half a tile high (n_tile/2 rows).  Needs n_tile % 32 == 0 and a.n_splits == 1.
+bool umma_pair_supported(int n_tile, int n_bundles);
+cudaError_t launch_conv_umma_pair(const UmmaArgs& a, const void* xmap, const void* wmap_half, int sm_count,
+                                  cudaStream_t stream);
+
 // Arguments of the small-C_in tensor-core kernel (C_in <= 8 at channel pitch 8, stride 1).
 struct SmallCArgs {
   ConvGeom g;

@@ -64,7 +64,8 @@ struct DeviceBlob {
     void* wtiles = nullptr;
     int32_t* step_ptr = nullptr;
     int32_t* steps = nullptr;
-    alignas(64) unsigned char wmap[128];   // CUtensorMap of wtiles
+    alignas(64) unsigned char wmap[128];   // CUtensorMap of wtiles, box = one [n_tile][64] tile
+    alignas(64) unsigned char wmap_half[128];   // same tensor, box = half a tile (CTA-pair kernel)
     bool ready = false;
   };
   std::map<int, Umma> umma;          // keyed by n_tile

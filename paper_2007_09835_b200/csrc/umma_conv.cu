@@ -211,7 +211,7 @@ conv3d_umma_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_consta
       const uint32_t idesc = instr_desc_bf16(a.n_tile);
       uint32_t j = 0, phase = 0;
       int stage = 0;
-      bool ok = true;
+      bool ok = true, ready = false;
       for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++j) {
         const ItemCoord c = decode_item(a, item, n_mtiles);
         int s_begin, nsteps, local0;
@@ -221,7 +221,11 @@ conv3d_umma_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_consta
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + buf * uint32_t(a.n_tile);
         for (int i = 0; i < nsteps; ++i) {
-          if (!mbar_wait(smem_u32(&bars->full[stage]), phase, bars, err, 3)) { ok = false; break; }
+          if (!ready && !mbar_wait(smem_u32(&bars->full[stage]), phase, bars, err, 3)) { ok = false; break; }
+          // poll the next stage's barrier now: its answer arrives while this stage's MMAs are issued
+          const int stage_n = stage + 1 == stages ? 0 : stage + 1;
+          const uint32_t phase_n = stage + 1 == stages ? phase ^ 1u : phase;
+          ready = mbar_try_wait(smem_u32(&bars->full[stage_n]), phase_n);
           tc_fence_after();
           const uint32_t a_addr = tiles_base + stage * stage_bytes;
           const uint64_t adesc = smem_desc_sw128(a_addr);
@@ -230,7 +234,7 @@ conv3d_umma_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_consta
           for (int kk = 0; kk < 4; ++kk)      // 4 x K=16 per 64-channel chunk: +32 bytes = +2 in descriptor units
             umma_bf16(d_tmem, adesc + 2 * kk, bdesc + 2 * kk, idesc, (i | kk) ? 1u : 0u);
           umma_commit(smem_u32(&bars->empty[stage]));
-          if (++stage == stages) { stage = 0; phase ^= 1u; }
+          stage = stage_n; phase = phase_n;
         }
         if (!ok) break;
         if (nsteps > 0) umma_commit(smem_u32(&bars->tmem_full[buf]));

@@ -1,0 +1,324 @@
+// Tensor-core KGS convolution on CTA pairs (tcgen05 cta_group::2).
+//
+// Same implicit GEMM as conv3d_umma_kernel, but two CTAs on neighbouring SMs form a cluster and
+// work on two output tiles of the same bundle at once: one MMA instruction, issued by a single
+// thread of the leader CTA, multiplies a 256-row A operand (128 voxels from each CTA's shared
+// memory) by the bundle's B tile, of which each CTA stages only half (n_tile/2 rows).  Per SM this
+// halves the weight bytes pulled from L2 per step and the per-step cost of the issuing thread,
+// which bound the single-CTA kernel.  Accumulators stay per CTA (128 TMEM lanes each), so the
+// epilogue is unchanged.
+//
+// Synchronisation: both producers wait on their own `empty[s]` (released for both CTAs by one
+// multicast commit), both send their loads' completion bytes to the leader's `full[s]`; the
+// leader's MMA thread waits there, issues, and commits to `empty[s]` / `tmem_full[b]` of both CTAs;
+// the epilogue warps of both CTAs release the accumulator on the leader's `tmem_empty[b]`.
+// All waits are bounded as in the single-CTA kernel.
+#include "kernels.h"
+#include "umma_common.cuh"
+
+namespace rt3d {
+namespace {
+
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// Address of the same shared-memory location in CTA `rank` of the cluster.
+__device__ __forceinline__ uint32_t mapa_shared(uint32_t addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ void tma_load_5d_pair(uint32_t dst, const CUtensorMap* map, uint32_t bar_cluster, int c0, int c1,
+                                                 int c2, int c3, int c4) {
+  asm volatile(
+      "cp.async.bulk.tensor.5d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar_cluster), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4)
+      : "memory");
+}
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, uint32_t bar_cluster, int c0, int c1) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar_cluster), "r"(c0), "r"(c1)
+      : "memory");
+}
+__device__ __forceinline__ void umma_bf16_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      "setp.ne.b32 p, %4, 0;\n"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n"
+      "}\n"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc)
+      : "memory");
+}
+// Arrive on the barrier at this shared-memory offset in both CTAs once all prior MMAs are done.
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
+  const uint16_t mask = 3;
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(bar), "h"(mask) : "memory");
+}
+// bf16 x bf16 -> fp32, K-major operands, M = 256 (128 rows per CTA), N = n.
+__device__ __forceinline__ uint32_t instr_desc_bf16_pair(int n) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | (uint32_t(n >> 3) << 17) | (uint32_t(256 >> 4) << 24);
+}
+
+struct PairItem {
+  int bundle;
+  int n0, t0, h0, w0;     // first output voxel of this CTA's box (beyond the tensor for a dummy tile)
+};
+
+__device__ __forceinline__ PairItem decode_pair_item(const UmmaArgs& a, int item, int pairs_per_bundle, int n_mtiles,
+                                                     uint32_t rank) {
+  PairItem c;
+  c.bundle = item / pairs_per_bundle;
+  int mt = (item - c.bundle * pairs_per_bundle) * 2 + int(rank);
+  if (mt >= n_mtiles) {            // odd tile count: the last pair's second tile does not exist
+    c.n0 = a.g.n; c.t0 = 0; c.h0 = 0; c.w0 = 0;
+    return c;
+  }
+  const int iw = mt % a.tiles_w; mt /= a.tiles_w;
+  const int ih = mt % a.tiles_h; mt /= a.tiles_h;
+  const int it = mt % a.tiles_t; mt /= a.tiles_t;
+  c.w0 = iw * a.box.bw; c.h0 = ih * a.box.bh; c.t0 = it * a.box.bt; c.n0 = mt * a.box.bn;
+  return c;
+}
+
+template <bool kDense>
+__global__ void __launch_bounds__(kThreadsUmma, 1)
+conv3d_umma_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CUtensorMap wmap_half,
+                        const UmmaArgs a, const int stages, const int tmem_cols) {
+  extern __shared__ unsigned char smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t tiles_base = (raw + 1023u) & ~1023u;
+  const int n_half = a.n_tile / 2;
+  const uint32_t b_bytes = uint32_t(n_half) * 128u;             // this CTA's half of the B tile
+  const uint32_t stage_bytes = kABytes + b_bytes;
+  Barriers* bars = reinterpret_cast<Barriers*>(smem_raw + (tiles_base - raw) + size_t(stages) * stage_bytes);
+  float* bias_s = reinterpret_cast<float*>(bars + 1);
+  int32_t* err = a.sched + 2;
+  for (int i = threadIdx.x; i < a.n_bundles * a.n_tile; i += blockDim.x)
+    bias_s[i] = (a.bias != nullptr && i < a.g.M) ? __ldg(a.bias + i) : 0.f;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();
+  const bool leader = rank == 0;
+  const int n_mtiles = a.tiles_n * a.tiles_t * a.tiles_h * a.tiles_w;
+  const int pairs_per_bundle = (n_mtiles + 1) / 2;
+  const int n_items = pairs_per_bundle * a.n_bundles;
+  const int cluster_id = blockIdx.x >> 1, n_clusters = gridDim.x >> 1;
+  const int box_rows = a.box.bn * a.box.bt * a.box.bh * a.box.bw;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < stages; ++s) {
+      mbar_init(smem_u32(&bars->full[s]), 1);     // leader: its producer's arrive + both CTAs' bytes
+      mbar_init(smem_u32(&bars->empty[s]), 1);    // multicast commit
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(smem_u32(&bars->tmem_full[b]), 1);    // multicast commit
+      mbar_init(smem_u32(&bars->tmem_empty[b]), 8);   // leader: 4 epilogue warps of each CTA
+    }
+    bars->abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
+                 ::"r"(smem_u32(&bars->tmem_base)), "r"(uint32_t(tmem_cols)) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();              // barriers of both CTAs are initialised before anyone signals them
+  tc_fence_after();
+  const uint32_t tmem_base = bars->tmem_base;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer (both CTAs)
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      const uint32_t tx_both = 2u * (uint32_t(box_rows) * 128u + b_bytes);
+      for (int item = cluster_id; item < n_items && ok; item += n_clusters) {
+        const PairItem c = decode_pair_item(a, item, pairs_per_bundle, n_mtiles, rank);
+        const int s_begin = kDense ? c.bundle * a.steps_dense : a.step_ptr[c.bundle];
+        const int nsteps = kDense ? a.steps_dense : a.step_ptr[c.bundle + 1] - s_begin;
+        const int wq = c.w0 * a.g.sw - a.g.pw, hq = c.h0 * a.g.sh - a.g.ph, tq = c.t0 * a.g.st - a.g.pt;
+        int kt = 0, kh = 0, kw = 0, ch = 0;
+        int enc_next = (!kDense && nsteps > 0) ? __ldg(a.steps + s_begin) : 0;
+        int wrow = s_begin * a.n_tile + int(rank) * n_half;
+        for (int i = 0; i < nsteps; ++i, wrow += a.n_tile) {
+          int c_ch, c_w, c_h, c_t;
+          if (kDense) {
+            c_ch = ch * 64; c_w = wq + kw; c_h = hq + kh; c_t = tq + kt;
+            if (++ch == a.n_chunks) { ch = 0; if (++kw == a.g.Kw) { kw = 0; if (++kh == a.g.Kh) { kh = 0; ++kt; } } }
+          } else {
+            const int enc = enc_next;
+            if (i + 1 < nsteps) enc_next = __ldg(a.steps + s_begin + i + 1);
+            c_t = tq + ((enc >> 24) & 63); c_h = hq + ((enc >> 18) & 63); c_w = wq + ((enc >> 12) & 63);
+            c_ch = (enc & 4095) * 64;
+          }
+          const uint32_t full_local = smem_u32(&bars->full[stage]);
+          const uint32_t full_leader = mapa_shared(full_local, 0);
+          const uint32_t a_dst = tiles_base + stage * stage_bytes;
+          if (!mbar_wait(smem_u32(&bars->empty[stage]), phase ^ 1u, bars, err, 21)) { ok = false; break; }
+          if (leader) mbar_expect_tx(full_local, tx_both);
+          tma_load_5d_pair(a_dst, &xmap, full_leader, c_ch, c_w, c_h, c_t, c.n0);
+          tma_load_2d_pair(a_dst + kABytes, &wmap_half, full_leader, 0, wrow);
+          if (++stage == stages) { stage = 0; phase ^= 1u; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer (leader CTA only)
+    if (lane == 0 && leader) {
+      const uint32_t idesc = instr_desc_bf16_pair(a.n_tile);
+      uint32_t j = 0, phase = 0;
+      int stage = 0;
+      bool ok = true, ready = false;
+      for (int item = cluster_id; item < n_items && ok; item += n_clusters, ++j) {
+        const int bundle = item / pairs_per_bundle;
+        const int nsteps = kDense ? a.steps_dense : a.step_ptr[bundle + 1] - a.step_ptr[bundle];
+        const uint32_t buf = j & 1u;
+        if (!mbar_wait(smem_u32(&bars->tmem_empty[buf]), ((j >> 1) & 1u) ^ 1u, bars, err, 22)) break;
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + buf * uint32_t(a.n_tile);
+        for (int i = 0; i < nsteps; ++i) {
+          if (!ready && !mbar_wait(smem_u32(&bars->full[stage]), phase, bars, err, 23)) { ok = false; break; }
+          // poll the next stage's barrier now: its answer arrives while this stage's MMAs are issued
+          const int stage_n = stage + 1 == stages ? 0 : stage + 1;
+          const uint32_t phase_n = stage + 1 == stages ? phase ^ 1u : phase;
+          ready = mbar_try_wait(smem_u32(&bars->full[stage_n]), phase_n);
+          tc_fence_after();
+          const uint32_t a_addr = tiles_base + stage * stage_bytes;
+          const uint64_t adesc = smem_desc_sw128(a_addr);
+          const uint64_t bdesc = smem_desc_sw128(a_addr + kABytes);
+#pragma unroll
+          for (int kk = 0; kk < 4; ++kk)
+            umma_bf16_pair(d_tmem, adesc + 2 * kk, bdesc + 2 * kk, idesc, (i | kk) ? 1u : 0u);
+          umma_commit_pair(smem_u32(&bars->empty[stage]));
+          stage = stage_n; phase = phase_n;
+        }
+        if (!ok) break;
+        umma_commit_pair(smem_u32(&bars->tmem_full[buf]));     // with no MMAs pending this arrives at once
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue (both CTAs)
+    const int quad = warp & 3;
+    const int row = quad * 32 + lane;
+    int r = row;
+    const int bw_i = r % a.box.bw; r /= a.box.bw;
+    const int bh_i = r % a.box.bh; r /= a.box.bh;
+    const int bt_i = r % a.box.bt; r /= a.box.bt;
+    const int bn_i = r;
+    __nv_bfloat16* yb = static_cast<__nv_bfloat16*>(a.y);
+    uint32_t j = 0;
+    for (int item = cluster_id; item < n_items; item += n_clusters, ++j) {
+      const PairItem c = decode_pair_item(a, item, pairs_per_bundle, n_mtiles, rank);
+      const int nsteps = kDense ? a.steps_dense : a.step_ptr[c.bundle + 1] - a.step_ptr[c.bundle];
+      const uint32_t buf = j & 1u;
+      if (!mbar_wait(smem_u32(&bars->tmem_full[buf]), (j >> 1) & 1u, bars, err, 24)) break;
+      tc_fence_after();
+      const int nn = c.n0 + bn_i, to = c.t0 + bt_i, ho = c.h0 + bh_i, wo = c.w0 + bw_i;
+      const bool in_range = row < box_rows && nn < a.g.n && to < a.g.To && ho < a.g.Ho && wo < a.g.Wo;
+      const long long vox = (((long long)nn * a.g.To + to) * a.g.Ho + ho) * a.g.Wo + wo;
+      const int m_base = c.bundle * a.n_tile;
+      const uint32_t taddr = tmem_base + (uint32_t(quad * 32) << 16) + buf * uint32_t(a.n_tile);
+      epilogue_row(taddr, a.n_tile, nsteps > 0, in_range, bias_s, a.g.relu, yb + vox * a.g.ycs + m_base, m_base, a.g.M);
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(mapa_shared(smem_u32(&bars->tmem_empty[buf]), 0));
+    }
+  }
+
+  // ---------------------------------------------------------------------- teardown
+  if (bars->abort_flag) {
+    const long long t0 = clock64();
+    while (clock64() - t0 < 2000000ll) { }
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();              // the peer may still be signalling barriers in this CTA's shared memory
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(uint32_t(tmem_cols)) : "memory");
+  }
+}
+
+int pick_stages_pair(int n_tile) {
+  const size_t stage = kABytes + size_t(n_tile / 2) * 128;
+  const int s = int(kSmemBudget / stage);
+  return s > kMaxStages ? kMaxStages : s;
+}
+
+size_t pair_smem_bytes(int n_tile, int n_bundles) {
+  return size_t(pick_stages_pair(n_tile)) * (kABytes + size_t(n_tile / 2) * 128) + 1024 + sizeof(Barriers) +
+         size_t(n_tile) * n_bundles * 4;
+}
+
+template <bool kDense>
+cudaError_t launch_pair_t(const UmmaArgs& a, const CUtensorMap& xm, const CUtensorMap& wm, int sm_count, int stages,
+                          int cols, size_t smem, long long n_items, cudaStream_t stream) {
+  static bool attr_done = false;
+  if (!attr_done) {
+    cudaError_t e = cudaFuncSetAttribute(conv3d_umma_pair_kernel<kDense>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    if (e != cudaSuccess) return e;
+    attr_done = true;
+  }
+  cudaLaunchConfig_t cfg = {};
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  cfg.blockDim = dim3(kThreadsUmma);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  // as many CTA pairs as can be resident at once (persistent kernel), never more than items
+  static int max_clusters = 0;
+  if (max_clusters == 0) {
+    cfg.gridDim = dim3(unsigned(sm_count & ~1));
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, conv3d_umma_pair_kernel<kDense>, &cfg) != cudaSuccess || n <= 0) n = sm_count / 2;
+    max_clusters = n;
+  }
+  long long clusters = max_clusters < sm_count / 2 ? max_clusters : sm_count / 2;
+  if (clusters > n_items) clusters = n_items;
+  cfg.gridDim = dim3(unsigned(2 * clusters));
+  return cudaLaunchKernelEx(&cfg, conv3d_umma_pair_kernel<kDense>, xm, wm, a, stages, cols);
+}
+
+}  // namespace
+
+bool umma_pair_supported(int n_tile, int n_bundles) {
+  return n_tile % 32 == 0 && n_tile <= 256 && pick_stages_pair(n_tile) >= 2 && pair_smem_bytes(n_tile, n_bundles) <= 227 * 1024;
+}
+
+cudaError_t launch_conv_umma_pair(const UmmaArgs& a, const void* xmap, const void* wmap_half, int sm_count,
+                                  cudaStream_t stream) {
+  if (!umma_pair_supported(a.n_tile, a.n_bundles) || a.n_splits != 1) return cudaErrorInvalidValue;
+  const int stages = pick_stages_pair(a.n_tile);
+  const size_t smem = pair_smem_bytes(a.n_tile, a.n_bundles);
+  int cols = 32;
+  while (cols < 2 * a.n_tile) cols *= 2;
+  if (cols > 512) return cudaErrorInvalidValue;
+  const long long n_mtiles = (long long)a.tiles_n * a.tiles_t * a.tiles_h * a.tiles_w;
+  const long long n_items = ((n_mtiles + 1) / 2) * a.n_bundles;
+  if (n_items <= 0) return cudaSuccess;
+  CUtensorMap xm, wm;
+  memcpy(&xm, xmap, sizeof(CUtensorMap));
+  memcpy(&wm, wmap_half, sizeof(CUtensorMap));
+  return a.dense ? launch_pair_t<true>(a, xm, wm, sm_count, stages, cols, smem, n_items, stream)
+                 : launch_pair_t<false>(a, xm, wm, sm_count, stages, cols, smem, n_items, stream);
+}
+
+}  // namespace rt3d
