@@ -98,7 +98,8 @@ typedef struct {
  *   w     host, [M][N][Kt][Kh][Kw] float
  *   mask  host, same shape, uint8, nonzero = keep; NULL = keep everything.  The mask is
  *         authoritative: kept weights are stored even if zero, pruned ones dropped even if not.
- *   g_m, g_n  group size, 1..8 each;  Kt*Kh*Kw <= 65535
+ *   g_m, g_n  group size, 1..256 each (the paper prefers g_n = 4, g_m = 4 or 8; groups wider than 8
+ *             run on the tensor-core kernels only);  Kt*Kh*Kw <= 65535
  *   compute_dtype  storage/compute precision of the tiles (RT3D_F32, or RT3D_BF16 = RNE-rounded)
  *   out   receives the new handle
  * Errors: INVALID_ARG, MASK_NOT_GROUP_UNIFORM (mask is not a KGS mask), ALLOC.

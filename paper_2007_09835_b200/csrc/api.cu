@@ -219,23 +219,35 @@ TileBox choose_box(const ConvGeom& g) {
 // the issuing thread about 175 ns of barrier hand-shake plus 4 MMA issues, or the tensor time of the
 // step if that is longer; a layer with few output tiles runs as many serial steps per CTA as its
 // step list is long, so it is split along K (at the price of writing and re-reading fp32 partial
-// tiles) until the SMs are occupied; narrower bundles are the fallback when K is short.
+// tiles) until the SMs are occupied.  The step count of each candidate bundle width comes from the
+// handle's real step lists: with kernel groups as wide as a bundle, pruned (location, chunk) steps
+// vanish and a narrower bundle that matches the group height can win.
 struct UmmaPlan { int n_tile, n_splits; };
 
-UmmaPlan pick_plan(int M, long long m_tiles, int steps, int sm_count) {
+UmmaPlan pick_plan(rt3d_packed* w, long long m_tiles, int sm_count) {
+  const int M = w->M;
   const int widest = default_n_tile(M);
   UmmaPlan best{widest, 1};
   double best_ns = -1.0;
   static const int kSplits[] = {1, 2, 3, 4, 6, 8};
   for (int n = widest; n >= 32; n = (n > 128 ? 128 : n / 2)) {
     if (n % 16) break;
-    const long long items = m_tiles * ceil_div(M, n);
-    const double issue = 175.0 + 4.0 * (25.0 + 0.06 * n), tensor = 1.02 * n;
+    // narrower bundles only pay when they let pruned steps drop out (groups at least 16 rows high)
+    // or when the layer has too few tiles; for the paper's 4..8-row groups the lists are full anyway
+    const int bundles = ceil_div(M, n);
+    const long long items = m_tiles * bundles;
+    double steps = double(w->Ks) * ceil_div(w->N, kChunk);      // full lists: true for groups a few rows high
+    if (w->g_m >= 16 && !w->is_dense) {
+      const UmmaLayout* L = get_umma_layout(w, n);
+      if (!L) break;
+      steps = items < sm_count ? double(L->max_steps) : double(L->steps.size()) / bundles;
+    }
+    const double issue = 175.0 + 4.0 * (25.0 + 0.06 * n), tensor = 1.4 * n;
     const double step_ns = issue > tensor ? issue : tensor;
     for (int S : kSplits) {
       if (S > 1 && (steps / S < 8 || items >= 2LL * sm_count)) continue;
       const double waves = double(ceil_div64(items * S, sm_count));
-      double ns = waves * ceil_div(steps, S) * step_ns;
+      double ns = waves * (steps / S) * step_ns;
       // partial tile out (every split) and S partial tiles back in (the CTA that arrives last), plus the
       // traffic of all partials (written once, read once) at about 2.5 TB/s
       if (S > 1) ns += 3000.0 + (1.0 + S) * n * 4.0 + double(items) * S * (kTileM * n * 4.0 * 2.0) / 2500.0;
@@ -318,19 +330,9 @@ rt3d_status launch_smallc(rt3d_packed* w, DeviceBlob* blob, const DeviceState* d
   cuuint64_t strides[4] = {cs, cs * x->w, cs * x->w * x->h, cs * x->w * x->h * x->t};
   cuuint32_t bx[5] = {8, cuuint32_t(L->halo_w), cuuint32_t(L->halo_h), cuuint32_t(L->halo_t), 1};
   cuuint32_t estr[5] = {1, 1, 1, 1, 1};
-#if defined(RT3D_EXPERIMENT) && RT3D_EXPERIMENT == 5
-  cuuint64_t dims4[4] = {cuuint64_t(x->w) * 8, cuuint64_t(x->h), cuuint64_t(x->t), cuuint64_t(x->n)};
-  cuuint64_t strides4[3] = {cs * x->w, cs * x->w * x->h, cs * x->w * x->h * x->t};
-  cuuint32_t bx4[4] = {cuuint32_t(L->halo_w) * 8, cuuint32_t(L->halo_h), cuuint32_t(L->halo_t), 1};
-  (void)dims; (void)strides; (void)bx;
-  if (g_encode(&xmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, x->data, dims4, strides4, bx4, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-               CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-    return RT3D_ERR_CUDA;
-#else
   if (g_encode(&xmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, x->data, dims, strides, bx, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
     return RT3D_ERR_CUDA;
-#endif
   if (launch_conv_umma_smallc(a, &xmap, d->sm_count, st) != cudaSuccess) return RT3D_ERR_CUDA;
   g_launches.fetch_add(1);
   return RT3D_OK;
@@ -353,6 +355,9 @@ rt3d_status conv_impl(const rt3d_tensor* x, const rt3d_packed* wc, const float* 
   cudaStream_t st = static_cast<cudaStream_t>(stream);
 
   const bool can_umma = umma_eligible(d, w, x, y, p);
+  const bool can_simt = w->g_m <= kMaxGroupSimt && w->g_n <= kMaxGroupSimt;
+  if (!can_umma && !can_simt) return RT3D_ERR_UNSUPPORTED;
+  if (p->algo == RT3D_ALGO_SIMT && !can_simt) return RT3D_ERR_UNSUPPORTED;
   if ((p->algo == RT3D_ALGO_UMMA || p->algo == RT3D_ALGO_UMMA_PAIR) && !can_umma) return RT3D_ERR_UNSUPPORTED;
   const bool use_umma = p->algo == RT3D_ALGO_UMMA || p->algo == RT3D_ALGO_UMMA_PAIR ||
                         (p->algo == RT3D_ALGO_AUTO && can_umma);
@@ -374,7 +379,7 @@ rt3d_status conv_impl(const rt3d_tensor* x, const rt3d_packed* wc, const float* 
   a.tiles_n = ceil_div(g.n, a.box.bn); a.tiles_t = ceil_div(g.To, a.box.bt);
   a.tiles_h = ceil_div(g.Ho, a.box.bh); a.tiles_w = ceil_div(g.Wo, a.box.bw);
   const long long m_tiles = (long long)a.tiles_n * a.tiles_t * a.tiles_h * a.tiles_w;
-  UmmaPlan plan = pick_plan(w->M, m_tiles, w->Ks * ceil_div(w->N, kChunk), d->sm_count);
+  UmmaPlan plan = pick_plan(w, m_tiles, d->sm_count);
   // CTA pairs: two tiles per MMA.  Worth it when every pair has work; forced by RT3D_ALGO_UMMA_PAIR.
   bool use_pair = false;
   if (p->algo == RT3D_ALGO_UMMA_PAIR) {

@@ -12,7 +12,8 @@
 
 namespace rt3d {
 
-constexpr int kMaxGroup = 8;        // g_m, g_n <= 8
+constexpr int kMaxGroup = 256;      // g_m, g_n <= 256 (pack, tensor-core kernels)
+constexpr int kMaxGroupSimt = 8;    // the CUDA-core kernel keeps one group row in registers: g_m, g_n <= 8
 constexpr int kChunk = 64;          // input channels per tensor-core K step (one 128-byte swizzle row of bf16)
 constexpr int kTileM = 128;         // output voxels per tensor-core tile (TMEM lanes)
 

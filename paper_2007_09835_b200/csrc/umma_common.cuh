@@ -41,11 +41,7 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   asm volatile(
       "{\n"
       ".reg .pred p;\n"
-#if defined(RT3D_EXPERIMENT) && RT3D_EXPERIMENT == 6
-      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n"
-#else
       "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
-#endif
       "selp.u32 %0, 1, 0, p;\n"
       "}\n"
       : "=r"(ok) : "r"(bar), "r"(parity) : "memory");

@@ -70,6 +70,8 @@ __device__ __forceinline__ uint32_t instr_desc_bf16_pair(int n) {
   return (1u << 4) | (1u << 7) | (1u << 10) | (uint32_t(n >> 3) << 17) | (uint32_t(256 >> 4) << 24);
 }
 
+constexpr int kCps = 1;     // K chunks (of 64 channels) per pipeline stage (2 was measured: no gain)
+
 struct PairItem {
   int bundle;
   int n0, t0, h0, w0;     // first output voxel of this CTA's box (beyond the tensor for a dummy tile)
@@ -100,7 +102,8 @@ conv3d_umma_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_c
   const uint32_t tiles_base = (raw + 1023u) & ~1023u;
   const int n_half = a.n_tile / 2;
   const uint32_t b_bytes = uint32_t(n_half) * 128u;             // this CTA's half of the B tile
-  const uint32_t stage_bytes = kABytes + b_bytes;
+  const uint32_t chunk_bytes = kABytes + b_bytes;
+  const uint32_t stage_bytes = kCps * chunk_bytes;
   Barriers* bars = reinterpret_cast<Barriers*>(smem_raw + (tiles_base - raw) + size_t(stages) * stage_bytes);
   float* bias_s = reinterpret_cast<float*>(bars + 1);
   int32_t* err = a.sched + 2;
@@ -146,33 +149,42 @@ conv3d_umma_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_c
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
-      const uint32_t tx_both = 2u * (uint32_t(box_rows) * 128u + b_bytes);
+      const uint32_t tx_chunk_both = 2u * (uint32_t(box_rows) * 128u + b_bytes);
       for (int item = cluster_id; item < n_items && ok; item += n_clusters) {
         const PairItem c = decode_pair_item(a, item, pairs_per_bundle, n_mtiles, rank);
         const int s_begin = kDense ? c.bundle * a.steps_dense : a.step_ptr[c.bundle];
         const int nsteps = kDense ? a.steps_dense : a.step_ptr[c.bundle + 1] - s_begin;
         const int wq = c.w0 * a.g.sw - a.g.pw, hq = c.h0 * a.g.sh - a.g.ph, tq = c.t0 * a.g.st - a.g.pt;
         int kt = 0, kh = 0, kw = 0, ch = 0;
-        int enc_next = (!kDense && nsteps > 0) ? __ldg(a.steps + s_begin) : 0;
         int wrow = s_begin * a.n_tile + int(rank) * n_half;
-        for (int i = 0; i < nsteps; ++i, wrow += a.n_tile) {
-          int c_ch, c_w, c_h, c_t;
-          if (kDense) {
-            c_ch = ch * 64; c_w = wq + kw; c_h = hq + kh; c_t = tq + kt;
-            if (++ch == a.n_chunks) { ch = 0; if (++kw == a.g.Kw) { kw = 0; if (++kh == a.g.Kh) { kh = 0; ++kt; } } }
-          } else {
-            const int enc = enc_next;
-            if (i + 1 < nsteps) enc_next = __ldg(a.steps + s_begin + i + 1);
-            c_t = tq + ((enc >> 24) & 63); c_h = hq + ((enc >> 18) & 63); c_w = wq + ((enc >> 12) & 63);
-            c_ch = (enc & 4095) * 64;
+        for (int i = 0; i < nsteps; i += kCps) {
+          const int nload = nsteps - i < kCps ? nsteps - i : kCps;
+          int c_ch[kCps], c_w[kCps], c_h[kCps], c_t[kCps];
+#pragma unroll
+          for (int q = 0; q < kCps; ++q) {
+            if (q >= nload) break;
+            if (kDense) {
+              c_ch[q] = ch * 64; c_w[q] = wq + kw; c_h[q] = hq + kh; c_t[q] = tq + kt;
+              if (++ch == a.n_chunks) { ch = 0; if (++kw == a.g.Kw) { kw = 0; if (++kh == a.g.Kh) { kh = 0; ++kt; } } }
+            } else {
+              const int enc = __ldg(a.steps + s_begin + i + q);
+              c_t[q] = tq + ((enc >> 24) & 63); c_h[q] = hq + ((enc >> 18) & 63); c_w[q] = wq + ((enc >> 12) & 63);
+              c_ch[q] = (enc & 4095) * 64;
+            }
           }
           const uint32_t full_local = smem_u32(&bars->full[stage]);
           const uint32_t full_leader = mapa_shared(full_local, 0);
-          const uint32_t a_dst = tiles_base + stage * stage_bytes;
+          const uint32_t s_dst = tiles_base + stage * stage_bytes;
           if (!mbar_wait(smem_u32(&bars->empty[stage]), phase ^ 1u, bars, err, 21)) { ok = false; break; }
-          if (leader) mbar_expect_tx(full_local, tx_both);
-          tma_load_5d_pair(a_dst, &xmap, full_leader, c_ch, c_w, c_h, c_t, c.n0);
-          tma_load_2d_pair(a_dst + kABytes, &wmap_half, full_leader, 0, wrow);
+          if (leader) mbar_expect_tx(full_local, tx_chunk_both * uint32_t(nload));
+#pragma unroll
+          for (int q = 0; q < kCps; ++q) {
+            if (q >= nload) break;
+            const uint32_t a_dst = s_dst + q * chunk_bytes;
+            tma_load_5d_pair(a_dst, &xmap, full_leader, c_ch[q], c_w[q], c_h[q], c_t[q], c.n0);
+            tma_load_2d_pair(a_dst + kABytes, &wmap_half, full_leader, 0, wrow);
+            wrow += a.n_tile;
+          }
           if (++stage == stages) { stage = 0; phase ^= 1u; }
         }
       }
@@ -191,19 +203,24 @@ conv3d_umma_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_c
         if (!mbar_wait(smem_u32(&bars->tmem_empty[buf]), ((j >> 1) & 1u) ^ 1u, bars, err, 22)) break;
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + buf * uint32_t(a.n_tile);
-        for (int i = 0; i < nsteps; ++i) {
+        for (int i = 0; i < nsteps; i += kCps) {
+          const int nload = nsteps - i < kCps ? nsteps - i : kCps;
           if (!ready && !mbar_wait(smem_u32(&bars->full[stage]), phase, bars, err, 23)) { ok = false; break; }
           // poll the next stage's barrier now: its answer arrives while this stage's MMAs are issued
           const int stage_n = stage + 1 == stages ? 0 : stage + 1;
           const uint32_t phase_n = stage + 1 == stages ? phase ^ 1u : phase;
           ready = mbar_try_wait(smem_u32(&bars->full[stage_n]), phase_n);
           tc_fence_after();
-          const uint32_t a_addr = tiles_base + stage * stage_bytes;
-          const uint64_t adesc = smem_desc_sw128(a_addr);
-          const uint64_t bdesc = smem_desc_sw128(a_addr + kABytes);
 #pragma unroll
-          for (int kk = 0; kk < 4; ++kk)
-            umma_bf16_pair(d_tmem, adesc + 2 * kk, bdesc + 2 * kk, idesc, (i | kk) ? 1u : 0u);
+          for (int q = 0; q < kCps; ++q) {
+            if (q >= nload) break;
+            const uint32_t a_addr = tiles_base + stage * stage_bytes + q * chunk_bytes;
+            const uint64_t adesc = smem_desc_sw128(a_addr);
+            const uint64_t bdesc = smem_desc_sw128(a_addr + kABytes);
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk)
+              umma_bf16_pair(d_tmem, adesc + 2 * kk, bdesc + 2 * kk, idesc, (i | q | kk) ? 1u : 0u);
+          }
           umma_commit_pair(smem_u32(&bars->empty[stage]));
           stage = stage_n; phase = phase_n;
         }
@@ -255,13 +272,13 @@ conv3d_umma_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_c
 }
 
 int pick_stages_pair(int n_tile) {
-  const size_t stage = kABytes + size_t(n_tile / 2) * 128;
+  const size_t stage = kCps * (kABytes + size_t(n_tile / 2) * 128);
   const int s = int(kSmemBudget / stage);
   return s > kMaxStages ? kMaxStages : s;
 }
 
 size_t pair_smem_bytes(int n_tile, int n_bundles) {
-  return size_t(pick_stages_pair(n_tile)) * (kABytes + size_t(n_tile / 2) * 128) + 1024 + sizeof(Barriers) +
+  return size_t(pick_stages_pair(n_tile)) * kCps * (kABytes + size_t(n_tile / 2) * 128) + 1024 + sizeof(Barriers) +
          size_t(n_tile) * n_bundles * 4;
 }
 

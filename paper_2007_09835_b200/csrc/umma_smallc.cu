@@ -87,13 +87,8 @@ conv3d_umma_smallc_kernel(const __grid_constant__ CUtensorMap xmap, const SmallC
         if (!mbar_wait(smem_u32(&bars->empty[stage]), phase ^ 1u, bars, err, 11)) break;
         const uint32_t full = smem_u32(&bars->full[stage]);
         mbar_expect_tx(full, uint32_t(a.halo_bytes));
-#if defined(RT3D_EXPERIMENT) && RT3D_EXPERIMENT == 5
-        tma_load_4d(halo_smem + stage * halo_stride, &xmap, full, (iw * kSmallCTileW - a.g.pw) * 8,
-                    ih * kSmallCTileH - a.g.ph, to - a.g.pt, nn);
-#else
         tma_load_5d(halo_smem + stage * halo_stride, &xmap, full, 0, iw * kSmallCTileW - a.g.pw,
                     ih * kSmallCTileH - a.g.ph, to - a.g.pt, nn);
-#endif
         if (++stage == kSmallCStages) { stage = 0; phase ^= 1u; }
       }
     }

@@ -178,6 +178,27 @@ def test_umma_pair_kernel_against_oracle(case, dense):
     assert np.abs(y1 - y).max() <= 1e-2 * np.abs(ref).max()
 
 
+WIDE_GROUP_CASES = [
+    # kernel groups matched to the tensor-core footprint (beyond the paper's 4..8): exact step skipping
+    (256, 256, (3, 3, 3), (2, 8, 14, 14), 256, 64, 0.25),
+    (256, 256, (3, 3, 3), (2, 8, 14, 14), 128, 64, 0.25),
+    (128, 256, (3, 3, 3), (4, 8, 14, 14), 64, 64, 0.5),
+    (192, 160, (1, 3, 3), (2, 4, 14, 14), 32, 16, 0.3),
+    (256, 256, (3, 3, 3), (1, 2, 7, 7), 256, 64, 0.125),       # few tiles: K split over short lists
+]
+
+
+@pytest.mark.parametrize("case", WIDE_GROUP_CASES)
+def test_wide_kernel_groups_against_oracle(case):
+    cin, cout, k, (n, t, h, w), g_m, g_n, d = case
+    spec = synth.ConvSpec("g", cin, cout, k, (1, 1, 1), tuple(kk // 2 for kk in k), True)
+    y, ref, lay, xd, yt = run_case(spec, n, t, h, w, g_m, g_n, "bernoulli", d, torch.bfloat16, rt3d.ALGO_AUTO)
+    check(y, ref, torch.bfloat16, f"wide groups {case}")
+    with pytest.raises(rt3d.Rt3dError) as e:               # the CUDA-core kernel stops at 8 x 8 groups
+        lay(xd, algo=rt3d.ALGO_SIMT)
+    assert e.value.status == rt3d.ERR_UNSUPPORTED
+
+
 SPLITK_CASES = [
     # few output tiles, long K: the tensor-core kernel splits K across CTAs and reduces fp32 partials
     (256, 256, (3, 3, 3), (1, 1, 1), (1, 1, 1), (1, 2, 7, 7), 4, 4, 0.4),

@@ -14,7 +14,8 @@ def _layer(M, N, k, g_m, g_n, density, seed):
 
 
 @pytest.mark.parametrize("M,N,k,g_m,g_n", [(32, 16, (3, 3, 3), 4, 4), (6, 5, (3, 3, 3), 4, 4), (64, 64, (3, 3, 3), 8, 4),
-                                           (45, 3, (1, 7, 7), 4, 4), (40, 24, (3, 1, 1), 8, 8), (7, 9, (2, 2, 1), 3, 2)])
+                                           (45, 3, (1, 7, 7), 4, 4), (40, 24, (3, 1, 1), 8, 8), (7, 9, (2, 2, 1), 3, 2),
+                                           (128, 128, (3, 3, 3), 64, 64), (200, 70, (1, 3, 3), 128, 16)])
 @pytest.mark.parametrize("dtype", [rt3d.RT3D_F32, rt3d.RT3D_BF16])
 def test_pack_bit_exact_against_oracle(M, N, k, g_m, g_n, dtype):
     L = _layer(M, N, k, g_m, g_n, 0.4, M + N)
@@ -49,7 +50,7 @@ def test_pack_errors():
     with pytest.raises(rt3d.Rt3dError) as e:
         rt3d.rt3d_pack_kgs(L["w"], bad, 4, 4, rt3d.RT3D_F32)
     assert e.value.status == rt3d.ERR_MASK_NOT_GROUP_UNIFORM
-    for g_m, g_n, dt in ((0, 4, 0), (4, 9, 0), (4, 4, 7)):
+    for g_m, g_n, dt in ((0, 4, 0), (4, 257, 0), (4, 4, 7)):
         with pytest.raises(rt3d.Rt3dError) as e:
             rt3d.rt3d_pack_kgs(L["w"], None, g_m, g_n, dt)
         assert e.value.status == rt3d.ERR_INVALID_ARG
@@ -67,13 +68,23 @@ def test_unpack_roundtrip(dtype):
 
 @pytest.mark.parametrize("M,N,k,g_m,g_n,n_tile", [(256, 128, (3, 3, 3), 4, 4, 0), (256, 128, (3, 3, 3), 4, 4, 64),
                                                   (45, 3, (1, 7, 7), 4, 4, 0), (144, 64, (1, 3, 3), 8, 4, 0),
-                                                  (64, 230, (3, 1, 1), 8, 8, 32), (512, 70, (1, 1, 1), 4, 4, 0)])
+                                                  (64, 230, (3, 1, 1), 8, 8, 32), (512, 70, (1, 1, 1), 4, 4, 0),
+                                                  (256, 128, (3, 3, 3), 64, 64, 64), (256, 256, (3, 3, 3), 256, 64, 0)])
 def test_tensor_core_layout_holds_exactly_the_masked_weights(M, N, k, g_m, g_n, n_tile):
     L = _layer(M, N, k, g_m, g_n, 0.3, 11)
     pk = rt3d.rt3d_pack_kgs(L["w"], L["mask"], g_m, g_n, rt3d.RT3D_BF16)
     np.testing.assert_array_equal(pk.unpack_device_layout(n_tile), oracle.bf16_round(L["w"] * L["mask"]))
     with pytest.raises(rt3d.Rt3dError):
         rt3d.rt3d_pack_kgs(L["w"], L["mask"], g_m, g_n, rt3d.RT3D_F32).unpack_device_layout(n_tile)
+
+
+def test_wide_groups_drop_whole_steps_from_the_layout():
+    # groups as wide as a bundle and as deep as a chunk: a pruned (location, chunk) is not a step at all
+    spec = synth.ConvSpec("t", 256, 256, (3, 3, 3), (1, 1, 1), (1, 1, 1))
+    L = synth.make_layer(spec, 9, 2, 256, 64, "exact_total", (1 * 4 * 27) // 4)
+    pk = rt3d.rt3d_pack_kgs(L["w"], L["mask"], 256, 64, rt3d.RT3D_BF16)
+    assert pk.view()["nnz"] == 27
+    np.testing.assert_array_equal(pk.unpack_device_layout(256), oracle.bf16_round(L["w"] * L["mask"]))
 
 
 def test_vanilla_high_rate_skips_steps_in_layout():
