@@ -37,6 +37,9 @@ import rt3d_synth as synth
 CFG = dict(n=8, t=8, h=28, w=28, cin=128, cout=256, k=(3, 3, 3), stride=(1, 1, 1), pad=(1, 1, 1),
            g_m=4, g_n=4, density=0.4)
 L2_BYTES = 126 * 1024 * 1024
+# DRAM bytes (read + write) of one launch of the timed kernel on this workload, from the ncu capture
+# summarised in profiles/conv3d_umma_pair_cfg1.md (14.65 MB read + 0.06 MB written; the output stays in L2).
+DRAM_TRAFFIC_PER_LAUNCH = 14.71e6
 WORKLOAD = "cfg1: C3D conv3a-shaped layer, batch 8, 128->256, 8x28x28, 3x3x3 s1 p1, KGS 4x4 ~2.5x, bf16"
 
 
@@ -318,7 +321,7 @@ def main():
                 "d2h_bytes_per_step": yh.numel() * 2},
         "gpu_launches": int(launches),
         "roofline": {"bound": "tensor", "achieved": ach, "peak": pk["bf16_tflops"], "unit": "TFLOP/s",
-                     "frac": ach / pk["bf16_tflops"], "traffic": None, "peak_source": pk["source"] + " (burst)",
+                     "frac": ach / pk["bf16_tflops"], "traffic": DRAM_TRAFFIC_PER_LAUNCH if algo == rt3d.ALGO_UMMA else None, "peak_source": pk["source"] + " (burst)",
                      "executed_tflops": 2.0 * dense_macs / (per_step_ms * 1e-3) / 1e12,
                      "alg_bytes_per_launch": alg_bytes},
     }
@@ -331,12 +334,6 @@ def main():
         out["cpu_baseline"] = {"value": flops_kept / dt / 1e12, "unit": "TFLOP/s", "cores": oracle.threads(),
                                "kind": "oracle", "seconds": dt,
                                "sample": f"all {clips} clips of one batch, one pass (masked dense weights, fp64 accumulation)"}
-    traffic_file = os.path.join(ROOT, "profiles", "traffic.json")
-    if os.path.exists(traffic_file):
-        try:
-            out["roofline"]["traffic"] = json.load(open(traffic_file)).get("cfg1_sparse_dram_bytes_per_launch")
-        except Exception:
-            pass
     if rank == 0:
         print(json.dumps(out))
     dist.shutdown(group)
