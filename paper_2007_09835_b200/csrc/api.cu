@@ -282,25 +282,28 @@ rt3d_status encode_xmap(const rt3d_tensor* x, const ConvGeom& g, const TileBox& 
   return r == CUDA_SUCCESS ? RT3D_OK : RT3D_ERR_CUDA;
 }
 
-// Small-C_in kernel: bf16, C_in <= 8 stored at pitch 8, stride 1, M <= 256.
+// Small-C_in kernel: bf16, C_in <= 8 stored at pitch 8, spatial strides <= 4, M <= 256.
 bool smallc_eligible(const DeviceState* d, rt3d_packed* w, const rt3d_tensor* x, const rt3d_tensor* y,
                      const rt3d_conv_params* p, const SmallCLayout** out) {
   if (d->cc_major != 10 || w->dtype != RT3D_BF16) return false;
   if (x->c > 8 || x->c_stride != 8 || y->c_stride % 8) return false;
-  if (p->st != 1 || p->sh != 1 || p->sw != 1) return false;
+  if (p->st > 8 || p->sh > 4 || p->sw > 4) return false;
   if (w->Kt > 16 || w->Kh > 32 || w->Kw > 32) return false;
-  const SmallCLayout* L = get_smallc_layout(w);
+  const SmallCLayout* L = get_smallc_layout(w, p->sh, p->sw);
   if (!L) return false;
-  if (smallc_smem_bytes(L->n_pairs, L->n_pad, L->halo_w * L->halo_h * L->halo_t * 16) > 227 * 1024) return false;
+  if (L->img_w * p->sw > 256 || L->img_h * p->sh > 256) return false;
+  if (smallc_smem_bytes(L->n_pairs, L->n_pad, L->n_phases * L->phase_stride) > 227 * 1024) return false;
   *out = L;
   return true;
 }
 
 rt3d_status launch_smallc(rt3d_packed* w, DeviceBlob* blob, const DeviceState* d, const SmallCLayout* L,
                           const rt3d_tensor* x, const ConvGeom& g, const float* bias, rt3d_tensor* y, cudaStream_t st) {
+  DeviceBlob::SmallC* sc = nullptr;
   {
     std::lock_guard<std::mutex> lock(w->mu);
-    if (!blob->smallc_wimg) {
+    sc = &blob->smallc[L->sh * 16 + L->sw];
+    if (!sc->wimg) {
       void* wi = nullptr;
       int32_t* po = nullptr;
       if (cudaMalloc(&wi, L->wimg.size() * 2 + 16) != cudaSuccess ||
@@ -310,26 +313,27 @@ rt3d_status launch_smallc(rt3d_packed* w, DeviceBlob* blob, const DeviceState* d
           (!L->pair_off.empty() &&
            cudaMemcpy(po, L->pair_off.data(), L->pair_off.size() * 4, cudaMemcpyHostToDevice) != cudaSuccess))
         return RT3D_ERR_CUDA;
-      blob->smallc_pairs = po;
-      blob->smallc_wimg = wi;
+      sc->pairs = po;
+      sc->wimg = wi;
     }
   }
   SmallCArgs a;
   a.g = g;
   a.n_pad = L->n_pad; a.n_pairs = L->n_pairs;
-  a.halo_w = L->halo_w; a.halo_h = L->halo_h; a.halo_t = L->halo_t;
-  a.halo_bytes = L->halo_w * L->halo_h * L->halo_t * 16;
+  a.n_phases = L->n_phases; a.phase_stride = L->phase_stride;
+  a.img_w = L->img_w; a.phase_bytes = L->img_w * L->img_h * L->img_t * 16;
   a.tiles_h = ceil_div(g.Ho, kSmallCTileH); a.tiles_w = ceil_div(g.Wo, kSmallCTileW);
   a.tmem_cols = 0;
-  a.wimg = blob->smallc_wimg; a.pair_off = blob->smallc_pairs;
+  a.wimg = sc->wimg; a.pair_off = sc->pairs;
   a.bias = bias; a.y = y->data; a.sched = d->sched;
-  // input as [n][t][h][w][8]: box = the halo of one 1 x 16 x 8 output tile, no swizzle
+  // input as [n][t][h][w][8]: one box = one phase image of a 1 x 16 x 8 output tile (every sh-th row and
+  // sw-th column: a traversal stride s loads ceil(box / s) elements), no swizzle
   CUtensorMap xmap;
   const cuuint64_t cs = 16;
   cuuint64_t dims[5] = {cuuint64_t(x->c), cuuint64_t(x->w), cuuint64_t(x->h), cuuint64_t(x->t), cuuint64_t(x->n)};
   cuuint64_t strides[4] = {cs, cs * x->w, cs * x->w * x->h, cs * x->w * x->h * x->t};
-  cuuint32_t bx[5] = {8, cuuint32_t(L->halo_w), cuuint32_t(L->halo_h), cuuint32_t(L->halo_t), 1};
-  cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+  cuuint32_t bx[5] = {8, cuuint32_t(L->img_w * g.sw), cuuint32_t(L->img_h * g.sh), cuuint32_t(L->img_t), 1};
+  cuuint32_t estr[5] = {1, cuuint32_t(g.sw), cuuint32_t(g.sh), 1, 1};
   if (g_encode(&xmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, x->data, dims, strides, bx, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
     return RT3D_ERR_CUDA;
@@ -509,7 +513,7 @@ void rt3d_packed_free(rt3d_packed* p) {
     cudaFree(b->group_ptr); cudaFree(b->pos_idx); cudaFree(b->tiles);
     for (auto& kv : b->umma) { cudaFree(kv.second.wtiles); cudaFree(kv.second.step_ptr); cudaFree(kv.second.steps); }
     cudaFree(b->stage_x); cudaFree(b->stage_y); cudaFree(b->stage_bias);
-    cudaFree(b->smallc_wimg); cudaFree(b->smallc_pairs);
+    for (auto& kv : b->smallc) { cudaFree(kv.second.wimg); cudaFree(kv.second.pairs); }
     cudaFree(b->splitk); cudaFree(b->splitk_cnt);
     delete b;
   }

@@ -61,21 +61,22 @@ bool umma_pair_supported(int n_tile, int n_bundles);
 cudaError_t launch_conv_umma_pair(const UmmaArgs& a, const void* xmap, const void* wmap_half, int sm_count,
                                   cudaStream_t stream);
 
-// Arguments of the small-C_in tensor-core kernel (C_in <= 8 at channel pitch 8, stride 1).
+// Arguments of the small-C_in tensor-core kernel (C_in <= 8 at channel pitch 8).
 struct SmallCArgs {
   ConvGeom g;
   int n_pad, n_pairs;                 // padded output channels; pairs of kept kernel locations
-  int halo_w, halo_h, halo_t, halo_bytes;
+  int n_phases, phase_stride;         // sh*sw phase images per tile, bytes between them in shared memory
+  int img_w, phase_bytes;             // voxels per image row; bytes one phase load delivers
   int tiles_h, tiles_w;               // 16 x 8 output tiles per frame
   int tmem_cols;                      // filled in by the launcher
   const void* wimg;                   // device: [n_pairs][2][n_pad/8][8][8] bf16
-  const int32_t* pair_off;            // device: [n_pairs][2] byte offsets inside the staged halo
+  const int32_t* pair_off;            // device: [n_pairs][2] byte offsets inside the staged images
   const float* bias;
   void* y;
   int32_t* sched;
 };
 cudaError_t launch_conv_umma_smallc(const SmallCArgs& a, const void* xmap, int sm_count, cudaStream_t stream);
-size_t smallc_smem_bytes(int n_pairs, int n_pad, int halo_bytes);
+size_t smallc_smem_bytes(int n_pairs, int n_pad, int stage_bytes);
 
 // Shared memory the tcgen05 kernel needs for a bundle width (for the host-side eligibility check).
 size_t umma_smem_bytes(int n_tile, int n_bundles);

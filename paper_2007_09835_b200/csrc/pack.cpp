@@ -1,8 +1,10 @@
 // Host-side weight reorganisation: the KGS pack (Section 3 / Section 5.2 of the paper), its
 // inverse, and the derivation of the tensor-core weight layout from the canonical arrays.
 // Pure host code: no CUDA calls, usable without a GPU.
+#include <algorithm>
 #include <cstring>
 #include <new>
+#include <utility>
 
 #include "rt3d_internal.h"
 
@@ -101,32 +103,41 @@ const UmmaLayout* get_umma_layout(rt3d_packed* p, int n_tile) {
   return &res.first->second;
 }
 
-// Small-C_in layout: kernel locations kept by at least one group are listed in ascending order and
-// paired; each pair is one K=16 MMA whose two K halves are the 8 (padded) channels at the two
-// locations.  Operands use the no-swizzle core-matrix layout (8 rows x 16 bytes).
-const SmallCLayout* get_smallc_layout(rt3d_packed* p) {
-  if (p->dtype != RT3D_BF16 || p->N > 8 || p->M > 256) return nullptr;
+// Small-C_in layout for spatial strides (sh, sw): kernel locations kept by at least one group are
+// sorted by the offset of their window inside the staged phase images and paired; each pair is one
+// K=16 MMA whose two K halves are the 8 (padded) channels at the two locations.  Operands use the
+// no-swizzle core-matrix layout (8 rows x 16 bytes).
+const SmallCLayout* get_smallc_layout(rt3d_packed* p, int sh, int sw) {
+  if (p->dtype != RT3D_BF16 || p->N > 8 || p->M > 256 || sh < 1 || sw < 1 || sh > 4 || sw > 4) return nullptr;
   std::lock_guard<std::mutex> lock(p->mu);
-  if (p->smallc_built) return &p->smallc;
-  SmallCLayout& L = p->smallc;
+  const int key = sh * 16 + sw;
+  auto it = p->smallc_layouts.find(key);
+  if (it != p->smallc_layouts.end()) return &it->second;
+  SmallCLayout L;
+  L.sh = sh; L.sw = sw;
   L.n_pad = round_up(p->M, 16);
-  L.halo_w = kSmallCTileW + p->Kw - 1;
-  L.halo_h = kSmallCTileH + p->Kh - 1;
-  L.halo_t = p->Kt;
+  L.n_phases = sh * sw;
+  L.img_w = kSmallCTileW - 1 + ceil_div(p->Kw, sw);
+  L.img_h = kSmallCTileH - 1 + ceil_div(p->Kh, sh);
+  L.img_t = p->Kt;
+  L.phase_stride = round_up(L.img_w * L.img_h * L.img_t * 16, 128);   // a TMA box must land on a 128-byte boundary
   std::vector<uint8_t> used(size_t(p->Ks), 0);
   for (int64_t e = 0; e < p->nnz; ++e) used[p->pos_idx[size_t(e)]] = 1;
-  std::vector<int> pos;
-  for (int k = 0; k < p->Ks; ++k)
-    if (used[size_t(k)]) pos.push_back(k);
+  std::vector<std::pair<int, int>> pos;            // (window offset, kernel location)
+  for (int k = 0; k < p->Ks; ++k) {
+    if (!used[size_t(k)]) continue;
+    const int kw = k % p->Kw, kh = (k / p->Kw) % p->Kh, kt = k / (p->Kw * p->Kh);
+    const int phase = (kh % sh) * sw + (kw % sw);
+    pos.emplace_back(phase * L.phase_stride + ((kt * L.img_h + kh / sh) * L.img_w + kw / sw) * 16, k);
+  }
+  std::sort(pos.begin(), pos.end());
   L.n_pairs = ceil_div(int(pos.size()), 2);
   L.pair_off.assign(size_t(L.n_pairs) * 2, 0);
   L.wimg.assign(size_t(L.n_pairs) * 2 * L.n_pad * 8, 0);
   std::vector<int> slot(size_t(p->Ks), -1);       // location -> pair*2 + half
   for (size_t i = 0; i < pos.size(); ++i) {
-    const int k = pos[i];
-    const int kw = k % p->Kw, kh = (k / p->Kw) % p->Kh, kt = k / (p->Kw * p->Kh);
-    L.pair_off[i] = ((kt * L.halo_h + kh) * L.halo_w + kw) * 16;
-    slot[size_t(k)] = int(i);
+    L.pair_off[i] = pos[i].first;
+    slot[size_t(pos[i].second)] = int(i);
   }
   if (pos.size() % 2) L.pair_off[pos.size()] = L.pair_off[pos.size() - 1] + 16;   // unused half: zero weights
   const uint16_t* tiles = reinterpret_cast<const uint16_t*>(p->tiles.data());
@@ -141,8 +152,8 @@ const SmallCLayout* get_smallc_layout(rt3d_packed* p) {
                 tiles[(size_t(e) * p->g_m + i) * p->g_n + j];
           }
       }
-  p->smallc_built = true;
-  return &L;
+  auto res = p->smallc_layouts.emplace(key, std::move(L));
+  return &res.first->second;
 }
 
 static rt3d_status pack_impl(const float* w, const uint8_t* mask, int M, int N, int Kt, int Kh, int Kw,

@@ -45,13 +45,19 @@ struct UmmaLayout {
   int max_steps = 0;                 // longest bundle list
 };
 
-// Layout for the small-C_in tensor-core kernel (C_in <= 8, channel pitch 8): the K dimension is
-// walked in pairs of kernel locations (8 padded channels each), one K=16 MMA per pair.
+// Layout for the small-C_in tensor-core kernel (C_in <= 8, channel pitch 8) at spatial strides
+// (sh, sw): the input under a 1x16x8 output tile is staged as sh*sw phase images (every sh-th row and
+// sw-th column), so that consecutive outputs are consecutive voxels of an image and every kernel
+// location is a shifted window of one image.  K is walked in pairs of kernel locations (8 padded
+// channels each), one K=16 MMA per pair.
 struct SmallCLayout {
+  int sh = 1, sw = 1;
   int n_pad = 0;                     // output channels rounded up to 16 (<= 256)
   int n_pairs = 0;
-  int halo_w = 0, halo_h = 0, halo_t = 0;   // input voxels staged per 1x16x8 output tile
-  std::vector<int32_t> pair_off;     // [n_pairs][2] byte offset of each location inside the staged halo
+  int n_phases = 1;                  // sh * sw
+  int img_w = 0, img_h = 0, img_t = 0;   // voxels of one phase image
+  int phase_stride = 0;              // bytes between phase images in shared memory
+  std::vector<int32_t> pair_off;     // [n_pairs][2] byte offset of each location's window inside the staged images
   std::vector<uint16_t> wimg;        // [n_pairs][2][n_pad/8][8][8] bf16 bits, zero where pruned / absent
 };
 
@@ -70,8 +76,8 @@ struct DeviceBlob {
     bool ready = false;
   };
   std::map<int, Umma> umma;          // keyed by n_tile
-  void* smallc_wimg = nullptr;       // small-C_in kernel: weight image and location-pair offsets
-  int32_t* smallc_pairs = nullptr;
+  struct SmallC { void* wimg = nullptr; int32_t* pairs = nullptr; };
+  std::map<int, SmallC> smallc;      // small-C_in kernel: weight image and pair offsets, keyed by sh*16+sw
   float* splitk = nullptr; size_t splitk_bytes = 0;            // split-K partial tiles (grown on demand)
   int32_t* splitk_cnt = nullptr; size_t splitk_cnt_bytes = 0;  // split-K arrival counters, zero between launches
   void* stage_x = nullptr; size_t stage_x_bytes = 0;   // staging for rt3d_conv3d_host
@@ -90,8 +96,7 @@ struct rt3d_packed {
   std::vector<unsigned char> tiles;  // nnz * g_m * g_n elements of float or bf16 bits
   std::mutex mu;                     // guards the lazily built members below
   std::map<int, rt3d::UmmaLayout> umma_layouts;   // keyed by n_tile
-  rt3d::SmallCLayout smallc;         // built on first use
-  bool smallc_built = false;
+  std::map<int, rt3d::SmallCLayout> smallc_layouts;   // keyed by sh*16+sw, built on first use
   std::vector<rt3d::DeviceBlob*> blobs;
 };
 
@@ -103,6 +108,6 @@ int default_n_tile(int M);
 const UmmaLayout* get_umma_layout(rt3d_packed* p, int n_tile);
 bool umma_layout_possible(const rt3d_packed* p);
 // Small-C_in layout (nullptr if the handle does not qualify: needs bf16, N <= 8, M <= 256).
-const SmallCLayout* get_smallc_layout(rt3d_packed* p);
+const SmallCLayout* get_smallc_layout(rt3d_packed* p, int sh, int sw);
 
 }  // namespace rt3d

@@ -1,5 +1,6 @@
 // Tensor-core convolution for layers with very few input channels (C_in <= 8 stored at a channel
-// pitch of 8, e.g. the RGB first layer of the C3D-shaped network), stride 1.
+// pitch of 8, e.g. the RGB first layers of the C3D- and R(2+1)D-shaped networks), any temporal
+// stride, spatial strides up to 4.
 //
 // With 16 bytes per voxel the input halo of an output tile of 1 x 16 x 8 voxels can be staged in
 // shared memory exactly as it lies in global memory, [t][h][w][8 channels], by one TMA box whose
@@ -10,6 +11,8 @@
 // kernel locations (leading byte offset = distance between the two shifted windows).  So each pair
 // of kept kernel locations is one MMA, the input is read from L2 once per tile, and the layer is
 // bound by writing its output.  Kernel locations that no group keeps are not in the pair list.
+// With a spatial stride the input is staged as one image per stride phase (strided TMA boxes), so
+// that consecutive outputs are again consecutive voxels and every location a window of one image.
 //
 // Roles as in the main kernel: warp 0 TMA producer, warp 1 MMA issuer / TMEM owner, warps 2..5
 // epilogue; bounded mbarrier waits.
@@ -30,7 +33,7 @@ conv3d_umma_smallc_kernel(const __grid_constant__ CUtensorMap xmap, const SmallC
   const uint32_t w_bytes = uint32_t(a.n_pairs) * 2u * uint32_t(a.n_pad) * 16u;
   const uint32_t w_smem = base;                                         // weight image, whole layer
   const uint32_t halo_smem = base + ((w_bytes + 127u) & ~127u);         // ring of staged halos
-  const uint32_t halo_stride = (uint32_t(a.halo_bytes) + 127u) & ~127u;
+  const uint32_t halo_stride = (uint32_t(a.n_phases * a.phase_stride) + 127u) & ~127u;
   unsigned char* gen = smem_raw + (base - raw);
   int32_t* pair_smem = reinterpret_cast<int32_t*>(gen + (halo_smem - base) + kSmallCStages * halo_stride);
   Barriers* bars = reinterpret_cast<Barriers*>(reinterpret_cast<unsigned char*>(pair_smem) +
@@ -86,16 +89,18 @@ conv3d_umma_smallc_kernel(const __grid_constant__ CUtensorMap xmap, const SmallC
         const int nn = r / a.g.To;
         if (!mbar_wait(smem_u32(&bars->empty[stage]), phase ^ 1u, bars, err, 11)) break;
         const uint32_t full = smem_u32(&bars->full[stage]);
-        mbar_expect_tx(full, uint32_t(a.halo_bytes));
-        tma_load_5d(halo_smem + stage * halo_stride, &xmap, full, 0, iw * kSmallCTileW - a.g.pw,
-                    ih * kSmallCTileH - a.g.ph, to - a.g.pt, nn);
+        mbar_expect_tx(full, uint32_t(a.n_phases * a.phase_bytes));
+        const int w0 = iw * kSmallCTileW * a.g.sw - a.g.pw, h0 = ih * kSmallCTileH * a.g.sh - a.g.ph;
+        for (int ph = 0; ph < a.n_phases; ++ph)      // one strided box per (row, column) stride phase
+          tma_load_5d(halo_smem + stage * halo_stride + ph * a.phase_stride, &xmap, full, 0, w0 + ph % a.g.sw,
+                      h0 + ph / a.g.sw, to * a.g.st - a.g.pt, nn);
         if (++stage == kSmallCStages) { stage = 0; phase ^= 1u; }
       }
     }
   } else if (warp == 1) {
     if (lane == 0) {
       const uint32_t idesc = instr_desc_bf16(a.n_pad);
-      const uint32_t sbo_a = uint32_t(a.halo_w) * 16u;            // next 8-voxel group = next halo row
+      const uint32_t sbo_a = uint32_t(a.img_w) * 16u;             // next 8-voxel group = next image row
       const uint32_t lbo_b = uint32_t(a.n_pad) * 16u;             // second K half of the weight image
       int stage = 0;
       uint32_t phase = 0, j = 0;
@@ -158,9 +163,9 @@ conv3d_umma_smallc_kernel(const __grid_constant__ CUtensorMap xmap, const SmallC
 
 }  // namespace
 
-size_t smallc_smem_bytes(int n_pairs, int n_pad, int halo_bytes) {
+size_t smallc_smem_bytes(int n_pairs, int n_pad, int stage_bytes) {
   const size_t w = (size_t(n_pairs) * 2 * n_pad * 16 + 127) & ~size_t(127);
-  const size_t halo = (size_t(halo_bytes) + 127) & ~size_t(127);
+  const size_t halo = (size_t(stage_bytes) + 127) & ~size_t(127);
   return 128 + w + kSmallCStages * halo + ((size_t(n_pairs) * 8 + 15) & ~size_t(15)) + sizeof(Barriers) + size_t(n_pad) * 4;
 }
 
@@ -170,7 +175,7 @@ cudaError_t launch_conv_umma_smallc(const SmallCArgs& a_in, const void* xmap, in
   while (cols < 2 * a.n_pad) cols *= 2;
   if (cols > 512) return cudaErrorInvalidValue;
   a.tmem_cols = cols;
-  const size_t smem = smallc_smem_bytes(a.n_pairs, a.n_pad, a.halo_bytes);
+  const size_t smem = smallc_smem_bytes(a.n_pairs, a.n_pad, a.n_phases * a.phase_stride);
   if (smem > 227 * 1024) return cudaErrorInvalidValue;
   const long long n_items = (long long)a.g.n * a.g.To * a.tiles_h * a.tiles_w;
   if (n_items <= 0) return cudaSuccess;

@@ -108,6 +108,10 @@ SMALLC_CASES = [
     (1, 16, (3, 1, 1), (1, 1, 1), (1, 0, 0), (1, 6, 9, 9), 4, 4, 0.7),
     (5, 256, (2, 2, 2), (1, 1, 1), (0, 0, 0), (1, 4, 18, 10), 8, 4, 0.5),    # no padding, even kernel
     (3, 32, (3, 3, 3), (1, 1, 1), (0, 1, 2), (1, 5, 17, 9), 4, 4, 0.05),     # very sparse: few pairs
+    (3, 45, (1, 7, 7), (1, 2, 2), (0, 3, 3), (2, 3, 56, 40), 4, 4, 0.4),     # R(2+1)D stem: 4 stride phases
+    (3, 64, (3, 3, 3), (2, 2, 2), (1, 1, 1), (1, 7, 35, 21), 4, 4, 0.6),     # strided in t, h and w, ragged
+    (8, 32, (3, 5, 3), (1, 3, 1), (1, 2, 1), (1, 3, 50, 12), 8, 8, 0.5),     # stride 3 along h only
+    (4, 16, (1, 2, 2), (1, 2, 2), (0, 0, 0), (1, 2, 32, 32), 4, 4, 1.0),     # kernel = stride: each phase one tap
 ]
 
 
