@@ -180,6 +180,36 @@ def time_networks(torch, rt3d, nets, dev, iters=20):
     return out
 
 
+def time_pruning_step(torch, rt3d, dev, hbm_gbs, iters=20):
+    """Device-side pruning step (group norms -> penalties + keep mask) on a weight tensor larger than L2:
+    2048 x 1024 x 3x3x3 fp32 = 226 MB, 4x4 groups.  Bound: HBM (the weights are read once)."""
+    M, N, k = 2048, 1024, (3, 3, 3)
+    w = torch.randn((M, N) + k, device=dev, dtype=torch.float32) * 0.05
+    P, Q, Ks = M // 4, N // 4, 27
+    norms = torch.empty((P, Q, Ks), device=dev, dtype=torch.float32)
+    pen = torch.empty_like(norms)
+    keep = torch.empty((P, Q, Ks), device=dev, dtype=torch.uint8)
+
+    def step():
+        rt3d.rt3d_kgs_group_norms(w, 4, 4, 2, norms)
+        rt3d.rt3d_kgs_reweight(norms, 1e-3, 0.2, pen, keep)
+
+    for _ in range(3):
+        step()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(iters):
+        step()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / iters
+    nbytes = w.numel() * 4 + norms.numel() * (4 + 4 + 4 + 1)
+    gbs = nbytes / ms / 1e6
+    return {"ms": ms, "alg_bytes": nbytes, "achieved_gbs": gbs, "hbm_peak_gbs": hbm_gbs, "frac": gbs / hbm_gbs,
+            "workload": "group norms + reweight, 2048x1024x3x3x3 fp32, 4x4 groups"}
+
+
 def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
@@ -296,6 +326,7 @@ def main():
     networks = None
     if not args.no_networks:
         networks = time_networks(torch, rt3d, nets, dev)
+        networks["pruning_step"] = time_pruning_step(torch, rt3d, dev, peaks()["hbm_gbs"])
 
     flops_kept = 2.0 * kept_macs
     per_step_ms = sparse_ms / args.steps

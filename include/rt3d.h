@@ -203,6 +203,25 @@ rt3d_status rt3d_maxpool3d(const rt3d_tensor* x, int kt, int kh, int kw, int st,
 /* y = a + b (optionally ReLU); equal extents and dtype; y may alias a or b. */
 rt3d_status rt3d_add_relu(const rt3d_tensor* a, const rt3d_tensor* b, int relu, rt3d_tensor* y, void* stream);
 
+/*
+ * Pruning step on the device (Section 4), the stage right before rt3d_pack_kgs.  All pointers DEVICE.
+ * rt3d_kgs_group_norms: norms[p][q][k] = group-lasso norm of the weights of kernel group (p,q) at
+ *   kernel location k (Fig. 2 caption; Eq. 2), norm = 1 (sum of magnitudes) or 2 (Euclidean);
+ *   w is float [M][N][Kt][Kh][Kw], norms float [P][Q][Kt*Kh*Kw]; missing kernels of ragged groups add 0.
+ * rt3d_kgs_reweight: one reweighting step on `count` norms (update rule below Eq. 3):
+ *   penalty[i] = 1 / (norms[i]^2 + eps), and the pruning decision keep[i] = norms[i] > threshold;
+ *   either output may be NULL; eps > 0.
+ * rt3d_kgs_expand_mask: group-level decisions [P][Q][Ks] -> per-weight mask [M][N][Ks] (uint8), the
+ *   form rt3d_pack_kgs takes once copied to the host.
+ * fp32 arithmetic; enqueue on `stream`, no synchronisation.  Errors: INVALID_ARG, CUDA.
+ */
+rt3d_status rt3d_kgs_group_norms(const float* w, int M, int N, int Kt, int Kh, int Kw, int g_m, int g_n, int norm,
+                                 float* norms, void* stream);
+rt3d_status rt3d_kgs_reweight(const float* norms, int64_t count, float eps, float threshold, float* penalty,
+                              uint8_t* keep, void* stream);
+rt3d_status rt3d_kgs_expand_mask(const uint8_t* group_mask, int M, int N, int Kt, int Kh, int Kw, int g_m, int g_n,
+                                 uint8_t* mask, void* stream);
+
 /* Work and traffic the method itself requires for one call (Section 3 cost model):
  * kept multiply-accumulates, dense multiply-accumulates, and algorithmic bytes
  * (input once + output once + packed weights and index once + bias). */

@@ -214,3 +214,28 @@ def add_relu(a, b, relu=True) -> np.ndarray:
     y = np.empty_like(a)
     lib.oracle_add_relu(_ptr(a, _f32p), _ptr(b, _f32p), ctypes.c_int64(a.size), int(relu), _ptr(y, _f32p))
     return y
+
+
+def group_norms(w, g_m: int, g_n: int, g: int = 2) -> np.ndarray:
+    """Group-lasso norm per (kernel group, kernel location): float32 [P, Q, Ks]; g = 1 or 2."""
+    lib = _load()
+    w = _f32(w)
+    M, N = w.shape[:2]
+    Ks = int(np.prod(w.shape[2:]))
+    P, Q = -(-M // g_m), -(-N // g_n)
+    out = np.empty((P, Q, Ks), dtype=np.float32)
+    rc = lib.oracle_group_norms(_ptr(w, _f32p), M, N, Ks, int(g_m), int(g_n), int(g), _ptr(out, _f32p))
+    if rc != 0:
+        raise ValueError("oracle_group_norms: bad arguments")
+    return out
+
+
+def reweight(norms, eps: float, threshold: float):
+    """(penalty = 1/(norm^2 + eps) as float32, keep = norm > threshold as uint8), same shape as norms."""
+    lib = _load()
+    norms = _f32(norms)
+    pen = np.empty_like(norms)
+    keep = np.empty(norms.shape, dtype=np.uint8)
+    lib.oracle_reweight(_ptr(norms, _f32p), ctypes.c_int64(norms.size), ctypes.c_float(eps), ctypes.c_float(threshold),
+                        _ptr(pen, _f32p), _ptr(keep, _u8p))
+    return pen, keep

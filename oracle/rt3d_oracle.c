@@ -344,3 +344,46 @@ int oracle_add_relu(const float* a, const float* b, int64_t count, int relu, flo
     }
     return 0;
 }
+
+/* -------------------------------------------- group norms, reweighting, mask (pruning step) ---- */
+/*
+ * Group-lasso norm of every (kernel group, kernel location), Section 4 (Fig. 2 caption, Eq. 2):
+ *   norms[p][q][k] = ( sum over kernels (i,j) of group (p,q) of |W[i][j][k]|^g )^(1/g),  g = 1 or 2.
+ * The printed caption drops the (i,j) subscript inside the sum; it is read as the sum over the
+ * kernels of the group.  Kernels that do not exist (ragged last groups) contribute nothing.
+ * Double accumulation, result cast to float.
+ */
+int oracle_group_norms(const float* w, int M, int N, int Ks, int g_m, int g_n, int g, float* norms)
+{
+    if (!w || !norms || (g != 1 && g != 2) || M <= 0 || N <= 0 || Ks <= 0 || g_m <= 0 || g_n <= 0) return -1;
+    const int P = (M + g_m - 1) / g_m, Q = (N + g_n - 1) / g_n;
+    for (int p = 0; p < P; ++p)
+      for (int q = 0; q < Q; ++q)
+        for (int k = 0; k < Ks; ++k) {
+            double s = 0.0;
+            for (int i = 0; i < g_m; ++i)
+              for (int j = 0; j < g_n; ++j) {
+                  const int m = p * g_m + i, c = q * g_n + j;
+                  if (m >= M || c >= N) continue;
+                  const double v = fabs((double)w[((int64_t)m * N + c) * Ks + k]);
+                  s += (g == 1) ? v : v * v;
+              }
+            norms[((int64_t)p * Q + q) * Ks + k] = (float)((g == 1) ? s : sqrt(s));
+        }
+    return 0;
+}
+
+/*
+ * One reweighting step (the update rule below Eq. 3): penalty = 1 / (norm^2 + eps); and the hard
+ * pruning decision that follows the last round ("prune the weights that converge to zero"):
+ * keep = norm > threshold.  The comparison is made on the float norm.
+ */
+int oracle_reweight(const float* norms, int64_t count, float eps, float threshold, float* penalty, uint8_t* keep)
+{
+    for (int64_t i = 0; i < count; ++i) {
+        const double n = (double)norms[i];
+        if (penalty) penalty[i] = (float)(1.0 / (n * n + (double)eps));
+        if (keep) keep[i] = norms[i] > threshold ? 1 : 0;
+    }
+    return 0;
+}

@@ -63,6 +63,9 @@ def _load():
     lib.rt3d_packed_free.restype = None
     for name in ("rt3d_conv3d_sparse", "rt3d_conv3d_dense", "rt3d_conv3d_host", "rt3d_conv3d_sparse_noalloc"):
         getattr(lib, name).argtypes = [TP, vp, vp, CP, TP, vp]
+    lib.rt3d_kgs_group_norms.argtypes = [vp, i, i, i, i, i, i, i, i, vp, vp]
+    lib.rt3d_kgs_reweight.argtypes = [vp, ctypes.c_int64, ctypes.c_float, ctypes.c_float, vp, vp, vp]
+    lib.rt3d_kgs_expand_mask.argtypes = [vp, i, i, i, i, i, i, i, vp, vp]
     lib.rt3d_maxpool3d.argtypes = [TP] + [i] * 9 + [TP, vp]
     lib.rt3d_add_relu.argtypes = [TP, TP, i, TP, vp]
     i64p = ctypes.POINTER(ctypes.c_int64)
@@ -243,6 +246,27 @@ def rt3d_maxpool3d(x: Tensor, k, stride, pad, y: Tensor, stream=None):
 def rt3d_add_relu(a: Tensor, b: Tensor, relu: bool, y: Tensor, stream=None):
     _check(_lib.rt3d_add_relu(ctypes.byref(a), ctypes.byref(b), int(bool(relu)), ctypes.byref(y),
                               _stream_ptr(stream)), "rt3d_add_relu")
+
+
+def rt3d_kgs_group_norms(w, g_m: int, g_n: int, norm: int, norms, stream=None):
+    """w: torch float32 device tensor [M,N,Kt,Kh,Kw]; norms: torch float32 device tensor [P,Q,Kt*Kh*Kw] (output)."""
+    M, N, Kt, Kh, Kw = w.shape
+    _check(_lib.rt3d_kgs_group_norms(ctypes.c_void_p(w.data_ptr()), M, N, Kt, Kh, Kw, int(g_m), int(g_n), int(norm),
+                                     ctypes.c_void_p(norms.data_ptr()), _stream_ptr(stream)), "rt3d_kgs_group_norms")
+
+
+def rt3d_kgs_reweight(norms, eps: float, threshold: float, penalty=None, keep=None, stream=None):
+    """norms: float32 device tensor; penalty (float32) / keep (uint8): device tensors of the same size or None."""
+    _check(_lib.rt3d_kgs_reweight(ctypes.c_void_p(norms.data_ptr()), norms.numel(), float(eps), float(threshold),
+                                  None if penalty is None else ctypes.c_void_p(penalty.data_ptr()),
+                                  None if keep is None else ctypes.c_void_p(keep.data_ptr()), _stream_ptr(stream)),
+           "rt3d_kgs_reweight")
+
+
+def rt3d_kgs_expand_mask(group_mask, M, N, Kt, Kh, Kw, g_m, g_n, mask, stream=None):
+    """group_mask: uint8 device [P,Q,Ks]; mask: uint8 device [M,N,Kt,Kh,Kw] (output)."""
+    _check(_lib.rt3d_kgs_expand_mask(ctypes.c_void_p(group_mask.data_ptr()), M, N, Kt, Kh, Kw, int(g_m), int(g_n),
+                                     ctypes.c_void_p(mask.data_ptr()), _stream_ptr(stream)), "rt3d_kgs_expand_mask")
 
 
 def rt3d_conv3d_cost(x: Tensor, w: Packed, stride=(1, 1, 1), pad=(0, 0, 0)):

@@ -350,3 +350,39 @@ def test_generator_is_counter_based_and_calibrated():
     assert synth.kgs_mask_exact_total(64, 64, 27, 12345, 3).sum() == 12345
     v = synth.vanilla_mask_exact_total(64, 64, 27, 100, 3)
     assert v.sum() == 2700 and set(np.unique(v.sum(-1))) == {0, 27}
+
+
+# ----------------------------------------------------- group norms and reweighting (Section 4)
+def test_group_norms_closed_forms_and_library():
+    M, N, k, g_m, g_n = 10, 7, (3, 3, 3), 4, 4
+    ones = np.ones((M, N) + k, np.float32)
+    n1 = oracle.group_norms(ones, g_m, g_n, 1)
+    n2 = oracle.group_norms(ones, g_m, g_n, 2)
+    rows = np.minimum(g_m, M - np.arange(0, M, g_m))          # kernels that exist in ragged groups
+    cols = np.minimum(g_n, N - np.arange(0, N, g_n))
+    cnt = np.outer(rows, cols).astype(np.float64)
+    np.testing.assert_array_equal(n1, np.broadcast_to(cnt[..., None], n1.shape).astype(np.float32))
+    np.testing.assert_allclose(n2, np.broadcast_to(np.sqrt(cnt)[..., None], n2.shape), rtol=1e-7)
+    w = _rand((M, N) + k, 4)
+    for g in (1, 2):                                           # library norm on each reshaped group
+        got = oracle.group_norms(w, g_m, g_n, g)
+        for p in range(3):
+            for q in range(2):
+                blk = w[p * g_m:(p + 1) * g_m, q * g_n:(q + 1) * g_n].reshape(-1, 27).astype(np.float64)
+                np.testing.assert_allclose(got[p, q], np.linalg.norm(blk, ord=g, axis=0), rtol=1e-6)
+        np.testing.assert_allclose(oracle.group_norms(-2.5 * w, g_m, g_n, g), 2.5 * got, rtol=1e-6)   # homogeneity
+
+
+def test_reweight_penalty_and_mask():
+    norms = np.array([0.0, 0.1, 0.5, 2.0], np.float32)
+    pen, keep = oracle.reweight(norms, 1e-3, 0.3)
+    np.testing.assert_allclose(pen, [1000.0, 1 / 0.011, 1 / 0.251, 1 / 4.001], rtol=1e-6)   # 1 / (n^2 + eps)
+    assert (np.diff(pen) < 0).all()                     # larger groups are penalised less
+    np.testing.assert_array_equal(keep, [0, 0, 1, 1])
+    # a mask made this way is a KGS mask: the packer accepts it and keeps exactly those locations
+    w = _rand((8, 8, 3, 3, 3), 5)
+    n = oracle.group_norms(w, 4, 4, 2)
+    thr = float(np.median(n))
+    _, gk = oracle.reweight(n, 1e-3, thr)
+    mask = synth.expand_group_mask(gk, 8, 8, 4, 4, 3, 3, 3)
+    assert oracle.pack_kgs(w, mask, 4, 4)["nnz"] == int(gk.sum()) == int((n > thr).sum())
