@@ -282,6 +282,28 @@ rt3d_status encode_xmap(const rt3d_tensor* x, const ConvGeom& g, const TileBox& 
   return r == CUDA_SUCCESS ? RT3D_OK : RT3D_ERR_CUDA;
 }
 
+// Output tensor map for the TMA-store epilogue: box = 32 channels x the 32 voxels one epilogue warp owns
+// (sub-box of the tile), 64-byte swizzle.  Returns false when a warp's rows are not a rectangular block
+// of voxels (then the kernels store directly).
+bool encode_ymap(const rt3d_tensor* y, const ConvGeom& g, int bw, int bh, int bt, int bn, CUtensorMap* map) {
+  if (g.M < 32 || (bw * bh * bt * bn) % 32) return false;
+  int rem = 32, sb[4] = {1, 1, 1, 1};
+  const int dims_box[4] = {bw, bh, bt, bn};
+  for (int i = 0; i < 4 && rem > 1; ++i) {
+    const int d = dims_box[i];
+    if (d >= rem) { if (d % rem) return false; sb[i] = rem; rem = 1; }
+    else { if (rem % d) return false; sb[i] = d; rem /= d; }
+  }
+  if (rem != 1) return false;
+  const cuuint64_t cs = cuuint64_t(g.ycs) * 2;
+  cuuint64_t dims[5] = {cuuint64_t(g.M), cuuint64_t(g.Wo), cuuint64_t(g.Ho), cuuint64_t(g.To), cuuint64_t(g.n)};
+  cuuint64_t strides[4] = {cs, cs * g.Wo, cs * g.Wo * g.Ho, cs * g.Wo * g.Ho * g.To};
+  cuuint32_t bx[5] = {32, cuuint32_t(sb[0]), cuuint32_t(sb[1]), cuuint32_t(sb[2]), cuuint32_t(sb[3])};
+  cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+  return g_encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, y->data, dims, strides, bx, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                  CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 // Small-C_in kernel: bf16, C_in <= 8 stored at pitch 8, spatial strides <= 4, M <= 256.
 bool smallc_eligible(const DeviceState* d, rt3d_packed* w, const rt3d_tensor* x, const rt3d_tensor* y,
                      const rt3d_conv_params* p, const SmallCLayout** out) {
@@ -337,7 +359,9 @@ rt3d_status launch_smallc(rt3d_packed* w, DeviceBlob* blob, const DeviceState* d
   if (g_encode(&xmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, x->data, dims, strides, bx, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
     return RT3D_ERR_CUDA;
-  if (launch_conv_umma_smallc(a, &xmap, d->sm_count, st) != cudaSuccess) return RT3D_ERR_CUDA;
+  CUtensorMap ymap;
+  a.store_tma = encode_ymap(y, g, kSmallCTileW, kSmallCTileH, 1, 1, &ymap) ? 1 : 0;
+  if (launch_conv_umma_smallc(a, &xmap, a.store_tma ? &ymap : nullptr, d->sm_count, st) != cudaSuccess) return RT3D_ERR_CUDA;
   g_launches.fetch_add(1);
   return RT3D_OK;
 }
@@ -428,8 +452,11 @@ rt3d_status conv_impl(const rt3d_tensor* x, const rt3d_packed* wc, const float* 
   }
   CUtensorMap xmap;
   if ((s = encode_xmap(x, g, a.box, &xmap)) != RT3D_OK) return s;
-  cudaError_t e = use_pair ? launch_conv_umma_pair(a, &xmap, u->wmap_half, d->sm_count, st)
-                           : launch_conv_umma(a, &xmap, u->wmap, d->sm_count, st);
+  CUtensorMap ymap;
+  a.store_tma = (a.n_splits == 1 && encode_ymap(y, g, a.box.bw, a.box.bh, a.box.bt, a.box.bn, &ymap)) ? 1 : 0;
+  const void* ym = a.store_tma ? &ymap : nullptr;
+  cudaError_t e = use_pair ? launch_conv_umma_pair(a, &xmap, u->wmap_half, ym, d->sm_count, st)
+                           : launch_conv_umma(a, &xmap, u->wmap, ym, d->sm_count, st);
   if (e != cudaSuccess) return RT3D_ERR_CUDA;
   g_launches.fetch_add(1);
   return RT3D_OK;
@@ -708,7 +735,9 @@ rt3d_status rt3d_conv3d_sparse_noalloc(const rt3d_tensor* x, const rt3d_packed* 
   }
   CUtensorMap xmap;
   if ((s = encode_xmap(x, g, a.box, &xmap)) != RT3D_OK) return s;
-  if (launch_conv_umma(a, &xmap, u->wmap, d->sm_count, st) != cudaSuccess) return RT3D_ERR_CUDA;
+  CUtensorMap ymap;
+  a.store_tma = (a.n_splits == 1 && encode_ymap(y, g, a.box.bw, a.box.bh, a.box.bt, a.box.bn, &ymap)) ? 1 : 0;
+  if (launch_conv_umma(a, &xmap, u->wmap, a.store_tma ? &ymap : nullptr, d->sm_count, st) != cudaSuccess) return RT3D_ERR_CUDA;
   g_launches.fetch_add(1);
   return RT3D_OK;
 }

@@ -46,20 +46,23 @@ struct UmmaArgs {
   const float* bias;                        // device or nullptr
   void* y;
   int32_t* sched;                           // device [8]: [2] = error word set by a bounded wait that gave up
+  int store_tma;                            // 1: epilogue stores go through shared memory + TMA (needs ymap)
   int n_splits;                             // K splits per output tile (1 = none)
   float* scratch;                           // device, split-K partial tiles [tile][split][128][n_tile] (n_splits > 1)
   int32_t* counters;                        // device, [tiles * 4] arrival counters, zero between launches
 };
 
 // xmap / wmap point to 128-byte CUtensorMap objects in host memory.
-cudaError_t launch_conv_umma(const UmmaArgs& a, const void* xmap, const void* wmap, int sm_count,
+// ymap: tensor map of the output for the TMA-store epilogue (box = 32 channels x one warp's 32 voxels,
+// 64-byte swizzle); used when a.store_tma != 0, may be nullptr otherwise.
+cudaError_t launch_conv_umma(const UmmaArgs& a, const void* xmap, const void* wmap, const void* ymap, int sm_count,
                              cudaStream_t stream);
 
 // CTA-pair variant (cta_group::2): wmap_half is a tensor map over the same weight tiles whose box is
 // half a tile high (n_tile/2 rows).  Needs n_tile % 32 == 0 and a.n_splits == 1.
 bool umma_pair_supported(int n_tile, int n_bundles);
-cudaError_t launch_conv_umma_pair(const UmmaArgs& a, const void* xmap, const void* wmap_half, int sm_count,
-                                  cudaStream_t stream);
+cudaError_t launch_conv_umma_pair(const UmmaArgs& a, const void* xmap, const void* wmap_half, const void* ymap,
+                                  int sm_count, cudaStream_t stream);
 
 // Arguments of the small-C_in tensor-core kernel (C_in <= 8 at channel pitch 8).
 struct SmallCArgs {
@@ -69,13 +72,15 @@ struct SmallCArgs {
   int img_w, phase_bytes;             // voxels per image row; bytes one phase load delivers
   int tiles_h, tiles_w;               // 16 x 8 output tiles per frame
   int tmem_cols;                      // filled in by the launcher
+  int store_tma;                      // 1: TMA-store epilogue (needs ymap)
   const void* wimg;                   // device: [n_pairs][2][n_pad/8][8][8] bf16
   const int32_t* pair_off;            // device: [n_pairs][2] byte offsets inside the staged images
   const float* bias;
   void* y;
   int32_t* sched;
 };
-cudaError_t launch_conv_umma_smallc(const SmallCArgs& a, const void* xmap, int sm_count, cudaStream_t stream);
+cudaError_t launch_conv_umma_smallc(const SmallCArgs& a, const void* xmap, const void* ymap, int sm_count,
+                                    cudaStream_t stream);
 size_t smallc_smem_bytes(int n_pairs, int n_pad, int stage_bytes);
 
 // Shared memory the tcgen05 kernel needs for a bundle width (for the host-side eligibility check).

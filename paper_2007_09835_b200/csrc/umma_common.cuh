@@ -186,6 +186,86 @@ __device__ __forceinline__ void epilogue_row(uint32_t taddr, int n_cols, bool ha
   }
 }
 
+// ------------------------------------------------------------------------------ TMA-store epilogue
+// Each epilogue warp owns 32 rows of a tile; when those rows are a rectangular block of output voxels
+// the warp writes 32-channel pieces (32 rows x 64 bytes of bf16) into its own two staging buffers in
+// shared memory, in the 64-byte swizzle pattern, and one lane hands each piece to the TMA engine as a
+// 5-D box store.  The stores drain asynchronously (full 64-byte rows, clipped at the tensor's edges and
+// at the channel count), so the threads never wait on global stores.  Only warp-level synchronisation
+// is used.
+constexpr uint32_t kStoreStageBytes = 32 * 64;          // one piece
+constexpr uint32_t kStoreWarpBytes = 2 * kStoreStageBytes;
+
+struct TmaStore {
+  const CUtensorMap* map;
+  uint32_t smem;              // this warp's two staging buffers (1024-byte aligned)
+  int c1, c2, c3, c4;         // output coordinates (w, h, t, n) of the warp's first row
+  uint32_t piece;             // pieces issued so far by this warp
+};
+
+__device__ __forceinline__ void tma_store_5d(const CUtensorMap* map, uint32_t src, int c0, int c1, int c2, int c3, int c4) {
+  asm volatile("cp.async.bulk.tensor.5d.global.shared::cta.tile.bulk_group [%0, {%2, %3, %4, %5, %6}], [%1];"
+               ::"l"(reinterpret_cast<uint64_t>(map)), "r"(src), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4)
+               : "memory");
+  asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+__device__ __forceinline__ void tma_store_wait_read_1() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
+// Before the warp leaves the kernel: all its bulk stores have completed (shared memory read, global written).
+__device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+
+// 32 accumulator columns of this thread's row -> bias, ReLU, bf16 -> staging buffer -> TMA box store of
+// channels [m0, m0+32) x the warp's 32 voxels.
+__device__ __forceinline__ void epilogue_piece_tma(const uint32_t* v, const float* bias_s, int relu, int m0, int lane,
+                                                   TmaStore& ts) {
+  uint4 o[4];
+  __nv_bfloat162* po = reinterpret_cast<__nv_bfloat162*>(o);
+#pragma unroll
+  for (int q = 0; q < 16; ++q) {
+    float a = __uint_as_float(v[2 * q]) + bias_s[2 * q], b = __uint_as_float(v[2 * q + 1]) + bias_s[2 * q + 1];
+    if (relu) { a = fmaxf(a, 0.f); b = fmaxf(b, 0.f); }
+    po[q] = __floats2bfloat162_rn(a, b);
+  }
+  const uint32_t buf = ts.smem + (ts.piece & 1u) * kStoreStageBytes;
+  if (lane == 0) tma_store_wait_read_1();          // the store issued two pieces ago has read this buffer
+  __syncwarp();
+  const uint32_t row = buf + uint32_t(lane) * 64u;
+  const uint32_t sw = (uint32_t(lane) >> 1) & 3u;  // 64-byte swizzle: 16-byte chunk index ^= address bits 7..8
+#pragma unroll
+  for (uint32_t k = 0; k < 4; ++k)
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(row + ((k ^ sw) << 4)), "r"(o[k].x), "r"(o[k].y),
+                 "r"(o[k].z), "r"(o[k].w) : "memory");
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  __syncwarp();
+  if (lane == 0) tma_store_5d(ts.map, buf, m0, ts.c1, ts.c2, ts.c3, ts.c4);
+  ++ts.piece;
+}
+
+// One voxel row of a finished accumulator tile through the TMA-store path: full 32-column pieces go
+// through the staging buffers, a 16-column tail (bundle widths that are not multiples of 32) is stored
+// directly.  `warp_rows_valid`: this warp's 32 rows belong to the tile (warp-uniform).
+__device__ __forceinline__ void epilogue_row_tma(uint32_t taddr, int n_cols, bool has_acc, bool warp_rows_valid,
+                                                 bool in_range, const float* bias_s, int relu, __nv_bfloat16* dst,
+                                                 int m_base, int M, int lane, TmaStore& ts) {
+  for (int col = 0; col < n_cols; col += 32) {
+    const int m0 = m_base + col;
+    if (m0 >= M) break;
+    uint32_t v[32];
+    const bool wide = col + 32 <= n_cols;
+    if (has_acc) {
+      if (wide) tmem_ld32(taddr + col, v);
+      else tmem_ld16(taddr + col, *reinterpret_cast<uint32_t(*)[16]>(v));
+    } else {
+#pragma unroll
+      for (int q = 0; q < 32; ++q) v[q] = 0u;
+    }
+    if (wide) {
+      if (warp_rows_valid) epilogue_piece_tma(v, bias_s + m0, relu, m0, lane, ts);
+    } else if (in_range) {
+      epilogue_cols<16>(v, bias_s + m0, relu, dst + col, M - m0);
+    }
+  }
+}
+
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 

@@ -122,13 +122,15 @@ __device__ __forceinline__ void reduce_partial_row(const float* part0, size_t sp
 template <bool kDense>
 __global__ void __launch_bounds__(kThreadsUmma, 1)
 conv3d_umma_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CUtensorMap wmap,
-                   const UmmaArgs a, const int stages, const int tmem_cols) {
+                   const __grid_constant__ CUtensorMap ymap, const UmmaArgs a, const int stages, const int tmem_cols) {
   extern __shared__ unsigned char smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t tiles_base = (raw + 1023u) & ~1023u;            // operand tiles need 1024-byte alignment
   const uint32_t b_bytes = uint32_t(a.n_tile) * 128u;
   const uint32_t stage_bytes = kABytes + b_bytes;
-  Barriers* bars = reinterpret_cast<Barriers*>(smem_raw + (tiles_base - raw) + size_t(stages) * stage_bytes);
+  const uint32_t store_smem = tiles_base + uint32_t(stages) * stage_bytes;     // 4 warps x 2 staging buffers
+  Barriers* bars = reinterpret_cast<Barriers*>(smem_raw + (tiles_base - raw) + size_t(stages) * stage_bytes +
+                                               4 * kStoreWarpBytes);
   float* bias_s = reinterpret_cast<float*>(bars + 1);              // bias of all bundles (zeros if none), padded
   int32_t* err = a.sched + 2;
   for (int i = threadIdx.x; i < a.n_bundles * a.n_tile; i += blockDim.x)
@@ -251,6 +253,12 @@ conv3d_umma_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_consta
     const int bt_i = r % a.box.bt; r /= a.box.bt;
     const int bn_i = r;
     __nv_bfloat16* yb = static_cast<__nv_bfloat16*>(a.y);
+    TmaStore ts{&ymap, store_smem + uint32_t(quad) * kStoreWarpBytes, 0, 0, 0, 0, 0u};
+    int r0 = quad * 32;                        // coordinates of the warp's first row inside the box
+    const int bw_0 = r0 % a.box.bw; r0 /= a.box.bw;
+    const int bh_0 = r0 % a.box.bh; r0 /= a.box.bh;
+    const int bt_0 = r0 % a.box.bt; r0 /= a.box.bt;
+    const int bn_0 = r0;
     const size_t part_tile = size_t(128) * a.n_tile;       // floats per partial tile
     uint32_t j = 0;
     for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++j) {
@@ -267,7 +275,13 @@ conv3d_umma_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_consta
       const uint32_t taddr = tmem_base + (uint32_t(quad * 32) << 16) + buf * uint32_t(a.n_tile);
       __nv_bfloat16* dst = yb + vox * a.g.ycs + m_base;
       if (a.n_splits == 1) {
-        epilogue_row(taddr, a.n_tile, nsteps > 0, in_range, bias_s, a.g.relu, dst, m_base, a.g.M);
+        if (a.store_tma) {
+          ts.c1 = c.w0 + bw_0; ts.c2 = c.h0 + bh_0; ts.c3 = c.t0 + bt_0; ts.c4 = c.n0 + bn_0;
+          epilogue_row_tma(taddr, a.n_tile, nsteps > 0, quad * 32 < box_rows, in_range, bias_s, a.g.relu, dst, m_base,
+                           a.g.M, lane, ts);
+        } else {
+          epilogue_row(taddr, a.n_tile, nsteps > 0, in_range, bias_s, a.g.relu, dst, m_base, a.g.M);
+        }
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&bars->tmem_empty[buf]));
@@ -293,6 +307,7 @@ conv3d_umma_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_consta
         }
       }
     }
+    if (lane == 0) tma_store_wait_all();         // all bulk stores done before shared memory goes away
   }
 
   // ---------------------------------------------------------------------- teardown
@@ -318,11 +333,11 @@ int pick_stages(int n_tile) {
 }  // namespace
 
 size_t umma_smem_bytes(int n_tile, int n_bundles) {
-  return size_t(pick_stages(n_tile)) * (kABytes + size_t(n_tile) * 128) + 1024 + sizeof(Barriers) +
+  return size_t(pick_stages(n_tile)) * (kABytes + size_t(n_tile) * 128) + 1024 + 4 * kStoreWarpBytes + sizeof(Barriers) +
          size_t(n_tile) * n_bundles * 4;
 }
 
-cudaError_t launch_conv_umma(const UmmaArgs& a, const void* xmap, const void* wmap, int sm_count,
+cudaError_t launch_conv_umma(const UmmaArgs& a, const void* xmap, const void* wmap, const void* ymap, int sm_count,
                              cudaStream_t stream) {
   const int stages = pick_stages(a.n_tile);
   if (stages < 2) return cudaErrorInvalidValue;
@@ -335,9 +350,11 @@ cudaError_t launch_conv_umma(const UmmaArgs& a, const void* xmap, const void* wm
   const long long n_items = (long long)a.tiles_n * a.tiles_t * a.tiles_h * a.tiles_w * a.n_bundles * a.n_splits;
   if (n_items <= 0) return cudaSuccess;
   const int grid = int(n_items < sm_count ? n_items : sm_count);
-  CUtensorMap xm, wm;
+  if (a.store_tma && ymap == nullptr) return cudaErrorInvalidValue;
+  CUtensorMap xm, wm, ym;
   memcpy(&xm, xmap, sizeof(CUtensorMap));
   memcpy(&wm, wmap, sizeof(CUtensorMap));
+  memcpy(&ym, ymap ? ymap : xmap, sizeof(CUtensorMap));
   cudaError_t e;
   if (a.dense) {
     static bool attr_done_d = false;
@@ -346,7 +363,7 @@ cudaError_t launch_conv_umma(const UmmaArgs& a, const void* xmap, const void* wm
       if (e != cudaSuccess) return e;
       attr_done_d = true;
     }
-    conv3d_umma_kernel<true><<<grid, kThreadsUmma, smem, stream>>>(xm, wm, a, stages, cols);
+    conv3d_umma_kernel<true><<<grid, kThreadsUmma, smem, stream>>>(xm, wm, ym, a, stages, cols);
   } else {
     static bool attr_done_s = false;
     if (!attr_done_s) {
@@ -354,7 +371,7 @@ cudaError_t launch_conv_umma(const UmmaArgs& a, const void* xmap, const void* wm
       if (e != cudaSuccess) return e;
       attr_done_s = true;
     }
-    conv3d_umma_kernel<false><<<grid, kThreadsUmma, smem, stream>>>(xm, wm, a, stages, cols);
+    conv3d_umma_kernel<false><<<grid, kThreadsUmma, smem, stream>>>(xm, wm, ym, a, stages, cols);
   }
   return cudaGetLastError();
 }

@@ -96,7 +96,7 @@ __device__ __forceinline__ PairItem decode_pair_item(const UmmaArgs& a, int item
 template <bool kDense>
 __global__ void __launch_bounds__(kThreadsUmma, 1)
 conv3d_umma_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CUtensorMap wmap_half,
-                        const UmmaArgs a, const int stages, const int tmem_cols) {
+                        const __grid_constant__ CUtensorMap ymap, const UmmaArgs a, const int stages, const int tmem_cols) {
   extern __shared__ unsigned char smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t tiles_base = (raw + 1023u) & ~1023u;
@@ -104,7 +104,9 @@ conv3d_umma_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_c
   const uint32_t b_bytes = uint32_t(n_half) * 128u;             // this CTA's half of the B tile
   const uint32_t chunk_bytes = kABytes + b_bytes;
   const uint32_t stage_bytes = kCps * chunk_bytes;
-  Barriers* bars = reinterpret_cast<Barriers*>(smem_raw + (tiles_base - raw) + size_t(stages) * stage_bytes);
+  const uint32_t store_smem = tiles_base + uint32_t(stages) * stage_bytes;     // 4 warps x 2 staging buffers
+  Barriers* bars = reinterpret_cast<Barriers*>(smem_raw + (tiles_base - raw) + size_t(stages) * stage_bytes +
+                                               4 * kStoreWarpBytes);
   float* bias_s = reinterpret_cast<float*>(bars + 1);
   int32_t* err = a.sched + 2;
   for (int i = threadIdx.x; i < a.n_bundles * a.n_tile; i += blockDim.x)
@@ -238,6 +240,12 @@ conv3d_umma_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_c
     const int bt_i = r % a.box.bt; r /= a.box.bt;
     const int bn_i = r;
     __nv_bfloat16* yb = static_cast<__nv_bfloat16*>(a.y);
+    TmaStore ts{&ymap, store_smem + uint32_t(quad) * kStoreWarpBytes, 0, 0, 0, 0, 0u};
+    int r0 = quad * 32;                        // coordinates of the warp's first row inside the box
+    const int bw_0 = r0 % a.box.bw; r0 /= a.box.bw;
+    const int bh_0 = r0 % a.box.bh; r0 /= a.box.bh;
+    const int bt_0 = r0 % a.box.bt; r0 /= a.box.bt;
+    const int bn_0 = r0;
     uint32_t j = 0;
     for (int item = cluster_id; item < n_items; item += n_clusters, ++j) {
       const PairItem c = decode_pair_item(a, item, pairs_per_bundle, n_mtiles, rank);
@@ -250,11 +258,18 @@ conv3d_umma_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_c
       const long long vox = (((long long)nn * a.g.To + to) * a.g.Ho + ho) * a.g.Wo + wo;
       const int m_base = c.bundle * a.n_tile;
       const uint32_t taddr = tmem_base + (uint32_t(quad * 32) << 16) + buf * uint32_t(a.n_tile);
-      epilogue_row(taddr, a.n_tile, nsteps > 0, in_range, bias_s, a.g.relu, yb + vox * a.g.ycs + m_base, m_base, a.g.M);
+      if (a.store_tma) {
+        ts.c1 = c.w0 + bw_0; ts.c2 = c.h0 + bh_0; ts.c3 = c.t0 + bt_0; ts.c4 = c.n0 + bn_0;
+        epilogue_row_tma(taddr, a.n_tile, nsteps > 0, quad * 32 < box_rows, in_range, bias_s, a.g.relu,
+                         yb + vox * a.g.ycs + m_base, m_base, a.g.M, lane, ts);
+      } else {
+        epilogue_row(taddr, a.n_tile, nsteps > 0, in_range, bias_s, a.g.relu, yb + vox * a.g.ycs + m_base, m_base, a.g.M);
+      }
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster(mapa_shared(smem_u32(&bars->tmem_empty[buf]), 0));
     }
+    if (lane == 0) tma_store_wait_all();         // all bulk stores done before shared memory goes away
   }
 
   // ---------------------------------------------------------------------- teardown
@@ -278,12 +293,14 @@ int pick_stages_pair(int n_tile) {
 }
 
 size_t pair_smem_bytes(int n_tile, int n_bundles) {
-  return size_t(pick_stages_pair(n_tile)) * kCps * (kABytes + size_t(n_tile / 2) * 128) + 1024 + sizeof(Barriers) +
+  return size_t(pick_stages_pair(n_tile)) * kCps * (kABytes + size_t(n_tile / 2) * 128) + 1024 + 4 * kStoreWarpBytes +
+         sizeof(Barriers) +
          size_t(n_tile) * n_bundles * 4;
 }
 
 template <bool kDense>
-cudaError_t launch_pair_t(const UmmaArgs& a, const CUtensorMap& xm, const CUtensorMap& wm, int sm_count, int stages,
+cudaError_t launch_pair_t(const UmmaArgs& a, const CUtensorMap& xm, const CUtensorMap& wm, const CUtensorMap& ym,
+                          int sm_count, int stages,
                           int cols, size_t smem, long long n_items, cudaStream_t stream) {
   static bool attr_done = false;
   if (!attr_done) {
@@ -311,7 +328,7 @@ cudaError_t launch_pair_t(const UmmaArgs& a, const CUtensorMap& xm, const CUtens
   long long clusters = max_clusters < sm_count / 2 ? max_clusters : sm_count / 2;
   if (clusters > n_items) clusters = n_items;
   cfg.gridDim = dim3(unsigned(2 * clusters));
-  return cudaLaunchKernelEx(&cfg, conv3d_umma_pair_kernel<kDense>, xm, wm, a, stages, cols);
+  return cudaLaunchKernelEx(&cfg, conv3d_umma_pair_kernel<kDense>, xm, wm, ym, a, stages, cols);
 }
 
 }  // namespace
@@ -320,8 +337,8 @@ bool umma_pair_supported(int n_tile, int n_bundles) {
   return n_tile % 32 == 0 && n_tile <= 256 && pick_stages_pair(n_tile) >= 2 && pair_smem_bytes(n_tile, n_bundles) <= 227 * 1024;
 }
 
-cudaError_t launch_conv_umma_pair(const UmmaArgs& a, const void* xmap, const void* wmap_half, int sm_count,
-                                  cudaStream_t stream) {
+cudaError_t launch_conv_umma_pair(const UmmaArgs& a, const void* xmap, const void* wmap_half, const void* ymap,
+                                  int sm_count, cudaStream_t stream) {
   if (!umma_pair_supported(a.n_tile, a.n_bundles) || a.n_splits != 1) return cudaErrorInvalidValue;
   const int stages = pick_stages_pair(a.n_tile);
   const size_t smem = pair_smem_bytes(a.n_tile, a.n_bundles);
@@ -331,11 +348,13 @@ cudaError_t launch_conv_umma_pair(const UmmaArgs& a, const void* xmap, const voi
   const long long n_mtiles = (long long)a.tiles_n * a.tiles_t * a.tiles_h * a.tiles_w;
   const long long n_items = ((n_mtiles + 1) / 2) * a.n_bundles;
   if (n_items <= 0) return cudaSuccess;
-  CUtensorMap xm, wm;
+  if (a.store_tma && ymap == nullptr) return cudaErrorInvalidValue;
+  CUtensorMap xm, wm, ym;
   memcpy(&xm, xmap, sizeof(CUtensorMap));
   memcpy(&wm, wmap_half, sizeof(CUtensorMap));
-  return a.dense ? launch_pair_t<true>(a, xm, wm, sm_count, stages, cols, smem, n_items, stream)
-                 : launch_pair_t<false>(a, xm, wm, sm_count, stages, cols, smem, n_items, stream);
+  memcpy(&ym, ymap ? ymap : xmap, sizeof(CUtensorMap));
+  return a.dense ? launch_pair_t<true>(a, xm, wm, ym, sm_count, stages, cols, smem, n_items, stream)
+                 : launch_pair_t<false>(a, xm, wm, ym, sm_count, stages, cols, smem, n_items, stream);
 }
 
 }  // namespace rt3d

@@ -26,10 +26,12 @@ constexpr int kSmallCStages = 3;
 
 template <int kDummy>
 __global__ void __launch_bounds__(kThreadsUmma, 1)
-conv3d_umma_smallc_kernel(const __grid_constant__ CUtensorMap xmap, const SmallCArgs a) {
+conv3d_umma_smallc_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CUtensorMap ymap,
+                          const SmallCArgs a) {
   extern __shared__ unsigned char smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
-  const uint32_t base = (raw + 127u) & ~127u;
+  const uint32_t store_smem = (raw + 1023u) & ~1023u;                   // 4 warps x 2 staging buffers (TMA stores)
+  const uint32_t base = store_smem + 4 * kStoreWarpBytes;
   const uint32_t w_bytes = uint32_t(a.n_pairs) * 2u * uint32_t(a.n_pad) * 16u;
   const uint32_t w_smem = base;                                         // weight image, whole layer
   const uint32_t halo_smem = base + ((w_bytes + 127u) & ~127u);         // ring of staged halos
@@ -128,6 +130,7 @@ conv3d_umma_smallc_kernel(const __grid_constant__ CUtensorMap xmap, const SmallC
     const int row = quad * 32 + lane;
     const int bh_i = row / kSmallCTileW, bw_i = row % kSmallCTileW;
     __nv_bfloat16* yb = static_cast<__nv_bfloat16*>(a.y);
+    TmaStore ts{&ymap, store_smem + uint32_t(quad) * kStoreWarpBytes, 0, 0, 0, 0, 0u};   // warp = 4 rows x 8 voxels
     uint32_t j = 0;
     for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++j) {
       int r = item;
@@ -142,11 +145,18 @@ conv3d_umma_smallc_kernel(const __grid_constant__ CUtensorMap xmap, const SmallC
       const bool in_range = ho < a.g.Ho && wo < a.g.Wo;
       const long long vox = (((long long)nn * a.g.To + to) * a.g.Ho + ho) * a.g.Wo + wo;
       const uint32_t taddr = tmem_base + (uint32_t(quad * 32) << 16) + buf * uint32_t(a.n_pad);
-      epilogue_row(taddr, a.n_pad, a.n_pairs > 0, in_range, bias_s, a.g.relu, yb + vox * a.g.ycs, 0, a.g.M);
+      if (a.store_tma) {
+        ts.c1 = iw * kSmallCTileW; ts.c2 = ih * kSmallCTileH + quad * 4; ts.c3 = to; ts.c4 = nn;
+        epilogue_row_tma(taddr, a.n_pad, a.n_pairs > 0, true, in_range, bias_s, a.g.relu, yb + vox * a.g.ycs, 0, a.g.M,
+                         lane, ts);
+      } else {
+        epilogue_row(taddr, a.n_pad, a.n_pairs > 0, in_range, bias_s, a.g.relu, yb + vox * a.g.ycs, 0, a.g.M);
+      }
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&bars->tmem_empty[buf]));
     }
+    if (lane == 0) tma_store_wait_all();         // all bulk stores done before shared memory goes away
   }
 
   if (bars->abort_flag) {
@@ -166,10 +176,11 @@ conv3d_umma_smallc_kernel(const __grid_constant__ CUtensorMap xmap, const SmallC
 size_t smallc_smem_bytes(int n_pairs, int n_pad, int stage_bytes) {
   const size_t w = (size_t(n_pairs) * 2 * n_pad * 16 + 127) & ~size_t(127);
   const size_t halo = (size_t(stage_bytes) + 127) & ~size_t(127);
-  return 128 + w + kSmallCStages * halo + ((size_t(n_pairs) * 8 + 15) & ~size_t(15)) + sizeof(Barriers) + size_t(n_pad) * 4;
+  return 1024 + 4 * kStoreWarpBytes + w + kSmallCStages * halo + ((size_t(n_pairs) * 8 + 15) & ~size_t(15)) + sizeof(Barriers) + size_t(n_pad) * 4;
 }
 
-cudaError_t launch_conv_umma_smallc(const SmallCArgs& a_in, const void* xmap, int sm_count, cudaStream_t stream) {
+cudaError_t launch_conv_umma_smallc(const SmallCArgs& a_in, const void* xmap, const void* ymap, int sm_count,
+                                    cudaStream_t stream) {
   SmallCArgs a = a_in;
   int cols = 32;
   while (cols < 2 * a.n_pad) cols *= 2;
@@ -187,15 +198,17 @@ cudaError_t launch_conv_umma_smallc(const SmallCArgs& a_in, const void* xmap, in
   if (per_sm < 1) per_sm = 1;
   const long long want = (long long)sm_count * per_sm;
   const int grid = int(n_items < want ? n_items : want);
-  CUtensorMap xm;
+  if (a.store_tma && ymap == nullptr) return cudaErrorInvalidValue;
+  CUtensorMap xm, ym;
   memcpy(&xm, xmap, sizeof(CUtensorMap));
+  memcpy(&ym, ymap ? ymap : xmap, sizeof(CUtensorMap));
   static bool attr_done = false;
   if (!attr_done) {
     cudaError_t e = cudaFuncSetAttribute(conv3d_umma_smallc_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
     if (e != cudaSuccess) return e;
     attr_done = true;
   }
-  conv3d_umma_smallc_kernel<0><<<grid, kThreadsUmma, smem, stream>>>(xm, a);
+  conv3d_umma_smallc_kernel<0><<<grid, kThreadsUmma, smem, stream>>>(xm, ym, a);
   return cudaGetLastError();
 }
 
