@@ -70,8 +70,6 @@ __device__ __forceinline__ uint32_t instr_desc_bf16_pair(int n) {
   return (1u << 4) | (1u << 7) | (1u << 10) | (uint32_t(n >> 3) << 17) | (uint32_t(256 >> 4) << 24);
 }
 
-constexpr int kCps = 1;     // K chunks (of 64 channels) per pipeline stage (2 was measured: no gain)
-
 struct PairItem {
   int bundle;
   int n0, t0, h0, w0;     // first output voxel of this CTA's box (beyond the tensor for a dummy tile)
@@ -93,7 +91,8 @@ __device__ __forceinline__ PairItem decode_pair_item(const UmmaArgs& a, int item
   return c;
 }
 
-template <bool kDense>
+// kCps: K steps per pipeline stage (and per barrier hand-shake): 1, or 2 for narrow bundles.
+template <bool kDense, int kCps>
 __global__ void __launch_bounds__(kThreadsUmma, 1)
 conv3d_umma_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CUtensorMap wmap_half,
                         const __grid_constant__ CUtensorMap ymap, const UmmaArgs a, const int stages, const int tmem_cols) {
@@ -286,25 +285,29 @@ conv3d_umma_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_c
   }
 }
 
+// Two K steps share one barrier hand-shake when a step is short (narrow bundles: the issuing thread, not
+// the tensor pipe, is the limit there); wide bundles keep one step per stage (deeper pipeline).
+int pick_cps(int n_tile) { return n_tile <= 128 ? 2 : 1; }
+
 int pick_stages_pair(int n_tile) {
-  const size_t stage = kCps * (kABytes + size_t(n_tile / 2) * 128);
+  const size_t stage = pick_cps(n_tile) * (kABytes + size_t(n_tile / 2) * 128);
   const int s = int(kSmemBudget / stage);
   return s > kMaxStages ? kMaxStages : s;
 }
 
 size_t pair_smem_bytes(int n_tile, int n_bundles) {
-  return size_t(pick_stages_pair(n_tile)) * kCps * (kABytes + size_t(n_tile / 2) * 128) + 1024 + 4 * kStoreWarpBytes +
+  return size_t(pick_stages_pair(n_tile)) * pick_cps(n_tile) * (kABytes + size_t(n_tile / 2) * 128) + 1024 + 4 * kStoreWarpBytes +
          sizeof(Barriers) +
          size_t(n_tile) * n_bundles * 4;
 }
 
-template <bool kDense>
+template <bool kDense, int kCps>
 cudaError_t launch_pair_t(const UmmaArgs& a, const CUtensorMap& xm, const CUtensorMap& wm, const CUtensorMap& ym,
                           int sm_count, int stages,
                           int cols, size_t smem, long long n_items, cudaStream_t stream) {
   static bool attr_done = false;
   if (!attr_done) {
-    cudaError_t e = cudaFuncSetAttribute(conv3d_umma_pair_kernel<kDense>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    cudaError_t e = cudaFuncSetAttribute(conv3d_umma_pair_kernel<kDense, kCps>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
     if (e != cudaSuccess) return e;
     attr_done = true;
   }
@@ -322,13 +325,13 @@ cudaError_t launch_pair_t(const UmmaArgs& a, const CUtensorMap& xm, const CUtens
   if (max_clusters == 0) {
     cfg.gridDim = dim3(unsigned(sm_count & ~1));
     int n = 0;
-    if (cudaOccupancyMaxActiveClusters(&n, conv3d_umma_pair_kernel<kDense>, &cfg) != cudaSuccess || n <= 0) n = sm_count / 2;
+    if (cudaOccupancyMaxActiveClusters(&n, conv3d_umma_pair_kernel<kDense, kCps>, &cfg) != cudaSuccess || n <= 0) n = sm_count / 2;
     max_clusters = n;
   }
   long long clusters = max_clusters < sm_count / 2 ? max_clusters : sm_count / 2;
   if (clusters > n_items) clusters = n_items;
   cfg.gridDim = dim3(unsigned(2 * clusters));
-  return cudaLaunchKernelEx(&cfg, conv3d_umma_pair_kernel<kDense>, xm, wm, ym, a, stages, cols);
+  return cudaLaunchKernelEx(&cfg, conv3d_umma_pair_kernel<kDense, kCps>, xm, wm, ym, a, stages, cols);
 }
 
 }  // namespace
@@ -353,8 +356,11 @@ cudaError_t launch_conv_umma_pair(const UmmaArgs& a, const void* xmap, const voi
   memcpy(&xm, xmap, sizeof(CUtensorMap));
   memcpy(&wm, wmap_half, sizeof(CUtensorMap));
   memcpy(&ym, ymap ? ymap : xmap, sizeof(CUtensorMap));
-  return a.dense ? launch_pair_t<true>(a, xm, wm, ym, sm_count, stages, cols, smem, n_items, stream)
-                 : launch_pair_t<false>(a, xm, wm, ym, sm_count, stages, cols, smem, n_items, stream);
+  if (pick_cps(a.n_tile) == 2)
+    return a.dense ? launch_pair_t<true, 2>(a, xm, wm, ym, sm_count, stages, cols, smem, n_items, stream)
+                   : launch_pair_t<false, 2>(a, xm, wm, ym, sm_count, stages, cols, smem, n_items, stream);
+  return a.dense ? launch_pair_t<true, 1>(a, xm, wm, ym, sm_count, stages, cols, smem, n_items, stream)
+                 : launch_pair_t<false, 1>(a, xm, wm, ym, sm_count, stages, cols, smem, n_items, stream);
 }
 
 }  // namespace rt3d
