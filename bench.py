@@ -141,7 +141,7 @@ def time_networks(torch, rt3d, nets, dev, iters=20):
         layers = {op.name: nets.ConvLayer(op, raw[op.name]["w"], raw[op.name]["bias"],
                                           None if mode == "dense" else raw[op.name]["mask"], 4, 4, torch.bfloat16,
                                           dense=(mode == "dense"), device=dev) for _, op in specs}
-        net = nets.C3DNet(plan, layers)
+        net = nets.C3DNet(plan, layers, fuse_pool=True)
         for batch in (1, 16):
             x = nets.to_device(synth.make_input(2, (batch, 16, 112, 112, 3)), torch.bfloat16, device=dev)
             ms = timed(nets.GraphedForward(net, x))
@@ -172,11 +172,12 @@ def time_networks(torch, rt3d, nets, dev, iters=20):
     for i, sp in enumerate(rspecs):
         L = synth.make_layer(sp, 3, i, 4, 4, "bernoulli", 0.4)
         rlayers[sp.name] = nets.ConvLayer(sp, L["w"], L["bias"], L["mask"], 4, 4, torch.bfloat16, device=dev)
-    rnet = nets.R2Plus1DNet(stem, blocks, rlayers)
+    rnet = nets.R2Plus1DNet(stem, blocks, rlayers, fuse_residual=True)
     x = nets.to_device(synth.make_input(3, (8, 16, 112, 112, 3)), torch.bfloat16, device=dev)
     ms = timed(nets.GraphedForward(rnet, x))
     out["r2plus1d_kgs_b8_clips_per_s"] = 8 / ms * 1e3
     out["r2plus1d_kgs_b8_ms"] = ms
+    out["r2plus1d_launches"] = rnet.n_launches()
     return out
 
 

@@ -156,6 +156,33 @@ rt3d_status rt3d_conv3d_dense(const rt3d_tensor* x, const rt3d_packed* w, const 
                               const rt3d_conv_params* p, rt3d_tensor* y, void* stream);
 
 /*
+ * Fused layer boundaries (the paper's framework applies "computational graph optimizations",
+ * Section 5.2, without detailing them; these two are the ones its models need).
+ *   residual  device tensor with the extents, dtype and alignment rules of the un-pooled output
+ *             (c == M), added to conv + bias BEFORE the ReLU of p->relu; NULL = none.  Must not
+ *             overlap y.  (R(2+1)D block end: y = relu(conv(x) + shortcut).)
+ *   pool_t/h/w  max-pool window applied AFTER the activation, window = stride, no padding, each
+ *             1 or 2 (1,1,1 = none); y then has extents floor(To/pool_t) x floor(Ho/pool_h) x
+ *             floor(Wo/pool_w).  (C3D: conv + ReLU + 1x2x2 or 2x2x2 pool.)
+ */
+typedef struct {
+  const rt3d_tensor* residual;
+  int32_t pool_t, pool_h, pool_w;
+} rt3d_fusion;
+
+/* rt3d_conv3d_sparse_fused - rt3d_conv3d_sparse (or the dense path for a dense handle) with the
+ * fusions above: y = pool(act(bias + conv(x, W (.) mask) + residual)).  Same argument rules; bf16
+ * results are rounded once, after the activation (pooling commutes with that rounding).
+ * RT3D_ERR_UNSUPPORTED when a fusion cannot be applied to this call (pooling needs the tensor-core
+ * kernels, tile shapes that hold whole windows and output bundles of whole 32-channel pieces); the
+ * caller then runs the steps separately.  With p->algo == RT3D_ALGO_AUTO pooling is also declined
+ * that way for layers with so few output tiles that the library would split K across SMs (the split
+ * plus a separate pool launch is the faster plan); RT3D_ALGO_UMMA fuses regardless. */
+rt3d_status rt3d_conv3d_sparse_fused(const rt3d_tensor* x, const rt3d_packed* w, const float* bias,
+                                     const rt3d_conv_params* p, const rt3d_fusion* fusion, rt3d_tensor* y,
+                                     void* stream);
+
+/*
  * rt3d_conv3d_sparse_noalloc - rt3d_conv3d_sparse for callers that must not allocate.
  * (No counterpart in the paper: this is a deployment variant of the tensor-core kernel.)
  * Some callers cannot call cudaMalloc at the point where they run a layer: code inside a

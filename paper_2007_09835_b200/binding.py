@@ -39,6 +39,11 @@ class ConvParams(ctypes.Structure):
                 ("relu", ctypes.c_int32), ("algo", ctypes.c_int32)]
 
 
+class Fusion(ctypes.Structure):
+    _fields_ = [("residual", ctypes.POINTER(Tensor)), ("pool_t", ctypes.c_int32), ("pool_h", ctypes.c_int32),
+                ("pool_w", ctypes.c_int32)]
+
+
 class PackedView(ctypes.Structure):
     _fields_ = [(k, ctypes.c_int32) for k in ("M", "N", "Kt", "Kh", "Kw", "g_m", "g_n", "P", "Q", "Ks",
                                               "dtype", "is_vanilla", "is_dense")] + \
@@ -63,6 +68,7 @@ def _load():
     lib.rt3d_packed_free.restype = None
     for name in ("rt3d_conv3d_sparse", "rt3d_conv3d_dense", "rt3d_conv3d_host", "rt3d_conv3d_sparse_noalloc"):
         getattr(lib, name).argtypes = [TP, vp, vp, CP, TP, vp]
+    lib.rt3d_conv3d_sparse_fused.argtypes = [TP, vp, vp, CP, ctypes.POINTER(Fusion), TP, vp]
     lib.rt3d_kgs_group_norms.argtypes = [vp, i, i, i, i, i, i, i, i, vp, vp]
     lib.rt3d_kgs_reweight.argtypes = [vp, ctypes.c_int64, ctypes.c_float, ctypes.c_float, vp, vp, vp]
     lib.rt3d_kgs_expand_mask.argtypes = [vp, i, i, i, i, i, i, i, vp, vp]
@@ -221,6 +227,16 @@ def rt3d_conv3d_sparse_noalloc(x: Tensor, w: Packed, bias, y: Tensor, stride=(1,
     _check(_lib.rt3d_conv3d_sparse_noalloc(ctypes.byref(x), w.handle, _bias_ptr(bias),
                                            ctypes.byref(_params(stride, pad, relu, algo)), ctypes.byref(y),
                                            _stream_ptr(stream)), "rt3d_conv3d_sparse_noalloc")
+
+
+def rt3d_conv3d_sparse_fused(x: Tensor, w: Packed, bias, y: Tensor, stride=(1, 1, 1), pad=(0, 0, 0), relu=False,
+                             residual: Tensor | None = None, pool=(1, 1, 1), algo=ALGO_AUTO, stream=None):
+    """y = pool(act(bias + conv(x) + residual)); residual: descriptor of a device tensor with the un-pooled
+    output's extents or None; pool: (1|2, 1|2, 1|2) max-pool window = stride applied after the activation."""
+    fz = Fusion(ctypes.pointer(residual) if residual is not None else None, int(pool[0]), int(pool[1]), int(pool[2]))
+    _check(_lib.rt3d_conv3d_sparse_fused(ctypes.byref(x), w.handle, _bias_ptr(bias),
+                                         ctypes.byref(_params(stride, pad, relu, algo)), ctypes.byref(fz),
+                                         ctypes.byref(y), _stream_ptr(stream)), "rt3d_conv3d_sparse_fused")
 
 
 def rt3d_conv3d_dense(x: Tensor, w: Packed, bias, y: Tensor, stride=(1, 1, 1), pad=(0, 0, 0), relu=False,

@@ -282,26 +282,60 @@ rt3d_status encode_xmap(const rt3d_tensor* x, const ConvGeom& g, const TileBox& 
   return r == CUDA_SUCCESS ? RT3D_OK : RT3D_ERR_CUDA;
 }
 
-// Output tensor map for the TMA-store epilogue: box = 32 channels x the 32 voxels one epilogue warp owns
-// (sub-box of the tile), 64-byte swizzle.  Returns false when a warp's rows are not a rectangular block
-// of voxels (then the kernels store directly).
-bool encode_ymap(const rt3d_tensor* y, const ConvGeom& g, int bw, int bh, int bt, int bn, CUtensorMap* map) {
-  if (g.M < 32 || (bw * bh * bt * bn) % 32) return false;
-  int rem = 32, sb[4] = {1, 1, 1, 1};
+// Block of 32 output voxels (w, h, t, n extents) that one epilogue warp owns in a box of bw x bh x bt x bn
+// voxels; false when 32 consecutive box rows are not a rectangular block.
+bool warp_block(int bw, int bh, int bt, int bn, int sb[4]) {
+  if ((bw * bh * bt * bn) % 32) return false;
+  int rem = 32;
   const int dims_box[4] = {bw, bh, bt, bn};
-  for (int i = 0; i < 4 && rem > 1; ++i) {
+  for (int i = 0; i < 4; ++i) {
+    sb[i] = 1;
+    if (rem == 1) continue;
     const int d = dims_box[i];
     if (d >= rem) { if (d % rem) return false; sb[i] = rem; rem = 1; }
     else { if (rem % d) return false; sb[i] = d; rem /= d; }
   }
-  if (rem != 1) return false;
-  const cuuint64_t cs = cuuint64_t(g.ycs) * 2;
-  cuuint64_t dims[5] = {cuuint64_t(g.M), cuuint64_t(g.Wo), cuuint64_t(g.Ho), cuuint64_t(g.To), cuuint64_t(g.n)};
-  cuuint64_t strides[4] = {cs, cs * g.Wo, cs * g.Wo * g.Ho, cs * g.Wo * g.Ho * g.To};
-  cuuint32_t bx[5] = {32, cuuint32_t(sb[0]), cuuint32_t(sb[1]), cuuint32_t(sb[2]), cuuint32_t(sb[3])};
+  return rem == 1;
+}
+
+// Output tensor map for the TMA-store epilogue: box = 32 channels x the voxels one epilogue warp stores per
+// piece (its block of 32 voxels, divided by the fused pooling window), 64-byte swizzle.  The tensor is y,
+// i.e. already the pooled one when pooling is fused.
+bool encode_ymap(const rt3d_tensor* y, const int sb[4], int pw, int ph, int pt, CUtensorMap* map) {
+  if (y->c < 32 || sb[0] % pw || sb[1] % ph || sb[2] % pt) return false;
+  const cuuint64_t cs = cuuint64_t(y->c_stride) * 2;
+  cuuint64_t dims[5] = {cuuint64_t(y->c), cuuint64_t(y->w), cuuint64_t(y->h), cuuint64_t(y->t), cuuint64_t(y->n)};
+  cuuint64_t strides[4] = {cs, cs * y->w, cs * y->w * y->h, cs * y->w * y->h * y->t};
+  cuuint32_t bx[5] = {32, cuuint32_t(sb[0] / pw), cuuint32_t(sb[1] / ph), cuuint32_t(sb[2] / pt), cuuint32_t(sb[3])};
   cuuint32_t estr[5] = {1, 1, 1, 1, 1};
   return g_encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, y->data, dims, strides, bx, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                   CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// Box for a call with fused pooling: fewest tiles among the boxes whose extents and whose per-warp block
+// are multiples of the pooling window (every window then lies inside one warp's 32 voxels).
+bool choose_box_pool(const ConvGeom& g, int pw, int ph, int pt, TileBox* out, int sb_out[4]) {
+  long long best_tiles = -1;
+  for (int bw = pw; bw <= kTileM && bw <= round_up(g.Wo, pw); bw += pw) {
+    if (bw * g.sw > 256) break;
+    for (int bh = ph; bw * bh <= kTileM && bh <= round_up(g.Ho, ph); bh += ph) {
+      if (bh * g.sh > 256) break;
+      for (int bt = pt; bw * bh * bt <= kTileM && bt <= round_up(g.To, pt); bt += pt) {
+        if (bt * g.st > 256) break;
+        int bn = kTileM / (bw * bh * bt);
+        if (bn > g.n) bn = g.n;
+        int sb[4];
+        if (!warp_block(bw, bh, bt, bn, sb) || sb[0] % pw || sb[1] % ph || sb[2] % pt) continue;
+        const long long tiles = (long long)ceil_div(g.n, bn) * ceil_div(g.To, bt) * ceil_div(g.Ho, bh) * ceil_div(g.Wo, bw);
+        if (best_tiles < 0 || tiles < best_tiles || (tiles == best_tiles && bw > out->bw)) {
+          best_tiles = tiles;
+          *out = TileBox{bn, bt, bh, bw};
+          for (int i = 0; i < 4; ++i) sb_out[i] = sb[i];
+        }
+      }
+    }
+  }
+  return best_tiles > 0;
 }
 
 // Small-C_in kernel: bf16, C_in <= 8 stored at pitch 8, spatial strides <= 4, M <= 256.
@@ -320,7 +354,8 @@ bool smallc_eligible(const DeviceState* d, rt3d_packed* w, const rt3d_tensor* x,
 }
 
 rt3d_status launch_smallc(rt3d_packed* w, DeviceBlob* blob, const DeviceState* d, const SmallCLayout* L,
-                          const rt3d_tensor* x, const ConvGeom& g, const float* bias, rt3d_tensor* y, cudaStream_t st) {
+                          const rt3d_tensor* x, const ConvGeom& g, const float* bias, rt3d_tensor* y, cudaStream_t st,
+                          const void* residual, int rcs, int pool_h, int pool_w) {
   DeviceBlob::SmallC* sc = nullptr;
   {
     std::lock_guard<std::mutex> lock(w->mu);
@@ -346,6 +381,8 @@ rt3d_status launch_smallc(rt3d_packed* w, DeviceBlob* blob, const DeviceState* d
   a.img_w = L->img_w; a.phase_bytes = L->img_w * L->img_h * L->img_t * 16;
   a.tiles_h = ceil_div(g.Ho, kSmallCTileH); a.tiles_w = ceil_div(g.Wo, kSmallCTileW);
   a.tmem_cols = 0;
+  a.residual = residual; a.rcs = rcs;
+  a.pool_t = 1; a.pool_h = pool_h; a.pool_w = pool_w;
   a.wimg = sc->wimg; a.pair_off = sc->pairs;
   a.bias = bias; a.y = y->data; a.sched = d->sched;
   // input as [n][t][h][w][8]: one box = one phase image of a 1 x 16 x 8 output tile (every sh-th row and
@@ -360,20 +397,43 @@ rt3d_status launch_smallc(rt3d_packed* w, DeviceBlob* blob, const DeviceState* d
                CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
     return RT3D_ERR_CUDA;
   CUtensorMap ymap;
-  a.store_tma = encode_ymap(y, g, kSmallCTileW, kSmallCTileH, 1, 1, &ymap) ? 1 : 0;
+  const int sb[4] = {kSmallCTileW, 4, 1, 1};          // a warp owns 4 rows of 8 voxels of the 16 x 8 tile
+  a.store_tma = encode_ymap(y, sb, pool_w, pool_h, 1, &ymap) ? 1 : 0;
+  if (!a.store_tma && pool_h * pool_w > 1) return RT3D_ERR_UNSUPPORTED;
   if (launch_conv_umma_smallc(a, &xmap, a.store_tma ? &ymap : nullptr, d->sm_count, st) != cudaSuccess) return RT3D_ERR_CUDA;
   g_launches.fetch_add(1);
   return RT3D_OK;
 }
 
 rt3d_status conv_impl(const rt3d_tensor* x, const rt3d_packed* wc, const float* bias, const rt3d_conv_params* p,
-                      rt3d_tensor* y, void* stream, bool dense_entry) {
+                      rt3d_tensor* y, void* stream, bool dense_entry, const rt3d_fusion* fz = nullptr) {
   ConvGeom g;
   if (!y) return RT3D_ERR_INVALID_ARG;
-  rt3d_status s = make_geom(x, wc, p, y, &g);
+  const bool pooled = fz && (fz->pool_t != 1 || fz->pool_h != 1 || fz->pool_w != 1);
+  if (fz && (fz->pool_t < 1 || fz->pool_t > 2 || fz->pool_h < 1 || fz->pool_h > 2 || fz->pool_w < 1 || fz->pool_w > 2))
+    return RT3D_ERR_INVALID_ARG;
+  const int pl_t = fz ? fz->pool_t : 1, pl_h = fz ? fz->pool_h : 1, pl_w = fz ? fz->pool_w : 1;
+  rt3d_status s = make_geom(x, wc, p, pooled ? nullptr : y, &g);
   if (s != RT3D_OK) return s;
+  if (pooled) {                     // y holds the pooled tensor; g keeps the extents of the convolution output
+    if ((s = check_tensor(y)) != RT3D_OK) return s;
+    if (y->n != g.n || y->t != g.To / pl_t || y->h != g.Ho / pl_h || y->w != g.Wo / pl_w || y->c != wc->M ||
+        y->dtype != wc->dtype || y->t < 1 || y->h < 1 || y->w < 1)
+      return RT3D_ERR_SHAPE;
+    if (fz->residual) return RT3D_ERR_UNSUPPORTED;
+    g.ycs = y->c_stride;
+  }
   if ((s = check_alignment(x)) != RT3D_OK || (s = check_alignment(y)) != RT3D_OK) return s;
   if (overlaps(x, y)) return RT3D_ERR_INVALID_ARG;
+  const rt3d_tensor* res = fz ? fz->residual : nullptr;
+  if (res) {
+    if ((s = check_tensor(res)) != RT3D_OK || (s = check_alignment(res)) != RT3D_OK) return s;
+    if (res->n != g.n || res->t != g.To || res->h != g.Ho || res->w != g.Wo || res->c != g.M || res->dtype != wc->dtype)
+      return RT3D_ERR_SHAPE;
+    if (overlaps(res, y)) return RT3D_ERR_INVALID_ARG;
+  }
+  const void* res_data = res ? res->data : nullptr;
+  const int res_pitch = res ? res->c_stride : 0;
   if (dense_entry && !wc->is_dense) return RT3D_ERR_INVALID_ARG;
   rt3d_packed* w = const_cast<rt3d_packed*>(wc);
   DeviceState* d = nullptr;
@@ -390,24 +450,39 @@ rt3d_status conv_impl(const rt3d_tensor* x, const rt3d_packed* wc, const float* 
   const bool use_umma = p->algo == RT3D_ALGO_UMMA || p->algo == RT3D_ALGO_UMMA_PAIR ||
                         (p->algo == RT3D_ALGO_AUTO && can_umma);
   if (!use_umma) {
+    if (pooled) return RT3D_ERR_UNSUPPORTED;
     cudaError_t e = launch_conv_simt(w->dtype, g, x->data, y->data, blob->group_ptr, blob->pos_idx, blob->tiles, bias,
-                                     w->g_m, w->g_n, w->P, w->Q, dense_entry, st);
+                                     w->g_m, w->g_n, w->P, w->Q, dense_entry, res_data, res_pitch, st);
     if (e != cudaSuccess) return RT3D_ERR_CUDA;
     g_launches.fetch_add(1);
     return RT3D_OK;
   }
 
   const SmallCLayout* SL = nullptr;
-  if (p->algo != RT3D_ALGO_UMMA_PAIR && smallc_eligible(d, w, x, y, p, &SL))
-    return launch_smallc(w, blob, d, SL, x, g, bias, y, st);
+  if (p->algo != RT3D_ALGO_UMMA_PAIR && (!pooled || pl_t == 1) && smallc_eligible(d, w, x, y, p, &SL))
+    return launch_smallc(w, blob, d, SL, x, g, bias, y, st, res_data, res_pitch, pl_h, pl_w);
 
   UmmaArgs a;
   a.g = g;
-  a.box = choose_box(g);
+  int sb[4] = {1, 1, 1, 1};
+  bool rect;
+  if (pooled) {
+    if (!choose_box_pool(g, pl_w, pl_h, pl_t, &a.box, sb)) return RT3D_ERR_UNSUPPORTED;
+    rect = true;
+  } else {
+    a.box = choose_box(g);
+    rect = warp_block(a.box.bw, a.box.bh, a.box.bt, a.box.bn, sb);
+  }
+  a.pool_t = pl_t; a.pool_h = pl_h; a.pool_w = pl_w; a.sbw = sb[0]; a.sbh = sb[1];
   a.tiles_n = ceil_div(g.n, a.box.bn); a.tiles_t = ceil_div(g.To, a.box.bt);
   a.tiles_h = ceil_div(g.Ho, a.box.bh); a.tiles_w = ceil_div(g.Wo, a.box.bw);
   const long long m_tiles = (long long)a.tiles_n * a.tiles_t * a.tiles_h * a.tiles_w;
   UmmaPlan plan = pick_plan(w, m_tiles, d->sm_count);
+  if (pooled) {                     // pooling lives in the TMA-store epilogue, which a K split does not use
+    // A layer this small is faster split over K and pooled by a second launch: AUTO declines the fusion.
+    if (p->algo == RT3D_ALGO_AUTO && plan.n_splits > 1) return RT3D_ERR_UNSUPPORTED;
+    plan.n_splits = 1;
+  }
   // CTA pairs: two tiles per MMA.  Worth it when every pair has work; forced by RT3D_ALGO_UMMA_PAIR.
   bool use_pair = false;
   if (p->algo == RT3D_ALGO_UMMA_PAIR) {
@@ -419,6 +494,7 @@ rt3d_status conv_impl(const rt3d_tensor* x, const rt3d_packed* wc, const float* 
              m_tiles * ceil_div(w->M, plan.n_tile) >= d->sm_count) {
     use_pair = true;
   }
+  if (pooled && plan.n_tile % 32) return RT3D_ERR_UNSUPPORTED;      // pooled rows leave as whole 32-channel pieces
   const UmmaLayout* L = get_umma_layout(w, plan.n_tile);
   if (!L) return RT3D_ERR_UNSUPPORTED;
   DeviceBlob::Umma* u = nullptr;
@@ -428,6 +504,7 @@ rt3d_status conv_impl(const rt3d_tensor* x, const rt3d_packed* wc, const float* 
   a.steps_dense = w->Ks * L->n_chunks;
   a.step_ptr = u->step_ptr; a.steps = u->steps;
   a.bias = bias; a.y = y->data; a.sched = d->sched;
+  a.residual = res_data; a.rcs = res_pitch;
   a.n_splits = plan.n_splits; a.scratch = nullptr; a.counters = nullptr;
   if (a.n_splits > 1) {
     // split-K workspace of this handle on this device: partial tiles + per-warp arrival counters
@@ -453,7 +530,8 @@ rt3d_status conv_impl(const rt3d_tensor* x, const rt3d_packed* wc, const float* 
   CUtensorMap xmap;
   if ((s = encode_xmap(x, g, a.box, &xmap)) != RT3D_OK) return s;
   CUtensorMap ymap;
-  a.store_tma = (a.n_splits == 1 && encode_ymap(y, g, a.box.bw, a.box.bh, a.box.bt, a.box.bn, &ymap)) ? 1 : 0;
+  a.store_tma = (a.n_splits == 1 && rect && encode_ymap(y, sb, pl_w, pl_h, pl_t, &ymap)) ? 1 : 0;
+  if (pooled && !a.store_tma) return RT3D_ERR_UNSUPPORTED;
   const void* ym = a.store_tma ? &ymap : nullptr;
   cudaError_t e = use_pair ? launch_conv_umma_pair(a, &xmap, u->wmap_half, ym, d->sm_count, st)
                            : launch_conv_umma(a, &xmap, u->wmap, ym, d->sm_count, st);
@@ -474,6 +552,13 @@ rt3d_status rt3d_conv3d_sparse(const rt3d_tensor* x, const rt3d_packed* w, const
 rt3d_status rt3d_conv3d_dense(const rt3d_tensor* x, const rt3d_packed* w, const float* bias,
                               const rt3d_conv_params* p, rt3d_tensor* y, void* stream) {
   return conv_impl(x, w, bias, p, y, stream, true);
+}
+
+rt3d_status rt3d_conv3d_sparse_fused(const rt3d_tensor* x, const rt3d_packed* w, const float* bias,
+                                     const rt3d_conv_params* p, const rt3d_fusion* fusion, rt3d_tensor* y,
+                                     void* stream) {
+  if (!fusion || !w) return RT3D_ERR_INVALID_ARG;
+  return conv_impl(x, w, bias, p, y, stream, w->is_dense != 0, fusion);
 }
 
 rt3d_status rt3d_conv3d_host(const rt3d_tensor* x, rt3d_packed* w, const float* bias, const rt3d_conv_params* p,
@@ -722,6 +807,7 @@ rt3d_status rt3d_conv3d_sparse_noalloc(const rt3d_tensor* x, const rt3d_packed* 
   if (splits > a.steps_dense / 8) splits = a.steps_dense / 8;
   if (splits < 1) splits = 1;
   a.n_splits = int(splits);
+  a.residual = nullptr; a.rcs = 0;
   a.scratch = nullptr; a.counters = nullptr;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (a.n_splits > 1) {
@@ -736,7 +822,10 @@ rt3d_status rt3d_conv3d_sparse_noalloc(const rt3d_tensor* x, const rt3d_packed* 
   CUtensorMap xmap;
   if ((s = encode_xmap(x, g, a.box, &xmap)) != RT3D_OK) return s;
   CUtensorMap ymap;
-  a.store_tma = (a.n_splits == 1 && encode_ymap(y, g, a.box.bw, a.box.bh, a.box.bt, a.box.bn, &ymap)) ? 1 : 0;
+  int sb[4];
+  a.pool_t = a.pool_h = a.pool_w = 1; a.sbw = a.sbh = 1;
+  a.store_tma = (a.n_splits == 1 && warp_block(a.box.bw, a.box.bh, a.box.bt, a.box.bn, sb) &&
+                 encode_ymap(y, sb, 1, 1, 1, &ymap)) ? 1 : 0;
   if (launch_conv_umma(a, &xmap, u->wmap, a.store_tma ? &ymap : nullptr, d->sm_count, st) != cudaSuccess) return RT3D_ERR_CUDA;
   g_launches.fetch_add(1);
   return RT3D_OK;

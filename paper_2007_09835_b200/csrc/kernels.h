@@ -18,10 +18,11 @@ struct ConvGeom {
 };
 
 // CUDA-core kernel driven by the canonical packed arrays.  dtype: 0 fp32, 1 bf16.
+// residual: tensor of the output's extents and dtype (pitch rcs) added before the ReLU, or nullptr.
 cudaError_t launch_conv_simt(int dtype, const ConvGeom& g, const void* x, void* y,
                              const int32_t* group_ptr, const uint16_t* pos_idx, const void* tiles,
                              const float* bias, int g_m, int g_n, int P, int Q, bool dense,
-                             cudaStream_t stream);
+                             const void* residual, int rcs, cudaStream_t stream);
 
 cudaError_t launch_maxpool3d(int dtype, const void* x, int n, int t, int h, int w, int c, int xcs,
                              int kt, int kh, int kw, int st, int sh, int sw, int pt, int ph, int pw,
@@ -47,6 +48,10 @@ struct UmmaArgs {
   void* y;
   int32_t* sched;                           // device [8]: [2] = error word set by a bounded wait that gave up
   int store_tma;                            // 1: epilogue stores go through shared memory + TMA (needs ymap)
+  const void* residual;                     // device bf16 tensor of the output's extents added before the ReLU, or nullptr
+  int rcs;                                  // its channel pitch
+  int pool_t, pool_h, pool_w;               // fused max-pool window (1,1,1 = none); needs store_tma, ymap over the pooled tensor
+  int sbw, sbh;                             // extents along w, h of the block of 32 voxels an epilogue warp owns
   int n_splits;                             // K splits per output tile (1 = none)
   float* scratch;                           // device, split-K partial tiles [tile][split][128][n_tile] (n_splits > 1)
   int32_t* counters;                        // device, [tiles * 4] arrival counters, zero between launches
@@ -73,6 +78,9 @@ struct SmallCArgs {
   int tiles_h, tiles_w;               // 16 x 8 output tiles per frame
   int tmem_cols;                      // filled in by the launcher
   int store_tma;                      // 1: TMA-store epilogue (needs ymap)
+  const void* residual;               // device bf16 tensor added before the ReLU, or nullptr
+  int rcs;                            // its channel pitch
+  int pool_t, pool_h, pool_w;         // fused max-pool window (1,1,1 = none; pool_t must be 1); needs store_tma
   const void* wimg;                   // device: [n_pairs][2][n_pad/8][8][8] bf16
   const int32_t* pair_off;            // device: [n_pairs][2] byte offsets inside the staged images
   const float* bias;

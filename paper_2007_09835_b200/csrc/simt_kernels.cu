@@ -29,7 +29,7 @@ __global__ void __launch_bounds__(kThreads)
 conv3d_kgs_simt_kernel(ConvGeom g, const T* __restrict__ x, T* __restrict__ y,
                        const int32_t* __restrict__ group_ptr, const uint16_t* __restrict__ pos_idx,
                        const T* __restrict__ tiles, const float* __restrict__ bias,
-                       int g_m_rt, int g_n_rt, int Q, long long total_voxels) {
+                       int g_m_rt, int g_n_rt, int Q, long long total_voxels, const T* __restrict__ residual, int rcs) {
   constexpr int MAXM = GM ? GM : 8;
   constexpr int MAXN = GN ? GN : 8;
   const int g_m = GM ? GM : g_m_rt;
@@ -82,6 +82,7 @@ conv3d_kgs_simt_kernel(ConvGeom g, const T* __restrict__ x, T* __restrict__ y,
     const int m = p * g_m + i;
     if (i < g_m && m < g.M) {
       float r = acc[i] + (bias ? bias[m] : 0.f);
+      if (residual) r += to_f32<T>(residual[v * rcs + m]);
       if (g.relu) r = fmaxf(r, 0.f);
       yp[i] = from_f32<T>(r);
     }
@@ -91,7 +92,7 @@ conv3d_kgs_simt_kernel(ConvGeom g, const T* __restrict__ x, T* __restrict__ y,
 template <typename T, bool DENSE>
 cudaError_t launch_conv_t(const ConvGeom& g, const void* x, void* y, const int32_t* group_ptr,
                           const uint16_t* pos_idx, const void* tiles, const float* bias, int g_m, int g_n,
-                          int P, int Q, cudaStream_t stream) {
+                          int P, int Q, const void* residual, int rcs, cudaStream_t stream) {
   const long long total = (long long)g.n * g.To * g.Ho * g.Wo;
   if (total == 0) return cudaSuccess;
   dim3 grid((unsigned)((total + kThreads - 1) / kThreads), (unsigned)P);
@@ -99,7 +100,7 @@ cudaError_t launch_conv_t(const ConvGeom& g, const void* x, void* y, const int32
   T* yt = static_cast<T*>(y);
   const T* tt = static_cast<const T*>(tiles);
 #define RT3D_LAUNCH(GM_, GN_) \
-  conv3d_kgs_simt_kernel<T, GM_, GN_, DENSE><<<grid, kThreads, 0, stream>>>(g, xt, yt, group_ptr, pos_idx, tt, bias, g_m, g_n, Q, total)
+  conv3d_kgs_simt_kernel<T, GM_, GN_, DENSE><<<grid, kThreads, 0, stream>>>(g, xt, yt, group_ptr, pos_idx, tt, bias, g_m, g_n, Q, total, static_cast<const T*>(residual), rcs)
   if (g_m == 4 && g_n == 4) RT3D_LAUNCH(4, 4);
   else if (g_m == 8 && g_n == 4) RT3D_LAUNCH(8, 4);
   else if (g_m == 8 && g_n == 8) RT3D_LAUNCH(8, 8);
@@ -214,12 +215,12 @@ __global__ void add_relu_bf16x8_kernel(const uint4* __restrict__ a, int acs8, co
 
 cudaError_t launch_conv_simt(int dtype, const ConvGeom& g, const void* x, void* y, const int32_t* group_ptr,
                              const uint16_t* pos_idx, const void* tiles, const float* bias, int g_m, int g_n,
-                             int P, int Q, bool dense, cudaStream_t stream) {
+                             int P, int Q, bool dense, const void* residual, int rcs, cudaStream_t stream) {
   if (dtype == 0)
-    return dense ? launch_conv_t<float, true>(g, x, y, group_ptr, pos_idx, tiles, bias, g_m, g_n, P, Q, stream)
-                 : launch_conv_t<float, false>(g, x, y, group_ptr, pos_idx, tiles, bias, g_m, g_n, P, Q, stream);
-  return dense ? launch_conv_t<__nv_bfloat16, true>(g, x, y, group_ptr, pos_idx, tiles, bias, g_m, g_n, P, Q, stream)
-               : launch_conv_t<__nv_bfloat16, false>(g, x, y, group_ptr, pos_idx, tiles, bias, g_m, g_n, P, Q, stream);
+    return dense ? launch_conv_t<float, true>(g, x, y, group_ptr, pos_idx, tiles, bias, g_m, g_n, P, Q, residual, rcs, stream)
+                 : launch_conv_t<float, false>(g, x, y, group_ptr, pos_idx, tiles, bias, g_m, g_n, P, Q, residual, rcs, stream);
+  return dense ? launch_conv_t<__nv_bfloat16, true>(g, x, y, group_ptr, pos_idx, tiles, bias, g_m, g_n, P, Q, residual, rcs, stream)
+               : launch_conv_t<__nv_bfloat16, false>(g, x, y, group_ptr, pos_idx, tiles, bias, g_m, g_n, P, Q, residual, rcs, stream);
 }
 
 cudaError_t launch_maxpool3d(int dtype, const void* x, int n, int t, int h, int w, int c, int xcs,

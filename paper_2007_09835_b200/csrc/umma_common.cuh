@@ -140,14 +140,31 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
 // Epilogue of NC (16 or 32) accumulator columns of one output voxel: + bias (from shared memory),
 // optional ReLU, round to bf16, store.  `valid` = number of real output channels among the NC
 // (>= NC: 16-byte vector stores; fewer: scalar tail, channels beyond are left untouched).
+// `res`: this voxel's residual channels starting at the same channel as v[0] (nullptr: none), of which
+// `res_avail` may be read (the channel pitch bounds the vector loads).
 template <int NC>
 __device__ __forceinline__ void epilogue_cols(const uint32_t* v, const float* bias_s, int relu,
-                                              __nv_bfloat16* dst, int valid) {
+                                              __nv_bfloat16* dst, int valid, const __nv_bfloat16* res, int res_avail) {
   float f[NC];
 #pragma unroll
-  for (int q = 0; q < NC; ++q) {
-    f[q] = __uint_as_float(v[q]) + bias_s[q];
-    if (relu) f[q] = fmaxf(f[q], 0.f);
+  for (int q = 0; q < NC; ++q) f[q] = __uint_as_float(v[q]) + bias_s[q];
+  if (res != nullptr) {
+#pragma unroll
+    for (int k = 0; k < NC / 8; ++k) {
+      if (8 * k < res_avail) {
+        const uint4 rv = *reinterpret_cast<const uint4*>(res + 8 * k);
+        const __nv_bfloat162* pr = reinterpret_cast<const __nv_bfloat162*>(&rv);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const float2 t = __bfloat1622float2(pr[e]);
+          f[8 * k + 2 * e] += t.x; f[8 * k + 2 * e + 1] += t.y;
+        }
+      }
+    }
+  }
+  if (relu) {
+#pragma unroll
+    for (int q = 0; q < NC; ++q) f[q] = fmaxf(f[q], 0.f);
   }
   if (valid >= NC) {
 #pragma unroll
@@ -166,8 +183,11 @@ __device__ __forceinline__ void epilogue_cols(const uint32_t* v, const float* bi
 // One voxel row of a finished accumulator tile: columns [0, n_cols) of the TMEM buffer at `taddr`
 // hold output channels m_base.. ; channels >= M are dropped.  Warp-uniform control flow around the
 // TMEM loads (.sync.aligned); `in_range` may differ per lane.
+// `res_row`: the voxel's residual row at channel m_base (nullptr: none); `res_pitch_left` = channels from
+// m_base to the end of the residual tensor's channel pitch.
 __device__ __forceinline__ void epilogue_row(uint32_t taddr, int n_cols, bool has_acc, bool in_range,
-                                             const float* bias_s, int relu, __nv_bfloat16* dst, int m_base, int M) {
+                                             const float* bias_s, int relu, __nv_bfloat16* dst, int m_base, int M,
+                                             const __nv_bfloat16* res_row = nullptr, int res_pitch_left = 0) {
   for (int col = 0; col < n_cols; col += 32) {
     const int m0 = m_base + col;
     if (m0 >= M) break;
@@ -181,8 +201,9 @@ __device__ __forceinline__ void epilogue_row(uint32_t taddr, int n_cols, bool ha
       for (int q = 0; q < 32; ++q) v[q] = 0u;
     }
     if (!in_range) continue;
-    if (wide) epilogue_cols<32>(v, bias_s + m0, relu, dst + col, M - m0);
-    else epilogue_cols<16>(v, bias_s + m0, relu, dst + col, M - m0);
+    const __nv_bfloat16* res = res_row ? res_row + col : nullptr;
+    if (wide) epilogue_cols<32>(v, bias_s + m0, relu, dst + col, M - m0, res, res_pitch_left - col);
+    else epilogue_cols<16>(v, bias_s + m0, relu, dst + col, M - m0, res, res_pitch_left - col);
   }
 }
 
@@ -203,6 +224,14 @@ struct TmaStore {
   uint32_t piece;             // pieces issued so far by this warp
 };
 
+// Fused max-pool (window = stride = 1 or 2 per axis) over the 32 voxels of an epilogue warp, which form a
+// block of sbw x sbh x sbt(...) voxels whose extents are multiples of the window: lane -> (w, h, t) inside
+// the block, partner lanes differ by 1, sbw and sbw*sbh.
+struct PoolLanes {
+  int pw, ph, pt;             // window
+  int sbw, sbh;               // block extents along w and h (lane = (t*sbh + h)*sbw + w)
+};
+
 __device__ __forceinline__ void tma_store_5d(const CUtensorMap* map, uint32_t src, int c0, int c1, int c2, int c3, int c4) {
   asm volatile("cp.async.bulk.tensor.5d.global.shared::cta.tile.bulk_group [%0, {%2, %3, %4, %5, %6}], [%1];"
                ::"l"(reinterpret_cast<uint64_t>(map)), "r"(src), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4)
@@ -216,24 +245,78 @@ __device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bu
 // 32 accumulator columns of this thread's row -> bias, ReLU, bf16 -> staging buffer -> TMA box store of
 // channels [m0, m0+32) x the warp's 32 voxels.
 __device__ __forceinline__ void epilogue_piece_tma(const uint32_t* v, const float* bias_s, int relu, int m0, int lane,
-                                                   TmaStore& ts) {
+                                                   TmaStore& ts, const __nv_bfloat16* res, int res_avail,
+                                                   const PoolLanes* pool) {
+  float f[32];
+#pragma unroll
+  for (int q = 0; q < 32; ++q) f[q] = __uint_as_float(v[q]) + bias_s[q];
+  if (res != nullptr) {
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      if (8 * k < res_avail) {
+        const uint4 rv = *reinterpret_cast<const uint4*>(res + 8 * k);
+        const __nv_bfloat162* pr = reinterpret_cast<const __nv_bfloat162*>(&rv);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const float2 t = __bfloat1622float2(pr[e]);
+          f[8 * k + 2 * e] += t.x; f[8 * k + 2 * e + 1] += t.y;
+        }
+      }
+    }
+  }
   uint4 o[4];
   __nv_bfloat162* po = reinterpret_cast<__nv_bfloat162*>(o);
 #pragma unroll
   for (int q = 0; q < 16; ++q) {
-    float a = __uint_as_float(v[2 * q]) + bias_s[2 * q], b = __uint_as_float(v[2 * q + 1]) + bias_s[2 * q + 1];
+    float a = f[2 * q], b = f[2 * q + 1];
     if (relu) { a = fmaxf(a, 0.f); b = fmaxf(b, 0.f); }
     po[q] = __floats2bfloat162_rn(a, b);
+  }
+  // optional max-pool: after the (monotonic) activation and bf16 rounding, so it equals pooling the stored tensor
+  int out_row = lane;
+  bool writer = true;
+  if (pool != nullptr) {
+    const int w = lane % pool->sbw, h = (lane / pool->sbw) % pool->sbh, t = lane / (pool->sbw * pool->sbh);
+    uint32_t* u = reinterpret_cast<uint32_t*>(o);
+    if (pool->pw == 2) {
+      const int src = lane ^ 1;
+#pragma unroll
+      for (int q = 0; q < 16; ++q) {
+        const uint32_t other = __shfl_sync(0xffffffffu, u[q], src);
+        po[q] = __hmax2(po[q], *reinterpret_cast<const __nv_bfloat162*>(&other));
+      }
+    }
+    if (pool->ph == 2) {
+      const int src = (h & 1) ? lane - pool->sbw : lane + pool->sbw;
+#pragma unroll
+      for (int q = 0; q < 16; ++q) {
+        const uint32_t other = __shfl_sync(0xffffffffu, u[q], src);
+        po[q] = __hmax2(po[q], *reinterpret_cast<const __nv_bfloat162*>(&other));
+      }
+    }
+    if (pool->pt == 2) {
+      const int plane = pool->sbw * pool->sbh;
+      const int src = (t & 1) ? lane - plane : lane + plane;
+#pragma unroll
+      for (int q = 0; q < 16; ++q) {
+        const uint32_t other = __shfl_sync(0xffffffffu, u[q], src);
+        po[q] = __hmax2(po[q], *reinterpret_cast<const __nv_bfloat162*>(&other));
+      }
+    }
+    writer = (w % pool->pw == 0) && (h % pool->ph == 0) && (t % pool->pt == 0);
+    out_row = ((t / pool->pt) * (pool->sbh / pool->ph) + h / pool->ph) * (pool->sbw / pool->pw) + w / pool->pw;
   }
   const uint32_t buf = ts.smem + (ts.piece & 1u) * kStoreStageBytes;
   if (lane == 0) tma_store_wait_read_1();          // the store issued two pieces ago has read this buffer
   __syncwarp();
-  const uint32_t row = buf + uint32_t(lane) * 64u;
-  const uint32_t sw = (uint32_t(lane) >> 1) & 3u;  // 64-byte swizzle: 16-byte chunk index ^= address bits 7..8
+  const uint32_t row = buf + uint32_t(out_row) * 64u;
+  const uint32_t sw = (uint32_t(out_row) >> 1) & 3u;  // 64-byte swizzle: 16-byte chunk index ^= address bits 7..8
+  if (writer) {
 #pragma unroll
-  for (uint32_t k = 0; k < 4; ++k)
-    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(row + ((k ^ sw) << 4)), "r"(o[k].x), "r"(o[k].y),
-                 "r"(o[k].z), "r"(o[k].w) : "memory");
+    for (uint32_t k = 0; k < 4; ++k)
+      asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(row + ((k ^ sw) << 4)), "r"(o[k].x), "r"(o[k].y),
+                   "r"(o[k].z), "r"(o[k].w) : "memory");
+  }
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   __syncwarp();
   if (lane == 0) tma_store_5d(ts.map, buf, m0, ts.c1, ts.c2, ts.c3, ts.c4);
@@ -245,7 +328,9 @@ __device__ __forceinline__ void epilogue_piece_tma(const uint32_t* v, const floa
 // directly.  `warp_rows_valid`: this warp's 32 rows belong to the tile (warp-uniform).
 __device__ __forceinline__ void epilogue_row_tma(uint32_t taddr, int n_cols, bool has_acc, bool warp_rows_valid,
                                                  bool in_range, const float* bias_s, int relu, __nv_bfloat16* dst,
-                                                 int m_base, int M, int lane, TmaStore& ts) {
+                                                 int m_base, int M, int lane, TmaStore& ts,
+                                                 const __nv_bfloat16* res_row = nullptr, int res_pitch_left = 0,
+                                                 const PoolLanes* pool = nullptr) {
   for (int col = 0; col < n_cols; col += 32) {
     const int m0 = m_base + col;
     if (m0 >= M) break;
@@ -258,10 +343,11 @@ __device__ __forceinline__ void epilogue_row_tma(uint32_t taddr, int n_cols, boo
 #pragma unroll
       for (int q = 0; q < 32; ++q) v[q] = 0u;
     }
+    const __nv_bfloat16* res = (res_row && in_range) ? res_row + col : nullptr;
     if (wide) {
-      if (warp_rows_valid) epilogue_piece_tma(v, bias_s + m0, relu, m0, lane, ts);
+      if (warp_rows_valid) epilogue_piece_tma(v, bias_s + m0, relu, m0, lane, ts, res, res_pitch_left - col, pool);
     } else if (in_range) {
-      epilogue_cols<16>(v, bias_s + m0, relu, dst + col, M - m0);
+      epilogue_cols<16>(v, bias_s + m0, relu, dst + col, M - m0, res, res_pitch_left - col);
     }
   }
 }

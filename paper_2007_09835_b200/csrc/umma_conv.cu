@@ -81,7 +81,8 @@ __device__ __forceinline__ void store_partial_row(uint32_t taddr, int n_cols, bo
 // for one output voxel; `part0` points at this thread's row of column 0 of split 0.
 template <int NC>
 __device__ __forceinline__ void reduce_partial_cols(const float* part0, size_t split_stride, int n_splits,
-                                                    const float* bias_s, int relu, __nv_bfloat16* dst, int valid) {
+                                                    const float* bias_s, int relu, __nv_bfloat16* dst, int valid,
+                                                    const __nv_bfloat16* res, int res_avail) {
   float acc[NC];
 #pragma unroll
   for (int q = 0; q < NC; ++q) acc[q] = 0.f;
@@ -103,19 +104,20 @@ __device__ __forceinline__ void reduce_partial_cols(const float* part0, size_t s
   uint32_t v[NC];
 #pragma unroll
   for (int q = 0; q < NC; ++q) v[q] = __float_as_uint(acc[q]);
-  epilogue_cols<NC>(v, bias_s, relu, dst, valid);
+  epilogue_cols<NC>(v, bias_s, relu, dst, valid, res, res_avail);
 }
 
 __device__ __forceinline__ void reduce_partial_row(const float* part0, size_t split_stride, int n_splits, int n_cols,
                                                    bool in_range, const float* bias_s, int relu, __nv_bfloat16* dst,
-                                                   int m_base, int M) {
+                                                   int m_base, int M, const __nv_bfloat16* res_row, int res_left) {
   if (!in_range) return;
   for (int col = 0; col < n_cols; col += 32) {
     const int m0 = m_base + col;
     if (m0 >= M) break;
     const float* p = part0 + size_t(col) * 128;
-    if (col + 32 <= n_cols) reduce_partial_cols<32>(p, split_stride, n_splits, bias_s + m0, relu, dst + col, M - m0);
-    else reduce_partial_cols<16>(p, split_stride, n_splits, bias_s + m0, relu, dst + col, M - m0);
+    const __nv_bfloat16* res = res_row ? res_row + col : nullptr;
+    if (col + 32 <= n_cols) reduce_partial_cols<32>(p, split_stride, n_splits, bias_s + m0, relu, dst + col, M - m0, res, res_left - col);
+    else reduce_partial_cols<16>(p, split_stride, n_splits, bias_s + m0, relu, dst + col, M - m0, res, res_left - col);
   }
 }
 
@@ -253,7 +255,10 @@ conv3d_umma_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_consta
     const int bt_i = r % a.box.bt; r /= a.box.bt;
     const int bn_i = r;
     __nv_bfloat16* yb = static_cast<__nv_bfloat16*>(a.y);
+    const __nv_bfloat16* rb = static_cast<const __nv_bfloat16*>(a.residual);
     TmaStore ts{&ymap, store_smem + uint32_t(quad) * kStoreWarpBytes, 0, 0, 0, 0, 0u};
+    const PoolLanes pool_lanes{a.pool_w, a.pool_h, a.pool_t, a.sbw, a.sbh};
+    const PoolLanes* pool = (a.pool_t * a.pool_h * a.pool_w > 1) ? &pool_lanes : nullptr;
     int r0 = quad * 32;                        // coordinates of the warp's first row inside the box
     const int bw_0 = r0 % a.box.bw; r0 /= a.box.bw;
     const int bh_0 = r0 % a.box.bh; r0 /= a.box.bh;
@@ -274,13 +279,15 @@ conv3d_umma_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_consta
       const int m_base = c.bundle * a.n_tile;
       const uint32_t taddr = tmem_base + (uint32_t(quad * 32) << 16) + buf * uint32_t(a.n_tile);
       __nv_bfloat16* dst = yb + vox * a.g.ycs + m_base;
+      const __nv_bfloat16* res = (rb != nullptr && in_range) ? rb + vox * a.rcs + m_base : nullptr;
+      const int res_left = a.rcs - m_base;
       if (a.n_splits == 1) {
         if (a.store_tma) {
-          ts.c1 = c.w0 + bw_0; ts.c2 = c.h0 + bh_0; ts.c3 = c.t0 + bt_0; ts.c4 = c.n0 + bn_0;
+          ts.c1 = (c.w0 + bw_0) / a.pool_w; ts.c2 = (c.h0 + bh_0) / a.pool_h; ts.c3 = (c.t0 + bt_0) / a.pool_t; ts.c4 = c.n0 + bn_0;
           epilogue_row_tma(taddr, a.n_tile, nsteps > 0, quad * 32 < box_rows, in_range, bias_s, a.g.relu, dst, m_base,
-                           a.g.M, lane, ts);
+                           a.g.M, lane, ts, res, res_left, pool);
         } else {
-          epilogue_row(taddr, a.n_tile, nsteps > 0, in_range, bias_s, a.g.relu, dst, m_base, a.g.M);
+          epilogue_row(taddr, a.n_tile, nsteps > 0, in_range, bias_s, a.g.relu, dst, m_base, a.g.M, res, res_left);
         }
         tc_fence_before();
         __syncwarp();
@@ -301,7 +308,7 @@ conv3d_umma_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_consta
         if (last) {
           __threadfence();
           reduce_partial_row(tile_part + row, part_tile, a.n_splits, a.n_tile, in_range, bias_s,
-                             a.g.relu, dst, m_base, a.g.M);
+                             a.g.relu, dst, m_base, a.g.M, res, res_left);
           __syncwarp();
           if (lane == 0) a.counters[c.tile_id * 4 + quad] = 0;              // ready for the next launch
         }

@@ -239,7 +239,10 @@ conv3d_umma_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_c
     const int bt_i = r % a.box.bt; r /= a.box.bt;
     const int bn_i = r;
     __nv_bfloat16* yb = static_cast<__nv_bfloat16*>(a.y);
+    const __nv_bfloat16* rb = static_cast<const __nv_bfloat16*>(a.residual);
     TmaStore ts{&ymap, store_smem + uint32_t(quad) * kStoreWarpBytes, 0, 0, 0, 0, 0u};
+    const PoolLanes pool_lanes{a.pool_w, a.pool_h, a.pool_t, a.sbw, a.sbh};
+    const PoolLanes* pool = (a.pool_t * a.pool_h * a.pool_w > 1) ? &pool_lanes : nullptr;
     int r0 = quad * 32;                        // coordinates of the warp's first row inside the box
     const int bw_0 = r0 % a.box.bw; r0 /= a.box.bw;
     const int bh_0 = r0 % a.box.bh; r0 /= a.box.bh;
@@ -257,12 +260,15 @@ conv3d_umma_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_c
       const long long vox = (((long long)nn * a.g.To + to) * a.g.Ho + ho) * a.g.Wo + wo;
       const int m_base = c.bundle * a.n_tile;
       const uint32_t taddr = tmem_base + (uint32_t(quad * 32) << 16) + buf * uint32_t(a.n_tile);
+      const __nv_bfloat16* res = (rb != nullptr && in_range) ? rb + vox * a.rcs + m_base : nullptr;
+      const int res_left = a.rcs - m_base;
       if (a.store_tma) {
-        ts.c1 = c.w0 + bw_0; ts.c2 = c.h0 + bh_0; ts.c3 = c.t0 + bt_0; ts.c4 = c.n0 + bn_0;
+        ts.c1 = (c.w0 + bw_0) / a.pool_w; ts.c2 = (c.h0 + bh_0) / a.pool_h; ts.c3 = (c.t0 + bt_0) / a.pool_t; ts.c4 = c.n0 + bn_0;
         epilogue_row_tma(taddr, a.n_tile, nsteps > 0, quad * 32 < box_rows, in_range, bias_s, a.g.relu,
-                         yb + vox * a.g.ycs + m_base, m_base, a.g.M, lane, ts);
+                         yb + vox * a.g.ycs + m_base, m_base, a.g.M, lane, ts, res, res_left, pool);
       } else {
-        epilogue_row(taddr, a.n_tile, nsteps > 0, in_range, bias_s, a.g.relu, yb + vox * a.g.ycs + m_base, m_base, a.g.M);
+        epilogue_row(taddr, a.n_tile, nsteps > 0, in_range, bias_s, a.g.relu, yb + vox * a.g.ycs + m_base, m_base, a.g.M,
+                     res, res_left);
       }
       tc_fence_before();
       __syncwarp();

@@ -131,6 +131,8 @@ conv3d_umma_smallc_kernel(const __grid_constant__ CUtensorMap xmap, const __grid
     const int bh_i = row / kSmallCTileW, bw_i = row % kSmallCTileW;
     __nv_bfloat16* yb = static_cast<__nv_bfloat16*>(a.y);
     TmaStore ts{&ymap, store_smem + uint32_t(quad) * kStoreWarpBytes, 0, 0, 0, 0, 0u};   // warp = 4 rows x 8 voxels
+    const PoolLanes pool_lanes{a.pool_w, a.pool_h, 1, kSmallCTileW, 4};
+    const PoolLanes* pool = (a.pool_h * a.pool_w > 1) ? &pool_lanes : nullptr;
     uint32_t j = 0;
     for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++j) {
       int r = item;
@@ -145,12 +147,14 @@ conv3d_umma_smallc_kernel(const __grid_constant__ CUtensorMap xmap, const __grid
       const bool in_range = ho < a.g.Ho && wo < a.g.Wo;
       const long long vox = (((long long)nn * a.g.To + to) * a.g.Ho + ho) * a.g.Wo + wo;
       const uint32_t taddr = tmem_base + (uint32_t(quad * 32) << 16) + buf * uint32_t(a.n_pad);
+      const __nv_bfloat16* res = (a.residual != nullptr && in_range)
+                                     ? static_cast<const __nv_bfloat16*>(a.residual) + vox * a.rcs : nullptr;
       if (a.store_tma) {
-        ts.c1 = iw * kSmallCTileW; ts.c2 = ih * kSmallCTileH + quad * 4; ts.c3 = to; ts.c4 = nn;
+        ts.c1 = iw * kSmallCTileW / a.pool_w; ts.c2 = (ih * kSmallCTileH + quad * 4) / a.pool_h; ts.c3 = to; ts.c4 = nn;
         epilogue_row_tma(taddr, a.n_pad, a.n_pairs > 0, true, in_range, bias_s, a.g.relu, yb + vox * a.g.ycs, 0, a.g.M,
-                         lane, ts);
+                         lane, ts, res, a.rcs, pool);
       } else {
-        epilogue_row(taddr, a.n_pad, a.n_pairs > 0, in_range, bias_s, a.g.relu, yb + vox * a.g.ycs, 0, a.g.M);
+        epilogue_row(taddr, a.n_pad, a.n_pairs > 0, in_range, bias_s, a.g.relu, yb + vox * a.g.ycs, 0, a.g.M, res, a.rcs);
       }
       tc_fence_before();
       __syncwarp();

@@ -62,6 +62,15 @@ class ConvLayer:
            self.spec.relu if relu is None else relu, algo, stream)
         return y
 
+    def fused(self, x: torch.Tensor, y: torch.Tensor, residual: torch.Tensor | None = None, pool=(1, 1, 1),
+              relu=None, algo=B.ALGO_AUTO, stream=None):
+        """y = pool(act(conv(x) + bias + residual)) in one launch (rt3d_conv3d_sparse_fused)."""
+        res = None if residual is None else B.tensor_desc(residual, self.spec.cout)
+        B.rt3d_conv3d_sparse_fused(B.tensor_desc(x, self.spec.cin), self.packed, self.bias,
+                                   B.tensor_desc(y, self.spec.cout), self.spec.stride, self.spec.pad,
+                                   self.spec.relu if relu is None else relu, res, pool, algo, stream)
+        return y
+
     def cost(self, x: torch.Tensor):
         return B.rt3d_conv3d_cost(B.tensor_desc(x, self.spec.cin), self.packed, self.spec.stride, self.spec.pad)
 
@@ -99,15 +108,50 @@ class Workspace:
 class C3DNet:
     """C3D-shaped forward: 8 convs (3x3x3, ReLU) and 5 max-pools.  `layers` maps conv name -> ConvLayer."""
 
-    def __init__(self, plan, layers):
+    def __init__(self, plan, layers, fuse_pool: bool = False):
         self.plan = plan
         self.layers = layers
+        self.fuse_pool = fuse_pool      # conv + ReLU + un-padded 2-wide max-pool in one launch where the library can
         self.ws = Workspace()
+        self.fused_ok = {}              # conv name -> did the fused call apply (decided on first use per shape)
+
+    def _try_fused(self, op, pool, x, algo, stream):
+        """Runs conv `op` with `pool` fused; returns the pooled tensor or None if the library declines."""
+        if any(pool.pad) or tuple(pool.k) != tuple(pool.stride) or any(k not in (1, 2) for k in pool.k):
+            return None
+        key = (op.name, tuple(x.shape))
+        if self.fused_ok.get(key) is False:
+            return None
+        layer = self.layers[op.name]
+        n, t, h, w, _ = x.shape
+        to, ho, wo = op.out_extent(t, h, w)
+        shape = (n, to // pool.k[0], ho // pool.k[1], wo // pool.k[2], pitch_for(op.cout, x.dtype))
+        y = self.ws.get(pool.name, shape, x.dtype, x.device)
+        try:
+            layer.fused(x, y, pool=pool.k, algo=algo, stream=stream)
+        except B.Rt3dError as e:
+            if e.status != B.ERR_UNSUPPORTED:
+                raise
+            self.fused_ok[key] = False
+            return None
+        self.fused_ok[key] = True
+        return y
 
     def forward(self, x: torch.Tensor, algo=B.ALGO_AUTO, keep=None, stream=None) -> torch.Tensor:
         c = self.plan[0].cin
-        for op in self.plan:
+        skip = None
+        for i, op in enumerate(self.plan):
+            if op is skip:
+                continue
             if hasattr(op, "cout"):
+                nxt = self.plan[i + 1] if i + 1 < len(self.plan) else None
+                if self.fuse_pool and nxt is not None and not hasattr(nxt, "cout"):
+                    y = self._try_fused(op, nxt, x, algo, stream)
+                    if y is not None:
+                        x, c, skip = y, op.cout, nxt
+                        if keep is not None:
+                            keep[nxt.name] = x
+                        continue
                 layer = self.layers[op.name]
                 y = self.ws.get(op.name, layer.out_shape(x), x.dtype, x.device)
                 x = layer(x, y, algo=algo, stream=stream)
@@ -129,8 +173,9 @@ class R2Plus1DNet:
     """R(2+1)D-18-shaped forward: stem, then residual blocks of two factorised convs each
     (spatial 1x3x3 then temporal 3x1x1), optional 1x1x1 strided projection, add + ReLU."""
 
-    def __init__(self, stem, blocks, layers):
+    def __init__(self, stem, blocks, layers, fuse_residual: bool = False):
         self.stem, self.blocks, self.layers = stem, blocks, layers
+        self.fuse_residual = fuse_residual      # block end = one fused launch instead of conv + add kernel
         self.ws = Workspace()
 
     def _conv(self, spec, x, algo, stream):
@@ -145,21 +190,28 @@ class R2Plus1DNet:
                 keep[spec.name] = x
         for blk in self.blocks:
             inp = x
-            for spec in blk.convs:
-                x = self._conv(spec, x, algo, stream)
-                if keep is not None:
-                    keep[spec.name] = x
             sc = inp if blk.shortcut is None else self._conv(blk.shortcut, inp, algo, stream)
             if keep is not None and blk.shortcut is not None:
                 keep[blk.shortcut.name] = sc
-            y = self.ws.get(blk.name + ".out", x.shape, x.dtype, x.device)
-            x = add_relu(x, sc, blk.convs[-1].cout, True, y, stream=stream)
+            last = blk.convs[-1]
+            for spec in blk.convs[:-1] if self.fuse_residual else blk.convs:
+                x = self._conv(spec, x, algo, stream)
+                if keep is not None:
+                    keep[spec.name] = x
+            if self.fuse_residual:
+                layer = self.layers[last.name]
+                y = self.ws.get(blk.name + ".out", layer.out_shape(x), x.dtype, x.device)
+                x = layer.fused(x, y, residual=sc, relu=True, algo=algo, stream=stream)
+            else:
+                y = self.ws.get(blk.name + ".out", x.shape, x.dtype, x.device)
+                x = add_relu(x, sc, last.cout, True, y, stream=stream)
             if keep is not None:
                 keep[blk.name + ".out"] = x
         return x
 
     def n_launches(self) -> int:
-        return len(self.stem) + sum(5 + (blk.shortcut is not None) for blk in self.blocks)
+        per_block = 4 if self.fuse_residual else 5
+        return len(self.stem) + sum(per_block + (blk.shortcut is not None) for blk in self.blocks)
 
 
 class GraphedForward:

@@ -66,11 +66,11 @@ def test_c3d_layers_teacher_forced(c3d):
     assert 3.2 < dense_macs / kept_macs < 4.0                    # about 3.6x FLOPs pruning overall
 
 
-@pytest.mark.parametrize("batch", [1, 16])
-def test_c3d_free_running_forward(c3d, batch):
+@pytest.mark.parametrize("batch,fuse", [(1, False), (16, False), (1, True), (16, True)])
+def test_c3d_free_running_forward(c3d, batch, fuse):
     plan, layers, specs, x2, rec, final = c3d
     dl = device_layers(layers, specs)
-    net = nets.C3DNet(plan, dl)
+    net = nets.C3DNet(plan, dl, fuse_pool=fuse)
     if batch == 1:
         x = x2[:1]
         pick = [0]
@@ -85,6 +85,8 @@ def test_c3d_free_running_forward(c3d, batch):
     assert (ref != 0).mean() > 0.10
     e = rel_err(y[pick], ref)
     assert e <= TOL_FREE, e
+    if fuse:
+        assert any(net.fused_ok.values())                        # at least conv1/conv2 really ran fused
 
 
 def test_c3d_dense_path_forward():
@@ -134,9 +136,10 @@ def test_r2plus1d_layers_teacher_forced(r21d):
     assert 2.2 < dense_macs / kept_macs < 2.8                    # about 2.5x
 
 
-def test_r2plus1d_free_running_batch8(r21d):
+@pytest.mark.parametrize("fuse", [False, True])
+def test_r2plus1d_free_running_batch8(r21d, fuse):
     stem, blocks, layers, specs, x2, rec, final = r21d
-    net = nets.R2Plus1DNet(stem, blocks, device_layers(layers, specs))
+    net = nets.R2Plus1DNet(stem, blocks, device_layers(layers, specs), fuse_residual=fuse)
     filler = oracle.bf16_round(synth.make_input(33, (6, 16, 112, 112, 3)))
     x = np.concatenate([x2[:1], filler, x2[1:]], axis=0)
     y = nets.to_numpy(net.forward(nets.to_device(x)), 512)
