@@ -38,8 +38,8 @@ CFG = dict(n=8, t=8, h=28, w=28, cin=128, cout=256, k=(3, 3, 3), stride=(1, 1, 1
            g_m=4, g_n=4, density=0.4)
 L2_BYTES = 126 * 1024 * 1024
 # DRAM bytes (read + write) of one launch of the timed kernel on this workload, from the ncu capture
-# summarised in profiles/conv3d_umma_pair_cfg1.md (14.65 MB read + 0.06 MB written; the output stays in L2).
-DRAM_TRAFFIC_PER_LAUNCH = 14.71e6
+# summarised in profiles/conv3d_umma_pair_cfg1.md (14.68 MB read + 0.01 MB written; the output stays in L2).
+DRAM_TRAFFIC_PER_LAUNCH = 14.69e6
 WORKLOAD = "cfg1: C3D conv3a-shaped layer, batch 8, 128->256, 8x28x28, 3x3x3 s1 p1, KGS 4x4 ~2.5x, bf16"
 
 
