@@ -255,6 +255,20 @@ rt3d_status rt3d_kgs_expand_mask(const uint8_t* group_mask, int M, int N, int Kt
 rt3d_status rt3d_conv3d_cost(const rt3d_tensor* x, const rt3d_packed* w, const rt3d_conv_params* p,
                              int64_t* kept_macs, int64_t* dense_macs, int64_t* alg_bytes);
 
+/* How the calling thread's most recent successful convolution call was run (for tests and profiling):
+ *   kernel       0 CUDA-core kernel, 1 tensor-core single-CTA kernel, 2 tensor-core CTA-pair kernel,
+ *                3 tensor-core small-C_in kernel
+ *   n_tile       output channels per accumulator tile (tensor-core kernels, else 0)
+ *   n_splits     K splits per output tile in the single-CTA kernel (1 = none)
+ *   tail_workers CTA pairs that share, cut along K, the output tiles which do not fill a last round
+ *                of the persistent CTA-pair grid (0 = every tile is computed by one pair)
+ *   fused_pool   1 if a max-pool ran in the epilogue
+ * RT3D_ERR_INVALID_ARG if info is NULL or the thread has not run a convolution yet. */
+typedef struct {
+  int32_t kernel, n_tile, n_splits, tail_workers, fused_pool;
+} rt3d_plan_info;
+rt3d_status rt3d_last_plan(rt3d_plan_info* info);
+
 /* Which kernel family RT3D_ALGO_AUTO would run for this call: writes an rt3d_algo to *algo. */
 rt3d_status rt3d_conv3d_query_algo(const rt3d_tensor* x, const rt3d_packed* w, const rt3d_conv_params* p,
                                    const rt3d_tensor* y, int* algo);

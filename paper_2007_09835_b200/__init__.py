@@ -7,8 +7,13 @@ module stays importable before the library exists.
 """
 
 
+_SUBMODULES = ("build", "binding", "nets", "dist", "sweep")
+
+
 def __getattr__(name):
     import importlib
+    if name in _SUBMODULES:             # `from package import build` must not load the (possibly stale) library
+        return importlib.import_module(__name__ + "." + name)
     binding = importlib.import_module(__name__ + ".binding")
     try:
         return getattr(binding, name)

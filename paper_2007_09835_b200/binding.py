@@ -44,6 +44,10 @@ class Fusion(ctypes.Structure):
                 ("pool_w", ctypes.c_int32)]
 
 
+class PlanInfo(ctypes.Structure):
+    _fields_ = [(k, ctypes.c_int32) for k in ("kernel", "n_tile", "n_splits", "tail_workers", "fused_pool")]
+
+
 class PackedView(ctypes.Structure):
     _fields_ = [(k, ctypes.c_int32) for k in ("M", "N", "Kt", "Kh", "Kw", "g_m", "g_n", "P", "Q", "Ks",
                                               "dtype", "is_vanilla", "is_dense")] + \
@@ -77,6 +81,7 @@ def _load():
     i64p = ctypes.POINTER(ctypes.c_int64)
     lib.rt3d_conv3d_cost.argtypes = [TP, vp, CP, i64p, i64p, i64p]
     lib.rt3d_conv3d_query_algo.argtypes = [TP, vp, CP, TP, ctypes.POINTER(ctypes.c_int)]
+    lib.rt3d_last_plan.argtypes = [ctypes.POINTER(PlanInfo)]
     lib.rt3d_last_device_status.argtypes = [vp]
     lib.rt3d_launch_count.restype = ctypes.c_int64
     lib.rt3d_status_string.restype = ctypes.c_char_p
@@ -298,6 +303,13 @@ def rt3d_conv3d_query_algo(x: Tensor, w: Packed, y: Tensor, stride=(1, 1, 1), pa
     _check(_lib.rt3d_conv3d_query_algo(ctypes.byref(x), w.handle, ctypes.byref(_params(stride, pad, False, algo)),
                                        ctypes.byref(y), ctypes.byref(a)), "rt3d_conv3d_query_algo")
     return a.value
+
+
+def rt3d_last_plan() -> dict:
+    """How this thread's most recent convolution call was run (kernel, n_tile, n_splits, tail_workers, fused_pool)."""
+    info = PlanInfo()
+    _check(_lib.rt3d_last_plan(ctypes.byref(info)), "rt3d_last_plan")
+    return {name: int(getattr(info, name)) for name, _ in PlanInfo._fields_}
 
 
 def rt3d_last_device_status(stream=None) -> int:

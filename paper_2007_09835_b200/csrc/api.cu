@@ -405,6 +405,28 @@ rt3d_status launch_smallc(rt3d_packed* w, DeviceBlob* blob, const DeviceState* d
   return RT3D_OK;
 }
 
+thread_local rt3d_plan_info t_last_plan = {-1, 0, 0, 0, 0};
+
+// Grows the handle's K-split workspace on this device: `bytes` of partial tiles and `cnt_bytes` of
+// counters / flags, which every kernel that uses them leaves zeroed.
+rt3d_status ensure_splitk(rt3d_packed* w, DeviceBlob* blob, size_t bytes, size_t cnt_bytes) {
+  std::lock_guard<std::mutex> lock(w->mu);
+  if (blob->splitk_bytes < bytes) {
+    cudaFree(blob->splitk);
+    blob->splitk = nullptr; blob->splitk_bytes = 0;
+    if (cudaMalloc(reinterpret_cast<void**>(&blob->splitk), bytes) != cudaSuccess) return RT3D_ERR_ALLOC;
+    blob->splitk_bytes = bytes;
+  }
+  if (blob->splitk_cnt_bytes < cnt_bytes) {
+    cudaFree(blob->splitk_cnt);
+    blob->splitk_cnt = nullptr; blob->splitk_cnt_bytes = 0;
+    if (cudaMalloc(reinterpret_cast<void**>(&blob->splitk_cnt), cnt_bytes) != cudaSuccess) return RT3D_ERR_ALLOC;
+    if (cudaMemset(blob->splitk_cnt, 0, cnt_bytes) != cudaSuccess) return RT3D_ERR_CUDA;
+    blob->splitk_cnt_bytes = cnt_bytes;
+  }
+  return RT3D_OK;
+}
+
 rt3d_status conv_impl(const rt3d_tensor* x, const rt3d_packed* wc, const float* bias, const rt3d_conv_params* p,
                       rt3d_tensor* y, void* stream, bool dense_entry, const rt3d_fusion* fz = nullptr) {
   ConvGeom g;
@@ -455,12 +477,16 @@ rt3d_status conv_impl(const rt3d_tensor* x, const rt3d_packed* wc, const float* 
                                      w->g_m, w->g_n, w->P, w->Q, dense_entry, res_data, res_pitch, st);
     if (e != cudaSuccess) return RT3D_ERR_CUDA;
     g_launches.fetch_add(1);
+    t_last_plan = rt3d_plan_info{0, 0, 1, 0, 0};
     return RT3D_OK;
   }
 
   const SmallCLayout* SL = nullptr;
-  if (p->algo != RT3D_ALGO_UMMA_PAIR && (!pooled || pl_t == 1) && smallc_eligible(d, w, x, y, p, &SL))
-    return launch_smallc(w, blob, d, SL, x, g, bias, y, st, res_data, res_pitch, pl_h, pl_w);
+  if (p->algo != RT3D_ALGO_UMMA_PAIR && (!pooled || pl_t == 1) && smallc_eligible(d, w, x, y, p, &SL)) {
+    s = launch_smallc(w, blob, d, SL, x, g, bias, y, st, res_data, res_pitch, pl_h, pl_w);
+    if (s == RT3D_OK) t_last_plan = rt3d_plan_info{3, SL->n_pad, 1, 0, pooled ? 1 : 0};
+    return s;
+  }
 
   UmmaArgs a;
   a.g = g;
@@ -506,25 +532,12 @@ rt3d_status conv_impl(const rt3d_tensor* x, const rt3d_packed* wc, const float* 
   a.bias = bias; a.y = y->data; a.sched = d->sched;
   a.residual = res_data; a.rcs = res_pitch;
   a.n_splits = plan.n_splits; a.scratch = nullptr; a.counters = nullptr;
+  a.tail_workers = 0; a.tail_scratch = nullptr; a.tail_flags = nullptr;
   if (a.n_splits > 1) {
     // split-K workspace of this handle on this device: partial tiles + per-warp arrival counters
     const long long tiles = m_tiles * L->n_bundles;
-    const size_t need = size_t(tiles) * a.n_splits * kTileM * L->n_tile * sizeof(float);
-    const size_t need_cnt = size_t(tiles) * 4 * sizeof(int32_t);
-    std::lock_guard<std::mutex> lock(w->mu);
-    if (blob->splitk_bytes < need) {
-      cudaFree(blob->splitk);
-      blob->splitk = nullptr; blob->splitk_bytes = 0;
-      if (cudaMalloc(reinterpret_cast<void**>(&blob->splitk), need) != cudaSuccess) return RT3D_ERR_ALLOC;
-      blob->splitk_bytes = need;
-    }
-    if (blob->splitk_cnt_bytes < need_cnt) {
-      cudaFree(blob->splitk_cnt);
-      blob->splitk_cnt = nullptr; blob->splitk_cnt_bytes = 0;
-      if (cudaMalloc(reinterpret_cast<void**>(&blob->splitk_cnt), need_cnt) != cudaSuccess) return RT3D_ERR_ALLOC;
-      if (cudaMemset(blob->splitk_cnt, 0, need_cnt) != cudaSuccess) return RT3D_ERR_CUDA;
-      blob->splitk_cnt_bytes = need_cnt;
-    }
+    if ((s = ensure_splitk(w, blob, size_t(tiles) * a.n_splits * kTileM * L->n_tile * sizeof(float),
+                           size_t(tiles) * 4 * sizeof(int32_t))) != RT3D_OK) return s;
     a.scratch = blob->splitk; a.counters = blob->splitk_cnt;
   }
   CUtensorMap xmap;
@@ -532,11 +545,21 @@ rt3d_status conv_impl(const rt3d_tensor* x, const rt3d_packed* wc, const float* 
   CUtensorMap ymap;
   a.store_tma = (a.n_splits == 1 && rect && encode_ymap(y, sb, pl_w, pl_h, pl_t, &ymap)) ? 1 : 0;
   if (pooled && !a.store_tma) return RT3D_ERR_UNSUPPORTED;
+  if (use_pair) {
+    // items that do not fill a last round of CTA pairs are cut along K and shared (same workspace as split-K)
+    size_t tail_bytes = 0, flag_bytes = 0;
+    umma_pair_tail_plan(&a, L->step_ptr.data(), d->sm_count, &tail_bytes, &flag_bytes);
+    if (a.tail_workers > 0) {
+      if ((s = ensure_splitk(w, blob, tail_bytes, flag_bytes)) != RT3D_OK) return s;
+      a.tail_scratch = blob->splitk; a.tail_flags = blob->splitk_cnt;
+    }
+  }
   const void* ym = a.store_tma ? &ymap : nullptr;
   cudaError_t e = use_pair ? launch_conv_umma_pair(a, &xmap, u->wmap_half, ym, d->sm_count, st)
                            : launch_conv_umma(a, &xmap, u->wmap, ym, d->sm_count, st);
   if (e != cudaSuccess) return RT3D_ERR_CUDA;
   g_launches.fetch_add(1);
+  t_last_plan = rt3d_plan_info{use_pair ? 2 : 1, a.n_tile, a.n_splits, a.tail_workers, pooled ? 1 : 0};
   return RT3D_OK;
 }
 
@@ -707,6 +730,12 @@ rt3d_status rt3d_conv3d_query_algo(const rt3d_tensor* x, const rt3d_packed* w, c
   return RT3D_OK;
 }
 
+rt3d_status rt3d_last_plan(rt3d_plan_info* info) {
+  if (!info || t_last_plan.kernel < 0) return RT3D_ERR_INVALID_ARG;
+  *info = t_last_plan;
+  return RT3D_OK;
+}
+
 rt3d_status rt3d_last_device_status(void* stream) {
   DeviceState* d = nullptr;
   rt3d_status s = get_device_state(&d);
@@ -824,6 +853,7 @@ rt3d_status rt3d_conv3d_sparse_noalloc(const rt3d_tensor* x, const rt3d_packed* 
   CUtensorMap ymap;
   int sb[4];
   a.pool_t = a.pool_h = a.pool_w = 1; a.sbw = a.sbh = 1;
+  a.tail_workers = 0; a.tail_scratch = nullptr; a.tail_flags = nullptr;
   a.store_tma = (a.n_splits == 1 && warp_block(a.box.bw, a.box.bh, a.box.bt, a.box.bn, sb) &&
                  encode_ymap(y, sb, 1, 1, 1, &ymap)) ? 1 : 0;
   if (launch_conv_umma(a, &xmap, u->wmap, a.store_tma ? &ymap : nullptr, d->sm_count, st) != cudaSuccess) return RT3D_ERR_CUDA;

@@ -55,6 +55,9 @@ struct UmmaArgs {
   int n_splits;                             // K splits per output tile (1 = none)
   float* scratch;                           // device, split-K partial tiles [tile][split][128][n_tile] (n_splits > 1)
   int32_t* counters;                        // device, [tiles * 4] arrival counters, zero between launches
+  int tail_workers;                         // CTA-pair kernel: pairs sharing the left-over items of the last round (0 = off)
+  float* tail_scratch;                      // device, [tail_workers][2 shares][2 CTAs][n_tile][128] fp32 partial tiles
+  int32_t* tail_flags;                      // device, [tail_workers][2][2][4 warps] "partial written" flags, zero between launches
 };
 
 // xmap / wmap point to 128-byte CUtensorMap objects in host memory.
@@ -66,6 +69,10 @@ cudaError_t launch_conv_umma(const UmmaArgs& a, const void* xmap, const void* wm
 // CTA-pair variant (cta_group::2): wmap_half is a tensor map over the same weight tiles whose box is
 // half a tile high (n_tile/2 rows).  Needs n_tile % 32 == 0 and a.n_splits == 1.
 bool umma_pair_supported(int n_tile, int n_bundles);
+// Fills a->tail_workers (0 = whole items only) and the scratch the tail split needs; the caller provides
+// a->tail_scratch / a->tail_flags of at least those sizes (flags zero-initialised).
+void umma_pair_tail_plan(UmmaArgs* a, const int32_t* step_ptr_host, int sm_count, size_t* scratch_bytes,
+                         size_t* flag_bytes);
 cudaError_t launch_conv_umma_pair(const UmmaArgs& a, const void* xmap, const void* wmap_half, const void* ymap,
                                   int sm_count, cudaStream_t stream);
 

@@ -330,7 +330,9 @@ __device__ __forceinline__ void epilogue_row_tma(uint32_t taddr, int n_cols, boo
                                                  bool in_range, const float* bias_s, int relu, __nv_bfloat16* dst,
                                                  int m_base, int M, int lane, TmaStore& ts,
                                                  const __nv_bfloat16* res_row = nullptr, int res_pitch_left = 0,
-                                                 const PoolLanes* pool = nullptr) {
+                                                 const PoolLanes* pool = nullptr, const float* extra_first = nullptr,
+                                                 const float* extra = nullptr, size_t extra_stride = 0,
+                                                 int n_extra = 0) {
   for (int col = 0; col < n_cols; col += 32) {
     const int m0 = m_base + col;
     if (m0 >= M) break;
@@ -343,12 +345,52 @@ __device__ __forceinline__ void epilogue_row_tma(uint32_t taddr, int n_cols, boo
 #pragma unroll
       for (int q = 0; q < 32; ++q) v[q] = 0u;
     }
+    // partial sums of the same tile left in scratch by this and other CTAs (column-major [column][128 rows],
+    // pointers at this thread's row), added in a fixed order: extra_first, then extra + p * extra_stride.
+    // Two partial tiles' loads are in flight at a time.
+    if (extra_first != nullptr) {
+      const float* e0 = extra_first + size_t(col) * 128;
+      for (int p = -1; p < n_extra; p += 2) {
+        const float* ea = p < 0 ? e0 : extra + size_t(p) * extra_stride + size_t(col) * 128;
+        const bool two = p + 1 < n_extra;
+        const float* eb = two ? extra + size_t(p + 1) * extra_stride + size_t(col) * 128 : ea;
+        float t0[32], t1[32];
+#pragma unroll
+        for (int q = 0; q < 32; ++q) {
+          const bool live = wide || q < 16;
+          t0[q] = live ? __ldcg(ea + size_t(q) * 128) : 0.f;
+          t1[q] = (live && two) ? __ldcg(eb + size_t(q) * 128) : 0.f;
+        }
+#pragma unroll
+        for (int q = 0; q < 32; ++q) v[q] = __float_as_uint((__uint_as_float(v[q]) + t0[q]) + t1[q]);
+      }
+    }
     const __nv_bfloat16* res = (res_row && in_range) ? res_row + col : nullptr;
     if (wide) {
       if (warp_rows_valid) epilogue_piece_tma(v, bias_s + m0, relu, m0, lane, ts, res, res_pitch_left - col, pool);
     } else if (in_range) {
       epilogue_cols<16>(v, bias_s + m0, relu, dst + col, M - m0, res, res_pitch_left - col);
     }
+  }
+}
+
+// Split-K partial tiles are stored column-major, [column][128 rows] floats, so that the 32 lanes of a
+// warp (32 consecutive rows) always touch 128 contiguous bytes.
+// Raw fp32 accumulator row -> scratch; `dst` already points at this thread's row of column 0.
+__device__ __forceinline__ void store_partial_row(uint32_t taddr, int n_cols, bool has_acc, float* dst) {
+  for (int col = 0; col < n_cols; col += 32) {
+    uint32_t v[32];
+    const bool wide = col + 32 <= n_cols;
+    if (has_acc) {
+      if (wide) tmem_ld32(taddr + col, v);
+      else tmem_ld16(taddr + col, *reinterpret_cast<uint32_t(*)[16]>(v));
+    } else {
+#pragma unroll
+      for (int q = 0; q < 32; ++q) v[q] = 0u;
+    }
+#pragma unroll
+    for (int q = 0; q < 32; ++q)
+      if (wide || q < 16) dst[size_t(col + q) * 128] = __uint_as_float(v[q]);
   }
 }
 

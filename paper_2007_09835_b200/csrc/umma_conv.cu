@@ -57,26 +57,6 @@ __device__ __forceinline__ void item_steps(const UmmaArgs& a, const ItemCoord& c
   nsteps = hi - local0;
 }
 
-// Split-K partial tiles are stored column-major, [column][128 rows] floats, so that the 32 lanes of a
-// warp (32 consecutive rows) always touch 128 contiguous bytes.
-// Raw fp32 accumulator row -> scratch; `dst` already points at this thread's row of column 0.
-__device__ __forceinline__ void store_partial_row(uint32_t taddr, int n_cols, bool has_acc, float* dst) {
-  for (int col = 0; col < n_cols; col += 32) {
-    uint32_t v[32];
-    const bool wide = col + 32 <= n_cols;
-    if (has_acc) {
-      if (wide) tmem_ld32(taddr + col, v);
-      else tmem_ld16(taddr + col, *reinterpret_cast<uint32_t(*)[16]>(v));
-    } else {
-#pragma unroll
-      for (int q = 0; q < 32; ++q) v[q] = 0u;
-    }
-#pragma unroll
-    for (int q = 0; q < 32; ++q)
-      if (wide || q < 16) dst[size_t(col + q) * 128] = __uint_as_float(v[q]);
-  }
-}
-
 // Sum of the partials of all splits (in split order, two splits' loads in flight at a time) + epilogue
 // for one output voxel; `part0` points at this thread's row of column 0 of split 0.
 template <int NC>

@@ -70,6 +70,27 @@ __device__ __forceinline__ uint32_t instr_desc_bf16_pair(int n) {
   return (1u << 4) | (1u << 7) | (1u << 10) | (uint32_t(n >> 3) << 17) | (uint32_t(256 >> 4) << 24);
 }
 
+// Work of one CTA pair: whole items dealt round-robin.  With the tail split, the items that would not
+// fill a last round are instead laid end to end as one line of K-step groups, cut into `tail_workers`
+// equal ranges and done FIRST: an item is then computed by up to a few pairs, each leaving its fp32
+// partial tile in global scratch.  The pair that holds the item's first steps owns it: once its own
+// share is stored, and while its tensor pipe is already busy with the first whole item, its epilogue
+// warps add the partial tiles in a fixed order and write the output.
+struct TailSeg { int item, g0, g1, part, nparts; };
+constexpr int kMaxTailSeg = 6;
+struct TailWork {
+  int n_full;                 // whole items of this pair: item = cluster_id + k * n_clusters
+  int n_seg;
+  TailSeg seg[kMaxTailSeg];
+};
+struct Work { int item, g0, g1, part, nparts; };
+
+__device__ __forceinline__ Work get_work(const TailWork* tw, int wi, int cluster_id, int n_clusters) {
+  if (wi >= tw->n_seg) return Work{cluster_id + (wi - tw->n_seg) * n_clusters, 0, 1 << 28, 0, 1};
+  const TailSeg& g = tw->seg[wi];
+  return Work{g.item, g.g0, g.g1, g.part, g.nparts};
+}
+
 struct PairItem {
   int bundle;
   int n0, t0, h0, w0;     // first output voxel of this CTA's box (beyond the tensor for a dummy tile)
@@ -106,7 +127,8 @@ conv3d_umma_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_c
   const uint32_t store_smem = tiles_base + uint32_t(stages) * stage_bytes;     // 4 warps x 2 staging buffers
   Barriers* bars = reinterpret_cast<Barriers*>(smem_raw + (tiles_base - raw) + size_t(stages) * stage_bytes +
                                                4 * kStoreWarpBytes);
-  float* bias_s = reinterpret_cast<float*>(bars + 1);
+  TailWork* tw = reinterpret_cast<TailWork*>(bars + 1);
+  float* bias_s = reinterpret_cast<float*>(tw + 1);
   int32_t* err = a.sched + 2;
   for (int i = threadIdx.x; i < a.n_bundles * a.n_tile; i += blockDim.x)
     bias_s[i] = (a.bias != nullptr && i < a.g.M) ? __ldg(a.bias + i) : 0.f;
@@ -132,6 +154,43 @@ conv3d_umma_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_c
     bars->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    // this pair's work list
+    tw->n_seg = 0;
+    if (a.tail_workers == 0) {
+      tw->n_full = cluster_id < n_items ? (n_items - cluster_id + n_clusters - 1) / n_clusters : 0;
+    } else {
+      const int rounds = n_items / n_clusters;
+      const int first_tail = rounds * n_clusters, n_tail = n_items - first_tail;
+      tw->n_full = rounds;
+      if (cluster_id < a.tail_workers) {
+        long long total = 0;
+        for (int t = 0; t < n_tail; ++t) {
+          const int b = (first_tail + t) / pairs_per_bundle;
+          const int ns = kDense ? a.steps_dense : a.step_ptr[b + 1] - a.step_ptr[b];
+          total += (ns + kCps - 1) / kCps;
+        }
+        const long long W = a.tail_workers;
+        const long long lo = cluster_id * total / W, hi = (cluster_id + 1) * total / W;
+        long long pre = 0;
+        int n_seg = 0;
+        for (int t = 0; t < n_tail && n_seg < kMaxTailSeg; ++t) {
+          const int b = (first_tail + t) / pairs_per_bundle;
+          const int ns = kDense ? a.steps_dense : a.step_ptr[b + 1] - a.step_ptr[b];
+          const long long G = (ns + kCps - 1) / kCps;
+          if (pre + G > lo && pre < hi) {
+            TailSeg& sg = tw->seg[n_seg++];
+            sg.item = first_tail + t;
+            sg.g0 = int((lo > pre ? lo : pre) - pre);
+            sg.g1 = int((hi < pre + G ? hi : pre + G) - pre);
+            const int first = int(((pre + 1) * W - 1) / total), last = int(((pre + G) * W - 1) / total);
+            sg.part = cluster_id - first;
+            sg.nparts = last - first + 1;
+          }
+          pre += G;
+        }
+        tw->n_seg = n_seg;
+      }
+    }
   }
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
@@ -151,15 +210,23 @@ conv3d_umma_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_c
       uint32_t phase = 0;
       bool ok = true;
       const uint32_t tx_chunk_both = 2u * (uint32_t(box_rows) * 128u + b_bytes);
-      for (int item = cluster_id; item < n_items && ok; item += n_clusters) {
-        const PairItem c = decode_pair_item(a, item, pairs_per_bundle, n_mtiles, rank);
+      const int n_work = tw->n_full + tw->n_seg;
+      for (int wi = 0; wi < n_work && ok; ++wi) {
+        const Work wk = get_work(tw, wi, cluster_id, n_clusters);
+        const PairItem c = decode_pair_item(a, wk.item, pairs_per_bundle, n_mtiles, rank);
         const int s_begin = kDense ? c.bundle * a.steps_dense : a.step_ptr[c.bundle];
         const int nsteps = kDense ? a.steps_dense : a.step_ptr[c.bundle + 1] - s_begin;
+        const int i0 = wk.g0 * kCps, i1 = wk.g1 * kCps < nsteps ? wk.g1 * kCps : nsteps;
         const int wq = c.w0 * a.g.sw - a.g.pw, hq = c.h0 * a.g.sh - a.g.ph, tq = c.t0 * a.g.st - a.g.pt;
         int kt = 0, kh = 0, kw = 0, ch = 0;
-        int wrow = s_begin * a.n_tile + int(rank) * n_half;
-        for (int i = 0; i < nsteps; i += kCps) {
-          const int nload = nsteps - i < kCps ? nsteps - i : kCps;
+        if (kDense && i0 > 0) {
+          ch = i0 % a.n_chunks;
+          const int pos = i0 / a.n_chunks;
+          kw = pos % a.g.Kw; kh = (pos / a.g.Kw) % a.g.Kh; kt = pos / (a.g.Kw * a.g.Kh);
+        }
+        int wrow = (s_begin + i0) * a.n_tile + int(rank) * n_half;
+        for (int i = i0; i < i1; i += kCps) {
+          const int nload = i1 - i < kCps ? i1 - i : kCps;
           int c_ch[kCps], c_w[kCps], c_h[kCps], c_t[kCps];
 #pragma unroll
           for (int q = 0; q < kCps; ++q) {
@@ -197,15 +264,18 @@ conv3d_umma_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_c
       uint32_t j = 0, phase = 0;
       int stage = 0;
       bool ok = true, ready = false;
-      for (int item = cluster_id; item < n_items && ok; item += n_clusters, ++j) {
-        const int bundle = item / pairs_per_bundle;
+      const int n_work = tw->n_full + tw->n_seg;
+      for (int wi = 0; wi < n_work && ok; ++wi, ++j) {
+        const Work wk = get_work(tw, wi, cluster_id, n_clusters);
+        const int bundle = wk.item / pairs_per_bundle;
         const int nsteps = kDense ? a.steps_dense : a.step_ptr[bundle + 1] - a.step_ptr[bundle];
+        const int i0 = wk.g0 * kCps, i1 = wk.g1 * kCps < nsteps ? wk.g1 * kCps : nsteps;
         const uint32_t buf = j & 1u;
         if (!mbar_wait(smem_u32(&bars->tmem_empty[buf]), ((j >> 1) & 1u) ^ 1u, bars, err, 22)) break;
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + buf * uint32_t(a.n_tile);
-        for (int i = 0; i < nsteps; i += kCps) {
-          const int nload = nsteps - i < kCps ? nsteps - i : kCps;
+        for (int i = i0; i < i1; i += kCps) {
+          const int nload = i1 - i < kCps ? i1 - i : kCps;
           if (!ready && !mbar_wait(smem_u32(&bars->full[stage]), phase, bars, err, 23)) { ok = false; break; }
           // poll the next stage's barrier now: its answer arrives while this stage's MMAs are issued
           const int stage_n = stage + 1 == stages ? 0 : stage + 1;
@@ -220,7 +290,7 @@ conv3d_umma_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_c
             const uint64_t bdesc = smem_desc_sw128(a_addr + kABytes);
 #pragma unroll
             for (int kk = 0; kk < 4; ++kk)
-              umma_bf16_pair(d_tmem, adesc + 2 * kk, bdesc + 2 * kk, idesc, (i | q | kk) ? 1u : 0u);
+              umma_bf16_pair(d_tmem, adesc + 2 * kk, bdesc + 2 * kk, idesc, ((i - i0) | q | kk) ? 1u : 0u);
           }
           umma_commit_pair(smem_u32(&bars->empty[stage]));
           stage = stage_n; phase = phase_n;
@@ -249,8 +319,13 @@ conv3d_umma_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_c
     const int bt_0 = r0 % a.box.bt; r0 /= a.box.bt;
     const int bn_0 = r0;
     uint32_t j = 0;
-    for (int item = cluster_id; item < n_items; item += n_clusters, ++j) {
-      const PairItem c = decode_pair_item(a, item, pairs_per_bundle, n_mtiles, rank);
+    const size_t part_tile = size_t(128) * a.n_tile;       // floats per partial tile
+    const int n_work = tw->n_full + tw->n_seg;
+    Work own{0, 0, 0, 0, 1};                               // the shared tile this pair owns, if any
+    int own_slot = 0;
+    for (int wi = 0; wi < n_work; ++wi, ++j) {
+      const Work wk = get_work(tw, wi, cluster_id, n_clusters);
+      const PairItem c = decode_pair_item(a, wk.item, pairs_per_bundle, n_mtiles, rank);
       const int nsteps = kDense ? a.steps_dense : a.step_ptr[c.bundle + 1] - a.step_ptr[c.bundle];
       const uint32_t buf = j & 1u;
       if (!mbar_wait(smem_u32(&bars->tmem_full[buf]), (j >> 1) & 1u, bars, err, 24)) break;
@@ -262,6 +337,61 @@ conv3d_umma_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_c
       const uint32_t taddr = tmem_base + (uint32_t(quad * 32) << 16) + buf * uint32_t(a.n_tile);
       const __nv_bfloat16* res = (rb != nullptr && in_range) ? rb + vox * a.rcs + m_base : nullptr;
       const int res_left = a.rcs - m_base;
+      if (wk.nparts > 1) {
+        // shared tile: leave the raw partial sums in scratch and raise this warp's flag.  A pair has at
+        // most two such shares, the first and the last segment of its range.
+        const int slot = (cluster_id * 2 + (wi == 0 ? 0 : 1)) * 2 + int(rank);
+        store_partial_row(taddr, a.n_tile, true, a.tail_scratch + size_t(slot) * part_tile + row);
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive_cluster(mapa_shared(smem_u32(&bars->tmem_empty[buf]), 0));
+        __threadfence();
+        __syncwarp();
+        if (lane == 0) *reinterpret_cast<volatile int32_t*>(a.tail_flags + slot * 4 + quad) = 1;
+        if (wk.part == 0) { own = wk; own_slot = slot; }
+        if (wi + 1 < tw->n_seg) continue;
+      }
+      if (wi + 1 == tw->n_seg && own.nparts > 1) {
+        // all shares of this pair are stored: finish the tile this pair owns.  The other shares were
+        // computed at the same time by the next pairs (each as the first segment of its range).
+        int ok = 1;
+        if (lane == 0) {
+          const long long start = clock64();
+          for (int p = 1; p < own.nparts && ok; ++p) {
+            const volatile int32_t* f = a.tail_flags + (((cluster_id + p) * 2) * 2 + int(rank)) * 4 + quad;
+            while (*f == 0) {
+              if (bars->abort_flag || clock64() - start > kWaitCycles) {
+                bars->abort_flag = 1;
+                atomicCAS(err, 0, 25);
+                ok = 0;
+                break;
+              }
+            }
+          }
+        }
+        ok = __shfl_sync(0xffffffffu, ok, 0);
+        if (!ok) break;
+        __threadfence();
+        const PairItem oc = decode_pair_item(a, own.item, pairs_per_bundle, n_mtiles, rank);
+        const int onn = oc.n0 + bn_i, oto = oc.t0 + bt_i, oho = oc.h0 + bh_i, owo = oc.w0 + bw_i;
+        const bool o_in = row < box_rows && onn < a.g.n && oto < a.g.To && oho < a.g.Ho && owo < a.g.Wo;
+        const long long ovox = (((long long)onn * a.g.To + oto) * a.g.Ho + oho) * a.g.Wo + owo;
+        const int om = oc.bundle * a.n_tile;
+        const __nv_bfloat16* ores = (rb != nullptr && o_in) ? rb + ovox * a.rcs + om : nullptr;
+        ts.c1 = (oc.w0 + bw_0) / a.pool_w; ts.c2 = (oc.h0 + bh_0) / a.pool_h; ts.c3 = (oc.t0 + bt_0) / a.pool_t; ts.c4 = oc.n0 + bn_0;
+        epilogue_row_tma(0u, a.n_tile, false, quad * 32 < box_rows, o_in, bias_s, a.g.relu,
+                         yb + ovox * a.g.ycs + om, om, a.g.M, lane, ts, ores, a.rcs - om, pool,
+                         a.tail_scratch + size_t(own_slot) * part_tile + row,
+                         a.tail_scratch + size_t(((cluster_id + 1) * 2) * 2 + int(rank)) * part_tile + row,
+                         4 * part_tile, own.nparts - 1);
+        __syncwarp();
+        if (lane == 0) {                                           // ready for the next launch
+          a.tail_flags[own_slot * 4 + quad] = 0;
+          for (int p = 1; p < own.nparts; ++p) a.tail_flags[(((cluster_id + p) * 2) * 2 + int(rank)) * 4 + quad] = 0;
+        }
+        own.nparts = 1;
+      }
+      if (wk.nparts > 1) continue;
       if (a.store_tma) {
         ts.c1 = (c.w0 + bw_0) / a.pool_w; ts.c2 = (c.h0 + bh_0) / a.pool_h; ts.c3 = (c.t0 + bt_0) / a.pool_t; ts.c4 = c.n0 + bn_0;
         epilogue_row_tma(taddr, a.n_tile, nsteps > 0, quad * 32 < box_rows, in_range, bias_s, a.g.relu,
@@ -303,40 +433,67 @@ int pick_stages_pair(int n_tile) {
 
 size_t pair_smem_bytes(int n_tile, int n_bundles) {
   return size_t(pick_stages_pair(n_tile)) * pick_cps(n_tile) * (kABytes + size_t(n_tile / 2) * 128) + 1024 + 4 * kStoreWarpBytes +
-         sizeof(Barriers) +
+         sizeof(Barriers) + sizeof(TailWork) +
          size_t(n_tile) * n_bundles * 4;
 }
 
 template <bool kDense, int kCps>
-cudaError_t launch_pair_t(const UmmaArgs& a, const CUtensorMap& xm, const CUtensorMap& wm, const CUtensorMap& ym,
-                          int sm_count, int stages,
-                          int cols, size_t smem, long long n_items, cudaStream_t stream) {
+cudaError_t prepare_pair_t() {
   static bool attr_done = false;
   if (!attr_done) {
     cudaError_t e = cudaFuncSetAttribute(conv3d_umma_pair_kernel<kDense, kCps>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
     if (e != cudaSuccess) return e;
     attr_done = true;
   }
-  cudaLaunchConfig_t cfg = {};
-  cudaLaunchAttribute attr[1];
+  return cudaSuccess;
+}
+
+void pair_launch_config(cudaLaunchConfig_t& cfg, cudaLaunchAttribute* attr, unsigned grid, size_t smem, cudaStream_t stream) {
+  cfg = cudaLaunchConfig_t{};
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  cfg.gridDim = dim3(grid);
   cfg.blockDim = dim3(kThreadsUmma);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = stream;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  // as many CTA pairs as can be resident at once (persistent kernel), never more than items
+}
+
+// CTA pairs that can be resident at once (the persistent grid), never more than SMs / 2.
+template <bool kDense, int kCps>
+int pair_max_clusters_t(int sm_count, size_t smem) {
   static int max_clusters = 0;
   if (max_clusters == 0) {
-    cfg.gridDim = dim3(unsigned(sm_count & ~1));
+    if (prepare_pair_t<kDense, kCps>() != cudaSuccess) return sm_count / 2;
+    cudaLaunchConfig_t cfg;
+    cudaLaunchAttribute attr[1];
+    pair_launch_config(cfg, attr, unsigned(sm_count & ~1), smem, nullptr);
     int n = 0;
     if (cudaOccupancyMaxActiveClusters(&n, conv3d_umma_pair_kernel<kDense, kCps>, &cfg) != cudaSuccess || n <= 0) n = sm_count / 2;
     max_clusters = n;
   }
-  long long clusters = max_clusters < sm_count / 2 ? max_clusters : sm_count / 2;
+  return max_clusters < sm_count / 2 ? max_clusters : sm_count / 2;
+}
+
+int pair_max_clusters(int n_tile, int n_bundles, bool dense, int sm_count) {
+  const size_t smem = pair_smem_bytes(n_tile, n_bundles);
+  if (pick_cps(n_tile) == 2)
+    return dense ? pair_max_clusters_t<true, 2>(sm_count, smem) : pair_max_clusters_t<false, 2>(sm_count, smem);
+  return dense ? pair_max_clusters_t<true, 1>(sm_count, smem) : pair_max_clusters_t<false, 1>(sm_count, smem);
+}
+
+template <bool kDense, int kCps>
+cudaError_t launch_pair_t(const UmmaArgs& a, const CUtensorMap& xm, const CUtensorMap& wm, const CUtensorMap& ym,
+                          int sm_count, int stages,
+                          int cols, size_t smem, long long n_items, cudaStream_t stream) {
+  cudaError_t e = prepare_pair_t<kDense, kCps>();
+  if (e != cudaSuccess) return e;
+  long long clusters = pair_max_clusters_t<kDense, kCps>(sm_count, smem);
   if (clusters > n_items) clusters = n_items;
-  cfg.gridDim = dim3(unsigned(2 * clusters));
+  cudaLaunchConfig_t cfg;
+  cudaLaunchAttribute attr[1];
+  pair_launch_config(cfg, attr, unsigned(2 * clusters), smem, stream);
   return cudaLaunchKernelEx(&cfg, conv3d_umma_pair_kernel<kDense, kCps>, xm, wm, ym, a, stages, cols);
 }
 
@@ -346,9 +503,52 @@ bool umma_pair_supported(int n_tile, int n_bundles) {
   return n_tile % 32 == 0 && n_tile <= 256 && pick_stages_pair(n_tile) >= 2 && pair_smem_bytes(n_tile, n_bundles) <= 227 * 1024;
 }
 
+// Tail split: decides how many CTA pairs share the items that do not fill a last round (0 = no split)
+// and how much scratch that needs.  `step_ptr_host`: the layout's per-bundle step offsets (sparse path).
+void umma_pair_tail_plan(UmmaArgs* a, const int32_t* step_ptr_host, int sm_count, size_t* scratch_bytes,
+                         size_t* flag_bytes) {
+  a->tail_workers = 0;
+  *scratch_bytes = 0; *flag_bytes = 0;
+  if (!a->store_tma || !umma_pair_supported(a->n_tile, a->n_bundles)) return;
+  const long long n_mtiles = (long long)a->tiles_n * a->tiles_t * a->tiles_h * a->tiles_w;
+  const long long pairs_per_bundle = (n_mtiles + 1) / 2;
+  const long long n_items = pairs_per_bundle * a->n_bundles;
+  const int clusters = pair_max_clusters(a->n_tile, a->n_bundles, a->dense != 0, sm_count);
+  if (clusters <= 0 || n_items <= clusters) return;
+  const long long rounds = n_items / clusters;
+  const int n_tail = int(n_items - rounds * clusters);
+  if (n_tail == 0) return;
+  const int cps = pick_cps(a->n_tile);
+  long long total = 0, g_min = 1 << 30, g_max = 0;
+  for (int t = 0; t < n_tail; ++t) {
+    const int b = int((rounds * clusters + t) / pairs_per_bundle);
+    const int ns = a->dense ? a->steps_dense : step_ptr_host[b + 1] - step_ptr_host[b];
+    if (ns < 8) return;                                   // nothing worth cutting
+    const long long g = (ns + cps - 1) / cps;
+    total += g;
+    g_min = g < g_min ? g : g_min; g_max = g > g_max ? g : g_max;
+  }
+  long long workers = clusters;
+  if (workers > 4LL * n_tail) workers = 4LL * n_tail;     // at most about four parts per item
+  if (workers > total / 4) workers = total / 4;           // at least four step groups per part
+  if (workers <= n_tail) return;
+  const long long range = (total + workers - 1) / workers;
+  if (range / g_min + 2 > kMaxTailSeg) return;
+  // Storing the shares and the owner's fix-up (four warps pulling the other shares through registers)
+  // cost about as much as this many K steps (measured on 256-wide bundles: the split pays for itself
+  // from about 100 steps per item).
+  const long long fixup_groups = (48 + cps - 1) / cps;
+  if (range + fixup_groups >= g_max) return;
+  a->tail_workers = int(workers);
+  // per pair: up to two shares (first and last segment of its range) x two CTAs
+  *scratch_bytes = size_t(workers) * 4 * 128 * a->n_tile * sizeof(float);
+  *flag_bytes = size_t(workers) * 4 * 4 * sizeof(int32_t);
+}
+
 cudaError_t launch_conv_umma_pair(const UmmaArgs& a, const void* xmap, const void* wmap_half, const void* ymap,
                                   int sm_count, cudaStream_t stream) {
   if (!umma_pair_supported(a.n_tile, a.n_bundles) || a.n_splits != 1) return cudaErrorInvalidValue;
+  if (a.tail_workers > 0 && (a.tail_scratch == nullptr || a.tail_flags == nullptr)) return cudaErrorInvalidValue;
   const int stages = pick_stages_pair(a.n_tile);
   const size_t smem = pair_smem_bytes(a.n_tile, a.n_bundles);
   int cols = 32;

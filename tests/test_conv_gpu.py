@@ -182,6 +182,37 @@ def test_umma_pair_kernel_against_oracle(case, dense):
     assert np.abs(y1 - y).max() <= 1e-2 * np.abs(ref).max()
 
 
+TAIL_CASES = [
+    # more tile pairs than CTA pairs, a last round that is not full, and long K: the left-over tiles are cut
+    # along K and shared by the pairs (fp32 partials through scratch, fixed summation order)
+    (256, 256, (3, 3, 3), (4, 8, 28, 28), False),      # 98 tile pairs on 74 CTA pairs, one step per hand-shake
+    (256, 512, (3, 3, 3), (2, 8, 28, 28), False),      # two bundles, left-over items all in the second
+    (256, 128, (3, 3, 3), (4, 8, 28, 28), False),      # narrow bundle: two steps per hand-shake
+    (256, 256, (3, 3, 3), (4, 8, 28, 28), True),       # dense path (computed steps)
+    (256, 256, (3, 3, 3), (4, 8, 27, 29), False),      # ragged boxes
+]
+
+
+@pytest.mark.parametrize("case", TAIL_CASES)
+def test_pair_kernel_tail_split_against_oracle(case):
+    cin, cout, k, (n, t, h, w), dense = case
+    spec = synth.ConvSpec("t", cin, cout, k, (1, 1, 1), tuple(kk // 2 for kk in k), True)
+    y, ref, lay, xd, yt = run_case(spec, n, t, h, w, 4, 4, "none" if dense else "bernoulli", 0.4, torch.bfloat16,
+                                   rt3d.ALGO_AUTO, dense=dense)
+    plan = rt3d.rt3d_last_plan()
+    assert plan["kernel"] == 2 and plan["tail_workers"] > 0, plan
+    check(y, ref, torch.bfloat16, f"tail split {case}")
+    first = yt.clone()
+    for _ in range(3):                       # flags reset themselves; the sum order is fixed
+        lay(xd, yt)
+        torch.cuda.synchronize()
+        assert torch.equal(first, yt)
+    assert rt3d.rt3d_last_device_status() == rt3d.OK
+    y1 = nets.to_numpy(lay(xd, algo=rt3d.ALGO_UMMA), cout)      # single-CTA kernel: whole tiles, other sum order
+    assert rt3d.rt3d_last_plan()["kernel"] == 1
+    assert np.abs(y1 - y).max() <= 1e-2 * np.abs(ref).max()
+
+
 WIDE_GROUP_CASES = [
     # kernel groups matched to the tensor-core footprint (beyond the paper's 4..8): exact step skipping
     (256, 256, (3, 3, 3), (2, 8, 14, 14), 256, 64, 0.25),
@@ -287,6 +318,7 @@ def test_cfg1_c3d_conv3a_full_size(mode):
                           dense=(mode == "dense"))
     rel = check(y, ref, torch.bfloat16, f"cfg1 {mode}")
     assert rel < 1e-2
+    assert rt3d.rt3d_last_plan()["kernel"] == 2                # CTA pairs: 196 tile pairs on 74 pairs of SMs
 
 
 # ------------------------------------------------------------------ host entry point, glue
