@@ -51,8 +51,12 @@ typedef enum {
   RT3D_ALGO_AUTO = 0,   /* tensor-core kernel when the shape allows it, else the CUDA-core kernel */
   RT3D_ALGO_SIMT = 1,   /* CUDA-core kernel driven by the canonical packed index (any shape)      */
   RT3D_ALGO_UMMA = 2,   /* tcgen05 tensor-core kernel, one CTA per tile; RT3D_ERR_UNSUPPORTED if not applicable */
-  RT3D_ALGO_UMMA_PAIR = 3 /* tcgen05 kernel on CTA pairs (two tiles per MMA, weight tile shared by the
+  RT3D_ALGO_UMMA_PAIR = 3, /* tcgen05 kernel on CTA pairs (two tiles per MMA, weight tile shared by the
                              pair); RT3D_ERR_UNSUPPORTED if not applicable                        */
+  RT3D_ALGO_UMMA_HALO = 4  /* tcgen05 kernel on CTA pairs for thin stride-1 layers: the layer's packed weights
+                             stay in shared memory and each output tile's input block (with halo) is
+                             staged once for all kernel locations; RT3D_ERR_UNSUPPORTED if the weights
+                             plus two input blocks do not fit, M > 256, or a stride is not 1      */
 } rt3d_algo;
 
 /* NDHWC activation tensor in DEVICE memory (HOST memory for the *_host entry point), caller-owned. */
@@ -257,7 +261,7 @@ rt3d_status rt3d_conv3d_cost(const rt3d_tensor* x, const rt3d_packed* w, const r
 
 /* How the calling thread's most recent successful convolution call was run (for tests and profiling):
  *   kernel       0 CUDA-core kernel, 1 tensor-core single-CTA kernel, 2 tensor-core CTA-pair kernel,
- *                3 tensor-core small-C_in kernel
+ *                3 tensor-core small-C_in kernel, 4 tensor-core resident-weight (halo) kernel
  *   n_tile       output channels per accumulator tile (tensor-core kernels, else 0)
  *   n_splits     K splits per output tile in the single-CTA kernel (1 = none)
  *   tail_workers CTA pairs that share, cut along K, the output tiles which do not fill a last round

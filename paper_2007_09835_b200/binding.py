@@ -16,7 +16,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.environ.get("RT3D_LIB") or os.path.join(_HERE, "librt3d.so")   # RT3D_LIB: alternative build of the same library
 
 RT3D_F32, RT3D_BF16 = 0, 1
-ALGO_AUTO, ALGO_SIMT, ALGO_UMMA, ALGO_UMMA_PAIR = 0, 1, 2, 3
+ALGO_AUTO, ALGO_SIMT, ALGO_UMMA, ALGO_UMMA_PAIR, ALGO_UMMA_HALO = 0, 1, 2, 3, 4
 OK, ERR_INVALID_ARG, ERR_SHAPE, ERR_MASK_NOT_GROUP_UNIFORM, ERR_UNSUPPORTED, ERR_ALLOC, ERR_CUDA, ERR_TIMEOUT = range(8)
 ERR_WORKSPACE, ERR_NOT_PREPARED = 8, 9
 

@@ -77,7 +77,7 @@ rt3d_status make_geom(const rt3d_tensor* x, const rt3d_packed* w, const rt3d_con
   if (s != RT3D_OK) return s;
   if (!w || !p) return RT3D_ERR_INVALID_ARG;
   if (p->st < 1 || p->sh < 1 || p->sw < 1 || p->pt < 0 || p->ph < 0 || p->pw < 0) return RT3D_ERR_INVALID_ARG;
-  if (p->algo < RT3D_ALGO_AUTO || p->algo > RT3D_ALGO_UMMA_PAIR) return RT3D_ERR_INVALID_ARG;
+  if (p->algo < RT3D_ALGO_AUTO || p->algo > RT3D_ALGO_UMMA_HALO) return RT3D_ERR_INVALID_ARG;
   if (x->c != w->N || x->dtype != w->dtype) return RT3D_ERR_SHAPE;
   const int64_t To = (int64_t(x->t) + 2 * p->pt - w->Kt) / p->st + 1;
   const int64_t Ho = (int64_t(x->h) + 2 * p->ph - w->Kh) / p->sh + 1;
@@ -175,7 +175,7 @@ rt3d_status get_umma_blob(rt3d_packed* h, DeviceBlob* blob, const UmmaLayout* L,
                           strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                           CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return RT3D_ERR_CUDA;
-    if (L->n_tile % 32 == 0) {
+    if (L->n_tile % 16 == 0) {
       cuuint32_t box_half[2] = {64, cuuint32_t(L->n_tile / 2)};
       r = g_encode(reinterpret_cast<CUtensorMap*>(u.wmap_half), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, u.wtiles, dims,
                    strides, box_half, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
@@ -427,6 +427,68 @@ rt3d_status ensure_splitk(rt3d_packed* w, DeviceBlob* blob, size_t bytes, size_t
   return RT3D_OK;
 }
 
+// Resident-weight kernel for thin stride-1 layers: used when the layer qualifies and (unless forced) has
+// at least one tile per SM.  *launched = false (and RT3D_OK) when the caller should take another kernel.
+rt3d_status try_halo(rt3d_packed* w, DeviceBlob* blob, DeviceState* d, const rt3d_tensor* x, const ConvGeom& g,
+                     const float* bias, rt3d_tensor* y, const void* res_data, int res_pitch, bool dense_entry,
+                     bool forced, cudaStream_t st, bool* launched) {
+  *launched = false;
+  if (g.st != 1 || g.sh != 1 || g.sw != 1 || w->M > 256) return RT3D_OK;
+  const int n_tile = round_up(w->M, 16);
+  const int n_chunks = ceil_div(w->N, kChunk);
+  // cheap size screen before the layout is built: all locations kept is the upper bound
+  if (!dense_entry && w->is_dense == 0 && size_t(w->Ks) * n_chunks * (n_tile / 2) * 128 > size_t(4) * 227 * 1024) return RT3D_OK;
+  HaloArgs h;
+  UmmaArgs& a = h.u;
+  a.g = g;
+  // tile: 8 voxels along w times 16 (t, h) lines; one frame thick unless the kernel is 1 high
+  int bt = 1, bh = 16;
+  if (g.Kh == 1) {
+    long long best = -1;
+    for (int t = 1; t <= 16; t *= 2) {
+      const int hh = 16 / t;
+      const long long cost = (long long)ceil_div(g.To, t) * ceil_div(g.Ho, hh) * (t + g.Kt - 1) * hh;
+      if (best < 0 || cost < best) { best = cost; bt = t; bh = hh; }
+    }
+  }
+  a.box = TileBox{1, bt, bh, 8};
+  a.tiles_n = g.n; a.tiles_t = ceil_div(g.To, bt); a.tiles_h = ceil_div(g.Ho, bh); a.tiles_w = ceil_div(g.Wo, 8);
+  const long long m_tiles = (long long)a.tiles_n * a.tiles_t * a.tiles_h * a.tiles_w;
+  if (!forced && m_tiles < d->sm_count) return RT3D_OK;
+  if (m_tiles > (1ll << 30)) return RT3D_OK;
+  const UmmaLayout* L = get_umma_layout(w, n_tile);
+  if (!L || L->n_bundles != 1) return RT3D_OK;
+  a.n_tile = L->n_tile; a.n_bundles = 1; a.n_chunks = L->n_chunks;
+  a.dense = dense_entry ? 1 : 0;
+  a.steps_dense = w->Ks * L->n_chunks;
+  h.n_steps = dense_entry ? a.steps_dense : L->step_ptr[1];
+  if (!umma_halo_plan(&h, dense_entry ? nullptr : L->steps.data())) return RT3D_OK;
+  // waste of the fixed 16 x 8 tile against the free-form boxes of the other kernels
+  if (!forced && m_tiles * 128 > 3 * ((long long)g.n * g.To * g.Ho * g.Wo) / 2) return RT3D_OK;
+  DeviceBlob::Umma* u = nullptr;
+  rt3d_status s = get_umma_blob(w, blob, L, &u);
+  if (s != RT3D_OK) return s;
+  a.step_ptr = u->step_ptr; a.steps = u->steps;
+  a.bias = bias; a.y = y->data; a.sched = d->sched;
+  a.residual = res_data; a.rcs = res_pitch;
+  a.pool_t = a.pool_h = a.pool_w = 1;
+  a.n_splits = 1; a.scratch = nullptr; a.counters = nullptr;
+  a.tail_workers = 0; a.tail_scratch = nullptr; a.tail_flags = nullptr;
+  ConvGeom unit = g;                       // the staged block is a plain box of input voxels
+  CUtensorMap xmap, ymap;
+  if ((s = encode_xmap(x, unit, TileBox{1, h.ht, h.hh, h.hw}, &xmap)) != RT3D_OK) return s;
+  int sb[4] = {1, 1, 1, 1};
+  const bool rect = warp_block(a.box.bw, a.box.bh, a.box.bt, a.box.bn, sb);
+  a.sbw = sb[0]; a.sbh = sb[1];
+  a.store_tma = (rect && encode_ymap(y, sb, 1, 1, 1, &ymap)) ? 1 : 0;
+  cudaError_t e = launch_conv_umma_halo(h, &xmap, u->wmap_half, a.store_tma ? &ymap : nullptr, d->sm_count, st);
+  if (e != cudaSuccess) return RT3D_ERR_CUDA;
+  g_launches.fetch_add(1);
+  t_last_plan = rt3d_plan_info{4, a.n_tile, 1, 0, 0};
+  *launched = true;
+  return RT3D_OK;
+}
+
 rt3d_status conv_impl(const rt3d_tensor* x, const rt3d_packed* wc, const float* bias, const rt3d_conv_params* p,
                       rt3d_tensor* y, void* stream, bool dense_entry, const rt3d_fusion* fz = nullptr) {
   ConvGeom g;
@@ -468,9 +530,9 @@ rt3d_status conv_impl(const rt3d_tensor* x, const rt3d_packed* wc, const float* 
   const bool can_simt = w->g_m <= kMaxGroupSimt && w->g_n <= kMaxGroupSimt;
   if (!can_umma && !can_simt) return RT3D_ERR_UNSUPPORTED;
   if (p->algo == RT3D_ALGO_SIMT && !can_simt) return RT3D_ERR_UNSUPPORTED;
-  if ((p->algo == RT3D_ALGO_UMMA || p->algo == RT3D_ALGO_UMMA_PAIR) && !can_umma) return RT3D_ERR_UNSUPPORTED;
-  const bool use_umma = p->algo == RT3D_ALGO_UMMA || p->algo == RT3D_ALGO_UMMA_PAIR ||
-                        (p->algo == RT3D_ALGO_AUTO && can_umma);
+  const bool want_umma = p->algo == RT3D_ALGO_UMMA || p->algo == RT3D_ALGO_UMMA_PAIR || p->algo == RT3D_ALGO_UMMA_HALO;
+  if (want_umma && !can_umma) return RT3D_ERR_UNSUPPORTED;
+  const bool use_umma = want_umma || (p->algo == RT3D_ALGO_AUTO && can_umma);
   if (!use_umma) {
     if (pooled) return RT3D_ERR_UNSUPPORTED;
     cudaError_t e = launch_conv_simt(w->dtype, g, x->data, y->data, blob->group_ptr, blob->pos_idx, blob->tiles, bias,
@@ -482,11 +544,18 @@ rt3d_status conv_impl(const rt3d_tensor* x, const rt3d_packed* wc, const float* 
   }
 
   const SmallCLayout* SL = nullptr;
-  if (p->algo != RT3D_ALGO_UMMA_PAIR && (!pooled || pl_t == 1) && smallc_eligible(d, w, x, y, p, &SL)) {
+  if (p->algo != RT3D_ALGO_UMMA_PAIR && p->algo != RT3D_ALGO_UMMA_HALO && (!pooled || pl_t == 1) && smallc_eligible(d, w, x, y, p, &SL)) {
     s = launch_smallc(w, blob, d, SL, x, g, bias, y, st, res_data, res_pitch, pl_h, pl_w);
     if (s == RT3D_OK) t_last_plan = rt3d_plan_info{3, SL->n_pad, 1, 0, pooled ? 1 : 0};
     return s;
   }
+
+  if ((p->algo == RT3D_ALGO_AUTO || p->algo == RT3D_ALGO_UMMA_HALO) && !pooled) {
+    bool launched = false;
+    s = try_halo(w, blob, d, x, g, bias, y, res_data, res_pitch, dense_entry, p->algo == RT3D_ALGO_UMMA_HALO, st, &launched);
+    if (s != RT3D_OK || launched) return s;
+  }
+  if (p->algo == RT3D_ALGO_UMMA_HALO) return RT3D_ERR_UNSUPPORTED;
 
   UmmaArgs a;
   a.g = g;

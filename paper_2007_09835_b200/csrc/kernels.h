@@ -76,6 +76,27 @@ void umma_pair_tail_plan(UmmaArgs* a, const int32_t* step_ptr_host, int sm_count
 cudaError_t launch_conv_umma_pair(const UmmaArgs& a, const void* xmap, const void* wmap_half, const void* ymap,
                                   int sm_count, cudaStream_t stream);
 
+constexpr int kHaloMaxMma = 112;      // MMAs per tile the resident-weight kernel can issue (table in the kernel parameters)
+
+// Resident-weight kernel for thin stride-1 layers (CTA pairs): u.box = {1, bt, bh, 8} with bt*bh = 16.
+struct HaloArgs {
+  UmmaArgs u;
+  int n_steps;                        // kept (location, chunk) steps of the single bundle (dense: Ks * n_chunks)
+  int n_mma;                          // K=16 MMAs per tile: 4 per step, fewer where the step is the last, partial chunk
+  uint32_t tab[2 * kHaloMaxMma];      // per MMA: low descriptor words of A (relative to the staged block) and of B
+                                      // (relative to the resident weights), both with the fixed LBO field set
+  int hw, hh, ht;                     // staged input block under one tile: box + kernel extent - 1 per axis
+  int halo_rows;                      // hw * hh * ht voxels
+  int plane_bytes;                    // halo_rows * 128 rounded up to 1024: one 64-channel chunk of the block
+  int stages;                         // staged blocks in flight (filled in by umma_halo_plan)
+};
+// Completes the staging geometry and the MMA table; false if the layer does not qualify (see
+// umma_conv_halo.cu).  steps_host: the bundle's encoded step list (nullptr for the dense path).
+bool umma_halo_plan(HaloArgs* h, const int32_t* steps_host);
+// xmap: input tensor map whose box is the staged block {64, hw, hh, ht, 1}; wmap_half as for the pair kernel.
+cudaError_t launch_conv_umma_halo(const HaloArgs& h, const void* xmap, const void* wmap_half, const void* ymap,
+                                  int sm_count, cudaStream_t stream);
+
 // Arguments of the small-C_in tensor-core kernel (C_in <= 8 at channel pitch 8).
 struct SmallCArgs {
   ConvGeom g;

@@ -137,6 +137,15 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
+// 16 columns into the low half of a 32-entry register array (upper half zero), without taking the array's
+// address in a way that would push it out of registers.
+__device__ __forceinline__ void tmem_ld16_into32(uint32_t taddr, uint32_t (&r)[32]) {
+  uint32_t t[16];
+  tmem_ld16(taddr, t);
+#pragma unroll
+  for (int q = 0; q < 16; ++q) { r[q] = t[q]; r[q + 16] = 0u; }
+}
+
 // Epilogue of NC (16 or 32) accumulator columns of one output voxel: + bias (from shared memory),
 // optional ReLU, round to bf16, store.  `valid` = number of real output channels among the NC
 // (>= NC: 16-byte vector stores; fewer: scalar tail, channels beyond are left untouched).
@@ -176,7 +185,9 @@ __device__ __forceinline__ void epilogue_cols(const uint32_t* v, const float* bi
       reinterpret_cast<uint4*>(dst)[q] = o;
     }
   } else {
-    for (int q = 0; q < valid; ++q) dst[q] = __float2bfloat16_rn(f[q]);
+#pragma unroll
+    for (int q = 0; q < NC; ++q)                 // static indices: f stays in registers
+      if (q < valid) dst[q] = __float2bfloat16_rn(f[q]);
   }
 }
 
@@ -195,7 +206,7 @@ __device__ __forceinline__ void epilogue_row(uint32_t taddr, int n_cols, bool ha
     const bool wide = col + 32 <= n_cols;
     if (has_acc) {
       if (wide) tmem_ld32(taddr + col, v);
-      else tmem_ld16(taddr + col, *reinterpret_cast<uint32_t(*)[16]>(v));
+      else tmem_ld16_into32(taddr + col, v);
     } else {
 #pragma unroll
       for (int q = 0; q < 32; ++q) v[q] = 0u;
@@ -215,7 +226,8 @@ __device__ __forceinline__ void epilogue_row(uint32_t taddr, int n_cols, bool ha
 // at the channel count), so the threads never wait on global stores.  Only warp-level synchronisation
 // is used.
 constexpr uint32_t kStoreStageBytes = 32 * 64;          // one piece
-constexpr uint32_t kStoreWarpBytes = 2 * kStoreStageBytes;
+constexpr uint32_t kStoreBufs = 2;                      // staging buffers per warp = bulk stores in flight per warp
+constexpr uint32_t kStoreWarpBytes = kStoreBufs * kStoreStageBytes;
 
 struct TmaStore {
   const CUtensorMap* map;
@@ -238,7 +250,10 @@ __device__ __forceinline__ void tma_store_5d(const CUtensorMap* map, uint32_t sr
                : "memory");
   asm volatile("cp.async.bulk.commit_group;" ::: "memory");
 }
-__device__ __forceinline__ void tma_store_wait_read_1() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
+// The store issued kStoreBufs pieces ago has finished reading its staging buffer.
+__device__ __forceinline__ void tma_store_wait_read_1() {
+  asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(kStoreBufs - 1) : "memory");
+}
 // Before the warp leaves the kernel: all its bulk stores have completed (shared memory read, global written).
 __device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 
@@ -306,8 +321,8 @@ __device__ __forceinline__ void epilogue_piece_tma(const uint32_t* v, const floa
     writer = (w % pool->pw == 0) && (h % pool->ph == 0) && (t % pool->pt == 0);
     out_row = ((t / pool->pt) * (pool->sbh / pool->ph) + h / pool->ph) * (pool->sbw / pool->pw) + w / pool->pw;
   }
-  const uint32_t buf = ts.smem + (ts.piece & 1u) * kStoreStageBytes;
-  if (lane == 0) tma_store_wait_read_1();          // the store issued two pieces ago has read this buffer
+  const uint32_t buf = ts.smem + (ts.piece % kStoreBufs) * kStoreStageBytes;
+  if (lane == 0) tma_store_wait_read_1();          // the store issued kStoreBufs pieces ago has read this buffer
   __syncwarp();
   const uint32_t row = buf + uint32_t(out_row) * 64u;
   const uint32_t sw = (uint32_t(out_row) >> 1) & 3u;  // 64-byte swizzle: 16-byte chunk index ^= address bits 7..8
@@ -340,7 +355,7 @@ __device__ __forceinline__ void epilogue_row_tma(uint32_t taddr, int n_cols, boo
     const bool wide = col + 32 <= n_cols;
     if (has_acc) {
       if (wide) tmem_ld32(taddr + col, v);
-      else tmem_ld16(taddr + col, *reinterpret_cast<uint32_t(*)[16]>(v));
+      else tmem_ld16_into32(taddr + col, v);
     } else {
 #pragma unroll
       for (int q = 0; q < 32; ++q) v[q] = 0u;
@@ -383,7 +398,7 @@ __device__ __forceinline__ void store_partial_row(uint32_t taddr, int n_cols, bo
     const bool wide = col + 32 <= n_cols;
     if (has_acc) {
       if (wide) tmem_ld32(taddr + col, v);
-      else tmem_ld16(taddr + col, *reinterpret_cast<uint32_t(*)[16]>(v));
+      else tmem_ld16_into32(taddr + col, v);
     } else {
 #pragma unroll
       for (int q = 0; q < 32; ++q) v[q] = 0u;

@@ -213,6 +213,57 @@ def test_pair_kernel_tail_split_against_oracle(case):
     assert np.abs(y1 - y).max() <= 1e-2 * np.abs(ref).max()
 
 
+HALO_CASES = [
+    # resident-weight kernel for thin stride-1 layers: cin, cout, k, pad, (n,t,h,w), dense
+    (64, 144, (1, 3, 3), (0, 1, 1), (2, 4, 24, 20), False),     # R(2+1)D stage-2 spatial conv; ragged tiles
+    (144, 64, (3, 1, 1), (1, 0, 0), (2, 6, 12, 16), False),     # its temporal conv: partial last chunk, tile 16 frames deep
+    (45, 64, (3, 1, 1), (1, 0, 0), (1, 5, 9, 11), False),       # stem temporal conv: 45 channels at pitch 48
+    (32, 32, (3, 3, 3), (1, 1, 1), (1, 4, 20, 12), False),      # 3x3x3: block of 3 x 18 x 10 voxels
+    (64, 128, (1, 1, 1), (0, 0, 0), (3, 3, 17, 9), False),      # one location: no halo; odd tile count
+    (64, 144, (1, 3, 3), (0, 1, 1), (1, 3, 16, 16), True),      # dense path (computed steps)
+    (64, 96, (1, 3, 3), (0, 0, 0), (1, 2, 19, 21), False),      # no padding: output smaller than input
+    (128, 64, (3, 1, 1), (0, 0, 0), (1, 9, 8, 8), False),       # two full chunks, no temporal padding
+]
+
+
+@pytest.mark.parametrize("case", HALO_CASES)
+def test_umma_halo_kernel_against_oracle(case):
+    cin, cout, k, pad, (n, t, h, w), dense = case
+    spec = synth.ConvSpec("h", cin, cout, k, (1, 1, 1), pad, True)
+    y, ref, lay, xd, yt = run_case(spec, n, t, h, w, 4, 4, "none" if dense else "bernoulli", 0.4, torch.bfloat16,
+                                   rt3d.ALGO_UMMA_HALO, dense=dense)
+    assert rt3d.rt3d_last_plan()["kernel"] == 4
+    check(y, ref, torch.bfloat16, f"halo {case}")
+    y1 = nets.to_numpy(lay(xd, algo=rt3d.ALGO_UMMA), cout)      # step-per-location kernel, same weights
+    assert rt3d.rt3d_last_plan()["kernel"] in (1, 2)
+    assert np.abs(y1 - y).max() <= 1e-2 * np.abs(ref).max()
+
+
+def test_umma_halo_kernel_refusals_and_auto_choice():
+    big = synth.ConvSpec("h", 128, 256, (3, 3, 3), (1, 1, 1), (1, 1, 1), True)          # weights far beyond shared memory
+    L = synth.make_layer(big, 7, 1, 4, 4, "bernoulli", 0.4)
+    lay = nets.ConvLayer(big, L["w"], L["bias"], L["mask"], 4, 4, torch.bfloat16)
+    xd = nets.to_device(synth.make_input(1, (1, 2, 8, 8, 128)))
+    with pytest.raises(rt3d.Rt3dError) as e:
+        lay(xd, algo=rt3d.ALGO_UMMA_HALO)
+    assert e.value.status == rt3d.ERR_UNSUPPORTED
+    strided = synth.ConvSpec("h", 64, 64, (1, 3, 3), (1, 2, 2), (0, 1, 1), True)
+    L = synth.make_layer(strided, 7, 2, 4, 4, "bernoulli", 0.4)
+    lay = nets.ConvLayer(strided, L["w"], L["bias"], L["mask"], 4, 4, torch.bfloat16)
+    with pytest.raises(rt3d.Rt3dError) as e:
+        lay(nets.to_device(synth.make_input(1, (1, 2, 16, 16, 64))), algo=rt3d.ALGO_UMMA_HALO)
+    assert e.value.status == rt3d.ERR_UNSUPPORTED
+    # a thin layer with at least one tile per SM: the library picks the resident-weight kernel by itself
+    thin = synth.ConvSpec("h", 64, 144, (1, 3, 3), (1, 1, 1), (0, 1, 1), True)
+    L = synth.make_layer(thin, 7, 3, 4, 4, "bernoulli", 0.4)
+    lay = nets.ConvLayer(thin, L["w"], L["bias"], L["mask"], 4, 4, torch.bfloat16)
+    x = synth.make_input(2, (2, 4, 48, 56, 64))
+    y = nets.to_numpy(lay(nets.to_device(x)), 144)
+    assert rt3d.rt3d_last_plan()["kernel"] == 4
+    ref = oracle.conv3d(x, L["w"], L["mask"], L["bias"], thin.stride, thin.pad, True, round_bf16=True)
+    check(y, ref, torch.bfloat16, "halo auto")
+
+
 WIDE_GROUP_CASES = [
     # kernel groups matched to the tensor-core footprint (beyond the paper's 4..8): exact step skipping
     (256, 256, (3, 3, 3), (2, 8, 14, 14), 256, 64, 0.25),
