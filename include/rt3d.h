@@ -72,6 +72,10 @@ typedef struct {
   int32_t pt, ph, pw;    /* zero padding on both sides of each axis (>= 0)                       */
   int32_t relu;          /* nonzero: y = max(y, 0) fused after the bias                          */
   int32_t algo;          /* rt3d_algo                                                            */
+  int32_t x_pad_zero;    /* nonzero: the caller guarantees that the padding channels c..c_stride-1 of x
+                            hold zeros.  Never needed for correctness (by default no kernel lets them
+                            reach the result); it lets the small-C_in kernel fetch whole image rows in
+                            one request instead of one voxel at a time                              */
 } rt3d_conv_params;
 
 typedef struct rt3d_packed rt3d_packed;   /* opaque; immutable after creation */

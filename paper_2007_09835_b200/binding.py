@@ -36,7 +36,7 @@ class Tensor(ctypes.Structure):
 class ConvParams(ctypes.Structure):
     _fields_ = [("st", ctypes.c_int32), ("sh", ctypes.c_int32), ("sw", ctypes.c_int32),
                 ("pt", ctypes.c_int32), ("ph", ctypes.c_int32), ("pw", ctypes.c_int32),
-                ("relu", ctypes.c_int32), ("algo", ctypes.c_int32)]
+                ("relu", ctypes.c_int32), ("algo", ctypes.c_int32), ("x_pad_zero", ctypes.c_int32)]
 
 
 class Fusion(ctypes.Structure):
@@ -199,9 +199,9 @@ def tensor_desc(t, c: int | None = None) -> Tensor:
     return Tensor(t.data_ptr(), n, tt, h, w, cs if c is None else int(c), cs, dt)
 
 
-def _params(stride, pad, relu, algo) -> ConvParams:
+def _params(stride, pad, relu, algo, x_pad_zero=False) -> ConvParams:
     return ConvParams(int(stride[0]), int(stride[1]), int(stride[2]), int(pad[0]), int(pad[1]), int(pad[2]),
-                      int(bool(relu)), int(algo))
+                      int(bool(relu)), int(algo), int(bool(x_pad_zero)))
 
 
 def _stream_ptr(stream):
@@ -216,10 +216,10 @@ def _bias_ptr(bias):
 
 
 def rt3d_conv3d_sparse(x: Tensor, w: Packed, bias, y: Tensor, stride=(1, 1, 1), pad=(0, 0, 0), relu=False,
-                       algo=ALGO_AUTO, stream=None):
+                       algo=ALGO_AUTO, stream=None, x_pad_zero=False):
     """x, y: Tensor descriptors (device); bias: torch float32 device tensor [M] or None."""
     _check(_lib.rt3d_conv3d_sparse(ctypes.byref(x), w.handle, _bias_ptr(bias),
-                                   ctypes.byref(_params(stride, pad, relu, algo)), ctypes.byref(y),
+                                   ctypes.byref(_params(stride, pad, relu, algo, x_pad_zero)), ctypes.byref(y),
                                    _stream_ptr(stream)), "rt3d_conv3d_sparse")
 
 
@@ -235,19 +235,20 @@ def rt3d_conv3d_sparse_noalloc(x: Tensor, w: Packed, bias, y: Tensor, stride=(1,
 
 
 def rt3d_conv3d_sparse_fused(x: Tensor, w: Packed, bias, y: Tensor, stride=(1, 1, 1), pad=(0, 0, 0), relu=False,
-                             residual: Tensor | None = None, pool=(1, 1, 1), algo=ALGO_AUTO, stream=None):
+                             residual: Tensor | None = None, pool=(1, 1, 1), algo=ALGO_AUTO, stream=None,
+                             x_pad_zero=False):
     """y = pool(act(bias + conv(x) + residual)); residual: descriptor of a device tensor with the un-pooled
     output's extents or None; pool: (1|2, 1|2, 1|2) max-pool window = stride applied after the activation."""
     fz = Fusion(ctypes.pointer(residual) if residual is not None else None, int(pool[0]), int(pool[1]), int(pool[2]))
     _check(_lib.rt3d_conv3d_sparse_fused(ctypes.byref(x), w.handle, _bias_ptr(bias),
-                                         ctypes.byref(_params(stride, pad, relu, algo)), ctypes.byref(fz),
+                                         ctypes.byref(_params(stride, pad, relu, algo, x_pad_zero)), ctypes.byref(fz),
                                          ctypes.byref(y), _stream_ptr(stream)), "rt3d_conv3d_sparse_fused")
 
 
 def rt3d_conv3d_dense(x: Tensor, w: Packed, bias, y: Tensor, stride=(1, 1, 1), pad=(0, 0, 0), relu=False,
-                      algo=ALGO_AUTO, stream=None):
+                       algo=ALGO_AUTO, stream=None, x_pad_zero=False):
     _check(_lib.rt3d_conv3d_dense(ctypes.byref(x), w.handle, _bias_ptr(bias),
-                                  ctypes.byref(_params(stride, pad, relu, algo)), ctypes.byref(y),
+                                  ctypes.byref(_params(stride, pad, relu, algo, x_pad_zero)), ctypes.byref(y),
                                   _stream_ptr(stream)), "rt3d_conv3d_dense")
 
 

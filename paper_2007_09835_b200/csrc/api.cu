@@ -355,7 +355,7 @@ bool smallc_eligible(const DeviceState* d, rt3d_packed* w, const rt3d_tensor* x,
 
 rt3d_status launch_smallc(rt3d_packed* w, DeviceBlob* blob, const DeviceState* d, const SmallCLayout* L,
                           const rt3d_tensor* x, const ConvGeom& g, const float* bias, rt3d_tensor* y, cudaStream_t st,
-                          const void* residual, int rcs, int pool_h, int pool_w) {
+                          const void* residual, int rcs, int pool_h, int pool_w, bool x_pad_zero) {
   DeviceBlob::SmallC* sc = nullptr;
   {
     std::lock_guard<std::mutex> lock(w->mu);
@@ -393,6 +393,17 @@ rt3d_status launch_smallc(rt3d_packed* w, DeviceBlob* blob, const DeviceState* d
   cuuint64_t strides[4] = {cs, cs * x->w, cs * x->w * x->h, cs * x->w * x->h * x->t};
   cuuint32_t bx[5] = {8, cuuint32_t(L->img_w * g.sw), cuuint32_t(L->img_h * g.sh), cuuint32_t(L->img_t), 1};
   cuuint32_t estr[5] = {1, cuuint32_t(g.sw), cuuint32_t(g.sh), 1, 1};
+  // Unit column stride and all 8 channels real (or the caller vouches for zero padding channels): merge the (w, channel) axes, so that the engine fetches each
+  // image row as one contiguous run instead of one 16-byte request per voxel (the tile load was the
+  // kernel's bottleneck).  Otherwise the separate channel axis stays: its out-of-range
+  // fill is what zeroes the padding channels, whatever the caller's buffer holds there.
+  a.merged_cw = (g.sw == 1 && (x->c == 8 || x_pad_zero) && L->img_w * 8 <= 256) ? 1 : 0;
+  if (a.merged_cw) {
+    dims[0] = cuuint64_t(x->w) * 8; dims[1] = 1;
+    strides[0] = cs;                                   // the unit axis never moves
+    bx[0] = cuuint32_t(L->img_w * 8); bx[1] = 1;
+    estr[1] = 1;
+  }
   if (g_encode(&xmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, x->data, dims, strides, bx, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
     return RT3D_ERR_CUDA;
@@ -545,7 +556,7 @@ rt3d_status conv_impl(const rt3d_tensor* x, const rt3d_packed* wc, const float* 
 
   const SmallCLayout* SL = nullptr;
   if (p->algo != RT3D_ALGO_UMMA_PAIR && p->algo != RT3D_ALGO_UMMA_HALO && (!pooled || pl_t == 1) && smallc_eligible(d, w, x, y, p, &SL)) {
-    s = launch_smallc(w, blob, d, SL, x, g, bias, y, st, res_data, res_pitch, pl_h, pl_w);
+    s = launch_smallc(w, blob, d, SL, x, g, bias, y, st, res_data, res_pitch, pl_h, pl_w, p->x_pad_zero != 0);
     if (s == RT3D_OK) t_last_plan = rt3d_plan_info{3, SL->n_pad, 1, 0, pooled ? 1 : 0};
     return s;
   }

@@ -103,6 +103,7 @@ struct SmallCArgs {
   int n_pad, n_pairs;                 // padded output channels; pairs of kept kernel locations
   int n_phases, phase_stride;         // sh*sw phase images per tile, bytes between them in shared memory
   int img_w, phase_bytes;             // voxels per image row; bytes one phase load delivers
+  int merged_cw;                      // 1: the tensor map's first axis is (w, channel) merged: one request per image row
   int tiles_h, tiles_w;               // 16 x 8 output tiles per frame
   int tmem_cols;                      // filled in by the launcher
   int store_tma;                      // 1: TMA-store epilogue (needs ymap)

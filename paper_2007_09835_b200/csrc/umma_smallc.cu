@@ -25,7 +25,7 @@ namespace {
 constexpr int kSmallCStages = 3;
 
 template <int kDummy>
-__global__ void __launch_bounds__(kThreadsUmma, 1)
+__global__ void __launch_bounds__(kThreadsUmma, 3)
 conv3d_umma_smallc_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CUtensorMap ymap,
                           const SmallCArgs a) {
   extern __shared__ unsigned char smem_raw[];
@@ -93,9 +93,15 @@ conv3d_umma_smallc_kernel(const __grid_constant__ CUtensorMap xmap, const __grid
         const uint32_t full = smem_u32(&bars->full[stage]);
         mbar_expect_tx(full, uint32_t(a.n_phases * a.phase_bytes));
         const int w0 = iw * kSmallCTileW * a.g.sw - a.g.pw, h0 = ih * kSmallCTileH * a.g.sh - a.g.ph;
-        for (int ph = 0; ph < a.n_phases; ++ph)      // one strided box per (row, column) stride phase
-          tma_load_5d(halo_smem + stage * halo_stride + ph * a.phase_stride, &xmap, full, 0, w0 + ph % a.g.sw,
-                      h0 + ph / a.g.sw, to * a.g.st - a.g.pt, nn);
+        if (a.merged_cw) {                           // unit column stride: a whole image row is one contiguous run
+          for (int ph = 0; ph < a.n_phases; ++ph)
+            tma_load_5d(halo_smem + stage * halo_stride + ph * a.phase_stride, &xmap, full, w0 * 8, 0, h0 + ph,
+                        to * a.g.st - a.g.pt, nn);
+        } else {
+          for (int ph = 0; ph < a.n_phases; ++ph)    // one strided box per (row, column) stride phase
+            tma_load_5d(halo_smem + stage * halo_stride + ph * a.phase_stride, &xmap, full, 0, w0 + ph % a.g.sw,
+                        h0 + ph / a.g.sw, to * a.g.st - a.g.pt, nn);
+        }
         if (++stage == kSmallCStages) { stage = 0; phase ^= 1u; }
       }
     }
@@ -194,14 +200,6 @@ cudaError_t launch_conv_umma_smallc(const SmallCArgs& a_in, const void* xmap, co
   if (smem > 227 * 1024) return cudaErrorInvalidValue;
   const long long n_items = (long long)a.g.n * a.g.To * a.tiles_h * a.tiles_w;
   if (n_items <= 0) return cudaSuccess;
-  // several CTAs per SM (the layer is bound by its epilogue / output stores): limited by shared
-  // memory, by the 512 TMEM columns of an SM, and kept at four.
-  int per_sm = int((220 * 1024) / (smem + 1024));
-  if (per_sm > 512 / cols) per_sm = 512 / cols;
-  if (per_sm > 4) per_sm = 4;
-  if (per_sm < 1) per_sm = 1;
-  const long long want = (long long)sm_count * per_sm;
-  const int grid = int(n_items < want ? n_items : want);
   if (a.store_tma && ymap == nullptr) return cudaErrorInvalidValue;
   CUtensorMap xm, ym;
   memcpy(&xm, xmap, sizeof(CUtensorMap));
@@ -210,8 +208,30 @@ cudaError_t launch_conv_umma_smallc(const SmallCArgs& a_in, const void* xmap, co
   if (!attr_done) {
     cudaError_t e = cudaFuncSetAttribute(conv3d_umma_smallc_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
     if (e != cudaSuccess) return e;
+    // ask for the largest shared-memory carve-out: with the default one fewer CTAs fit an SM than the sizes allow
+    e = cudaFuncSetAttribute(conv3d_umma_smallc_kernel<0>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+    if (e != cudaSuccess) return e;
     attr_done = true;
   }
+  // Several CTAs per SM (the layer is bound by the latencies of its epilogue): as many as are really resident
+  // at once, counted here from the register file, the shared memory (228 KB per SM, 1 KB reserved per CTA)
+  // and the 512 TMEM columns of an SM (a CTA that cannot allocate its columns would spin inside
+  // tcgen05.alloc), at most four.  (cudaOccupancyMaxActiveBlocksPerMultiprocessor answers 1 for this kernel
+  // whatever the sizes, while two and three CTAs per SM measurably run side by side.)  The grid is exactly
+  // that many persistent CTAs: surplus CTAs would run as a ragged second wave.
+  static int regs_per_thread = 0;
+  if (regs_per_thread == 0) {
+    cudaFuncAttributes fa;
+    regs_per_thread = cudaFuncGetAttributes(&fa, conv3d_umma_smallc_kernel<0>) == cudaSuccess ? fa.numRegs : 128;
+  }
+  int per_sm = 65536 / (((regs_per_thread + 7) & ~7) * kThreadsUmma);
+  const int by_smem = int((228 * 1024) / (smem + 1024));
+  if (per_sm > by_smem) per_sm = by_smem;
+  if (per_sm > 512 / cols) per_sm = 512 / cols;
+  if (per_sm > 4) per_sm = 4;
+  if (per_sm < 1) per_sm = 1;
+  const long long want = (long long)sm_count * per_sm;
+  const int grid = int(n_items < want ? n_items : want);
   conv3d_umma_smallc_kernel<0><<<grid, kThreadsUmma, smem, stream>>>(xm, ym, a);
   return cudaGetLastError();
 }

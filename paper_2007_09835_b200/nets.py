@@ -52,23 +52,26 @@ class ConvLayer:
     def alloc_out(self, x: torch.Tensor) -> torch.Tensor:
         return torch.zeros(self.out_shape(x), dtype=self.dtype, device=x.device)
 
-    def __call__(self, x: torch.Tensor, y: torch.Tensor | None = None, algo=B.ALGO_AUTO, relu=None, stream=None):
+    def __call__(self, x: torch.Tensor, y: torch.Tensor | None = None, algo=B.ALGO_AUTO, relu=None, stream=None,
+                 x_pad_zero=False):
+        """x_pad_zero: the channels of x beyond spec.cin are known to hold zeros (true for tensors made by
+        `to_device`); lets the first-layer kernel fetch whole image rows per request."""
         if y is None:
             y = self.alloc_out(x)
         xd = B.tensor_desc(x, self.spec.cin)
         yd = B.tensor_desc(y, self.spec.cout)
         fn = B.rt3d_conv3d_dense if self.dense else B.rt3d_conv3d_sparse
         fn(xd, self.packed, self.bias, yd, self.spec.stride, self.spec.pad,
-           self.spec.relu if relu is None else relu, algo, stream)
+           self.spec.relu if relu is None else relu, algo, stream, x_pad_zero)
         return y
 
     def fused(self, x: torch.Tensor, y: torch.Tensor, residual: torch.Tensor | None = None, pool=(1, 1, 1),
-              relu=None, algo=B.ALGO_AUTO, stream=None):
+              relu=None, algo=B.ALGO_AUTO, stream=None, x_pad_zero=False):
         """y = pool(act(conv(x) + bias + residual)) in one launch (rt3d_conv3d_sparse_fused)."""
         res = None if residual is None else B.tensor_desc(residual, self.spec.cout)
         B.rt3d_conv3d_sparse_fused(B.tensor_desc(x, self.spec.cin), self.packed, self.bias,
                                    B.tensor_desc(y, self.spec.cout), self.spec.stride, self.spec.pad,
-                                   self.spec.relu if relu is None else relu, res, pool, algo, stream)
+                                   self.spec.relu if relu is None else relu, res, pool, algo, stream, x_pad_zero)
         return y
 
     def cost(self, x: torch.Tensor):
@@ -108,14 +111,15 @@ class Workspace:
 class C3DNet:
     """C3D-shaped forward: 8 convs (3x3x3, ReLU) and 5 max-pools.  `layers` maps conv name -> ConvLayer."""
 
-    def __init__(self, plan, layers, fuse_pool: bool = False):
+    def __init__(self, plan, layers, fuse_pool: bool = False, input_pad_zero: bool = True):
         self.plan = plan
         self.layers = layers
         self.fuse_pool = fuse_pool      # conv + ReLU + un-padded 2-wide max-pool in one launch where the library can
+        self.input_pad_zero = input_pad_zero    # the clip tensor comes from to_device(): channels 3..7 are zeros
         self.ws = Workspace()
         self.fused_ok = {}              # conv name -> did the fused call apply (decided on first use per shape)
 
-    def _try_fused(self, op, pool, x, algo, stream):
+    def _try_fused(self, op, pool, x, algo, stream, x_pad_zero=False):
         """Runs conv `op` with `pool` fused; returns the pooled tensor or None if the library declines."""
         if any(pool.pad) or tuple(pool.k) != tuple(pool.stride) or any(k not in (1, 2) for k in pool.k):
             return None
@@ -128,7 +132,7 @@ class C3DNet:
         shape = (n, to // pool.k[0], ho // pool.k[1], wo // pool.k[2], pitch_for(op.cout, x.dtype))
         y = self.ws.get(pool.name, shape, x.dtype, x.device)
         try:
-            layer.fused(x, y, pool=pool.k, algo=algo, stream=stream)
+            layer.fused(x, y, pool=pool.k, algo=algo, stream=stream, x_pad_zero=x_pad_zero)
         except B.Rt3dError as e:
             if e.status != B.ERR_UNSUPPORTED:
                 raise
@@ -144,9 +148,10 @@ class C3DNet:
             if op is skip:
                 continue
             if hasattr(op, "cout"):
+                pad0 = self.input_pad_zero and i == 0
                 nxt = self.plan[i + 1] if i + 1 < len(self.plan) else None
                 if self.fuse_pool and nxt is not None and not hasattr(nxt, "cout"):
-                    y = self._try_fused(op, nxt, x, algo, stream)
+                    y = self._try_fused(op, nxt, x, algo, stream, pad0)
                     if y is not None:
                         x, c, skip = y, op.cout, nxt
                         if keep is not None:
@@ -154,7 +159,7 @@ class C3DNet:
                         continue
                 layer = self.layers[op.name]
                 y = self.ws.get(op.name, layer.out_shape(x), x.dtype, x.device)
-                x = layer(x, y, algo=algo, stream=stream)
+                x = layer(x, y, algo=algo, stream=stream, x_pad_zero=pad0)
                 c = op.cout
             else:
                 n, t, h, w, cs = x.shape

@@ -125,6 +125,27 @@ def test_small_cin_kernel_against_oracle(case):
     check(ys, ref, torch.bfloat16, f"small-cin simt {case}")
 
 
+def test_small_cin_padding_channels():
+    """Channels 3..7 of a 3-channel input at pitch 8 are padding.  By default nothing the caller left there
+    may reach the result; with x_pad_zero the caller vouches for zeros and the kernel fetches whole rows."""
+    spec = synth.ConvSpec("c1", 3, 64, (3, 3, 3), (1, 1, 1), (1, 1, 1), True)
+    L = synth.make_layer(spec, 7, 21, 4, 4, "bernoulli", 0.4)
+    x = synth.make_input(721, (2, 5, 21, 19, 3))
+    ref = oracle.conv3d(x, L["w"], L["mask"], L["bias"], spec.stride, spec.pad, True, round_bf16=True)
+    lay = nets.ConvLayer(spec, L["w"], L["bias"], L["mask"], 4, 4, torch.bfloat16)
+    xd = nets.to_device(x)
+    y0 = lay(xd).clone()
+    assert rt3d.rt3d_last_plan()["kernel"] == 3
+    check(nets.to_numpy(y0, 64), ref, torch.bfloat16, "small-C default")
+    y1 = lay(xd, x_pad_zero=True)
+    assert rt3d.rt3d_last_plan()["kernel"] == 3
+    assert torch.equal(y0, y1)                               # same arithmetic, only the loads differ
+    dirty = xd.clone()
+    dirty[..., 3:] = float("nan")                            # garbage in the padding channels
+    y2 = lay(dirty)
+    assert torch.equal(y0, y2)
+
+
 def test_small_cin_all_pruned_outputs_bias():
     spec = synth.ConvSpec("c", 3, 32, (3, 3, 3), (1, 1, 1), (1, 1, 1), False)
     L = synth.make_layer(spec, 7, 4, 4, 4, "bernoulli", 0.5)
