@@ -178,6 +178,19 @@ def time_networks(torch, rt3d, nets, dev, iters=20):
     out["r2plus1d_kgs_b8_clips_per_s"] = 8 / ms * 1e3
     out["r2plus1d_kgs_b8_ms"] = ms
     out["r2plus1d_launches"] = rnet.n_launches()
+    del rnet, rlayers
+
+    # S3D-shaped network (separable 3-D Inception, 16 x 224 x 224 clips, KGS about 2.1x), batch 8
+    splan = synth.s3d_plan()
+    slayers = {}
+    for i, sp in enumerate(synth.s3d_convs(splan)):
+        L = synth.make_layer(sp, 5, i, 4, 4, "bernoulli", 1 / 2.1)
+        slayers[sp.name] = nets.ConvLayer(sp, L["w"], L["bias"], L["mask"], 4, 4, torch.bfloat16, device=dev)
+    snet = nets.S3DNet(splan, slayers)
+    x = nets.to_device(synth.make_input(5, (8, 16, 224, 224, 3)), torch.bfloat16, device=dev)
+    ms = timed(nets.GraphedForward(snet, x))
+    out["s3d_kgs_b8_clips_per_s"] = 8 / ms * 1e3
+    out["s3d_kgs_b8_ms"] = ms
     return out
 
 

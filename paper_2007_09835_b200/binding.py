@@ -199,6 +199,17 @@ def tensor_desc(t, c: int | None = None) -> Tensor:
     return Tensor(t.data_ptr(), n, tt, h, w, cs if c is None else int(c), cs, dt)
 
 
+def channel_slice_desc(t, offset: int, c: int) -> Tensor:
+    """Channels [offset, offset + c) of a dense NDHWC torch tensor as an rt3d_tensor (same voxel pitch): lets a
+    layer write its output straight into its place of a channel concatenation.  offset must keep the data
+    pointer 16-byte aligned (a multiple of 8 bf16 / 4 fp32 channels)."""
+    d = tensor_desc(t)
+    if offset < 0 or c < 1 or offset + c > d.c_stride:
+        raise ValueError("channel slice out of range")
+    es = 2 if d.dtype == RT3D_BF16 else 4
+    return Tensor(t.data_ptr() + offset * es, d.n, d.t, d.h, d.w, int(c), d.c_stride, d.dtype)
+
+
 def _params(stride, pad, relu, algo, x_pad_zero=False) -> ConvParams:
     return ConvParams(int(stride[0]), int(stride[1]), int(stride[2]), int(pad[0]), int(pad[1]), int(pad[2]),
                       int(bool(relu)), int(algo), int(bool(x_pad_zero)))

@@ -65,6 +65,11 @@ class ConvLayer:
            self.spec.relu if relu is None else relu, algo, stream, x_pad_zero)
         return y
 
+    def run_desc(self, xd, yd, algo=B.ALGO_AUTO, stream=None):
+        """Same call on ready-made descriptors (e.g. a channel slice of a concatenation buffer as output)."""
+        fn = B.rt3d_conv3d_dense if self.dense else B.rt3d_conv3d_sparse
+        fn(xd, self.packed, self.bias, yd, self.spec.stride, self.spec.pad, self.spec.relu, algo, stream)
+
     def fused(self, x: torch.Tensor, y: torch.Tensor, residual: torch.Tensor | None = None, pool=(1, 1, 1),
               relu=None, algo=B.ALGO_AUTO, stream=None, x_pad_zero=False):
         """y = pool(act(conv(x) + bias + residual)) in one launch (rt3d_conv3d_sparse_fused)."""
@@ -217,6 +222,56 @@ class R2Plus1DNet:
     def n_launches(self) -> int:
         per_block = 4 if self.fuse_residual else 5
         return len(self.stem) + sum(per_block + (blk.shortcut is not None) for blk in self.blocks)
+
+
+class S3DNet:
+    """S3D-shaped forward (separable 3-D Inception): stem convs and pools, then Inception blocks whose four
+    branches write straight into their channel slice of the block's output tensor (no concat pass)."""
+
+    def __init__(self, plan, layers, input_pad_zero: bool = True):
+        self.plan, self.layers = plan, layers
+        self.input_pad_zero = input_pad_zero
+        self.ws = Workspace()
+
+    def _conv(self, spec, x, algo, stream, pad0=False):
+        layer = self.layers[spec.name]
+        y = self.ws.get(spec.name, layer.out_shape(x), x.dtype, x.device)
+        return layer(x, y, algo=algo, stream=stream, x_pad_zero=pad0)
+
+    def _pool(self, spec, x, c, stream):
+        n, t, h, w, cs = x.shape
+        ext = [(d + 2 * p - k) // s + 1 for d, p, k, s in zip((t, h, w), spec.pad, spec.k, spec.stride)]
+        y = self.ws.get(spec.name, (n, ext[0], ext[1], ext[2], cs), x.dtype, x.device)
+        return maxpool(x, c, spec, y, stream=stream)
+
+    def forward(self, x: torch.Tensor, algo=B.ALGO_AUTO, keep=None, stream=None) -> torch.Tensor:
+        c = self.plan[0].cin
+        for i, op in enumerate(self.plan):
+            if hasattr(op, "b0"):                                   # Inception block
+                n, t, h, w, _ = x.shape
+                out = self.ws.get(op.name, (n, t, h, w, op.cout), x.dtype, x.device)
+                xd = B.tensor_desc(x, op.cin)
+                off = 0
+                self.layers[op.b0.name].run_desc(xd, B.channel_slice_desc(out, off, op.b0.cout), algo, stream)
+                off += op.b0.cout
+                for br in (op.b1, op.b2):
+                    a = self._conv(br[0], x, algo, stream)
+                    b = self._conv(br[1], a, algo, stream)
+                    self.layers[br[2].name].run_desc(B.tensor_desc(b, br[2].cin), B.channel_slice_desc(out, off, br[2].cout),
+                                                     algo, stream)
+                    off += br[2].cout
+                p = self._pool(op.pool, x, op.cin, stream)
+                self.layers[op.b3.name].run_desc(B.tensor_desc(p, op.cin), B.channel_slice_desc(out, off, op.b3.cout),
+                                                 algo, stream)
+                x, c = out, op.cout
+            elif hasattr(op, "cout"):
+                x = self._conv(op, x, algo, stream, pad0=self.input_pad_zero and i == 0)
+                c = op.cout
+            else:
+                x = self._pool(op, x, c, stream)
+            if keep is not None:
+                keep[op.name] = x
+        return x
 
 
 class GraphedForward:

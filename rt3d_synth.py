@@ -199,6 +199,75 @@ def r2plus1d18_plan():
 
 
 # --------------------------------------------------------------------- layer instances
+@dataclasses.dataclass(frozen=True)
+class InceptionSpec:
+    """One Inception block of the S3D-shaped network: four branches whose outputs are concatenated along
+    the channels in this order: 1x1x1; 1x1x1 then separable 3x3x3 (1x3x3 + 3x1x1); the same again with other
+    widths; 3x3x3 stride-1 max-pool then 1x1x1.  Every conv is followed by ReLU."""
+    name: str
+    b0: ConvSpec
+    b1: tuple            # (1x1x1 reduce, 1x3x3, 3x1x1)
+    b2: tuple            # (1x1x1 reduce, 1x3x3, 3x1x1)
+    pool: PoolSpec
+    b3: ConvSpec
+
+    @property
+    def cin(self):
+        return self.b0.cin
+
+    @property
+    def cout(self):
+        return self.b0.cout + self.b1[2].cout + self.b2[2].cout + self.b3.cout
+
+    def convs(self):
+        return (self.b0,) + tuple(self.b1) + tuple(self.b2) + (self.b3,)
+
+
+def _sep3(name, cin, cout):
+    return (ConvSpec(name + ".s", cin, cout, (1, 3, 3), (1, 1, 1), (0, 1, 1), True),
+            ConvSpec(name + ".t", cout, cout, (3, 1, 1), (1, 1, 1), (1, 0, 0), True))
+
+
+def s3d_plan():
+    """S3D-shaped network (separable 3-D Inception): list of ConvSpec / PoolSpec / InceptionSpec in execution
+    order; input is 16 x 224 x 224 x 3.  Widths are those of the Inception-v1 table the architecture uses."""
+    plan = [ConvSpec("conv1.s", 3, 64, (1, 7, 7), (1, 2, 2), (0, 3, 3), True),
+            ConvSpec("conv1.t", 64, 64, (7, 1, 1), (2, 1, 1), (3, 0, 0), True),
+            PoolSpec("pool1", (1, 3, 3), (1, 2, 2), (0, 1, 1)),
+            ConvSpec("conv2b", 64, 64, (1, 1, 1), (1, 1, 1), (0, 0, 0), True)]
+    plan += list(_sep3("conv2c", 64, 192))
+    plan.append(PoolSpec("pool2", (1, 3, 3), (1, 2, 2), (0, 1, 1)))
+    table = [("mixed3b", 192, 64, 96, 128, 16, 32, 32), ("mixed3c", 256, 128, 128, 192, 32, 96, 64), "pool3",
+             ("mixed4b", 480, 192, 96, 208, 16, 48, 64), ("mixed4c", 512, 160, 112, 224, 24, 64, 64),
+             ("mixed4d", 512, 128, 128, 256, 24, 64, 64), ("mixed4e", 512, 112, 144, 288, 32, 64, 64),
+             ("mixed4f", 528, 256, 160, 320, 32, 128, 128), "pool4",
+             ("mixed5b", 832, 256, 160, 320, 32, 128, 128), ("mixed5c", 832, 384, 192, 384, 48, 128, 128)]
+    for row in table:
+        if row == "pool3":
+            plan.append(PoolSpec("pool3", (3, 3, 3), (2, 2, 2), (1, 1, 1)))
+        elif row == "pool4":
+            plan.append(PoolSpec("pool4", (2, 2, 2), (2, 2, 2), (0, 0, 0)))
+        else:
+            nm, cin, b0, b1a, b1b, b2a, b2b, b3 = row
+            one = lambda tag, ci, co: ConvSpec(f"{nm}.{tag}", ci, co, (1, 1, 1), (1, 1, 1), (0, 0, 0), True)  # noqa: E731
+            plan.append(InceptionSpec(nm, one("b0", cin, b0),
+                                      (one("b1a", cin, b1a),) + _sep3(nm + ".b1", b1a, b1b),
+                                      (one("b2a", cin, b2a),) + _sep3(nm + ".b2", b2a, b2b),
+                                      PoolSpec(nm + ".pool", (3, 3, 3), (1, 1, 1), (1, 1, 1)), one("b3", cin, b3)))
+    return plan
+
+
+def s3d_convs(plan):
+    """All ConvSpec of an S3D-shaped plan in execution order."""
+    out = []
+    for op in plan:
+        if isinstance(op, ConvSpec):
+            out.append(op)
+        elif isinstance(op, InceptionSpec):
+            out += list(op.convs())
+    return out
+
+
 def make_layer(spec: ConvSpec, cfg: int, layer: int, g_m: int, g_n: int, mask_kind: str,
                mask_arg, seed: int = BASE_SEED):
     """Draw weights, bias and a KGS / vanilla mask for one layer.

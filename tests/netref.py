@@ -71,3 +71,46 @@ def r2plus1d_reference(stem, blocks, layers, x):
         rec[blk.name + ".out"] = ((cur, sc), out)
         cur = oracle.bf16_round(out)
     return rec, cur
+
+
+def make_s3d_layers(cfg, density, g_m=4, g_n=4):
+    plan = synth.s3d_plan()
+    layers = {sp.name: synth.make_layer(sp, cfg, i, g_m, g_n, "bernoulli", density)
+              for i, sp in enumerate(synth.s3d_convs(plan))}
+    return plan, layers
+
+
+def s3d_reference(plan, layers, x):
+    """Oracle forward of the S3D-shaped network; records[name] = (input, unrounded output) per conv / pool,
+    records[block] = (input, concatenated bf16 output) per Inception block."""
+    rec = {}
+
+    def conv(sp, inp):
+        L = layers[sp.name]
+        out = oracle.conv3d(inp, L["w"], L["mask"], L["bias"], sp.stride, sp.pad, sp.relu, round_bf16=True)
+        rec[sp.name] = (inp, out)
+        return oracle.bf16_round(out)
+
+    def pool(sp, inp):
+        out = oracle.maxpool3d(inp, sp.k, sp.stride, sp.pad)
+        rec[sp.name] = (inp, out)
+        return out
+
+    cur = x
+    for op in plan:
+        if isinstance(op, synth.ConvSpec):
+            cur = conv(op, cur)
+        elif isinstance(op, synth.PoolSpec):
+            cur = pool(op, cur)
+        else:
+            inp = cur
+            parts = [conv(op.b0, inp)]
+            for br in (op.b1, op.b2):
+                t = inp
+                for sp in br:
+                    t = conv(sp, t)
+                parts.append(t)
+            parts.append(conv(op.b3, pool(op.pool, inp)))
+            cur = np.concatenate(parts, axis=-1)
+            rec[op.name] = (inp, cur)
+    return rec, cur

@@ -150,6 +150,55 @@ def test_r2plus1d_free_running_batch8(r21d, fuse):
     assert e <= TOL_FREE, e
 
 
+# ------------------------------------------------------------------------------ S3D-shaped
+@pytest.fixture(scope="module")
+def s3d():
+    plan, layers = netref.make_s3d_layers(5, 1 / 2.1)
+    x = oracle.bf16_round(synth.make_input(5, (1, 16, 224, 224, 3)))
+    rec, final = netref.s3d_reference(plan, layers, x)
+    return plan, layers, x, rec, final
+
+
+def test_s3d_layers_teacher_forced(s3d):
+    plan, layers, x, rec, final = s3d
+    specs = synth.s3d_convs(plan)
+    dl = device_layers(layers, specs)
+    dense_macs = kept_macs = 0
+    for sp in specs:
+        inp, ref = rec[sp.name]
+        xd = nets.to_device(inp)
+        y = nets.to_numpy(dl[sp.name](xd), sp.cout)
+        assert (ref != 0).mean() > 0.10, sp.name
+        e = rel_err(y, ref)
+        assert e <= TOL, (sp.name, e)
+        k, d, _ = dl[sp.name].cost(xd)
+        kept_macs += k; dense_macs += d
+    for op in plan:
+        pools = [op] if isinstance(op, synth.PoolSpec) else ([op.pool] if isinstance(op, synth.InceptionSpec) else [])
+        for ps in pools:
+            inp, ref = rec[ps.name]
+            c = inp.shape[-1]
+            y = nets.to_numpy(nets.maxpool(nets.to_device(inp), c, ps), c)
+            np.testing.assert_array_equal(y, ref)
+    assert rt3d.rt3d_last_device_status() == rt3d.OK
+    assert abs(dense_macs / 1e9 - 17.978) < 0.01                 # dense conv work of the S3D-shaped stack per clip
+    assert 1.9 < dense_macs / kept_macs < 2.3                    # about 2.1x FLOPs pruning (Table 2)
+
+
+def test_s3d_free_running_forward(s3d):
+    plan, layers, x, rec, final = s3d
+    net = nets.S3DNet(plan, device_layers(layers, synth.s3d_convs(plan)))
+    keep = {}
+    y = nets.to_numpy(net.forward(nets.to_device(x), keep=keep), 1024)
+    assert y.shape == (1, 2, 7, 7, 1024)
+    assert rt3d.rt3d_last_device_status() == rt3d.OK
+    # the first Inception block: every branch landed in its channel slice
+    blk = nets.to_numpy(keep["mixed3b"], 256)
+    assert rel_err(blk, rec["mixed3b"][1]) <= TOL_FREE
+    assert (final != 0).mean() > 0.10
+    assert rel_err(y, final) <= TOL_FREE
+
+
 # --------------------------------------------------------------------------- sparsity sweep
 SWEEP_SPEC = synth.ConvSpec("sweep", 256, 256, (3, 3, 3), (1, 1, 1), (1, 1, 1), True)
 
