@@ -337,6 +337,37 @@ def test_layer_plans_reproduce_paper_totals():
 
 
 # -------------------------------------------------------------------- generator sanity
+def test_s3d_plan_is_consistent():
+    """The paper gives no S3D totals (only its 2.1x FLOPs pruning rate), so this pins the plan's internal
+    consistency: every op consumes what the previous one produces, Inception branches concatenate to the
+    next block's input width, extents follow the pooling schedule, slices stay 16-byte aligned."""
+    plan = synth.s3d_plan()
+    t, h, w, c = 16, 224, 224, 3
+    n_convs = 0
+    for op in plan:
+        if isinstance(op, synth.ConvSpec):
+            assert op.cin == c, op.name
+            t, h, w = op.out_extent(t, h, w)
+            c = op.cout
+            n_convs += 1
+        elif isinstance(op, synth.PoolSpec):
+            t, h, w = [(d + 2 * p - k) // s + 1 for d, p, k, s in zip((t, h, w), op.pad, op.k, op.stride)]
+        else:
+            assert op.cin == c, op.name
+            for br in (op.b1, op.b2):
+                assert br[0].cin == c and br[1].cin == br[0].cout and br[2].cin == br[1].cout == br[2].cout
+            assert op.b3.cin == c and op.b0.cin == c
+            assert [(d + 2 * p - k) // s + 1 for d, p, k, s in zip((t, h, w), op.pool.pad, op.pool.k, op.pool.stride)] == [t, h, w]
+            for sp in op.convs():
+                assert sp.out_extent(t, h, w) == (t, h, w)            # branches keep the extents
+                assert sp.cout % 8 == 0                               # channel slices start on 16-byte boundaries
+            c = op.cout
+            n_convs += 8
+    assert (t, h, w, c) == (2, 7, 7, 1024)
+    assert n_convs == 5 + 9 * 8 == len(synth.s3d_convs(plan))
+    assert [op.cout for op in plan if isinstance(op, synth.InceptionSpec)] == [256, 480, 512, 512, 512, 528, 832, 832, 1024]
+
+
 def test_generator_is_counter_based_and_calibrated():
     a = synth.splitmix64(123, 0, 1000)
     b = synth.splitmix64(123, 500, 500)
