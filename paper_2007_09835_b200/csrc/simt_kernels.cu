@@ -10,6 +10,7 @@
 #include <cuda_bf16.h>
 
 #include "kernels.h"
+#include "pdl.cuh"
 
 namespace rt3d {
 namespace {
@@ -30,6 +31,7 @@ conv3d_kgs_simt_kernel(ConvGeom g, const T* __restrict__ x, T* __restrict__ y,
                        const int32_t* __restrict__ group_ptr, const uint16_t* __restrict__ pos_idx,
                        const T* __restrict__ tiles, const float* __restrict__ bias,
                        int g_m_rt, int g_n_rt, int Q, long long total_voxels, const T* __restrict__ residual, int rcs) {
+  pdl_entry();
   constexpr int MAXM = GM ? GM : 8;
   constexpr int MAXN = GN ? GN : 8;
   const int g_m = GM ? GM : g_m_rt;
@@ -99,14 +101,17 @@ cudaError_t launch_conv_t(const ConvGeom& g, const void* x, void* y, const int32
   const T* xt = static_cast<const T*>(x);
   T* yt = static_cast<T*>(y);
   const T* tt = static_cast<const T*>(tiles);
+  LaunchSetup ls(grid, dim3(kThreads), 0, stream);
+  const T* rt = static_cast<const T*>(residual);
+  cudaError_t le = cudaSuccess;
 #define RT3D_LAUNCH(GM_, GN_) \
-  conv3d_kgs_simt_kernel<T, GM_, GN_, DENSE><<<grid, kThreads, 0, stream>>>(g, xt, yt, group_ptr, pos_idx, tt, bias, g_m, g_n, Q, total, static_cast<const T*>(residual), rcs)
+  le = cudaLaunchKernelEx(&ls.cfg, conv3d_kgs_simt_kernel<T, GM_, GN_, DENSE>, g, xt, yt, group_ptr, pos_idx, tt, bias, g_m, g_n, Q, total, rt, rcs)
   if (g_m == 4 && g_n == 4) RT3D_LAUNCH(4, 4);
   else if (g_m == 8 && g_n == 4) RT3D_LAUNCH(8, 4);
   else if (g_m == 8 && g_n == 8) RT3D_LAUNCH(8, 8);
   else RT3D_LAUNCH(0, 0);
 #undef RT3D_LAUNCH
-  return cudaGetLastError();
+  return le;
 }
 
 // ------------------------------------------------------------------------------- max-pool
@@ -114,6 +119,7 @@ template <typename T>
 __global__ void maxpool3d_kernel(const T* __restrict__ x, int t, int h, int w, int c, int xcs,
                                  int kt, int kh, int kw, int st, int sh, int sw, int pt, int ph, int pw,
                                  T* __restrict__ y, int To, int Ho, int Wo, int ycs, long long total) {
+  pdl_entry();
   const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= total) return;
   const int cc = int(idx % c);
@@ -143,6 +149,7 @@ __global__ void maxpool3d_kernel(const T* __restrict__ x, int t, int h, int w, i
 __global__ void maxpool3d_bf16x8_kernel(const uint4* __restrict__ x, int t, int h, int w, int c8, int xcs8,
                                         int kt, int kh, int kw, int st, int sh, int sw, int pt, int ph, int pw,
                                         uint4* __restrict__ y, int To, int Ho, int Wo, int ycs8, long long total) {
+  pdl_entry();
   const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= total) return;
   const int cc = int(idx % c8);
@@ -180,6 +187,7 @@ __global__ void maxpool3d_bf16x8_kernel(const uint4* __restrict__ x, int t, int 
 template <typename T>
 __global__ void add_relu_kernel(const T* __restrict__ a, int acs, const T* __restrict__ b, int bcs,
                                 T* __restrict__ y, int ycs, int c, int relu, long long total) {
+  pdl_entry();
   const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= total) return;
   const int cc = int(idx % c);
@@ -192,6 +200,7 @@ __global__ void add_relu_kernel(const T* __restrict__ a, int acs, const T* __res
 __global__ void add_relu_bf16x8_kernel(const uint4* __restrict__ a, int acs8, const uint4* __restrict__ b,
                                        int bcs8, uint4* __restrict__ y, int ycs8, int c8, int relu,
                                        long long total) {
+  pdl_entry();
   const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= total) return;
   const int cc = int(idx % c8);
@@ -231,22 +240,19 @@ cudaError_t launch_maxpool3d(int dtype, const void* x, int n, int t, int h, int 
   const int threads = 256;
   if (dtype == 1 && c % 8 == 0 && xcs % 8 == 0 && ycs % 8 == 0) {
     const long long total = vox * (c / 8);
-    maxpool3d_bf16x8_kernel<<<(unsigned)((total + threads - 1) / threads), threads, 0, stream>>>(
-        static_cast<const uint4*>(x), t, h, w, c / 8, xcs / 8, kt, kh, kw, st, sh, sw, pt, ph, pw,
-        static_cast<uint4*>(y), To, Ho, Wo, ycs / 8, total);
+    LaunchSetup ls(dim3((unsigned)((total + threads - 1) / threads)), dim3(threads), 0, stream);
+    return cudaLaunchKernelEx(&ls.cfg, maxpool3d_bf16x8_kernel, static_cast<const uint4*>(x), t, h, w, c / 8, xcs / 8, kt, kh, kw,
+                              st, sh, sw, pt, ph, pw, static_cast<uint4*>(y), To, Ho, Wo, ycs / 8, total);
   } else {
     const long long total = vox * c;
     const unsigned blocks = (unsigned)((total + threads - 1) / threads);
+    LaunchSetup ls(dim3(blocks), dim3(threads), 0, stream);
     if (dtype == 0)
-      maxpool3d_kernel<float><<<blocks, threads, 0, stream>>>(static_cast<const float*>(x), t, h, w, c, xcs, kt, kh, kw,
-                                                             st, sh, sw, pt, ph, pw, static_cast<float*>(y), To, Ho, Wo,
-                                                             ycs, total);
-    else
-      maxpool3d_kernel<__nv_bfloat16><<<blocks, threads, 0, stream>>>(
-          static_cast<const __nv_bfloat16*>(x), t, h, w, c, xcs, kt, kh, kw, st, sh, sw, pt, ph, pw,
-          static_cast<__nv_bfloat16*>(y), To, Ho, Wo, ycs, total);
+      return cudaLaunchKernelEx(&ls.cfg, maxpool3d_kernel<float>, static_cast<const float*>(x), t, h, w, c, xcs, kt, kh, kw,
+                                st, sh, sw, pt, ph, pw, static_cast<float*>(y), To, Ho, Wo, ycs, total);
+    return cudaLaunchKernelEx(&ls.cfg, maxpool3d_kernel<__nv_bfloat16>, static_cast<const __nv_bfloat16*>(x), t, h, w, c, xcs,
+                              kt, kh, kw, st, sh, sw, pt, ph, pw, static_cast<__nv_bfloat16*>(y), To, Ho, Wo, ycs, total);
   }
-  return cudaGetLastError();
 }
 
 cudaError_t launch_add_relu(int dtype, const void* a, int acs, const void* b, int bcs, void* y, int ycs,
@@ -255,21 +261,19 @@ cudaError_t launch_add_relu(int dtype, const void* a, int acs, const void* b, in
   const int threads = 256;
   if (dtype == 1 && c % 8 == 0 && acs % 8 == 0 && bcs % 8 == 0 && ycs % 8 == 0) {
     const long long total = voxels * (c / 8);
-    add_relu_bf16x8_kernel<<<(unsigned)((total + threads - 1) / threads), threads, 0, stream>>>(
-        static_cast<const uint4*>(a), acs / 8, static_cast<const uint4*>(b), bcs / 8, static_cast<uint4*>(y),
-        ycs / 8, c / 8, relu, total);
+    LaunchSetup ls(dim3((unsigned)((total + threads - 1) / threads)), dim3(threads), 0, stream);
+    return cudaLaunchKernelEx(&ls.cfg, add_relu_bf16x8_kernel, static_cast<const uint4*>(a), acs / 8, static_cast<const uint4*>(b),
+                              bcs / 8, static_cast<uint4*>(y), ycs / 8, c / 8, relu, total);
   } else {
     const long long total = voxels * c;
     const unsigned blocks = (unsigned)((total + threads - 1) / threads);
+    LaunchSetup ls(dim3(blocks), dim3(threads), 0, stream);
     if (dtype == 0)
-      add_relu_kernel<float><<<blocks, threads, 0, stream>>>(static_cast<const float*>(a), acs, static_cast<const float*>(b),
-                                                            bcs, static_cast<float*>(y), ycs, c, relu, total);
-    else
-      add_relu_kernel<__nv_bfloat16><<<blocks, threads, 0, stream>>>(
-          static_cast<const __nv_bfloat16*>(a), acs, static_cast<const __nv_bfloat16*>(b), bcs,
-          static_cast<__nv_bfloat16*>(y), ycs, c, relu, total);
+      return cudaLaunchKernelEx(&ls.cfg, add_relu_kernel<float>, static_cast<const float*>(a), acs, static_cast<const float*>(b),
+                                bcs, static_cast<float*>(y), ycs, c, relu, total);
+    return cudaLaunchKernelEx(&ls.cfg, add_relu_kernel<__nv_bfloat16>, static_cast<const __nv_bfloat16*>(a), acs,
+                              static_cast<const __nv_bfloat16*>(b), bcs, static_cast<__nv_bfloat16*>(y), ycs, c, relu, total);
   }
-  return cudaGetLastError();
 }
 
 }  // namespace rt3d

@@ -23,6 +23,7 @@
 // memory, all roles fall through, TMEM is released and the kernel returns.
 #include "kernels.h"
 #include "umma_common.cuh"
+#include "pdl.cuh"
 
 namespace rt3d {
 namespace {
@@ -105,6 +106,7 @@ template <bool kDense>
 __global__ void __launch_bounds__(kThreadsUmma, 1)
 conv3d_umma_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CUtensorMap wmap,
                    const __grid_constant__ CUtensorMap ymap, const UmmaArgs a, const int stages, const int tmem_cols) {
+  pdl_launch();
   extern __shared__ unsigned char smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t tiles_base = (raw + 1023u) & ~1023u;            // operand tiles need 1024-byte alignment
@@ -115,8 +117,6 @@ conv3d_umma_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_consta
                                                4 * kStoreWarpBytes);
   float* bias_s = reinterpret_cast<float*>(bars + 1);              // bias of all bundles (zeros if none), padded
   int32_t* err = a.sched + 2;
-  for (int i = threadIdx.x; i < a.n_bundles * a.n_tile; i += blockDim.x)
-    bias_s[i] = (a.bias != nullptr && i < a.g.M) ? __ldg(a.bias + i) : 0.f;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n_mtiles = a.tiles_n * a.tiles_t * a.tiles_h * a.tiles_w;
@@ -145,6 +145,12 @@ conv3d_umma_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_consta
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = bars->tmem_base;
+
+  // Everything above touched only shared memory, barriers and TMEM; global memory from here on.
+  pdl_wait();
+  for (int i = threadIdx.x; i < a.n_bundles * a.n_tile; i += blockDim.x)
+    bias_s[i] = (a.bias != nullptr && i < a.g.M) ? __ldg(a.bias + i) : 0.f;
+  __syncthreads();
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
@@ -350,7 +356,8 @@ cudaError_t launch_conv_umma(const UmmaArgs& a, const void* xmap, const void* wm
       if (e != cudaSuccess) return e;
       attr_done_d = true;
     }
-    conv3d_umma_kernel<true><<<grid, kThreadsUmma, smem, stream>>>(xm, wm, ym, a, stages, cols);
+    LaunchSetup ls(dim3(grid), dim3(kThreadsUmma), smem, stream);
+    return cudaLaunchKernelEx(&ls.cfg, conv3d_umma_kernel<true>, xm, wm, ym, a, stages, cols);
   } else {
     static bool attr_done_s = false;
     if (!attr_done_s) {
@@ -358,9 +365,9 @@ cudaError_t launch_conv_umma(const UmmaArgs& a, const void* xmap, const void* wm
       if (e != cudaSuccess) return e;
       attr_done_s = true;
     }
-    conv3d_umma_kernel<false><<<grid, kThreadsUmma, smem, stream>>>(xm, wm, ym, a, stages, cols);
+    LaunchSetup ls(dim3(grid), dim3(kThreadsUmma), smem, stream);
+    return cudaLaunchKernelEx(&ls.cfg, conv3d_umma_kernel<false>, xm, wm, ym, a, stages, cols);
   }
-  return cudaGetLastError();
 }
 
 }  // namespace rt3d

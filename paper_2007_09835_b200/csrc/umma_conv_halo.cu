@@ -35,6 +35,7 @@
 #include "kernels.h"
 #include "umma_common.cuh"
 #include "umma_pair.cuh"
+#include "pdl.cuh"
 
 namespace rt3d {
 namespace {
@@ -71,6 +72,7 @@ template <bool kDense>
 __global__ void __launch_bounds__(kThreadsHalo, 1)
 conv3d_umma_halo_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CUtensorMap wmap_half,
                         const __grid_constant__ CUtensorMap ymap, const HaloArgs h, const int tmem_cols) {
+  pdl_launch();
   const UmmaArgs& a = h.u;
   extern __shared__ unsigned char smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
@@ -87,7 +89,6 @@ conv3d_umma_halo_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_c
   float* bias_s = reinterpret_cast<float*>(hb + 1);
   int32_t* err = a.sched + 2;
 
-  for (int i = threadIdx.x; i < a.n_tile; i += blockDim.x) bias_s[i] = (a.bias != nullptr && i < a.g.M) ? __ldg(a.bias + i) : 0.f;
   // warp index and CTA rank in forms the compiler can prove uniform (the MMA warp must stay convergent)
   const int warp = __shfl_sync(0xffffffffu, threadIdx.x >> 5, 0), lane = threadIdx.x & 31;
   const uint32_t rank = blockIdx.x & 1u;          // clusters are pairs of consecutive CTAs of a 1-D grid
@@ -121,6 +122,11 @@ conv3d_umma_halo_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_c
   cluster_sync_all();
   tc_fence_after();
   const uint32_t tmem_base = bars->tmem_base;
+
+  // Everything above touched only shared memory, barriers and TMEM; global memory from here on.
+  pdl_wait();
+  for (int i = threadIdx.x; i < a.n_tile; i += blockDim.x) bias_s[i] = (a.bias != nullptr && i < a.g.M) ? __ldg(a.bias + i) : 0.f;
+  __syncthreads();
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer (both CTAs)
@@ -269,17 +275,8 @@ cudaError_t launch_halo_t(const HaloArgs& h, const CUtensorMap& xm, const CUtens
   }
   long long clusters = sm_count / 2;
   if (clusters > n_items) clusters = n_items;
-  cudaLaunchConfig_t cfg = {};
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
-  cfg.gridDim = dim3(unsigned(2 * clusters));
-  cfg.blockDim = dim3(kThreadsHalo);
-  cfg.dynamicSmemBytes = smem;
-  cfg.stream = stream;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, conv3d_umma_halo_kernel<kDense>, xm, wm, ym, h, cols);
+  LaunchSetup ls(dim3(unsigned(2 * clusters)), dim3(kThreadsHalo), smem, stream, 2);
+  return cudaLaunchKernelEx(&ls.cfg, conv3d_umma_halo_kernel<kDense>, xm, wm, ym, h, cols);
 }
 
 }  // namespace

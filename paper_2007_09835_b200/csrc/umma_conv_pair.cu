@@ -16,6 +16,7 @@
 #include "kernels.h"
 #include "umma_common.cuh"
 #include "umma_pair.cuh"
+#include "pdl.cuh"
 
 namespace rt3d {
 namespace {
@@ -46,6 +47,7 @@ template <bool kDense, int kCps>
 __global__ void __launch_bounds__(kThreadsUmma, 1)
 conv3d_umma_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CUtensorMap wmap_half,
                         const __grid_constant__ CUtensorMap ymap, const UmmaArgs a, const int stages, const int tmem_cols) {
+  pdl_launch();
   extern __shared__ unsigned char smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t tiles_base = (raw + 1023u) & ~1023u;
@@ -59,8 +61,6 @@ conv3d_umma_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_c
   TailWork* tw = reinterpret_cast<TailWork*>(bars + 1);
   float* bias_s = reinterpret_cast<float*>(tw + 1);
   int32_t* err = a.sched + 2;
-  for (int i = threadIdx.x; i < a.n_bundles * a.n_tile; i += blockDim.x)
-    bias_s[i] = (a.bias != nullptr && i < a.g.M) ? __ldg(a.bias + i) : 0.f;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_ctarank();
@@ -83,6 +83,23 @@ conv3d_umma_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_c
     bars->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
+                 ::"r"(smem_u32(&bars->tmem_base)), "r"(uint32_t(tmem_cols)) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();              // barriers of both CTAs are initialised before anyone signals them
+  tc_fence_after();
+  const uint32_t tmem_base = bars->tmem_base;
+
+  // Everything above touched only shared memory, barriers and TMEM; global memory from here on.
+  pdl_wait();
+  for (int i = threadIdx.x; i < a.n_bundles * a.n_tile; i += blockDim.x)
+    bias_s[i] = (a.bias != nullptr && i < a.g.M) ? __ldg(a.bias + i) : 0.f;
+  if (threadIdx.x == 0) {
     // this pair's work list
     tw->n_seg = 0;
     if (a.tail_workers == 0) {
@@ -121,16 +138,7 @@ conv3d_umma_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_c
       }
     }
   }
-  if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
-                 ::"r"(smem_u32(&bars->tmem_base)), "r"(uint32_t(tmem_cols)) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
-  }
-  tc_fence_before();
   __syncthreads();
-  cluster_sync_all();              // barriers of both CTAs are initialised before anyone signals them
-  tc_fence_after();
-  const uint32_t tmem_base = bars->tmem_base;
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer (both CTAs)
@@ -420,10 +428,8 @@ cudaError_t launch_pair_t(const UmmaArgs& a, const CUtensorMap& xm, const CUtens
   if (e != cudaSuccess) return e;
   long long clusters = pair_max_clusters_t<kDense, kCps>(sm_count, smem);
   if (clusters > n_items) clusters = n_items;
-  cudaLaunchConfig_t cfg;
-  cudaLaunchAttribute attr[1];
-  pair_launch_config(cfg, attr, unsigned(2 * clusters), smem, stream);
-  return cudaLaunchKernelEx(&cfg, conv3d_umma_pair_kernel<kDense, kCps>, xm, wm, ym, a, stages, cols);
+  LaunchSetup ls(dim3(unsigned(2 * clusters)), dim3(kThreadsUmma), smem, stream, 2);
+  return cudaLaunchKernelEx(&ls.cfg, conv3d_umma_pair_kernel<kDense, kCps>, xm, wm, ym, a, stages, cols);
 }
 
 }  // namespace

@@ -18,6 +18,7 @@
 // epilogue; bounded mbarrier waits.
 #include "kernels.h"
 #include "umma_common.cuh"
+#include "pdl.cuh"
 
 namespace rt3d {
 namespace {
@@ -28,6 +29,7 @@ template <int kDummy>
 __global__ void __launch_bounds__(kThreadsUmma, 3)
 conv3d_umma_smallc_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CUtensorMap ymap,
                           const SmallCArgs a) {
+  pdl_launch();
   extern __shared__ unsigned char smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t store_smem = (raw + 1023u) & ~1023u;                   // 4 warps x 2 staging buffers (TMA stores)
@@ -43,18 +45,9 @@ conv3d_umma_smallc_kernel(const __grid_constant__ CUtensorMap xmap, const __grid
   float* bias_s = reinterpret_cast<float*>(bars + 1);
   int32_t* err = a.sched + 2;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  for (int i = threadIdx.x; i < a.n_pad; i += blockDim.x)
-    bias_s[i] = (a.bias != nullptr && i < a.g.M) ? __ldg(a.bias + i) : 0.f;
   const int tiles_per_frame = a.tiles_h * a.tiles_w;
   const int n_items = a.g.n * a.g.To * tiles_per_frame;
 
-  // weight image and pair offsets: plain cooperative copy, once per CTA
-  {
-    const uint4* src = reinterpret_cast<const uint4*>(a.wimg);
-    uint4* dst = reinterpret_cast<uint4*>(gen);
-    for (uint32_t i = threadIdx.x; i < w_bytes / 16; i += blockDim.x) dst[i] = __ldg(src + i);
-    for (int i = threadIdx.x; i < a.n_pairs * 2; i += blockDim.x) pair_smem[i] = __ldg(a.pair_off + i);
-  }
   if (threadIdx.x == 0) {
     for (int s = 0; s < kSmallCStages; ++s) {
       mbar_init(smem_u32(&bars->full[s]), 1);
@@ -67,8 +60,6 @@ conv3d_umma_smallc_kernel(const __grid_constant__ CUtensorMap xmap, const __grid
     bars->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  // generic-proxy writes of the weight image must be visible to the tensor core (async proxy)
-  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
                  ::"r"(smem_u32(&bars->tmem_base)), "r"(uint32_t(a.tmem_cols)) : "memory");
@@ -78,6 +69,21 @@ conv3d_umma_smallc_kernel(const __grid_constant__ CUtensorMap xmap, const __grid
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = bars->tmem_base;
+
+  // Everything above touched only shared memory, barriers and TMEM; global memory from here on.
+  pdl_wait();
+  for (int i = threadIdx.x; i < a.n_pad; i += blockDim.x)
+    bias_s[i] = (a.bias != nullptr && i < a.g.M) ? __ldg(a.bias + i) : 0.f;
+  // weight image and pair offsets: plain cooperative copy, once per CTA
+  {
+    const uint4* src = reinterpret_cast<const uint4*>(a.wimg);
+    uint4* dst = reinterpret_cast<uint4*>(gen);
+    for (uint32_t i = threadIdx.x; i < w_bytes / 16; i += blockDim.x) dst[i] = __ldg(src + i);
+    for (int i = threadIdx.x; i < a.n_pairs * 2; i += blockDim.x) pair_smem[i] = __ldg(a.pair_off + i);
+  }
+  // generic-proxy writes of the weight image must be visible to the tensor core (async proxy)
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  __syncthreads();
 
   if (warp == 0) {
     if (lane == 0 && a.n_pairs > 0) {
@@ -232,8 +238,8 @@ cudaError_t launch_conv_umma_smallc(const SmallCArgs& a_in, const void* xmap, co
   if (per_sm < 1) per_sm = 1;
   const long long want = (long long)sm_count * per_sm;
   const int grid = int(n_items < want ? n_items : want);
-  conv3d_umma_smallc_kernel<0><<<grid, kThreadsUmma, smem, stream>>>(xm, ym, a);
-  return cudaGetLastError();
+  LaunchSetup ls(dim3(grid), dim3(kThreadsUmma), smem, stream);
+  return cudaLaunchKernelEx(&ls.cfg, conv3d_umma_smallc_kernel<0>, xm, ym, a);
 }
 
 }  // namespace rt3d
