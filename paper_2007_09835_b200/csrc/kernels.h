@@ -67,7 +67,7 @@ cudaError_t launch_conv_umma(const UmmaArgs& a, const void* xmap, const void* wm
                              cudaStream_t stream);
 
 // CTA-pair variant (cta_group::2): wmap_half is a tensor map over the same weight tiles whose box is
-// half a tile high (n_tile/2 rows).  Needs n_tile % 32 == 0 and a.n_splits == 1.
+// half a tile high (n_tile/2 rows).  Needs n_tile % 16 == 0 and a.n_splits == 1.
 bool umma_pair_supported(int n_tile, int n_bundles);
 // Fills a->tail_workers (0 = whole items only) and the scratch the tail split needs; the caller provides
 // a->tail_scratch / a->tail_flags of at least those sizes (flags zero-initialised).

@@ -435,7 +435,7 @@ cudaError_t launch_pair_t(const UmmaArgs& a, const CUtensorMap& xm, const CUtens
 }  // namespace
 
 bool umma_pair_supported(int n_tile, int n_bundles) {
-  return n_tile % 32 == 0 && n_tile <= 256 && pick_stages_pair(n_tile) >= 2 && pair_smem_bytes(n_tile, n_bundles) <= 227 * 1024;
+  return n_tile % 16 == 0 && n_tile <= 256 && pick_stages_pair(n_tile) >= 2 && pair_smem_bytes(n_tile, n_bundles) <= 227 * 1024;
 }
 
 // Tail split: decides how many CTA pairs share the items that do not fill a last round (0 = no split)
