@@ -145,6 +145,51 @@ __global__ void maxpool3d_kernel(const T* __restrict__ x, int t, int h, int w, i
   y[((((long long)nn * To + to) * Ho + ho) * Wo + wo) * ycs + cc] = from_f32<T>(best);
 }
 
+// Same for a window known at compile time: all loads of the window are issued together (clamped address,
+// result masked to -inf outside the tensor) instead of one after the other behind run-time branches.
+template <int KT, int KH, int KW>
+__global__ void maxpool3d_bf16x8_win_kernel(const uint4* __restrict__ x, int t, int h, int w, int c8, int xcs8,
+                                            int st, int sh, int sw, int pt, int ph, int pw,
+                                            uint4* __restrict__ y, int To, int Ho, int Wo, int ycs8, long long total) {
+  pdl_entry();
+  const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= total) return;
+  const int cc = int(idx % c8);
+  long long r = idx / c8;
+  const int wo = int(r % Wo); r /= Wo;
+  const int ho = int(r % Ho); r /= Ho;
+  const int to = int(r % To);
+  const int nn = int(r / To);
+  const int t0 = to * st - pt, h0 = ho * sh - ph, w0 = wo * sw - pw;
+  uint4 v[KT * KH * KW];
+  bool ok[KT * KH * KW];
+#pragma unroll
+  for (int a = 0; a < KT; ++a)
+#pragma unroll
+    for (int b = 0; b < KH; ++b)
+#pragma unroll
+      for (int d = 0; d < KW; ++d) {
+        const int ti = t0 + a, hi = h0 + b, wi = w0 + d;
+        const bool in = ti >= 0 && ti < t && hi >= 0 && hi < h && wi >= 0 && wi < w;
+        const int tc = min(max(ti, 0), t - 1), hc = min(max(hi, 0), h - 1), wc = min(max(wi, 0), w - 1);
+        ok[(a * KH + b) * KW + d] = in;
+        v[(a * KH + b) * KW + d] = __ldg(x + ((((long long)nn * t + tc) * h + hc) * w + wc) * xcs8 + cc);
+      }
+  const __nv_bfloat162 ninf = __float2bfloat162_rn(-INFINITY);
+  __nv_bfloat162 best[4] = {ninf, ninf, ninf, ninf};
+#pragma unroll
+  for (int i = 0; i < KT * KH * KW; ++i) {
+    const __nv_bfloat162* pv = reinterpret_cast<const __nv_bfloat162*>(&v[i]);
+#pragma unroll
+    for (int k = 0; k < 4; ++k) best[k] = ok[i] ? __hmax2(best[k], pv[k]) : best[k];
+  }
+  uint4 out;
+  __nv_bfloat162* po = reinterpret_cast<__nv_bfloat162*>(&out);
+#pragma unroll
+  for (int k = 0; k < 4; ++k) po[k] = best[k];
+  y[((((long long)nn * To + to) * Ho + ho) * Wo + wo) * ycs8 + cc] = out;
+}
+
 // bf16, 8 channels (16 bytes) per thread; needs c % 8 == 0 and 8-element pitches.
 __global__ void maxpool3d_bf16x8_kernel(const uint4* __restrict__ x, int t, int h, int w, int c8, int xcs8,
                                         int kt, int kh, int kw, int st, int sh, int sw, int pt, int ph, int pw,
@@ -241,6 +286,15 @@ cudaError_t launch_maxpool3d(int dtype, const void* x, int n, int t, int h, int 
   if (dtype == 1 && c % 8 == 0 && xcs % 8 == 0 && ycs % 8 == 0) {
     const long long total = vox * (c / 8);
     LaunchSetup ls(dim3((unsigned)((total + threads - 1) / threads)), dim3(threads), 0, stream);
+#define RT3D_POOL_WIN(KT_, KH_, KW_)                                                                                   \
+  if (kt == KT_ && kh == KH_ && kw == KW_)                                                                              \
+    return cudaLaunchKernelEx(&ls.cfg, maxpool3d_bf16x8_win_kernel<KT_, KH_, KW_>, static_cast<const uint4*>(x), t, h, w, \
+                              c / 8, xcs / 8, st, sh, sw, pt, ph, pw, static_cast<uint4*>(y), To, Ho, Wo, ycs / 8, total)
+    RT3D_POOL_WIN(3, 3, 3);
+    RT3D_POOL_WIN(1, 3, 3);
+    RT3D_POOL_WIN(2, 2, 2);
+    RT3D_POOL_WIN(1, 2, 2);
+#undef RT3D_POOL_WIN
     return cudaLaunchKernelEx(&ls.cfg, maxpool3d_bf16x8_kernel, static_cast<const uint4*>(x), t, h, w, c / 8, xcs / 8, kt, kh, kw,
                               st, sh, sw, pt, ph, pw, static_cast<uint4*>(y), To, Ho, Wo, ycs / 8, total);
   } else {
