@@ -375,10 +375,16 @@ def main():
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         import oracle
         clips = CFG["n"]
-        dt = oracle_timed(spec, L, x, clips)
+        oracle_timed(spec, L, x, 1)                       # first call: builds / loads the oracle, warms the caches
+        passes, total = 0, 0.0
+        while total < 10.0 and passes < 32:               # about 10-15 s of CPU work
+            total += oracle_timed(spec, L, x, clips)
+            passes += 1
+        dt = total / passes
         out["cpu_baseline"] = {"value": flops_kept / dt / 1e12, "unit": "TFLOP/s", "cores": oracle.threads(),
-                               "kind": "oracle", "seconds": dt,
-                               "sample": f"all {clips} clips of one batch, one pass (masked dense weights, fp64 accumulation)"}
+                               "kind": "oracle", "seconds": total,
+                               "sample": f"all {clips} clips of one batch, mean of {passes} passes "
+                                         f"(masked dense weights, fp64 accumulation)"}
     if rank == 0:
         print(json.dumps(out))
     dist.shutdown(group)
