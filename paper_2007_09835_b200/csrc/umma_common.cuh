@@ -24,6 +24,11 @@ struct __align__(8) Barriers {
   volatile int abort_flag;
 };
 
+// Bias staging area of a kernel, rounded up to 16 bytes so that the epilogue reads it as float4.
+__device__ __forceinline__ float* align16_f32(void* p) {
+  return reinterpret_cast<float*>((reinterpret_cast<uintptr_t>(p) + 15) & ~uintptr_t(15));
+}
+
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return static_cast<uint32_t>(__cvta_generic_to_shared(p));
 }
@@ -155,8 +160,13 @@ template <int NC>
 __device__ __forceinline__ void epilogue_cols(const uint32_t* v, const float* bias_s, int relu,
                                               __nv_bfloat16* dst, int valid, const __nv_bfloat16* res, int res_avail) {
   float f[NC];
+  const float4* b4 = reinterpret_cast<const float4*>(bias_s);      // 16-byte aligned by construction
 #pragma unroll
-  for (int q = 0; q < NC; ++q) f[q] = __uint_as_float(v[q]) + bias_s[q];
+  for (int k = 0; k < NC / 4; ++k) {
+    const float4 b = b4[k];
+    f[4 * k] = __uint_as_float(v[4 * k]) + b.x; f[4 * k + 1] = __uint_as_float(v[4 * k + 1]) + b.y;
+    f[4 * k + 2] = __uint_as_float(v[4 * k + 2]) + b.z; f[4 * k + 3] = __uint_as_float(v[4 * k + 3]) + b.w;
+  }
   if (res != nullptr) {
 #pragma unroll
     for (int k = 0; k < NC / 8; ++k) {
@@ -263,8 +273,13 @@ __device__ __forceinline__ void epilogue_piece_tma(const uint32_t* v, const floa
                                                    TmaStore& ts, const __nv_bfloat16* res, int res_avail,
                                                    const PoolLanes* pool) {
   float f[32];
+  const float4* b4 = reinterpret_cast<const float4*>(bias_s);      // 16-byte aligned by construction
 #pragma unroll
-  for (int q = 0; q < 32; ++q) f[q] = __uint_as_float(v[q]) + bias_s[q];
+  for (int k = 0; k < 8; ++k) {
+    const float4 b = b4[k];
+    f[4 * k] = __uint_as_float(v[4 * k]) + b.x; f[4 * k + 1] = __uint_as_float(v[4 * k + 1]) + b.y;
+    f[4 * k + 2] = __uint_as_float(v[4 * k + 2]) + b.z; f[4 * k + 3] = __uint_as_float(v[4 * k + 3]) + b.w;
+  }
   if (res != nullptr) {
 #pragma unroll
     for (int k = 0; k < 4; ++k) {

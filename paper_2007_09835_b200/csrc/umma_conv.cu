@@ -115,7 +115,7 @@ conv3d_umma_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_consta
   const uint32_t store_smem = tiles_base + uint32_t(stages) * stage_bytes;     // 4 warps x 2 staging buffers
   Barriers* bars = reinterpret_cast<Barriers*>(smem_raw + (tiles_base - raw) + size_t(stages) * stage_bytes +
                                                4 * kStoreWarpBytes);
-  float* bias_s = reinterpret_cast<float*>(bars + 1);              // bias of all bundles (zeros if none), padded
+  float* bias_s = align16_f32(bars + 1);                            // bias of all bundles (zeros if none), padded
   int32_t* err = a.sched + 2;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -326,7 +326,7 @@ int pick_stages(int n_tile) {
 }  // namespace
 
 size_t umma_smem_bytes(int n_tile, int n_bundles) {
-  return size_t(pick_stages(n_tile)) * (kABytes + size_t(n_tile) * 128) + 1024 + 4 * kStoreWarpBytes + sizeof(Barriers) +
+  return size_t(pick_stages(n_tile)) * (kABytes + size_t(n_tile) * 128) + 1024 + 4 * kStoreWarpBytes + sizeof(Barriers) + 16 +
          size_t(n_tile) * n_bundles * 4;
 }
 

@@ -86,7 +86,7 @@ conv3d_umma_halo_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_c
   unsigned char* tail = smem_raw + (store_smem - raw) + 8 * kStoreWarpBytes;
   HaloBars* hb = reinterpret_cast<HaloBars*>(tail);
   Barriers* bars = &hb->b;
-  float* bias_s = reinterpret_cast<float*>(hb + 1);
+  float* bias_s = align16_f32(hb + 1);
   int32_t* err = a.sched + 2;
 
   // warp index and CTA rank in forms the compiler can prove uniform (the MMA warp must stay convergent)

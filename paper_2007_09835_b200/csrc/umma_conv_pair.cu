@@ -59,7 +59,7 @@ conv3d_umma_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_c
   Barriers* bars = reinterpret_cast<Barriers*>(smem_raw + (tiles_base - raw) + size_t(stages) * stage_bytes +
                                                4 * kStoreWarpBytes);
   TailWork* tw = reinterpret_cast<TailWork*>(bars + 1);
-  float* bias_s = reinterpret_cast<float*>(tw + 1);
+  float* bias_s = align16_f32(tw + 1);
   int32_t* err = a.sched + 2;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -370,7 +370,7 @@ int pick_stages_pair(int n_tile) {
 
 size_t pair_smem_bytes(int n_tile, int n_bundles) {
   return size_t(pick_stages_pair(n_tile)) * pick_cps(n_tile) * (kABytes + size_t(n_tile / 2) * 128) + 1024 + 4 * kStoreWarpBytes +
-         sizeof(Barriers) + sizeof(TailWork) +
+         sizeof(Barriers) + sizeof(TailWork) + 16 +
          size_t(n_tile) * n_bundles * 4;
 }
 

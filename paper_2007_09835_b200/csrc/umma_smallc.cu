@@ -42,7 +42,7 @@ conv3d_umma_smallc_kernel(const __grid_constant__ CUtensorMap xmap, const __grid
   int32_t* pair_smem = reinterpret_cast<int32_t*>(gen + (halo_smem - base) + kSmallCStages * halo_stride);
   Barriers* bars = reinterpret_cast<Barriers*>(reinterpret_cast<unsigned char*>(pair_smem) +
                                                ((size_t(a.n_pairs) * 8 + 15) & ~size_t(15)));
-  float* bias_s = reinterpret_cast<float*>(bars + 1);
+  float* bias_s = align16_f32(bars + 1);
   int32_t* err = a.sched + 2;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int tiles_per_frame = a.tiles_h * a.tiles_w;
@@ -192,7 +192,7 @@ conv3d_umma_smallc_kernel(const __grid_constant__ CUtensorMap xmap, const __grid
 size_t smallc_smem_bytes(int n_pairs, int n_pad, int stage_bytes) {
   const size_t w = (size_t(n_pairs) * 2 * n_pad * 16 + 127) & ~size_t(127);
   const size_t halo = (size_t(stage_bytes) + 127) & ~size_t(127);
-  return 1024 + 4 * kStoreWarpBytes + w + kSmallCStages * halo + ((size_t(n_pairs) * 8 + 15) & ~size_t(15)) + sizeof(Barriers) + size_t(n_pad) * 4;
+  return 1024 + 4 * kStoreWarpBytes + w + kSmallCStages * halo + ((size_t(n_pairs) * 8 + 15) & ~size_t(15)) + sizeof(Barriers) + 16 + size_t(n_pad) * 4;
 }
 
 cudaError_t launch_conv_umma_smallc(const SmallCArgs& a_in, const void* xmap, const void* ymap, int sm_count,
