@@ -13,7 +13,13 @@
  *   - Compute calls enqueue work on the given CUDA stream (a cudaStream_t passed as
  *     void*, NULL = default stream) and return without synchronising.  The first compute
  *     call that uses a handle on a device uploads the handle's device blobs (allocation +
- *     copy); later calls allocate nothing.  rt3d_packed_prepare does that upload ahead of time.
+ *     copy), and the first call of a shape that splits K grows the handle's scratch buffer;
+ *     later calls allocate nothing.  rt3d_packed_prepare does the upload ahead of time.
+ *     That scratch belongs to the handle: two calls on the SAME handle whose kernels may overlap
+ *     on the GPU (different streams) must be serialised by the caller.
+ *   - Kernels are launched with programmatic stream serialisation: a kernel's set-up may overlap
+ *     the tail of the previous kernel on its stream, but it reads and writes global memory only
+ *     after that kernel has completed (environment RT3D_PDL=0 turns the attribute off).
  *   - Argument errors are detected on the host before anything is launched.
  *   - Activation layout: NDHWC = [n][t][h][w][c] with a channel pitch c_stride >= c
  *     (elements between consecutive voxels).  Weight layout handed to the packers:
