@@ -17,7 +17,9 @@
 
 namespace rt3d {
 
-// At kernel entry: the successor may be scheduled.
+// The successor may be scheduled.  The tensor-core kernels call this only after their TMEM allocation: a
+// successor's CTA that became resident on the same SM and allocated TMEM first could otherwise block a CTA of
+// the kernel it is waiting for.
 __device__ __forceinline__ void pdl_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 // Before the first access to global memory: the predecessor has completed and its writes are visible.
 // Set-up that touches only shared memory, barriers and TMEM may run before it.

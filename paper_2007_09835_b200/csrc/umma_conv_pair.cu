@@ -47,7 +47,6 @@ template <bool kDense, int kCps>
 __global__ void __launch_bounds__(kThreadsUmma, 1)
 conv3d_umma_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CUtensorMap wmap_half,
                         const __grid_constant__ CUtensorMap ymap, const UmmaArgs a, const int stages, const int tmem_cols) {
-  pdl_launch();
   extern __shared__ unsigned char smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t tiles_base = (raw + 1023u) & ~1023u;
@@ -95,7 +94,10 @@ conv3d_umma_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_c
   tc_fence_after();
   const uint32_t tmem_base = bars->tmem_base;
 
-  // Everything above touched only shared memory, barriers and TMEM; global memory from here on.
+  // Everything above touched only shared memory, barriers and TMEM.  The successor may be scheduled now that
+  // this CTA holds its TMEM columns (a successor CTA that shared the SM and allocated first could otherwise
+  // starve this one while waiting for it); global memory from here on.
+  pdl_launch();
   pdl_wait();
   for (int i = threadIdx.x; i < a.n_bundles * a.n_tile; i += blockDim.x)
     bias_s[i] = (a.bias != nullptr && i < a.g.M) ? __ldg(a.bias + i) : 0.f;

@@ -29,7 +29,6 @@ template <int kDummy>
 __global__ void __launch_bounds__(kThreadsUmma, 3)
 conv3d_umma_smallc_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CUtensorMap ymap,
                           const SmallCArgs a) {
-  pdl_launch();
   extern __shared__ unsigned char smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t store_smem = (raw + 1023u) & ~1023u;                   // 4 warps x 2 staging buffers (TMA stores)
@@ -70,7 +69,10 @@ conv3d_umma_smallc_kernel(const __grid_constant__ CUtensorMap xmap, const __grid
   tc_fence_after();
   const uint32_t tmem_base = bars->tmem_base;
 
-  // Everything above touched only shared memory, barriers and TMEM; global memory from here on.
+  // Everything above touched only shared memory, barriers and TMEM.  The successor may be scheduled now that
+  // this CTA holds its TMEM columns (a successor CTA that shared the SM and allocated first could otherwise
+  // starve this one while waiting for it); global memory from here on.
+  pdl_launch();
   pdl_wait();
   for (int i = threadIdx.x; i < a.n_pad; i += blockDim.x)
     bias_s[i] = (a.bias != nullptr && i < a.g.M) ? __ldg(a.bias + i) : 0.f;
