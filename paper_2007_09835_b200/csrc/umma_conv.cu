@@ -102,7 +102,9 @@ __device__ __forceinline__ void reduce_partial_row(const float* part0, size_t sp
   }
 }
 
-template <bool kDense>
+// kCps: K steps per pipeline stage (and per barrier hand-shake): 1, or 2 for narrow bundles, where the
+// issuing thread's hand-shake, not the tensor pipe, bounds a step.
+template <bool kDense, int kCps>
 __global__ void __launch_bounds__(kThreadsUmma, 1)
 conv3d_umma_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CUtensorMap wmap,
                    const __grid_constant__ CUtensorMap ymap, const UmmaArgs a, const int stages, const int tmem_cols) {
@@ -110,7 +112,8 @@ conv3d_umma_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_consta
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t tiles_base = (raw + 1023u) & ~1023u;            // operand tiles need 1024-byte alignment
   const uint32_t b_bytes = uint32_t(a.n_tile) * 128u;
-  const uint32_t stage_bytes = kABytes + b_bytes;
+  const uint32_t chunk_bytes = kABytes + b_bytes;
+  const uint32_t stage_bytes = kCps * chunk_bytes;
   const uint32_t store_smem = tiles_base + uint32_t(stages) * stage_bytes;     // 4 warps x 2 staging buffers
   Barriers* bars = reinterpret_cast<Barriers*>(smem_raw + (tiles_base - raw) + size_t(stages) * stage_bytes +
                                                4 * kStoreWarpBytes);
@@ -174,25 +177,34 @@ conv3d_umma_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_consta
           const int pos = local0 / a.n_chunks;
           kw = pos % a.g.Kw; kh = (pos / a.g.Kw) % a.g.Kh; kt = pos / (a.g.Kw * a.g.Kh);
         }
-        int enc_next = (!kDense && nsteps > 0) ? __ldg(a.steps + s_begin) : 0;
         int wrow = s_begin * a.n_tile;
-        for (int i = 0; i < nsteps; ++i, wrow += a.n_tile) {
-          int c_ch, c_w, c_h, c_t;
-          if (kDense) {
-            c_ch = ch * 64; c_w = wq + kw; c_h = hq + kh; c_t = tq + kt;
-            if (++ch == a.n_chunks) { ch = 0; if (++kw == a.g.Kw) { kw = 0; if (++kh == a.g.Kh) { kh = 0; ++kt; } } }
-          } else {
-            const int enc = enc_next;
-            if (i + 1 < nsteps) enc_next = __ldg(a.steps + s_begin + i + 1);
-            c_t = tq + ((enc >> 24) & 63); c_h = hq + ((enc >> 18) & 63); c_w = wq + ((enc >> 12) & 63);
-            c_ch = (enc & 4095) * 64;
+        for (int i = 0; i < nsteps; i += kCps) {
+          const int nload = nsteps - i < kCps ? nsteps - i : kCps;
+          int c_ch[kCps], c_w[kCps], c_h[kCps], c_t[kCps];
+#pragma unroll
+          for (int q = 0; q < kCps; ++q) {
+            if (q >= nload) break;
+            if (kDense) {
+              c_ch[q] = ch * 64; c_w[q] = wq + kw; c_h[q] = hq + kh; c_t[q] = tq + kt;
+              if (++ch == a.n_chunks) { ch = 0; if (++kw == a.g.Kw) { kw = 0; if (++kh == a.g.Kh) { kh = 0; ++kt; } } }
+            } else {
+              const int enc = __ldg(a.steps + s_begin + i + q);
+              c_t[q] = tq + ((enc >> 24) & 63); c_h[q] = hq + ((enc >> 18) & 63); c_w[q] = wq + ((enc >> 12) & 63);
+              c_ch[q] = (enc & 4095) * 64;
+            }
           }
           const uint32_t full = smem_u32(&bars->full[stage]);
-          const uint32_t a_dst = tiles_base + stage * stage_bytes;
+          const uint32_t s_dst = tiles_base + stage * stage_bytes;
           if (!mbar_wait(smem_u32(&bars->empty[stage]), phase ^ 1u, bars, err, 1)) { ok = false; break; }
-          mbar_expect_tx(full, tx_bytes);
-          tma_load_5d(a_dst, &xmap, full, c_ch, c_w, c_h, c_t, c.n0);
-          tma_load_2d(a_dst + kABytes, &wmap, full, 0, wrow);
+          mbar_expect_tx(full, tx_bytes * uint32_t(nload));
+#pragma unroll
+          for (int q = 0; q < kCps; ++q) {
+            if (q >= nload) break;
+            const uint32_t a_dst = s_dst + q * chunk_bytes;
+            tma_load_5d(a_dst, &xmap, full, c_ch[q], c_w[q], c_h[q], c_t[q], c.n0);
+            tma_load_2d(a_dst + kABytes, &wmap, full, 0, wrow);
+            wrow += a.n_tile;
+          }
           if (++stage == stages) { stage = 0; phase ^= 1u; }
         }
       }
@@ -212,19 +224,24 @@ conv3d_umma_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_consta
         if (!mbar_wait(smem_u32(&bars->tmem_empty[buf]), ((j >> 1) & 1u) ^ 1u, bars, err, 2)) break;
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + buf * uint32_t(a.n_tile);
-        for (int i = 0; i < nsteps; ++i) {
+        for (int i = 0; i < nsteps; i += kCps) {
+          const int nload = nsteps - i < kCps ? nsteps - i : kCps;
           if (!ready && !mbar_wait(smem_u32(&bars->full[stage]), phase, bars, err, 3)) { ok = false; break; }
           // poll the next stage's barrier now: its answer arrives while this stage's MMAs are issued
           const int stage_n = stage + 1 == stages ? 0 : stage + 1;
           const uint32_t phase_n = stage + 1 == stages ? phase ^ 1u : phase;
           ready = mbar_try_wait(smem_u32(&bars->full[stage_n]), phase_n);
           tc_fence_after();
-          const uint32_t a_addr = tiles_base + stage * stage_bytes;
-          const uint64_t adesc = smem_desc_sw128(a_addr);
-          const uint64_t bdesc = smem_desc_sw128(a_addr + kABytes);
 #pragma unroll
-          for (int kk = 0; kk < 4; ++kk)      // 4 x K=16 per 64-channel chunk: +32 bytes = +2 in descriptor units
-            umma_bf16(d_tmem, adesc + 2 * kk, bdesc + 2 * kk, idesc, (i | kk) ? 1u : 0u);
+          for (int q = 0; q < kCps; ++q) {
+            if (q >= nload) break;
+            const uint32_t a_addr = tiles_base + stage * stage_bytes + q * chunk_bytes;
+            const uint64_t adesc = smem_desc_sw128(a_addr);
+            const uint64_t bdesc = smem_desc_sw128(a_addr + kABytes);
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk)    // 4 x K=16 per 64-channel chunk: +32 bytes = +2 in descriptor units
+              umma_bf16(d_tmem, adesc + 2 * kk, bdesc + 2 * kk, idesc, (i | q | kk) ? 1u : 0u);
+          }
           umma_commit(smem_u32(&bars->empty[stage]));
           stage = stage_n; phase = phase_n;
         }
@@ -319,16 +336,31 @@ conv3d_umma_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_consta
   }
 }
 
+int pick_cps_single(int n_tile) { return n_tile <= 128 ? 2 : 1; }
+
 int pick_stages(int n_tile) {
-  const size_t stage = kABytes + size_t(n_tile) * 128;
+  const size_t stage = pick_cps_single(n_tile) * (kABytes + size_t(n_tile) * 128);
   const int s = int(kSmemBudget / stage);
   return s > kMaxStages ? kMaxStages : s;
+}
+
+template <bool kDense, int kCps>
+cudaError_t launch_single_t(const UmmaArgs& a, const CUtensorMap& xm, const CUtensorMap& wm, const CUtensorMap& ym, int grid,
+                            size_t smem, int stages, int cols, cudaStream_t stream) {
+  static bool attr_done = false;
+  if (!attr_done) {
+    cudaError_t e = cudaFuncSetAttribute(conv3d_umma_kernel<kDense, kCps>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    if (e != cudaSuccess) return e;
+    attr_done = true;
+  }
+  LaunchSetup ls(dim3(grid), dim3(kThreadsUmma), smem, stream);
+  return cudaLaunchKernelEx(&ls.cfg, conv3d_umma_kernel<kDense, kCps>, xm, wm, ym, a, stages, cols);
 }
 
 }  // namespace
 
 size_t umma_smem_bytes(int n_tile, int n_bundles) {
-  return size_t(pick_stages(n_tile)) * (kABytes + size_t(n_tile) * 128) + 1024 + 4 * kStoreWarpBytes + sizeof(Barriers) + 16 +
+  return size_t(pick_stages(n_tile)) * pick_cps_single(n_tile) * (kABytes + size_t(n_tile) * 128) + 1024 + 4 * kStoreWarpBytes + sizeof(Barriers) + 16 +
          size_t(n_tile) * n_bundles * 4;
 }
 
@@ -350,26 +382,11 @@ cudaError_t launch_conv_umma(const UmmaArgs& a, const void* xmap, const void* wm
   memcpy(&xm, xmap, sizeof(CUtensorMap));
   memcpy(&wm, wmap, sizeof(CUtensorMap));
   memcpy(&ym, ymap ? ymap : xmap, sizeof(CUtensorMap));
-  cudaError_t e;
-  if (a.dense) {
-    static bool attr_done_d = false;
-    if (!attr_done_d) {
-      e = cudaFuncSetAttribute(conv3d_umma_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-      if (e != cudaSuccess) return e;
-      attr_done_d = true;
-    }
-    LaunchSetup ls(dim3(grid), dim3(kThreadsUmma), smem, stream);
-    return cudaLaunchKernelEx(&ls.cfg, conv3d_umma_kernel<true>, xm, wm, ym, a, stages, cols);
-  } else {
-    static bool attr_done_s = false;
-    if (!attr_done_s) {
-      e = cudaFuncSetAttribute(conv3d_umma_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-      if (e != cudaSuccess) return e;
-      attr_done_s = true;
-    }
-    LaunchSetup ls(dim3(grid), dim3(kThreadsUmma), smem, stream);
-    return cudaLaunchKernelEx(&ls.cfg, conv3d_umma_kernel<false>, xm, wm, ym, a, stages, cols);
-  }
+  const bool two = pick_cps_single(a.n_tile) == 2;
+  if (a.dense) return two ? launch_single_t<true, 2>(a, xm, wm, ym, grid, smem, stages, cols, stream)
+                          : launch_single_t<true, 1>(a, xm, wm, ym, grid, smem, stages, cols, stream);
+  return two ? launch_single_t<false, 2>(a, xm, wm, ym, grid, smem, stages, cols, stream)
+             : launch_single_t<false, 1>(a, xm, wm, ym, grid, smem, stages, cols, stream);
 }
 
 }  // namespace rt3d
