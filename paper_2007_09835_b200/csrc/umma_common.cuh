@@ -71,6 +71,11 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, Barrier
   }
 }
 
+// Pulls a tensor map (a kernel parameter) into the descriptor cache ahead of its first use.
+__device__ __forceinline__ void tma_prefetch_map(const CUtensorMap* map) {
+  asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(map)) : "memory");
+}
+
 __device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2,
                                             int c3, int c4) {
   asm volatile(
@@ -264,8 +269,15 @@ __device__ __forceinline__ void tma_store_5d(const CUtensorMap* map, uint32_t sr
 __device__ __forceinline__ void tma_store_wait_read_1() {
   asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(kStoreBufs - 1) : "memory");
 }
-// Before the warp leaves the kernel: all its bulk stores have completed (shared memory read, global written).
+// Before the warp leaves the kernel: all its bulk stores have read their staging buffers (shared memory may go
+// away).  Their global writes are part of the grid's memory operations, complete before the grid does.
 __device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+
+// Barrier among the epilogue warps only (named barrier 1): the bias staged after the dependent-launch wait is
+// needed by nobody else, so the producer and MMA warps do not stop for it.
+__device__ __forceinline__ void epilogue_bar_sync(int n_threads) {
+  asm volatile("bar.sync 1, %0;" ::"r"(n_threads) : "memory");
+}
 
 // 32 accumulator columns of this thread's row -> bias, ReLU, bf16 -> staging buffer -> TMA box store of
 // channels [m0, m0+32) x the warp's 32 voxels.

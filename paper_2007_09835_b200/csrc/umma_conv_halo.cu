@@ -97,6 +97,11 @@ conv3d_umma_halo_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_c
   const int cluster_id = blockIdx.x >> 1, n_clusters = gridDim.x >> 1;
   const int box_rows = a.box.bn * a.box.bt * a.box.bh * a.box.bw;
 
+  if (threadIdx.x == 32) {                     // descriptor fetches overlap the rest of the set-up
+    tma_prefetch_map(&xmap);
+    tma_prefetch_map(&wmap_half);
+    tma_prefetch_map(&ymap);
+  }
   if (threadIdx.x == 0) {
     for (int s = 0; s < h.stages; ++s) {
       mbar_init(smem_u32(&bars->full[s]), 1);
@@ -127,8 +132,10 @@ conv3d_umma_halo_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_c
   // starve this one while waiting for it); global memory from here on.
   pdl_launch();
   pdl_wait();
-  for (int i = threadIdx.x; i < a.n_tile; i += blockDim.x) bias_s[i] = (a.bias != nullptr && i < a.g.M) ? __ldg(a.bias + i) : 0.f;
-  __syncthreads();
+  if (warp >= 2) {                               // epilogue warps stage the bias; the other roles start at once
+    for (int i = threadIdx.x - 64; i < a.n_tile; i += 256) bias_s[i] = (a.bias != nullptr && i < a.g.M) ? __ldg(a.bias + i) : 0.f;
+    epilogue_bar_sync(256);
+  }
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer (both CTAs)

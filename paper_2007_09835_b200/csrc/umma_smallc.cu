@@ -47,6 +47,10 @@ conv3d_umma_smallc_kernel(const __grid_constant__ CUtensorMap xmap, const __grid
   const int tiles_per_frame = a.tiles_h * a.tiles_w;
   const int n_items = a.g.n * a.g.To * tiles_per_frame;
 
+  if (threadIdx.x == 32) {                     // descriptor fetches overlap the rest of the set-up
+    tma_prefetch_map(&xmap);
+    tma_prefetch_map(&ymap);
+  }
   if (threadIdx.x == 0) {
     for (int s = 0; s < kSmallCStages; ++s) {
       mbar_init(smem_u32(&bars->full[s]), 1);
