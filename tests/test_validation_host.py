@@ -62,3 +62,47 @@ def test_pool_and_add_argument_errors():
     assert lib.rt3d_maxpool3d(ctypes.byref(x), 0, 2, 2, 2, 2, 2, 0, 0, 0, ctypes.byref(y), None) == B.ERR_INVALID_ARG
     a, b = tensor(1, 2, 4, 4, 16), tensor(1, 2, 4, 4, 24)
     assert lib.rt3d_add_relu(ctypes.byref(a), ctypes.byref(b), 1, ctypes.byref(a), None) == B.ERR_SHAPE
+
+
+def test_fused_call_argument_errors_need_no_device(packed):
+    lib = B.lib()
+    x, y = tensor(1, 4, 8, 8, 16), tensor(1, 4, 8, 8, 32, data=FAKE + (1 << 24))
+    p = B.ConvParams(1, 1, 1, 1, 1, 1, 1, 0)
+
+    def fused(fz, yy=y):
+        return lib.rt3d_conv3d_sparse_fused(ctypes.byref(x), packed.handle, None, ctypes.byref(p), ctypes.byref(fz),
+                                            ctypes.byref(yy), None)
+
+    assert fused(B.Fusion(None, 3, 1, 1)) == B.ERR_INVALID_ARG                         # window must be 1 or 2
+    assert fused(B.Fusion(None, 1, 0, 1)) == B.ERR_INVALID_ARG
+    assert fused(B.Fusion(None, 2, 2, 2)) == B.ERR_SHAPE                               # y is not the pooled extent
+    pooled = tensor(1, 2, 4, 4, 32, data=FAKE + (1 << 24))
+    res = tensor(1, 4, 8, 8, 32, data=FAKE + (1 << 25))
+    assert fused(B.Fusion(ctypes.pointer(res), 2, 2, 2), pooled) == B.ERR_UNSUPPORTED  # residual and pooling together
+    bad_res = tensor(1, 4, 8, 7, 32, data=FAKE + (1 << 25))
+    assert fused(B.Fusion(ctypes.pointer(bad_res), 1, 1, 1)) == B.ERR_SHAPE
+
+
+def test_last_plan_before_any_convolution():
+    import threading
+    out = {}
+
+    def worker():                                   # the record is per thread: a fresh thread has none
+        out["null"] = B.lib().rt3d_last_plan(None)
+        out["fresh"] = B.lib().rt3d_last_plan(ctypes.byref(B.PlanInfo()))
+
+    th = threading.Thread(target=worker)
+    th.start(); th.join()
+    assert out == {"null": B.ERR_INVALID_ARG, "fresh": B.ERR_INVALID_ARG}
+
+
+def test_channel_slice_descriptor():
+    import torch
+    t = torch.zeros((1, 2, 3, 4, 64), dtype=torch.bfloat16)
+    d = B.channel_slice_desc(t, 16, 24)
+    assert (d.c, d.c_stride, d.n, d.t, d.h, d.w) == (24, 64, 1, 2, 3, 4)
+    assert d.data == t.data_ptr() + 32
+    with pytest.raises(ValueError):
+        B.channel_slice_desc(t, 48, 24)             # runs past the pitch
+    with pytest.raises(ValueError):
+        B.channel_slice_desc(t[..., :32], 0, 8)     # not a dense tensor
