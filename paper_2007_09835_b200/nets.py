@@ -186,6 +186,7 @@ class R2Plus1DNet:
     def __init__(self, stem, blocks, layers, fuse_residual: bool = False):
         self.stem, self.blocks, self.layers = stem, blocks, layers
         self.fuse_residual = fuse_residual      # block end = one fused launch instead of conv + add kernel
+        self.side = None
         self.ws = Workspace()
 
     def _conv(self, spec, x, algo, stream):
@@ -200,7 +201,24 @@ class R2Plus1DNet:
                 keep[spec.name] = x
         for blk in self.blocks:
             inp = x
-            sc = inp if blk.shortcut is None else self._conv(blk.shortcut, inp, algo, stream)
+            join = None
+            if blk.shortcut is None:
+                sc = inp
+            elif stream is None:
+                # the strided 1x1x1 projection is independent of the block's main path: side stream, joined
+                # before the residual is added (a parallel branch when captured into a CUDA graph)
+                if self.side is None:
+                    self.side = torch.cuda.Stream(device=x.device)
+                main = torch.cuda.current_stream(x.device)
+                fork = torch.cuda.Event()
+                fork.record(main)
+                self.side.wait_event(fork)
+                with torch.cuda.stream(self.side):
+                    sc = self._conv(blk.shortcut, inp, algo, None)
+                    join = torch.cuda.Event()
+                    join.record(self.side)
+            else:
+                sc = self._conv(blk.shortcut, inp, algo, stream)
             if keep is not None and blk.shortcut is not None:
                 keep[blk.shortcut.name] = sc
             last = blk.convs[-1]
@@ -208,6 +226,8 @@ class R2Plus1DNet:
                 x = self._conv(spec, x, algo, stream)
                 if keep is not None:
                     keep[spec.name] = x
+            if join is not None:
+                torch.cuda.current_stream(x.device).wait_event(join)
             if self.fuse_residual:
                 layer = self.layers[last.name]
                 y = self.ws.get(blk.name + ".out", layer.out_shape(x), x.dtype, x.device)
@@ -228,10 +248,20 @@ class S3DNet:
     """S3D-shaped forward (separable 3-D Inception): stem convs and pools, then Inception blocks whose four
     branches write straight into their channel slice of the block's output tensor (no concat pass)."""
 
-    def __init__(self, plan, layers, input_pad_zero: bool = True):
+    def __init__(self, plan, layers, input_pad_zero: bool = True, parallel_branches: bool = True):
         self.plan, self.layers = plan, layers
         self.input_pad_zero = input_pad_zero
+        # The four branches of an Inception block are independent and mostly too small to fill the GPU (a few
+        # dozen tiles each): run them on separate streams, joined before the next block.  Inside a CUDA graph
+        # capture this becomes parallel branches of the graph.  (Only with the default stream argument.)
+        self.parallel_branches = parallel_branches
+        self.side = None
         self.ws = Workspace()
+
+    def _branch_streams(self, device):
+        if self.side is None:
+            self.side = [torch.cuda.Stream(device=device) for _ in range(3)]
+        return self.side
 
     def _conv(self, spec, x, algo, stream, pad0=False):
         layer = self.layers[spec.name]
@@ -251,18 +281,42 @@ class S3DNet:
                 n, t, h, w, _ = x.shape
                 out = self.ws.get(op.name, (n, t, h, w, op.cout), x.dtype, x.device)
                 xd = B.tensor_desc(x, op.cin)
-                off = 0
-                self.layers[op.b0.name].run_desc(xd, B.channel_slice_desc(out, off, op.b0.cout), algo, stream)
-                off += op.b0.cout
-                for br in (op.b1, op.b2):
+                offs = [0, op.b0.cout, op.b0.cout + op.b1[2].cout, op.b0.cout + op.b1[2].cout + op.b2[2].cout]
+
+                def branch0(x=x, xd=xd, out=out, op=op):
+                    self.layers[op.b0.name].run_desc(xd, B.channel_slice_desc(out, offs[0], op.b0.cout), algo, stream)
+
+                def branch_sep(br, off, x=x, out=out):
                     a = self._conv(br[0], x, algo, stream)
                     b = self._conv(br[1], a, algo, stream)
                     self.layers[br[2].name].run_desc(B.tensor_desc(b, br[2].cin), B.channel_slice_desc(out, off, br[2].cout),
                                                      algo, stream)
-                    off += br[2].cout
-                p = self._pool(op.pool, x, op.cin, stream)
-                self.layers[op.b3.name].run_desc(B.tensor_desc(p, op.cin), B.channel_slice_desc(out, off, op.b3.cout),
-                                                 algo, stream)
+
+                def branch3(x=x, out=out, op=op):
+                    p = self._pool(op.pool, x, op.cin, stream)
+                    self.layers[op.b3.name].run_desc(B.tensor_desc(p, op.cin), B.channel_slice_desc(out, offs[3], op.b3.cout),
+                                                     algo, stream)
+
+                work = [lambda: branch_sep(op.b1, offs[1]), lambda: branch_sep(op.b2, offs[2]), branch3]
+                if self.parallel_branches and stream is None:
+                    main = torch.cuda.current_stream(x.device)
+                    fork = torch.cuda.Event()
+                    fork.record(main)
+                    joins = []
+                    for fn, side in zip(work, self._branch_streams(x.device)):
+                        side.wait_event(fork)
+                        with torch.cuda.stream(side):
+                            fn()
+                            ev = torch.cuda.Event()
+                            ev.record(side)
+                        joins.append(ev)
+                    branch0()                                        # the main stream takes the 1x1x1 branch
+                    for ev in joins:
+                        main.wait_event(ev)
+                else:
+                    branch0()
+                    for fn in work:
+                        fn()
                 x, c = out, op.cout
             elif hasattr(op, "cout"):
                 x = self._conv(op, x, algo, stream, pad0=self.input_pad_zero and i == 0)
