@@ -2,7 +2,7 @@
 
     python -m paper_2007_09835_b200.net_bench --net r2plus1d --batch 8
 
---net c3d | r2plus1d | s3d; synthetic clips and KGS-pruned layers from the seeded generators of rt3d_synth
+--net c3d | c3d_fc (with the fully connected tail) | r2plus1d | s3d; synthetic clips and KGS-pruned layers from the seeded generators of rt3d_synth
 (4x4 groups; keep probability 1/3.6, 0.4 and 1/2.1 as in the paper's Table 2 rates).  By default the pass is
 captured in a CUDA graph and replayed `--iters` times between CUDA events; `--eager` launches the kernels one
 by one instead (what a profiler should see: `--eager --iters 1 --warmup 2` gives one forward pass to capture).
@@ -28,10 +28,16 @@ def build(net: str, dense: bool = False):
         L = synth.make_layer(sp, cfg, i, 4, 4, "none" if dense else "bernoulli", None if dense else density)
         return nets.ConvLayer(sp, L["w"], L["bias"], L["mask"], 4, 4, torch.bfloat16, dense=dense)
 
-    if net == "c3d":
+    if net in ("c3d", "c3d_fc"):
         plan = synth.c3d_plan()
         layers = {op.name: layer(op, 2, i, 1 / 3.6) for i, op in enumerate(plan) if isinstance(op, synth.ConvSpec)}
-        return nets.C3DNet(plan, layers, fuse_pool=True), (16, 112, 112, 3)
+        fc = None
+        if net == "c3d_fc":                     # with the three (unpruned) fully connected layers after pool5
+            fc = []
+            for i, sp in enumerate(synth.c3d_fc_tail()):
+                L = synth.make_layer(sp, 2, 100 + i, 4, 4, "none", None)
+                fc.append(nets.ConvLayer(sp, L["w"], L["bias"], None, 4, 4, torch.bfloat16, dense=True))
+        return nets.C3DNet(plan, layers, fuse_pool=True, fc_layers=fc), (16, 112, 112, 3)
     if net == "r2plus1d":
         stem, blocks = synth.r2plus1d18_plan()
         specs = list(stem)
@@ -48,7 +54,7 @@ def build(net: str, dense: bool = False):
 
 def main(argv=None) -> int:
     ap = argparse.ArgumentParser(description=__doc__, formatter_class=argparse.RawDescriptionHelpFormatter)
-    ap.add_argument("--net", choices=["c3d", "r2plus1d", "s3d"], required=True)
+    ap.add_argument("--net", choices=["c3d", "c3d_fc", "r2plus1d", "s3d"], required=True)
     ap.add_argument("--batch", type=int, default=8)
     ap.add_argument("--dense", action="store_true", help="unpruned weights through the dense path")
     ap.add_argument("--eager", action="store_true", help="no CUDA graph")

@@ -116,9 +116,10 @@ class Workspace:
 class C3DNet:
     """C3D-shaped forward: 8 convs (3x3x3, ReLU) and 5 max-pools.  `layers` maps conv name -> ConvLayer."""
 
-    def __init__(self, plan, layers, fuse_pool: bool = False, input_pad_zero: bool = True):
+    def __init__(self, plan, layers, fuse_pool: bool = False, input_pad_zero: bool = True, fc_layers=None):
         self.plan = plan
         self.layers = layers
+        self.fc_layers = fc_layers      # optional list of dense 1x1x1 ConvLayer (fc6, fc7, fc8) run on the flattened pool5 block
         self.fuse_pool = fuse_pool      # conv + ReLU + un-padded 2-wide max-pool in one launch where the library can
         self.input_pad_zero = input_pad_zero    # the clip tensor comes from to_device(): channels 3..7 are zeros
         self.ws = Workspace()
@@ -173,6 +174,22 @@ class C3DNet:
                 x = maxpool(x, c, op, y, stream=stream)
             if keep is not None:
                 keep[op.name] = x
+        if self.fc_layers:
+            x = self.fc_tail(x, c, algo=algo, keep=keep, stream=stream)
+        return x
+
+    def fc_tail(self, feat: torch.Tensor, c: int, algo=B.ALGO_AUTO, keep=None, stream=None) -> torch.Tensor:
+        """Fully connected layers as 1x1x1 convolutions over the flattened feature block (memory order t, h, w, c;
+        needs the block stored without channel padding)."""
+        n, t, h, w, cs = feat.shape
+        if cs != c:
+            raise ValueError("the feature block must have no channel padding to be flattened in place")
+        x = feat.view(n, 1, 1, 1, t * h * w * c)
+        for layer in self.fc_layers:
+            y = self.ws.get(layer.spec.name, layer.out_shape(x), x.dtype, x.device)
+            x = layer(x, y, algo=algo, stream=stream)
+            if keep is not None:
+                keep[layer.spec.name] = x
         return x
 
     def n_launches(self) -> int:

@@ -160,6 +160,14 @@ def c3d_plan():
     return plan
 
 
+def c3d_fc_tail(n_classes: int = 101):
+    """The three fully connected layers that follow pool5 of the C3D-shaped stack, as 1x1x1 convolutions over
+    the flattened 1 x 4 x 4 x 512 feature block (flattened in memory order h, w, c): 8192 -> 4096 -> 4096 ->
+    classes, ReLU after the first two.  Not pruned (the paper's FLOPs rates are over the conv layers)."""
+    one = lambda nm, ci, co, relu: ConvSpec(nm, ci, co, (1, 1, 1), (1, 1, 1), (0, 0, 0), relu)  # noqa: E731
+    return [one("fc6", 8192, 4096, True), one("fc7", 4096, 4096, True), one("fc8", 4096, n_classes, False)]
+
+
 def r2plus1d_mid(cin: int, cout: int) -> int:
     """Width of the intermediate tensor of a factorised (2+1)D block, chosen so the
     factorised pair has about as many parameters as the 3x3x3 conv it replaces."""

@@ -114,3 +114,19 @@ def s3d_reference(plan, layers, x):
             cur = np.concatenate(parts, axis=-1)
             rec[op.name] = (inp, cur)
     return rec, cur
+
+
+def make_c3d_fc_layers(cfg):
+    return {sp.name: synth.make_layer(sp, cfg, 100 + i, 4, 4, "none", None) for i, sp in enumerate(synth.c3d_fc_tail())}
+
+
+def c3d_fc_reference(fc_layers, feat):
+    """feat: bf16-representable pool5 output [n,1,4,4,512]; returns records and the logits [n,1,1,1,101]."""
+    rec = {}
+    cur = feat.reshape(feat.shape[0], 1, 1, 1, -1)
+    for sp in synth.c3d_fc_tail():
+        L = fc_layers[sp.name]
+        out = oracle.conv3d(cur, L["w"], None, L["bias"], sp.stride, sp.pad, sp.relu, round_bf16=True)
+        rec[sp.name] = (cur, out)
+        cur = oracle.bf16_round(out)
+    return rec, cur

@@ -89,6 +89,25 @@ def test_c3d_free_running_forward(c3d, batch, fuse):
         assert any(net.fused_ok.values())                        # at least conv1/conv2 really ran fused
 
 
+def test_c3d_fc_tail(c3d):
+    """fc6-fc8 as dense 1x1x1 convolutions over the flattened pool5 block: teacher-forced per layer, then the
+    whole stack (convs + pools + FC) free-running against the oracle's logits."""
+    plan, layers, specs, x2, rec, final = c3d
+    fc = netref.make_c3d_fc_layers(2)
+    fc_rec, logits = netref.c3d_fc_reference(fc, final)
+    fc_specs = synth.c3d_fc_tail()
+    fc_dl = [nets.ConvLayer(sp, fc[sp.name]["w"], fc[sp.name]["bias"], None, 4, 4, torch.bfloat16, dense=True) for sp in fc_specs]
+    for sp, lay in zip(fc_specs, fc_dl):
+        inp, ref = fc_rec[sp.name]
+        y = nets.to_numpy(lay(nets.to_device(inp)), sp.cout)
+        assert rel_err(y, ref) <= TOL, sp.name
+    net = nets.C3DNet(plan, device_layers(layers, specs), fuse_pool=True, fc_layers=fc_dl)
+    y = nets.to_numpy(net.forward(nets.to_device(x2)), 101)
+    assert y.shape == (2, 1, 1, 1, 101)
+    assert rt3d.rt3d_last_device_status() == rt3d.OK
+    assert rel_err(y, logits) <= TOL_FREE
+
+
 def test_c3d_dense_path_forward():
     plan, layers = netref.make_c3d_layers(2, 1.0, dense=True)
     specs = [op for op in plan if isinstance(op, synth.ConvSpec)]
