@@ -172,7 +172,7 @@ def time_networks(torch, rt3d, nets, dev, iters=20):
     for i, sp in enumerate(rspecs):
         L = synth.make_layer(sp, 3, i, 4, 4, "bernoulli", 0.4)
         rlayers[sp.name] = nets.ConvLayer(sp, L["w"], L["bias"], L["mask"], 4, 4, torch.bfloat16, device=dev)
-    rnet = nets.R2Plus1DNet(stem, blocks, rlayers, fuse_residual=True)
+    rnet = nets.R2Plus1DNet(stem, blocks, rlayers, fuse_residual=True, fuse_pairs=True)
     x = nets.to_device(synth.make_input(3, (8, 16, 112, 112, 3)), torch.bfloat16, device=dev)
     ms = timed(nets.GraphedForward(rnet, x))
     out["r2plus1d_kgs_b8_clips_per_s"] = 8 / ms * 1e3

@@ -197,6 +197,33 @@ rt3d_status rt3d_conv3d_sparse_fused(const rt3d_tensor* x, const rt3d_packed* w,
                                      void* stream);
 
 /*
+ * rt3d_conv2plus1d_fused - a factorised (2+1)D convolution in one launch: a spatial 1 x Kh x Kw
+ * convolution followed by a temporal Kt x 1 x 1 convolution (the R(2+1)D building block among the
+ * paper's models, Section 5.1), both with KGS-pruned (or dense) packed weights:
+ *     mid = round_bf16(act_s(bias_s + conv(x, W_s (.) mask_s)))        act_s = ReLU iff p_s->relu
+ *     y   = act_t(bias_t + conv(mid, W_t (.) mask_t) + residual)       act_t = ReLU iff p_t->relu
+ * i.e. exactly what rt3d_conv3d_sparse on (x, w_s) into a bf16 tensor `mid`, then
+ * rt3d_conv3d_sparse_fused on (mid, w_t, residual) compute, but `mid` (usually the widest tensor
+ * of the block) stays in shared memory / TMEM and never reaches device memory.
+ *   x, y, residual   device NDHWC tensors as elsewhere; residual has y's extents and dtype, or NULL.
+ *                    y must not overlap x or residual.
+ *   w_s, w_t         packed handles (w_t->N == w_s->M); bias_s [w_s->M], bias_t [w_t->M]: device
+ *                    fp32 or NULL.  p_s / p_t: strides, padding, relu of the two convolutions
+ *                    (algo ignored).
+ * Shape and argument errors are reported as by the separate calls and nothing is launched.
+ * RT3D_ERR_UNSUPPORTED (nothing launched; run the two layers separately) unless: bf16; w_s is
+ * 1 x Kh x Kw with at most 64 input channels; w_t is 3 x 1 x 1 with temporal padding 1; every stride 1;
+ * at most 256 intermediate and 256 output channels with 2*ceil16(mid) + 3*ceil16(out) <= 512; every
+ * temporal tap keeps at least one weight group; both packed weight tensors plus one intermediate
+ * frame of a 16 x 8 patch fit in shared memory; compute capability 10.x.
+ * rt3d_last_plan reports kernel 5.  Same stream, ownership and error conventions as above.
+ */
+rt3d_status rt3d_conv2plus1d_fused(const rt3d_tensor* x, const rt3d_packed* w_s, const float* bias_s,
+                                   const rt3d_conv_params* p_s, const rt3d_packed* w_t, const float* bias_t,
+                                   const rt3d_conv_params* p_t, const rt3d_tensor* residual, rt3d_tensor* y,
+                                   void* stream);
+
+/*
  * rt3d_conv3d_sparse_noalloc - rt3d_conv3d_sparse for callers that must not allocate.
  * (No counterpart in the paper: this is a deployment variant of the tensor-core kernel.)
  * Some callers cannot call cudaMalloc at the point where they run a layer: code inside a
@@ -271,7 +298,8 @@ rt3d_status rt3d_conv3d_cost(const rt3d_tensor* x, const rt3d_packed* w, const r
 
 /* How the calling thread's most recent successful convolution call was run (for tests and profiling):
  *   kernel       0 CUDA-core kernel, 1 tensor-core single-CTA kernel, 2 tensor-core CTA-pair kernel,
- *                3 tensor-core small-C_in kernel, 4 tensor-core resident-weight (halo) kernel
+ *                3 tensor-core small-C_in kernel, 4 tensor-core resident-weight (halo) kernel,
+ *                5 fused (2+1)D kernel (rt3d_conv2plus1d_fused; n_tile = intermediate width)
  *   n_tile       output channels per accumulator tile (tensor-core kernels, else 0)
  *   n_splits     K splits per output tile in the single-CTA kernel (1 = none)
  *   tail_workers CTA pairs that share, cut along K, the output tiles which do not fill a last round

@@ -73,6 +73,7 @@ def _load():
     for name in ("rt3d_conv3d_sparse", "rt3d_conv3d_dense", "rt3d_conv3d_host", "rt3d_conv3d_sparse_noalloc"):
         getattr(lib, name).argtypes = [TP, vp, vp, CP, TP, vp]
     lib.rt3d_conv3d_sparse_fused.argtypes = [TP, vp, vp, CP, ctypes.POINTER(Fusion), TP, vp]
+    lib.rt3d_conv2plus1d_fused.argtypes = [TP, vp, vp, CP, vp, vp, CP, TP, TP, vp]
     lib.rt3d_kgs_group_norms.argtypes = [vp, i, i, i, i, i, i, i, i, vp, vp]
     lib.rt3d_kgs_reweight.argtypes = [vp, ctypes.c_int64, ctypes.c_float, ctypes.c_float, vp, vp, vp]
     lib.rt3d_kgs_expand_mask.argtypes = [vp, i, i, i, i, i, i, i, vp, vp]
@@ -254,6 +255,17 @@ def rt3d_conv3d_sparse_fused(x: Tensor, w: Packed, bias, y: Tensor, stride=(1, 1
     _check(_lib.rt3d_conv3d_sparse_fused(ctypes.byref(x), w.handle, _bias_ptr(bias),
                                          ctypes.byref(_params(stride, pad, relu, algo, x_pad_zero)), ctypes.byref(fz),
                                          ctypes.byref(y), _stream_ptr(stream)), "rt3d_conv3d_sparse_fused")
+
+
+def rt3d_conv2plus1d_fused(x: Tensor, w_s: Packed, bias_s, pad_s, relu_s, w_t: Packed, bias_t, pad_t, relu_t,
+                           y: Tensor, residual: Tensor | None = None, stream=None):
+    """Spatial 1xKhxKw conv then temporal 3x1x1 conv in one launch (all strides 1); Rt3dError with status
+    ERR_UNSUPPORTED when the pair does not fit the fused kernel (run the two layers separately then)."""
+    res = ctypes.pointer(residual) if residual is not None else None
+    _check(_lib.rt3d_conv2plus1d_fused(ctypes.byref(x), w_s.handle, _bias_ptr(bias_s),
+                                       ctypes.byref(_params((1, 1, 1), pad_s, relu_s, ALGO_AUTO)), w_t.handle,
+                                       _bias_ptr(bias_t), ctypes.byref(_params((1, 1, 1), pad_t, relu_t, ALGO_AUTO)),
+                                       res, ctypes.byref(y), _stream_ptr(stream)), "rt3d_conv2plus1d_fused")
 
 
 def rt3d_conv3d_dense(x: Tensor, w: Packed, bias, y: Tensor, stride=(1, 1, 1), pad=(0, 0, 0), relu=False,

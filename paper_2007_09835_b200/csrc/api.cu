@@ -643,9 +643,83 @@ rt3d_status conv_impl(const rt3d_tensor* x, const rt3d_packed* wc, const float* 
   return RT3D_OK;
 }
 
+
+// Fused spatial -> temporal pair.  Argument errors first (as the two separate calls would report them), then
+// the eligibility screen of the one-kernel path.
+rt3d_status conv2plus1d_impl(const rt3d_tensor* x, const rt3d_packed* wsc, const float* bias_s, const rt3d_conv_params* ps,
+                             const rt3d_packed* wtc, const float* bias_t, const rt3d_conv_params* pt,
+                             const rt3d_tensor* res, rt3d_tensor* y, void* stream) {
+  if (!wsc || !wtc || !ps || !pt || !y) return RT3D_ERR_INVALID_ARG;
+  ConvGeom g;
+  rt3d_status s = make_geom(x, wsc, ps, nullptr, &g);
+  if (s != RT3D_OK) return s;
+  if (pt->st < 1 || pt->sh < 1 || pt->sw < 1 || pt->pt < 0 || pt->ph < 0 || pt->pw < 0) return RT3D_ERR_INVALID_ARG;
+  if ((s = check_tensor(y)) != RT3D_OK) return s;
+  if (wtc->N != wsc->M || wtc->dtype != wsc->dtype) return RT3D_ERR_SHAPE;
+  if (g.To + 2 * pt->pt < wtc->Kt || g.Ho + 2 * pt->ph < wtc->Kh || g.Wo + 2 * pt->pw < wtc->Kw) return RT3D_ERR_SHAPE;
+  const int64_t To2 = (int64_t(g.To) + 2 * pt->pt - wtc->Kt) / pt->st + 1;
+  const int64_t Ho2 = (int64_t(g.Ho) + 2 * pt->ph - wtc->Kh) / pt->sh + 1;
+  const int64_t Wo2 = (int64_t(g.Wo) + 2 * pt->pw - wtc->Kw) / pt->sw + 1;
+  if (y->n != g.n || y->t != To2 || y->h != Ho2 || y->w != Wo2 || y->c != wtc->M || y->dtype != wtc->dtype)
+    return RT3D_ERR_SHAPE;
+  if ((s = check_alignment(x)) != RT3D_OK || (s = check_alignment(y)) != RT3D_OK) return s;
+  if (overlaps(x, y)) return RT3D_ERR_INVALID_ARG;
+  if (res) {
+    if ((s = check_tensor(res)) != RT3D_OK || (s = check_alignment(res)) != RT3D_OK) return s;
+    if (res->n != y->n || res->t != y->t || res->h != y->h || res->w != y->w || res->c != y->c || res->dtype != y->dtype)
+      return RT3D_ERR_SHAPE;
+    if (overlaps(res, y)) return RT3D_ERR_INVALID_ARG;
+  }
+  // what the one-kernel path takes
+  if (wsc->dtype != RT3D_BF16) return RT3D_ERR_UNSUPPORTED;
+  if (wsc->Kt != 1 || g.st != 1 || g.sh != 1 || g.sw != 1 || g.pt != 0 || wsc->N > kChunk || wsc->M > 256) return RT3D_ERR_UNSUPPORTED;
+  if (wtc->Kt != 3 || wtc->Kh != 1 || wtc->Kw != 1 || pt->st != 1 || pt->sh != 1 || pt->sw != 1 || pt->pt != 1 ||
+      pt->ph != 0 || pt->pw != 0 || wtc->M > 256)
+    return RT3D_ERR_UNSUPPORTED;
+  rt3d_packed* ws = const_cast<rt3d_packed*>(wsc);
+  rt3d_packed* wt = const_cast<rt3d_packed*>(wtc);
+  DeviceState* d = nullptr;
+  if ((s = get_device_state(&d)) != RT3D_OK) return s;
+  if (!umma_eligible(d, ws, x, y, ps) || !umma_layout_possible(wt)) return RT3D_ERR_UNSUPPORTED;
+  if (res && res->c_stride % 8) return RT3D_ERR_UNSUPPORTED;
+  StArgs a;
+  a.g = g;
+  a.c_mid = ws->M;
+  a.n1 = round_up(ws->M, 16); a.n2 = round_up(wt->M, 16);
+  if (2 * a.n1 + 3 * a.n2 > 512) return RT3D_ERR_UNSUPPORTED;
+  const UmmaLayout* L1 = get_umma_layout(ws, a.n1);
+  const UmmaLayout* L2 = get_umma_layout(wt, a.n2);
+  if (!L1 || !L2 || L1->n_bundles != 1 || L2->n_bundles != 1 || L1->n_chunks != 1) return RT3D_ERR_UNSUPPORTED;
+  a.n_steps1 = L1->step_ptr[1]; a.n_steps2 = L2->step_ptr[1];
+  if (!umma_st_plan(&a, L1->steps.data(), L2->steps.data())) return RT3D_ERR_UNSUPPORTED;
+  DeviceBlob *blob1 = nullptr, *blob2 = nullptr;
+  if ((s = get_blob(ws, &blob1)) != RT3D_OK || (s = get_blob(wt, &blob2)) != RT3D_OK) return s;
+  DeviceBlob::Umma *u1 = nullptr, *u2 = nullptr;
+  if ((s = get_umma_blob(ws, blob1, L1, &u1)) != RT3D_OK || (s = get_umma_blob(wt, blob2, L2, &u2)) != RT3D_OK) return s;
+  a.M2 = wt->M; a.ycs = y->c_stride; a.relu2 = pt->relu ? 1 : 0;
+  a.bias1 = bias_s; a.bias2 = bias_t; a.y = y->data;
+  a.residual = res ? res->data : nullptr; a.rcs = res ? res->c_stride : 0;
+  a.sched = d->sched;
+  CUtensorMap xmap;
+  ConvGeom unit = g;
+  if ((s = encode_xmap(x, unit, TileBox{1, 1, a.hh, a.hw}, &xmap)) != RT3D_OK) return s;
+  cudaError_t e = launch_conv_umma_st(a, &xmap, u1->wmap_half, u2->wmap_half, d->sm_count, static_cast<cudaStream_t>(stream));
+  if (e != cudaSuccess) return RT3D_ERR_CUDA;
+  g_launches.fetch_add(1);
+  t_last_plan = rt3d_plan_info{5, a.n1, 1, 0, 0};
+  return RT3D_OK;
+}
+
 }  // namespace
 
 extern "C" {
+
+rt3d_status rt3d_conv2plus1d_fused(const rt3d_tensor* x, const rt3d_packed* w_s, const float* bias_s,
+                                   const rt3d_conv_params* p_s, const rt3d_packed* w_t, const float* bias_t,
+                                   const rt3d_conv_params* p_t, const rt3d_tensor* residual, rt3d_tensor* y,
+                                   void* stream) {
+  return conv2plus1d_impl(x, w_s, bias_s, p_s, w_t, bias_t, p_t, residual, y, stream);
+}
 
 rt3d_status rt3d_conv3d_sparse(const rt3d_tensor* x, const rt3d_packed* w, const float* bias,
                                const rt3d_conv_params* p, rt3d_tensor* y, void* stream) {

@@ -97,6 +97,35 @@ bool umma_halo_plan(HaloArgs* h, const int32_t* steps_host);
 cudaError_t launch_conv_umma_halo(const HaloArgs& h, const void* xmap, const void* wmap_half, const void* ymap,
                                   int sm_count, cudaStream_t stream);
 
+constexpr int kStMaxMma1 = 64;        // spatial / temporal MMAs per frame the fused (2+1)D kernel can issue
+constexpr int kStMaxMma2 = 48;
+
+// Fused spatial (1 x Kh x Kw) -> temporal (3 x 1 x 1) convolution pair (umma_conv_st.cu).
+struct StArgs {
+  ConvGeom g;                         // the spatial conv: input -> intermediate tensor (To, Ho, Wo; relu = its ReLU)
+  int c_mid;                          // intermediate channels = g.M
+  int n1, n2;                         // accumulator widths: intermediate / output channels rounded up to 16
+  int M2, ycs, relu2;                 // output channels, output channel pitch, final ReLU
+  int n_steps1, n_steps2;             // kept (location, chunk) steps of each layer's single bundle
+  int n_mma1;                         // K=16 MMAs of S per frame
+  int mma2_ptr[4];                    // temporal MMAs of tap dt: [mma2_ptr[dt], mma2_ptr[dt+1])
+  uint32_t tab1[2 * kStMaxMma1];      // per MMA: low descriptor words of A (staged frame) and B (resident weights)
+  uint32_t tab2[2 * kStMaxMma2];      // same for T: A = intermediate frame, B = temporal weights
+  int hw, hh, halo_rows, plane_bytes; // staged input frame under a 16 x 8 patch (patch + kernel extent - 1)
+  int stages;                         // staged frames in flight
+  int tiles_h, tiles_w;               // patches per frame
+  const float* bias1;                 // device or nullptr
+  const float* bias2;
+  void* y;
+  const void* residual;               // device bf16 tensor of the output's extents added before the final ReLU, or nullptr
+  int rcs;
+  int32_t* sched;                     // [2] = error word
+};
+bool umma_st_plan(StArgs* a, const int32_t* steps1_host, const int32_t* steps2_host);
+// xmap: input tensor map with box {64, hw, hh, 1, 1}; w?map_half: half-tile weight maps of the two layers.
+cudaError_t launch_conv_umma_st(const StArgs& a, const void* xmap, const void* w1map_half, const void* w2map_half,
+                                int sm_count, cudaStream_t stream);
+
 // Arguments of the small-C_in tensor-core kernel (C_in <= 8 at channel pitch 8).
 struct SmallCArgs {
   ConvGeom g;

@@ -34,6 +34,11 @@ def main(argv=None) -> int:
     ap.add_argument("--dense", action="store_true")
     ap.add_argument("--algo", type=int, default=B.ALGO_AUTO)
     ap.add_argument("--pool", type=int, nargs=3, default=(1, 1, 1), help="fused max-pool window")
+    ap.add_argument("--temporal-cout", type=int, default=0,
+                    help="follow the (1 x Kh x Kw) layer by a 3x1x1 conv to this many channels, fused into ONE launch "
+                         "(rt3d_conv2plus1d_fused); --separate runs the same pair as two launches")
+    ap.add_argument("--separate", action="store_true")
+    ap.add_argument("--residual", action="store_true", help="with --temporal-cout: add a residual tensor before the final ReLU")
     ap.add_argument("--iters", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     a = ap.parse_args(argv)
@@ -46,7 +51,27 @@ def main(argv=None) -> int:
     x = (torch.rand((n, t, h, w, nets.pitch_for(a.cin, torch.bfloat16)), device="cuda") - 0.5).to(torch.bfloat16)
     x[..., a.cin:] = 0
     pooled = tuple(a.pool) != (1, 1, 1)
-    if pooled:
+    lay_t = None
+    if a.temporal_cout:
+        spec_t = synth.ConvSpec("temporal", a.cout, a.temporal_cout, (3, 1, 1), (1, 1, 1), (1, 0, 0), True)
+        Lt = synth.make_layer(spec_t, 3, 2, a.group[0], a.group[1], "none" if a.dense else "bernoulli", None if a.dense else a.density)
+        lay_t = nets.ConvLayer(spec_t, Lt["w"], Lt["bias"], Lt["mask"], a.group[0], a.group[1], torch.bfloat16, dense=a.dense)
+        y = torch.zeros((n, t, h, w, nets.pitch_for(a.temporal_cout, torch.bfloat16)), dtype=torch.bfloat16, device="cuda")
+        res = (torch.rand_like(y, dtype=torch.float32) - 0.5).to(torch.bfloat16) if a.residual else None
+        if a.separate:
+            mid = lay.alloc_out(x)
+
+            def run():
+                lay(x, mid, x_pad_zero=True)
+                lay_t.fused(mid, y, residual=res)
+        else:
+            xd, yd = B.tensor_desc(x, a.cin), B.tensor_desc(y, a.temporal_cout)
+            rd = None if res is None else B.tensor_desc(res, a.temporal_cout)
+
+            def run():
+                B.rt3d_conv2plus1d_fused(xd, lay.packed, lay.bias, pad, True, lay_t.packed, lay_t.bias, (1, 0, 0), True, yd,
+                                         residual=rd)
+    elif pooled:
         to, ho, wo = spec.out_extent(t, h, w)
         y = torch.zeros((n, to // a.pool[0], ho // a.pool[1], wo // a.pool[2], nets.pitch_for(a.cout, torch.bfloat16)),
                         dtype=torch.bfloat16, device="cuda")
@@ -65,6 +90,11 @@ def main(argv=None) -> int:
     torch.cuda.synchronize()
     us = e0.elapsed_time(e1) / a.iters * 1e3
     kept, dense_macs, alg_bytes = lay.cost(x)
+    if lay_t is not None:                # the pair: MACs of both layers; bytes = input + output (+ residual) + both weight sets
+        k2, d2, b2 = lay_t.cost(lay.alloc_out(x))
+        mid_bytes = n * t * h * w * a.cout * 2
+        kept, dense_macs = kept + k2, dense_macs + d2
+        alg_bytes = alg_bytes + b2 - 2 * mid_bytes + (n * t * h * w * a.temporal_cout * 2 if a.residual else 0)
     print(json.dumps({"us_per_call": us, "plan": B.rt3d_last_plan(), "kept_gmac": kept / 1e9, "dense_gmac": dense_macs / 1e9,
                       "executed_tflops": 2 * dense_macs / us / 1e6, "algorithmic_tflops": 2 * kept / us / 1e6,
                       "algorithmic_gbs": alg_bytes / us / 1e3, "status": B.rt3d_last_device_status()}))

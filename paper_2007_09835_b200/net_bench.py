@@ -22,7 +22,7 @@ from paper_2007_09835_b200 import binding as B  # noqa: E402
 from paper_2007_09835_b200 import nets  # noqa: E402
 
 
-def build(net: str, dense: bool = False):
+def build(net: str, dense: bool = False, pair_fusion: bool = True):
     """Returns (network object, clip shape (t, h, w, c))."""
     def layer(sp, cfg, i, density):
         L = synth.make_layer(sp, cfg, i, 4, 4, "none" if dense else "bernoulli", None if dense else density)
@@ -44,7 +44,7 @@ def build(net: str, dense: bool = False):
         for blk in blocks:
             specs += list(blk.convs) + ([blk.shortcut] if blk.shortcut is not None else [])
         layers = {sp.name: layer(sp, 3, i, 0.4) for i, sp in enumerate(specs)}
-        return nets.R2Plus1DNet(stem, blocks, layers, fuse_residual=True), (16, 112, 112, 3)
+        return nets.R2Plus1DNet(stem, blocks, layers, fuse_residual=True, fuse_pairs=pair_fusion), (16, 112, 112, 3)
     if net == "s3d":
         plan = synth.s3d_plan()
         layers = {sp.name: layer(sp, 5, i, 1 / 2.1) for i, sp in enumerate(synth.s3d_convs(plan))}
@@ -58,11 +58,13 @@ def main(argv=None) -> int:
     ap.add_argument("--batch", type=int, default=8)
     ap.add_argument("--dense", action="store_true", help="unpruned weights through the dense path")
     ap.add_argument("--eager", action="store_true", help="no CUDA graph")
+    ap.add_argument("--no-pair-fusion", action="store_true",
+                    help="r2plus1d: run every factorised pair as two launches (default: one launch where the library fuses it)")
     ap.add_argument("--iters", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     a = ap.parse_args(argv)
 
-    net, clip = build(a.net, a.dense)
+    net, clip = build(a.net, a.dense, not a.no_pair_fusion)
     x = nets.to_device(synth.make_input(7, (a.batch,) + clip))
     fwd = (lambda: net.forward(x)) if a.eager else nets.GraphedForward(net, x)
     for _ in range(a.warmup):

@@ -200,11 +200,38 @@ class R2Plus1DNet:
     """R(2+1)D-18-shaped forward: stem, then residual blocks of two factorised convs each
     (spatial 1x3x3 then temporal 3x1x1), optional 1x1x1 strided projection, add + ReLU."""
 
-    def __init__(self, stem, blocks, layers, fuse_residual: bool = False):
+    def __init__(self, stem, blocks, layers, fuse_residual: bool = False, fuse_pairs: bool = False):
         self.stem, self.blocks, self.layers = stem, blocks, layers
         self.fuse_residual = fuse_residual      # block end = one fused launch instead of conv + add kernel
+        # spatial conv + temporal conv of a factorised pair in ONE launch (rt3d_conv2plus1d_fused) wherever the
+        # library takes the pair; the wide intermediate tensor then never reaches device memory.  Needs
+        # fuse_residual (the block's second pair ends in the residual add) and is skipped while `keep` collects
+        # every layer's output.
+        self.fuse_pairs = fuse_pairs and fuse_residual
+        self.pairs_fused, self.pairs_declined = set(), set()
         self.side = None
         self.ws = Workspace()
+
+    def _pair(self, s_spec, t_spec, x, residual, relu_t, stream, out_name):
+        """The pair in one launch; None if the library declines it (remembered, so it is asked only once)."""
+        if s_spec.name in self.pairs_declined or s_spec.stride != (1, 1, 1) or t_spec.stride != (1, 1, 1):
+            return None
+        ls, lt = self.layers[s_spec.name], self.layers[t_spec.name]
+        n, t, h, w, _ = x.shape
+        t, h, w = t_spec.out_extent(*s_spec.out_extent(t, h, w))
+        y = self.ws.get(out_name, (n, t, h, w, pitch_for(t_spec.cout, x.dtype)), x.dtype, x.device)
+        try:
+            B.rt3d_conv2plus1d_fused(B.tensor_desc(x, s_spec.cin), ls.packed, ls.bias, s_spec.pad, s_spec.relu, lt.packed,
+                                     lt.bias, t_spec.pad, relu_t, B.tensor_desc(y, t_spec.cout),
+                                     residual=None if residual is None else B.tensor_desc(residual, t_spec.cout),
+                                     stream=stream)
+        except B.Rt3dError as e:
+            if e.status != B.ERR_UNSUPPORTED:
+                raise
+            self.pairs_declined.add(s_spec.name)
+            return None
+        self.pairs_fused.add(s_spec.name)
+        return y
 
     def _conv(self, spec, x, algo, stream):
         layer = self.layers[spec.name]
@@ -239,6 +266,20 @@ class R2Plus1DNet:
             if keep is not None and blk.shortcut is not None:
                 keep[blk.shortcut.name] = sc
             last = blk.convs[-1]
+            if self.fuse_pairs and keep is None and algo == B.ALGO_AUTO:
+                c = blk.convs
+                y = self._pair(c[0], c[1], x, None, c[1].relu, stream, c[1].name)
+                x = y if y is not None else self._conv(c[1], self._conv(c[0], x, algo, stream), algo, stream)
+                if join is not None:
+                    torch.cuda.current_stream(x.device).wait_event(join)
+                y = self._pair(c[2], c[3], x, sc, True, stream, blk.name + ".out")
+                if y is None:
+                    x = self._conv(c[2], x, algo, stream)
+                    layer = self.layers[last.name]
+                    y = self.ws.get(blk.name + ".out", layer.out_shape(x), x.dtype, x.device)
+                    y = layer.fused(x, y, residual=sc, relu=True, algo=algo, stream=stream)
+                x = y
+                continue
             for spec in blk.convs[:-1] if self.fuse_residual else blk.convs:
                 x = self._conv(spec, x, algo, stream)
                 if keep is not None:
@@ -257,8 +298,9 @@ class R2Plus1DNet:
         return x
 
     def n_launches(self) -> int:
+        """Launches of one forward pass (after a first pass has found out which pairs the library fuses)."""
         per_block = 4 if self.fuse_residual else 5
-        return len(self.stem) + sum(per_block + (blk.shortcut is not None) for blk in self.blocks)
+        return len(self.stem) + sum(per_block + (blk.shortcut is not None) for blk in self.blocks) - len(self.pairs_fused)
 
 
 class S3DNet:

@@ -155,10 +155,10 @@ def test_r2plus1d_layers_teacher_forced(r21d):
     assert 2.2 < dense_macs / kept_macs < 2.8                    # about 2.5x
 
 
-@pytest.mark.parametrize("fuse", [False, True])
+@pytest.mark.parametrize("fuse", [False, True, "pairs"])
 def test_r2plus1d_free_running_batch8(r21d, fuse):
     stem, blocks, layers, specs, x2, rec, final = r21d
-    net = nets.R2Plus1DNet(stem, blocks, device_layers(layers, specs), fuse_residual=fuse)
+    net = nets.R2Plus1DNet(stem, blocks, device_layers(layers, specs), fuse_residual=bool(fuse), fuse_pairs=fuse == "pairs")
     filler = oracle.bf16_round(synth.make_input(33, (6, 16, 112, 112, 3)))
     x = np.concatenate([x2[:1], filler, x2[1:]], axis=0)
     y = nets.to_numpy(net.forward(nets.to_device(x)), 512)
@@ -167,6 +167,11 @@ def test_r2plus1d_free_running_batch8(r21d, fuse):
     assert (final != 0).mean() > 0.10
     e = rel_err(y[[0, 7]], final)
     assert e <= TOL_FREE, e
+    if fuse == "pairs":       # the two stage-2 blocks run their four factorised pairs as one launch each
+        assert net.pairs_fused == {"s2b1.c1.s", "s2b1.c2.s", "s2b2.c1.s", "s2b2.c2.s"}, (net.pairs_fused, net.pairs_declined)
+        launches = rt3d.rt3d_launch_count()
+        net.forward(nets.to_device(x))
+        assert rt3d.rt3d_launch_count() - launches == net.n_launches()
 
 
 # ------------------------------------------------------------------------------ S3D-shaped
