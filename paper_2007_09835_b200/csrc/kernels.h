@@ -105,12 +105,13 @@ struct StArgs {
   ConvGeom g;                         // the spatial conv: input -> intermediate tensor (To, Ho, Wo; relu = its ReLU)
   int c_mid;                          // intermediate channels = g.M
   int n1, n2;                         // accumulator widths: intermediate / output channels rounded up to 16
+  int c_split;                        // intermediate channels [0, c_split) / [c_split, n1) are converted by different warps
   int M2, ycs, relu2;                 // output channels, output channel pitch, final ReLU
   int n_steps1, n_steps2;             // kept (location, chunk) steps of each layer's single bundle
   int n_mma1;                         // K=16 MMAs of S per frame
   int mma2_ptr[4];                    // temporal MMAs of tap dt: [mma2_ptr[dt], mma2_ptr[dt+1])
   uint32_t tab1[2 * kStMaxMma1];      // per MMA: low descriptor words of A (staged frame) and B (resident weights)
-  uint32_t tab2[2 * kStMaxMma2];      // same for T: A = intermediate frame, B = temporal weights
+  uint32_t tab2[2 * kStMaxMma2];      // T: TMEM column offset of the A slice (intermediate frame), low descriptor word of B
   int hw, hh, halo_rows, plane_bytes; // staged input frame under a 16 x 8 patch (patch + kernel extent - 1)
   int stages;                         // staged frames in flight
   int tiles_h, tiles_w;               // patches per frame

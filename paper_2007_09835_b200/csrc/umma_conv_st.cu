@@ -6,12 +6,13 @@
 // along t: for every frame p it
 //   S(p)  contracts the staged input frame (patch + spatial halo, one TMA box) with the resident spatial
 //         weights into a TMEM accumulator D1 (double buffered),
-//   E1(p) eight epilogue warps turn D1 into the intermediate frame: + bias, ReLU, round to bf16, written to
-//         shared memory as the K-major A operand of the second contraction (no-swizzle layout: 8-channel
-//         slices [slice][128 voxels][16 bytes], so a warp's 32 rows of one slice are 512 contiguous bytes),
+//   E1(p) eight epilogue warps turn D1 into the intermediate frame IN PLACE: + bias, ReLU, round to bf16, and
+//         the packed bf16 values go back into the first half of the same TMEM columns (tcgen05.st), where
+//         they are the A operand of the second contraction (tcgen05.mma with A in tensor memory): the
+//         intermediate tensor never touches shared memory either,
 //   T(p)  adds that frame's contribution to the THREE output frames it touches, out(p-1) += mid(p) Wt[2],
 //         out(p) += mid(p) Wt[1], out(p+1) += mid(p) Wt[0]: three output accumulators live in TMEM, so only
-//         one intermediate frame is ever held (36 KB for 144 channels) and nothing is recomputed along t,
+//         one intermediate frame is ever held and nothing is recomputed along t,
 //   E2    four more epilogue warps drain each output frame once its last contribution has landed
 //         (+ bias, residual, ReLU, bf16, 16-byte global stores).
 // CTA pairs (tcgen05 cta_group::2): two patches per MMA, each CTA holds half of both weight tensors.
@@ -25,7 +26,7 @@
 //
 // Limits (else the caller runs the two layers separately): bf16; C_in <= 64; intermediate and output
 // channels <= 256 with 2 * n1 + 3 * n2 <= 512 TMEM columns; all strides 1; temporal kernel 3 with padding 1;
-// both weight tensors, one intermediate frame and two staged input frames within 227 KB of shared memory.
+// both weight tensors and two staged input frames within 227 KB of shared memory.
 // Every wait is bounded (error word + abort flag, as in the other tensor-core kernels).
 #include "kernels.h"
 #include "umma_common.cuh"
@@ -41,8 +42,7 @@ constexpr int kStOuts = 3;              // output accumulators in flight = tempo
 struct StBars {
   Barriers b;                           // full/empty: staged input frames; tmem_full/empty: D1 buffers
   unsigned long long w_full;            // leader: both weight tensors of both CTAs have landed
-  unsigned long long mid_full;          // leader: 16 E1 warps wrote the intermediate frame
-  unsigned long long mid_empty;         // both: the MMAs reading the intermediate frame are done
+  unsigned long long mid_full;          // leader: 16 E1 warps wrote the intermediate frame back into D1
   unsigned long long out_full[kStOuts]; // both: last contribution to an output accumulator is done
   unsigned long long out_empty[kStOuts];// leader: 8 E2 warps drained it
 };
@@ -52,22 +52,22 @@ struct StBars {
 // min(tb, T-1).
 struct StWalk {
   int T;
-  long long g0, g, g_end;
+  int g0, g, g_end;                     // the launcher keeps the step count below 2^31
   int item, ta, tb, p, pb;
   bool live;
 };
 __device__ __forceinline__ void st_segment(StWalk& k) {
-  k.item = int(k.g / k.T);
-  k.ta = int(k.g - (long long)k.item * k.T);
-  const long long left = k.g_end - k.g;
-  k.tb = (left < k.T - k.ta) ? k.ta + int(left) : k.T;
+  k.item = k.g / k.T;
+  k.ta = k.g - k.item * k.T;
+  const int left = k.g_end - k.g;
+  k.tb = (left < k.T - k.ta) ? k.ta + left : k.T;
   k.p = k.ta > 0 ? k.ta - 1 : 0;
   k.pb = k.tb < k.T ? k.tb : k.T - 1;
 }
 __device__ __forceinline__ void st_init(StWalk& k, int T, long long total, int cluster, int n_clusters) {
   k.T = T;
-  k.g0 = k.g = total * cluster / n_clusters;
-  k.g_end = total * (cluster + 1) / n_clusters;
+  k.g0 = k.g = int(total * cluster / n_clusters);
+  k.g_end = int(total * (cluster + 1) / n_clusters);
   k.live = k.g < k.g_end;
   if (k.live) st_segment(k);
 }
@@ -79,6 +79,32 @@ __device__ __forceinline__ void st_next(StWalk& k) {
   }
 }
 
+// D[tmem] (+)= A[tmem] * B[smem]: the A operand (this CTA's 128 rows, K-major, two bf16 per 32-bit column) is
+// read from tensor memory.
+__device__ __forceinline__ void umma_bf16_pair_ta(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      "setp.ne.b32 p, %4, 0;\n"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], [%1], %2, %3, p;\n"
+      "}\n"
+      ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(acc)
+      : "memory");
+}
+// 16 (8) consecutive 32-bit columns of this thread's TMEM lane <- 4 (2) uint4 of packed bf16 pairs.
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint4 (&o)[4]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
+      ::"r"(taddr), "r"(o[0].x), "r"(o[0].y), "r"(o[0].z), "r"(o[0].w), "r"(o[1].x), "r"(o[1].y), "r"(o[1].z), "r"(o[1].w),
+        "r"(o[2].x), "r"(o[2].y), "r"(o[2].z), "r"(o[2].w), "r"(o[3].x), "r"(o[3].y), "r"(o[3].z), "r"(o[3].w)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st8(uint32_t taddr, const uint4 (&o)[4]) {
+  asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+               ::"r"(taddr), "r"(o[0].x), "r"(o[0].y), "r"(o[0].z), "r"(o[0].w), "r"(o[1].x), "r"(o[1].y), "r"(o[1].z), "r"(o[1].w)
+               : "memory");
+}
+
 __global__ void __launch_bounds__(kThreadsSt, 1)
 conv3d_umma_st_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CUtensorMap w1map,
                       const __grid_constant__ CUtensorMap w2map, const StArgs a, const int tmem_cols) {
@@ -88,8 +114,7 @@ conv3d_umma_st_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_con
   const uint32_t b1_bytes = uint32_t(a.n1 / 2) * 128u, b2_bytes = uint32_t(a.n2 / 2) * 128u;
   const uint32_t w1_smem = base;
   const uint32_t w2_smem = w1_smem + uint32_t(a.n_steps1) * b1_bytes;
-  const uint32_t mid_smem = w2_smem + uint32_t(a.n_steps2) * b2_bytes;
-  const uint32_t in_smem = mid_smem + uint32_t(a.n1) * 256u;            // 128 voxels x n1 channels of bf16
+  const uint32_t in_smem = w2_smem + uint32_t(a.n_steps2) * b2_bytes;
   unsigned char* tail = smem_raw + (in_smem - raw) + size_t(a.stages) * a.plane_bytes;
   StBars* sb = reinterpret_cast<StBars*>(tail);
   Barriers* bars = &sb->b;
@@ -115,13 +140,9 @@ conv3d_umma_st_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_con
       mbar_init(smem_u32(&bars->full[s]), 1);
       mbar_init(smem_u32(&bars->empty[s]), 1);
     }
-    for (int b = 0; b < 2; ++b) {
-      mbar_init(smem_u32(&bars->tmem_full[b]), 1);
-      mbar_init(smem_u32(&bars->tmem_empty[b]), 16);     // leader: 8 E1 warps of each CTA
-    }
+    for (int b = 0; b < 2; ++b) mbar_init(smem_u32(&bars->tmem_full[b]), 1);
     mbar_init(smem_u32(&sb->w_full), 1);
-    mbar_init(smem_u32(&sb->mid_full), 16);
-    mbar_init(smem_u32(&sb->mid_empty), 1);
+    mbar_init(smem_u32(&sb->mid_full), 16);              // leader: 8 E1 warps of each CTA
     for (int s = 0; s < kStOuts; ++s) {
       mbar_init(smem_u32(&sb->out_full[s]), 1);
       mbar_init(smem_u32(&sb->out_empty[s]), 8);         // leader: 4 E2 warps of each CTA
@@ -194,12 +215,10 @@ conv3d_umma_st_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_con
       asm volatile("{\n.reg .pred p;\nelect.sync _|p, 0xffffffff;\nselp.u32 %0, 1, 0, p;\n}\n" : "=r"(elected));
       const uint32_t idesc1 = instr_desc_bf16_pair(a.n1), idesc2 = instr_desc_bf16_pair(a.n2);
       // high descriptor words.  Staged input: 128-byte swizzle, 8-row groups one halo row apart.  Weights:
-      // 128-byte swizzle, groups 1024 bytes apart.  Intermediate frame: no swizzle, groups 128 bytes apart
-      // (the distance between its two 8-channel slices sits in the low word, in the table).
+      // 128-byte swizzle, groups 1024 bytes apart.  (The intermediate frame is read from tensor memory.)
       const uint64_t a1_hi = uint64_t(((uint32_t(a.hw) * 128u) >> 4) | (1u << 14) | (2u << 29)) << 32;
       const uint64_t b_hi = uint64_t((1024u >> 4) | (1u << 14) | (2u << 29)) << 32;
-      const uint64_t a2_hi = uint64_t((128u >> 4) | (1u << 14)) << 32;
-      const uint32_t w1_16 = w1_smem >> 4, w2_16 = w2_smem >> 4, mid16 = mid_smem >> 4;
+      const uint32_t w1_16 = w1_smem >> 4, w2_16 = w2_smem >> 4;
       int stage = 0;
       uint32_t phase = 0;
       bool ok = mbar_wait(smem_u32(&sb->w_full), 0, bars, err, 42);
@@ -208,10 +227,11 @@ conv3d_umma_st_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_con
       nxt = cur;
       if (nxt.live) st_next(nxt);
       uint32_t j = 0;
-      // S of job jj into D1 buffer jj & 1
+      // S of job jj into D1 buffer jj & 1.  The buffer's previous contents (the intermediate frame of job jj - 2)
+      // were last read by T(jj - 2), issued earlier from this same thread: the tensor pipe keeps that order, so
+      // no barrier guards the reuse.
       auto issue_s = [&](uint32_t jj) -> bool {
         const uint32_t buf = jj & 1u;
-        if (!mbar_wait(smem_u32(&bars->tmem_empty[buf]), ((jj >> 1) & 1u) ^ 1u, bars, err, 43)) return false;
         if (!mbar_wait(smem_u32(&bars->full[stage]), phase, bars, err, 44)) return false;
         tc_fence_after();
         const uint32_t d = tmem_base + buf * uint32_t(a.n1);
@@ -229,31 +249,48 @@ conv3d_umma_st_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_con
         if (++stage == a.stages) { stage = 0; phase ^= 1u; }
         return true;
       };
+      // Per job j: all of S(j+1), then T(j), so that E1 converts frame j while the tensor pipe works on S(j+1).
+      // (Mixing the two shapes more finely is slower: alternating single MMAs of S and T took 143 us, and
+      // alternating T's taps with thirds of S 122 us, against 93 us in this order for the R(2+1)D stage-2 block.)
       if (ok && cur.live) ok = issue_s(0);
       while (ok && cur.live) {
         if (nxt.live) { if (!issue_s(j + 1)) break; }
         if (!mbar_wait(smem_u32(&sb->mid_full), j & 1u, bars, err, 45)) break;
         tc_fence_after();
-        const int qb = int(cur.g - cur.g0) - cur.ta;       // running number of output frame o is qb + o
-        for (int dt = 2; dt >= 0 && ok; --dt) {
+        const int qb = cur.g - cur.g0 - cur.ta;            // running number of output frame o is qb + o
+        const uint32_t mid_tmem = tmem_base + (j & 1u) * uint32_t(a.n1);
+        // the taps this job issues, oldest output frame first; a frame that starts here needs its accumulator
+        // drained of the frame that used it before.  All waiting is done before the first MMA is issued.
+        bool live[3];
+        uint32_t dd[3], acc0[3];
+#pragma unroll
+        for (int dt = 0; dt < 3; ++dt) {
           const int o = cur.p + 1 - dt;
-          if (o < cur.ta || o >= cur.tb) continue;
+          live[dt] = o >= cur.ta && o < cur.tb;
           const uint32_t q = uint32_t(qb + o), slot = q % kStOuts;
           const bool first = cur.p == (o > 0 ? o - 1 : 0);
-          if (first && !mbar_wait(smem_u32(&sb->out_empty[slot]), ((q / kStOuts) & 1u) ^ 1u, bars, err, 46)) { ok = false; break; }
-          if (first) tc_fence_after();
-          const uint32_t d = out_tmem + slot * uint32_t(a.n2);
+          dd[dt] = out_tmem + slot * uint32_t(a.n2);
+          acc0[dt] = first ? 0u : 1u;
+          if (live[dt] && first && ok)
+            ok = mbar_wait(smem_u32(&sb->out_empty[slot]), ((q / kStOuts) & 1u) ^ 1u, bars, err, 46);
+        }
+        if (!ok) break;
+        tc_fence_after();
+#pragma unroll
+        for (int dt = 2; dt >= 0; --dt) {
+          if (!live[dt]) continue;
           const int m0 = a.mma2_ptr[dt], m1 = a.mma2_ptr[dt + 1];
+          const uint32_t d = dd[dt];
+          uint32_t acc = acc0[dt];
 #pragma unroll 2
           for (int m = m0; m < m1; ++m) {
-            const uint64_t adesc = a2_hi | uint64_t(mid16 + a.tab2[2 * m]);
             const uint64_t bdesc = b_hi | uint64_t(w2_16 + a.tab2[2 * m + 1]);
-            if (elected) umma_bf16_pair(d, adesc, bdesc, idesc2, (m > m0 || !first) ? 1u : 0u);
+            if (elected) umma_bf16_pair_ta(d, mid_tmem + a.tab2[2 * m], bdesc, idesc2, acc);
+            acc = 1u;
           }
         }
         if (!ok) break;
         if (elected) {
-          umma_commit_pair(smem_u32(&sb->mid_empty));
           const int o1 = cur.p - 1;
           if (o1 >= cur.ta && o1 < cur.tb) umma_commit_pair(smem_u32(&sb->out_full[uint32_t(qb + o1) % kStOuts]));
           if (cur.p == T - 1 && cur.p >= cur.ta && cur.p < cur.tb)
@@ -268,8 +305,7 @@ conv3d_umma_st_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_con
   } else if (warp < 10) {
     // ------------------------------------------------------------------ E1: D1 -> intermediate frame (both CTAs, 8 warps)
     const int quad = warp & 3;
-    const int half = (warp - 2) >> 2;           // 0: even 32-column pieces, 1: odd ones
-    const uint32_t row16 = uint32_t(quad * 32 + lane) * 16u;
+    const int half = (warp - 2) >> 2;           // 0: columns [0, c_split), 1: [c_split, n1)
     const uint32_t mid_full_leader = mapa_shared(smem_u32(&sb->mid_full), 0);
     StWalk k;
     uint32_t j = 0;
@@ -278,16 +314,17 @@ conv3d_umma_st_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_con
       if (!mbar_wait(smem_u32(&bars->tmem_full[buf]), (j >> 1) & 1u, bars, err, 47)) break;
       tc_fence_after();
       const uint32_t taddr = tmem_base + (uint32_t(quad * 32) << 16) + buf * uint32_t(a.n1);
-      // All of this warp's pieces (up to four of 32 columns) are converted into registers first, so that D1 is
-      // released at once and only the shared-memory stores remain once the previous frame's temporal MMAs
-      // have finished reading the buffer.
+      // The two warps of a lane quadrant split the columns at c_split (a multiple of 16); each converts all of its
+      // pieces (up to four of 32 columns) into registers and then writes the packed values back over the
+      // first half of ITS OWN column range, so neither overwrites columns the other still has to read.
+      const int r0 = half ? a.c_split : 0, r1 = half ? a.n1 : a.c_split;
       uint4 o[4][4];
 #pragma unroll
       for (int pc = 0; pc < 4; ++pc) {
-        const int col = half * 32 + pc * 64;
-        if (col < a.n1) {
+        const int col = r0 + pc * 32;
+        if (col < r1) {
           uint32_t v[32];
-          const bool wide = col + 32 <= a.n1;
+          const bool wide = col + 32 <= r1;
           if (wide) tmem_ld32(taddr + col, v);
           else tmem_ld16_into32(taddr + col, v);
           __nv_bfloat162* po = reinterpret_cast<__nv_bfloat162*>(o[pc]);
@@ -303,29 +340,18 @@ conv3d_umma_st_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_con
           }
         }
       }
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive_cluster(mapa_shared(smem_u32(&bars->tmem_empty[buf]), 0));
-      {
-        if (!mbar_wait(smem_u32(&sb->mid_empty), (j & 1u) ^ 1u, bars, err, 48)) break;
-      }
 #pragma unroll
       for (int pc = 0; pc < 4; ++pc) {
-        const int col = half * 32 + pc * 64;
-        if (col < a.n1) {
-          const bool wide = col + 32 <= a.n1;
-          const uint32_t dst = mid_smem + uint32_t(col >> 3) * 2048u + row16;
-#pragma unroll
-          for (uint32_t s = 0; s < 4; ++s)
-            if (wide || s < 2)
-              asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst + s * 2048u), "r"(o[pc][s].x),
-                           "r"(o[pc][s].y), "r"(o[pc][s].z), "r"(o[pc][s].w) : "memory");
+        const int col = r0 + pc * 32;
+        if (col < r1) {
+          const uint32_t dst = taddr + uint32_t(r0 + pc * 16);       // two bf16 per 32-bit column
+          if (col + 32 <= r1) tmem_st16(dst, o[pc]);
+          else tmem_st8(dst, o[pc]);
         }
       }
-      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+      tc_fence_before();
       __syncwarp();
-      // default arrive semantics: each CTA's tensor core reads its OWN shared memory, made visible to the async
-      // proxy by the fence above; the barrier only tells the issuing thread that both halves are ready
       if (lane == 0) mbar_arrive_cluster(mid_full_leader);
     }
   } else {
@@ -339,7 +365,7 @@ conv3d_umma_st_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_con
     StWalk k;
     bool ok = true;
     for (st_init(k, T, total, cluster_id, n_clusters); k.live && ok; st_next(k)) {
-      const int qb = int(k.g - k.g0) - k.ta;
+      const int qb = k.g - k.g0 - k.ta;
       for (int which = 0; which < 2 && ok; ++which) {
         const int o = which == 0 ? k.p - 1 : k.p;
         if (o < k.ta || o >= k.tb || (which == 1 && k.p != T - 1)) continue;
@@ -435,7 +461,7 @@ conv3d_umma_st_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_con
 
 
 size_t st_smem_bytes(const StArgs& a) {
-  return 1024 + size_t(a.n_steps1) * (a.n1 / 2) * 128 + size_t(a.n_steps2) * (a.n2 / 2) * 128 + size_t(a.n1) * 256 +
+  return 1024 + size_t(a.n_steps1) * (a.n1 / 2) * 128 + size_t(a.n_steps2) * (a.n2 / 2) * 128 +
          size_t(a.stages) * a.plane_bytes + sizeof(StBars) + size_t(a.n1 + a.n2) * 4 + 16;
 }
 
@@ -474,6 +500,7 @@ bool umma_st_plan(StArgs* a, const int32_t* steps1_host, const int32_t* steps2_h
   }
   a->n_mma1 = m;
   for (int q = 2 * m; q < 2 * kStMaxMma1; ++q) a->tab1[q] = 0u;
+  a->c_split = 16 * ((a->n1 / 16 + 1) / 2);
   // temporal MMAs, grouped by dt: step = (dt, 64-channel chunk of the intermediate frame)
   const int chunks2 = (a->c_mid + 63) / 64;
   const int last_k16 = (a->c_mid - (chunks2 - 1) * 64 + 15) / 16;
@@ -491,8 +518,10 @@ bool umma_st_plan(StArgs* a, const int32_t* steps1_host, const int32_t* steps2_h
       if (m + kc > kStMaxMma2) return false;
       const uint32_t b_off = uint32_t(size_t(s) * b2 >> 4);
       for (int kk = 0; kk < kc; ++kk, ++m) {
-        // 8-channel slices (ch*8 + 2kk, +1) of the frame, 2048 bytes each; LBO field = slice distance
-        a->tab2[2 * m] = (uint32_t(ch * 8 + 2 * kk) * (2048u >> 4)) | ((2048u >> 4) << 16);
+        // 16 channels of the intermediate frame = 8 TMEM columns of packed bf16 pairs; the slices of the second
+        // half of the channels start at column c_split (see E1 in the kernel)
+        const int s16 = ch * 4 + kk, s_half = a->c_split / 16;
+        a->tab2[2 * m] = uint32_t(s16 < s_half ? s16 * 8 : a->c_split + (s16 - s_half) * 8);
         a->tab2[2 * m + 1] = (b_off + 2u * uint32_t(kk)) | (1u << 16);
       }
     }
@@ -501,7 +530,7 @@ bool umma_st_plan(StArgs* a, const int32_t* steps1_host, const int32_t* steps2_h
   if (s != a->n_steps2) return false;
   a->mma2_ptr[3] = m;
   for (int q = 2 * m; q < 2 * kStMaxMma2; ++q) a->tab2[q] = 0u;
-  for (a->stages = 3; a->stages >= 2; --a->stages)
+  for (a->stages = 4; a->stages >= 2; --a->stages)
     if (st_smem_bytes(*a) <= 227 * 1024) return true;
   return false;
 }
@@ -517,6 +546,7 @@ cudaError_t launch_conv_umma_st(const StArgs& a, const void* xmap, const void* w
   const long long n_patches = (long long)a.g.n * a.tiles_h * a.tiles_w;
   const long long total = ((n_patches + 1) / 2) * a.g.To;
   if (total <= 0) return cudaSuccess;
+  if (total >= (1ll << 31)) return cudaErrorInvalidValue;
   CUtensorMap xm, w1m, w2m;
   memcpy(&xm, xmap, sizeof(CUtensorMap));
   memcpy(&w1m, w1map_half, sizeof(CUtensorMap));
