@@ -24,6 +24,12 @@
 // balanced at a few per cent of extra work, where whole patches per pair would leave half the SMs idle in
 // the second round (112 patch pairs over 74 CTA pairs for the R(2+1)D stage-2 shapes).
 //
+// Tried and not kept: the three taps of T as ONE MMA of N = 3 x C_out per 16 channels over the three adjacent
+// accumulators (taps stacked in shared memory as the cyclic sequence Wt2 Wt1 Wt0 Wt2 Wt1, of which a rotation
+// picks three blocks; E2 clearing each accumulator after use since a wide MMA cannot start one frame from zero):
+// correct, 9 instead of 27 temporal MMAs per frame, and the same 90-92 us, with narrower limits
+// (3 x C_out <= 256, two input stages).  The kernel is not bound by the temporal MMAs' issue rate alone.
+//
 // Limits (else the caller runs the two layers separately): bf16; C_in <= 64; intermediate and output
 // channels <= 256 with 2 * n1 + 3 * n2 <= 512 TMEM columns; all strides 1; temporal kernel 3 with padding 1;
 // both weight tensors and two staged input frames within 227 KB of shared memory.
@@ -314,40 +320,29 @@ conv3d_umma_st_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_con
       if (!mbar_wait(smem_u32(&bars->tmem_full[buf]), (j >> 1) & 1u, bars, err, 47)) break;
       tc_fence_after();
       const uint32_t taddr = tmem_base + (uint32_t(quad * 32) << 16) + buf * uint32_t(a.n1);
-      // The two warps of a lane quadrant split the columns at c_split (a multiple of 16); each converts all of its
-      // pieces (up to four of 32 columns) into registers and then writes the packed values back over the
-      // first half of ITS OWN column range, so neither overwrites columns the other still has to read.
+      // The two warps of a lane quadrant split the columns at c_split (a multiple of 16).  Each walks its range in
+      // pieces of 32 columns and writes the packed values of piece k back over columns [16k, 16k + 16) of ITS OWN
+      // range: those belong to piece k / 2, which it has read already, and never to the other warp's range.
       const int r0 = half ? a.c_split : 0, r1 = half ? a.n1 : a.c_split;
-      uint4 o[4][4];
+      for (int col = r0, dst_col = r0; col < r1; col += 32, dst_col += 16) {
+        uint32_t v[32];
+        const bool wide = col + 32 <= r1;
+        if (wide) tmem_ld32(taddr + col, v);
+        else tmem_ld16_into32(taddr + col, v);
+        uint4 o[4];
+        __nv_bfloat162* po = reinterpret_cast<__nv_bfloat162*>(o);
+        const float4* b4 = reinterpret_cast<const float4*>(bias1_s + col);
 #pragma unroll
-      for (int pc = 0; pc < 4; ++pc) {
-        const int col = r0 + pc * 32;
-        if (col < r1) {
-          uint32_t v[32];
-          const bool wide = col + 32 <= r1;
-          if (wide) tmem_ld32(taddr + col, v);
-          else tmem_ld16_into32(taddr + col, v);
-          __nv_bfloat162* po = reinterpret_cast<__nv_bfloat162*>(o[pc]);
-          const float4* b4 = reinterpret_cast<const float4*>(bias1_s + col);
-#pragma unroll
-          for (int q = 0; q < 8; ++q) {
-            const float4 b = (wide || q < 4) ? b4[q] : make_float4(0.f, 0.f, 0.f, 0.f);
-            float f0 = __uint_as_float(v[4 * q]) + b.x, f1 = __uint_as_float(v[4 * q + 1]) + b.y;
-            float f2 = __uint_as_float(v[4 * q + 2]) + b.z, f3 = __uint_as_float(v[4 * q + 3]) + b.w;
-            if (a.g.relu) { f0 = fmaxf(f0, 0.f); f1 = fmaxf(f1, 0.f); f2 = fmaxf(f2, 0.f); f3 = fmaxf(f3, 0.f); }
-            po[2 * q] = __floats2bfloat162_rn(f0, f1);
-            po[2 * q + 1] = __floats2bfloat162_rn(f2, f3);
-          }
+        for (int q = 0; q < 8; ++q) {
+          const float4 b = (wide || q < 4) ? b4[q] : make_float4(0.f, 0.f, 0.f, 0.f);
+          float f0 = __uint_as_float(v[4 * q]) + b.x, f1 = __uint_as_float(v[4 * q + 1]) + b.y;
+          float f2 = __uint_as_float(v[4 * q + 2]) + b.z, f3 = __uint_as_float(v[4 * q + 3]) + b.w;
+          if (a.g.relu) { f0 = fmaxf(f0, 0.f); f1 = fmaxf(f1, 0.f); f2 = fmaxf(f2, 0.f); f3 = fmaxf(f3, 0.f); }
+          po[2 * q] = __floats2bfloat162_rn(f0, f1);
+          po[2 * q + 1] = __floats2bfloat162_rn(f2, f3);
         }
-      }
-#pragma unroll
-      for (int pc = 0; pc < 4; ++pc) {
-        const int col = r0 + pc * 32;
-        if (col < r1) {
-          const uint32_t dst = taddr + uint32_t(r0 + pc * 16);       // two bf16 per 32-bit column
-          if (col + 32 <= r1) tmem_st16(dst, o[pc]);
-          else tmem_st8(dst, o[pc]);
-        }
+        if (wide) tmem_st16(taddr + uint32_t(dst_col), o);
+        else tmem_st8(taddr + uint32_t(dst_col), o);
       }
       asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
       tc_fence_before();
