@@ -83,6 +83,40 @@ def test_fused_call_argument_errors_need_no_device(packed):
     assert fused(B.Fusion(ctypes.pointer(bad_res), 1, 1, 1)) == B.ERR_SHAPE
 
 
+def test_fused_pair_argument_errors_need_no_device():
+    """rt3d_conv2plus1d_fused: argument and shape errors as the two separate calls would give them, and the
+    refusals that depend on the layers alone, all before any CUDA call."""
+    def pack(cin, cout, k, dtype=B.RT3D_BF16):
+        spec = synth.ConvSpec("p", cin, cout, k, (1, 1, 1), tuple(kk // 2 for kk in k))
+        L = synth.make_layer(spec, 6, cin + cout, 4, 4, "bernoulli", 0.5)
+        return B.rt3d_pack_kgs(L["w"], L["mask"], 4, 4, dtype)
+
+    ws, wt = pack(16, 48, (1, 3, 3)), pack(48, 32, (3, 1, 1))
+    lib = B.lib()
+    x, y = tensor(1, 4, 8, 8, 16), tensor(1, 4, 8, 8, 32, data=FAKE + (1 << 24))
+    ps, pt = B.ConvParams(1, 1, 1, 0, 1, 1, 1, 0), B.ConvParams(1, 1, 1, 1, 0, 0, 1, 0)
+
+    def pair(xx=x, yy=y, w1=ws, w2=wt, p1=ps, p2=pt, res=None):
+        return lib.rt3d_conv2plus1d_fused(ctypes.byref(xx), w1.handle, None, ctypes.byref(p1), w2.handle, None,
+                                          ctypes.byref(p2), None if res is None else ctypes.byref(res), ctypes.byref(yy), None)
+
+    assert pair(xx=tensor(1, 4, 8, 8, 24)) == B.ERR_SHAPE                              # x channels != w_s->N
+    assert pair(yy=tensor(1, 4, 8, 8, 48, data=FAKE + (1 << 24))) == B.ERR_SHAPE       # y channels != w_t->M
+    assert pair(yy=tensor(1, 2, 8, 8, 32, data=FAKE + (1 << 24))) == B.ERR_SHAPE       # wrong output extent
+    assert pair(w2=pack(40, 32, (3, 1, 1))) == B.ERR_SHAPE                             # w_t->N != w_s->M
+    assert pair(p2=B.ConvParams(0, 1, 1, 1, 0, 0, 1, 0)) == B.ERR_INVALID_ARG          # stride 0
+    assert pair(yy=tensor(1, 4, 8, 8, 32)) == B.ERR_INVALID_ARG                        # y overlaps x
+    assert pair(res=tensor(1, 4, 8, 7, 32, data=FAKE + (1 << 25))) == B.ERR_SHAPE      # residual extent
+    assert pair(res=y) == B.ERR_INVALID_ARG                                            # residual overlaps y
+    # layer pairs the one-kernel path does not take: refused on the host, nothing launched
+    assert pair(w1=pack(16, 48, (3, 3, 3)), p1=B.ConvParams(1, 1, 1, 1, 1, 1, 1, 0)) == B.ERR_UNSUPPORTED    # not 1xKhxKw
+    assert pair(yy=tensor(1, 4, 4, 4, 32, data=FAKE + (1 << 24)), p1=B.ConvParams(1, 2, 2, 0, 1, 1, 1, 0)) == B.ERR_UNSUPPORTED   # strided
+    f32s, f32t = pack(16, 48, (1, 3, 3), B.RT3D_F32), pack(48, 32, (3, 1, 1), B.RT3D_F32)
+    xf = tensor(1, 4, 8, 8, 16, dtype=B.RT3D_F32)
+    yf = tensor(1, 4, 8, 8, 32, dtype=B.RT3D_F32, data=FAKE + (1 << 24))
+    assert pair(xx=xf, yy=yf, w1=f32s, w2=f32t) == B.ERR_UNSUPPORTED                   # fp32
+
+
 def test_last_plan_before_any_convolution():
     import threading
     out = {}
