@@ -253,11 +253,25 @@ struct TmaStore {
 
 // Fused max-pool (window = stride = 1 or 2 per axis) over the 32 voxels of an epilogue warp, which form a
 // block of sbw x sbh x sbt(...) voxels whose extents are multiples of the window: lane -> (w, h, t) inside
-// the block, partner lanes differ by 1, sbw and sbw*sbh.
+// the block, partner lanes differ by 1, sbw and sbw*sbh.  Everything that depends only on the lane is worked
+// out once per thread (make_pool_lanes), not once per 32-channel piece: it takes a dozen integer divisions.
 struct PoolLanes {
   int pw, ph, pt;             // window
-  int sbw, sbh;               // block extents along w and h (lane = (t*sbh + h)*sbw + w)
+  int src_w, src_h, src_t;    // partner lane along each axis
+  int out_row;                // row of the pooled block this lane's window leader writes
+  bool writer;                // this lane is the leader of its window
 };
+__device__ __forceinline__ PoolLanes make_pool_lanes(int pw, int ph, int pt, int sbw, int sbh, int lane) {
+  PoolLanes p;
+  p.pw = pw; p.ph = ph; p.pt = pt;
+  const int w = lane % sbw, h = (lane / sbw) % sbh, t = lane / (sbw * sbh);
+  p.src_w = lane ^ 1;
+  p.src_h = (h & 1) ? lane - sbw : lane + sbw;
+  p.src_t = (t & 1) ? lane - sbw * sbh : lane + sbw * sbh;
+  p.writer = (w % pw == 0) && (h % ph == 0) && (t % pt == 0);
+  p.out_row = ((t / pt) * (sbh / ph) + h / ph) * (sbw / pw) + w / pw;
+  return p;
+}
 
 __device__ __forceinline__ void tma_store_5d(const CUtensorMap* map, uint32_t src, int c0, int c1, int c2, int c3, int c4) {
   asm volatile("cp.async.bulk.tensor.5d.global.shared::cta.tile.bulk_group [%0, {%2, %3, %4, %5, %6}], [%1];"
@@ -318,35 +332,30 @@ __device__ __forceinline__ void epilogue_piece_tma(const uint32_t* v, const floa
   int out_row = lane;
   bool writer = true;
   if (pool != nullptr) {
-    const int w = lane % pool->sbw, h = (lane / pool->sbw) % pool->sbh, t = lane / (pool->sbw * pool->sbh);
     uint32_t* u = reinterpret_cast<uint32_t*>(o);
     if (pool->pw == 2) {
-      const int src = lane ^ 1;
 #pragma unroll
       for (int q = 0; q < 16; ++q) {
-        const uint32_t other = __shfl_sync(0xffffffffu, u[q], src);
+        const uint32_t other = __shfl_sync(0xffffffffu, u[q], pool->src_w);
         po[q] = __hmax2(po[q], *reinterpret_cast<const __nv_bfloat162*>(&other));
       }
     }
     if (pool->ph == 2) {
-      const int src = (h & 1) ? lane - pool->sbw : lane + pool->sbw;
 #pragma unroll
       for (int q = 0; q < 16; ++q) {
-        const uint32_t other = __shfl_sync(0xffffffffu, u[q], src);
+        const uint32_t other = __shfl_sync(0xffffffffu, u[q], pool->src_h);
         po[q] = __hmax2(po[q], *reinterpret_cast<const __nv_bfloat162*>(&other));
       }
     }
     if (pool->pt == 2) {
-      const int plane = pool->sbw * pool->sbh;
-      const int src = (t & 1) ? lane - plane : lane + plane;
 #pragma unroll
       for (int q = 0; q < 16; ++q) {
-        const uint32_t other = __shfl_sync(0xffffffffu, u[q], src);
+        const uint32_t other = __shfl_sync(0xffffffffu, u[q], pool->src_t);
         po[q] = __hmax2(po[q], *reinterpret_cast<const __nv_bfloat162*>(&other));
       }
     }
-    writer = (w % pool->pw == 0) && (h % pool->ph == 0) && (t % pool->pt == 0);
-    out_row = ((t / pool->pt) * (pool->sbh / pool->ph) + h / pool->ph) * (pool->sbw / pool->pw) + w / pool->pw;
+    writer = pool->writer;
+    out_row = pool->out_row;
   }
   const uint32_t buf = ts.smem + (ts.piece % kStoreBufs) * kStoreStageBytes;
   if (lane == 0) tma_store_wait_read_1();          // the store issued kStoreBufs pieces ago has read this buffer

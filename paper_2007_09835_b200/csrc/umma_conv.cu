@@ -269,7 +269,7 @@ conv3d_umma_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_consta
     __nv_bfloat16* yb = static_cast<__nv_bfloat16*>(a.y);
     const __nv_bfloat16* rb = static_cast<const __nv_bfloat16*>(a.residual);
     TmaStore ts{&ymap, store_smem + uint32_t(quad) * kStoreWarpBytes, 0, 0, 0, 0, 0u};
-    const PoolLanes pool_lanes{a.pool_w, a.pool_h, a.pool_t, a.sbw, a.sbh};
+    const PoolLanes pool_lanes = make_pool_lanes(a.pool_w, a.pool_h, a.pool_t, a.sbw, a.sbh, lane);
     const PoolLanes* pool = (a.pool_t * a.pool_h * a.pool_w > 1) ? &pool_lanes : nullptr;
     int r0 = quad * 32;                        // coordinates of the warp's first row inside the box
     const int bw_0 = r0 % a.box.bw; r0 /= a.box.bw;

@@ -149,7 +149,7 @@ conv3d_umma_smallc_kernel(const __grid_constant__ CUtensorMap xmap, const __grid
     const int bh_i = row / kSmallCTileW, bw_i = row % kSmallCTileW;
     __nv_bfloat16* yb = static_cast<__nv_bfloat16*>(a.y);
     TmaStore ts{&ymap, store_smem + uint32_t(quad) * kStoreWarpBytes, 0, 0, 0, 0, 0u};   // warp = 4 rows x 8 voxels
-    const PoolLanes pool_lanes{a.pool_w, a.pool_h, 1, kSmallCTileW, 4};
+    const PoolLanes pool_lanes = make_pool_lanes(a.pool_w, a.pool_h, 1, kSmallCTileW, 4, lane);
     const PoolLanes* pool = (a.pool_h * a.pool_w > 1) ? &pool_lanes : nullptr;
     uint32_t j = 0;
     for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++j) {
