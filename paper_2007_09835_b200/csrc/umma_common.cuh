@@ -71,6 +71,28 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, Barrier
   }
 }
 
+// Walk over a 4-digit mixed-radix index (digits i0 fastest .. i3 slowest, radices r0, r1, r2) that advances by a
+// constant step per iteration: the step is decomposed once, after that every advance is four adds with carries
+// instead of the three divisions a fresh decode costs.  i3 is unbounded.
+struct Walk4 {
+  int i0, i1, i2, i3;
+  int d0, d1, d2, d3;
+  int r0, r1, r2;
+};
+__device__ __forceinline__ void walk4_init(Walk4& k, int first, int step, int r0, int r1, int r2) {
+  k.r0 = r0; k.r1 = r1; k.r2 = r2;
+  int m = first;
+  k.i0 = m % r0; m /= r0; k.i1 = m % r1; m /= r1; k.i2 = m % r2; k.i3 = m / r2;
+  m = step;
+  k.d0 = m % r0; m /= r0; k.d1 = m % r1; m /= r1; k.d2 = m % r2; k.d3 = m / r2;
+}
+__device__ __forceinline__ void walk4_next(Walk4& k) {
+  k.i0 += k.d0; int c = k.i0 >= k.r0; k.i0 -= c * k.r0;
+  k.i1 += k.d1 + c; c = k.i1 >= k.r1; k.i1 -= c * k.r1;
+  k.i2 += k.d2 + c; c = k.i2 >= k.r2; k.i2 -= c * k.r2;
+  k.i3 += k.d3 + c;
+}
+
 // Pulls a tensor map (a kernel parameter) into the descriptor cache ahead of its first use.
 __device__ __forceinline__ void tma_prefetch_map(const CUtensorMap* map) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(map)) : "memory");
@@ -323,10 +345,13 @@ __device__ __forceinline__ void epilogue_piece_tma(const uint32_t* v, const floa
   uint4 o[4];
   __nv_bfloat162* po = reinterpret_cast<__nv_bfloat162*>(o);
 #pragma unroll
-  for (int q = 0; q < 16; ++q) {
-    float a = f[2 * q], b = f[2 * q + 1];
-    if (relu) { a = fmaxf(a, 0.f); b = fmaxf(b, 0.f); }
-    po[q] = __floats2bfloat162_rn(a, b);
+  for (int q = 0; q < 16; ++q) po[q] = __floats2bfloat162_rn(f[2 * q], f[2 * q + 1]);
+  // ReLU on the packed pairs: rounding is monotonic and keeps zero, so max(round(x), 0) = round(max(x, 0)), at
+  // half the instructions
+  if (relu) {
+    const __nv_bfloat162 zero2 = __floats2bfloat162_rn(0.f, 0.f);
+#pragma unroll
+    for (int q = 0; q < 16; ++q) po[q] = __hmax2(po[q], zero2);
   }
   // optional max-pool: after the (monotonic) activation and bf16 rounding, so it equals pooling the stored tensor
   int out_row = lane;

@@ -95,12 +95,10 @@ conv3d_umma_smallc_kernel(const __grid_constant__ CUtensorMap xmap, const __grid
     if (lane == 0 && a.n_pairs > 0) {
       int stage = 0;
       uint32_t phase = 0;
-      for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
-        int r = item;
-        const int iw = r % a.tiles_w; r /= a.tiles_w;
-        const int ih = r % a.tiles_h; r /= a.tiles_h;
-        const int to = r % a.g.To;
-        const int nn = r / a.g.To;
+      Walk4 k;
+      walk4_init(k, blockIdx.x, gridDim.x, a.tiles_w, a.tiles_h, a.g.To);
+      for (int item = blockIdx.x; item < n_items; item += gridDim.x, walk4_next(k)) {
+        const int iw = k.i0, ih = k.i1, to = k.i2, nn = k.i3;
         if (!mbar_wait(smem_u32(&bars->empty[stage]), phase ^ 1u, bars, err, 11)) break;
         const uint32_t full = smem_u32(&bars->full[stage]);
         mbar_expect_tx(full, uint32_t(a.n_phases * a.phase_bytes));
@@ -152,23 +150,24 @@ conv3d_umma_smallc_kernel(const __grid_constant__ CUtensorMap xmap, const __grid
     const PoolLanes pool_lanes = make_pool_lanes(a.pool_w, a.pool_h, 1, kSmallCTileW, 4, lane);
     const PoolLanes* pool = (a.pool_h * a.pool_w > 1) ? &pool_lanes : nullptr;
     uint32_t j = 0;
-    for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++j) {
-      int r = item;
-      const int iw = r % a.tiles_w; r /= a.tiles_w;
-      const int ih = r % a.tiles_h; r /= a.tiles_h;
-      const int to = r % a.g.To;
-      const int nn = r / a.g.To;
+    Walk4 k;
+    walk4_init(k, blockIdx.x, gridDim.x, a.tiles_w, a.tiles_h, a.g.To);
+    for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++j, walk4_next(k)) {
+      const int iw = k.i0, ih = k.i1, to = k.i2, nn = k.i3;
       const uint32_t buf = j & 1u;
       if (!mbar_wait(smem_u32(&bars->tmem_full[buf]), (j >> 1) & 1u, bars, err, 14)) break;
       tc_fence_after();
       const int ho = ih * kSmallCTileH + bh_i, wo = iw * kSmallCTileW + bw_i;
       const bool in_range = ho < a.g.Ho && wo < a.g.Wo;
-      const long long vox = (((long long)nn * a.g.To + to) * a.g.Ho + ho) * a.g.Wo + wo;
+      // the voxel's linear index is needed only by the direct-store paths and the residual (uniform condition)
+      const bool need_vox = a.residual != nullptr || !a.store_tma || (a.n_pad & 31);
+      const long long vox = need_vox ? (((long long)nn * a.g.To + to) * a.g.Ho + ho) * a.g.Wo + wo : 0;
       const uint32_t taddr = tmem_base + (uint32_t(quad * 32) << 16) + buf * uint32_t(a.n_pad);
       const __nv_bfloat16* res = (a.residual != nullptr && in_range)
                                      ? static_cast<const __nv_bfloat16*>(a.residual) + vox * a.rcs : nullptr;
       if (a.store_tma) {
-        ts.c1 = iw * kSmallCTileW / a.pool_w; ts.c2 = (ih * kSmallCTileH + quad * 4) / a.pool_h; ts.c3 = to; ts.c4 = nn;
+        // pooling windows are 1 or 2 wide: the division is a shift
+        ts.c1 = (iw * kSmallCTileW) >> (a.pool_w - 1); ts.c2 = (ih * kSmallCTileH + quad * 4) >> (a.pool_h - 1); ts.c3 = to; ts.c4 = nn;
         epilogue_row_tma(taddr, a.n_pad, a.n_pairs > 0, true, in_range, bias_s, a.g.relu, yb + vox * a.g.ycs, 0, a.g.M,
                          lane, ts, res, a.rcs, pool);
       } else {
