@@ -187,12 +187,17 @@ template <int NC>
 __device__ __forceinline__ void epilogue_cols(const uint32_t* v, const float* bias_s, int relu,
                                               __nv_bfloat16* dst, int valid, const __nv_bfloat16* res, int res_avail) {
   float f[NC];
-  const float4* b4 = reinterpret_cast<const float4*>(bias_s);      // 16-byte aligned by construction
+  if (bias_s != nullptr) {                                            // nullptr: the bias is in the accumulator already
+    const float4* b4 = reinterpret_cast<const float4*>(bias_s);      // 16-byte aligned by construction
 #pragma unroll
-  for (int k = 0; k < NC / 4; ++k) {
-    const float4 b = b4[k];
-    f[4 * k] = __uint_as_float(v[4 * k]) + b.x; f[4 * k + 1] = __uint_as_float(v[4 * k + 1]) + b.y;
-    f[4 * k + 2] = __uint_as_float(v[4 * k + 2]) + b.z; f[4 * k + 3] = __uint_as_float(v[4 * k + 3]) + b.w;
+    for (int k = 0; k < NC / 4; ++k) {
+      const float4 b = b4[k];
+      f[4 * k] = __uint_as_float(v[4 * k]) + b.x; f[4 * k + 1] = __uint_as_float(v[4 * k + 1]) + b.y;
+      f[4 * k + 2] = __uint_as_float(v[4 * k + 2]) + b.z; f[4 * k + 3] = __uint_as_float(v[4 * k + 3]) + b.w;
+    }
+  } else {
+#pragma unroll
+    for (int q = 0; q < NC; ++q) f[q] = __uint_as_float(v[q]);
   }
   if (res != nullptr) {
 #pragma unroll
@@ -250,8 +255,9 @@ __device__ __forceinline__ void epilogue_row(uint32_t taddr, int n_cols, bool ha
     }
     if (!in_range) continue;
     const __nv_bfloat16* res = res_row ? res_row + col : nullptr;
-    if (wide) epilogue_cols<32>(v, bias_s + m0, relu, dst + col, M - m0, res, res_pitch_left - col);
-    else epilogue_cols<16>(v, bias_s + m0, relu, dst + col, M - m0, res, res_pitch_left - col);
+    const float* bs = bias_s ? bias_s + m0 : nullptr;
+    if (wide) epilogue_cols<32>(v, bs, relu, dst + col, M - m0, res, res_pitch_left - col);
+    else epilogue_cols<16>(v, bs, relu, dst + col, M - m0, res, res_pitch_left - col);
   }
 }
 
@@ -321,12 +327,17 @@ __device__ __forceinline__ void epilogue_piece_tma(const uint32_t* v, const floa
                                                    TmaStore& ts, const __nv_bfloat16* res, int res_avail,
                                                    const PoolLanes* pool) {
   float f[32];
-  const float4* b4 = reinterpret_cast<const float4*>(bias_s);      // 16-byte aligned by construction
+  if (bias_s != nullptr) {                                            // nullptr: the bias is in the accumulator already
+    const float4* b4 = reinterpret_cast<const float4*>(bias_s);      // 16-byte aligned by construction
 #pragma unroll
-  for (int k = 0; k < 8; ++k) {
-    const float4 b = b4[k];
-    f[4 * k] = __uint_as_float(v[4 * k]) + b.x; f[4 * k + 1] = __uint_as_float(v[4 * k + 1]) + b.y;
-    f[4 * k + 2] = __uint_as_float(v[4 * k + 2]) + b.z; f[4 * k + 3] = __uint_as_float(v[4 * k + 3]) + b.w;
+    for (int k = 0; k < 8; ++k) {
+      const float4 b = b4[k];
+      f[4 * k] = __uint_as_float(v[4 * k]) + b.x; f[4 * k + 1] = __uint_as_float(v[4 * k + 1]) + b.y;
+      f[4 * k + 2] = __uint_as_float(v[4 * k + 2]) + b.z; f[4 * k + 3] = __uint_as_float(v[4 * k + 3]) + b.w;
+    }
+  } else {
+#pragma unroll
+    for (int q = 0; q < 32; ++q) f[q] = __uint_as_float(v[q]);
   }
   if (res != nullptr) {
 #pragma unroll
@@ -443,9 +454,9 @@ __device__ __forceinline__ void epilogue_row_tma(uint32_t taddr, int n_cols, boo
     }
     const __nv_bfloat16* res = (res_row && in_range) ? res_row + col : nullptr;
     if (wide) {
-      if (warp_rows_valid) epilogue_piece_tma(v, bias_s + m0, relu, m0, lane, ts, res, res_pitch_left - col, pool);
+      if (warp_rows_valid) epilogue_piece_tma(v, bias_s ? bias_s + m0 : nullptr, relu, m0, lane, ts, res, res_pitch_left - col, pool);
     } else if (in_range) {
-      epilogue_cols<16>(v, bias_s + m0, relu, dst + col, M - m0, res, res_pitch_left - col);
+      epilogue_cols<16>(v, bias_s ? bias_s + m0 : nullptr, relu, dst + col, M - m0, res, res_pitch_left - col);
     }
   }
 }

@@ -11,6 +11,8 @@
 // kernel locations (leading byte offset = distance between the two shifted windows).  So each pair
 // of kept kernel locations is one MMA, the input is read from L2 once per tile, and the layer is
 // bound by writing its output.  Kernel locations that no group keeps are not in the pair list.
+// The bias is one more MMA (a ones column times the bias as two bf16 terms): the kernel is bound by the
+// instruction count of its epilogue warps, and that removes a third of it.
 // With a spatial stride the input is staged as one image per stride phase (strided TMA boxes), so
 // that consecutive outputs are again consecutive voxels and every location a window of one image.
 //
@@ -35,7 +37,13 @@ conv3d_umma_smallc_kernel(const __grid_constant__ CUtensorMap xmap, const __grid
   const uint32_t base = store_smem + 4 * kStoreWarpBytes;
   const uint32_t w_bytes = uint32_t(a.n_pairs) * 2u * uint32_t(a.n_pad) * 16u;
   const uint32_t w_smem = base;                                         // weight image, whole layer
-  const uint32_t halo_smem = base + ((w_bytes + 127u) & ~127u);         // ring of staged halos
+  // The bias enters the accumulator through one more MMA instead of 32 additions per 32-channel piece in the
+  // epilogue (which is what bounds this kernel): B = one extra "pair" of the weight image whose k = 0 rows hold
+  // the bias split into two bf16 terms (high part + remainder: fp32 accuracy to about 2^-17), A = a single core
+  // matrix with ones in its k = 0 column that every 8-row group and both K halves read (strides 0).
+  const uint32_t bias_b_smem = w_smem + w_bytes;                        // [2 K halves][n_pad][8] bf16
+  const uint32_t ones_smem = bias_b_smem + 2u * uint32_t(a.n_pad) * 16u; // [8 rows][8] bf16
+  const uint32_t halo_smem = base + ((w_bytes + 2u * uint32_t(a.n_pad) * 16u + 128u + 127u) & ~127u);   // ring of staged halos
   const uint32_t halo_stride = (uint32_t(a.n_phases * a.phase_stride) + 127u) & ~127u;
   unsigned char* gen = smem_raw + (base - raw);
   int32_t* pair_smem = reinterpret_cast<int32_t*>(gen + (halo_smem - base) + kSmallCStages * halo_stride);
@@ -86,6 +94,21 @@ conv3d_umma_smallc_kernel(const __grid_constant__ CUtensorMap xmap, const __grid
     uint4* dst = reinterpret_cast<uint4*>(gen);
     for (uint32_t i = threadIdx.x; i < w_bytes / 16; i += blockDim.x) dst[i] = __ldg(src + i);
     for (int i = threadIdx.x; i < a.n_pairs * 2; i += blockDim.x) pair_smem[i] = __ldg(a.pair_off + i);
+    // bias operand and ones tile
+    __nv_bfloat16* bb = reinterpret_cast<__nv_bfloat16*>(gen + (bias_b_smem - base));
+    const int n8 = a.n_pad * 8;
+    for (int i = threadIdx.x; i < 2 * n8 + 64; i += blockDim.x) {
+      float val = 0.f;
+      if (i >= 2 * n8) {
+        val = ((i - 2 * n8) & 7) == 0 ? 1.f : 0.f;                    // ones tile: k = 0 column
+      } else if ((i & 7) == 0) {                                      // k = 0 of output channel m, K half i / n8
+        const int m = (i % n8) >> 3;
+        const float b = (a.bias != nullptr && m < a.g.M) ? __ldg(a.bias + m) : 0.f;
+        const float hi = __bfloat162float(__float2bfloat16_rn(b));
+        val = i < n8 ? hi : b - hi;
+      }
+      bb[i] = __float2bfloat16_rn(val);
+    }
   }
   // generic-proxy writes of the weight image must be visible to the tensor core (async proxy)
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -136,6 +159,7 @@ conv3d_umma_smallc_kernel(const __grid_constant__ CUtensorMap xmap, const __grid
           const uint64_t bdesc = smem_desc_noswizzle(w_smem + uint32_t(p) * 2u * lbo_b, lbo_b, 128u);
           umma_bf16(d_tmem, adesc, bdesc, idesc, p ? 1u : 0u);
         }
+        umma_bf16(d_tmem, smem_desc_noswizzle(ones_smem, 0u, 0u), smem_desc_noswizzle(bias_b_smem, lbo_b, 128u), idesc, 1u);
         umma_commit(smem_u32(&bars->empty[stage]));
         umma_commit(smem_u32(&bars->tmem_full[buf]));
         if (++stage == kSmallCStages) { stage = 0; phase ^= 1u; }
@@ -148,6 +172,7 @@ conv3d_umma_smallc_kernel(const __grid_constant__ CUtensorMap xmap, const __grid
     __nv_bfloat16* yb = static_cast<__nv_bfloat16*>(a.y);
     TmaStore ts{&ymap, store_smem + uint32_t(quad) * kStoreWarpBytes, 0, 0, 0, 0, 0u};   // warp = 4 rows x 8 voxels
     const PoolLanes pool_lanes = make_pool_lanes(a.pool_w, a.pool_h, 1, kSmallCTileW, 4, lane);
+    const float* bias_e = a.n_pairs > 0 ? nullptr : bias_s;   // with MMAs the bias is in the accumulator already
     const PoolLanes* pool = (a.pool_h * a.pool_w > 1) ? &pool_lanes : nullptr;
     uint32_t j = 0;
     Walk4 k;
@@ -168,10 +193,10 @@ conv3d_umma_smallc_kernel(const __grid_constant__ CUtensorMap xmap, const __grid
       if (a.store_tma) {
         // pooling windows are 1 or 2 wide: the division is a shift
         ts.c1 = (iw * kSmallCTileW) >> (a.pool_w - 1); ts.c2 = (ih * kSmallCTileH + quad * 4) >> (a.pool_h - 1); ts.c3 = to; ts.c4 = nn;
-        epilogue_row_tma(taddr, a.n_pad, a.n_pairs > 0, true, in_range, bias_s, a.g.relu, yb + vox * a.g.ycs, 0, a.g.M,
+        epilogue_row_tma(taddr, a.n_pad, a.n_pairs > 0, true, in_range, bias_e, a.g.relu, yb + vox * a.g.ycs, 0, a.g.M,
                          lane, ts, res, a.rcs, pool);
       } else {
-        epilogue_row(taddr, a.n_pad, a.n_pairs > 0, in_range, bias_s, a.g.relu, yb + vox * a.g.ycs, 0, a.g.M, res, a.rcs);
+        epilogue_row(taddr, a.n_pad, a.n_pairs > 0, in_range, bias_e, a.g.relu, yb + vox * a.g.ycs, 0, a.g.M, res, a.rcs);
       }
       tc_fence_before();
       __syncwarp();
@@ -195,7 +220,7 @@ conv3d_umma_smallc_kernel(const __grid_constant__ CUtensorMap xmap, const __grid
 }  // namespace
 
 size_t smallc_smem_bytes(int n_pairs, int n_pad, int stage_bytes) {
-  const size_t w = (size_t(n_pairs) * 2 * n_pad * 16 + 127) & ~size_t(127);
+  const size_t w = (size_t(n_pairs + 1) * 2 * n_pad * 16 + 128 + 127) & ~size_t(127);   // + bias operand and ones tile
   const size_t halo = (size_t(stage_bytes) + 127) & ~size_t(127);
   return 1024 + 4 * kStoreWarpBytes + w + kSmallCStages * halo + ((size_t(n_pairs) * 8 + 15) & ~size_t(15)) + sizeof(Barriers) + 16 + size_t(n_pad) * 4;
 }

@@ -146,6 +146,25 @@ def test_small_cin_padding_channels():
     assert torch.equal(y0, y2)
 
 
+def test_small_cin_bias_enters_through_the_accumulator():
+    """The first-layer kernel adds the bias by one extra MMA (bias split into two bf16 terms) instead of in the
+    epilogue.  The usual synthetic bias is too small for the layer tolerance to notice a wrong one, so: a bias
+    of order 3 with full fp32 mantissas over a weak convolution; the result must be within half a bf16 step
+    of the oracle's."""
+    for cout, stride in ((64, (1, 1, 1)), (45, (1, 2, 2)), (24, (1, 1, 1))):
+        spec = synth.ConvSpec("c1", 3, cout, (3, 3, 3), stride, (1, 1, 1), False)
+        L = synth.make_layer(spec, 2, 31, 4, 4, "bernoulli", 0.5)
+        bias = (np.random.default_rng(31).standard_normal(cout) * 3.0).astype(np.float32)
+        w = (L["w"] * 0.01).astype(np.float32)
+        x = synth.make_input(731, (2, 4, 32, 24, 3))
+        ref = oracle.conv3d(x, w, L["mask"], bias, stride, (1, 1, 1), False, round_bf16=True)
+        lay = nets.ConvLayer(spec, w, bias, L["mask"], 4, 4, torch.bfloat16)
+        y = nets.to_numpy(lay(nets.to_device(x), x_pad_zero=True), cout)
+        assert rt3d.rt3d_last_plan()["kernel"] == 3
+        assert rt3d.rt3d_last_device_status() == rt3d.OK
+        assert np.abs(y - ref).max() <= np.abs(ref).max() * 2.0 ** -8, (cout, stride)
+
+
 def test_small_cin_all_pruned_outputs_bias():
     spec = synth.ConvSpec("c", 3, 32, (3, 3, 3), (1, 1, 1), (1, 1, 1), False)
     L = synth.make_layer(spec, 7, 4, 4, 4, "bernoulli", 0.5)
