@@ -256,9 +256,14 @@ rt3d_status rt3d_conv3d_sparse_noalloc(const rt3d_tensor* x, const rt3d_packed* 
 /*
  * rt3d_conv3d_host - end-to-end variant: x->data and y->data are HOST buffers (pinned
  * memory recommended), bias is HOST [M] or NULL.  Copies x to a library-owned device staging
- * buffer, runs rt3d_conv3d_sparse (or _dense for a dense handle) and copies y back, all on
- * `stream`; returns after the stream has been synchronised.  Staging buffers are cached
- * in the handle and grow on demand.
+ * buffer, runs rt3d_conv3d_sparse (or _dense for a dense handle) and copies y back; the work is
+ * ordered after what `stream` holds on entry, and the call returns after the stream has been
+ * synchronised.  Batches of at least two clips and 8 MiB go through in up to eight chunks of whole
+ * clips (clips are independent), with the copies of neighbouring chunks on two internal streams, so
+ * that copy-in, convolution and copy-out overlap; each chunk is one rt3d_conv3d_sparse call, so the
+ * result agrees with a single call on the whole batch within the library's tolerance (the K split, and
+ * with it the fp32 summation order, may differ), not necessarily bit for bit.  Staging buffers, streams
+ * and events are cached in the handle (one call at a time per handle).
  */
 rt3d_status rt3d_conv3d_host(const rt3d_tensor* x, rt3d_packed* w, const float* bias,
                              const rt3d_conv_params* p, rt3d_tensor* y, void* stream);

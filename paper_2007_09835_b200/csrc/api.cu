@@ -765,17 +765,75 @@ rt3d_status rt3d_conv3d_host(const rt3d_tensor* x, rt3d_packed* w, const float* 
       return RT3D_ERR_ALLOC;
   }
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  if (cudaMemcpyAsync(blob->stage_x, x->data, xb, cudaMemcpyHostToDevice, st) != cudaSuccess) return RT3D_ERR_CUDA;
   if (bias && cudaMemcpyAsync(blob->stage_bias, bias, size_t(w->M) * 4, cudaMemcpyHostToDevice, st) != cudaSuccess)
     return RT3D_ERR_CUDA;
-  rt3d_tensor xd = *x, yd = *y;
-  xd.data = blob->stage_x;
-  yd.data = blob->stage_y;
-  s = conv_impl(&xd, w, bias ? blob->stage_bias : nullptr, p, &yd, stream, w->is_dense != 0);
-  if (s != RT3D_OK) return s;
-  if (cudaMemcpyAsync(y->data, blob->stage_y, yb, cudaMemcpyDeviceToHost, st) != cudaSuccess) return RT3D_ERR_CUDA;
-  if (cudaStreamSynchronize(st) != cudaSuccess) return RT3D_ERR_CUDA;
-  return RT3D_OK;
+  const float* bias_d = bias ? blob->stage_bias : nullptr;
+  // Clips are independent, so a large batch goes through in up to eight chunks of whole clips: chunk k+1 is
+  // copied in on one stream while chunk k is convolved on the caller's stream and chunk k-1 is copied out on a
+  // third (PCIe is full duplex; the call is bound by the larger of the two copies instead of their sum).
+  constexpr int kHostChunks = 8;
+  const int n_chunks = (x->n >= 2 && xb + yb >= (size_t(8) << 20)) ? (x->n < kHostChunks ? x->n : kHostChunks) : 1;
+  if (n_chunks == 1) {
+    if (cudaMemcpyAsync(blob->stage_x, x->data, xb, cudaMemcpyHostToDevice, st) != cudaSuccess) return RT3D_ERR_CUDA;
+    rt3d_tensor xd = *x, yd = *y;
+    xd.data = blob->stage_x;
+    yd.data = blob->stage_y;
+    s = conv_impl(&xd, w, bias_d, p, &yd, stream, w->is_dense != 0);
+    if (s != RT3D_OK) return s;
+    if (cudaMemcpyAsync(y->data, blob->stage_y, yb, cudaMemcpyDeviceToHost, st) != cudaSuccess) return RT3D_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return RT3D_ERR_CUDA;
+    return RT3D_OK;
+  }
+  {
+    std::lock_guard<std::mutex> lock(w->mu);
+    for (void*& hs : blob->host_streams)
+      if (!hs) {
+        cudaStream_t ns;
+        if (cudaStreamCreateWithFlags(&ns, cudaStreamNonBlocking) != cudaSuccess) return RT3D_ERR_CUDA;
+        hs = ns;
+      }
+    for (void*& he : blob->host_events)
+      if (!he) {
+        cudaEvent_t ne;
+        if (cudaEventCreateWithFlags(&ne, cudaEventDisableTiming) != cudaSuccess) return RT3D_ERR_CUDA;
+        he = ne;
+      }
+  }
+  cudaStream_t s_in = static_cast<cudaStream_t>(blob->host_streams[0]);
+  cudaStream_t s_out = static_cast<cudaStream_t>(blob->host_streams[1]);
+  auto ev = [&](int i) { return static_cast<cudaEvent_t>(blob->host_events[i]); };
+  const size_t es = elem_size(x->dtype);
+  const size_t x_clip = size_t(x->t) * x->h * x->w * x->c_stride * es, y_clip = size_t(y->t) * y->h * y->w * y->c_stride * es;
+  bool cuda_ok = cudaEventRecord(ev(0), st) == cudaSuccess && cudaStreamWaitEvent(s_in, ev(0), 0) == cudaSuccess &&
+                 cudaStreamWaitEvent(s_out, ev(0), 0) == cudaSuccess;
+  rt3d_status cs = RT3D_OK;
+  int n0 = 0;
+  for (int k = 0; k < n_chunks && cuda_ok && cs == RT3D_OK; ++k) {
+    const int n1 = int((long long)x->n * (k + 1) / n_chunks), nc = n1 - n0;
+    const size_t xo = size_t(n0) * x_clip, yo = size_t(n0) * y_clip;
+    const size_t xn = n1 == x->n ? xb - xo : size_t(nc) * x_clip, yn = n1 == x->n ? yb - yo : size_t(nc) * y_clip;
+    cuda_ok = cudaMemcpyAsync(static_cast<char*>(blob->stage_x) + xo, static_cast<const char*>(x->data) + xo, xn,
+                              cudaMemcpyHostToDevice, s_in) == cudaSuccess &&
+              cudaEventRecord(ev(1 + k), s_in) == cudaSuccess && cudaStreamWaitEvent(st, ev(1 + k), 0) == cudaSuccess;
+    if (!cuda_ok) break;
+    rt3d_tensor xd = *x, yd = *y;
+    xd.n = nc; yd.n = nc;
+    xd.data = static_cast<char*>(blob->stage_x) + xo;
+    yd.data = static_cast<char*>(blob->stage_y) + yo;
+    cs = conv_impl(&xd, w, bias_d, p, &yd, stream, w->is_dense != 0);
+    if (cs != RT3D_OK) break;
+    cuda_ok = cudaEventRecord(ev(1 + kHostChunks + k), st) == cudaSuccess &&
+              cudaStreamWaitEvent(s_out, ev(1 + kHostChunks + k), 0) == cudaSuccess &&
+              cudaMemcpyAsync(static_cast<char*>(y->data) + yo, static_cast<char*>(blob->stage_y) + yo, yn,
+                              cudaMemcpyDeviceToHost, s_out) == cudaSuccess;
+    n0 = n1;
+  }
+  // the caller's stream ends up behind everything this call enqueued, whatever happened
+  const bool joined = cudaEventRecord(ev(17), s_out) == cudaSuccess && cudaStreamWaitEvent(st, ev(17), 0) == cudaSuccess &&
+                      cudaEventRecord(ev(0), s_in) == cudaSuccess && cudaStreamWaitEvent(st, ev(0), 0) == cudaSuccess;
+  const bool synced = cudaStreamSynchronize(st) == cudaSuccess;
+  if (cs != RT3D_OK) return cs;
+  return (cuda_ok && joined && synced) ? RT3D_OK : RT3D_ERR_CUDA;
 }
 
 rt3d_status rt3d_packed_prepare(rt3d_packed* p) {
@@ -802,6 +860,8 @@ void rt3d_packed_free(rt3d_packed* p) {
     cudaFree(b->group_ptr); cudaFree(b->pos_idx); cudaFree(b->tiles);
     for (auto& kv : b->umma) { cudaFree(kv.second.wtiles); cudaFree(kv.second.step_ptr); cudaFree(kv.second.steps); }
     cudaFree(b->stage_x); cudaFree(b->stage_y); cudaFree(b->stage_bias);
+    for (void* hs : b->host_streams) if (hs) cudaStreamDestroy(static_cast<cudaStream_t>(hs));
+    for (void* he : b->host_events) if (he) cudaEventDestroy(static_cast<cudaEvent_t>(he));
     for (auto& kv : b->smallc) { cudaFree(kv.second.wimg); cudaFree(kv.second.pairs); }
     cudaFree(b->splitk); cudaFree(b->splitk_cnt);
     delete b;

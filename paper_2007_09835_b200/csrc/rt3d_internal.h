@@ -83,6 +83,10 @@ struct DeviceBlob {
   void* stage_x = nullptr; size_t stage_x_bytes = 0;   // staging for rt3d_conv3d_host
   void* stage_y = nullptr; size_t stage_y_bytes = 0;
   float* stage_bias = nullptr;
+  // rt3d_conv3d_host pipelines a large batch in chunks: copy-in and copy-out streams and events
+  // (cudaStream_t / cudaEvent_t, created on first use)
+  void* host_streams[2] = {nullptr, nullptr};
+  void* host_events[18] = {};
 };
 
 }  // namespace rt3d

@@ -419,6 +419,28 @@ def test_conv3d_host_entry_point_matches_device_call():
     assert torch.equal(yh, yd.cpu())
 
 
+def test_conv3d_host_entry_point_pipelines_large_batches_in_chunks():
+    """Above 8 MiB the host entry point copies, convolves and copies back chunks of whole clips on three
+    streams.  Every output element must arrive, in the right place (11 clips = chunks of one or two clips)."""
+    spec = synth.ConvSpec("h", 64, 128, (3, 3, 3), (1, 1, 1), (1, 1, 1), True)
+    L = synth.make_layer(spec, 7, 10, 4, 4, "bernoulli", 0.4)
+    x = synth.make_input(710, (11, 4, 28, 28, 64))
+    lay = nets.ConvLayer(spec, L["w"], L["bias"], L["mask"], 4, 4, torch.bfloat16)
+    yd = lay(nets.to_device(x)).cpu().float()
+    xh = torch.from_numpy(x).to(torch.bfloat16).pin_memory()
+    yh = torch.full((11, 4, 28, 28, 128), 55.0, dtype=torch.bfloat16).pin_memory()
+    bh = torch.from_numpy(L["bias"]).pin_memory()
+    launches = rt3d.rt3d_launch_count()
+    for _ in range(2):                                   # the second call reuses streams, events and staging
+        rt3d.rt3d_conv3d_host(rt3d.tensor_desc(xh), lay.packed, bh, rt3d.tensor_desc(yh), spec.stride, spec.pad, True)
+    assert rt3d.rt3d_launch_count() - launches == 16     # eight chunks per call
+    assert rt3d.rt3d_last_device_status() == rt3d.OK
+    assert (yd != 0).float().mean() > 0.1
+    assert (yh.float() - yd).abs().max() <= 1e-2 * yd.abs().max()
+    ref0 = oracle.conv3d(x[10:], L["w"], L["mask"], L["bias"], spec.stride, spec.pad, True, round_bf16=True)
+    check(yh[10:].float().numpy(), ref0, torch.bfloat16, "host path, last clip")
+
+
 def test_maxpool_and_add_relu_against_oracle():
     for dtype in (torch.bfloat16, torch.float32):
         for c, shape, pool in ((64, (2, 4, 8, 8), synth.PoolSpec("p", (2, 2, 2), (2, 2, 2), (0, 0, 0))),
