@@ -155,9 +155,27 @@ conv3d_umma_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_consta
 
   // Everything above touched only shared memory, barriers and TMEM.  The successor may be scheduled now that
   // this CTA holds its TMEM columns (a successor CTA that shared the SM and allocated first could otherwise
-  // starve this one while waiting for it); global memory from here on.
+  // starve this one while waiting for it).
   pdl_launch();
-  pdl_wait();
+  // Work that needs none of the predecessor's results is done while the CTA still waits for it: every thread
+  // decodes the CTA's first item (a chain of integer divisions: half a microsecond in the single producer
+  // thread) and reads that item's bounds in the step list, the producer also its first encoded steps.  The
+  // step lists belong to the packed handle, which no kernel writes; after the wait these reads are two
+  // dependent trips to L2 in front of the first TMA request of a layer that takes 4 to 10 us in all.
+  // (Only registers survive the wait: a plain prefetch into L1 did not help.)
+  constexpr int kPreSteps = 4;
+  ItemCoord pre_c = {};
+  int pre_sbegin = 0, pre_nsteps = 0, pre_local0 = 0, pre_enc[kPreSteps] = {0, 0, 0, 0};
+  if (int(blockIdx.x) < n_items) {
+    pre_c = decode_item(a, blockIdx.x, n_mtiles);
+    item_steps<kDense>(a, pre_c, pre_sbegin, pre_nsteps, pre_local0);
+    if (!kDense && threadIdx.x == 0) {
+#pragma unroll
+      for (int q = 0; q < kPreSteps; ++q)
+        if (q < pre_nsteps) pre_enc[q] = __ldg(a.steps + pre_sbegin + q);
+    }
+  }
+  pdl_wait();                                    // predecessor complete: activations, bias, residual are visible
   if (warp >= 2) {                               // epilogue warps stage the bias; the other roles start at once
     for (int i = threadIdx.x - 64; i < a.n_bundles * a.n_tile; i += 128)
       bias_s[i] = (a.bias != nullptr && i < a.g.M) ? __ldg(a.bias + i) : 0.f;
@@ -172,9 +190,10 @@ conv3d_umma_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_consta
       bool ok = true;
       const uint32_t tx_bytes = uint32_t(box_rows) * 128u + b_bytes;
       for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
-        const ItemCoord c = decode_item(a, item, n_mtiles);
-        int s_begin, nsteps, local0;
-        item_steps<kDense>(a, c, s_begin, nsteps, local0);
+        const bool first_item = item == int(blockIdx.x);                // decoded before the dependency wait
+        const ItemCoord c = first_item ? pre_c : decode_item(a, item, n_mtiles);
+        int s_begin = pre_sbegin, nsteps = pre_nsteps, local0 = pre_local0;
+        if (!first_item) item_steps<kDense>(a, c, s_begin, nsteps, local0);
         const int wq = c.w0 * a.g.sw - a.g.pw, hq = c.h0 * a.g.sh - a.g.ph, tq = c.t0 * a.g.st - a.g.pt;
         // Everything a step needs is computed (dense) or fetched one step ahead (indexed) before the
         // wait on the stage, so a freed stage is re-armed without further latency.
@@ -195,7 +214,14 @@ conv3d_umma_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_consta
               c_ch[q] = ch * 64; c_w[q] = wq + kw; c_h[q] = hq + kh; c_t[q] = tq + kt;
               if (++ch == a.n_chunks) { ch = 0; if (++kw == a.g.Kw) { kw = 0; if (++kh == a.g.Kh) { kh = 0; ++kt; } } }
             } else {
-              const int enc = __ldg(a.steps + s_begin + i + q);
+              int enc;
+              if (first_item && i + q < kPreSteps) {             // kDense is false here
+                enc = pre_enc[0];
+#pragma unroll
+                for (int e = 1; e < kPreSteps; ++e) enc = (i + q == e) ? pre_enc[e] : enc;
+              } else {
+                enc = __ldg(a.steps + s_begin + i + q);
+              }
               c_t[q] = tq + ((enc >> 24) & 63); c_h[q] = hq + ((enc >> 18) & 63); c_w[q] = wq + ((enc >> 12) & 63);
               c_ch[q] = (enc & 4095) * 64;
             }
@@ -224,9 +250,10 @@ conv3d_umma_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_consta
       int stage = 0;
       bool ok = true, ready = false;
       for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++j) {
-        const ItemCoord c = decode_item(a, item, n_mtiles);
-        int s_begin, nsteps, local0;
-        item_steps<kDense>(a, c, s_begin, nsteps, local0);
+        const bool first_item = item == int(blockIdx.x);
+        const ItemCoord c = first_item ? pre_c : decode_item(a, item, n_mtiles);
+        int s_begin = pre_sbegin, nsteps = pre_nsteps, local0 = pre_local0;
+        if (!first_item) item_steps<kDense>(a, c, s_begin, nsteps, local0);
         const uint32_t buf = j & 1u;
         if (!mbar_wait(smem_u32(&bars->tmem_empty[buf]), ((j >> 1) & 1u) ^ 1u, bars, err, 2)) break;
         tc_fence_after();
@@ -279,9 +306,10 @@ conv3d_umma_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_consta
     const size_t part_tile = size_t(128) * a.n_tile;       // floats per partial tile
     uint32_t j = 0;
     for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++j) {
-      const ItemCoord c = decode_item(a, item, n_mtiles);
-      int s_begin, nsteps, local0;
-      item_steps<kDense>(a, c, s_begin, nsteps, local0);
+      const bool first_item = item == int(blockIdx.x);
+      const ItemCoord c = first_item ? pre_c : decode_item(a, item, n_mtiles);
+      int s_begin = pre_sbegin, nsteps = pre_nsteps, local0 = pre_local0;
+      if (!first_item) item_steps<kDense>(a, c, s_begin, nsteps, local0);
       const uint32_t buf = j & 1u;
       if (!mbar_wait(smem_u32(&bars->tmem_full[buf]), (j >> 1) & 1u, bars, err, 4)) break;
       tc_fence_after();
