@@ -104,8 +104,15 @@ __device__ __forceinline__ void reduce_partial_row(const float* part0, size_t sp
 
 // kCps: K steps per pipeline stage (and per barrier hand-shake): 1, or 2 for narrow bundles, where the
 // issuing thread's hand-shake, not the tensor pipe, bounds a step.
+// Threads of the single-CTA kernel: producer warp, MMA warp, two sets of four epilogue warps.  The second set
+// works only on plain (unsplit, unpooled) calls, where it takes the odd 32-column pieces of a tile and stores
+// them directly: most layers that run here give a CTA a single tile, so the epilogue is a pure latency chain
+// of up to eight pieces per warp, and sharing it between two warps per lane quadrant halves the tail of the
+// layer.
+constexpr int kThreadsSingle = 320;
+
 template <bool kDense, int kCps>
-__global__ void __launch_bounds__(kThreadsUmma, 1)
+__global__ void __launch_bounds__(kThreadsSingle, 1)
 conv3d_umma_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CUtensorMap wmap,
                    const __grid_constant__ CUtensorMap ymap, const UmmaArgs a, const int stages, const int tmem_cols) {
   extern __shared__ unsigned char smem_raw[];
@@ -124,6 +131,7 @@ conv3d_umma_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_consta
   const int n_mtiles = a.tiles_n * a.tiles_t * a.tiles_h * a.tiles_w;
   const int n_items = n_mtiles * a.n_bundles * a.n_splits;
   const int box_rows = a.box.bn * a.box.bt * a.box.bh * a.box.bw;
+  const bool two_sets = a.n_splits == 1 && a.pool_t * a.pool_h * a.pool_w == 1;   // both epilogue warp sets work
 
   if (threadIdx.x == 32) {                     // descriptor fetches overlap the rest of the set-up
     tma_prefetch_map(&xmap);
@@ -137,7 +145,7 @@ conv3d_umma_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_consta
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(smem_u32(&bars->tmem_full[b]), 1);
-      mbar_init(smem_u32(&bars->tmem_empty[b]), 4);
+      mbar_init(smem_u32(&bars->tmem_empty[b]), two_sets ? 8 : 4);
     }
     bars->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -177,9 +185,9 @@ conv3d_umma_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_consta
   }
   pdl_wait();                                    // predecessor complete: activations, bias, residual are visible
   if (warp >= 2) {                               // epilogue warps stage the bias; the other roles start at once
-    for (int i = threadIdx.x - 64; i < a.n_bundles * a.n_tile; i += 128)
+    for (int i = threadIdx.x - 64; i < a.n_bundles * a.n_tile; i += 256)
       bias_s[i] = (a.bias != nullptr && i < a.g.M) ? __ldg(a.bias + i) : 0.f;
-    epilogue_bar_sync(128);
+    epilogue_bar_sync(256);
   }
 
   if (warp == 0) {
@@ -284,9 +292,10 @@ conv3d_umma_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_consta
         else mbar_arrive(smem_u32(&bars->tmem_full[buf]));
       }
     }
-  } else {
-    // ------------------------------------------------------------------ epilogue (warps 2..5)
+  } else if (warp < 6 || two_sets) {
+    // ------------------------------------------------------------------ epilogue (warps 2..5, and 6..9 on plain calls)
     const int quad = warp & 3;                 // TMEM lane quadrant this warp may read
+    const int half = (warp - 2) >> 2;          // second set: odd pieces, direct stores
     const int row = quad * 32 + lane;          // voxel row inside the box
     int r = row;
     const int bw_i = r % a.box.bw; r /= a.box.bw;
@@ -321,7 +330,32 @@ conv3d_umma_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_consta
       __nv_bfloat16* dst = yb + vox * a.g.ycs + m_base;
       const __nv_bfloat16* res = (rb != nullptr && in_range) ? rb + vox * a.rcs + m_base : nullptr;
       const int res_left = a.rcs - m_base;
-      if (a.n_splits == 1) {
+      if (two_sets) {
+        ts.c1 = c.w0 + bw_0; ts.c2 = c.h0 + bh_0; ts.c3 = c.t0 + bt_0; ts.c4 = c.n0 + bn_0;
+        for (int col = half * 32; col < a.n_tile; col += 64) {
+          const int m0 = m_base + col;
+          if (m0 >= a.g.M) break;
+          uint32_t v[32];
+          const bool wide = col + 32 <= a.n_tile;
+          if (nsteps > 0) {
+            if (wide) tmem_ld32(taddr + col, v);
+            else tmem_ld16_into32(taddr + col, v);
+          } else {
+#pragma unroll
+            for (int q = 0; q < 32; ++q) v[q] = 0u;
+          }
+          const __nv_bfloat16* rp = res ? res + col : nullptr;
+          if (half == 0 && wide && a.store_tma) {
+            if (quad * 32 < box_rows) epilogue_piece_tma(v, bias_s + m0, a.g.relu, m0, lane, ts, rp, res_left - col, nullptr);
+          } else if (in_range) {
+            if (wide) epilogue_cols<32>(v, bias_s + m0, a.g.relu, dst + col, a.g.M - m0, rp, res_left - col);
+            else epilogue_cols<16>(v, bias_s + m0, a.g.relu, dst + col, a.g.M - m0, rp, res_left - col);
+          }
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&bars->tmem_empty[buf]));
+      } else if (a.n_splits == 1) {
         if (a.store_tma) {
           ts.c1 = (c.w0 + bw_0) / a.pool_w; ts.c2 = (c.h0 + bh_0) / a.pool_h; ts.c3 = (c.t0 + bt_0) / a.pool_t; ts.c4 = c.n0 + bn_0;
           epilogue_row_tma(taddr, a.n_tile, nsteps > 0, quad * 32 < box_rows, in_range, bias_s, a.g.relu, dst, m_base,
@@ -388,7 +422,7 @@ cudaError_t launch_single_t(const UmmaArgs& a, const CUtensorMap& xm, const CUte
     if (e != cudaSuccess) return e;
     attr_done = true;
   }
-  LaunchSetup ls(dim3(grid), dim3(kThreadsUmma), smem, stream);
+  LaunchSetup ls(dim3(grid), dim3(kThreadsSingle), smem, stream);
   return cudaLaunchKernelEx(&ls.cfg, conv3d_umma_kernel<kDense, kCps>, xm, wm, ym, a, stages, cols);
 }
 
