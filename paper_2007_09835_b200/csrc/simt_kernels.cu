@@ -190,6 +190,69 @@ __global__ void maxpool3d_bf16x8_win_kernel(const uint4* __restrict__ x, int t, 
   y[((((long long)nn * To + to) * Ho + ho) * Wo + wo) * ycs8 + cc] = out;
 }
 
+// Unit stride along w: a thread produces WB consecutive outputs of one image row.  The windows of neighbouring
+// outputs share KW - 1 columns, so the (t, h) maximum of each of the WB + KW - 1 input columns is formed once and
+// every output is the maximum of KW adjacent column maxima: (WB + KW - 1) * KT * KH loads for WB outputs instead
+// of WB * KT * KH * KW (a 3x3x3 stride-1 pool is bound by L1 bandwidth: 27 loads of 16 bytes per 16 bytes written).
+template <int KT, int KH, int KW, int WB>
+__global__ void maxpool3d_bf16x8_row_kernel(const uint4* __restrict__ x, int t, int h, int w, int c8, int xcs8,
+                                            int st, int sh, int pt, int ph, int pw,
+                                            uint4* __restrict__ y, int To, int Ho, int Wo, int ycs8, int w_blocks, long long total) {
+  pdl_entry();
+  const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= total) return;
+  const int cc = int(idx % c8);
+  long long r = idx / c8;
+  const int wb = int(r % w_blocks); r /= w_blocks;
+  const int ho = int(r % Ho); r /= Ho;
+  const int to = int(r % To);
+  const int nn = int(r / To);
+  const int t0 = to * st - pt, h0 = ho * sh - ph, w0 = wb * WB - pw;
+  const __nv_bfloat162 ninf = __float2bfloat162_rn(-INFINITY);
+  __nv_bfloat162 cm[WB + KW - 1][4];
+#pragma unroll
+  for (int d = 0; d < WB + KW - 1; ++d) {
+    const int wi = w0 + d;
+    const bool w_in = wi >= 0 && wi < w;
+    const int wc = min(max(wi, 0), w - 1);
+    uint4 v[KT * KH];
+    bool ok[KT * KH];
+#pragma unroll
+    for (int a = 0; a < KT; ++a)
+#pragma unroll
+      for (int b = 0; b < KH; ++b) {
+        const int ti = t0 + a, hi = h0 + b;
+        ok[a * KH + b] = w_in && ti >= 0 && ti < t && hi >= 0 && hi < h;
+        const int tc = min(max(ti, 0), t - 1), hc = min(max(hi, 0), h - 1);
+        v[a * KH + b] = __ldg(x + ((((long long)nn * t + tc) * h + hc) * w + wc) * xcs8 + cc);
+      }
+#pragma unroll
+    for (int k = 0; k < 4; ++k) cm[d][k] = ninf;
+#pragma unroll
+    for (int i = 0; i < KT * KH; ++i) {
+      const __nv_bfloat162* pv = reinterpret_cast<const __nv_bfloat162*>(&v[i]);
+#pragma unroll
+      for (int k = 0; k < 4; ++k) cm[d][k] = ok[i] ? __hmax2(cm[d][k], pv[k]) : cm[d][k];
+    }
+  }
+  uint4* yrow = y + ((((long long)nn * To + to) * Ho + ho) * Wo) * ycs8 + cc;
+#pragma unroll
+  for (int j = 0; j < WB; ++j) {
+    const int wo = wb * WB + j;
+    if (wo >= Wo) break;
+    uint4 out;
+    __nv_bfloat162* po = reinterpret_cast<__nv_bfloat162*>(&out);
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      __nv_bfloat162 m = cm[j][k];
+#pragma unroll
+      for (int d = 1; d < KW; ++d) m = __hmax2(m, cm[j + d][k]);
+      po[k] = m;
+    }
+    yrow[(long long)wo * ycs8] = out;
+  }
+}
+
 // bf16, 8 channels (16 bytes) per thread; needs c % 8 == 0 and 8-element pitches.
 __global__ void maxpool3d_bf16x8_kernel(const uint4* __restrict__ x, int t, int h, int w, int c8, int xcs8,
                                         int kt, int kh, int kw, int st, int sh, int sw, int pt, int ph, int pw,
@@ -286,6 +349,16 @@ cudaError_t launch_maxpool3d(int dtype, const void* x, int n, int t, int h, int 
   if (dtype == 1 && c % 8 == 0 && xcs % 8 == 0 && ycs % 8 == 0) {
     const long long total = vox * (c / 8);
     LaunchSetup ls(dim3((unsigned)((total + threads - 1) / threads)), dim3(threads), 0, stream);
+    if (sw == 1 && kw == 3 && kh == 3 && (kt == 3 || kt == 1) && Wo >= 4) {       // unit stride along w: shared column maxima
+      const int w_blocks = (Wo + 3) / 4;
+      const long long total_r = (long long)n * To * Ho * w_blocks * (c / 8);
+      LaunchSetup lr(dim3((unsigned)((total_r + threads - 1) / threads)), dim3(threads), 0, stream);
+      if (kt == 3)
+        return cudaLaunchKernelEx(&lr.cfg, maxpool3d_bf16x8_row_kernel<3, 3, 3, 4>, static_cast<const uint4*>(x), t, h, w, c / 8,
+                                  xcs / 8, st, sh, pt, ph, pw, static_cast<uint4*>(y), To, Ho, Wo, ycs / 8, w_blocks, total_r);
+      return cudaLaunchKernelEx(&lr.cfg, maxpool3d_bf16x8_row_kernel<1, 3, 3, 4>, static_cast<const uint4*>(x), t, h, w, c / 8,
+                                xcs / 8, st, sh, pt, ph, pw, static_cast<uint4*>(y), To, Ho, Wo, ycs / 8, w_blocks, total_r);
+    }
 #define RT3D_POOL_WIN(KT_, KH_, KW_)                                                                                   \
   if (kt == KT_ && kh == KH_ && kw == KW_)                                                                              \
     return cudaLaunchKernelEx(&ls.cfg, maxpool3d_bf16x8_win_kernel<KT_, KH_, KW_>, static_cast<const uint4*>(x), t, h, w, \

@@ -446,7 +446,14 @@ def test_maxpool_and_add_relu_against_oracle():
         for c, shape, pool in ((64, (2, 4, 8, 8), synth.PoolSpec("p", (2, 2, 2), (2, 2, 2), (0, 0, 0))),
                                (64, (1, 3, 14, 14), synth.PoolSpec("p", (1, 2, 2), (1, 2, 2), (0, 0, 0))),
                                (16, (1, 2, 7, 7), synth.PoolSpec("p", (2, 2, 2), (2, 2, 2), (0, 1, 1))),
-                               (5, (1, 2, 6, 6), synth.PoolSpec("p", (2, 2, 2), (2, 2, 2), (0, 0, 0)))):
+                               (5, (1, 2, 6, 6), synth.PoolSpec("p", (2, 2, 2), (2, 2, 2), (0, 0, 0))),
+                               # unit stride along w: four outputs per thread share their column maxima
+                               (32, (2, 5, 9, 13), synth.PoolSpec("p", (3, 3, 3), (1, 1, 1), (1, 1, 1))),
+                               (16, (1, 4, 7, 4), synth.PoolSpec("p", (3, 3, 3), (1, 1, 1), (1, 1, 1))),
+                               (16, (1, 4, 7, 3), synth.PoolSpec("p", (3, 3, 3), (1, 1, 1), (1, 1, 1))),
+                               (24, (2, 6, 11, 10), synth.PoolSpec("p", (3, 3, 3), (2, 2, 1), (1, 1, 1))),
+                               (8, (1, 3, 12, 17), synth.PoolSpec("p", (1, 3, 3), (1, 1, 1), (0, 1, 1))),
+                               (8, (1, 3, 12, 17), synth.PoolSpec("p", (1, 3, 3), (1, 2, 1), (0, 0, 0)))):
             x = synth.make_input(800 + c, shape + (c,))
             xr = oracle.bf16_round(x) if dtype == torch.bfloat16 else x
             y = nets.to_numpy(nets.maxpool(nets.to_device(x, dtype), c, pool), c)
