@@ -22,6 +22,8 @@ ST_CASES = [
     (32, 80, 48, (1, 1), (1, 9, 16, 24), 0.7, True, True, True),        # pointwise spatial conv, 16-column tails
     (64, 96, 96, (3, 1), (2, 7, 33, 10), 0.5, False, True, False),
     (16, 160, 64, (3, 3), (1, 4, 12, 12), None, True, True, True),      # dense weights
+    (64, 144, 64, (3, 3), (1, 40, 16, 8), 0.4, True, True, True),       # one patch, 40 frames: every CTA pair gets one frame of a cut clip
+    (48, 112, 64, (3, 3), (2, 37, 24, 16), 0.5, False, True, True),     # long clips cut at odd places
 ]
 
 
