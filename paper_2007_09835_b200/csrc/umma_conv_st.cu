@@ -13,8 +13,8 @@
 //   T(p)  adds that frame's contribution to the THREE output frames it touches, out(p-1) += mid(p) Wt[2],
 //         out(p) += mid(p) Wt[1], out(p+1) += mid(p) Wt[0]: three output accumulators live in TMEM, so only
 //         one intermediate frame is ever held and nothing is recomputed along t,
-//   E2    four more epilogue warps drain each output frame once its last contribution has landed
-//         (+ bias, residual, ReLU, bf16, 16-byte global stores).
+//   E2    eight more epilogue warps (two per lane quadrant, alternating 32-channel pieces) drain each output
+//         frame once its last contribution has landed (+ bias, residual, ReLU, bf16, 16-byte global stores).
 // CTA pairs (tcgen05 cta_group::2): two patches per MMA, each CTA holds half of both weight tensors.
 // The MMA warp issues S(p+1) before T(p), so E1(p) overlaps S(p+1) on the tensor pipe.
 //
@@ -42,7 +42,7 @@
 namespace rt3d {
 namespace {
 
-constexpr int kThreadsSt = 448;         // producer, MMA, 8 x E1, 4 x E2 warps
+constexpr int kThreadsSt = 576;         // producer, MMA, 8 x E1, 8 x E2 warps
 constexpr int kStOuts = 3;              // output accumulators in flight = temporal kernel extent
 
 struct StBars {
@@ -50,7 +50,7 @@ struct StBars {
   unsigned long long w_full;            // leader: both weight tensors of both CTAs have landed
   unsigned long long mid_full;          // leader: 16 E1 warps wrote the intermediate frame back into D1
   unsigned long long out_full[kStOuts]; // both: last contribution to an output accumulator is done
-  unsigned long long out_empty[kStOuts];// leader: 8 E2 warps drained it
+  unsigned long long out_empty[kStOuts];// leader: 16 E2 warps drained it
 };
 
 // Walk over this CTA pair's frame jobs.  g counts (patch pair, output frame) steps; a segment is the part of
@@ -151,7 +151,7 @@ conv3d_umma_st_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_con
     mbar_init(smem_u32(&sb->mid_full), 16);              // leader: 8 E1 warps of each CTA
     for (int s = 0; s < kStOuts; ++s) {
       mbar_init(smem_u32(&sb->out_full[s]), 1);
-      mbar_init(smem_u32(&sb->out_empty[s]), 8);         // leader: 4 E2 warps of each CTA
+      mbar_init(smem_u32(&sb->out_empty[s]), 16);        // leader: 8 E2 warps of each CTA
     }
     bars->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -350,8 +350,9 @@ conv3d_umma_st_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_con
       if (lane == 0) mbar_arrive_cluster(mid_full_leader);
     }
   } else {
-    // ------------------------------------------------------------------ E2: output accumulators -> y (both CTAs, 4 warps)
+    // ------------------------------------------------------------------ E2: output accumulators -> y (both CTAs, 8 warps)
     const int quad = warp & 3;
+    const int half2 = (warp - 10) >> 2;        // two warps per lane quadrant: even / odd 32-column pieces
     const int row = quad * 32 + lane;
     const int bh_i = row >> 3, bw_i = row & 7;
     __nv_bfloat16* yb = static_cast<__nv_bfloat16*>(a.y);
@@ -379,11 +380,12 @@ conv3d_umma_st_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_con
         uint4 rv[4];
 #pragma unroll
         for (int e = 0; e < 4; ++e)
-          rv[e] = (res_row != nullptr && 8 * e < a.rcs) ? __ldg(reinterpret_cast<const uint4*>(res_row) + e) : make_uint4(0u, 0u, 0u, 0u);
+          rv[e] = (res_row != nullptr && half2 * 32 + 8 * e < a.rcs)
+                      ? __ldg(reinterpret_cast<const uint4*>(res_row + half2 * 32) + e) : make_uint4(0u, 0u, 0u, 0u);
         if (!mbar_wait(smem_u32(&sb->out_full[slot]), (q / kStOuts) & 1u, bars, err, 49)) { ok = false; break; }
         tc_fence_after();
         const uint32_t taddr = out_tmem + (uint32_t(quad * 32) << 16) + slot * uint32_t(a.n2);
-        for (int col = 0; col < a.n2 && col < a.M2; col += 32) {
+        for (int col = half2 * 32; col < a.n2 && col < a.M2; col += 64) {
           uint32_t v[32];
           const bool wide = col + 32 <= a.n2;
           if (wide) tmem_ld32(taddr + col, v);
@@ -391,11 +393,11 @@ conv3d_umma_st_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_con
           uint4 rc[4];
 #pragma unroll
           for (int e = 0; e < 4; ++e) rc[e] = rv[e];
-          if (col + 32 < a.n2) {
+          if (col + 64 < a.n2) {
 #pragma unroll
             for (int e = 0; e < 4; ++e)
-              rv[e] = (res_row != nullptr && col + 32 + 8 * e < a.rcs)
-                          ? __ldg(reinterpret_cast<const uint4*>(res_row + col + 32) + e) : make_uint4(0u, 0u, 0u, 0u);
+              rv[e] = (res_row != nullptr && col + 64 + 8 * e < a.rcs)
+                          ? __ldg(reinterpret_cast<const uint4*>(res_row + col + 64) + e) : make_uint4(0u, 0u, 0u, 0u);
           }
           const float4* b4 = reinterpret_cast<const float4*>(bias2_s + col);
           uint4 ov[4];
