@@ -15,6 +15,7 @@ CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "librt3d.so")
 SOURCES = ["api.cu", "pack.cpp", "simt_kernels.cu", "umma_conv.cu", "umma_conv_pair.cu", "umma_conv_halo.cu", "umma_conv_st.cu", "umma_smallc.cu", "reweight.cu"]
 HEADERS = ["kernels.h", "rt3d_internal.h", "umma_common.cuh", "umma_pair.cuh", "pdl.cuh", "tile_consts.h"]
+MICROBENCH = os.path.join(HERE, "rt3d_microbench")       # stand-alone instruction-rate microbenchmarks
 
 
 def _nvcc() -> str:
@@ -45,5 +46,20 @@ def build(force: bool = False, verbose: bool = False) -> str:
     return LIB
 
 
+def build_microbench(force: bool = False) -> str:
+    """Compiles csrc/microbench_mma.cu into the stand-alone program `rt3d_microbench` (prints a markdown report)."""
+    src = os.path.join(CSRC, "microbench_mma.cu")
+    deps = [src, os.path.join(CSRC, "umma_common.cuh"), os.path.join(CSRC, "umma_pair.cuh")]
+    if not force and os.path.exists(MICROBENCH) and all(os.path.getmtime(d) <= os.path.getmtime(MICROBENCH) for d in deps):
+        return MICROBENCH
+    tmp = MICROBENCH + f".tmp{os.getpid()}"
+    subprocess.check_call([_nvcc(), "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
+                           "-I", os.path.join(ROOT, "include"), "-I", CSRC, "-o", tmp, src])
+    os.replace(tmp, MICROBENCH)
+    return MICROBENCH
+
+
 if __name__ == "__main__":
     print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    if "--microbench" in sys.argv:
+        print(build_microbench(force="--force" in sys.argv))

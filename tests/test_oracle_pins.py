@@ -220,6 +220,41 @@ def test_pack_roundtrip_and_counts(M, N, g_m, g_n, to_bf16):
     assert np.isclose(np.abs(tiles).sum(dtype=np.float64), np.abs(back).sum(dtype=np.float64))
 
 
+def test_pack_tile_element_order_by_direct_indexing():
+    """Pins the order INSIDE a tile without going through the oracle's own unpack: element [i][j] of the
+    tile stored for group (p, q) at kernel location kpos is W[p*g_m + i][q*g_n + j][kpos], zero where the
+    kernel does not exist (ragged last groups).  A non-square group size and weights that encode their own
+    (m, n, kpos) make a transposed or differently flattened layout fail."""
+    M, N, k, g_m, g_n = 19, 14, (2, 3, 2), 8, 4
+    Ks = k[0] * k[1] * k[2]
+    m_i, n_i, k_i = np.meshgrid(np.arange(M), np.arange(N), np.arange(Ks), indexing="ij")
+    # m + n/16 + kpos/256 + 1: distinct per (m, n, kpos); 5 + 4 + 4 significant bits, but bf16 keeps 8, so
+    # the bf16 case uses a code with 8 bits that is still distinct inside every tile and across locations
+    codes = {False: (1.0 + m_i + n_i / 16.0 + k_i / 256.0), True: (1.0 + (m_i % 8) * 16 + (n_i % 4) * 4 + (k_i % 4))}
+    P, Q = synth.n_groups(M, N, g_m, g_n)
+    gm = synth.kgs_mask_bernoulli(P, Q, Ks, 0.5, 77)
+    mask = synth.expand_group_mask(gm, M, N, g_m, g_n, *k)
+    for to_bf16 in (False, True):
+        wv = codes[to_bf16].astype(np.float32).reshape((M, N) + k)
+        pk = oracle.pack_kgs(wv, mask, g_m, g_n, to_bf16)
+        tiles = pk["tiles"] if not to_bf16 else oracle.bf16_widen(pk["tiles"])
+        assert tiles.shape == (pk["nnz"], g_m, g_n) and pk["nnz"] > 0
+        w3 = wv.reshape(M, N, Ks)
+        seen_ragged = False
+        for p in range(P):
+            for q in range(Q):
+                g = p * Q + q
+                for e in range(pk["group_ptr"][g], pk["group_ptr"][g + 1]):
+                    kpos = int(pk["pos_idx"][e])
+                    for i in range(g_m):
+                        for j in range(g_n):
+                            m, n = p * g_m + i, q * g_n + j
+                            inside = m < M and n < N
+                            seen_ragged |= not inside
+                            assert tiles[e, i, j] == (w3[m, n, kpos] if inside else 0.0), (to_bf16, p, q, kpos, i, j)
+        assert seen_ragged
+
+
 def test_pack_rejects_non_uniform_mask():
     wt = _rand((8, 8, 3, 3, 3), 1)
     mask = np.ones_like(wt, dtype=np.uint8)
@@ -279,9 +314,17 @@ def test_maxpool_ramp_closed_form_and_library():
 
 
 def test_add_relu():
-    a, b = _rand((3, 5), 1), _rand((3, 5), 2)
-    np.testing.assert_array_equal(oracle.add_relu(a, b, True), np.maximum(a.astype(np.float64) + b, 0).astype(np.float32))
-    np.testing.assert_array_equal(oracle.add_relu(a, b, False), (a.astype(np.float64) + b).astype(np.float32))
+    # hand values: sums that are exact in binary, one negative, one exactly zero, one positive
+    a = np.array([[1.5, -2.0, 0.25], [-0.5, 3.0, -4.0]], np.float32)
+    b = np.array([[0.5, 1.0, -0.25], [-0.5, -1.0, 4.5]], np.float32)
+    np.testing.assert_array_equal(oracle.add_relu(a, b, False), np.array([[2.0, -1.0, 0.0], [-1.0, 2.0, 0.5]], np.float32))
+    np.testing.assert_array_equal(oracle.add_relu(a, b, True), np.array([[2.0, 0.0, 0.0], [0.0, 2.0, 0.5]], np.float32))
+    # and commutativity / idempotence of the activation on random data
+    x, y = _rand((3, 5), 1), _rand((3, 5), 2)
+    r = oracle.add_relu(x, y, True)
+    np.testing.assert_array_equal(r, oracle.add_relu(y, x, True))
+    np.testing.assert_array_equal(oracle.add_relu(r, np.zeros_like(r), True), r)
+    assert (r >= 0).all() and (r[oracle.add_relu(x, y, False) > 0] > 0).all()
 
 
 # -------------------------------------------------------------------- workload shapes
