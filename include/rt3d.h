@@ -59,10 +59,16 @@ typedef enum {
   RT3D_ALGO_UMMA = 2,   /* tcgen05 tensor-core kernel, one CTA per tile; RT3D_ERR_UNSUPPORTED if not applicable */
   RT3D_ALGO_UMMA_PAIR = 3, /* tcgen05 kernel on CTA pairs (two tiles per MMA, weight tile shared by the
                              pair); RT3D_ERR_UNSUPPORTED if not applicable                        */
-  RT3D_ALGO_UMMA_HALO = 4  /* tcgen05 kernel on CTA pairs for thin stride-1 layers: the layer's packed weights
+  RT3D_ALGO_UMMA_HALO = 4, /* tcgen05 kernel on CTA pairs for thin stride-1 layers: the layer's packed weights
                              stay in shared memory and each output tile's input block (with halo) is
                              staged once for all kernel locations; RT3D_ERR_UNSUPPORTED if the weights
                              plus two input blocks do not fit, M > 256, or a stride is not 1      */
+  RT3D_ALGO_UMMA_SUB = 5   /* tcgen05 kernel that skips pruned kernel locations per block of 16 output x 16
+                             input channels (input tiles held in tensor memory, eight issuing warps).
+                             Never chosen by RT3D_ALGO_AUTO: on B200 it is slower than multiplying the
+                             zero-filled tiles (see the kernel's header comment); kept as the measured
+                             answer to "can skipping at the paper's group sizes pay on this hardware".
+                             RT3D_ERR_UNSUPPORTED for dense handles, fused pooling and fp32         */
 } rt3d_algo;
 
 /* NDHWC activation tensor in DEVICE memory (HOST memory for the *_host entry point), caller-owned. */
@@ -138,6 +144,12 @@ rt3d_status rt3d_unpack_to_dense(const rt3d_packed* p, float* w_out);
  * `n_tile` output channels (0 = the library's choice): w_out as above.  Lets a host-only
  * test check that derived layout against the canonical one. */
 rt3d_status rt3d_unpack_device_layout(const rt3d_packed* p, int n_tile, float* w_out);
+
+/* The same check for the layout of the sub-tile kernel (RT3D_ALGO_UMMA_SUB): w_out is rebuilt from the
+ * 16 x 16 weight blocks and the step headers; RT3D_ERR_INVALID_ARG if they are inconsistent (a non-zero
+ * weight outside the tensor, a block index out of range, a first step that does not start every range of
+ * its bundle).  Pure host work. */
+rt3d_status rt3d_unpack_sub_layout(const rt3d_packed* p, int n_tile, float* w_out);
 
 /* Upload the handle's device blobs to the current CUDA device now (otherwise done by the
  * first compute call).  Synchronises the device. */
@@ -304,7 +316,8 @@ rt3d_status rt3d_conv3d_cost(const rt3d_tensor* x, const rt3d_packed* w, const r
 /* How the calling thread's most recent successful convolution call was run (for tests and profiling):
  *   kernel       0 CUDA-core kernel, 1 tensor-core single-CTA kernel, 2 tensor-core CTA-pair kernel,
  *                3 tensor-core small-C_in kernel, 4 tensor-core resident-weight (halo) kernel,
- *                5 fused (2+1)D kernel (rt3d_conv2plus1d_fused; n_tile = intermediate width)
+ *                5 fused (2+1)D kernel (rt3d_conv2plus1d_fused; n_tile = intermediate width),
+ *                6 tensor-core sub-tile kernel (RT3D_ALGO_UMMA_SUB)
  *   n_tile       output channels per accumulator tile (tensor-core kernels, else 0)
  *   n_splits     K splits per output tile in the single-CTA kernel (1 = none)
  *   tail_workers CTA pairs that share, cut along K, the output tiles which do not fill a last round

@@ -16,7 +16,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.environ.get("RT3D_LIB") or os.path.join(_HERE, "librt3d.so")   # RT3D_LIB: alternative build of the same library
 
 RT3D_F32, RT3D_BF16 = 0, 1
-ALGO_AUTO, ALGO_SIMT, ALGO_UMMA, ALGO_UMMA_PAIR, ALGO_UMMA_HALO = 0, 1, 2, 3, 4
+ALGO_AUTO, ALGO_SIMT, ALGO_UMMA, ALGO_UMMA_PAIR, ALGO_UMMA_HALO, ALGO_UMMA_SUB = 0, 1, 2, 3, 4, 5
 OK, ERR_INVALID_ARG, ERR_SHAPE, ERR_MASK_NOT_GROUP_UNIFORM, ERR_UNSUPPORTED, ERR_ALLOC, ERR_CUDA, ERR_TIMEOUT = range(8)
 ERR_WORKSPACE, ERR_NOT_PREPARED = 8, 9
 
@@ -67,6 +67,7 @@ def _load():
     lib.rt3d_packed_view_get.argtypes = [vp, ctypes.POINTER(PackedView)]
     lib.rt3d_unpack_to_dense.argtypes = [vp, f32p]
     lib.rt3d_unpack_device_layout.argtypes = [vp, i, f32p]
+    lib.rt3d_unpack_sub_layout.argtypes = [vp, i, f32p]
     lib.rt3d_packed_prepare.argtypes = [vp]
     lib.rt3d_packed_free.argtypes = [vp]
     lib.rt3d_packed_free.restype = None
@@ -141,6 +142,13 @@ class Packed:
         _check(_lib.rt3d_unpack_device_layout(self.handle, int(n_tile),
                                               out.ctypes.data_as(ctypes.POINTER(ctypes.c_float))),
                "rt3d_unpack_device_layout")
+        return out
+
+    def unpack_sub_layout(self, n_tile: int = 0) -> np.ndarray:
+        v = self.view()
+        out = np.empty((v["M"], v["N"], v["Kt"], v["Kh"], v["Kw"]), np.float32)
+        _check(_lib.rt3d_unpack_sub_layout(self.handle, int(n_tile), out.ctypes.data_as(ctypes.POINTER(ctypes.c_float))),
+               "rt3d_unpack_sub_layout")
         return out
 
     def prepare(self):

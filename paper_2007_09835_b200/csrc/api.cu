@@ -3,6 +3,7 @@
 #include <cuda.h>
 #include <cuda_runtime.h>
 
+#include <algorithm>
 #include <atomic>
 #include <cstdio>
 #include <cstdlib>
@@ -41,8 +42,8 @@ rt3d_status get_device_state(DeviceState** out) {
   if (!d.init) {
     if (cudaDeviceGetAttribute(&d.sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return RT3D_ERR_CUDA;
     if (cudaDeviceGetAttribute(&d.cc_major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return RT3D_ERR_CUDA;
-    if (cudaMalloc(&d.sched, 8 * sizeof(int32_t)) != cudaSuccess) return RT3D_ERR_ALLOC;
-    if (cudaMemset(d.sched, 0, 8 * sizeof(int32_t)) != cudaSuccess) return RT3D_ERR_CUDA;
+    if (cudaMalloc(&d.sched, 256 * sizeof(int32_t)) != cudaSuccess) return RT3D_ERR_ALLOC;
+    if (cudaMemset(d.sched, 0, 256 * sizeof(int32_t)) != cudaSuccess) return RT3D_ERR_CUDA;
     if (!g_encode) {
       void* fn = nullptr;
       cudaDriverEntryPointQueryResult qres;
@@ -77,7 +78,7 @@ rt3d_status make_geom(const rt3d_tensor* x, const rt3d_packed* w, const rt3d_con
   if (s != RT3D_OK) return s;
   if (!w || !p) return RT3D_ERR_INVALID_ARG;
   if (p->st < 1 || p->sh < 1 || p->sw < 1 || p->pt < 0 || p->ph < 0 || p->pw < 0) return RT3D_ERR_INVALID_ARG;
-  if (p->algo < RT3D_ALGO_AUTO || p->algo > RT3D_ALGO_UMMA_HALO) return RT3D_ERR_INVALID_ARG;
+  if (p->algo < RT3D_ALGO_AUTO || p->algo > RT3D_ALGO_UMMA_SUB) return RT3D_ERR_INVALID_ARG;
   if (x->c != w->N || x->dtype != w->dtype) return RT3D_ERR_SHAPE;
   const int64_t To = (int64_t(x->t) + 2 * p->pt - w->Kt) / p->st + 1;
   const int64_t Ho = (int64_t(x->h) + 2 * p->ph - w->Kh) / p->sh + 1;
@@ -182,6 +183,26 @@ rt3d_status get_umma_blob(rt3d_packed* h, DeviceBlob* blob, const UmmaLayout* L,
                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
       if (r != CUDA_SUCCESS) return RT3D_ERR_CUDA;
     }
+    u.ready = true;
+  }
+  *out = &u;
+  return RT3D_OK;
+}
+
+// Device copy of the sub-tile kernel's layout (step records, step offsets, weight blocks).
+rt3d_status get_sub_blob(rt3d_packed* h, DeviceBlob* blob, const SubLayout* L, DeviceBlob::Sub** out) {
+  std::lock_guard<std::mutex> lock(h->mu);
+  DeviceBlob::Sub& u = blob->sub[L->n_tile];
+  if (!u.ready) {
+    const size_t sbytes = L->steps.size() * sizeof(SubStep), bbytes = L->payload.size();
+    if (cudaMalloc(&u.steps, sbytes + 64) != cudaSuccess ||
+        cudaMalloc(reinterpret_cast<void**>(&u.step_ptr), L->step_ptr.size() * 4) != cudaSuccess ||
+        cudaMalloc(&u.blocks, bbytes + 512) != cudaSuccess)
+      return RT3D_ERR_ALLOC;
+    if ((sbytes && cudaMemcpy(u.steps, L->steps.data(), sbytes, cudaMemcpyHostToDevice) != cudaSuccess) ||
+        cudaMemcpy(u.step_ptr, L->step_ptr.data(), L->step_ptr.size() * 4, cudaMemcpyHostToDevice) != cudaSuccess ||
+        (bbytes && cudaMemcpy(u.blocks, L->payload.data(), bbytes, cudaMemcpyHostToDevice) != cudaSuccess))
+      return RT3D_ERR_CUDA;
     u.ready = true;
   }
   *out = &u;
@@ -500,6 +521,46 @@ rt3d_status try_halo(rt3d_packed* w, DeviceBlob* blob, DeviceState* d, const rt3
   return RT3D_OK;
 }
 
+// Sub-tile kernel: blocks of 16 x 16 channels in which no kernel group keeps the step's location are skipped.
+// Runs only when asked for (RT3D_ALGO_UMMA_SUB): measured on B200 it loses to the masked-dense CTA-pair kernel at
+// every group size and pruning rate of the sweep, because moving a step's input tile through shared memory into
+// tensor memory costs about as much as the dense MMAs of that step.
+// *launched = false (and RT3D_OK) when the handle cannot use it.
+rt3d_status try_sub(rt3d_packed* w, DeviceBlob* blob, DeviceState* d, const rt3d_tensor* x, const ConvGeom& g,
+                    const float* bias, rt3d_tensor* y, const void* res_data, int res_pitch, cudaStream_t st, bool* launched) {
+  *launched = false;
+  if (w->is_dense) return RT3D_OK;
+  SubArgs a;
+  a.g = g;
+  a.box = choose_box(g);
+  a.tiles_n = ceil_div(g.n, a.box.bn); a.tiles_t = ceil_div(g.To, a.box.bt);
+  a.tiles_h = ceil_div(g.Ho, a.box.bh); a.tiles_w = ceil_div(g.Wo, a.box.bw);
+  const long long m_tiles = (long long)a.tiles_n * a.tiles_t * a.tiles_h * a.tiles_w;
+  if (m_tiles > (1ll << 30)) return RT3D_OK;
+  const SubLayout* L = get_sub_layout(w, 0);
+  if (!L) return RT3D_OK;
+  a.n_tile = L->n_tile; a.n_bundles = L->n_bundles;
+  if (!umma_sub_plan(&a, L->max_blocks)) return RT3D_OK;
+  DeviceBlob::Sub* u = nullptr;
+  rt3d_status s = get_sub_blob(w, blob, L, &u);
+  if (s != RT3D_OK) return s;
+  a.steps = static_cast<const SubStep*>(u->steps); a.step_ptr = u->step_ptr; a.blocks = u->blocks;
+  a.bias = bias; a.y = y->data; a.sched = d->sched;
+  a.residual = res_data; a.rcs = res_pitch;
+  CUtensorMap xmap, ymap;
+  if ((s = encode_xmap(x, g, a.box, &xmap)) != RT3D_OK) return s;
+  int sb[4] = {1, 1, 1, 1};
+  const bool rect = warp_block(a.box.bw, a.box.bh, a.box.bt, a.box.bn, sb);
+  a.store_tma = (rect && encode_ymap(y, sb, 1, 1, 1, &ymap)) ? 1 : 0;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return RT3D_ERR_CUDA;
+  if (launch_conv_umma_sub(a, &xmap, a.store_tma ? &ymap : nullptr, d->sm_count, dev, st) != cudaSuccess) return RT3D_ERR_CUDA;
+  g_launches.fetch_add(1);
+  t_last_plan = rt3d_plan_info{6, a.n_tile, 1, 0, 0};
+  *launched = true;
+  return RT3D_OK;
+}
+
 rt3d_status conv_impl(const rt3d_tensor* x, const rt3d_packed* wc, const float* bias, const rt3d_conv_params* p,
                       rt3d_tensor* y, void* stream, bool dense_entry, const rt3d_fusion* fz = nullptr) {
   ConvGeom g;
@@ -541,7 +602,8 @@ rt3d_status conv_impl(const rt3d_tensor* x, const rt3d_packed* wc, const float* 
   const bool can_simt = w->g_m <= kMaxGroupSimt && w->g_n <= kMaxGroupSimt;
   if (!can_umma && !can_simt) return RT3D_ERR_UNSUPPORTED;
   if (p->algo == RT3D_ALGO_SIMT && !can_simt) return RT3D_ERR_UNSUPPORTED;
-  const bool want_umma = p->algo == RT3D_ALGO_UMMA || p->algo == RT3D_ALGO_UMMA_PAIR || p->algo == RT3D_ALGO_UMMA_HALO;
+  const bool want_umma = p->algo == RT3D_ALGO_UMMA || p->algo == RT3D_ALGO_UMMA_PAIR || p->algo == RT3D_ALGO_UMMA_HALO ||
+                         p->algo == RT3D_ALGO_UMMA_SUB;
   if (want_umma && !can_umma) return RT3D_ERR_UNSUPPORTED;
   const bool use_umma = want_umma || (p->algo == RT3D_ALGO_AUTO && can_umma);
   if (!use_umma) {
@@ -555,7 +617,8 @@ rt3d_status conv_impl(const rt3d_tensor* x, const rt3d_packed* wc, const float* 
   }
 
   const SmallCLayout* SL = nullptr;
-  if (p->algo != RT3D_ALGO_UMMA_PAIR && p->algo != RT3D_ALGO_UMMA_HALO && (!pooled || pl_t == 1) && smallc_eligible(d, w, x, y, p, &SL)) {
+  if (p->algo != RT3D_ALGO_UMMA_PAIR && p->algo != RT3D_ALGO_UMMA_HALO && p->algo != RT3D_ALGO_UMMA_SUB && (!pooled || pl_t == 1) &&
+      smallc_eligible(d, w, x, y, p, &SL)) {
     s = launch_smallc(w, blob, d, SL, x, g, bias, y, st, res_data, res_pitch, pl_h, pl_w, p->x_pad_zero != 0);
     if (s == RT3D_OK) t_last_plan = rt3d_plan_info{3, SL->n_pad, 1, 0, pooled ? 1 : 0};
     return s;
@@ -567,6 +630,14 @@ rt3d_status conv_impl(const rt3d_tensor* x, const rt3d_packed* wc, const float* 
     if (s != RT3D_OK || launched) return s;
   }
   if (p->algo == RT3D_ALGO_UMMA_HALO) return RT3D_ERR_UNSUPPORTED;
+  if (p->algo == RT3D_ALGO_UMMA_SUB) {
+    bool launched = false;
+    if (!pooled && !dense_entry) {
+      s = try_sub(w, blob, d, x, g, bias, y, res_data, res_pitch, st, &launched);
+      if (s != RT3D_OK || launched) return s;
+    }
+    return RT3D_ERR_UNSUPPORTED;
+  }
 
   UmmaArgs a;
   a.g = g;
@@ -863,6 +934,7 @@ void rt3d_packed_free(rt3d_packed* p) {
     for (void* hs : b->host_streams) if (hs) cudaStreamDestroy(static_cast<cudaStream_t>(hs));
     for (void* he : b->host_events) if (he) cudaEventDestroy(static_cast<cudaEvent_t>(he));
     for (auto& kv : b->smallc) { cudaFree(kv.second.wimg); cudaFree(kv.second.pairs); }
+    for (auto& kv : b->sub) { cudaFree(kv.second.steps); cudaFree(kv.second.step_ptr); cudaFree(kv.second.blocks); }
     cudaFree(b->splitk); cudaFree(b->splitk_cnt);
     delete b;
   }
@@ -1076,6 +1148,7 @@ rt3d_status rt3d_conv3d_sparse_noalloc(const rt3d_tensor* x, const rt3d_packed* 
 }
 
 int64_t rt3d_launch_count(void) { return g_launches.load(); }
+
 
 const char* rt3d_status_string(rt3d_status s) {
   switch (s) {

@@ -127,6 +127,28 @@ bool umma_st_plan(StArgs* a, const int32_t* steps1_host, const int32_t* steps2_h
 cudaError_t launch_conv_umma_st(const StArgs& a, const void* xmap, const void* w1map_half, const void* w2map_half,
                                 int sm_count, cudaStream_t stream);
 
+// Sub-tile kernel (umma_conv_sub.cu): skips pruned kernel locations per block of 16 output x 16 input channels.
+struct SubArgs {
+  ConvGeom g;
+  TileBox box;
+  int n_tile, n_bundles;
+  int tiles_n, tiles_t, tiles_h, tiles_w;
+  const SubStep* steps;               // device: the bundles' step records
+  const int32_t* step_ptr;            // device, [n_bundles + 1]
+  const void* blocks;                 // device: 512-byte weight blocks
+  const float* bias;                  // device or nullptr
+  void* y;
+  int32_t* sched;                     // [2] = error word
+  int store_tma;                      // 1: TMA-store epilogue (needs ymap)
+  const void* residual;               // device bf16 tensor of the output's extents added before the ReLU, or nullptr
+  int rcs;
+  int stages;                         // ring depth (filled in by umma_sub_plan)
+  uint32_t slot_bytes;                // bytes of one stage of the block ring
+};
+bool umma_sub_plan(SubArgs* a, int max_blocks);
+// xmap: input tensor map whose box is the tile box (as for the step-list kernels).
+cudaError_t launch_conv_umma_sub(const SubArgs& a, const void* xmap, const void* ymap, int sm_count, int device, cudaStream_t stream);
+
 // Arguments of the small-C_in tensor-core kernel (C_in <= 8 at channel pitch 8).
 struct SmallCArgs {
   ConvGeom g;

@@ -404,6 +404,222 @@ smem_share_kernel(long long* out, int mma_warps, int mma_count, int cp_warps, in
   }
 }
 
+// ------------------------------------------------------------------------------------------ M8
+// Tensor-memory traffic next to the MMAs.  Eight warps issue chains of N = 16 MMAs with A in tensor memory;
+// B is a 512-byte block in the 128-byte-swizzle layout (b_noswizzle = 0) or in the no-swizzle core-matrix
+// layout (1).  Meanwhile `st_warps` (0 or 4) further warps each write 32 lanes x 32 columns (4 KB) per
+// iteration with tcgen05.st + wait::st, as a kernel that stages its A operand through registers would, and
+// `ld_warps` (0 or 4) read 32 x 32 columns per iteration with tcgen05.ld (an epilogue).
+// out[0] = clocks of the MMA chains, out[1] = clocks of the store loops, out[2] = clocks of the load loops.
+__global__ void __launch_bounds__(512, 1)
+tmem_share_kernel(long long* out, int mma_count, int b_noswizzle, int st_warps, int st_iters, int ld_warps, int ld_iters,
+                  float* sink, int32_t* err) {
+  extern __shared__ unsigned char smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  const uint32_t b_smem = base + kARegion;
+  Barriers* bars = reinterpret_cast<Barriers*>(smem_raw + (base - raw) + kARegion + kBRegion);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  for (uint32_t i = threadIdx.x; i < (kARegion + kBRegion) / 4; i += blockDim.x)
+    reinterpret_cast<uint32_t*>(smem_raw + (base - raw))[i] = 0x3c003c00u;
+  if (threadIdx.x == 0) {
+    for (int q = 0; q < kMaxStages; ++q) mbar_init(smem_u32(&bars->full[q]), 1);
+    bars->abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 0) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&bars->tmem_base)), "r"(512u) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = bars->tmem_base;
+  if (warp < 4) {
+    const uint32_t taddr = tmem_base + (uint32_t(warp * 32) << 16) + 256u;
+    for (int c = 0; c < 32; c += 8)
+      asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %1, %1, %1, %1, %1, %1, %1};" ::"r"(taddr + c), "r"(0x3c003c00u) : "memory");
+    asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const long long t0 = clock64();
+  if (warp < 8) {
+    if (lane == 0) {
+      const uint32_t idesc = idesc_any(0, 128, 16);
+      const uint32_t d = tmem_base + uint32_t(warp) * 16u;
+      for (int i = 0; i < mma_count; ++i) {
+        const uint32_t blk = b_smem + uint32_t((i + warp) & 15) * 2048u;
+        const uint64_t bdesc = b_noswizzle ? smem_desc_noswizzle(blk + uint32_t(i & 3) * 512u, 128u, 256u) : smem_desc_sw128(blk) + 2 * (i & 3);
+        mma_any<0, true, 1>(d, 0ull, tmem_base + 256u + uint32_t(i & 3) * 8u, bdesc, idesc, i ? 1u : 0u);
+      }
+      umma_commit(smem_u32(&bars->full[warp]));
+      mbar_wait(smem_u32(&bars->full[warp]), 0, bars, err, 10);
+      atomicMax(reinterpret_cast<unsigned long long*>(out), (unsigned long long)(clock64() - t0));
+    }
+  } else if (warp < 8 + st_warps) {
+    // columns 320..447 (four 32-column stages), never read by the MMAs
+    uint32_t v[32];
+#pragma unroll
+    for (int q = 0; q < 32; ++q) v[q] = 0x3c003c00u + q + lane;
+    const uint32_t lanes = uint32_t((warp & 3) * 32) << 16;
+    for (int it = 0; it < st_iters; ++it) {
+      const uint32_t taddr = tmem_base + lanes + 320u + uint32_t(it & 3) * 32u;
+      asm volatile(
+          "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+          "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+          ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]), "r"(v[8]), "r"(v[9]),
+            "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]), "r"(v[16]), "r"(v[17]), "r"(v[18]), "r"(v[19]),
+            "r"(v[20]), "r"(v[21]), "r"(v[22]), "r"(v[23]), "r"(v[24]), "r"(v[25]), "r"(v[26]), "r"(v[27]), "r"(v[28]), "r"(v[29]),
+            "r"(v[30]), "r"(v[31]) : "memory");
+      asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+      v[it & 31] += 1u;
+    }
+    if (lane == 0) atomicMax(reinterpret_cast<unsigned long long*>(out + 1), (unsigned long long)(clock64() - t0));
+  } else if (warp < 12 + ld_warps) {
+    float acc = 0.f;
+    const uint32_t lanes = uint32_t((warp & 3) * 32) << 16;
+    for (int it = 0; it < ld_iters; ++it) {
+      uint32_t v[32];
+      tmem_ld32(tmem_base + lanes + 128u + uint32_t(it & 3) * 32u, v);
+#pragma unroll
+      for (int q = 0; q < 32; ++q) acc += __uint_as_float(v[q]);
+    }
+    if (acc == 123.456f) sink[threadIdx.x] = acc;
+    if (lane == 0) atomicMax(reinterpret_cast<unsigned long long*>(out + 2), (unsigned long long)(clock64() - t0));
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+  }
+}
+
+// ------------------------------------------------------------------------------------------ M9
+// The issue loop of a kernel that works in K steps: eight warps, per step each warp (optionally) executes
+// tcgen05.fence::after_thread_sync, issues `per_step` N = 16 MMAs (A in tensor memory, stage step % 8 of an
+// eight-stage ring) and (optionally) commits to the step's barrier (count 8); with `ring` the warp first waits
+// until the barrier of the step eight earlier has completed.  out[0] = clocks for all steps.
+__global__ void __launch_bounds__(256, 1)
+stepped_issue_kernel(long long* out, int steps, int per_step, int use_fence, int use_commit, int ring, int a_stages, int d_stride, int n, int32_t* err) {
+  extern __shared__ unsigned char smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  const uint32_t b_smem = base + kARegion;
+  Barriers* bars = reinterpret_cast<Barriers*>(smem_raw + (base - raw) + kARegion + kBRegion);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  for (uint32_t i = threadIdx.x; i < (kARegion + kBRegion) / 4; i += blockDim.x)
+    reinterpret_cast<uint32_t*>(smem_raw + (base - raw))[i] = 0x3c003c00u;
+  if (threadIdx.x == 0) {
+    for (int q = 0; q < kMaxStages; ++q) { mbar_init(smem_u32(&bars->full[q]), 8); mbar_init(smem_u32(&bars->empty[q]), 1); }
+    bars->abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 0) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&bars->tmem_base)), "r"(512u) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = bars->tmem_base;
+  if (warp < 4) {
+    for (int c = 0; c < 256; c += 8)
+      asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %1, %1, %1, %1, %1, %1, %1};"
+                   ::"r"(tmem_base + (uint32_t(warp * 32) << 16) + 256u + c), "r"(0x3c003c00u) : "memory");
+    asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  if (lane == 0) {
+    const uint32_t idesc = idesc_any(0, 128, n);
+    const uint32_t d = tmem_base + uint32_t(warp) * uint32_t(d_stride);
+    const long long t0 = clock64();
+    for (int st = 0; st < steps; ++st) {
+      const int stage = st & 7;
+      const int a_stage = st % a_stages;
+      if (ring && st >= 8 && !mbar_wait(smem_u32(&bars->full[stage]), uint32_t((st >> 3) - 1) & 1u, bars, err, 11)) break;
+      if (use_fence) tc_fence_after();
+      for (int i = 0; i < per_step; ++i) {
+        const uint64_t bdesc = smem_desc_noswizzle(b_smem + uint32_t((st + warp) & 15) * 2048u + uint32_t(i & 3) * 512u, 128u, 256u);
+        mma_any<0, true, 1>(d, 0ull, tmem_base + 256u + uint32_t(a_stage) * 32u + uint32_t(i & 3) * 8u, bdesc, idesc, (st | i) ? 1u : 0u);
+      }
+      if (use_commit) umma_commit(smem_u32(&bars->full[stage]));
+    }
+    if (warp == 0) {
+      umma_commit(smem_u32(&bars->empty[0]));
+      mbar_wait(smem_u32(&bars->empty[0]), 0, bars, err, 12);
+    }
+    atomicMax(reinterpret_cast<unsigned long long*>(out), (unsigned long long)(clock64() - t0));
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+  }
+}
+
+// ------------------------------------------------------------------------------------------ M10
+// Several lanes of one warp issuing: lanes 0..L-1 of each of W warps each run their own chain of N = 16 MMAs
+// (A in tensor memory) into their own 16 accumulator columns.  out[0] = clocks until all chains are done.
+__global__ void __launch_bounds__(512, 1)
+lane_issue_kernel(long long* out, int count, int warps, int lanes, int a_slices, int32_t* err) {
+  extern __shared__ unsigned char smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  const uint32_t b_smem = base + kARegion;
+  Barriers* bars = reinterpret_cast<Barriers*>(smem_raw + (base - raw) + kARegion + kBRegion);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  for (uint32_t i = threadIdx.x; i < (kARegion + kBRegion) / 4; i += blockDim.x)
+    reinterpret_cast<uint32_t*>(smem_raw + (base - raw))[i] = 0x3c003c00u;
+  if (threadIdx.x == 0) {
+    mbar_init(smem_u32(&bars->full[0]), uint32_t(warps * lanes));
+    bars->abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 0) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&bars->tmem_base)), "r"(512u) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = bars->tmem_base;
+  if (warp < 4) {
+    for (int c = 0; c < 256; c += 8)
+      asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %1, %1, %1, %1, %1, %1, %1};"
+                   ::"r"(tmem_base + (uint32_t(warp * 32) << 16) + 256u + c), "r"(0x3c003c00u) : "memory");
+    asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  if (warp < warps && lane < lanes) {
+    const uint32_t idesc = idesc_any(0, 128, 16);
+    const uint32_t d = tmem_base + uint32_t(warp * lanes + lane) * 16u;
+    const uint64_t bdesc = smem_desc_noswizzle(b_smem + uint32_t(warp * lanes + lane) * 2048u, 128u, 256u);
+    const long long t0 = clock64();
+    for (int i = 0; i < count; ++i)
+      mma_any<0, true, 1>(d, 0ull, tmem_base + 256u + uint32_t(i & (a_slices - 1)) * 8u, bdesc + uint64_t(i & 3) * 32u, idesc, i ? 1u : 0u);
+    umma_commit(smem_u32(&bars->full[0]));
+    mbar_wait(smem_u32(&bars->full[0]), 0, bars, err, 13);
+    atomicMax(reinterpret_cast<unsigned long long*>(out), (unsigned long long)(clock64() - t0));
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+  }
+}
+
 // ------------------------------------------------------------------------------------------ M3
 // kShape: 0 m16n8k16 bf16, 1 m16n8k8 bf16, 2 m16n8k8 tf32, 3 m16n8k4 tf32.  Eight independent accumulator
 // tiles per warp, operands in registers.
@@ -709,6 +925,68 @@ int main(int argc, char** argv) {
              cp_bw, bk_clk, bk_bw, mma_bw + cp_bw + bk_bw);
     }
     cudaFree(gsrc);
+  }
+
+  printf("\n## M8: tensor-memory stores and loads next to 8 warps issuing N = 16 MMAs (A in TMEM), one CTA\n\n");
+  printf("| B layout | st warps | ld warps | clk/MMA | st clk per 4 KB (one warp) | TMEM write B/clk (all st warps) | ld clk per 4 KB |\n|---|---|---|---|---|---|---|\n");
+  {
+    const size_t smem = 1024 + kARegion + kBRegion + sizeof(Barriers) + 64;
+    cudaFuncSetAttribute(tmem_share_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
+    const int combos[][4] = {{0, 0, 0, 1}, {1, 0, 0, 1}, {1, 4, 0, 0}, {1, 4, 0, 1}, {0, 4, 0, 1}, {1, 0, 4, 1}, {1, 4, 4, 1}};
+    for (const auto& cb : combos) {
+      const int mma_count = cb[3] ? 512 : 0, st_iters = cb[1] ? 256 : 0, ld_iters = cb[2] ? 256 : 0;
+      long long h[3] = {0, 0, 0};
+      for (int rep = 0; rep < 2; ++rep) {
+        cudaMemset(d_out, 0, 32);
+        tmem_share_kernel<<<1, 512, smem>>>(d_out, mma_count, cb[0], cb[1], st_iters, cb[2], ld_iters, d_sink, d_err);
+        if (!sync_ok("tmem_share")) return 1;
+      }
+      cudaMemcpy(h, d_out, 24, cudaMemcpyDeviceToHost);
+      printf("| %s | %d | %d | %.1f | %.1f | %.0f | %.1f |\n", cb[0] ? "no swizzle" : "128-byte swizzle", cb[1], cb[2],
+             mma_count ? double(h[0]) / (mma_count * 8.0) : 0.0, st_iters ? double(h[1]) / st_iters : 0.0,
+             st_iters ? 4096.0 * cb[1] * st_iters / double(h[1]) : 0.0, ld_iters ? double(h[2]) / ld_iters : 0.0);
+    }
+  }
+
+  printf("\n## M9: issue loop in K steps (8 warps, N = 16 MMAs with A in TMEM, per-step fence / commit / ring wait)\n\n");
+  printf("| MMAs per warp and step | N | fence | commit | ring wait | A stages cycled | D column stride per warp | clk/step | clk/MMA |\n|---|---|---|---|---|---|---|---|---|\n");
+  {
+    const size_t smem = 1024 + kARegion + kBRegion + sizeof(Barriers) + 64;
+    cudaFuncSetAttribute(stepped_issue_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
+    const int combos[][7] = {{4, 0, 0, 0, 1, 16, 16}, {4, 0, 0, 0, 1, 32, 16}, {4, 0, 0, 0, 8, 16, 16}, {4, 0, 0, 0, 8, 32, 16}, {4, 0, 0, 0, 2, 32, 16},
+                             {4, 1, 1, 1, 8, 32, 16}, {2, 1, 1, 1, 8, 32, 16}, {1, 1, 1, 1, 8, 32, 16}, {1, 1, 1, 1, 1, 32, 16},
+                             {4, 1, 1, 1, 8, 32, 32}, {2, 1, 1, 1, 8, 32, 32}, {1, 1, 1, 1, 8, 32, 32}};
+    for (const auto& cb : combos) {
+      const int steps = 256;
+      long long h[1] = {0};
+      for (int rep = 0; rep < 2; ++rep) {
+        cudaMemset(d_out, 0, 32);
+        stepped_issue_kernel<<<1, 256, smem>>>(d_out, steps, cb[0], cb[1], cb[2], cb[3], cb[4], cb[5], cb[6], d_err);
+        if (!sync_ok("stepped_issue")) return 1;
+      }
+      cudaMemcpy(h, d_out, 8, cudaMemcpyDeviceToHost);
+      printf("| %d | %d | %s | %s | %s | %d | %d | %.1f | %.1f |\n", cb[0], cb[6], cb[1] ? "yes" : "no", cb[2] ? "yes" : "no", cb[3] ? "yes" : "no",
+             cb[4], cb[5], double(h[0]) / steps, double(h[0]) / steps / (cb[0] * 8.0));
+    }
+  }
+
+  printf("\n## M10: several lanes of a warp issuing N = 16 MMAs (A in TMEM), each lane its own accumulator\n\n");
+  printf("| warps | lanes per warp | A slices cycled | clk per MMA (all chains) | clk per MMA of one lane |\n|---|---|---|---|---|\n");
+  {
+    const size_t smem = 1024 + kARegion + kBRegion + sizeof(Barriers) + 64;
+    cudaFuncSetAttribute(lane_issue_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
+    const int combos[][3] = {{1, 1, 4}, {1, 2, 4}, {1, 4, 4}, {1, 16, 4}, {4, 4, 4}, {8, 2, 4}, {8, 1, 4}, {16, 1, 4}, {8, 1, 1}, {8, 1, 8}, {8, 1, 32}, {16, 1, 32}, {1, 1, 32}};
+    for (const auto& cb : combos) {
+      const int cnt = 256;
+      long long h[1] = {0};
+      for (int rep = 0; rep < 2; ++rep) {
+        cudaMemset(d_out, 0, 32);
+        lane_issue_kernel<<<1, 512, smem>>>(d_out, cnt, cb[0], cb[1], cb[2], d_err);
+        if (!sync_ok("lane_issue")) return 1;
+      }
+      cudaMemcpy(h, d_out, 8, cudaMemcpyDeviceToHost);
+      printf("| %d | %d | %d | %.1f | %.1f |\n", cb[0], cb[1], cb[2], double(h[0]) / (double(cnt) * cb[0] * cb[1]), double(h[0]) / cnt);
+    }
   }
 
   printf("\n## M2: tcgen05.mma cta_group::1 kind::tf32 (K = 8)\n\n");

@@ -103,6 +103,93 @@ const UmmaLayout* get_umma_layout(rt3d_packed* p, int n_tile) {
   return &res.first->second;
 }
 
+// Layout of the sub-tile kernel (see SubLayout and SubStep).
+const SubLayout* get_sub_layout(rt3d_packed* p, int n_tile) {
+  if (!umma_layout_possible(p)) return nullptr;
+  if (n_tile <= 0) n_tile = default_n_tile(p->M);
+  if (n_tile % 16 || n_tile > 256) return nullptr;
+  std::lock_guard<std::mutex> lock(p->mu);
+  auto it = p->sub_layouts.find(n_tile);
+  if (it != p->sub_layouts.end()) return &it->second;
+
+  SubLayout L;
+  L.n_tile = n_tile;
+  L.n_bundles = ceil_div(p->M, n_tile);
+  L.n_chunks = ceil_div(p->N, kChunk);
+  L.step_ptr.assign(L.n_bundles + 1, 0);
+  const int Ks = p->Ks;
+  const uint16_t* tiles = reinterpret_cast<const uint16_t*>(p->tiles.data());
+  std::vector<uint64_t> pres(size_t(Ks) * L.n_chunks);     // bit ks*16 + r: block (range r, K slice ks) exists
+  std::vector<int32_t> slot(size_t(Ks) * L.n_chunks);
+  for (int b = 0; b < L.n_bundles; ++b) {
+    const int m_lo = b * n_tile, m_hi = std::min(p->M, m_lo + n_tile);
+    const int n_ranges = ceil_div(m_hi - m_lo, kSubRange);
+    const int p_lo = m_lo / p->g_m, p_hi = ceil_div(m_hi, p->g_m);
+    // pass 1: which (range, K slice) blocks exist in which (location, chunk) step
+    std::fill(pres.begin(), pres.end(), uint64_t(0));
+    for (int pr = p_lo; pr < p_hi; ++pr) {
+      const int r_lo = (std::max(pr * p->g_m, m_lo) - m_lo) / kSubRange;
+      const int r_hi = (std::min(std::min((pr + 1) * p->g_m, p->M), m_hi) - 1 - m_lo) / kSubRange;
+      uint64_t rbits = 0;
+      for (int r = r_lo; r <= r_hi; ++r) rbits |= uint64_t(1) << r;
+      for (int q = 0; q < p->Q; ++q) {
+        const int c_lo = q * p->g_n, c_hi = std::min(p->N, c_lo + p->g_n);
+        for (int32_t e = p->group_ptr[size_t(pr) * p->Q + q]; e < p->group_ptr[size_t(pr) * p->Q + q + 1]; ++e)
+          for (int sl = c_lo / 16; sl <= (c_hi - 1) / 16; ++sl)       // 16-channel slices the group touches
+            pres[size_t(p->pos_idx[e]) * L.n_chunks + sl / 4] |= rbits << ((sl % 4) * 16);
+      }
+    }
+    const int32_t first_step = int32_t(L.steps.size());
+    for (int ch = 0; ch < L.n_chunks; ++ch)
+      for (int kpos = 0; kpos < Ks; ++kpos) {
+        uint64_t m = pres[size_t(kpos) * L.n_chunks + ch];
+        slot[size_t(kpos) * L.n_chunks + ch] = -1;
+        if (!m) continue;
+        if (int32_t(L.steps.size()) == first_step) {          // first step: every range starts its accumulator here
+          m |= (uint64_t(1) << n_ranges) - 1;
+          pres[size_t(kpos) * L.n_chunks + ch] = m;
+        }
+        slot[size_t(kpos) * L.n_chunks + ch] = int32_t(L.steps.size());
+        const int kw = kpos % p->Kw, kh = (kpos / p->Kw) % p->Kh, kt = kpos / (p->Kw * p->Kh);
+        SubStep st{};
+        st.enc = encode_step(kt, kh, kw, ch);
+        st.off64 = unsigned(L.payload.size() / 64);
+        st.nblk = __builtin_popcountll(m);
+        L.steps.push_back(st);
+        L.max_blocks = std::max(L.max_blocks, st.nblk);
+        const size_t base = L.payload.size();
+        L.payload.resize(base + kSubHeaderBytes + size_t(st.nblk) * kSubBlockBytes, 0);
+        int idx = 0;
+        for (int bit = 0; bit < 64; ++bit)
+          if ((m >> bit) & 1) L.payload[base + size_t(4 * (bit % 16) + bit / 16)] = uint8_t(0x80 | idx++);
+      }
+    const int32_t end_step = int32_t(L.steps.size());
+    L.step_ptr[b + 1] = end_step;
+    L.max_steps = std::max(L.max_steps, int(end_step - first_step));
+    // pass 2: scatter the kept weights into their blocks
+    for (int pr = p_lo; pr < p_hi; ++pr)
+      for (int q = 0; q < p->Q; ++q)
+        for (int32_t e = p->group_ptr[size_t(pr) * p->Q + q]; e < p->group_ptr[size_t(pr) * p->Q + q + 1]; ++e)
+          for (int i = 0; i < p->g_m; ++i) {
+            const int m = pr * p->g_m + i;
+            if (m < m_lo || m >= m_hi) continue;
+            const int r = (m - m_lo) / kSubRange, ri = (m - m_lo) % kSubRange;
+            for (int j = 0; j < p->g_n; ++j) {
+              const int c = q * p->g_n + j;
+              if (c >= p->N) continue;
+              const SubStep& st = L.steps[slot[size_t(p->pos_idx[e]) * L.n_chunks + c / kChunk]];
+              const size_t base = size_t(st.off64) * 64;
+              const int ks = (c % kChunk) / 16, kj = c % 16;
+              const size_t blk = L.payload[base + size_t(4 * r + ks)] & 0x3F;
+              uint16_t* dst = reinterpret_cast<uint16_t*>(L.payload.data() + base + kSubHeaderBytes + blk * kSubBlockBytes);
+              dst[((ri / 8) * 2 + kj / 8) * 64 + (ri % 8) * 8 + kj % 8] = tiles[(int64_t(e) * p->g_m + i) * p->g_n + j];
+            }
+          }
+  }
+  auto res = p->sub_layouts.emplace(n_tile, std::move(L));
+  return &res.first->second;
+}
+
 // Small-C_in layout for spatial strides (sh, sw): kernel locations kept by at least one group are
 // sorted by the offset of their window inside the staged phase images and paired; each pair is one
 // K=16 MMA whose two K halves are the 8 (padded) channels at the two locations.  Operands use the
@@ -284,6 +371,43 @@ rt3d_status rt3d_unpack_device_layout(const rt3d_packed* p, int n_tile, float* w
           w_out[(int64_t(b * L->n_tile + r) * p->N + (ch * kChunk + j)) * p->Ks + kpos] =
               bf16_bits_to_f32(L->wtiles[(size_t(s) * L->n_tile + r) * kChunk + j]);
     }
+  return RT3D_OK;
+}
+
+rt3d_status rt3d_unpack_sub_layout(const rt3d_packed* p, int n_tile, float* w_out) {
+  if (!p || !w_out) return RT3D_ERR_INVALID_ARG;
+  const SubLayout* L = get_sub_layout(const_cast<rt3d_packed*>(p), n_tile);
+  if (!L) return RT3D_ERR_UNSUPPORTED;
+  std::memset(w_out, 0, sizeof(float) * size_t(p->M) * p->N * p->Ks);
+  for (int b = 0; b < L->n_bundles; ++b) {
+    const int n_ranges = ceil_div(std::min(L->n_tile, p->M - b * L->n_tile), kSubRange);
+    for (int32_t s = L->step_ptr[b]; s < L->step_ptr[b + 1]; ++s) {
+      const SubStep& st = L->steps[s];
+      int kt, kh, kw, ch;
+      decode_step(st.enc, kt, kh, kw, ch);
+      const int kpos = (kt * p->Kh + kh) * p->Kw + kw;
+      const unsigned char* hdr = L->payload.data() + size_t(st.off64) * 64;
+      int seen = 0;
+      for (int r = 0; r < 16; ++r)
+        for (int ks = 0; ks < 4; ++ks) {
+          const unsigned char cmd = hdr[4 * r + ks];
+          // the first step of a bundle must start every range's accumulator in K slice 0
+          if (s == L->step_ptr[b] && ks == 0 && r < n_ranges && !(cmd & 0x80)) return RT3D_ERR_INVALID_ARG;
+          if (!(cmd & 0x80)) continue;
+          if (r >= n_ranges || (cmd & 0x3F) >= st.nblk) return RT3D_ERR_INVALID_ARG;
+          ++seen;
+          const uint16_t* blk = reinterpret_cast<const uint16_t*>(hdr + kSubHeaderBytes + size_t(cmd & 0x3F) * kSubBlockBytes);
+          for (int i = 0; i < 16; ++i)
+            for (int j = 0; j < 16; ++j) {
+              const int m = b * L->n_tile + r * 16 + i, c = ch * kChunk + ks * 16 + j;
+              const float v = bf16_bits_to_f32(blk[((i / 8) * 2 + j / 8) * 64 + (i % 8) * 8 + j % 8]);
+              if (m < p->M && c < p->N) w_out[(int64_t(m) * p->N + c) * p->Ks + kpos] += v;
+              else if (v != 0.f) return RT3D_ERR_INVALID_ARG;
+            }
+        }
+      if (seen != st.nblk) return RT3D_ERR_INVALID_ARG;
+    }
+  }
   return RT3D_OK;
 }
 

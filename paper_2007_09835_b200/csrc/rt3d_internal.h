@@ -61,6 +61,21 @@ struct SmallCLayout {
   std::vector<uint16_t> wimg;        // [n_pairs][2][n_pad/8][8][8] bf16 bits, zero where pruned / absent
 };
 
+// Layout consumed by the sub-tile kernel: per bundle of n_tile output channels the list of non-empty K steps in
+// chunk-major order (all kernel locations of a 64-channel chunk, then the next chunk: the input block under a
+// tile is then re-read from the L1 cache), each with its block mask, and the blocks themselves.  A block holds
+// W[16 output channels][16 input channels] of one kernel location as four 8 x 8 core matrices
+// [row group][K half][8 rows][8 channels] (no-swizzle K-major operand: 128 bytes between K halves, 256 between
+// row groups).
+struct SubLayout {
+  int n_tile = 0, n_bundles = 0, n_chunks = 0;
+  std::vector<int32_t> step_ptr;     // [n_bundles + 1]
+  std::vector<SubStep> steps;
+  std::vector<unsigned char> payload; // per step: 64-byte header + its blocks ([nblk][256] bf16 bits)
+  int max_blocks = 0;                // most blocks in one step
+  int max_steps = 0;                 // longest bundle list
+};
+
 // Per-device copies of a handle's arrays.
 struct DeviceBlob {
   int device = -1;
@@ -76,6 +91,8 @@ struct DeviceBlob {
     bool ready = false;
   };
   std::map<int, Umma> umma;          // keyed by n_tile
+  struct Sub { void* steps = nullptr; int32_t* step_ptr = nullptr; void* blocks = nullptr; bool ready = false; };
+  std::map<int, Sub> sub;            // sub-tile kernel, keyed by n_tile
   struct SmallC { void* wimg = nullptr; int32_t* pairs = nullptr; };
   std::map<int, SmallC> smallc;      // small-C_in kernel: weight image and pair offsets, keyed by sh*16+sw
   float* splitk = nullptr; size_t splitk_bytes = 0;            // split-K partial tiles (grown on demand)
@@ -100,6 +117,7 @@ struct rt3d_packed {
   std::vector<unsigned char> tiles;  // nnz * g_m * g_n elements of float or bf16 bits
   std::mutex mu;                     // guards the lazily built members below
   std::map<int, rt3d::UmmaLayout> umma_layouts;   // keyed by n_tile
+  std::map<int, rt3d::SubLayout> sub_layouts;     // keyed by n_tile
   std::map<int, rt3d::SmallCLayout> smallc_layouts;   // keyed by sh*16+sw, built on first use
   std::vector<rt3d::DeviceBlob*> blobs;
 };
@@ -111,6 +129,9 @@ int default_n_tile(int M);
 // Builds (or returns the cached) tensor-core layout; nullptr if the handle cannot use it.
 const UmmaLayout* get_umma_layout(rt3d_packed* p, int n_tile);
 bool umma_layout_possible(const rt3d_packed* p);
+// Builds (or returns the cached) layout of the sub-tile kernel; nullptr if the handle cannot use it.
+const SubLayout* get_sub_layout(rt3d_packed* p, int n_tile);
+
 // Small-C_in layout (nullptr if the handle does not qualify: needs bf16, N <= 8, M <= 256).
 const SmallCLayout* get_smallc_layout(rt3d_packed* p, int sh, int sw);
 

@@ -93,3 +93,15 @@ def test_vanilla_high_rate_skips_steps_in_layout():
     L = synth.make_layer(spec, 9, 1, 4, 4, "vanilla_total", (16 * 64) // 8)
     pk = rt3d.rt3d_pack_kgs(L["w"], L["mask"], 4, 4, rt3d.RT3D_BF16)
     np.testing.assert_array_equal(pk.unpack_device_layout(16), oracle.bf16_round(L["w"] * L["mask"]))
+
+
+@pytest.mark.parametrize("M,N,k,g_m,g_n,density", [(256, 256, (3, 3, 3), 8, 8, 0.125), (256, 128, (3, 3, 3), 4, 4, 0.4),
+                                                   (230, 72, (1, 3, 3), 8, 4, 0.2), (64, 40, (3, 1, 1), 8, 8, 0.3),
+                                                   (512, 64, (3, 3, 3), 64, 64, 0.5), (40, 16, (3, 3, 3), 8, 8, 0.05),
+                                                   (300, 256, (3, 3, 3), 16, 16, 0.25)])
+def test_sub_tile_layout_holds_exactly_the_masked_weights(M, N, k, g_m, g_n, density):
+    # blocks of 16 x 16 channels + per-step command headers: rebuilt weights equal W * mask after bf16 rounding, and the
+    # library's own consistency checks (first step starts every range, block indices in range, zeros outside) pass
+    L = _layer(M, N, k, g_m, g_n, density, 3)
+    pk = rt3d.rt3d_pack_kgs(L["w"], L["mask"], g_m, g_n, rt3d.RT3D_BF16)
+    np.testing.assert_array_equal(pk.unpack_sub_layout(0), oracle.bf16_round(L["w"] * L["mask"]))
