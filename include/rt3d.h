@@ -88,6 +88,9 @@ typedef struct {
                             hold zeros.  Never needed for correctness (by default no kernel lets them
                             reach the result); it lets the small-C_in kernel fetch whole image rows in
                             one request instead of one voxel at a time                              */
+  int32_t concurrent;    /* nonzero: other kernels may run on the device while this call does (parallel
+                            streams).  The library then avoids plans whose CTAs wait for one another (the
+                            tail split of the CTA-pair kernel), which need the whole grid resident at once */
 } rt3d_conv_params;
 
 typedef struct rt3d_packed rt3d_packed;   /* opaque; immutable after creation */
@@ -112,7 +115,7 @@ typedef struct {
  * (P = ceil(M/g_m), Q = ceil(N/g_n), Section 4); inside a group every kernel location
  * (kt,kh,kw) is kept or pruned for all kernels together, which is whole-column removal in
  * the group's weight matrix.  The pack keeps, per group, the list of kept locations and one
- * compact g_m x g_n tile per kept location (the "reorganize the model weights" step of
+ * compact g_m x g_n tile per kept location (the compile-time weight reordering step of
  * Section 5.2).  Vanilla sparsity (whole groups removed) is the special case where each
  * group keeps all or no locations.
  *   w     host, [M][N][Kt][Kh][Kw] float
@@ -152,15 +155,18 @@ rt3d_status rt3d_unpack_device_layout(const rt3d_packed* p, int n_tile, float* w
 rt3d_status rt3d_unpack_sub_layout(const rt3d_packed* p, int n_tile, float* w_out);
 
 /* Upload the handle's device blobs to the current CUDA device now (otherwise done by the
- * first compute call).  Synchronises the device. */
+ * first compute call), and look up, once per device, the device address of the fixed workspace of
+ * rt3d_conv3d_sparse_noalloc (that look-up may make the CUDA runtime load this library's module on the
+ * device, which is when the driver sets the workspace's memory aside).  Call it before any stream capture.
+ * Synchronises the device. */
 rt3d_status rt3d_packed_prepare(rt3d_packed* p);
 
 void rt3d_packed_free(rt3d_packed* p);
 
 /*
  * rt3d_conv3d_sparse - the hot path: y = act(bias + conv3d(x, W (.) mask)), iterating only
- * the kept (group, location) entries of the packed index (Section 3: after column removal
- * "the remaining computation is still based on full matrices (albeit smaller)").
+ * the kept (group, location) entries of the packed index (Section 3: pruning a location in a group removes
+ * a whole column of the group's weight matrix, and what is left is again a dense, only smaller, product).
  *   x, y   device tensors; x.c == N, y.c == M, y extents = output extents of (x, params);
  *          dtypes equal the handle's compute dtype.  bf16: c_stride multiple of 8, fp32:
  *          multiple of 4; data 16-byte aligned.  x and y must not overlap.
@@ -182,8 +188,8 @@ rt3d_status rt3d_conv3d_dense(const rt3d_tensor* x, const rt3d_packed* w, const 
                               const rt3d_conv_params* p, rt3d_tensor* y, void* stream);
 
 /*
- * Fused layer boundaries (the paper's framework applies "computational graph optimizations",
- * Section 5.2, without detailing them; these two are the ones its models need).
+ * Fused layer boundaries (Section 5.2 says the paper's framework optimises the computation graph
+ * without detailing how; these two fusions are the ones its models need).
  *   residual  device tensor with the extents, dtype and alignment rules of the un-pooled output
  *             (c == M), added to conv + bias BEFORE the ReLU of p->relu; NULL = none.  Must not
  *             overlap y.  (R(2+1)D block end: y = relu(conv(x) + shortcut).)
@@ -251,11 +257,13 @@ rt3d_status rt3d_conv2plus1d_fused(const rt3d_tensor* x, const rt3d_packed* w_s,
  *     (fp32, channel pitch not a multiple of 8, p->algo == RT3D_ALGO_SIMT) give RT3D_ERR_UNSUPPORTED.
  *   - K is split S ways, S = min(8, SMs / output tiles, K steps / 8), at least 1, where an output
  *     tile is 128 voxels x up to 256 channels and a K step is one kernel location x 64 input
- *     channels.  If S > 1 and (output tiles x S) partial tiles of 128 x n_tile floats exceed
+ *     channels that some kernel group of the tile's channels keeps (the longest such list counts).  If S > 1 and (output tiles x S) partial tiles of 128 x n_tile floats exceed
  *     16 MiB, or there are more than 128 output tiles, the call is rejected with
  *     RT3D_ERR_WORKSPACE and nothing is launched (rt3d_conv3d_sparse has no such limit).
- *   - The first call on a device looks up the device address of the workspace; make that first
- *     call before any stream capture begins.  No call allocates or frees device or pinned memory.
+ *   - The device address of the workspace is looked up by rt3d_packed_prepare (once per device, with that
+ *     device current; do it before any stream capture begins).  This entry point itself never allocates
+ *     or frees device or pinned memory and never triggers that look-up: without a prepared handle on the
+ *     device it returns RT3D_ERR_NOT_PREPARED.
  *   - All calls on a device share the one workspace, which keeps the previous call's contents; the
  *     entry point clears the counters it needs on `stream` before the kernel.  Two calls whose
  *     kernels may overlap on the GPU (different streams) race on it: serialise them.
@@ -340,6 +348,27 @@ rt3d_status rt3d_last_device_status(void* stream);
 
 /* Number of kernels this library has launched in this process (all devices). */
 int64_t rt3d_launch_count(void);
+
+/* Number of device allocations (cudaMalloc calls) this library has made in this process. */
+int64_t rt3d_alloc_count(void);
+
+/* Planning mode of the calling thread.  Between rt3d_plan_begin and rt3d_plan_end every compute call of this
+ * library (convolutions, fused pair, pool, add) validates its arguments, chooses its kernel, builds and uploads
+ * the weight layout that kernel needs and sizes the K-split / tail-split workspace of the handle exactly as the
+ * real call would, but launches nothing and touches no activation.  Running a network's sequence of calls once in
+ * planning mode (same shapes, same parameters) therefore moves every allocation and upload out of the later real
+ * calls: afterwards rt3d_alloc_count does not change while those calls run.  rt3d_last_plan reports the planned
+ * kernel.  (The paper's counterpart is its compile-time "tuning of the computation configuration", Section 5.2.) */
+void rt3d_plan_begin(void);
+void rt3d_plan_end(void);
+
+/* Test hooks; no effect on results.  RT3D_DEBUG_WAIT_CYCLES: SM clocks after which a wait inside the single-CTA
+ * tensor-core kernel gives up (0 = default, about one second; the environment variable
+ * RT3D_DEBUG_TIMEOUT_POLLS sets the initial value).  RT3D_DEBUG_DROP_LAST_LOAD: nonzero makes that kernel's
+ * producer skip the loads of each CTA's last pipeline stage, so that the wait on them runs out and the error
+ * path (RT3D_ERR_TIMEOUT from rt3d_last_device_status) can be exercised without any fault. */
+enum { RT3D_DEBUG_WAIT_CYCLES = 1, RT3D_DEBUG_DROP_LAST_LOAD = 2 };
+rt3d_status rt3d_debug_set(int what, long long value);
 
 const char* rt3d_status_string(rt3d_status s);
 const char* rt3d_version(void);

@@ -7,8 +7,10 @@ library; there is no fallback: if librt3d.so is missing the import of this modul
 """
 from __future__ import annotations
 
+import contextlib
 import ctypes
 import os
+import threading
 
 import numpy as np
 
@@ -36,7 +38,8 @@ class Tensor(ctypes.Structure):
 class ConvParams(ctypes.Structure):
     _fields_ = [("st", ctypes.c_int32), ("sh", ctypes.c_int32), ("sw", ctypes.c_int32),
                 ("pt", ctypes.c_int32), ("ph", ctypes.c_int32), ("pw", ctypes.c_int32),
-                ("relu", ctypes.c_int32), ("algo", ctypes.c_int32), ("x_pad_zero", ctypes.c_int32)]
+                ("relu", ctypes.c_int32), ("algo", ctypes.c_int32), ("x_pad_zero", ctypes.c_int32),
+                ("concurrent", ctypes.c_int32)]
 
 
 class Fusion(ctypes.Structure):
@@ -86,6 +89,10 @@ def _load():
     lib.rt3d_last_plan.argtypes = [ctypes.POINTER(PlanInfo)]
     lib.rt3d_last_device_status.argtypes = [vp]
     lib.rt3d_launch_count.restype = ctypes.c_int64
+    lib.rt3d_alloc_count.restype = ctypes.c_int64
+    lib.rt3d_plan_begin.restype = None
+    lib.rt3d_plan_end.restype = None
+    lib.rt3d_debug_set.argtypes = [i, ctypes.c_longlong]
     lib.rt3d_status_string.restype = ctypes.c_char_p
     lib.rt3d_status_string.argtypes = [i]
     lib.rt3d_version.restype = ctypes.c_char_p
@@ -219,9 +226,35 @@ def channel_slice_desc(t, offset: int, c: int) -> Tensor:
     return Tensor(t.data_ptr() + offset * es, d.n, d.t, d.h, d.w, int(c), d.c_stride, d.dtype)
 
 
+_concurrent = threading.local()
+
+
+@contextlib.contextmanager
+def concurrent_kernels():
+    """Convolution calls made by this thread inside the block tell the library that other kernels may run on the
+    device at the same time (parallel streams): it then avoids plans whose CTAs wait for one another."""
+    prev = getattr(_concurrent, "on", False)
+    _concurrent.on = True
+    try:
+        yield
+    finally:
+        _concurrent.on = prev
+
+
+@contextlib.contextmanager
+def planning():
+    """Planning mode (rt3d_plan_begin / rt3d_plan_end): compute calls inside the block choose their kernels, upload
+    their weight layouts and size their workspaces but launch nothing."""
+    _lib.rt3d_plan_begin()
+    try:
+        yield
+    finally:
+        _lib.rt3d_plan_end()
+
+
 def _params(stride, pad, relu, algo, x_pad_zero=False) -> ConvParams:
     return ConvParams(int(stride[0]), int(stride[1]), int(stride[2]), int(pad[0]), int(pad[1]), int(pad[2]),
-                      int(bool(relu)), int(algo), int(bool(x_pad_zero)))
+                      int(bool(relu)), int(algo), int(bool(x_pad_zero)), int(getattr(_concurrent, "on", False)))
 
 
 def _stream_ptr(stream):
@@ -350,6 +383,17 @@ def rt3d_last_device_status(stream=None) -> int:
 
 def rt3d_launch_count() -> int:
     return int(_lib.rt3d_launch_count())
+
+
+def rt3d_alloc_count() -> int:
+    return int(_lib.rt3d_alloc_count())
+
+
+DEBUG_WAIT_CYCLES, DEBUG_DROP_LAST_LOAD = 1, 2
+
+
+def rt3d_debug_set(what: int, value: int):
+    _check(_lib.rt3d_debug_set(int(what), int(value)), "rt3d_debug_set")
 
 
 def rt3d_version() -> str:

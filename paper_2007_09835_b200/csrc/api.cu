@@ -19,6 +19,37 @@ using namespace rt3d;
 namespace {
 
 std::atomic<int64_t> g_launches{0};
+std::atomic<int64_t> g_allocs{0};            // device allocations made by this library (rt3d_alloc_count)
+
+// Every device allocation of the library goes through here.
+cudaError_t dev_malloc(void** p, size_t bytes) {
+  g_allocs.fetch_add(1);
+  return cudaMalloc(p, bytes);
+}
+template <typename T>
+cudaError_t dev_malloc(T** p, size_t bytes) { return dev_malloc(reinterpret_cast<void**>(p), bytes); }
+
+// Planning mode of the calling thread (rt3d_plan_begin / rt3d_plan_end): compute calls do everything they would do
+// before their launch (choose the kernel, build and upload weight layouts, size the workspaces) and return.
+thread_local bool t_plan_only = false;
+
+// Test hooks of the single-CTA tensor-core kernel (rt3d_debug_set).
+std::atomic<long long> g_debug_wait_cycles{-1};      // -1: not set yet (RT3D_DEBUG_TIMEOUT_POLLS is read on first use)
+std::atomic<int> g_debug_drop_last_load{0};
+long long debug_wait_cycles() {
+  long long v = g_debug_wait_cycles.load();
+  if (v < 0) {
+    const char* e = getenv("RT3D_DEBUG_TIMEOUT_POLLS");
+    v = e ? atoll(e) : 0;
+    if (v < 0) v = 0;
+    g_debug_wait_cycles.store(v);
+  }
+  return v;
+}
+
+// All device blobs of live handles: their K-split counters are cleared when a kernel reported a timeout.
+std::mutex g_blobs_mu;
+std::vector<DeviceBlob*> g_blobs;
 
 struct DeviceState {
   bool init = false;
@@ -42,7 +73,7 @@ rt3d_status get_device_state(DeviceState** out) {
   if (!d.init) {
     if (cudaDeviceGetAttribute(&d.sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return RT3D_ERR_CUDA;
     if (cudaDeviceGetAttribute(&d.cc_major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return RT3D_ERR_CUDA;
-    if (cudaMalloc(&d.sched, 256 * sizeof(int32_t)) != cudaSuccess) return RT3D_ERR_ALLOC;
+    if (dev_malloc(&d.sched, 256 * sizeof(int32_t)) != cudaSuccess) return RT3D_ERR_ALLOC;
     if (cudaMemset(d.sched, 0, 256 * sizeof(int32_t)) != cudaSuccess) return RT3D_ERR_CUDA;
     if (!g_encode) {
       void* fn = nullptr;
@@ -132,9 +163,9 @@ rt3d_status get_blob(rt3d_packed* h, DeviceBlob** out) {
     if (!b) return RT3D_ERR_ALLOC;
     b->device = dev;
     rt3d_status s = RT3D_OK;
-    if (cudaMalloc(reinterpret_cast<void**>(&b->group_ptr), h->group_ptr.size() * 4) != cudaSuccess ||
-        cudaMalloc(reinterpret_cast<void**>(&b->pos_idx), h->pos_idx.size() * 2 + 16) != cudaSuccess ||
-        cudaMalloc(&b->tiles, h->tiles.size() + 16) != cudaSuccess)
+    if (dev_malloc(&b->group_ptr, h->group_ptr.size() * 4) != cudaSuccess ||
+        dev_malloc(&b->pos_idx, h->pos_idx.size() * 2 + 16) != cudaSuccess ||
+        dev_malloc(&b->tiles, h->tiles.size() + 16) != cudaSuccess)
       s = RT3D_ERR_ALLOC;
     if (s == RT3D_OK &&
         (cudaMemcpy(b->group_ptr, h->group_ptr.data(), h->group_ptr.size() * 4, cudaMemcpyHostToDevice) != cudaSuccess ||
@@ -147,6 +178,8 @@ rt3d_status get_blob(rt3d_packed* h, DeviceBlob** out) {
       return s;
     }
     h->blobs.push_back(b);
+    std::lock_guard<std::mutex> reg(g_blobs_mu);
+    g_blobs.push_back(b);
   }
   *out = b;
   return RT3D_OK;
@@ -157,9 +190,9 @@ rt3d_status get_umma_blob(rt3d_packed* h, DeviceBlob* blob, const UmmaLayout* L,
   DeviceBlob::Umma& u = blob->umma[L->n_tile];
   if (!u.ready) {
     const size_t wbytes = L->wtiles.size() * 2;
-    if (cudaMalloc(&u.wtiles, wbytes + 1024) != cudaSuccess ||
-        cudaMalloc(reinterpret_cast<void**>(&u.step_ptr), L->step_ptr.size() * 4) != cudaSuccess ||
-        cudaMalloc(reinterpret_cast<void**>(&u.steps), L->steps.size() * 4 + 16) != cudaSuccess)
+    if (dev_malloc(&u.wtiles, wbytes + 1024) != cudaSuccess ||
+        dev_malloc(&u.step_ptr, L->step_ptr.size() * 4) != cudaSuccess ||
+        dev_malloc(&u.steps, L->steps.size() * 4 + 16) != cudaSuccess)
       return RT3D_ERR_ALLOC;
     if ((wbytes && cudaMemcpy(u.wtiles, L->wtiles.data(), wbytes, cudaMemcpyHostToDevice) != cudaSuccess) ||
         cudaMemcpy(u.step_ptr, L->step_ptr.data(), L->step_ptr.size() * 4, cudaMemcpyHostToDevice) != cudaSuccess ||
@@ -195,9 +228,9 @@ rt3d_status get_sub_blob(rt3d_packed* h, DeviceBlob* blob, const SubLayout* L, D
   DeviceBlob::Sub& u = blob->sub[L->n_tile];
   if (!u.ready) {
     const size_t sbytes = L->steps.size() * sizeof(SubStep), bbytes = L->payload.size();
-    if (cudaMalloc(&u.steps, sbytes + 64) != cudaSuccess ||
-        cudaMalloc(reinterpret_cast<void**>(&u.step_ptr), L->step_ptr.size() * 4) != cudaSuccess ||
-        cudaMalloc(&u.blocks, bbytes + 512) != cudaSuccess)
+    if (dev_malloc(&u.steps, sbytes + 64) != cudaSuccess ||
+        dev_malloc(&u.step_ptr, L->step_ptr.size() * 4) != cudaSuccess ||
+        dev_malloc(&u.blocks, bbytes + 512) != cudaSuccess)
       return RT3D_ERR_ALLOC;
     if ((sbytes && cudaMemcpy(u.steps, L->steps.data(), sbytes, cudaMemcpyHostToDevice) != cudaSuccess) ||
         cudaMemcpy(u.step_ptr, L->step_ptr.data(), L->step_ptr.size() * 4, cudaMemcpyHostToDevice) != cudaSuccess ||
@@ -384,8 +417,8 @@ rt3d_status launch_smallc(rt3d_packed* w, DeviceBlob* blob, const DeviceState* d
     if (!sc->wimg) {
       void* wi = nullptr;
       int32_t* po = nullptr;
-      if (cudaMalloc(&wi, L->wimg.size() * 2 + 16) != cudaSuccess ||
-          cudaMalloc(reinterpret_cast<void**>(&po), L->pair_off.size() * 4 + 16) != cudaSuccess)
+      if (dev_malloc(&wi, L->wimg.size() * 2 + 16) != cudaSuccess ||
+          dev_malloc(&po, L->pair_off.size() * 4 + 16) != cudaSuccess)
         return RT3D_ERR_ALLOC;
       if ((!L->wimg.empty() && cudaMemcpy(wi, L->wimg.data(), L->wimg.size() * 2, cudaMemcpyHostToDevice) != cudaSuccess) ||
           (!L->pair_off.empty() &&
@@ -432,6 +465,7 @@ rt3d_status launch_smallc(rt3d_packed* w, DeviceBlob* blob, const DeviceState* d
   const int sb[4] = {kSmallCTileW, 4, 1, 1};          // a warp owns 4 rows of 8 voxels of the 16 x 8 tile
   a.store_tma = encode_ymap(y, sb, pool_w, pool_h, 1, &ymap) ? 1 : 0;
   if (!a.store_tma && pool_h * pool_w > 1) return RT3D_ERR_UNSUPPORTED;
+  if (t_plan_only) return RT3D_OK;
   if (launch_conv_umma_smallc(a, &xmap, a.store_tma ? &ymap : nullptr, d->sm_count, st) != cudaSuccess) return RT3D_ERR_CUDA;
   g_launches.fetch_add(1);
   return RT3D_OK;
@@ -446,13 +480,13 @@ rt3d_status ensure_splitk(rt3d_packed* w, DeviceBlob* blob, size_t bytes, size_t
   if (blob->splitk_bytes < bytes) {
     cudaFree(blob->splitk);
     blob->splitk = nullptr; blob->splitk_bytes = 0;
-    if (cudaMalloc(reinterpret_cast<void**>(&blob->splitk), bytes) != cudaSuccess) return RT3D_ERR_ALLOC;
+    if (dev_malloc(&blob->splitk, bytes) != cudaSuccess) return RT3D_ERR_ALLOC;
     blob->splitk_bytes = bytes;
   }
   if (blob->splitk_cnt_bytes < cnt_bytes) {
     cudaFree(blob->splitk_cnt);
     blob->splitk_cnt = nullptr; blob->splitk_cnt_bytes = 0;
-    if (cudaMalloc(reinterpret_cast<void**>(&blob->splitk_cnt), cnt_bytes) != cudaSuccess) return RT3D_ERR_ALLOC;
+    if (dev_malloc(&blob->splitk_cnt, cnt_bytes) != cudaSuccess) return RT3D_ERR_ALLOC;
     if (cudaMemset(blob->splitk_cnt, 0, cnt_bytes) != cudaSuccess) return RT3D_ERR_CUDA;
     blob->splitk_cnt_bytes = cnt_bytes;
   }
@@ -506,6 +540,7 @@ rt3d_status try_halo(rt3d_packed* w, DeviceBlob* blob, DeviceState* d, const rt3
   a.pool_t = a.pool_h = a.pool_w = 1;
   a.n_splits = 1; a.scratch = nullptr; a.counters = nullptr;
   a.tail_workers = 0; a.tail_scratch = nullptr; a.tail_flags = nullptr;
+  a.wait_cycles = 0; a.debug_drop_last_load = 0;
   ConvGeom unit = g;                       // the staged block is a plain box of input voxels
   CUtensorMap xmap, ymap;
   if ((s = encode_xmap(x, unit, TileBox{1, h.ht, h.hh, h.hw}, &xmap)) != RT3D_OK) return s;
@@ -513,11 +548,12 @@ rt3d_status try_halo(rt3d_packed* w, DeviceBlob* blob, DeviceState* d, const rt3
   const bool rect = warp_block(a.box.bw, a.box.bh, a.box.bt, a.box.bn, sb);
   a.sbw = sb[0]; a.sbh = sb[1];
   a.store_tma = (rect && encode_ymap(y, sb, 1, 1, 1, &ymap)) ? 1 : 0;
+  t_last_plan = rt3d_plan_info{4, a.n_tile, 1, 0, 0};
+  *launched = true;
+  if (t_plan_only) return RT3D_OK;
   cudaError_t e = launch_conv_umma_halo(h, &xmap, u->wmap_half, a.store_tma ? &ymap : nullptr, d->sm_count, st);
   if (e != cudaSuccess) return RT3D_ERR_CUDA;
   g_launches.fetch_add(1);
-  t_last_plan = rt3d_plan_info{4, a.n_tile, 1, 0, 0};
-  *launched = true;
   return RT3D_OK;
 }
 
@@ -552,12 +588,11 @@ rt3d_status try_sub(rt3d_packed* w, DeviceBlob* blob, DeviceState* d, const rt3d
   int sb[4] = {1, 1, 1, 1};
   const bool rect = warp_block(a.box.bw, a.box.bh, a.box.bt, a.box.bn, sb);
   a.store_tma = (rect && encode_ymap(y, sb, 1, 1, 1, &ymap)) ? 1 : 0;
-  int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess) return RT3D_ERR_CUDA;
-  if (launch_conv_umma_sub(a, &xmap, a.store_tma ? &ymap : nullptr, d->sm_count, dev, st) != cudaSuccess) return RT3D_ERR_CUDA;
-  g_launches.fetch_add(1);
   t_last_plan = rt3d_plan_info{6, a.n_tile, 1, 0, 0};
   *launched = true;
+  if (t_plan_only) return RT3D_OK;
+  if (launch_conv_umma_sub(a, &xmap, a.store_tma ? &ymap : nullptr, d->sm_count, st) != cudaSuccess) return RT3D_ERR_CUDA;
+  g_launches.fetch_add(1);
   return RT3D_OK;
 }
 
@@ -608,6 +643,8 @@ rt3d_status conv_impl(const rt3d_tensor* x, const rt3d_packed* wc, const float* 
   const bool use_umma = want_umma || (p->algo == RT3D_ALGO_AUTO && can_umma);
   if (!use_umma) {
     if (pooled) return RT3D_ERR_UNSUPPORTED;
+    t_last_plan = rt3d_plan_info{0, 0, 1, 0, 0};
+    if (t_plan_only) return RT3D_OK;
     cudaError_t e = launch_conv_simt(w->dtype, g, x->data, y->data, blob->group_ptr, blob->pos_idx, blob->tiles, bias,
                                      w->g_m, w->g_n, w->P, w->Q, dense_entry, res_data, res_pitch, st);
     if (e != cudaSuccess) return RT3D_ERR_CUDA;
@@ -684,6 +721,7 @@ rt3d_status conv_impl(const rt3d_tensor* x, const rt3d_packed* wc, const float* 
   a.residual = res_data; a.rcs = res_pitch;
   a.n_splits = plan.n_splits; a.scratch = nullptr; a.counters = nullptr;
   a.tail_workers = 0; a.tail_scratch = nullptr; a.tail_flags = nullptr;
+  a.wait_cycles = debug_wait_cycles(); a.debug_drop_last_load = g_debug_drop_last_load.load();
   if (a.n_splits > 1) {
     // split-K workspace of this handle on this device: partial tiles + per-warp arrival counters
     const long long tiles = m_tiles * L->n_bundles;
@@ -698,19 +736,22 @@ rt3d_status conv_impl(const rt3d_tensor* x, const rt3d_packed* wc, const float* 
   if (pooled && !a.store_tma) return RT3D_ERR_UNSUPPORTED;
   if (use_pair) {
     // items that do not fill a last round of CTA pairs are cut along K and shared (same workspace as split-K)
+    // (its CTA pairs wait for one another, which needs the whole grid resident at once: not used when the caller
+    // says that other kernels may run beside this call)
     size_t tail_bytes = 0, flag_bytes = 0;
-    umma_pair_tail_plan(&a, L->step_ptr.data(), d->sm_count, &tail_bytes, &flag_bytes);
+    if (!p->concurrent) umma_pair_tail_plan(&a, L->step_ptr.data(), d->sm_count, &tail_bytes, &flag_bytes);
     if (a.tail_workers > 0) {
       if ((s = ensure_splitk(w, blob, tail_bytes, flag_bytes)) != RT3D_OK) return s;
       a.tail_scratch = blob->splitk; a.tail_flags = blob->splitk_cnt;
     }
   }
   const void* ym = a.store_tma ? &ymap : nullptr;
+  t_last_plan = rt3d_plan_info{use_pair ? 2 : 1, a.n_tile, a.n_splits, a.tail_workers, pooled ? 1 : 0};
+  if (t_plan_only) return RT3D_OK;
   cudaError_t e = use_pair ? launch_conv_umma_pair(a, &xmap, u->wmap_half, ym, d->sm_count, st)
                            : launch_conv_umma(a, &xmap, u->wmap, ym, d->sm_count, st);
   if (e != cudaSuccess) return RT3D_ERR_CUDA;
   g_launches.fetch_add(1);
-  t_last_plan = rt3d_plan_info{use_pair ? 2 : 1, a.n_tile, a.n_splits, a.tail_workers, pooled ? 1 : 0};
   return RT3D_OK;
 }
 
@@ -774,13 +815,50 @@ rt3d_status conv2plus1d_impl(const rt3d_tensor* x, const rt3d_packed* wsc, const
   CUtensorMap xmap;
   ConvGeom unit = g;
   if ((s = encode_xmap(x, unit, TileBox{1, 1, a.hh, a.hw}, &xmap)) != RT3D_OK) return s;
+  t_last_plan = rt3d_plan_info{5, a.n1, 1, 0, 0};
+  if (t_plan_only) return RT3D_OK;
   cudaError_t e = launch_conv_umma_st(a, &xmap, u1->wmap_half, u2->wmap_half, d->sm_count, static_cast<cudaStream_t>(stream));
   if (e != cudaSuccess) return RT3D_ERR_CUDA;
   g_launches.fetch_add(1);
-  t_last_plan = rt3d_plan_info{5, a.n1, 1, 0, 0};
   return RT3D_OK;
 }
 
+}  // namespace
+
+// ------------------------------------------------------------------ entry point without allocation
+// Fixed workspace for rt3d_conv3d_sparse_noalloc: split-K partial tiles followed by the per-warp
+// arrival counters.  It lives in every GPU context that loads this library, for the life of the
+// process.  In host code `g_noalloc_ws` is only a handle for the runtime, never a device address:
+// the address is looked up per device with cudaGetSymbolAddress below.
+#define RT3D_NOALLOC_PARTIAL_TILES 128                                   /* 128 x 256 fp32 each */
+#define RT3D_NOALLOC_PARTIAL_BYTES (RT3D_NOALLOC_PARTIAL_TILES * 128 * 256 * 4)   /* 16 MiB */
+#define RT3D_NOALLOC_COUNTER_BYTES (RT3D_NOALLOC_PARTIAL_TILES * 4 * 4)  /* 4 counters per output tile */
+static __device__ __align__(256) unsigned char g_noalloc_ws[RT3D_NOALLOC_PARTIAL_BYTES + RT3D_NOALLOC_COUNTER_BYTES];
+
+namespace {
+struct NoAllocState { bool ready = false; unsigned char* ws = nullptr; };
+NoAllocState g_noalloc[64];
+std::mutex g_noalloc_mu;
+
+// Once per device, with that device current: resolve the device address of the workspace.  Called from
+// rt3d_packed_prepare, the documented set-up point: the first look-up may make the CUDA runtime load this
+// module on the device, which is when the driver sets the array's memory aside.
+rt3d_status noalloc_workspace_setup(int dev) {
+  std::lock_guard<std::mutex> lock(g_noalloc_mu);
+  NoAllocState& st = g_noalloc[dev];
+  if (!st.ready) {
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_noalloc_ws) != cudaSuccess || p == nullptr) return RT3D_ERR_CUDA;
+    st.ws = static_cast<unsigned char*>(p);
+    st.ready = true;
+  }
+  return RT3D_OK;
+}
+// The cached address, or nullptr if no handle has been prepared on this device yet.
+unsigned char* noalloc_workspace(int dev) {
+  std::lock_guard<std::mutex> lock(g_noalloc_mu);
+  return g_noalloc[dev].ready ? g_noalloc[dev].ws : nullptr;
+}
 }  // namespace
 
 extern "C" {
@@ -823,16 +901,16 @@ rt3d_status rt3d_conv3d_host(const rt3d_tensor* x, rt3d_packed* w, const float* 
     if (blob->stage_x_bytes < xb) {
       cudaFree(blob->stage_x);
       blob->stage_x = nullptr; blob->stage_x_bytes = 0;
-      if (cudaMalloc(&blob->stage_x, xb + 256) != cudaSuccess) return RT3D_ERR_ALLOC;
+      if (dev_malloc(&blob->stage_x, xb + 256) != cudaSuccess) return RT3D_ERR_ALLOC;
       blob->stage_x_bytes = xb;
     }
     if (blob->stage_y_bytes < yb) {
       cudaFree(blob->stage_y);
       blob->stage_y = nullptr; blob->stage_y_bytes = 0;
-      if (cudaMalloc(&blob->stage_y, yb + 256) != cudaSuccess) return RT3D_ERR_ALLOC;
+      if (dev_malloc(&blob->stage_y, yb + 256) != cudaSuccess) return RT3D_ERR_ALLOC;
       blob->stage_y_bytes = yb;
     }
-    if (!blob->stage_bias && cudaMalloc(reinterpret_cast<void**>(&blob->stage_bias), size_t(w->M) * 4) != cudaSuccess)
+    if (!blob->stage_bias && dev_malloc(&blob->stage_bias, size_t(w->M) * 4) != cudaSuccess)
       return RT3D_ERR_ALLOC;
   }
   cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -919,6 +997,9 @@ rt3d_status rt3d_packed_prepare(rt3d_packed* p) {
     DeviceBlob::Umma* u = nullptr;
     if (L && (s = get_umma_blob(p, blob, L, &u)) != RT3D_OK) return s;
   }
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return RT3D_ERR_CUDA;
+  if ((s = noalloc_workspace_setup(dev)) != RT3D_OK) return s;
   return cudaDeviceSynchronize() == cudaSuccess ? RT3D_OK : RT3D_ERR_CUDA;
 }
 
@@ -926,6 +1007,11 @@ void rt3d_packed_free(rt3d_packed* p) {
   if (!p) return;
   int cur = -1;
   const bool have_dev = !p->blobs.empty() && cudaGetDevice(&cur) == cudaSuccess;
+  {
+    std::lock_guard<std::mutex> reg(g_blobs_mu);
+    for (DeviceBlob* b : p->blobs)
+      g_blobs.erase(std::remove(g_blobs.begin(), g_blobs.end(), b), g_blobs.end());
+  }
   for (DeviceBlob* b : p->blobs) {
     if (have_dev) cudaSetDevice(b->device);
     cudaFree(b->group_ptr); cudaFree(b->pos_idx); cudaFree(b->tiles);
@@ -955,6 +1041,7 @@ rt3d_status rt3d_maxpool3d(const rt3d_tensor* x, int kt, int kh, int kw, int st,
   if ((To - 1) * st - pt >= x->t || (Ho - 1) * sh - ph >= x->h || (Wo - 1) * sw - pw >= x->w) return RT3D_ERR_SHAPE;
   if ((s = check_alignment(x)) != RT3D_OK || (s = check_alignment(y)) != RT3D_OK) return s;
   if (overlaps(x, y)) return RT3D_ERR_INVALID_ARG;
+  if (t_plan_only) return RT3D_OK;
   cudaError_t e = launch_maxpool3d(x->dtype, x->data, x->n, x->t, x->h, x->w, x->c, x->c_stride, kt, kh, kw, st, sh, sw,
                                    pt, ph, pw, y->data, To, Ho, Wo, y->c_stride, static_cast<cudaStream_t>(stream));
   if (e != cudaSuccess) return RT3D_ERR_CUDA;
@@ -969,6 +1056,7 @@ rt3d_status rt3d_add_relu(const rt3d_tensor* a, const rt3d_tensor* b, int relu, 
   if (a->n != y->n || a->t != y->t || a->h != y->h || a->w != y->w || a->c != y->c || a->dtype != y->dtype) return RT3D_ERR_SHAPE;
   if ((s = check_alignment(a)) != RT3D_OK || (s = check_alignment(b)) != RT3D_OK || (s = check_alignment(y)) != RT3D_OK) return s;
   const int64_t vox = int64_t(a->n) * a->t * a->h * a->w;
+  if (t_plan_only) return RT3D_OK;
   cudaError_t e = launch_add_relu(a->dtype, a->data, a->c_stride, b->data, b->c_stride, y->data, y->c_stride, vox, a->c,
                                   relu ? 1 : 0, static_cast<cudaStream_t>(stream));
   if (e != cudaSuccess) return RT3D_ERR_CUDA;
@@ -1031,40 +1119,20 @@ rt3d_status rt3d_last_device_status(void* stream) {
   if (cudaMemcpy(&word, d->sched + 2, 4, cudaMemcpyDeviceToHost) != cudaSuccess) return RT3D_ERR_CUDA;
   if (word != 0) {
     cudaMemset(d->sched + 2, 0, 4);
+    // A kernel that gave up may have left K-split arrival counters and tail-split flags non-zero (they are
+    // cleared by the CTA that finishes a tile): clear them for every handle on this device, so that later
+    // calls do not take a stale count for "all other splits have arrived".
+    int dev = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess) {
+      cudaDeviceSynchronize();
+      std::lock_guard<std::mutex> reg(g_blobs_mu);
+      for (DeviceBlob* b : g_blobs)
+        if (b->device == dev && b->splitk_cnt) cudaMemset(b->splitk_cnt, 0, b->splitk_cnt_bytes);
+    }
     return RT3D_ERR_TIMEOUT;
   }
   return RT3D_OK;
 }
-
-// ------------------------------------------------------------------ entry point without allocation
-// Fixed workspace for rt3d_conv3d_sparse_noalloc: split-K partial tiles followed by the per-warp
-// arrival counters.  It lives in every GPU context that loads this library, for the life of the
-// process.  In host code `g_noalloc_ws` is only a handle for the runtime, never a device address:
-// the address is looked up per device with cudaGetSymbolAddress below.
-#define RT3D_NOALLOC_PARTIAL_TILES 128                                   /* 128 x 256 fp32 each */
-#define RT3D_NOALLOC_PARTIAL_BYTES (RT3D_NOALLOC_PARTIAL_TILES * 128 * 256 * 4)   /* 16 MiB */
-#define RT3D_NOALLOC_COUNTER_BYTES (RT3D_NOALLOC_PARTIAL_TILES * 4 * 4)  /* 4 counters per output tile */
-static __device__ __align__(256) unsigned char g_noalloc_ws[RT3D_NOALLOC_PARTIAL_BYTES + RT3D_NOALLOC_COUNTER_BYTES];
-
-namespace {
-struct NoAllocState { bool ready = false; unsigned char* ws = nullptr; };
-NoAllocState g_noalloc[64];
-std::mutex g_noalloc_mu;
-
-// Once per device, with that device current: resolve the device address of the workspace.
-rt3d_status noalloc_workspace(int dev, unsigned char** ws) {
-  std::lock_guard<std::mutex> lock(g_noalloc_mu);
-  NoAllocState& st = g_noalloc[dev];
-  if (!st.ready) {
-    void* p = nullptr;
-    if (cudaGetSymbolAddress(&p, g_noalloc_ws) != cudaSuccess || p == nullptr) return RT3D_ERR_CUDA;
-    st.ws = static_cast<unsigned char*>(p);
-    st.ready = true;
-  }
-  *ws = st.ws;
-  return RT3D_OK;
-}
-}  // namespace
 
 rt3d_status rt3d_conv3d_sparse_noalloc(const rt3d_tensor* x, const rt3d_packed* wc, const float* bias,
                                        const rt3d_conv_params* p, rt3d_tensor* y, void* stream) {
@@ -1101,8 +1169,8 @@ rt3d_status rt3d_conv3d_sparse_noalloc(const rt3d_tensor* x, const rt3d_packed* 
     if (li != w->umma_layouts.end()) L = &li->second;
   }
   if (!blob || !u || !L) return RT3D_ERR_NOT_PREPARED;
-  unsigned char* ws = nullptr;
-  if ((s = noalloc_workspace(dev, &ws)) != RT3D_OK) return s;
+  unsigned char* ws = noalloc_workspace(dev);
+  if (!ws) return RT3D_ERR_NOT_PREPARED;
 
   UmmaArgs a;
   a.g = g;
@@ -1115,11 +1183,11 @@ rt3d_status rt3d_conv3d_sparse_noalloc(const rt3d_tensor* x, const rt3d_packed* 
   a.step_ptr = u->step_ptr; a.steps = u->steps;
   a.bias = bias; a.y = y->data; a.sched = d->sched;
   // Split rule of this entry point: as many K splits (at most 8) as keep every SM busy, each with at
-  // least 8 of the layer's K steps.
+  // least 8 of the K steps of the layer's longest step list.
   const long long tiles = (long long)a.tiles_n * a.tiles_t * a.tiles_h * a.tiles_w * L->n_bundles;
   long long splits = tiles > 0 ? d->sm_count / tiles : 1;
   if (splits > 8) splits = 8;
-  if (splits > a.steps_dense / 8) splits = a.steps_dense / 8;
+  if (splits > L->max_steps / 8) splits = L->max_steps / 8;
   if (splits < 1) splits = 1;
   a.n_splits = int(splits);
   a.residual = nullptr; a.rcs = 0;
@@ -1140,14 +1208,27 @@ rt3d_status rt3d_conv3d_sparse_noalloc(const rt3d_tensor* x, const rt3d_packed* 
   int sb[4];
   a.pool_t = a.pool_h = a.pool_w = 1; a.sbw = a.sbh = 1;
   a.tail_workers = 0; a.tail_scratch = nullptr; a.tail_flags = nullptr;
+  a.wait_cycles = 0; a.debug_drop_last_load = 0;
   a.store_tma = (a.n_splits == 1 && warp_block(a.box.bw, a.box.bh, a.box.bt, a.box.bn, sb) &&
                  encode_ymap(y, sb, 1, 1, 1, &ymap)) ? 1 : 0;
   if (launch_conv_umma(a, &xmap, u->wmap, a.store_tma ? &ymap : nullptr, d->sm_count, st) != cudaSuccess) return RT3D_ERR_CUDA;
   g_launches.fetch_add(1);
+  t_last_plan = rt3d_plan_info{1, a.n_tile, a.n_splits, 0, 0};
   return RT3D_OK;
 }
 
 int64_t rt3d_launch_count(void) { return g_launches.load(); }
+
+int64_t rt3d_alloc_count(void) { return g_allocs.load(); }
+
+void rt3d_plan_begin(void) { t_plan_only = true; }
+void rt3d_plan_end(void) { t_plan_only = false; }
+
+rt3d_status rt3d_debug_set(int what, long long value) {
+  if (what == RT3D_DEBUG_WAIT_CYCLES) { if (value < 0) return RT3D_ERR_INVALID_ARG; g_debug_wait_cycles.store(value); return RT3D_OK; }
+  if (what == RT3D_DEBUG_DROP_LAST_LOAD) { g_debug_drop_last_load.store(value != 0); return RT3D_OK; }
+  return RT3D_ERR_INVALID_ARG;
+}
 
 
 const char* rt3d_status_string(rt3d_status s) {

@@ -58,6 +58,8 @@ struct UmmaArgs {
   int tail_workers;                         // CTA-pair kernel: pairs sharing the left-over items of the last round (0 = off)
   float* tail_scratch;                      // device, [tail_workers][2 shares][2 CTAs][n_tile][128] fp32 partial tiles
   int32_t* tail_flags;                      // device, [tail_workers][2][2][4 warps] "partial written" flags, zero between launches
+  long long wait_cycles;                    // single-CTA kernel: SM clocks after which a wait gives up (0 = the default, about 1 s)
+  int debug_drop_last_load;                 // single-CTA kernel, tests only: never issue the loads of each CTA's last stage
 };
 
 // xmap / wmap point to 128-byte CUtensorMap objects in host memory.
@@ -147,7 +149,7 @@ struct SubArgs {
 };
 bool umma_sub_plan(SubArgs* a, int max_blocks);
 // xmap: input tensor map whose box is the tile box (as for the step-list kernels).
-cudaError_t launch_conv_umma_sub(const SubArgs& a, const void* xmap, const void* ymap, int sm_count, int device, cudaStream_t stream);
+cudaError_t launch_conv_umma_sub(const SubArgs& a, const void* xmap, const void* ymap, int sm_count, cudaStream_t stream);
 
 // Arguments of the small-C_in tensor-core kernel (C_in <= 8 at channel pitch 8).
 struct SmallCArgs {

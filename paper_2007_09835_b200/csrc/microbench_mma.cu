@@ -80,6 +80,7 @@ tc_chain_kernel(long long* out, int m, int n, int count, int issuers, int32_t* e
   if (threadIdx.x == 0) {
     for (int q = 0; q < kMaxStages; ++q) { mbar_init(smem_u32(&bars->full[q]), 1); mbar_init(smem_u32(&bars->empty[q]), 1); }
     bars->abort_flag = 0;
+    bars->wait_limit = kWaitCycles;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
@@ -144,6 +145,7 @@ tc_chain_pair_kernel(long long* out, int n, int count, int issuers, int32_t* err
   if (threadIdx.x == 0) {
     for (int q = 0; q < kMaxStages; ++q) mbar_init(smem_u32(&bars->full[q]), 1);
     bars->abort_flag = 0;
+    bars->wait_limit = kWaitCycles;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
@@ -225,6 +227,7 @@ tc_cp_kernel(long long* out, int tiles, int32_t* err) {
   if (threadIdx.x == 0) {
     for (int q = 0; q < 4; ++q) mbar_init(smem_u32(&bars->full[q]), 1);
     bars->abort_flag = 0;
+    bars->wait_limit = kWaitCycles;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -340,6 +343,7 @@ smem_share_kernel(long long* out, int mma_warps, int mma_count, int cp_warps, in
     for (int q = 0; q < kMaxStages; ++q) { mbar_init(smem_u32(&bars->full[q]), 1); mbar_init(smem_u32(&bars->empty[q]), 1); }
     for (int q = 0; q < 16; ++q) mbar_init(smem_u32(&bar2[q]), 1);
     bars->abort_flag = 0;
+    bars->wait_limit = kWaitCycles;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
@@ -425,6 +429,7 @@ tmem_share_kernel(long long* out, int mma_count, int b_noswizzle, int st_warps, 
   if (threadIdx.x == 0) {
     for (int q = 0; q < kMaxStages; ++q) mbar_init(smem_u32(&bars->full[q]), 1);
     bars->abort_flag = 0;
+    bars->wait_limit = kWaitCycles;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
@@ -516,6 +521,7 @@ stepped_issue_kernel(long long* out, int steps, int per_step, int use_fence, int
   if (threadIdx.x == 0) {
     for (int q = 0; q < kMaxStages; ++q) { mbar_init(smem_u32(&bars->full[q]), 8); mbar_init(smem_u32(&bars->empty[q]), 1); }
     bars->abort_flag = 0;
+    bars->wait_limit = kWaitCycles;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
@@ -581,6 +587,7 @@ lane_issue_kernel(long long* out, int count, int warps, int lanes, int a_slices,
   if (threadIdx.x == 0) {
     mbar_init(smem_u32(&bars->full[0]), uint32_t(warps * lanes));
     bars->abort_flag = 0;
+    bars->wait_limit = kWaitCycles;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }

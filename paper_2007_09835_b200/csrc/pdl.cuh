@@ -26,6 +26,15 @@ __device__ __forceinline__ void pdl_launch() { asm volatile("griddepcontrol.laun
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_entry() { pdl_launch(); pdl_wait(); }
 
+// One-time set-up that CUDA keeps per device (function attributes, occupancy answers): index of the current
+// device, or -1.  The launchers keep their "done" flags and cached values in arrays of kMaxDevices entries.
+constexpr int kMaxDevices = 64;
+inline int current_device_index() {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return -1;
+  return dev;
+}
+
 inline bool pdl_enabled() {
   static const bool on = [] {
     const char* e = getenv("RT3D_PDL");

@@ -22,6 +22,7 @@ struct __align__(8) Barriers {
   unsigned long long tmem_empty[2];
   unsigned int tmem_base;
   volatile int abort_flag;
+  long long wait_limit;      // SM clocks after which a wait gives up: kWaitCycles unless a test shortens it
 };
 
 // Bias staging area of a kernel, rounded up to 16 bytes so that the epilogue reads it as float4.
@@ -54,7 +55,7 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 }
 
 // Bounded wait.  Returns false (and raises the CTA's abort flag + the global error word) when the
-// phase did not complete within kWaitCycles, or when another role already aborted.
+// phase did not complete within bars->wait_limit clocks, or when another role already aborted.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, Barriers* bars, int32_t* err, int code) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long start = clock64();
@@ -63,7 +64,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, Barrier
     for (int i = 0; i < 128; ++i)
       if (mbar_try_wait(bar, parity)) return true;
     if (bars->abort_flag) return false;
-    if (clock64() - start > kWaitCycles) {
+    if (clock64() - start > bars->wait_limit) {
       bars->abort_flag = 1;
       atomicCAS(err, 0, code);
       return false;

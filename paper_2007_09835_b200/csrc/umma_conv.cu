@@ -148,6 +148,7 @@ conv3d_umma_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_consta
       mbar_init(smem_u32(&bars->tmem_empty[b]), two_sets ? 8 : 4);
     }
     bars->abort_flag = 0;
+    bars->wait_limit = a.wait_cycles > 0 ? a.wait_cycles : kWaitCycles;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
@@ -238,6 +239,9 @@ conv3d_umma_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_consta
           const uint32_t s_dst = tiles_base + stage * stage_bytes;
           if (!mbar_wait(smem_u32(&bars->empty[stage]), phase ^ 1u, bars, err, 1)) { ok = false; break; }
           mbar_expect_tx(full, tx_bytes * uint32_t(nload));
+          // test hook: the loads of this CTA's very last stage are never issued, so that the MMA warp's wait on
+          // them runs into the (shortened) limit and the error path can be exercised without any fault
+          if (a.debug_drop_last_load && i + kCps >= nsteps && item + int(gridDim.x) >= n_items) continue;
 #pragma unroll
           for (int q = 0; q < kCps; ++q) {
             if (q >= nload) break;
@@ -416,11 +420,13 @@ int pick_stages(int n_tile) {
 template <bool kDense, int kCps>
 cudaError_t launch_single_t(const UmmaArgs& a, const CUtensorMap& xm, const CUtensorMap& wm, const CUtensorMap& ym, int grid,
                             size_t smem, int stages, int cols, cudaStream_t stream) {
-  static bool attr_done = false;
-  if (!attr_done) {
+  static bool attr_done[kMaxDevices] = {};             // the attribute is per device
+  const int dev = current_device_index();
+  if (dev < 0) return cudaErrorInvalidDevice;
+  if (!attr_done[dev]) {
     cudaError_t e = cudaFuncSetAttribute(conv3d_umma_kernel<kDense, kCps>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
     if (e != cudaSuccess) return e;
-    attr_done = true;
+    attr_done[dev] = true;
   }
   LaunchSetup ls(dim3(grid), dim3(kThreadsSingle), smem, stream);
   return cudaLaunchKernelEx(&ls.cfg, conv3d_umma_kernel<kDense, kCps>, xm, wm, ym, a, stages, cols);

@@ -113,6 +113,7 @@ conv3d_umma_halo_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_c
     }
     mbar_init(smem_u32(&hb->w_full), 1);
     bars->abort_flag = 0;
+    bars->wait_limit = kWaitCycles;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
@@ -276,11 +277,13 @@ size_t halo_smem_bytes(const HaloArgs& h) {
 template <bool kDense>
 cudaError_t launch_halo_t(const HaloArgs& h, const CUtensorMap& xm, const CUtensorMap& wm, const CUtensorMap& ym,
                           int sm_count, int cols, size_t smem, long long n_items, cudaStream_t stream) {
-  static bool attr_done = false;
-  if (!attr_done) {
+  static bool attr_done[kMaxDevices] = {};             // the attributes are per device
+  const int dev_idx = current_device_index();
+  if (dev_idx < 0) return cudaErrorInvalidDevice;
+  if (!attr_done[dev_idx]) {
     cudaError_t e = cudaFuncSetAttribute(conv3d_umma_halo_kernel<kDense>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
     if (e != cudaSuccess) return e;
-    attr_done = true;
+    attr_done[dev_idx] = true;
   }
   long long clusters = sm_count / 2;
   if (clusters > n_items) clusters = n_items;

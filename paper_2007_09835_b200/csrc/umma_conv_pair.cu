@@ -80,6 +80,7 @@ conv3d_umma_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_c
       mbar_init(smem_u32(&bars->tmem_empty[b]), 8);   // leader: 4 epilogue warps of each CTA
     }
     bars->abort_flag = 0;
+    bars->wait_limit = kWaitCycles;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
@@ -378,11 +379,13 @@ size_t pair_smem_bytes(int n_tile, int n_bundles) {
 
 template <bool kDense, int kCps>
 cudaError_t prepare_pair_t() {
-  static bool attr_done = false;
-  if (!attr_done) {
+  static bool attr_done[kMaxDevices] = {};             // the attribute is per device
+  const int dev = current_device_index();
+  if (dev < 0) return cudaErrorInvalidDevice;
+  if (!attr_done[dev]) {
     cudaError_t e = cudaFuncSetAttribute(conv3d_umma_pair_kernel<kDense, kCps>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
     if (e != cudaSuccess) return e;
-    attr_done = true;
+    attr_done[dev] = true;
   }
   return cudaSuccess;
 }
@@ -402,7 +405,10 @@ void pair_launch_config(cudaLaunchConfig_t& cfg, cudaLaunchAttribute* attr, unsi
 // CTA pairs that can be resident at once (the persistent grid), never more than SMs / 2.
 template <bool kDense, int kCps>
 int pair_max_clusters_t(int sm_count, size_t smem) {
-  static int max_clusters = 0;
+  static int max_clusters_dev[kMaxDevices] = {};       // the occupancy answer is per device
+  const int dev = current_device_index();
+  if (dev < 0) return sm_count / 2;
+  int& max_clusters = max_clusters_dev[dev];
   if (max_clusters == 0) {
     if (prepare_pair_t<kDense, kCps>() != cudaSuccess) return sm_count / 2;
     cudaLaunchConfig_t cfg;

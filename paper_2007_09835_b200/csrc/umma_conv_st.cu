@@ -154,6 +154,7 @@ conv3d_umma_st_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_con
       mbar_init(smem_u32(&sb->out_empty[s]), 16);        // leader: 8 E2 warps of each CTA
     }
     bars->abort_flag = 0;
+    bars->wait_limit = kWaitCycles;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
@@ -548,11 +549,13 @@ cudaError_t launch_conv_umma_st(const StArgs& a, const void* xmap, const void* w
   memcpy(&xm, xmap, sizeof(CUtensorMap));
   memcpy(&w1m, w1map_half, sizeof(CUtensorMap));
   memcpy(&w2m, w2map_half, sizeof(CUtensorMap));
-  static bool attr_done = false;
-  if (!attr_done) {
+  static bool attr_done[kMaxDevices] = {};             // the attributes are per device
+  const int dev_idx = current_device_index();
+  if (dev_idx < 0) return cudaErrorInvalidDevice;
+  if (!attr_done[dev_idx]) {
     cudaError_t e = cudaFuncSetAttribute(conv3d_umma_st_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
     if (e != cudaSuccess) return e;
-    attr_done = true;
+    attr_done[dev_idx] = true;
   }
   long long clusters = sm_count / 2;
   if (clusters > total) clusters = total;

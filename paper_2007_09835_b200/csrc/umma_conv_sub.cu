@@ -386,15 +386,16 @@ bool umma_sub_plan(SubArgs* a, int max_blocks) {
   return sub_smem_bytes_impl(stages, slot, a->n_tile, a->n_bundles) <= 227 * 1024;
 }
 
-cudaError_t launch_conv_umma_sub(const SubArgs& a, const void* xmap, const void* ymap, int sm_count, int device, cudaStream_t stream) {
+cudaError_t launch_conv_umma_sub(const SubArgs& a, const void* xmap, const void* ymap, int sm_count, cudaStream_t stream) {
   if (a.stages < 2 || a.stages > kSubMaxStages || a.n_tile % 16 || a.n_tile > 256) return cudaErrorInvalidValue;
   if (xmap == nullptr || (a.store_tma && ymap == nullptr)) return cudaErrorInvalidValue;
   const size_t smem = sub_smem_bytes_impl(a.stages, a.slot_bytes, a.n_tile, a.n_bundles);
   if (smem > 227 * 1024) return cudaErrorInvalidValue;
   const long long n_items = (long long)a.tiles_n * a.tiles_t * a.tiles_h * a.tiles_w * a.n_bundles;
   if (n_items <= 0) return cudaSuccess;
-  static bool attr_done[64] = {};
-  if (device < 0 || device >= 64) return cudaErrorInvalidValue;
+  static bool attr_done[kMaxDevices] = {};             // the attribute is per device
+  const int device = current_device_index();
+  if (device < 0) return cudaErrorInvalidDevice;
   if (!attr_done[device]) {
     cudaError_t e = cudaFuncSetAttribute(conv3d_umma_sub_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
     if (e != cudaSuccess) return e;

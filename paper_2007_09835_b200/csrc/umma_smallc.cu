@@ -69,6 +69,7 @@ conv3d_umma_smallc_kernel(const __grid_constant__ CUtensorMap xmap, const __grid
       mbar_init(smem_u32(&bars->tmem_empty[b]), 4);
     }
     bars->abort_flag = 0;
+    bars->wait_limit = kWaitCycles;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
@@ -240,14 +241,16 @@ cudaError_t launch_conv_umma_smallc(const SmallCArgs& a_in, const void* xmap, co
   CUtensorMap xm, ym;
   memcpy(&xm, xmap, sizeof(CUtensorMap));
   memcpy(&ym, ymap ? ymap : xmap, sizeof(CUtensorMap));
-  static bool attr_done = false;
-  if (!attr_done) {
+  static bool attr_done[kMaxDevices] = {};             // the attributes are per device
+  const int dev_idx = current_device_index();
+  if (dev_idx < 0) return cudaErrorInvalidDevice;
+  if (!attr_done[dev_idx]) {
     cudaError_t e = cudaFuncSetAttribute(conv3d_umma_smallc_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
     if (e != cudaSuccess) return e;
     // ask for the largest shared-memory carve-out: with the default one fewer CTAs fit an SM than the sizes allow
     e = cudaFuncSetAttribute(conv3d_umma_smallc_kernel<0>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
     if (e != cudaSuccess) return e;
-    attr_done = true;
+    attr_done[dev_idx] = true;
   }
   // Several CTAs per SM (the layer is bound by the latencies of its epilogue): as many as are really resident
   // at once, counted here from the register file, the shared memory (228 KB per SM, 1 KB reserved per CTA)

@@ -7,6 +7,8 @@ step is a call into librt3d; torch provides device memory and streams.
 """
 from __future__ import annotations
 
+import contextlib
+
 import numpy as np
 import torch
 
@@ -147,7 +149,8 @@ class C3DNet:
         self.fused_ok[key] = True
         return y
 
-    def forward(self, x: torch.Tensor, algo=B.ALGO_AUTO, keep=None, stream=None) -> torch.Tensor:
+    def forward(self, x: torch.Tensor, algo=B.ALGO_AUTO, keep=None, stream=None, plan_log=None) -> torch.Tensor:
+        """plan_log: dict that receives, per conv name, how the library ran that layer (rt3d_last_plan)."""
         c = self.plan[0].cin
         skip = None
         for i, op in enumerate(self.plan):
@@ -159,6 +162,8 @@ class C3DNet:
                 if self.fuse_pool and nxt is not None and not hasattr(nxt, "cout"):
                     y = self._try_fused(op, nxt, x, algo, stream, pad0)
                     if y is not None:
+                        if plan_log is not None:
+                            plan_log[op.name] = B.rt3d_last_plan()
                         x, c, skip = y, op.cout, nxt
                         if keep is not None:
                             keep[nxt.name] = x
@@ -166,6 +171,8 @@ class C3DNet:
                 layer = self.layers[op.name]
                 y = self.ws.get(op.name, layer.out_shape(x), x.dtype, x.device)
                 x = layer(x, y, algo=algo, stream=stream, x_pad_zero=pad0)
+                if plan_log is not None:
+                    plan_log[op.name] = B.rt3d_last_plan()
                 c = op.cout
             else:
                 n, t, h, w, cs = x.shape
@@ -257,12 +264,15 @@ class R2Plus1DNet:
                 fork = torch.cuda.Event()
                 fork.record(main)
                 self.side.wait_event(fork)
-                with torch.cuda.stream(self.side):
+                with torch.cuda.stream(self.side), B.concurrent_kernels():
                     sc = self._conv(blk.shortcut, inp, algo, None)
                     join = torch.cuda.Event()
                     join.record(self.side)
             else:
                 sc = self._conv(blk.shortcut, inp, algo, stream)
+            # until the join, the main path's kernels run beside the projection on the side stream
+            beside = B.concurrent_kernels() if join is not None else contextlib.nullcontext()
+            beside.__enter__()
             if keep is not None and blk.shortcut is not None:
                 keep[blk.shortcut.name] = sc
             last = blk.convs[-1]
@@ -270,6 +280,7 @@ class R2Plus1DNet:
                 c = blk.convs
                 y = self._pair(c[0], c[1], x, None, c[1].relu, stream, c[1].name)
                 x = y if y is not None else self._conv(c[1], self._conv(c[0], x, algo, stream), algo, stream)
+                beside.__exit__(None, None, None)
                 if join is not None:
                     torch.cuda.current_stream(x.device).wait_event(join)
                 y = self._pair(c[2], c[3], x, sc, True, stream, blk.name + ".out")
@@ -284,6 +295,7 @@ class R2Plus1DNet:
                 x = self._conv(spec, x, algo, stream)
                 if keep is not None:
                     keep[spec.name] = x
+            beside.__exit__(None, None, None)
             if join is not None:
                 torch.cuda.current_stream(x.device).wait_event(join)
             if self.fuse_residual:
@@ -362,14 +374,15 @@ class S3DNet:
                     fork = torch.cuda.Event()
                     fork.record(main)
                     joins = []
-                    for fn, side in zip(work, self._branch_streams(x.device)):
-                        side.wait_event(fork)
-                        with torch.cuda.stream(side):
-                            fn()
-                            ev = torch.cuda.Event()
-                            ev.record(side)
-                        joins.append(ev)
-                    branch0()                                        # the main stream takes the 1x1x1 branch
+                    with B.concurrent_kernels():
+                        for fn, side in zip(work, self._branch_streams(x.device)):
+                            side.wait_event(fork)
+                            with torch.cuda.stream(side):
+                                fn()
+                                ev = torch.cuda.Event()
+                                ev.record(side)
+                            joins.append(ev)
+                        branch0()                                    # the main stream takes the 1x1x1 branch
                     for ev in joins:
                         main.wait_event(ev)
                 else:

@@ -3,10 +3,12 @@
 Per layer the CUDA library receives exactly the input the oracle consumed (teacher forcing),
 so every conv output is held to max|err| <= 2e-2 * max|ref| and every pool / add output must be
 bit-identical.  The free-running forward pass (the library feeding itself) is compared at the
-network output with the same norm at 3e-2: the two data flows round each layer's output to
-bf16 independently, and a one-ulp rounding difference (2^-8 relative) of an activation is then
-an input perturbation of the next layer, which the per-layer bound does not cover.
+network output with the same norm and the same 2e-2: the two data flows round each layer's output to
+bf16 independently, so a one-ulp rounding difference (2^-8 relative) of an activation perturbs the
+next layer's input, but the measured errors (4e-3 to 1e-2, recorded by record_error) stay well inside.
 """
+import os
+
 import numpy as np
 import pytest
 import torch
@@ -20,12 +22,22 @@ import netref
 
 pytestmark = pytest.mark.gpu
 TOL = 2e-2
-TOL_FREE = 3e-2
+TOL_FREE = 2e-2
 
 
 def rel_err(y, ref):
     assert np.isfinite(y).all()
     return float(np.abs(y - ref).max() / np.abs(ref).max())
+
+
+def record_error(name, err, tol):
+    """Keeps the measured error of a free-running forward pass on record (one line per case in
+    parity_errors.txt under RT3D_PARITY_LOG_DIR, default gpurun_out/, when that folder exists): the distance
+    from the 2e-2 single-layer tolerance is otherwise invisible behind a passing assertion."""
+    folder = os.environ.get("RT3D_PARITY_LOG_DIR", os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "gpurun_out"))
+    if os.path.isdir(folder):
+        with open(os.path.join(folder, "parity_errors.txt"), "a") as f:
+            f.write(f"{name}: max|err|/max|ref| = {err:.4e} (asserted <= {tol:g})\n")
 
 
 def device_layers(layers, specs, dense=False):
@@ -84,9 +96,48 @@ def test_c3d_free_running_forward(c3d, batch, fuse):
     ref = final[: len(pick)]
     assert (ref != 0).mean() > 0.10
     e = rel_err(y[pick], ref)
+    record_error(f"C3D-shaped free-running forward, batch {batch}, fused pools {fuse}", e, TOL_FREE)
     assert e <= TOL_FREE, e
     if fuse:
         assert any(net.fused_ok.values())                        # at least conv1/conv2 really ran fused
+
+
+def test_c3d_layers_teacher_forced_at_the_batch16_plan(c3d):
+    """The eight conv layers once more, each called exactly as the batch-16 forward pass calls it (same shapes, fused
+    pools where that forward fuses them), so that the kernel plans a large batch selects (CTA-pair kernel, tail
+    split, pooling epilogue) are checked per layer against the oracle and not only at the network output.  The
+    batch is made of the oracle's two clips in an irregular order: clips are independent, so EVERY clip of the
+    batch has a full reference (a superset of sampling outputs on the clips between the first and the last)."""
+    plan, layers, specs, x2, rec, final = c3d
+    dl = device_layers(layers, specs)
+    net = nets.C3DNet(plan, dl, fuse_pool=True)
+    order = [0, 1, 1, 0, 1, 0, 0, 1, 0, 0, 1, 1, 1, 0, 0, 1]
+    x16 = x2[order]
+    plans_fwd = {}
+    net.forward(nets.to_device(x16), plan_log=plans_fwd)          # what the real forward pass runs per layer
+    assert rt3d.rt3d_last_device_status() == rt3d.OK
+    assert plans_fwd["conv3a"]["kernel"] == 2 and plans_fwd["conv1"]["kernel"] == 3
+    assert plans_fwd["conv1"]["fused_pool"] == 1 and plans_fwd["conv2"]["fused_pool"] == 1
+    assert any(p["tail_workers"] > 0 for p in plans_fwd.values())  # the batch-16 pass does use the tail split
+    for i, op in enumerate(plan):
+        if not isinstance(op, synth.ConvSpec):
+            continue
+        inp, ref = rec[op.name]
+        xd = nets.to_device(inp[order])
+        nxt = plan[i + 1] if i + 1 < len(plan) else None
+        fused = plans_fwd[op.name]["fused_pool"] == 1
+        if fused:
+            y = net._try_fused(op, nxt, xd, rt3d.ALGO_AUTO, None, i == 0)
+            assert y is not None
+            expect = rec[nxt.name][1]                             # the oracle's pooled tensor
+        else:
+            y = dl[op.name](xd, x_pad_zero=(i == 0))
+            expect = ref
+        assert rt3d.rt3d_last_plan() == plans_fwd[op.name], (op.name, rt3d.rt3d_last_plan(), plans_fwd[op.name])
+        got = nets.to_numpy(y, op.cout)
+        e = rel_err(got, expect[order])
+        assert e <= TOL, (op.name, e)
+    assert rt3d.rt3d_last_device_status() == rt3d.OK
 
 
 def test_c3d_fc_tail(c3d):
@@ -105,7 +156,9 @@ def test_c3d_fc_tail(c3d):
     y = nets.to_numpy(net.forward(nets.to_device(x2)), 101)
     assert y.shape == (2, 1, 1, 1, 101)
     assert rt3d.rt3d_last_device_status() == rt3d.OK
-    assert rel_err(y, logits) <= TOL_FREE
+    e = rel_err(y, logits)
+    record_error("C3D-shaped + FC tail, free-running, 2 clips", e, TOL_FREE)
+    assert e <= TOL_FREE
 
 
 def test_c3d_dense_path_forward():
@@ -166,6 +219,7 @@ def test_r2plus1d_free_running_batch8(r21d, fuse):
     assert rt3d.rt3d_last_device_status() == rt3d.OK
     assert (final != 0).mean() > 0.10
     e = rel_err(y[[0, 7]], final)
+    record_error(f"R(2+1)D-shaped free-running forward, batch 8, fusion {fuse}", e, TOL_FREE)
     assert e <= TOL_FREE, e
     if fuse == "pairs":       # the two stage-2 blocks run their four factorised pairs as one launch each
         assert net.pairs_fused == {"s2b1.c1.s", "s2b1.c2.s", "s2b2.c1.s", "s2b2.c2.s"}, (net.pairs_fused, net.pairs_declined)
@@ -220,7 +274,9 @@ def test_s3d_free_running_forward(s3d):
     blk = nets.to_numpy(keep["mixed3b"], 256)
     assert rel_err(blk, rec["mixed3b"][1]) <= TOL_FREE
     assert (final != 0).mean() > 0.10
-    assert rel_err(y, final) <= TOL_FREE
+    e = rel_err(y, final)
+    record_error("S3D-shaped free-running forward, batch 1", e, TOL_FREE)
+    assert e <= TOL_FREE
 
 
 # --------------------------------------------------------------------------- sparsity sweep
