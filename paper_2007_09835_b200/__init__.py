@@ -7,7 +7,7 @@ module stays importable before the library exists.
 """
 
 
-_SUBMODULES = ("build", "binding", "nets", "dist", "sweep", "layer_bench", "net_bench")
+_SUBMODULES = ("build", "binding", "nets", "dist", "sweep")
 
 
 def __getattr__(name):

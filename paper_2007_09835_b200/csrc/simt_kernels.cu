@@ -25,6 +25,13 @@ template <> __device__ __forceinline__ float from_f32<float>(float v) { return v
 template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
 
 // GM/GN > 0: compile-time group size; 0: run-time size (<= 8).
+// All threads of a block work on the same row p of kernel groups, so the row's packed index and weight tiles are
+// staged once per block in shared memory (in pieces of kStageEntries kept entries across the row's Q groups, which
+// are contiguous in the packed arrays), with each kept location
+// decoded to its (kt, kh, kw) there: the inner loop then has no integer division and no dependent global load
+// besides the input voxel itself, which is fetched with one 16-byte load when the group is four channels wide.
+constexpr int kStageEntries = 64;
+
 template <typename T, int GM, int GN, bool DENSE>
 __global__ void __launch_bounds__(kThreads)
 conv3d_kgs_simt_kernel(ConvGeom g, const T* __restrict__ x, T* __restrict__ y,
@@ -34,6 +41,9 @@ conv3d_kgs_simt_kernel(ConvGeom g, const T* __restrict__ x, T* __restrict__ y,
   pdl_entry();
   constexpr int MAXM = GM ? GM : 8;
   constexpr int MAXN = GN ? GN : 8;
+  __shared__ float w_s[kStageEntries * MAXM * MAXN];
+  __shared__ int off_s[kStageEntries];             // (kt << 20) | (kh << 10) | kw
+  __shared__ int c0_s[kStageEntries];              // first input channel of the entry's group
   const int g_m = GM ? GM : g_m_rt;
   const int g_n = GN ? GN : g_n_rt;
   const int p = blockIdx.y;
@@ -52,27 +62,47 @@ conv3d_kgs_simt_kernel(ConvGeom g, const T* __restrict__ x, T* __restrict__ y,
   for (int i = 0; i < MAXM; ++i) acc[i] = 0.f;
 
   const int tile_elems = g_m * g_n;
-  for (int q = 0; q < Q; ++q) {
-    const int e0 = group_ptr[p * Q + q], e1 = group_ptr[p * Q + q + 1];
-    const int c0 = q * g_n;
-    for (int e = e0; e < e1; ++e) {
-      const int kpos = DENSE ? (e - e0) : int(pos_idx[e]);
-      const int kw = kpos % g.Kw;
-      const int kh = (kpos / g.Kw) % g.Kh;
-      const int kt = kpos / (g.Kw * g.Kh);
-      const int ti = t0 + kt, hi = h0 + kh, wi = w0 + kw;
-      if (!valid || ti < 0 || ti >= g.t || hi < 0 || hi >= g.h || wi < 0 || wi >= g.w) continue;
-      const T* xp = x + ((((long long)nn * g.t + ti) * g.h + hi) * g.w + wi) * g.xcs + c0;
+  const bool vec4 = GN == 4 && sizeof(T) == 4 && (g.xcs & 3) == 0 && (g.c & 3) == 0;
+  // the kept entries of all Q groups of row p are one contiguous range of the packed arrays
+  const int row0 = group_ptr[p * Q], row1 = group_ptr[p * Q + Q];
+  for (int eb = row0; eb < row1; eb += kStageEntries) {
+    const int n_e = row1 - eb < kStageEntries ? row1 - eb : kStageEntries;
+    __syncthreads();                               // the previous piece has been consumed
+    for (int i = threadIdx.x; i < n_e * tile_elems; i += kThreads) {
+      const int e = i / tile_elems, k = i - e * tile_elems;
+      w_s[e * (MAXM * MAXN) + (k / g_n) * MAXN + k % g_n] = to_f32<T>(tiles[(long long)(eb + e) * tile_elems + k]);
+    }
+    for (int e = threadIdx.x; e < n_e; e += kThreads) {
+      int q = 0;                                     // the group this entry belongs to
+      while (q + 1 < Q && group_ptr[p * Q + q + 1] <= eb + e) ++q;
+      const int kpos = DENSE ? (eb + e - group_ptr[p * Q + q]) : int(pos_idx[eb + e]);
+      off_s[e] = ((kpos / (g.Kw * g.Kh)) << 20) | (((kpos / g.Kw) % g.Kh) << 10) | (kpos % g.Kw);
+      c0_s[e] = q * g_n;
+    }
+    __syncthreads();
+#pragma unroll 4
+    for (int e = 0; e < n_e; ++e) {
+      const int off = off_s[e], c0 = c0_s[e];
+      const int ti = t0 + (off >> 20), hi = h0 + ((off >> 10) & 1023), wi = w0 + (off & 1023);
+      const bool inb = valid && unsigned(ti) < unsigned(g.t) && unsigned(hi) < unsigned(g.h) && unsigned(wi) < unsigned(g.w);
+      const T* xp = x + ((((long long)nn * g.t + (inb ? ti : 0)) * g.h + (inb ? hi : 0)) * g.w + (inb ? wi : 0)) * g.xcs + c0;
       float xv[MAXN];
+      if (vec4) {
+        const float4 t4 = inb ? __ldg(reinterpret_cast<const float4*>(xp)) : make_float4(0.f, 0.f, 0.f, 0.f);
+        xv[0] = t4.x; xv[1] = t4.y; xv[2] = t4.z; xv[3] = t4.w;
 #pragma unroll
-      for (int j = 0; j < MAXN; ++j) xv[j] = (j < g_n && c0 + j < g.c) ? to_f32<T>(xp[j]) : 0.f;
-      const T* tp = tiles + (long long)e * tile_elems;
+        for (int j = 4; j < MAXN; ++j) xv[j] = 0.f;
+      } else {
+#pragma unroll
+        for (int j = 0; j < MAXN; ++j) xv[j] = (inb && j < g_n && c0 + j < g.c) ? to_f32<T>(xp[j]) : 0.f;
+      }
+      const float* tp = w_s + e * (MAXM * MAXN);
 #pragma unroll
       for (int i = 0; i < MAXM; ++i) {
         if (i < g_m) {
 #pragma unroll
           for (int j = 0; j < MAXN; ++j)
-            if (j < g_n) acc[i] = fmaf(xv[j], to_f32<T>(tp[i * g_n + j]), acc[i]);
+            if (j < g_n) acc[i] = fmaf(xv[j], tp[i * MAXN + j], acc[i]);
         }
       }
     }

@@ -45,7 +45,7 @@ def time_layer(layer, x, y, iters, algo=B.ALGO_AUTO):
     return e0.elapsed_time(e1) / iters * 1e3        # microseconds
 
 
-def run(iters=30, groups=None, rates=None, algo=B.ALGO_AUTO):
+def run(iters=30, groups=None, rates=None, algo=B.ALGO_AUTO, schemes=("kgs", "vanilla")):
     spec = synth.ConvSpec("sweep", 256, 256, (3, 3, 3), (1, 1, 1), (1, 1, 1), True)
     x = nets.to_device(synth.make_input(4, (32, 8, 14, 14, 256)))
     base = synth.make_layer(spec, 4, 0, 4, 4, "none", None)
@@ -58,7 +58,7 @@ def run(iters=30, groups=None, rates=None, algo=B.ALGO_AUTO):
     for g_m, g_n in (groups or PAPER_GROUPS + WIDE_GROUPS):
         P, Q = synth.n_groups(256, 256, g_m, g_n)
         for rate in (rates or RATES):
-            for scheme in ("kgs", "vanilla"):
+            for scheme in schemes:
                 if scheme == "vanilla" and (rate == 1 or round(P * Q / rate) < 1):
                     continue
                 if scheme == "kgs":
