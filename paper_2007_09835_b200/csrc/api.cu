@@ -55,7 +55,7 @@ struct DeviceState {
   bool init = false;
   int sm_count = 0;
   int cc_major = 0;
-  int32_t* sched = nullptr;     // [8] words: [2] = error word written by kernels on a bounded-wait expiry
+  int32_t* sched = nullptr;     // [256] words: [2] = error word written by kernels on a bounded-wait expiry
 };
 std::mutex g_dev_mu;
 DeviceState g_dev[64];
