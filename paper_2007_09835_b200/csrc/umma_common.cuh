@@ -241,8 +241,9 @@ __device__ __forceinline__ void epilogue_cols(const uint32_t* v, const float* bi
 // m_base to the end of the residual tensor's channel pitch.
 __device__ __forceinline__ void epilogue_row(uint32_t taddr, int n_cols, bool has_acc, bool in_range,
                                              const float* bias_s, int relu, __nv_bfloat16* dst, int m_base, int M,
-                                             const __nv_bfloat16* res_row = nullptr, int res_pitch_left = 0) {
-  for (int col = 0; col < n_cols; col += 32) {
+                                             const __nv_bfloat16* res_row = nullptr, int res_pitch_left = 0,
+                                             int col0 = 0, int col_step = 32) {
+  for (int col = col0; col < n_cols; col += col_step) {
     const int m0 = m_base + col;
     if (m0 >= M) break;
     uint32_t v[32];
@@ -278,6 +279,7 @@ struct TmaStore {
   uint32_t smem;              // this warp's two staging buffers (1024-byte aligned)
   int c1, c2, c3, c4;         // output coordinates (w, h, t, n) of the warp's first row
   uint32_t piece;             // pieces issued so far by this warp
+  uint32_t bufs = kStoreBufs; // staging buffers this warp cycles through (1 when two warps share a quadrant's pair)
 };
 
 // Fused max-pool (window = stride = 1 or 2 per axis) over the 32 voxels of an epilogue warp, which form a
@@ -312,6 +314,8 @@ __device__ __forceinline__ void tma_store_5d(const CUtensorMap* map, uint32_t sr
 __device__ __forceinline__ void tma_store_wait_read_1() {
   asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(kStoreBufs - 1) : "memory");
 }
+// The warp's previous store has finished reading its (single) staging buffer.
+__device__ __forceinline__ void tma_store_wait_read_0() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 // Before the warp leaves the kernel: all its bulk stores have read their staging buffers (shared memory may go
 // away).  Their global writes are part of the grid's memory operations, complete before the grid does.
 __device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
@@ -394,8 +398,11 @@ __device__ __forceinline__ void epilogue_piece_tma(const uint32_t* v, const floa
     writer = pool->writer;
     out_row = pool->out_row;
   }
-  const uint32_t buf = ts.smem + (ts.piece % kStoreBufs) * kStoreStageBytes;
-  if (lane == 0) tma_store_wait_read_1();          // the store issued kStoreBufs pieces ago has read this buffer
+  const uint32_t buf = ts.smem + (ts.piece % ts.bufs) * kStoreStageBytes;
+  if (lane == 0) {                                 // the store issued ts.bufs pieces ago has read this buffer
+    if (ts.bufs == 1) tma_store_wait_read_0();
+    else tma_store_wait_read_1();
+  }
   __syncwarp();
   const uint32_t row = buf + uint32_t(out_row) * 64u;
   const uint32_t sw = (uint32_t(out_row) >> 1) & 3u;  // 64-byte swizzle: 16-byte chunk index ^= address bits 7..8
@@ -420,8 +427,9 @@ __device__ __forceinline__ void epilogue_row_tma(uint32_t taddr, int n_cols, boo
                                                  const __nv_bfloat16* res_row = nullptr, int res_pitch_left = 0,
                                                  const PoolLanes* pool = nullptr, const float* extra_first = nullptr,
                                                  const float* extra = nullptr, size_t extra_stride = 0,
-                                                 int n_extra = 0) {
-  for (int col = 0; col < n_cols; col += 32) {
+                                                 int n_extra = 0, int col0 = 0, int col_step = 32) {
+  // col0 / col_step: a second warp on the same TMEM lane quadrant takes every other 32-column piece
+  for (int col = col0; col < n_cols; col += col_step) {
     const int m0 = m_base + col;
     if (m0 >= M) break;
     uint32_t v[32];

@@ -42,9 +42,15 @@ __device__ __forceinline__ Work get_work(const TailWork* tw, int wi, int cluster
   return Work{g.item, g.g0, g.g1, g.part, g.nparts};
 }
 
+// Threads of a CTA: producer warp, MMA warp, two sets of four epilogue warps.  The second set (warps 6..9) takes the
+// odd 32-column pieces of every tile, so that a tile with few K steps (a heavily pruned layer with tall kernel
+// groups, a 1x1x1 or 1x3x3 layer) is not bound by its epilogue: four warps need about 15 k clocks for a 128 x 256
+// tile, as long as 30 K steps.  With the tail split only the first set works (the fix-up of shared tiles is theirs).
+constexpr int kThreadsPair = 320;
+
 // kCps: K steps per pipeline stage (and per barrier hand-shake): 1, or 2 for narrow bundles.
 template <bool kDense, int kCps>
-__global__ void __launch_bounds__(kThreadsUmma, 1)
+__global__ void __launch_bounds__(kThreadsPair, 1)
 conv3d_umma_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CUtensorMap wmap_half,
                         const __grid_constant__ CUtensorMap ymap, const UmmaArgs a, const int stages, const int tmem_cols) {
   extern __shared__ unsigned char smem_raw[];
@@ -69,6 +75,7 @@ conv3d_umma_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_c
   const int n_items = pairs_per_bundle * a.n_bundles;
   const int cluster_id = blockIdx.x >> 1, n_clusters = gridDim.x >> 1;
   const int box_rows = a.box.bn * a.box.bt * a.box.bh * a.box.bw;
+  const int epi_sets = a.tail_workers == 0 ? 2 : 1;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < stages; ++s) {
@@ -77,7 +84,7 @@ conv3d_umma_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_c
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(smem_u32(&bars->tmem_full[b]), 1);    // multicast commit
-      mbar_init(smem_u32(&bars->tmem_empty[b]), 8);   // leader: 4 epilogue warps of each CTA
+      mbar_init(smem_u32(&bars->tmem_empty[b]), uint32_t(8 * epi_sets));   // leader: the working epilogue warps of both CTAs
     }
     bars->abort_flag = 0;
     bars->wait_limit = kWaitCycles;
@@ -239,9 +246,11 @@ conv3d_umma_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_c
         umma_commit_pair(smem_u32(&bars->tmem_full[buf]));     // with no MMAs pending this arrives at once
       }
     }
-  } else {
+  } else if (warp < 6 || epi_sets == 2) {
     // ------------------------------------------------------------------ epilogue (both CTAs)
     const int quad = warp & 3;
+    const int set = (warp - 2) >> 2;                       // 0: warps 2..5, 1: warps 6..9
+    const int col0 = set * 32, col_step = 32 * epi_sets;   // which 32-column pieces this warp takes
     const int row = quad * 32 + lane;
     int r = row;
     const int bw_i = r % a.box.bw; r /= a.box.bw;
@@ -250,7 +259,9 @@ conv3d_umma_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_c
     const int bn_i = r;
     __nv_bfloat16* yb = static_cast<__nv_bfloat16*>(a.y);
     const __nv_bfloat16* rb = static_cast<const __nv_bfloat16*>(a.residual);
-    TmaStore ts{&ymap, store_smem + uint32_t(quad) * kStoreWarpBytes, 0, 0, 0, 0, 0u};
+    // two sets: each warp of a quadrant uses one of the quadrant's two staging buffers
+    TmaStore ts{&ymap, store_smem + uint32_t(quad) * kStoreWarpBytes + uint32_t(set) * kStoreStageBytes, 0, 0, 0, 0, 0u,
+                epi_sets == 2 ? 1u : kStoreBufs};
     const PoolLanes pool_lanes = make_pool_lanes(a.pool_w, a.pool_h, a.pool_t, a.sbw, a.sbh, lane);
     const PoolLanes* pool = (a.pool_t * a.pool_h * a.pool_w > 1) ? &pool_lanes : nullptr;
     int r0 = quad * 32;                        // coordinates of the warp's first row inside the box
@@ -335,10 +346,11 @@ conv3d_umma_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_c
       if (a.store_tma) {
         ts.c1 = (c.w0 + bw_0) / a.pool_w; ts.c2 = (c.h0 + bh_0) / a.pool_h; ts.c3 = (c.t0 + bt_0) / a.pool_t; ts.c4 = c.n0 + bn_0;
         epilogue_row_tma(taddr, a.n_tile, nsteps > 0, quad * 32 < box_rows, in_range, bias_s, a.g.relu,
-                         yb + vox * a.g.ycs + m_base, m_base, a.g.M, lane, ts, res, res_left, pool);
+                         yb + vox * a.g.ycs + m_base, m_base, a.g.M, lane, ts, res, res_left, pool, nullptr, nullptr, 0, 0,
+                         col0, col_step);
       } else {
         epilogue_row(taddr, a.n_tile, nsteps > 0, in_range, bias_s, a.g.relu, yb + vox * a.g.ycs + m_base, m_base, a.g.M,
-                     res, res_left);
+                     res, res_left, col0, col_step);
       }
       tc_fence_before();
       __syncwarp();
@@ -395,7 +407,7 @@ void pair_launch_config(cudaLaunchConfig_t& cfg, cudaLaunchAttribute* attr, unsi
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
   cfg.gridDim = dim3(grid);
-  cfg.blockDim = dim3(kThreadsUmma);
+  cfg.blockDim = dim3(kThreadsPair);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = stream;
   cfg.attrs = attr;
@@ -436,7 +448,7 @@ cudaError_t launch_pair_t(const UmmaArgs& a, const CUtensorMap& xm, const CUtens
   if (e != cudaSuccess) return e;
   long long clusters = pair_max_clusters_t<kDense, kCps>(sm_count, smem);
   if (clusters > n_items) clusters = n_items;
-  LaunchSetup ls(dim3(unsigned(2 * clusters)), dim3(kThreadsUmma), smem, stream, 2);
+  LaunchSetup ls(dim3(unsigned(2 * clusters)), dim3(kThreadsPair), smem, stream, 2);
   return cudaLaunchKernelEx(&ls.cfg, conv3d_umma_pair_kernel<kDense, kCps>, xm, wm, ym, a, stages, cols);
 }
 
