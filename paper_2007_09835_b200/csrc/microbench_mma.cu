@@ -627,6 +627,70 @@ lane_issue_kernel(long long* out, int count, int warps, int lanes, int a_slices,
   }
 }
 
+// ------------------------------------------------------------------------------------------ M11
+// Two issuing warps with DIFFERENT instruction shapes at once: warp 0 a chain of N = n0 MMAs with A in shared
+// memory (a spatial convolution's steps), warp 1 a chain of N = n1 MMAs with A in tensor memory (a temporal
+// convolution fed from the intermediate frame).  out[0] / out[1] = clocks until each chain is done.
+__global__ void __launch_bounds__(128, 1)
+mixed_issue_kernel(long long* out, int n0, int count0, int n1, int count1, int32_t* err) {
+  extern __shared__ unsigned char smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  const uint32_t a_smem = base, b_smem = base + kARegion;
+  Barriers* bars = reinterpret_cast<Barriers*>(smem_raw + (base - raw) + kARegion + kBRegion);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  for (uint32_t i = threadIdx.x; i < (kARegion + kBRegion) / 4; i += blockDim.x)
+    reinterpret_cast<uint32_t*>(smem_raw + (base - raw))[i] = 0x3c003c00u;
+  if (threadIdx.x == 0) {
+    mbar_init(smem_u32(&bars->full[0]), 1);
+    mbar_init(smem_u32(&bars->full[1]), 1);
+    bars->abort_flag = 0;
+    bars->wait_limit = kWaitCycles;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 0) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&bars->tmem_base)), "r"(512u) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = bars->tmem_base;
+  {
+    const uint32_t taddr = tmem_base + (uint32_t(warp * 32) << 16) + 448u;
+    for (int c = 0; c < 32; c += 8)
+      asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %1, %1, %1, %1, %1, %1, %1};" ::"r"(taddr + c), "r"(0x3c003c00u) : "memory");
+    asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  if (lane == 0 && warp < 2) {
+    const int n = warp == 0 ? n0 : n1, count = warp == 0 ? count0 : count1;
+    const uint32_t idesc = idesc_any(0, 128, n);
+    const uint64_t bdesc = smem_desc_sw128(b_smem);
+    const uint32_t d = tmem_base + uint32_t(warp) * 256u;          // accumulators at columns 0.. and 256..
+    const long long t0 = clock64();
+    for (int i = 0; i < count; ++i) {
+      const uint64_t adesc = smem_desc_sw128(a_smem + uint32_t(i & 3) * 16384u) + 2 * (i & 3);
+      if (warp == 0) mma_any<0, false, 1>(d, adesc, 0u, bdesc + 2 * (i & 3), idesc, i ? 1u : 0u);
+      else mma_any<0, true, 1>(d, 0ull, tmem_base + 448u + uint32_t(i & 3) * 8u, bdesc + 2 * (i & 3), idesc, i ? 1u : 0u);
+    }
+    if (count > 0) {
+      umma_commit(smem_u32(&bars->full[warp]));
+      mbar_wait(smem_u32(&bars->full[warp]), 0, bars, err, 14);
+    }
+    out[warp] = clock64() - t0;
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+  }
+}
+
 // ------------------------------------------------------------------------------------------ M3
 // kShape: 0 m16n8k16 bf16, 1 m16n8k8 bf16, 2 m16n8k8 tf32, 3 m16n8k4 tf32.  Eight independent accumulator
 // tiles per warp, operands in registers.
@@ -993,6 +1057,24 @@ int main(int argc, char** argv) {
       }
       cudaMemcpy(h, d_out, 8, cudaMemcpyDeviceToHost);
       printf("| %d | %d | %d | %.1f | %.1f |\n", cb[0], cb[1], cb[2], double(h[0]) / (double(cnt) * cb[0] * cb[1]), double(h[0]) / cnt);
+    }
+  }
+
+  printf("\n## M11: two issuing warps with different shapes (warp 0: N = 144, A in shared memory; warp 1: N = 64, A in TMEM)\n\n");
+  printf("| MMAs of warp 0 | MMAs of warp 1 | clocks warp 0 | clocks warp 1 | tensor clocks of all MMAs |\n|---|---|---|---|---|\n");
+  {
+    const size_t smem = 1024 + kARegion + kBRegion + sizeof(Barriers) + 64;
+    cudaFuncSetAttribute(mixed_issue_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
+    const int combos[][2] = {{360, 0}, {0, 270}, {360, 270}, {360, 540}};
+    for (const auto& cb : combos) {
+      long long h[2] = {0, 0};
+      for (int rep = 0; rep < 2; ++rep) {
+        cudaMemset(d_out, 0, 32);
+        mixed_issue_kernel<<<1, 128, smem>>>(d_out, 144, cb[0], 64, cb[1], d_err);
+        if (!sync_ok("mixed_issue")) return 1;
+      }
+      cudaMemcpy(h, d_out, 16, cudaMemcpyDeviceToHost);
+      printf("| %d | %d | %lld | %lld | %.0f |\n", cb[0], cb[1], h[0], h[1], cb[0] * 72.0 + cb[1] * 32.0);
     }
   }
 
