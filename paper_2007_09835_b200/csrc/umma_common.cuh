@@ -473,8 +473,9 @@ __device__ __forceinline__ void epilogue_row_tma(uint32_t taddr, int n_cols, boo
 // Split-K partial tiles are stored column-major, [column][128 rows] floats, so that the 32 lanes of a
 // warp (32 consecutive rows) always touch 128 contiguous bytes.
 // Raw fp32 accumulator row -> scratch; `dst` already points at this thread's row of column 0.
-__device__ __forceinline__ void store_partial_row(uint32_t taddr, int n_cols, bool has_acc, float* dst) {
-  for (int col = 0; col < n_cols; col += 32) {
+__device__ __forceinline__ void store_partial_row(uint32_t taddr, int n_cols, bool has_acc, float* dst, int col0 = 0,
+                                                  int col_step = 32) {
+  for (int col = col0; col < n_cols; col += col_step) {
     uint32_t v[32];
     const bool wide = col + 32 <= n_cols;
     if (has_acc) {

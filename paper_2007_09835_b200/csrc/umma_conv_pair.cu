@@ -24,18 +24,23 @@ namespace {
 // Work of one CTA pair: whole items dealt round-robin.  With the tail split, the items that would not
 // fill a last round are instead laid end to end as one line of K-step groups, cut into `tail_workers`
 // equal ranges and done FIRST: an item is then computed by up to a few pairs, each leaving its fp32
-// partial tile in global scratch.  The pair that holds the item's first steps owns it: once its own
-// share is stored, and while its tensor pipe is already busy with the first whole item, its epilogue
-// warps add the partial tiles in a fixed order and write the output.
+// partial tile in global scratch.  The pair that holds the item's first steps owns it: its own share
+// stays in tensor memory, and while its tensor pipe is already busy with the first whole item, its
+// epilogue warps add the other pairs' partial tiles to it in a fixed order and write the output.
 struct TailSeg { int item, g0, g1, part, nparts; };
 constexpr int kMaxTailSeg = 6;
+constexpr int kMaxTail = 128;  // left-over items are fewer than the pairs of the grid (at most 74)
 struct TailWork {
   int n_full;                 // whole items of this pair: item = cluster_id + k * n_clusters
   int n_seg;
+  int t_first;                // first left-over item this pair has a share of
   TailSeg seg[kMaxTailSeg];
+  int g[kMaxTail];            // step groups of each left-over item
 };
 struct Work { int item, g0, g1, part, nparts; };
 
+// Order of a pair's work: its tail segments first (the first one is a share of a tile another pair owns and is
+// wanted early by that pair), then its whole items.
 __device__ __forceinline__ Work get_work(const TailWork* tw, int wi, int cluster_id, int n_clusters) {
   if (wi >= tw->n_seg) return Work{cluster_id + (wi - tw->n_seg) * n_clusters, 0, 1 << 28, 0, 1};
   const TailSeg& g = tw->seg[wi];
@@ -45,7 +50,7 @@ __device__ __forceinline__ Work get_work(const TailWork* tw, int wi, int cluster
 // Threads of a CTA: producer warp, MMA warp, two sets of four epilogue warps.  The second set (warps 6..9) takes the
 // odd 32-column pieces of every tile, so that a tile with few K steps (a heavily pruned layer with tall kernel
 // groups, a 1x1x1 or 1x3x3 layer) is not bound by its epilogue: four warps need about 15 k clocks for a 128 x 256
-// tile, as long as 30 K steps.  With the tail split only the first set works (the fix-up of shared tiles is theirs).
+// tile, as long as 30 K steps.  Shares and fix-ups of split tiles are divided between the sets the same way.
 constexpr int kThreadsPair = 320;
 
 // kCps: K steps per pipeline stage (and per barrier hand-shake): 1, or 2 for narrow bundles.
@@ -75,7 +80,7 @@ conv3d_umma_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_c
   const int n_items = pairs_per_bundle * a.n_bundles;
   const int cluster_id = blockIdx.x >> 1, n_clusters = gridDim.x >> 1;
   const int box_rows = a.box.bn * a.box.bt * a.box.bh * a.box.bw;
-  const int epi_sets = a.tail_workers == 0 ? 2 : 1;
+  constexpr int epi_sets = 2;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < stages; ++s) {
@@ -106,48 +111,57 @@ conv3d_umma_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_c
   // this CTA holds its TMEM columns (a successor CTA that shared the SM and allocated first could otherwise
   // starve this one while waiting for it); global memory from here on.
   pdl_launch();
+  // The step counts belong to the packed layout, which only host uploads write, never a kernel: the work list
+  // is built before the wait on the predecessor grid (the caller's tensors, bias included, are read after it).
+  // This pair's work list.  The tail split's segment table is built by one thread per left-over item (a lone
+  // thread walking the items, two dependent global loads each, took longer than the split saved).
+  if (threadIdx.x == 0) {
+    tw->n_seg = 0;
+    tw->t_first = 1 << 30;
+    const int rounds = n_items / n_clusters;
+    tw->n_full = a.tail_workers == 0 ? (cluster_id < n_items ? (n_items - cluster_id + n_clusters - 1) / n_clusters : 0)
+                                     : rounds;
+  }
+  if (a.tail_workers > 0) {                                 // uniform over the grid
+    const int first_tail = (n_items / n_clusters) * n_clusters, n_tail = n_items - first_tail;   // n_tail < kMaxTail
+    const int t = threadIdx.x;
+    if (t < n_tail) {
+      const int b = (first_tail + t) / pairs_per_bundle;
+      const int ns = kDense ? a.steps_dense : __ldg(a.step_ptr + b + 1) - __ldg(a.step_ptr + b);
+      tw->g[t] = (ns + kCps - 1) / kCps;
+    }
+    __syncthreads();
+    bool mine = false;
+    long long pre = 0, lo = 0, hi = 0, total = 0;
+    int G = 0;
+    if (t < n_tail && cluster_id < a.tail_workers) {
+      for (int u = 0; u < n_tail; ++u) {
+        const int gu = tw->g[u];
+        if (u < t) pre += gu;
+        total += gu;
+      }
+      G = tw->g[t];
+      const long long W = a.tail_workers;
+      lo = cluster_id * total / W; hi = (cluster_id + 1) * total / W;
+      mine = pre + G > lo && pre < hi;
+      if (mine) atomicMin(&tw->t_first, t);
+    }
+    __syncthreads();
+    if (mine && t - tw->t_first < kMaxTailSeg) {
+      const long long W = a.tail_workers;
+      TailSeg& sg = tw->seg[t - tw->t_first];
+      sg.item = first_tail + t;
+      sg.g0 = int((lo > pre ? lo : pre) - pre);
+      sg.g1 = int((hi < pre + G ? hi : pre + G) - pre);
+      const int first = int(((pre + 1) * W - 1) / total), last = int(((pre + G) * W - 1) / total);
+      sg.part = cluster_id - first;
+      sg.nparts = last - first + 1;
+      atomicAdd(&tw->n_seg, 1);
+    }
+  }
   pdl_wait();
   for (int i = threadIdx.x; i < a.n_bundles * a.n_tile; i += blockDim.x)
     bias_s[i] = (a.bias != nullptr && i < a.g.M) ? __ldg(a.bias + i) : 0.f;
-  if (threadIdx.x == 0) {
-    // this pair's work list
-    tw->n_seg = 0;
-    if (a.tail_workers == 0) {
-      tw->n_full = cluster_id < n_items ? (n_items - cluster_id + n_clusters - 1) / n_clusters : 0;
-    } else {
-      const int rounds = n_items / n_clusters;
-      const int first_tail = rounds * n_clusters, n_tail = n_items - first_tail;
-      tw->n_full = rounds;
-      if (cluster_id < a.tail_workers) {
-        long long total = 0;
-        for (int t = 0; t < n_tail; ++t) {
-          const int b = (first_tail + t) / pairs_per_bundle;
-          const int ns = kDense ? a.steps_dense : a.step_ptr[b + 1] - a.step_ptr[b];
-          total += (ns + kCps - 1) / kCps;
-        }
-        const long long W = a.tail_workers;
-        const long long lo = cluster_id * total / W, hi = (cluster_id + 1) * total / W;
-        long long pre = 0;
-        int n_seg = 0;
-        for (int t = 0; t < n_tail && n_seg < kMaxTailSeg; ++t) {
-          const int b = (first_tail + t) / pairs_per_bundle;
-          const int ns = kDense ? a.steps_dense : a.step_ptr[b + 1] - a.step_ptr[b];
-          const long long G = (ns + kCps - 1) / kCps;
-          if (pre + G > lo && pre < hi) {
-            TailSeg& sg = tw->seg[n_seg++];
-            sg.item = first_tail + t;
-            sg.g0 = int((lo > pre ? lo : pre) - pre);
-            sg.g1 = int((hi < pre + G ? hi : pre + G) - pre);
-            const int first = int(((pre + 1) * W - 1) / total), last = int(((pre + G) * W - 1) / total);
-            sg.part = cluster_id - first;
-            sg.nparts = last - first + 1;
-          }
-          pre += G;
-        }
-        tw->n_seg = n_seg;
-      }
-    }
-  }
   __syncthreads();
 
   if (warp == 0) {
@@ -246,7 +260,7 @@ conv3d_umma_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_c
         umma_commit_pair(smem_u32(&bars->tmem_full[buf]));     // with no MMAs pending this arrives at once
       }
     }
-  } else if (warp < 6 || epi_sets == 2) {
+  } else {
     // ------------------------------------------------------------------ epilogue (both CTAs)
     const int quad = warp & 3;
     const int set = (warp - 2) >> 2;                       // 0: warps 2..5, 1: warps 6..9
@@ -261,7 +275,7 @@ conv3d_umma_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_c
     const __nv_bfloat16* rb = static_cast<const __nv_bfloat16*>(a.residual);
     // two sets: each warp of a quadrant uses one of the quadrant's two staging buffers
     TmaStore ts{&ymap, store_smem + uint32_t(quad) * kStoreWarpBytes + uint32_t(set) * kStoreStageBytes, 0, 0, 0, 0, 0u,
-                epi_sets == 2 ? 1u : kStoreBufs};
+                1u};
     const PoolLanes pool_lanes = make_pool_lanes(a.pool_w, a.pool_h, a.pool_t, a.sbw, a.sbh, lane);
     const PoolLanes* pool = (a.pool_t * a.pool_h * a.pool_w > 1) ? &pool_lanes : nullptr;
     int r0 = quad * 32;                        // coordinates of the warp's first row inside the box
@@ -272,8 +286,6 @@ conv3d_umma_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_c
     uint32_t j = 0;
     const size_t part_tile = size_t(128) * a.n_tile;       // floats per partial tile
     const int n_work = tw->n_full + tw->n_seg;
-    Work own{0, 0, 0, 0, 1};                               // the shared tile this pair owns, if any
-    int own_slot = 0;
     for (int wi = 0; wi < n_work; ++wi, ++j) {
       const Work wk = get_work(tw, wi, cluster_id, n_clusters);
       const PairItem c = decode_pair_item(a, wk.item, pairs_per_bundle, n_mtiles, rank);
@@ -288,28 +300,28 @@ conv3d_umma_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_c
       const uint32_t taddr = tmem_base + (uint32_t(quad * 32) << 16) + buf * uint32_t(a.n_tile);
       const __nv_bfloat16* res = (rb != nullptr && in_range) ? rb + vox * a.rcs + m_base : nullptr;
       const int res_left = a.rcs - m_base;
-      if (wk.nparts > 1) {
-        // shared tile: leave the raw partial sums in scratch and raise this warp's flag.  A pair has at
-        // most two such shares, the first and the last segment of its range.
-        const int slot = (cluster_id * 2 + (wi == 0 ? 0 : 1)) * 2 + int(rank);
-        store_partial_row(taddr, a.n_tile, true, a.tail_scratch + size_t(slot) * part_tile + row);
+      if (wk.nparts > 1 && wk.part != 0) {
+        // A share of a tile another pair owns: leave the raw partial sums in scratch and raise this warp's flag.
+        // It is the first segment of this pair's range.
+        const int slot = cluster_id * 2 + int(rank);
+        store_partial_row(taddr, a.n_tile, true, a.tail_scratch + size_t(slot) * part_tile + row, col0, col_step);
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive_cluster(mapa_shared(smem_u32(&bars->tmem_empty[buf]), 0));
         __threadfence();
         __syncwarp();
-        if (lane == 0) *reinterpret_cast<volatile int32_t*>(a.tail_flags + slot * 4 + quad) = 1;
-        if (wk.part == 0) { own = wk; own_slot = slot; }
-        if (wi + 1 < tw->n_seg) continue;
+        if (lane == 0) *reinterpret_cast<volatile int32_t*>(a.tail_flags + slot * 8 + set * 4 + quad) = 1;
+        continue;
       }
-      if (wi + 1 == tw->n_seg && own.nparts > 1) {
-        // all shares of this pair are stored: finish the tile this pair owns.  The other shares were
-        // computed at the same time by the next pairs (each as the first segment of its range).
+      if (wk.nparts > 1) {
+        // The share of the tile this pair owns (the last segment of its range; its accumulator is still in tensor
+        // memory).  The other shares were computed at the same time by the next pairs, each as the first segment of
+        // its range: wait for their flags, then add their partial tiles to the accumulator in the epilogue.
         int ok = 1;
         if (lane == 0) {
           const long long start = clock64();
-          for (int p = 1; p < own.nparts && ok; ++p) {
-            const volatile int32_t* f = a.tail_flags + (((cluster_id + p) * 2) * 2 + int(rank)) * 4 + quad;
+          for (int p = 1; p < wk.nparts && ok; ++p) {
+            const volatile int32_t* f = a.tail_flags + ((cluster_id + p) * 2 + int(rank)) * 8 + set * 4 + quad;
             while (*f == 0) {
               if (bars->abort_flag || clock64() - start > kWaitCycles) {
                 bars->abort_flag = 1;
@@ -323,26 +335,21 @@ conv3d_umma_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_c
         ok = __shfl_sync(0xffffffffu, ok, 0);
         if (!ok) break;
         __threadfence();
-        const PairItem oc = decode_pair_item(a, own.item, pairs_per_bundle, n_mtiles, rank);
-        const int onn = oc.n0 + bn_i, oto = oc.t0 + bt_i, oho = oc.h0 + bh_i, owo = oc.w0 + bw_i;
-        const bool o_in = row < box_rows && onn < a.g.n && oto < a.g.To && oho < a.g.Ho && owo < a.g.Wo;
-        const long long ovox = (((long long)onn * a.g.To + oto) * a.g.Ho + oho) * a.g.Wo + owo;
-        const int om = oc.bundle * a.n_tile;
-        const __nv_bfloat16* ores = (rb != nullptr && o_in) ? rb + ovox * a.rcs + om : nullptr;
-        ts.c1 = (oc.w0 + bw_0) / a.pool_w; ts.c2 = (oc.h0 + bh_0) / a.pool_h; ts.c3 = (oc.t0 + bt_0) / a.pool_t; ts.c4 = oc.n0 + bn_0;
-        epilogue_row_tma(0u, a.n_tile, false, quad * 32 < box_rows, o_in, bias_s, a.g.relu,
-                         yb + ovox * a.g.ycs + om, om, a.g.M, lane, ts, ores, a.rcs - om, pool,
-                         a.tail_scratch + size_t(own_slot) * part_tile + row,
-                         a.tail_scratch + size_t(((cluster_id + 1) * 2) * 2 + int(rank)) * part_tile + row,
-                         4 * part_tile, own.nparts - 1);
+        ts.c1 = (c.w0 + bw_0) / a.pool_w; ts.c2 = (c.h0 + bh_0) / a.pool_h; ts.c3 = (c.t0 + bt_0) / a.pool_t; ts.c4 = c.n0 + bn_0;
+        epilogue_row_tma(taddr, a.n_tile, true, quad * 32 < box_rows, in_range, bias_s, a.g.relu,
+                         yb + vox * a.g.ycs + m_base, m_base, a.g.M, lane, ts, res, res_left, pool,
+                         a.tail_scratch + size_t((cluster_id + 1) * 2 + int(rank)) * part_tile + row,
+                         a.tail_scratch + size_t((cluster_id + 2) * 2 + int(rank)) * part_tile + row,
+                         2 * part_tile, wk.nparts - 2, col0, col_step);
+        tc_fence_before();
         __syncwarp();
-        if (lane == 0) {                                           // ready for the next launch
-          a.tail_flags[own_slot * 4 + quad] = 0;
-          for (int p = 1; p < own.nparts; ++p) a.tail_flags[(((cluster_id + p) * 2) * 2 + int(rank)) * 4 + quad] = 0;
+        if (lane == 0) {
+          mbar_arrive_cluster(mapa_shared(smem_u32(&bars->tmem_empty[buf]), 0));
+          for (int p = 1; p < wk.nparts; ++p)                        // ready for the next launch
+            a.tail_flags[((cluster_id + p) * 2 + int(rank)) * 8 + set * 4 + quad] = 0;
         }
-        own.nparts = 1;
+        continue;
       }
-      if (wk.nparts > 1) continue;
       if (a.store_tma) {
         ts.c1 = (c.w0 + bw_0) / a.pool_w; ts.c2 = (c.h0 + bh_0) / a.pool_h; ts.c3 = (c.t0 + bt_0) / a.pool_t; ts.c4 = c.n0 + bn_0;
         epilogue_row_tma(taddr, a.n_tile, nsteps > 0, quad * 32 < box_rows, in_range, bias_s, a.g.relu,
@@ -472,7 +479,7 @@ void umma_pair_tail_plan(UmmaArgs* a, const int32_t* step_ptr_host, int sm_count
   if (clusters <= 0 || n_items <= clusters) return;
   const long long rounds = n_items / clusters;
   const int n_tail = int(n_items - rounds * clusters);
-  if (n_tail == 0) return;
+  if (n_tail == 0 || n_tail > kMaxTail) return;
   const int cps = pick_cps(a->n_tile);
   long long total = 0, g_min = 1 << 30, g_max = 0;
   for (int t = 0; t < n_tail; ++t) {
@@ -492,12 +499,12 @@ void umma_pair_tail_plan(UmmaArgs* a, const int32_t* step_ptr_host, int sm_count
   // Storing the shares and the owner's fix-up (four warps pulling the other shares through registers)
   // cost about as much as this many K steps (measured on 256-wide bundles: the split pays for itself
   // from about 100 steps per item).
-  const long long fixup_groups = (48 + cps - 1) / cps;
+  const long long fixup_groups = (12 + cps - 1) / cps;
   if (range + fixup_groups >= g_max) return;
   a->tail_workers = int(workers);
-  // per pair: up to two shares (first and last segment of its range) x two CTAs
-  *scratch_bytes = size_t(workers) * 4 * 128 * a->n_tile * sizeof(float);
-  *flag_bytes = size_t(workers) * 4 * 4 * sizeof(int32_t);
+  // per pair: one share (the first segment of its range) x two CTAs; one flag per epilogue warp
+  *scratch_bytes = size_t(workers) * 2 * 128 * a->n_tile * sizeof(float);
+  *flag_bytes = size_t(workers) * 2 * 8 * sizeof(int32_t);
 }
 
 cudaError_t launch_conv_umma_pair(const UmmaArgs& a, const void* xmap, const void* wmap_half, const void* ymap,
