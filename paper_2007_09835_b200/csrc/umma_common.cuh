@@ -178,6 +178,19 @@ __device__ __forceinline__ void tmem_ld16_into32(uint32_t taddr, uint32_t (&r)[3
 #pragma unroll
   for (int q = 0; q < 16; ++q) { r[q] = t[q]; r[q + 16] = 0u; }
 }
+// 32 (or 16) accumulator columns of this thread's row; `acc2_off` != 0: the tile was accumulated in two halves by
+// two issuing threads, the second one `acc2_off` columns further on, and the two are added here (warp-uniform).
+__device__ __forceinline__ void tmem_ld_acc(uint32_t taddr, bool wide, uint32_t acc2_off, uint32_t (&v)[32]) {
+  if (wide) tmem_ld32(taddr, v);
+  else tmem_ld16_into32(taddr, v);
+  if (acc2_off) {
+    uint32_t v2[32];
+    if (wide) tmem_ld32(taddr + acc2_off, v2);
+    else tmem_ld16_into32(taddr + acc2_off, v2);
+#pragma unroll
+    for (int q = 0; q < 32; ++q) v[q] = __float_as_uint(__uint_as_float(v[q]) + __uint_as_float(v2[q]));
+  }
+}
 
 // Epilogue of NC (16 or 32) accumulator columns of one output voxel: + bias (from shared memory),
 // optional ReLU, round to bf16, store.  `valid` = number of real output channels among the NC
@@ -234,6 +247,28 @@ __device__ __forceinline__ void epilogue_cols(const uint32_t* v, const float* bi
   }
 }
 
+// Partial sums of the same tile left in scratch by other CTAs (column-major [column][128 rows] floats, pointers
+// at this thread's row), added to the 32 (or 16) accumulator columns from `col` on in a fixed order: extra_first,
+// then extra + p * extra_stride.  Two partial tiles' loads are in flight at a time.
+__device__ __forceinline__ void add_partials(uint32_t (&v)[32], bool wide, int col, const float* extra_first,
+                                             const float* extra, size_t extra_stride, int n_extra) {
+  const float* e0 = extra_first + size_t(col) * 128;
+  for (int p = -1; p < n_extra; p += 2) {
+    const float* ea = p < 0 ? e0 : extra + size_t(p) * extra_stride + size_t(col) * 128;
+    const bool two = p + 1 < n_extra;
+    const float* eb = two ? extra + size_t(p + 1) * extra_stride + size_t(col) * 128 : ea;
+    float t0[32], t1[32];
+#pragma unroll
+    for (int q = 0; q < 32; ++q) {
+      const bool live = wide || q < 16;
+      t0[q] = live ? __ldcg(ea + size_t(q) * 128) : 0.f;
+      t1[q] = (live && two) ? __ldcg(eb + size_t(q) * 128) : 0.f;
+    }
+#pragma unroll
+    for (int q = 0; q < 32; ++q) v[q] = __float_as_uint((__uint_as_float(v[q]) + t0[q]) + t1[q]);
+  }
+}
+
 // One voxel row of a finished accumulator tile: columns [0, n_cols) of the TMEM buffer at `taddr`
 // hold output channels m_base.. ; channels >= M are dropped.  Warp-uniform control flow around the
 // TMEM loads (.sync.aligned); `in_range` may differ per lane.
@@ -242,20 +277,22 @@ __device__ __forceinline__ void epilogue_cols(const uint32_t* v, const float* bi
 __device__ __forceinline__ void epilogue_row(uint32_t taddr, int n_cols, bool has_acc, bool in_range,
                                              const float* bias_s, int relu, __nv_bfloat16* dst, int m_base, int M,
                                              const __nv_bfloat16* res_row = nullptr, int res_pitch_left = 0,
-                                             int col0 = 0, int col_step = 32) {
+                                             int col0 = 0, int col_step = 32, const float* extra_first = nullptr,
+                                             const float* extra = nullptr, size_t extra_stride = 0, int n_extra = 0,
+                                             uint32_t acc2_off = 0) {
   for (int col = col0; col < n_cols; col += col_step) {
     const int m0 = m_base + col;
     if (m0 >= M) break;
     uint32_t v[32];
     const bool wide = col + 32 <= n_cols;
     if (has_acc) {
-      if (wide) tmem_ld32(taddr + col, v);
-      else tmem_ld16_into32(taddr + col, v);
+      tmem_ld_acc(taddr + col, wide, acc2_off, v);
     } else {
 #pragma unroll
       for (int q = 0; q < 32; ++q) v[q] = 0u;
     }
     if (!in_range) continue;
+    if (extra_first != nullptr) add_partials(v, wide, col, extra_first, extra, extra_stride, n_extra);
     const __nv_bfloat16* res = res_row ? res_row + col : nullptr;
     const float* bs = bias_s ? bias_s + m0 : nullptr;
     if (wide) epilogue_cols<32>(v, bs, relu, dst + col, M - m0, res, res_pitch_left - col);
@@ -427,7 +464,8 @@ __device__ __forceinline__ void epilogue_row_tma(uint32_t taddr, int n_cols, boo
                                                  const __nv_bfloat16* res_row = nullptr, int res_pitch_left = 0,
                                                  const PoolLanes* pool = nullptr, const float* extra_first = nullptr,
                                                  const float* extra = nullptr, size_t extra_stride = 0,
-                                                 int n_extra = 0, int col0 = 0, int col_step = 32) {
+                                                 int n_extra = 0, int col0 = 0, int col_step = 32,
+                                                 uint32_t acc2_off = 0) {
   // col0 / col_step: a second warp on the same TMEM lane quadrant takes every other 32-column piece
   for (int col = col0; col < n_cols; col += col_step) {
     const int m0 = m_base + col;
@@ -435,32 +473,12 @@ __device__ __forceinline__ void epilogue_row_tma(uint32_t taddr, int n_cols, boo
     uint32_t v[32];
     const bool wide = col + 32 <= n_cols;
     if (has_acc) {
-      if (wide) tmem_ld32(taddr + col, v);
-      else tmem_ld16_into32(taddr + col, v);
+      tmem_ld_acc(taddr + col, wide, acc2_off, v);
     } else {
 #pragma unroll
       for (int q = 0; q < 32; ++q) v[q] = 0u;
     }
-    // partial sums of the same tile left in scratch by this and other CTAs (column-major [column][128 rows],
-    // pointers at this thread's row), added in a fixed order: extra_first, then extra + p * extra_stride.
-    // Two partial tiles' loads are in flight at a time.
-    if (extra_first != nullptr) {
-      const float* e0 = extra_first + size_t(col) * 128;
-      for (int p = -1; p < n_extra; p += 2) {
-        const float* ea = p < 0 ? e0 : extra + size_t(p) * extra_stride + size_t(col) * 128;
-        const bool two = p + 1 < n_extra;
-        const float* eb = two ? extra + size_t(p + 1) * extra_stride + size_t(col) * 128 : ea;
-        float t0[32], t1[32];
-#pragma unroll
-        for (int q = 0; q < 32; ++q) {
-          const bool live = wide || q < 16;
-          t0[q] = live ? __ldcg(ea + size_t(q) * 128) : 0.f;
-          t1[q] = (live && two) ? __ldcg(eb + size_t(q) * 128) : 0.f;
-        }
-#pragma unroll
-        for (int q = 0; q < 32; ++q) v[q] = __float_as_uint((__uint_as_float(v[q]) + t0[q]) + t1[q]);
-      }
-    }
+    if (extra_first != nullptr) add_partials(v, wide, col, extra_first, extra, extra_stride, n_extra);
     const __nv_bfloat16* res = (res_row && in_range) ? res_row + col : nullptr;
     if (wide) {
       if (warp_rows_valid) epilogue_piece_tma(v, bias_s ? bias_s + m0 : nullptr, relu, m0, lane, ts, res, res_pitch_left - col, pool);
@@ -474,13 +492,12 @@ __device__ __forceinline__ void epilogue_row_tma(uint32_t taddr, int n_cols, boo
 // warp (32 consecutive rows) always touch 128 contiguous bytes.
 // Raw fp32 accumulator row -> scratch; `dst` already points at this thread's row of column 0.
 __device__ __forceinline__ void store_partial_row(uint32_t taddr, int n_cols, bool has_acc, float* dst, int col0 = 0,
-                                                  int col_step = 32) {
+                                                  int col_step = 32, uint32_t acc2_off = 0) {
   for (int col = col0; col < n_cols; col += col_step) {
     uint32_t v[32];
     const bool wide = col + 32 <= n_cols;
     if (has_acc) {
-      if (wide) tmem_ld32(taddr + col, v);
-      else tmem_ld16_into32(taddr + col, v);
+      tmem_ld_acc(taddr + col, wide, acc2_off, v);
     } else {
 #pragma unroll
       for (int q = 0; q < 32; ++q) v[q] = 0u;

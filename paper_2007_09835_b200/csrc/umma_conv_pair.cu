@@ -47,11 +47,12 @@ __device__ __forceinline__ Work get_work(const TailWork* tw, int wi, int cluster
   return Work{g.item, g.g0, g.g1, g.part, g.nparts};
 }
 
-// Threads of a CTA: producer warp, MMA warp, two sets of four epilogue warps.  The second set (warps 6..9) takes the
+// Threads of a CTA: producer warp, MMA warp, two sets of four epilogue warps, and a second MMA warp (warp 10) that
+// only narrow bundles use.  The second epilogue set (warps 6..9) takes the
 // odd 32-column pieces of every tile, so that a tile with few K steps (a heavily pruned layer with tall kernel
 // groups, a 1x1x1 or 1x3x3 layer) is not bound by its epilogue: four warps need about 15 k clocks for a 128 x 256
 // tile, as long as 30 K steps.  Shares and fix-ups of split tiles are divided between the sets the same way.
-constexpr int kThreadsPair = 320;
+constexpr int kThreadsPair = 352;
 
 // kCps: K steps per pipeline stage (and per barrier hand-shake): 1, or 2 for narrow bundles.
 template <bool kDense, int kCps>
@@ -81,6 +82,11 @@ conv3d_umma_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_c
   const int cluster_id = blockIdx.x >> 1, n_clusters = gridDim.x >> 1;
   const int box_rows = a.box.bn * a.box.bt * a.box.bh * a.box.bw;
   constexpr int epi_sets = 2;
+  // Narrow bundles (kCps == 2, N <= 128): one thread cannot issue MMAs and run the barrier hand-shakes as fast as
+  // the tensor pipe executes them, so two threads issue alternate step groups, each into its own accumulator
+  // (2 buffers x 2 x N <= 512 columns); the epilogue adds the two.  Fixed order, so results stay repeatable.
+  constexpr bool kDual = kCps == 2;
+  constexpr int kIss = kDual ? 2 : 1;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < stages; ++s) {
@@ -88,7 +94,7 @@ conv3d_umma_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_c
       mbar_init(smem_u32(&bars->empty[s]), 1);    // multicast commit
     }
     for (int b = 0; b < 2; ++b) {
-      mbar_init(smem_u32(&bars->tmem_full[b]), 1);    // multicast commit
+      mbar_init(smem_u32(&bars->tmem_full[b]), kIss);  // multicast commit of every issuing thread
       mbar_init(smem_u32(&bars->tmem_empty[b]), uint32_t(8 * epi_sets));   // leader: the working epilogue warps of both CTAs
     }
     bars->abort_flag = 0;
@@ -218,9 +224,10 @@ conv3d_umma_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_c
         }
       }
     }
-  } else if (warp == 1) {
-    // ------------------------------------------------------------------ MMA issuer (leader CTA only)
+  } else if (warp == 1 || (kDual && warp == 10)) {
+    // ------------------------------------------------------------------ MMA issuer(s) (leader CTA only)
     if (lane == 0 && leader) {
+      const int me = warp == 1 ? 0 : 1;                      // which step groups of an item: even / odd
       const uint32_t idesc = instr_desc_bf16_pair(a.n_tile);
       uint32_t j = 0, phase = 0;
       int stage = 0;
@@ -234,33 +241,36 @@ conv3d_umma_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_c
         const uint32_t buf = j & 1u;
         if (!mbar_wait(smem_u32(&bars->tmem_empty[buf]), ((j >> 1) & 1u) ^ 1u, bars, err, 22)) break;
         tc_fence_after();
-        const uint32_t d_tmem = tmem_base + buf * uint32_t(a.n_tile);
-        for (int i = i0; i < i1; i += kCps) {
+        const uint32_t d_tmem = tmem_base + (buf * uint32_t(kIss) + uint32_t(me)) * uint32_t(a.n_tile);
+        int gl = 0;                                          // step group inside this item
+        for (int i = i0; i < i1; i += kCps, ++gl) {
           const int nload = i1 - i < kCps ? i1 - i : kCps;
-          if (!ready && !mbar_wait(smem_u32(&bars->full[stage]), phase, bars, err, 23)) { ok = false; break; }
-          // poll the next stage's barrier now: its answer arrives while this stage's MMAs are issued
           const int stage_n = stage + 1 == stages ? 0 : stage + 1;
           const uint32_t phase_n = stage + 1 == stages ? phase ^ 1u : phase;
-          ready = mbar_try_wait(smem_u32(&bars->full[stage_n]), phase_n);
-          tc_fence_after();
+          if (!kDual || (gl & 1) == me) {
+            if (!ready && !mbar_wait(smem_u32(&bars->full[stage]), phase, bars, err, 23)) { ok = false; break; }
+            // one issuer: poll the next stage's barrier now, its answer arrives while this stage's MMAs are issued
+            ready = kDual ? false : mbar_try_wait(smem_u32(&bars->full[stage_n]), phase_n);
+            tc_fence_after();
 #pragma unroll
-          for (int q = 0; q < kCps; ++q) {
-            if (q >= nload) break;
-            const uint32_t a_addr = tiles_base + stage * stage_bytes + q * chunk_bytes;
-            const uint64_t adesc = smem_desc_sw128(a_addr);
-            const uint64_t bdesc = smem_desc_sw128(a_addr + kABytes);
+            for (int q = 0; q < kCps; ++q) {
+              if (q >= nload) break;
+              const uint32_t a_addr = tiles_base + stage * stage_bytes + q * chunk_bytes;
+              const uint64_t adesc = smem_desc_sw128(a_addr);
+              const uint64_t bdesc = smem_desc_sw128(a_addr + kABytes);
 #pragma unroll
-            for (int kk = 0; kk < 4; ++kk)
-              umma_bf16_pair(d_tmem, adesc + 2 * kk, bdesc + 2 * kk, idesc, ((i - i0) | q | kk) ? 1u : 0u);
+              for (int kk = 0; kk < 4; ++kk)
+                umma_bf16_pair(d_tmem, adesc + 2 * kk, bdesc + 2 * kk, idesc, ((gl >= kIss) | q | kk) ? 1u : 0u);
+            }
+            umma_commit_pair(smem_u32(&bars->empty[stage]));
           }
-          umma_commit_pair(smem_u32(&bars->empty[stage]));
           stage = stage_n; phase = phase_n;
         }
         if (!ok) break;
         umma_commit_pair(smem_u32(&bars->tmem_full[buf]));     // with no MMAs pending this arrives at once
       }
     }
-  } else {
+  } else if (warp < 10) {
     // ------------------------------------------------------------------ epilogue (both CTAs)
     const int quad = warp & 3;
     const int set = (warp - 2) >> 2;                       // 0: warps 2..5, 1: warps 6..9
@@ -297,14 +307,17 @@ conv3d_umma_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_c
       const bool in_range = row < box_rows && nn < a.g.n && to < a.g.To && ho < a.g.Ho && wo < a.g.Wo;
       const long long vox = (((long long)nn * a.g.To + to) * a.g.Ho + ho) * a.g.Wo + wo;
       const int m_base = c.bundle * a.n_tile;
-      const uint32_t taddr = tmem_base + (uint32_t(quad * 32) << 16) + buf * uint32_t(a.n_tile);
+      const uint32_t taddr = tmem_base + (uint32_t(quad * 32) << 16) + buf * uint32_t(kIss * a.n_tile);
+      // the second issuer's accumulator holds something once the item (or share) has two step groups
+      const int steps_here = (wk.g1 * kCps < nsteps ? wk.g1 * kCps : nsteps) - wk.g0 * kCps;
+      const uint32_t acc2 = (kDual && steps_here > kCps) ? uint32_t(a.n_tile) : 0u;
       const __nv_bfloat16* res = (rb != nullptr && in_range) ? rb + vox * a.rcs + m_base : nullptr;
       const int res_left = a.rcs - m_base;
       if (wk.nparts > 1 && wk.part != 0) {
         // A share of a tile another pair owns: leave the raw partial sums in scratch and raise this warp's flag.
         // It is the first segment of this pair's range.
         const int slot = cluster_id * 2 + int(rank);
-        store_partial_row(taddr, a.n_tile, true, a.tail_scratch + size_t(slot) * part_tile + row, col0, col_step);
+        store_partial_row(taddr, a.n_tile, true, a.tail_scratch + size_t(slot) * part_tile + row, col0, col_step, acc2);
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive_cluster(mapa_shared(smem_u32(&bars->tmem_empty[buf]), 0));
@@ -335,12 +348,17 @@ conv3d_umma_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_c
         ok = __shfl_sync(0xffffffffu, ok, 0);
         if (!ok) break;
         __threadfence();
-        ts.c1 = (c.w0 + bw_0) / a.pool_w; ts.c2 = (c.h0 + bh_0) / a.pool_h; ts.c3 = (c.t0 + bt_0) / a.pool_t; ts.c4 = c.n0 + bn_0;
-        epilogue_row_tma(taddr, a.n_tile, true, quad * 32 < box_rows, in_range, bias_s, a.g.relu,
-                         yb + vox * a.g.ycs + m_base, m_base, a.g.M, lane, ts, res, res_left, pool,
-                         a.tail_scratch + size_t((cluster_id + 1) * 2 + int(rank)) * part_tile + row,
-                         a.tail_scratch + size_t((cluster_id + 2) * 2 + int(rank)) * part_tile + row,
-                         2 * part_tile, wk.nparts - 2, col0, col_step);
+        const float* e_first = a.tail_scratch + size_t((cluster_id + 1) * 2 + int(rank)) * part_tile + row;
+        const float* e_more = a.tail_scratch + size_t((cluster_id + 2) * 2 + int(rank)) * part_tile + row;
+        if (a.store_tma) {
+          ts.c1 = (c.w0 + bw_0) / a.pool_w; ts.c2 = (c.h0 + bh_0) / a.pool_h; ts.c3 = (c.t0 + bt_0) / a.pool_t; ts.c4 = c.n0 + bn_0;
+          epilogue_row_tma(taddr, a.n_tile, true, quad * 32 < box_rows, in_range, bias_s, a.g.relu,
+                           yb + vox * a.g.ycs + m_base, m_base, a.g.M, lane, ts, res, res_left, pool,
+                           e_first, e_more, 2 * part_tile, wk.nparts - 2, col0, col_step, acc2);
+        } else {
+          epilogue_row(taddr, a.n_tile, true, in_range, bias_s, a.g.relu, yb + vox * a.g.ycs + m_base, m_base, a.g.M,
+                       res, res_left, col0, col_step, e_first, e_more, 2 * part_tile, wk.nparts - 2, acc2);
+        }
         tc_fence_before();
         __syncwarp();
         if (lane == 0) {
@@ -354,10 +372,10 @@ conv3d_umma_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_c
         ts.c1 = (c.w0 + bw_0) / a.pool_w; ts.c2 = (c.h0 + bh_0) / a.pool_h; ts.c3 = (c.t0 + bt_0) / a.pool_t; ts.c4 = c.n0 + bn_0;
         epilogue_row_tma(taddr, a.n_tile, nsteps > 0, quad * 32 < box_rows, in_range, bias_s, a.g.relu,
                          yb + vox * a.g.ycs + m_base, m_base, a.g.M, lane, ts, res, res_left, pool, nullptr, nullptr, 0, 0,
-                         col0, col_step);
+                         col0, col_step, acc2);
       } else {
         epilogue_row(taddr, a.n_tile, nsteps > 0, in_range, bias_s, a.g.relu, yb + vox * a.g.ycs + m_base, m_base, a.g.M,
-                     res, res_left, col0, col_step);
+                     res, res_left, col0, col_step, nullptr, nullptr, 0, 0, acc2);
       }
       tc_fence_before();
       __syncwarp();
@@ -454,7 +472,8 @@ cudaError_t launch_pair_t(const UmmaArgs& a, const CUtensorMap& xm, const CUtens
   cudaError_t e = prepare_pair_t<kDense, kCps>();
   if (e != cudaSuccess) return e;
   long long clusters = pair_max_clusters_t<kDense, kCps>(sm_count, smem);
-  if (clusters > n_items) clusters = n_items;
+  const long long want = n_items > a.tail_workers ? n_items : a.tail_workers;
+  if (clusters > want) clusters = want;
   LaunchSetup ls(dim3(unsigned(2 * clusters)), dim3(kThreadsPair), smem, stream, 2);
   return cudaLaunchKernelEx(&ls.cfg, conv3d_umma_pair_kernel<kDense, kCps>, xm, wm, ym, a, stages, cols);
 }
@@ -471,12 +490,13 @@ void umma_pair_tail_plan(UmmaArgs* a, const int32_t* step_ptr_host, int sm_count
                          size_t* flag_bytes) {
   a->tail_workers = 0;
   *scratch_bytes = 0; *flag_bytes = 0;
-  if (!a->store_tma || !umma_pair_supported(a->n_tile, a->n_bundles)) return;
+  if (!umma_pair_supported(a->n_tile, a->n_bundles)) return;
   const long long n_mtiles = (long long)a->tiles_n * a->tiles_t * a->tiles_h * a->tiles_w;
   const long long pairs_per_bundle = (n_mtiles + 1) / 2;
   const long long n_items = pairs_per_bundle * a->n_bundles;
   const int clusters = pair_max_clusters(a->n_tile, a->n_bundles, a->dense != 0, sm_count);
-  if (clusters <= 0 || n_items <= clusters) return;
+  if (clusters <= 0) return;
+  // fewer items than pairs: every item is a left-over item, the grid is `tail_workers` pairs
   const long long rounds = n_items / clusters;
   const int n_tail = int(n_items - rounds * clusters);
   if (n_tail == 0 || n_tail > kMaxTail) return;
@@ -491,7 +511,8 @@ void umma_pair_tail_plan(UmmaArgs* a, const int32_t* step_ptr_host, int sm_count
     g_min = g < g_min ? g : g_min; g_max = g > g_max ? g : g_max;
   }
   long long workers = clusters;
-  if (workers > 4LL * n_tail) workers = 4LL * n_tail;     // at most about four parts per item
+  const long long max_parts = rounds == 0 ? 8 : 4;        // parts per item, about
+  if (workers > max_parts * n_tail) workers = max_parts * n_tail;
   if (workers > total / 4) workers = total / 4;           // at least four step groups per part
   if (workers <= n_tail) return;
   const long long range = (total + workers - 1) / workers;
@@ -514,7 +535,7 @@ cudaError_t launch_conv_umma_pair(const UmmaArgs& a, const void* xmap, const voi
   const int stages = pick_stages_pair(a.n_tile);
   const size_t smem = pair_smem_bytes(a.n_tile, a.n_bundles);
   int cols = 32;
-  while (cols < 2 * a.n_tile) cols *= 2;
+  while (cols < 2 * a.n_tile * (pick_cps(a.n_tile) == 2 ? 2 : 1)) cols *= 2;     // two issuing threads: two accumulators
   if (cols > 512) return cudaErrorInvalidValue;
   const long long n_mtiles = (long long)a.tiles_n * a.tiles_t * a.tiles_h * a.tiles_w;
   const long long n_items = ((n_mtiles + 1) / 2) * a.n_bundles;
