@@ -147,6 +147,11 @@ rt3d_status rt3d_unpack_to_dense(const rt3d_packed* p, float* w_out);
  * `n_tile` output channels (0 = the library's choice): w_out as above.  Lets a host-only
  * test check that derived layout against the canonical one. */
 rt3d_status rt3d_unpack_device_layout(const rt3d_packed* p, int n_tile, float* w_out);
+/* The same for the t-grouped order of that layout (steps ordered by (kh, kw), channel chunk, kt; the runs that
+ * differ only in kt are the groups whose steps share one staged input tile in the CTA-pair kernel).  Also checks
+ * the group tables: RT3D_ERR_INVALID_ARG if the groups do not tile every bundle's list or a group mixes
+ * locations other than along kt. */
+rt3d_status rt3d_unpack_device_layout_tgroups(const rt3d_packed* p, int n_tile, float* w_out);
 
 /* The same check for the layout of the sub-tile kernel (RT3D_ALGO_UMMA_SUB): w_out is rebuilt from the
  * 16 x 16 weight blocks and the step headers; RT3D_ERR_INVALID_ARG if they are inconsistent (a non-zero
@@ -326,6 +331,7 @@ rt3d_status rt3d_conv3d_cost(const rt3d_tensor* x, const rt3d_packed* w, const r
  *                3 tensor-core small-C_in kernel, 4 tensor-core resident-weight (halo) kernel,
  *                5 fused (2+1)D kernel (rt3d_conv2plus1d_fused; n_tile = intermediate width),
  *                6 tensor-core sub-tile kernel (RT3D_ALGO_UMMA_SUB)
+ *                7 tensor-core CTA-pair kernel, one deeper input tile per (kh, kw, chunk) shared by all kt
  *   n_tile       output channels per accumulator tile (tensor-core kernels, else 0)
  *   n_splits     K splits per output tile in the single-CTA kernel (1 = none)
  *   tail_workers CTA pairs that share, cut along K, the output tiles which do not fill a last round
@@ -366,8 +372,11 @@ void rt3d_plan_end(void);
  * tensor-core kernel gives up (0 = default, about one second; the environment variable
  * RT3D_DEBUG_TIMEOUT_POLLS sets the initial value).  RT3D_DEBUG_DROP_LAST_LOAD: nonzero makes that kernel's
  * producer skip the loads of each CTA's last pipeline stage, so that the wait on them runs out and the error
- * path (RT3D_ERR_TIMEOUT from rt3d_last_device_status) can be exercised without any fault. */
-enum { RT3D_DEBUG_WAIT_CYCLES = 1, RT3D_DEBUG_DROP_LAST_LOAD = 2 };
+ * path (RT3D_ERR_TIMEOUT from rt3d_last_device_status) can be exercised without any fault.
+ * RT3D_DEBUG_T_GROUPS: 0 switches off the CTA-pair kernel's variant that stages one deeper input tile per
+ * (kh, kw, channel chunk) for all kt (plan kernel 7), so that it can be compared with the step-per-location
+ * form (kernel 2) on the same handle; default 1. */
+enum { RT3D_DEBUG_WAIT_CYCLES = 1, RT3D_DEBUG_DROP_LAST_LOAD = 2, RT3D_DEBUG_T_GROUPS = 3 };
 rt3d_status rt3d_debug_set(int what, long long value);
 
 const char* rt3d_status_string(rt3d_status s);

@@ -70,6 +70,7 @@ def _load():
     lib.rt3d_packed_view_get.argtypes = [vp, ctypes.POINTER(PackedView)]
     lib.rt3d_unpack_to_dense.argtypes = [vp, f32p]
     lib.rt3d_unpack_device_layout.argtypes = [vp, i, f32p]
+    lib.rt3d_unpack_device_layout_tgroups.argtypes = [vp, i, f32p]
     lib.rt3d_unpack_sub_layout.argtypes = [vp, i, f32p]
     lib.rt3d_packed_prepare.argtypes = [vp]
     lib.rt3d_packed_free.argtypes = [vp]
@@ -143,11 +144,11 @@ class Packed:
                "rt3d_unpack_to_dense")
         return out
 
-    def unpack_device_layout(self, n_tile: int = 0) -> np.ndarray:
+    def unpack_device_layout(self, n_tile: int = 0, t_groups: bool = False) -> np.ndarray:
         v = self.view()
         out = np.empty((v["M"], v["N"], v["Kt"], v["Kh"], v["Kw"]), np.float32)
-        _check(_lib.rt3d_unpack_device_layout(self.handle, int(n_tile),
-                                              out.ctypes.data_as(ctypes.POINTER(ctypes.c_float))),
+        fn = _lib.rt3d_unpack_device_layout_tgroups if t_groups else _lib.rt3d_unpack_device_layout
+        _check(fn(self.handle, int(n_tile), out.ctypes.data_as(ctypes.POINTER(ctypes.c_float))),
                "rt3d_unpack_device_layout")
         return out
 
@@ -389,7 +390,7 @@ def rt3d_alloc_count() -> int:
     return int(_lib.rt3d_alloc_count())
 
 
-DEBUG_WAIT_CYCLES, DEBUG_DROP_LAST_LOAD = 1, 2
+DEBUG_WAIT_CYCLES, DEBUG_DROP_LAST_LOAD, DEBUG_T_GROUPS = 1, 2, 3
 
 
 def rt3d_debug_set(what: int, value: int):

@@ -36,6 +36,7 @@ thread_local bool t_plan_only = false;
 // Test hooks of the single-CTA tensor-core kernel (rt3d_debug_set).
 std::atomic<long long> g_debug_wait_cycles{-1};      // -1: not set yet (RT3D_DEBUG_TIMEOUT_POLLS is read on first use)
 std::atomic<int> g_debug_drop_last_load{0};
+std::atomic<int> g_ts_enabled{1};            // t-grouped CTA-pair variant (RT3D_DEBUG_T_GROUPS switches it off for comparisons)
 long long debug_wait_cycles() {
   long long v = g_debug_wait_cycles.load();
   if (v < 0) {
@@ -187,7 +188,7 @@ rt3d_status get_blob(rt3d_packed* h, DeviceBlob** out) {
 
 rt3d_status get_umma_blob(rt3d_packed* h, DeviceBlob* blob, const UmmaLayout* L, DeviceBlob::Umma** out) {
   std::lock_guard<std::mutex> lock(h->mu);
-  DeviceBlob::Umma& u = blob->umma[L->n_tile];
+  DeviceBlob::Umma& u = blob->umma[L->n_tile + (L->t_groups ? 4096 : 0)];
   if (!u.ready) {
     const size_t wbytes = L->wtiles.size() * 2;
     if (dev_malloc(&u.wtiles, wbytes + 1024) != cudaSuccess ||
@@ -199,6 +200,14 @@ rt3d_status get_umma_blob(rt3d_packed* h, DeviceBlob* blob, const UmmaLayout* L,
         (!L->steps.empty() &&
          cudaMemcpy(u.steps, L->steps.data(), L->steps.size() * 4, cudaMemcpyHostToDevice) != cudaSuccess))
       return RT3D_ERR_CUDA;
+    if (L->t_groups) {
+      if (dev_malloc(&u.grp_ptr, L->grp_ptr.size() * 4) != cudaSuccess ||
+          dev_malloc(&u.grp_first, L->grp_first.size() * 4) != cudaSuccess)
+        return RT3D_ERR_ALLOC;
+      if (cudaMemcpy(u.grp_ptr, L->grp_ptr.data(), L->grp_ptr.size() * 4, cudaMemcpyHostToDevice) != cudaSuccess ||
+          cudaMemcpy(u.grp_first, L->grp_first.data(), L->grp_first.size() * 4, cudaMemcpyHostToDevice) != cudaSuccess)
+        return RT3D_ERR_CUDA;
+    }
     // 2-D map over the weight tiles: rows of 64 bf16 (128 bytes), one box = one [n_tile][64] tile
     const cuuint64_t rows = L->steps.empty() ? cuuint64_t(L->n_tile) : cuuint64_t(L->steps.size()) * L->n_tile;
     cuuint64_t dims[2] = {64, rows};
@@ -245,7 +254,9 @@ rt3d_status get_sub_blob(rt3d_packed* h, DeviceBlob* blob, const SubLayout* L, D
 // ------------------------------------------------------------------------ tile planning
 // Box of output voxels (bn x bt x bh x bw <= 128) that covers the output with the fewest tiles;
 // ties go to the wider box along w, then h (longer contiguous runs for the TMA engine).
-TileBox choose_box(const ConvGeom& g) {
+// `prefer_deep`: ties go first to boxes inside one clip, then to the deeper box along t (the t-grouped CTA-pair
+// variant shares one staged input tile between the kt steps; the deeper the box, the less the extra frames weigh).
+TileBox choose_box(const ConvGeom& g, bool prefer_deep = false) {
   TileBox best{1, 1, 1, 1};
   long long best_tiles = -1;
   for (int bw = 1; bw <= g.Wo && bw <= kTileM; ++bw) {
@@ -258,7 +269,9 @@ TileBox choose_box(const ConvGeom& g) {
         if (bn > g.n) bn = g.n;
         const long long tiles = (long long)ceil_div(g.n, bn) * ceil_div(g.To, bt) * ceil_div(g.Ho, bh) * ceil_div(g.Wo, bw);
         bool better = best_tiles < 0 || tiles < best_tiles;
-        if (!better && tiles == best_tiles) {
+        if (!better && tiles == best_tiles && prefer_deep && ((bn == 1) != (best.bn == 1) || bt != best.bt)) {
+          better = (bn == 1) != (best.bn == 1) ? bn == 1 : bt > best.bt;
+        } else if (!better && tiles == best_tiles) {
           if (bw > best.bw) better = true;
           else if (bw == best.bw && bh > best.bh) better = true;
         }
@@ -322,12 +335,13 @@ bool umma_eligible(const DeviceState* d, const rt3d_packed* w, const rt3d_tensor
   return true;
 }
 
-rt3d_status encode_xmap(const rt3d_tensor* x, const ConvGeom& g, const TileBox& box, CUtensorMap* map) {
+// `extra_t`: frames added to the box along t (the t-grouped CTA-pair variant stages Kt - 1 more; temporal stride 1).
+rt3d_status encode_xmap(const rt3d_tensor* x, const ConvGeom& g, const TileBox& box, CUtensorMap* map, int extra_t = 0) {
   const cuuint64_t cs = cuuint64_t(x->c_stride) * 2;
   cuuint64_t dims[5] = {cuuint64_t(x->c), cuuint64_t(x->w), cuuint64_t(x->h), cuuint64_t(x->t), cuuint64_t(x->n)};
   cuuint64_t strides[4] = {cs, cs * x->w, cs * x->w * x->h, cs * x->w * x->h * x->t};
   // with a traversal stride s the engine loads ceil(box / s) elements, so a box of b outputs spans b*s inputs
-  cuuint32_t bx[5] = {64, cuuint32_t(box.bw * g.sw), cuuint32_t(box.bh * g.sh), cuuint32_t(box.bt * g.st),
+  cuuint32_t bx[5] = {64, cuuint32_t(box.bw * g.sw), cuuint32_t(box.bh * g.sh), cuuint32_t(box.bt * g.st + extra_t),
                       cuuint32_t(box.bn)};
   cuuint32_t estr[5] = {1, cuuint32_t(g.sw), cuuint32_t(g.sh), cuuint32_t(g.st), 1};
   CUresult r = g_encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, x->data, dims, strides, bx, estr,
@@ -368,7 +382,7 @@ bool encode_ymap(const rt3d_tensor* y, const int sb[4], int pw, int ph, int pt, 
 
 // Box for a call with fused pooling: fewest tiles among the boxes whose extents and whose per-warp block
 // are multiples of the pooling window (every window then lies inside one warp's 32 voxels).
-bool choose_box_pool(const ConvGeom& g, int pw, int ph, int pt, TileBox* out, int sb_out[4]) {
+bool choose_box_pool(const ConvGeom& g, int pw, int ph, int pt, TileBox* out, int sb_out[4], bool prefer_deep = false) {
   long long best_tiles = -1;
   for (int bw = pw; bw <= kTileM && bw <= round_up(g.Wo, pw); bw += pw) {
     if (bw * g.sw > 256) break;
@@ -381,7 +395,12 @@ bool choose_box_pool(const ConvGeom& g, int pw, int ph, int pt, TileBox* out, in
         int sb[4];
         if (!warp_block(bw, bh, bt, bn, sb) || sb[0] % pw || sb[1] % ph || sb[2] % pt) continue;
         const long long tiles = (long long)ceil_div(g.n, bn) * ceil_div(g.To, bt) * ceil_div(g.Ho, bh) * ceil_div(g.Wo, bw);
-        if (best_tiles < 0 || tiles < best_tiles || (tiles == best_tiles && bw > out->bw)) {
+        bool better = best_tiles < 0 || tiles < best_tiles;
+        if (!better && tiles == best_tiles) {
+          if (prefer_deep && ((bn == 1) != (out->bn == 1) || bt != out->bt)) better = (bn == 1) != (out->bn == 1) ? bn == 1 : bt > out->bt;
+          else better = bw > out->bw;
+        }
+        if (better) {
           best_tiles = tiles;
           *out = TileBox{bn, bt, bh, bw};
           for (int i = 0; i < 4; ++i) sb_out[i] = sb[i];
@@ -540,6 +559,7 @@ rt3d_status try_halo(rt3d_packed* w, DeviceBlob* blob, DeviceState* d, const rt3
   a.pool_t = a.pool_h = a.pool_w = 1;
   a.n_splits = 1; a.scratch = nullptr; a.counters = nullptr;
   a.tail_workers = 0; a.tail_scratch = nullptr; a.tail_flags = nullptr;
+  a.ts = 0; a.grp_ptr = nullptr; a.grp_first = nullptr; a.ts_a_bytes = 0; a.ts_frame_bytes = 0;
   a.wait_cycles = 0; a.debug_drop_last_load = 0;
   ConvGeom unit = g;                       // the staged block is a plain box of input voxels
   CUtensorMap xmap, ymap;
@@ -680,11 +700,12 @@ rt3d_status conv_impl(const rt3d_tensor* x, const rt3d_packed* wc, const float* 
   a.g = g;
   int sb[4] = {1, 1, 1, 1};
   bool rect;
+  const bool prefer_deep = g_ts_enabled.load() && g.st == 1 && (g.Kt == 2 || g.Kt == 3) && default_n_tile(w->M) <= 128;
   if (pooled) {
-    if (!choose_box_pool(g, pl_w, pl_h, pl_t, &a.box, sb)) return RT3D_ERR_UNSUPPORTED;
+    if (!choose_box_pool(g, pl_w, pl_h, pl_t, &a.box, sb, prefer_deep)) return RT3D_ERR_UNSUPPORTED;
     rect = true;
   } else {
-    a.box = choose_box(g);
+    a.box = choose_box(g, prefer_deep);
     rect = warp_block(a.box.bw, a.box.bh, a.box.bt, a.box.bn, sb);
   }
   a.pool_t = pl_t; a.pool_h = pl_h; a.pool_w = pl_w; a.sbw = sb[0]; a.sbh = sb[1];
@@ -709,7 +730,14 @@ rt3d_status conv_impl(const rt3d_tensor* x, const rt3d_packed* wc, const float* 
     use_pair = true;
   }
   if (pooled && plan.n_tile % 32) return RT3D_ERR_UNSUPPORTED;      // pooled rows leave as whole 32-channel pieces
-  const UmmaLayout* L = get_umma_layout(w, plan.n_tile);
+  // CTA pairs on bundles up to 128 wide with a kernel that is 2 or 3 deep: one deeper input tile per (kh, kw, chunk)
+  bool use_ts = false;
+  if (use_pair && g_ts_enabled.load()) {
+    UmmaArgs probe = a;
+    probe.n_tile = plan.n_tile; probe.n_bundles = ceil_div(w->M, plan.n_tile); probe.dense = dense_entry ? 1 : 0;
+    use_ts = umma_pair_ts_supported(probe, w->Ks * ceil_div(w->N, kChunk) * probe.n_bundles);
+  }
+  const UmmaLayout* L = get_umma_layout(w, plan.n_tile, use_ts);
   if (!L) return RT3D_ERR_UNSUPPORTED;
   DeviceBlob::Umma* u = nullptr;
   if ((s = get_umma_blob(w, blob, L, &u)) != RT3D_OK) return s;
@@ -721,6 +749,7 @@ rt3d_status conv_impl(const rt3d_tensor* x, const rt3d_packed* wc, const float* 
   a.residual = res_data; a.rcs = res_pitch;
   a.n_splits = plan.n_splits; a.scratch = nullptr; a.counters = nullptr;
   a.tail_workers = 0; a.tail_scratch = nullptr; a.tail_flags = nullptr;
+  a.ts = 0; a.grp_ptr = nullptr; a.grp_first = nullptr; a.ts_a_bytes = 0; a.ts_frame_bytes = 0;
   a.wait_cycles = debug_wait_cycles(); a.debug_drop_last_load = g_debug_drop_last_load.load();
   if (a.n_splits > 1) {
     // split-K workspace of this handle on this device: partial tiles + per-warp arrival counters
@@ -729,8 +758,13 @@ rt3d_status conv_impl(const rt3d_tensor* x, const rt3d_packed* wc, const float* 
                            size_t(tiles) * 4 * sizeof(int32_t))) != RT3D_OK) return s;
     a.scratch = blob->splitk; a.counters = blob->splitk_cnt;
   }
+  if (use_ts) {
+    a.ts = 1; a.grp_ptr = u->grp_ptr; a.grp_first = u->grp_first;
+    a.ts_frame_bytes = a.box.bh * a.box.bw * 128;
+    a.ts_a_bytes = (a.box.bt + g.Kt - 1) * a.ts_frame_bytes;
+  }
   CUtensorMap xmap;
-  if ((s = encode_xmap(x, g, a.box, &xmap)) != RT3D_OK) return s;
+  if ((s = encode_xmap(x, g, a.box, &xmap, use_ts ? g.Kt - 1 : 0)) != RT3D_OK) return s;
   CUtensorMap ymap;
   a.store_tma = (a.n_splits == 1 && rect && encode_ymap(y, sb, pl_w, pl_h, pl_t, &ymap)) ? 1 : 0;
   if (pooled && !a.store_tma) return RT3D_ERR_UNSUPPORTED;
@@ -739,14 +773,15 @@ rt3d_status conv_impl(const rt3d_tensor* x, const rt3d_packed* wc, const float* 
     // (its CTA pairs wait for one another, which needs the whole grid resident at once: not used when the caller
     // says that other kernels may run beside this call)
     size_t tail_bytes = 0, flag_bytes = 0;
-    if (!p->concurrent) umma_pair_tail_plan(&a, L->step_ptr.data(), d->sm_count, &tail_bytes, &flag_bytes);
+    if (!p->concurrent)
+      umma_pair_tail_plan(&a, L->step_ptr.data(), d->sm_count, &tail_bytes, &flag_bytes, use_ts ? L->grp_ptr.data() : nullptr);
     if (a.tail_workers > 0) {
       if ((s = ensure_splitk(w, blob, tail_bytes, flag_bytes)) != RT3D_OK) return s;
       a.tail_scratch = blob->splitk; a.tail_flags = blob->splitk_cnt;
     }
   }
   const void* ym = a.store_tma ? &ymap : nullptr;
-  t_last_plan = rt3d_plan_info{use_pair ? 2 : 1, a.n_tile, a.n_splits, a.tail_workers, pooled ? 1 : 0};
+  t_last_plan = rt3d_plan_info{use_pair ? (use_ts ? 7 : 2) : 1, a.n_tile, a.n_splits, a.tail_workers, pooled ? 1 : 0};
   if (t_plan_only) return RT3D_OK;
   cudaError_t e = use_pair ? launch_conv_umma_pair(a, &xmap, u->wmap_half, ym, d->sm_count, st)
                            : launch_conv_umma(a, &xmap, u->wmap, ym, d->sm_count, st);
@@ -1015,7 +1050,10 @@ void rt3d_packed_free(rt3d_packed* p) {
   for (DeviceBlob* b : p->blobs) {
     if (have_dev) cudaSetDevice(b->device);
     cudaFree(b->group_ptr); cudaFree(b->pos_idx); cudaFree(b->tiles);
-    for (auto& kv : b->umma) { cudaFree(kv.second.wtiles); cudaFree(kv.second.step_ptr); cudaFree(kv.second.steps); }
+    for (auto& kv : b->umma) {
+      cudaFree(kv.second.wtiles); cudaFree(kv.second.step_ptr); cudaFree(kv.second.steps);
+      cudaFree(kv.second.grp_ptr); cudaFree(kv.second.grp_first);
+    }
     cudaFree(b->stage_x); cudaFree(b->stage_y); cudaFree(b->stage_bias);
     for (void* hs : b->host_streams) if (hs) cudaStreamDestroy(static_cast<cudaStream_t>(hs));
     for (void* he : b->host_events) if (he) cudaEventDestroy(static_cast<cudaEvent_t>(he));
@@ -1208,6 +1246,7 @@ rt3d_status rt3d_conv3d_sparse_noalloc(const rt3d_tensor* x, const rt3d_packed* 
   int sb[4];
   a.pool_t = a.pool_h = a.pool_w = 1; a.sbw = a.sbh = 1;
   a.tail_workers = 0; a.tail_scratch = nullptr; a.tail_flags = nullptr;
+  a.ts = 0; a.grp_ptr = nullptr; a.grp_first = nullptr; a.ts_a_bytes = 0; a.ts_frame_bytes = 0;
   a.wait_cycles = 0; a.debug_drop_last_load = 0;
   a.store_tma = (a.n_splits == 1 && warp_block(a.box.bw, a.box.bh, a.box.bt, a.box.bn, sb) &&
                  encode_ymap(y, sb, 1, 1, 1, &ymap)) ? 1 : 0;
@@ -1227,6 +1266,7 @@ void rt3d_plan_end(void) { t_plan_only = false; }
 rt3d_status rt3d_debug_set(int what, long long value) {
   if (what == RT3D_DEBUG_WAIT_CYCLES) { if (value < 0) return RT3D_ERR_INVALID_ARG; g_debug_wait_cycles.store(value); return RT3D_OK; }
   if (what == RT3D_DEBUG_DROP_LAST_LOAD) { g_debug_drop_last_load.store(value != 0); return RT3D_OK; }
+  if (what == RT3D_DEBUG_T_GROUPS) { g_ts_enabled.store(value != 0); return RT3D_OK; }
   return RT3D_ERR_INVALID_ARG;
 }
 

@@ -58,6 +58,13 @@ struct UmmaArgs {
   int tail_workers;                         // CTA-pair kernel: pairs sharing the left-over items of the last round (0 = off)
   float* tail_scratch;                      // device, [tail_workers][2 shares][2 CTAs][n_tile][128] fp32 partial tiles
   int32_t* tail_flags;                      // device, [tail_workers][2][2][4 warps] "partial written" flags, zero between launches
+  // CTA-pair kernel, t-grouped layout (ts != 0): steps that differ only in kt share one staged input tile that is
+  // Kt - 1 frames deeper (the xmap's box); needs temporal stride 1, one clip per box and bundles up to 128 wide.
+  int ts;
+  const int32_t* grp_ptr;                   // device, [n_bundles + 1]
+  const int32_t* grp_first;                 // device, first step of each group + sentinel
+  int ts_a_bytes;                           // bytes of the deeper input tile
+  int ts_frame_bytes;                       // bytes of one frame of it (bh * bw rows of 128 bytes)
   long long wait_cycles;                    // single-CTA kernel: SM clocks after which a wait gives up (0 = the default, about 1 s)
   int debug_drop_last_load;                 // single-CTA kernel, tests only: never issue the loads of each CTA's last stage
 };
@@ -73,8 +80,11 @@ cudaError_t launch_conv_umma(const UmmaArgs& a, const void* xmap, const void* wm
 bool umma_pair_supported(int n_tile, int n_bundles);
 // Fills a->tail_workers (0 = whole items only) and the scratch the tail split needs; the caller provides
 // a->tail_scratch / a->tail_flags of at least those sizes (flags zero-initialised).
+// With a->ts the unit of the split is a group: `grp_ptr_host` = the layout's per-bundle group offsets.
 void umma_pair_tail_plan(UmmaArgs* a, const int32_t* step_ptr_host, int sm_count, size_t* scratch_bytes,
-                         size_t* flag_bytes);
+                         size_t* flag_bytes, const int32_t* grp_ptr_host = nullptr);
+// Whether the t-grouped variant can run this shape (and is expected to pay).
+bool umma_pair_ts_supported(const UmmaArgs& a, int total_steps);
 cudaError_t launch_conv_umma_pair(const UmmaArgs& a, const void* xmap, const void* wmap_half, const void* ymap,
                                   int sm_count, cudaStream_t stream);
 

@@ -44,16 +44,21 @@ static float tile_value(const rt3d_packed* p, int64_t e, int i, int j) {
 // steps in which at least one kernel group of the bundle keeps that location, and build the
 // matching [n_tile][64] weight tiles (zeros where a group prunes the location).  Steps are
 // ordered by location, then chunk.
-const UmmaLayout* get_umma_layout(rt3d_packed* p, int n_tile) {
+// `t_groups`: the order is (kh, kw), chunk, kt instead, and the steps that differ only in kt form a
+// group (grp_ptr / grp_first): the CTA-pair kernel stages one input tile, Kt - 1 frames deeper, per group.
+const UmmaLayout* get_umma_layout(rt3d_packed* p, int n_tile, bool t_groups) {
   if (!umma_layout_possible(p)) return nullptr;
   if (n_tile <= 0) n_tile = default_n_tile(p->M);
   if (n_tile % 16 || n_tile > 256) return nullptr;
   std::lock_guard<std::mutex> lock(p->mu);
-  auto it = p->umma_layouts.find(n_tile);
+  const int key = n_tile + (t_groups ? 4096 : 0);
+  auto it = p->umma_layouts.find(key);
   if (it != p->umma_layouts.end()) return &it->second;
 
   UmmaLayout L;
   L.n_tile = n_tile;
+  L.t_groups = t_groups;
+  if (t_groups) L.grp_ptr.assign(1, 0);
   L.n_bundles = ceil_div(p->M, n_tile);
   L.n_chunks = ceil_div(p->N, kChunk);
   L.step_ptr.assign(L.n_bundles + 1, 0);
@@ -73,13 +78,28 @@ const UmmaLayout* get_umma_layout(rt3d_packed* p, int n_tile) {
       }
     const int32_t base = L.step_ptr[b];
     int32_t cnt = 0;
-    for (int kpos = 0; kpos < Ks; ++kpos)
-      for (int ch = 0; ch < L.n_chunks; ++ch)
-        if (slot[size_t(kpos) * L.n_chunks + ch] == 0) {
-          slot[size_t(kpos) * L.n_chunks + ch] = base + cnt++;
-          const int kw = kpos % p->Kw, kh = (kpos / p->Kw) % p->Kh, kt = kpos / (p->Kw * p->Kh);
-          L.steps.push_back(encode_step(kt, kh, kw, ch));
+    if (!t_groups) {
+      for (int kpos = 0; kpos < Ks; ++kpos)
+        for (int ch = 0; ch < L.n_chunks; ++ch)
+          if (slot[size_t(kpos) * L.n_chunks + ch] == 0) {
+            slot[size_t(kpos) * L.n_chunks + ch] = base + cnt++;
+            const int kw = kpos % p->Kw, kh = (kpos / p->Kw) % p->Kh, kt = kpos / (p->Kw * p->Kh);
+            L.steps.push_back(encode_step(kt, kh, kw, ch));
+          }
+    } else {
+      for (int hw = 0; hw < p->Kh * p->Kw; ++hw)
+        for (int ch = 0; ch < L.n_chunks; ++ch) {
+          bool open = false;
+          for (int kt = 0; kt < p->Kt; ++kt) {
+            const int kpos = kt * p->Kh * p->Kw + hw;
+            if (slot[size_t(kpos) * L.n_chunks + ch] != 0) continue;
+            if (!open) { L.grp_first.push_back(base + cnt); open = true; }
+            slot[size_t(kpos) * L.n_chunks + ch] = base + cnt++;
+            L.steps.push_back(encode_step(kt, hw / p->Kw, hw % p->Kw, ch));
+          }
         }
+      L.grp_ptr.push_back(int32_t(L.grp_first.size()));
+    }
     L.step_ptr[b + 1] = base + cnt;
     L.max_steps = std::max(L.max_steps, int(cnt));
     L.wtiles.resize(size_t(base + cnt) * n_tile * kChunk, 0);
@@ -99,7 +119,8 @@ const UmmaLayout* get_umma_layout(rt3d_packed* p, int n_tile) {
             }
           }
   }
-  auto res = p->umma_layouts.emplace(n_tile, std::move(L));
+  if (t_groups) L.grp_first.push_back(int32_t(L.steps.size()));     // sentinel: end of the last group
+  auto res = p->umma_layouts.emplace(key, std::move(L));
   return &res.first->second;
 }
 
@@ -356,10 +377,43 @@ rt3d_status rt3d_unpack_to_dense(const rt3d_packed* p, float* w_out) {
   return RT3D_OK;
 }
 
+namespace {
+rt3d_status unpack_device_layout(const rt3d_packed* p, int n_tile, bool t_groups, float* w_out);
+}
 rt3d_status rt3d_unpack_device_layout(const rt3d_packed* p, int n_tile, float* w_out) {
+  return unpack_device_layout(p, n_tile, false, w_out);
+}
+rt3d_status rt3d_unpack_device_layout_tgroups(const rt3d_packed* p, int n_tile, float* w_out) {
+  return unpack_device_layout(p, n_tile, true, w_out);
+}
+namespace {
+rt3d_status unpack_device_layout(const rt3d_packed* p, int n_tile, bool t_groups, float* w_out) {
   if (!p || !w_out) return RT3D_ERR_INVALID_ARG;
-  const UmmaLayout* L = get_umma_layout(const_cast<rt3d_packed*>(p), n_tile);
+  const UmmaLayout* L = get_umma_layout(const_cast<rt3d_packed*>(p), n_tile, t_groups);
   if (!L) return RT3D_ERR_UNSUPPORTED;
+  if (t_groups) {
+    // groups tile each bundle's list exactly; inside a group only kt changes, upwards
+    if (int(L->grp_ptr.size()) != L->n_bundles + 1 || L->grp_first.size() != size_t(L->grp_ptr.back()) + 1 ||
+        L->grp_first.back() != int32_t(L->steps.size()))
+      return RT3D_ERR_INVALID_ARG;
+    for (int b = 0; b < L->n_bundles; ++b) {
+      if (L->grp_ptr[b] > L->grp_ptr[b + 1]) return RT3D_ERR_INVALID_ARG;
+      const int32_t first = L->grp_ptr[b] < L->grp_ptr[b + 1] ? L->grp_first[L->grp_ptr[b]] : L->step_ptr[b];
+      if (first != L->step_ptr[b]) return RT3D_ERR_INVALID_ARG;
+      for (int32_t g = L->grp_ptr[b]; g < L->grp_ptr[b + 1]; ++g) {
+        const int32_t s0 = L->grp_first[g], s1 = L->grp_first[g + 1];
+        if (s1 <= s0 || s1 - s0 > p->Kt || s1 > L->step_ptr[b + 1]) return RT3D_ERR_INVALID_ARG;
+        int kt0, kh0, kw0, ch0;
+        decode_step(L->steps[s0], kt0, kh0, kw0, ch0);
+        for (int32_t s = s0 + 1; s < s1; ++s) {
+          int kt, kh, kw, ch;
+          decode_step(L->steps[s], kt, kh, kw, ch);
+          if (kh != kh0 || kw != kw0 || ch != ch0 || kt <= kt0) return RT3D_ERR_INVALID_ARG;
+          kt0 = kt;
+        }
+      }
+    }
+  }
   std::memset(w_out, 0, sizeof(float) * size_t(p->M) * p->N * p->Ks);
   for (int b = 0; b < L->n_bundles; ++b)
     for (int32_t s = L->step_ptr[b]; s < L->step_ptr[b + 1]; ++s) {
@@ -373,6 +427,7 @@ rt3d_status rt3d_unpack_device_layout(const rt3d_packed* p, int n_tile, float* w
     }
   return RT3D_OK;
 }
+}  // namespace
 
 rt3d_status rt3d_unpack_sub_layout(const rt3d_packed* p, int n_tile, float* w_out) {
   if (!p || !w_out) return RT3D_ERR_INVALID_ARG;

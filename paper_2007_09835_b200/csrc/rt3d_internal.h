@@ -43,6 +43,9 @@ struct UmmaLayout {
   std::vector<int32_t> steps;        // encoded (kt,kh,kw,chunk), only non-empty steps of each bundle
   std::vector<uint16_t> wtiles;      // [steps.size()][n_tile][64] bf16 bits, zero where pruned / absent
   int max_steps = 0;                 // longest bundle list
+  bool t_groups = false;             // steps ordered (kh, kw), chunk, kt; groups = runs that differ only in kt
+  std::vector<int32_t> grp_ptr;      // [n_bundles + 1] offsets into grp_first            (t_groups only)
+  std::vector<int32_t> grp_first;    // first step of each group, + one sentinel           (t_groups only)
 };
 
 // Layout for the small-C_in tensor-core kernel (C_in <= 8, channel pitch 8) at spatial strides
@@ -88,9 +91,11 @@ struct DeviceBlob {
     int32_t* steps = nullptr;
     alignas(64) unsigned char wmap[128];   // CUtensorMap of wtiles, box = one [n_tile][64] tile
     alignas(64) unsigned char wmap_half[128];   // same tensor, box = half a tile (CTA-pair kernel)
+    int32_t* grp_ptr = nullptr;                 // t-grouped layouts only
+    int32_t* grp_first = nullptr;
     bool ready = false;
   };
-  std::map<int, Umma> umma;          // keyed by n_tile
+  std::map<int, Umma> umma;          // keyed like the handle's layouts
   struct Sub { void* steps = nullptr; int32_t* step_ptr = nullptr; void* blocks = nullptr; bool ready = false; };
   std::map<int, Sub> sub;            // sub-tile kernel, keyed by n_tile
   struct SmallC { void* wimg = nullptr; int32_t* pairs = nullptr; };
@@ -116,7 +121,7 @@ struct rt3d_packed {
   std::vector<uint16_t> pos_idx;
   std::vector<unsigned char> tiles;  // nnz * g_m * g_n elements of float or bf16 bits
   std::mutex mu;                     // guards the lazily built members below
-  std::map<int, rt3d::UmmaLayout> umma_layouts;   // keyed by n_tile
+  std::map<int, rt3d::UmmaLayout> umma_layouts;   // keyed by n_tile (+ 4096: the t-grouped order)
   std::map<int, rt3d::SubLayout> sub_layouts;     // keyed by n_tile
   std::map<int, rt3d::SmallCLayout> smallc_layouts;   // keyed by sh*16+sw, built on first use
   std::vector<rt3d::DeviceBlob*> blobs;
@@ -127,7 +132,7 @@ namespace rt3d {
 // Default bundle width for M output channels: as few bundles as possible with n_tile <= 256.
 int default_n_tile(int M);
 // Builds (or returns the cached) tensor-core layout; nullptr if the handle cannot use it.
-const UmmaLayout* get_umma_layout(rt3d_packed* p, int n_tile);
+const UmmaLayout* get_umma_layout(rt3d_packed* p, int n_tile, bool t_groups = false);
 bool umma_layout_possible(const rt3d_packed* p);
 // Builds (or returns the cached) layout of the sub-tile kernel; nullptr if the handle cannot use it.
 const SubLayout* get_sub_layout(rt3d_packed* p, int n_tile);

@@ -54,8 +54,15 @@ __device__ __forceinline__ Work get_work(const TailWork* tw, int wi, int cluster
 // tile, as long as 30 K steps.  Shares and fix-ups of split tiles are divided between the sets the same way.
 constexpr int kThreadsPair = 352;
 
+// t-grouped variant: step and group tables (all bundles together) live in shared memory, up to this many entries each.
+constexpr int kTsTable = 1024;
+
 // kCps: K steps per pipeline stage (and per barrier hand-shake): 1, or 2 for narrow bundles.
-template <bool kDense, int kCps>
+// kTS: t-grouped layout.  A pipeline stage then holds ONE input tile that is Kt - 1 frames deeper and the weight
+// tiles of the up to Kt steps (kt = 0 .. Kt-1 at one (kh, kw, chunk)) that read it, each through a descriptor that
+// starts kt frames into the tile: a third as many input bytes per step cross from L2, so more steps are in flight
+// in the same shared memory (a 64 -> 128 channel 3x3x3 layer was bound by that, at 387 clocks per step against 256).
+template <bool kDense, int kCps, bool kTS>
 __global__ void __launch_bounds__(kThreadsPair, 1)
 conv3d_umma_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CUtensorMap wmap_half,
                         const __grid_constant__ CUtensorMap ymap, const UmmaArgs a, const int stages, const int tmem_cols) {
@@ -65,12 +72,16 @@ conv3d_umma_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_c
   const int n_half = a.n_tile / 2;
   const uint32_t b_bytes = uint32_t(n_half) * 128u;             // this CTA's half of the B tile
   const uint32_t chunk_bytes = kABytes + b_bytes;
-  const uint32_t stage_bytes = kCps * chunk_bytes;
+  const uint32_t ts_a_slot = (uint32_t(a.ts_a_bytes) + 1023u) & ~1023u;
+  const uint32_t stage_bytes = kTS ? ts_a_slot + uint32_t(a.g.Kt) * b_bytes : kCps * chunk_bytes;
   const uint32_t store_smem = tiles_base + uint32_t(stages) * stage_bytes;     // 4 warps x 2 staging buffers
   Barriers* bars = reinterpret_cast<Barriers*>(smem_raw + (tiles_base - raw) + size_t(stages) * stage_bytes +
                                                4 * kStoreWarpBytes);
   TailWork* tw = reinterpret_cast<TailWork*>(bars + 1);
   float* bias_s = align16_f32(tw + 1);
+  int32_t* steps_s = reinterpret_cast<int32_t*>(bias_s + a.n_bundles * a.n_tile);   // kTS only: steps, then group starts
+  int32_t* grp_s = steps_s + kTsTable;
+  const int ts_groups_dense = a.g.Kh * a.g.Kw * a.n_chunks;
   int32_t* err = a.sched + 2;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -133,8 +144,12 @@ conv3d_umma_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_c
     const int t = threadIdx.x;
     if (t < n_tail) {
       const int b = (first_tail + t) / pairs_per_bundle;
-      const int ns = kDense ? a.steps_dense : __ldg(a.step_ptr + b + 1) - __ldg(a.step_ptr + b);
-      tw->g[t] = (ns + kCps - 1) / kCps;
+      if (kTS) {
+        tw->g[t] = kDense ? ts_groups_dense : __ldg(a.grp_ptr + b + 1) - __ldg(a.grp_ptr + b);
+      } else {
+        const int ns = kDense ? a.steps_dense : __ldg(a.step_ptr + b + 1) - __ldg(a.step_ptr + b);
+        tw->g[t] = (ns + kCps - 1) / kCps;
+      }
     }
     __syncthreads();
     bool mine = false;
@@ -165,6 +180,11 @@ conv3d_umma_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_c
       atomicAdd(&tw->n_seg, 1);
     }
   }
+  if (kTS && !kDense) {                    // the layout's tables (host uploads only, as above)
+    const int total_steps = __ldg(a.step_ptr + a.n_bundles), total_groups = __ldg(a.grp_ptr + a.n_bundles);
+    for (int i = threadIdx.x; i < total_steps; i += blockDim.x) steps_s[i] = __ldg(a.steps + i);
+    for (int i = threadIdx.x; i <= total_groups; i += blockDim.x) grp_s[i] = __ldg(a.grp_first + i);
+  }
   pdl_wait();
   for (int i = threadIdx.x; i < a.n_bundles * a.n_tile; i += blockDim.x)
     bias_s[i] = (a.bias != nullptr && i < a.g.M) ? __ldg(a.bias + i) : 0.f;
@@ -178,7 +198,38 @@ conv3d_umma_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_c
       bool ok = true;
       const uint32_t tx_chunk_both = 2u * (uint32_t(box_rows) * 128u + b_bytes);
       const int n_work = tw->n_full + tw->n_seg;
-      for (int wi = 0; wi < n_work && ok; ++wi) {
+      for (int wi = 0; kTS && wi < n_work && ok; ++wi) {
+        const Work wk = get_work(tw, wi, cluster_id, n_clusters);
+        const PairItem c = decode_pair_item(a, wk.item, pairs_per_bundle, n_mtiles, rank);
+        const int gbase = kDense ? 0 : a.grp_ptr[c.bundle];
+        const int ngrp = kDense ? ts_groups_dense : a.grp_ptr[c.bundle + 1] - gbase;
+        const int g1 = wk.g1 < ngrp ? wk.g1 : ngrp;
+        const int wq = c.w0 * a.g.sw - a.g.pw, hq = c.h0 * a.g.sh - a.g.ph, tq = c.t0 - a.g.pt;
+        for (int g = wk.g0; g < g1; ++g) {
+          int s0, ns, kh, kw, ch;
+          if (kDense) {
+            s0 = c.bundle * a.steps_dense + g * a.g.Kt; ns = a.g.Kt;
+            ch = g % a.n_chunks;
+            const int hw = g / a.n_chunks;
+            kw = hw % a.g.Kw; kh = hw / a.g.Kw;
+          } else {
+            s0 = grp_s[gbase + g]; ns = grp_s[gbase + g + 1] - s0;
+            const int enc = steps_s[s0];
+            kh = (enc >> 18) & 63; kw = (enc >> 12) & 63; ch = enc & 4095;
+          }
+          const uint32_t full_local = smem_u32(&bars->full[stage]);
+          const uint32_t full_leader = mapa_shared(full_local, 0);
+          const uint32_t s_dst = tiles_base + stage * stage_bytes;
+          if (!mbar_wait(smem_u32(&bars->empty[stage]), phase ^ 1u, bars, err, 21)) { ok = false; break; }
+          if (leader) mbar_expect_tx(full_local, 2u * (uint32_t(a.ts_a_bytes) + uint32_t(ns) * b_bytes));
+          tma_load_5d_pair(s_dst, &xmap, full_leader, ch * 64, wq + kw, hq + kh, tq, c.n0);
+          const int wrow = s0 * a.n_tile + int(rank) * n_half;
+          for (int q = 0; q < ns; ++q)
+            tma_load_2d_pair(s_dst + ts_a_slot + uint32_t(q) * b_bytes, &wmap_half, full_leader, 0, wrow + q * a.n_tile);
+          if (++stage == stages) { stage = 0; phase ^= 1u; }
+        }
+      }
+      for (int wi = 0; !kTS && wi < n_work && ok; ++wi) {
         const Work wk = get_work(tw, wi, cluster_id, n_clusters);
         const PairItem c = decode_pair_item(a, wk.item, pairs_per_bundle, n_mtiles, rank);
         const int s_begin = kDense ? c.bundle * a.steps_dense : a.step_ptr[c.bundle];
@@ -233,7 +284,40 @@ conv3d_umma_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_c
       int stage = 0;
       bool ok = true, ready = false;
       const int n_work = tw->n_full + tw->n_seg;
-      for (int wi = 0; wi < n_work && ok; ++wi, ++j) {
+      for (int wi = 0; kTS && wi < n_work && ok; ++wi, ++j) {
+        const Work wk = get_work(tw, wi, cluster_id, n_clusters);
+        const int bundle = wk.item / pairs_per_bundle;
+        const int gbase = kDense ? 0 : a.grp_ptr[bundle];
+        const int ngrp = kDense ? ts_groups_dense : a.grp_ptr[bundle + 1] - gbase;
+        const int g1 = wk.g1 < ngrp ? wk.g1 : ngrp;
+        const uint32_t buf = j & 1u;
+        if (!mbar_wait(smem_u32(&bars->tmem_empty[buf]), ((j >> 1) & 1u) ^ 1u, bars, err, 22)) break;
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (buf * uint32_t(kIss) + uint32_t(me)) * uint32_t(a.n_tile);
+        int gl = 0;                                          // group inside this item (or share)
+        for (int g = wk.g0; g < g1; ++g, ++gl) {
+          if (!kDual || (gl & 1) == me) {
+            int s0 = 0, ns = a.g.Kt;
+            if (!kDense) { s0 = grp_s[gbase + g]; ns = grp_s[gbase + g + 1] - s0; }
+            if (!mbar_wait(smem_u32(&bars->full[stage]), phase, bars, err, 23)) { ok = false; break; }
+            tc_fence_after();
+            const uint32_t s_base = tiles_base + stage * stage_bytes;
+            for (int q = 0; q < ns; ++q) {
+              const int kt = kDense ? q : (steps_s[s0 + q] >> 24) & 63;
+              const uint64_t adesc = smem_desc_sw128(s_base + uint32_t(kt) * uint32_t(a.ts_frame_bytes));
+              const uint64_t bdesc = smem_desc_sw128(s_base + ts_a_slot + uint32_t(q) * b_bytes);
+#pragma unroll
+              for (int kk = 0; kk < 4; ++kk)
+                umma_bf16_pair(d_tmem, adesc + 2 * kk, bdesc + 2 * kk, idesc, ((gl >= kIss) | q | kk) ? 1u : 0u);
+            }
+            umma_commit_pair(smem_u32(&bars->empty[stage]));
+          }
+          if (++stage == stages) { stage = 0; phase ^= 1u; }
+        }
+        if (!ok) break;
+        umma_commit_pair(smem_u32(&bars->tmem_full[buf]));
+      }
+      for (int wi = 0; !kTS && wi < n_work && ok; ++wi, ++j) {
         const Work wk = get_work(tw, wi, cluster_id, n_clusters);
         const int bundle = wk.item / pairs_per_bundle;
         const int nsteps = kDense ? a.steps_dense : a.step_ptr[bundle + 1] - a.step_ptr[bundle];
@@ -309,8 +393,14 @@ conv3d_umma_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_c
       const int m_base = c.bundle * a.n_tile;
       const uint32_t taddr = tmem_base + (uint32_t(quad * 32) << 16) + buf * uint32_t(kIss * a.n_tile);
       // the second issuer's accumulator holds something once the item (or share) has two step groups
-      const int steps_here = (wk.g1 * kCps < nsteps ? wk.g1 * kCps : nsteps) - wk.g0 * kCps;
-      const uint32_t acc2 = (kDual && steps_here > kCps) ? uint32_t(a.n_tile) : 0u;
+      int units_here;                                      // step groups (of kCps steps, or t-groups) of this item or share
+      if (kTS) {
+        const int ngrp = kDense ? ts_groups_dense : a.grp_ptr[c.bundle + 1] - a.grp_ptr[c.bundle];
+        units_here = (wk.g1 < ngrp ? wk.g1 : ngrp) - wk.g0;
+      } else {
+        units_here = ((wk.g1 * kCps < nsteps ? wk.g1 * kCps : nsteps) - wk.g0 * kCps + kCps - 1) / kCps;
+      }
+      const uint32_t acc2 = (kDual && units_here >= 2) ? uint32_t(a.n_tile) : 0u;
       const __nv_bfloat16* res = (rb != nullptr && in_range) ? rb + vox * a.rcs + m_base : nullptr;
       const int res_left = a.rcs - m_base;
       if (wk.nparts > 1 && wk.part != 0) {
@@ -414,13 +504,26 @@ size_t pair_smem_bytes(int n_tile, int n_bundles) {
          size_t(n_tile) * n_bundles * 4;
 }
 
-template <bool kDense, int kCps>
+// t-grouped variant: a stage = one deeper input tile + Kt weight half-tiles; the tables come after the bias.
+size_t ts_stage_bytes(const UmmaArgs& a) {
+  return ((size_t(a.ts_a_bytes) + 1023) & ~size_t(1023)) + size_t(a.g.Kt) * size_t(a.n_tile / 2) * 128;
+}
+int pick_stages_pair_ts(const UmmaArgs& a) {
+  const int s = int(kSmemBudget / ts_stage_bytes(a));
+  return s > kMaxStages ? kMaxStages : s;
+}
+size_t pair_smem_bytes_ts(const UmmaArgs& a) {
+  return size_t(pick_stages_pair_ts(a)) * ts_stage_bytes(a) + 1024 + 4 * kStoreWarpBytes + sizeof(Barriers) + sizeof(TailWork) +
+         16 + size_t(a.n_tile) * a.n_bundles * 4 + (2 * size_t(kTsTable) + 8) * 4;
+}
+
+template <bool kDense, int kCps, bool kTS>
 cudaError_t prepare_pair_t() {
   static bool attr_done[kMaxDevices] = {};             // the attribute is per device
   const int dev = current_device_index();
   if (dev < 0) return cudaErrorInvalidDevice;
   if (!attr_done[dev]) {
-    cudaError_t e = cudaFuncSetAttribute(conv3d_umma_pair_kernel<kDense, kCps>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    cudaError_t e = cudaFuncSetAttribute(conv3d_umma_pair_kernel<kDense, kCps, kTS>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
     if (e != cudaSuccess) return e;
     attr_done[dev] = true;
   }
@@ -440,19 +543,19 @@ void pair_launch_config(cudaLaunchConfig_t& cfg, cudaLaunchAttribute* attr, unsi
 }
 
 // CTA pairs that can be resident at once (the persistent grid), never more than SMs / 2.
-template <bool kDense, int kCps>
+template <bool kDense, int kCps, bool kTS>
 int pair_max_clusters_t(int sm_count, size_t smem) {
   static int max_clusters_dev[kMaxDevices] = {};       // the occupancy answer is per device
   const int dev = current_device_index();
   if (dev < 0) return sm_count / 2;
   int& max_clusters = max_clusters_dev[dev];
   if (max_clusters == 0) {
-    if (prepare_pair_t<kDense, kCps>() != cudaSuccess) return sm_count / 2;
+    if (prepare_pair_t<kDense, kCps, kTS>() != cudaSuccess) return sm_count / 2;
     cudaLaunchConfig_t cfg;
     cudaLaunchAttribute attr[1];
     pair_launch_config(cfg, attr, unsigned(sm_count & ~1), smem, nullptr);
     int n = 0;
-    if (cudaOccupancyMaxActiveClusters(&n, conv3d_umma_pair_kernel<kDense, kCps>, &cfg) != cudaSuccess || n <= 0) n = sm_count / 2;
+    if (cudaOccupancyMaxActiveClusters(&n, conv3d_umma_pair_kernel<kDense, kCps, kTS>, &cfg) != cudaSuccess || n <= 0) n = sm_count / 2;
     max_clusters = n;
   }
   return max_clusters < sm_count / 2 ? max_clusters : sm_count / 2;
@@ -461,21 +564,25 @@ int pair_max_clusters_t(int sm_count, size_t smem) {
 int pair_max_clusters(int n_tile, int n_bundles, bool dense, int sm_count) {
   const size_t smem = pair_smem_bytes(n_tile, n_bundles);
   if (pick_cps(n_tile) == 2)
-    return dense ? pair_max_clusters_t<true, 2>(sm_count, smem) : pair_max_clusters_t<false, 2>(sm_count, smem);
-  return dense ? pair_max_clusters_t<true, 1>(sm_count, smem) : pair_max_clusters_t<false, 1>(sm_count, smem);
+    return dense ? pair_max_clusters_t<true, 2, false>(sm_count, smem) : pair_max_clusters_t<false, 2, false>(sm_count, smem);
+  return dense ? pair_max_clusters_t<true, 1, false>(sm_count, smem) : pair_max_clusters_t<false, 1, false>(sm_count, smem);
+}
+int pair_max_clusters_ts(const UmmaArgs& a, int sm_count) {
+  const size_t smem = pair_smem_bytes_ts(a);
+  return a.dense ? pair_max_clusters_t<true, 2, true>(sm_count, smem) : pair_max_clusters_t<false, 2, true>(sm_count, smem);
 }
 
-template <bool kDense, int kCps>
+template <bool kDense, int kCps, bool kTS>
 cudaError_t launch_pair_t(const UmmaArgs& a, const CUtensorMap& xm, const CUtensorMap& wm, const CUtensorMap& ym,
                           int sm_count, int stages,
                           int cols, size_t smem, long long n_items, cudaStream_t stream) {
-  cudaError_t e = prepare_pair_t<kDense, kCps>();
+  cudaError_t e = prepare_pair_t<kDense, kCps, kTS>();
   if (e != cudaSuccess) return e;
-  long long clusters = pair_max_clusters_t<kDense, kCps>(sm_count, smem);
+  long long clusters = pair_max_clusters_t<kDense, kCps, kTS>(sm_count, smem);
   const long long want = n_items > a.tail_workers ? n_items : a.tail_workers;
   if (clusters > want) clusters = want;
   LaunchSetup ls(dim3(unsigned(2 * clusters)), dim3(kThreadsPair), smem, stream, 2);
-  return cudaLaunchKernelEx(&ls.cfg, conv3d_umma_pair_kernel<kDense, kCps>, xm, wm, ym, a, stages, cols);
+  return cudaLaunchKernelEx(&ls.cfg, conv3d_umma_pair_kernel<kDense, kCps, kTS>, xm, wm, ym, a, stages, cols);
 }
 
 }  // namespace
@@ -486,27 +593,39 @@ bool umma_pair_supported(int n_tile, int n_bundles) {
 
 // Tail split: decides how many CTA pairs share the items that do not fill a last round (0 = no split)
 // and how much scratch that needs.  `step_ptr_host`: the layout's per-bundle step offsets (sparse path).
+bool umma_pair_ts_supported(const UmmaArgs& a, int total_steps) {
+  if (a.n_tile > 128 || a.n_tile % 16 || a.g.st != 1 || a.box.bn != 1 || a.box.bt < 2) return false;
+  if (a.g.Kt < 2 || a.g.Kt > 3) return false;
+  if (a.box.bt + a.g.Kt - 1 > 256) return false;
+  if (!a.dense && total_steps > kTsTable) return false;
+  UmmaArgs t = a;
+  t.ts_a_bytes = (a.box.bt + a.g.Kt - 1) * a.box.bh * a.box.bw * 128;
+  return pick_stages_pair_ts(t) >= 3 && pair_smem_bytes_ts(t) <= 227 * 1024;
+}
+
 void umma_pair_tail_plan(UmmaArgs* a, const int32_t* step_ptr_host, int sm_count, size_t* scratch_bytes,
-                         size_t* flag_bytes) {
+                         size_t* flag_bytes, const int32_t* grp_ptr_host) {
   a->tail_workers = 0;
   *scratch_bytes = 0; *flag_bytes = 0;
   if (!umma_pair_supported(a->n_tile, a->n_bundles)) return;
   const long long n_mtiles = (long long)a->tiles_n * a->tiles_t * a->tiles_h * a->tiles_w;
   const long long pairs_per_bundle = (n_mtiles + 1) / 2;
   const long long n_items = pairs_per_bundle * a->n_bundles;
-  const int clusters = pair_max_clusters(a->n_tile, a->n_bundles, a->dense != 0, sm_count);
+  const int clusters = a->ts ? pair_max_clusters_ts(*a, sm_count)
+                             : pair_max_clusters(a->n_tile, a->n_bundles, a->dense != 0, sm_count);
   if (clusters <= 0) return;
   // fewer items than pairs: every item is a left-over item, the grid is `tail_workers` pairs
   const long long rounds = n_items / clusters;
   const int n_tail = int(n_items - rounds * clusters);
   if (n_tail == 0 || n_tail > kMaxTail) return;
-  const int cps = pick_cps(a->n_tile);
+  const int cps = a->ts ? a->g.Kt : pick_cps(a->n_tile);   // steps per unit of the split, about
   long long total = 0, g_min = 1 << 30, g_max = 0;
   for (int t = 0; t < n_tail; ++t) {
     const int b = int((rounds * clusters + t) / pairs_per_bundle);
     const int ns = a->dense ? a->steps_dense : step_ptr_host[b + 1] - step_ptr_host[b];
     if (ns < 8) return;                                   // nothing worth cutting
-    const long long g = (ns + cps - 1) / cps;
+    long long g = (ns + cps - 1) / cps;
+    if (a->ts) g = a->dense ? (long long)a->g.Kh * a->g.Kw * a->n_chunks : grp_ptr_host[b + 1] - grp_ptr_host[b];
     total += g;
     g_min = g < g_min ? g : g_min; g_max = g > g_max ? g : g_max;
   }
@@ -532,8 +651,9 @@ cudaError_t launch_conv_umma_pair(const UmmaArgs& a, const void* xmap, const voi
                                   int sm_count, cudaStream_t stream) {
   if (!umma_pair_supported(a.n_tile, a.n_bundles) || a.n_splits != 1) return cudaErrorInvalidValue;
   if (a.tail_workers > 0 && (a.tail_scratch == nullptr || a.tail_flags == nullptr)) return cudaErrorInvalidValue;
-  const int stages = pick_stages_pair(a.n_tile);
-  const size_t smem = pair_smem_bytes(a.n_tile, a.n_bundles);
+  const int stages = a.ts ? pick_stages_pair_ts(a) : pick_stages_pair(a.n_tile);
+  const size_t smem = a.ts ? pair_smem_bytes_ts(a) : pair_smem_bytes(a.n_tile, a.n_bundles);
+  if (a.ts && (a.n_tile > 128 || smem > 227 * 1024 || stages < 2)) return cudaErrorInvalidValue;
   int cols = 32;
   while (cols < 2 * a.n_tile * (pick_cps(a.n_tile) == 2 ? 2 : 1)) cols *= 2;     // two issuing threads: two accumulators
   if (cols > 512) return cudaErrorInvalidValue;
@@ -545,11 +665,14 @@ cudaError_t launch_conv_umma_pair(const UmmaArgs& a, const void* xmap, const voi
   memcpy(&xm, xmap, sizeof(CUtensorMap));
   memcpy(&wm, wmap_half, sizeof(CUtensorMap));
   memcpy(&ym, ymap ? ymap : xmap, sizeof(CUtensorMap));
+  if (a.ts)
+    return a.dense ? launch_pair_t<true, 2, true>(a, xm, wm, ym, sm_count, stages, cols, smem, n_items, stream)
+                   : launch_pair_t<false, 2, true>(a, xm, wm, ym, sm_count, stages, cols, smem, n_items, stream);
   if (pick_cps(a.n_tile) == 2)
-    return a.dense ? launch_pair_t<true, 2>(a, xm, wm, ym, sm_count, stages, cols, smem, n_items, stream)
-                   : launch_pair_t<false, 2>(a, xm, wm, ym, sm_count, stages, cols, smem, n_items, stream);
-  return a.dense ? launch_pair_t<true, 1>(a, xm, wm, ym, sm_count, stages, cols, smem, n_items, stream)
-                 : launch_pair_t<false, 1>(a, xm, wm, ym, sm_count, stages, cols, smem, n_items, stream);
+    return a.dense ? launch_pair_t<true, 2, false>(a, xm, wm, ym, sm_count, stages, cols, smem, n_items, stream)
+                   : launch_pair_t<false, 2, false>(a, xm, wm, ym, sm_count, stages, cols, smem, n_items, stream);
+  return a.dense ? launch_pair_t<true, 1, false>(a, xm, wm, ym, sm_count, stages, cols, smem, n_items, stream)
+                 : launch_pair_t<false, 1, false>(a, xm, wm, ym, sm_count, stages, cols, smem, n_items, stream);
 }
 
 }  // namespace rt3d

@@ -233,7 +233,7 @@ def test_pair_kernel_tail_split_against_oracle(case):
     y, ref, lay, xd, yt = run_case(spec, n, t, h, w, 4, 4, "none" if dense else "bernoulli", 0.4, torch.bfloat16,
                                    rt3d.ALGO_AUTO, dense=dense)
     plan = rt3d.rt3d_last_plan()
-    assert plan["kernel"] == 2 and plan["tail_workers"] > 0, plan
+    assert plan["kernel"] in (2, 7) and plan["tail_workers"] > 0, plan     # 7: narrow bundle, one deeper input tile per kt group
     check(y, ref, torch.bfloat16, f"tail split {case}")
     first = yt.clone()
     for _ in range(3):                       # flags reset themselves; the sum order is fixed

@@ -74,6 +74,8 @@ def test_tensor_core_layout_holds_exactly_the_masked_weights(M, N, k, g_m, g_n, 
     L = _layer(M, N, k, g_m, g_n, 0.3, 11)
     pk = rt3d.rt3d_pack_kgs(L["w"], L["mask"], g_m, g_n, rt3d.RT3D_BF16)
     np.testing.assert_array_equal(pk.unpack_device_layout(n_tile), oracle.bf16_round(L["w"] * L["mask"]))
+    # the t-grouped order of the same layout (its group tables are checked inside the call)
+    np.testing.assert_array_equal(pk.unpack_device_layout(n_tile, t_groups=True), oracle.bf16_round(L["w"] * L["mask"]))
     with pytest.raises(rt3d.Rt3dError):
         rt3d.rt3d_pack_kgs(L["w"], L["mask"], g_m, g_n, rt3d.RT3D_F32).unpack_device_layout(n_tile)
 
@@ -93,6 +95,7 @@ def test_vanilla_high_rate_skips_steps_in_layout():
     L = synth.make_layer(spec, 9, 1, 4, 4, "vanilla_total", (16 * 64) // 8)
     pk = rt3d.rt3d_pack_kgs(L["w"], L["mask"], 4, 4, rt3d.RT3D_BF16)
     np.testing.assert_array_equal(pk.unpack_device_layout(16), oracle.bf16_round(L["w"] * L["mask"]))
+    np.testing.assert_array_equal(pk.unpack_device_layout(16, t_groups=True), oracle.bf16_round(L["w"] * L["mask"]))
 
 
 @pytest.mark.parametrize("M,N,k,g_m,g_n,density", [(256, 256, (3, 3, 3), 8, 8, 0.125), (256, 128, (3, 3, 3), 4, 4, 0.4),
