@@ -559,7 +559,7 @@ rt3d_status try_halo(rt3d_packed* w, DeviceBlob* blob, DeviceState* d, const rt3
   a.pool_t = a.pool_h = a.pool_w = 1;
   a.n_splits = 1; a.scratch = nullptr; a.counters = nullptr;
   a.tail_workers = 0; a.tail_scratch = nullptr; a.tail_flags = nullptr;
-  a.ts = 0; a.grp_ptr = nullptr; a.grp_first = nullptr; a.ts_a_bytes = 0; a.ts_frame_bytes = 0;
+  a.ts = 0; a.grp_ptr = nullptr; a.grp_first = nullptr; a.ts_a_bytes = 0; a.ts_frame_bytes = 0; a.ts_table = 0;
   a.wait_cycles = 0; a.debug_drop_last_load = 0;
   ConvGeom unit = g;                       // the staged block is a plain box of input voxels
   CUtensorMap xmap, ymap;
@@ -700,7 +700,7 @@ rt3d_status conv_impl(const rt3d_tensor* x, const rt3d_packed* wc, const float* 
   a.g = g;
   int sb[4] = {1, 1, 1, 1};
   bool rect;
-  const bool prefer_deep = g_ts_enabled.load() && g.st == 1 && (g.Kt == 2 || g.Kt == 3) && default_n_tile(w->M) <= 128;
+  const bool prefer_deep = g_ts_enabled.load() && g.st == 1 && (g.Kt == 2 || g.Kt == 3);
   if (pooled) {
     if (!choose_box_pool(g, pl_w, pl_h, pl_t, &a.box, sb, prefer_deep)) return RT3D_ERR_UNSUPPORTED;
     rect = true;
@@ -732,10 +732,10 @@ rt3d_status conv_impl(const rt3d_tensor* x, const rt3d_packed* wc, const float* 
   if (pooled && plan.n_tile % 32) return RT3D_ERR_UNSUPPORTED;      // pooled rows leave as whole 32-channel pieces
   // CTA pairs on bundles up to 128 wide with a kernel that is 2 or 3 deep: one deeper input tile per (kh, kw, chunk)
   bool use_ts = false;
+  UmmaArgs probe = a;
   if (use_pair && g_ts_enabled.load()) {
-    UmmaArgs probe = a;
     probe.n_tile = plan.n_tile; probe.n_bundles = ceil_div(w->M, plan.n_tile); probe.dense = dense_entry ? 1 : 0;
-    use_ts = umma_pair_ts_supported(probe, w->Ks * ceil_div(w->N, kChunk) * probe.n_bundles);
+    use_ts = umma_pair_ts_supported(&probe, w->Ks * ceil_div(w->N, kChunk) * probe.n_bundles);
   }
   const UmmaLayout* L = get_umma_layout(w, plan.n_tile, use_ts);
   if (!L) return RT3D_ERR_UNSUPPORTED;
@@ -749,7 +749,7 @@ rt3d_status conv_impl(const rt3d_tensor* x, const rt3d_packed* wc, const float* 
   a.residual = res_data; a.rcs = res_pitch;
   a.n_splits = plan.n_splits; a.scratch = nullptr; a.counters = nullptr;
   a.tail_workers = 0; a.tail_scratch = nullptr; a.tail_flags = nullptr;
-  a.ts = 0; a.grp_ptr = nullptr; a.grp_first = nullptr; a.ts_a_bytes = 0; a.ts_frame_bytes = 0;
+  a.ts = 0; a.grp_ptr = nullptr; a.grp_first = nullptr; a.ts_a_bytes = 0; a.ts_frame_bytes = 0; a.ts_table = 0;
   a.wait_cycles = debug_wait_cycles(); a.debug_drop_last_load = g_debug_drop_last_load.load();
   if (a.n_splits > 1) {
     // split-K workspace of this handle on this device: partial tiles + per-warp arrival counters
@@ -760,8 +760,7 @@ rt3d_status conv_impl(const rt3d_tensor* x, const rt3d_packed* wc, const float* 
   }
   if (use_ts) {
     a.ts = 1; a.grp_ptr = u->grp_ptr; a.grp_first = u->grp_first;
-    a.ts_frame_bytes = a.box.bh * a.box.bw * 128;
-    a.ts_a_bytes = (a.box.bt + g.Kt - 1) * a.ts_frame_bytes;
+    a.ts_a_bytes = probe.ts_a_bytes; a.ts_frame_bytes = probe.ts_frame_bytes; a.ts_table = probe.ts_table;
   }
   CUtensorMap xmap;
   if ((s = encode_xmap(x, g, a.box, &xmap, use_ts ? g.Kt - 1 : 0)) != RT3D_OK) return s;
@@ -1246,7 +1245,7 @@ rt3d_status rt3d_conv3d_sparse_noalloc(const rt3d_tensor* x, const rt3d_packed* 
   int sb[4];
   a.pool_t = a.pool_h = a.pool_w = 1; a.sbw = a.sbh = 1;
   a.tail_workers = 0; a.tail_scratch = nullptr; a.tail_flags = nullptr;
-  a.ts = 0; a.grp_ptr = nullptr; a.grp_first = nullptr; a.ts_a_bytes = 0; a.ts_frame_bytes = 0;
+  a.ts = 0; a.grp_ptr = nullptr; a.grp_first = nullptr; a.ts_a_bytes = 0; a.ts_frame_bytes = 0; a.ts_table = 0;
   a.wait_cycles = 0; a.debug_drop_last_load = 0;
   a.store_tma = (a.n_splits == 1 && warp_block(a.box.bw, a.box.bh, a.box.bt, a.box.bn, sb) &&
                  encode_ymap(y, sb, 1, 1, 1, &ymap)) ? 1 : 0;

@@ -65,6 +65,7 @@ struct UmmaArgs {
   const int32_t* grp_first;                 // device, first step of each group + sentinel
   int ts_a_bytes;                           // bytes of the deeper input tile
   int ts_frame_bytes;                       // bytes of one frame of it (bh * bw rows of 128 bytes)
+  int ts_table;                             // entries reserved in shared memory for the step list (the group list follows)
   long long wait_cycles;                    // single-CTA kernel: SM clocks after which a wait gives up (0 = the default, about 1 s)
   int debug_drop_last_load;                 // single-CTA kernel, tests only: never issue the loads of each CTA's last stage
 };
@@ -83,8 +84,9 @@ bool umma_pair_supported(int n_tile, int n_bundles);
 // With a->ts the unit of the split is a group: `grp_ptr_host` = the layout's per-bundle group offsets.
 void umma_pair_tail_plan(UmmaArgs* a, const int32_t* step_ptr_host, int sm_count, size_t* scratch_bytes,
                          size_t* flag_bytes, const int32_t* grp_ptr_host = nullptr);
-// Whether the t-grouped variant can run this shape (and is expected to pay).
-bool umma_pair_ts_supported(const UmmaArgs& a, int total_steps);
+// Whether the t-grouped variant can run this shape (and is expected to pay); `total_steps`: all bundles' lists.
+// Fills a->ts_a_bytes, ts_frame_bytes and ts_table when it can.
+bool umma_pair_ts_supported(UmmaArgs* a, int total_steps);
 cudaError_t launch_conv_umma_pair(const UmmaArgs& a, const void* xmap, const void* wmap_half, const void* ymap,
                                   int sm_count, cudaStream_t stream);
 

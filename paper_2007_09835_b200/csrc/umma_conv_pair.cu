@@ -54,8 +54,8 @@ __device__ __forceinline__ Work get_work(const TailWork* tw, int wi, int cluster
 // tile, as long as 30 K steps.  Shares and fix-ups of split tiles are divided between the sets the same way.
 constexpr int kThreadsPair = 352;
 
-// t-grouped variant: step and group tables (all bundles together) live in shared memory, up to this many entries each.
-constexpr int kTsTable = 1024;
+// t-grouped variant: step and group tables (all bundles together) live in shared memory, up to this many steps.
+constexpr int kTsTable = 2048;
 
 // kCps: K steps per pipeline stage (and per barrier hand-shake): 1, or 2 for narrow bundles.
 // kTS: t-grouped layout.  A pipeline stage then holds ONE input tile that is Kt - 1 frames deeper and the weight
@@ -80,7 +80,7 @@ conv3d_umma_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_c
   TailWork* tw = reinterpret_cast<TailWork*>(bars + 1);
   float* bias_s = align16_f32(tw + 1);
   int32_t* steps_s = reinterpret_cast<int32_t*>(bias_s + a.n_bundles * a.n_tile);   // kTS only: steps, then group starts
-  int32_t* grp_s = steps_s + kTsTable;
+  int32_t* grp_s = steps_s + a.ts_table;
   const int ts_groups_dense = a.g.Kh * a.g.Kw * a.n_chunks;
   int32_t* err = a.sched + 2;
 
@@ -509,12 +509,14 @@ size_t ts_stage_bytes(const UmmaArgs& a) {
   return ((size_t(a.ts_a_bytes) + 1023) & ~size_t(1023)) + size_t(a.g.Kt) * size_t(a.n_tile / 2) * 128;
 }
 int pick_stages_pair_ts(const UmmaArgs& a) {
-  const int s = int(kSmemBudget / ts_stage_bytes(a));
+  const size_t fixed = 1024 + 4 * kStoreWarpBytes + sizeof(Barriers) + sizeof(TailWork) + 16 +
+                       size_t(a.n_tile) * a.n_bundles * 4 + (2 * size_t(a.ts_table) + 8) * 4;
+  const int s = int((size_t(227) * 1024 - fixed) / ts_stage_bytes(a));
   return s > kMaxStages ? kMaxStages : s;
 }
 size_t pair_smem_bytes_ts(const UmmaArgs& a) {
   return size_t(pick_stages_pair_ts(a)) * ts_stage_bytes(a) + 1024 + 4 * kStoreWarpBytes + sizeof(Barriers) + sizeof(TailWork) +
-         16 + size_t(a.n_tile) * a.n_bundles * 4 + (2 * size_t(kTsTable) + 8) * 4;
+         16 + size_t(a.n_tile) * a.n_bundles * 4 + (2 * size_t(a.ts_table) + 8) * 4;
 }
 
 template <bool kDense, int kCps, bool kTS>
@@ -569,7 +571,9 @@ int pair_max_clusters(int n_tile, int n_bundles, bool dense, int sm_count) {
 }
 int pair_max_clusters_ts(const UmmaArgs& a, int sm_count) {
   const size_t smem = pair_smem_bytes_ts(a);
-  return a.dense ? pair_max_clusters_t<true, 2, true>(sm_count, smem) : pair_max_clusters_t<false, 2, true>(sm_count, smem);
+  if (pick_cps(a.n_tile) == 2)
+    return a.dense ? pair_max_clusters_t<true, 2, true>(sm_count, smem) : pair_max_clusters_t<false, 2, true>(sm_count, smem);
+  return a.dense ? pair_max_clusters_t<true, 1, true>(sm_count, smem) : pair_max_clusters_t<false, 1, true>(sm_count, smem);
 }
 
 template <bool kDense, int kCps, bool kTS>
@@ -593,14 +597,18 @@ bool umma_pair_supported(int n_tile, int n_bundles) {
 
 // Tail split: decides how many CTA pairs share the items that do not fill a last round (0 = no split)
 // and how much scratch that needs.  `step_ptr_host`: the layout's per-bundle step offsets (sparse path).
-bool umma_pair_ts_supported(const UmmaArgs& a, int total_steps) {
-  if (a.n_tile > 128 || a.n_tile % 16 || a.g.st != 1 || a.box.bn != 1 || a.box.bt < 2) return false;
-  if (a.g.Kt < 2 || a.g.Kt > 3) return false;
-  if (a.box.bt + a.g.Kt - 1 > 256) return false;
-  if (!a.dense && total_steps > kTsTable) return false;
-  UmmaArgs t = a;
-  t.ts_a_bytes = (a.box.bt + a.g.Kt - 1) * a.box.bh * a.box.bw * 128;
-  return pick_stages_pair_ts(t) >= 3 && pair_smem_bytes_ts(t) <= 227 * 1024;
+bool umma_pair_ts_supported(UmmaArgs* a, int total_steps) {
+  if (a->n_tile > 256 || a->n_tile % 16 || a->g.st != 1 || a->box.bn != 1 || a->box.bt < 2) return false;
+  if (a->g.Kt < 2 || a->g.Kt > 3) return false;
+  if (a->box.bt + a->g.Kt - 1 > 256 || total_steps > kTsTable) return false;
+  UmmaArgs t = *a;
+  t.ts_frame_bytes = a->box.bh * a->box.bw * 128;
+  t.ts_a_bytes = (a->box.bt + a->g.Kt - 1) * t.ts_frame_bytes;
+  t.ts_table = a->dense ? 0 : (total_steps + 3) & ~3;
+  // at least as many steps in flight as the step-per-location form has, and it has to fit
+  if (pick_stages_pair_ts(t) < 3 || pair_smem_bytes_ts(t) > 227 * 1024) return false;
+  a->ts_frame_bytes = t.ts_frame_bytes; a->ts_a_bytes = t.ts_a_bytes; a->ts_table = t.ts_table;
+  return true;
 }
 
 void umma_pair_tail_plan(UmmaArgs* a, const int32_t* step_ptr_host, int sm_count, size_t* scratch_bytes,
@@ -653,7 +661,7 @@ cudaError_t launch_conv_umma_pair(const UmmaArgs& a, const void* xmap, const voi
   if (a.tail_workers > 0 && (a.tail_scratch == nullptr || a.tail_flags == nullptr)) return cudaErrorInvalidValue;
   const int stages = a.ts ? pick_stages_pair_ts(a) : pick_stages_pair(a.n_tile);
   const size_t smem = a.ts ? pair_smem_bytes_ts(a) : pair_smem_bytes(a.n_tile, a.n_bundles);
-  if (a.ts && (a.n_tile > 128 || smem > 227 * 1024 || stages < 2)) return cudaErrorInvalidValue;
+  if (a.ts && (smem > 227 * 1024 || stages < 2)) return cudaErrorInvalidValue;
   int cols = 32;
   while (cols < 2 * a.n_tile * (pick_cps(a.n_tile) == 2 ? 2 : 1)) cols *= 2;     // two issuing threads: two accumulators
   if (cols > 512) return cudaErrorInvalidValue;
@@ -665,9 +673,12 @@ cudaError_t launch_conv_umma_pair(const UmmaArgs& a, const void* xmap, const voi
   memcpy(&xm, xmap, sizeof(CUtensorMap));
   memcpy(&wm, wmap_half, sizeof(CUtensorMap));
   memcpy(&ym, ymap ? ymap : xmap, sizeof(CUtensorMap));
-  if (a.ts)
+  if (a.ts && pick_cps(a.n_tile) == 2)
     return a.dense ? launch_pair_t<true, 2, true>(a, xm, wm, ym, sm_count, stages, cols, smem, n_items, stream)
                    : launch_pair_t<false, 2, true>(a, xm, wm, ym, sm_count, stages, cols, smem, n_items, stream);
+  if (a.ts)
+    return a.dense ? launch_pair_t<true, 1, true>(a, xm, wm, ym, sm_count, stages, cols, smem, n_items, stream)
+                   : launch_pair_t<false, 1, true>(a, xm, wm, ym, sm_count, stages, cols, smem, n_items, stream);
   if (pick_cps(a.n_tile) == 2)
     return a.dense ? launch_pair_t<true, 2, false>(a, xm, wm, ym, sm_count, stages, cols, smem, n_items, stream)
                    : launch_pair_t<false, 2, false>(a, xm, wm, ym, sm_count, stages, cols, smem, n_items, stream);

@@ -402,7 +402,7 @@ def test_cfg1_c3d_conv3a_full_size(mode):
                           dense=(mode == "dense"))
     rel = check(y, ref, torch.bfloat16, f"cfg1 {mode}")
     assert rel < 1e-2
-    assert rt3d.rt3d_last_plan()["kernel"] == 2                # CTA pairs: 196 tile pairs on 74 pairs of SMs
+    assert rt3d.rt3d_last_plan()["kernel"] in (2, 7)           # CTA pairs: 196 tile pairs on 74 pairs of SMs
 
 
 # ------------------------------------------------------------------ host entry point, glue

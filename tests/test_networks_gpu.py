@@ -116,7 +116,7 @@ def test_c3d_layers_teacher_forced_at_the_batch16_plan(c3d):
     plans_fwd = {}
     net.forward(nets.to_device(x16), plan_log=plans_fwd)          # what the real forward pass runs per layer
     assert rt3d.rt3d_last_device_status() == rt3d.OK
-    assert plans_fwd["conv3a"]["kernel"] == 2 and plans_fwd["conv1"]["kernel"] == 3
+    assert plans_fwd["conv3a"]["kernel"] in (2, 7) and plans_fwd["conv1"]["kernel"] == 3
     assert plans_fwd["conv1"]["fused_pool"] == 1 and plans_fwd["conv2"]["fused_pool"] == 1
     assert any(p["tail_workers"] > 0 for p in plans_fwd.values())  # the batch-16 pass does use the tail split
     for i, op in enumerate(plan):
