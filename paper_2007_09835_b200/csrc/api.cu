@@ -36,7 +36,8 @@ thread_local bool t_plan_only = false;
 // Test hooks of the single-CTA tensor-core kernel (rt3d_debug_set).
 std::atomic<long long> g_debug_wait_cycles{-1};      // -1: not set yet (RT3D_DEBUG_TIMEOUT_POLLS is read on first use)
 std::atomic<int> g_debug_drop_last_load{0};
-std::atomic<int> g_ts_enabled{1};            // t-grouped CTA-pair variant (RT3D_DEBUG_T_GROUPS switches it off for comparisons)
+// t-grouped CTA-pair variant: on unless the environment says RT3D_T_GROUPS=0; RT3D_DEBUG_T_GROUPS switches it at run time
+std::atomic<int> g_ts_enabled{[] { const char* e = getenv("RT3D_T_GROUPS"); return (e && e[0] == '0') ? 0 : 1; }()};
 long long debug_wait_cycles() {
   long long v = g_debug_wait_cycles.load();
   if (v < 0) {
@@ -700,12 +701,11 @@ rt3d_status conv_impl(const rt3d_tensor* x, const rt3d_packed* wc, const float* 
   a.g = g;
   int sb[4] = {1, 1, 1, 1};
   bool rect;
-  const bool prefer_deep = g_ts_enabled.load() && g.st == 1 && (g.Kt == 2 || g.Kt == 3);
   if (pooled) {
-    if (!choose_box_pool(g, pl_w, pl_h, pl_t, &a.box, sb, prefer_deep)) return RT3D_ERR_UNSUPPORTED;
+    if (!choose_box_pool(g, pl_w, pl_h, pl_t, &a.box, sb)) return RT3D_ERR_UNSUPPORTED;
     rect = true;
   } else {
-    a.box = choose_box(g, prefer_deep);
+    a.box = choose_box(g);
     rect = warp_block(a.box.bw, a.box.bh, a.box.bt, a.box.bn, sb);
   }
   a.pool_t = pl_t; a.pool_h = pl_h; a.pool_w = pl_w; a.sbw = sb[0]; a.sbh = sb[1];
@@ -731,11 +731,30 @@ rt3d_status conv_impl(const rt3d_tensor* x, const rt3d_packed* wc, const float* 
   }
   if (pooled && plan.n_tile % 32) return RT3D_ERR_UNSUPPORTED;      // pooled rows leave as whole 32-channel pieces
   // CTA pairs on bundles up to 128 wide with a kernel that is 2 or 3 deep: one deeper input tile per (kh, kw, chunk)
+  // (its box: among the boxes with as few tiles, one inside a single clip and as deep along t as possible)
   bool use_ts = false;
   UmmaArgs probe = a;
-  if (use_pair && g_ts_enabled.load()) {
+  // (wide bundles: only kernels that are also wide in space; a 3x1x1 layer with 192-wide bundles lost 8 us of 43
+  // inside the S3D-shaped forward with it, while 3x3x3 layers gain 1-4 %)
+  if (use_pair && g_ts_enabled.load() && g.st == 1 && (g.Kt == 2 || g.Kt == 3) && (plan.n_tile <= 128 || g.Kh * g.Kw >= 4)) {
+    int sb2[4] = {1, 1, 1, 1};
+    TileBox deep = a.box;
+    const bool ok2 = pooled ? choose_box_pool(g, pl_w, pl_h, pl_t, &deep, sb2, true)
+                            : (deep = choose_box(g, true), warp_block(deep.bw, deep.bh, deep.bt, deep.bn, sb2) == rect);
+    const long long tiles2 = (long long)ceil_div(g.n, deep.bn) * ceil_div(g.To, deep.bt) * ceil_div(g.Ho, deep.bh) * ceil_div(g.Wo, deep.bw);
+    if (ok2 && tiles2 == m_tiles) {
+      probe.box = deep;
+      probe.sbw = sb2[0]; probe.sbh = sb2[1];
+      probe.tiles_n = ceil_div(g.n, deep.bn); probe.tiles_t = ceil_div(g.To, deep.bt);
+      probe.tiles_h = ceil_div(g.Ho, deep.bh); probe.tiles_w = ceil_div(g.Wo, deep.bw);
+    }
     probe.n_tile = plan.n_tile; probe.n_bundles = ceil_div(w->M, plan.n_tile); probe.dense = dense_entry ? 1 : 0;
     use_ts = umma_pair_ts_supported(&probe, w->Ks * ceil_div(w->N, kChunk) * probe.n_bundles);
+    if (use_ts) {
+      a.box = probe.box; a.sbw = probe.sbw; a.sbh = probe.sbh;
+      a.tiles_n = probe.tiles_n; a.tiles_t = probe.tiles_t; a.tiles_h = probe.tiles_h; a.tiles_w = probe.tiles_w;
+      for (int i = 0; i < 4; ++i) sb[i] = sb2[i];
+    }
   }
   const UmmaLayout* L = get_umma_layout(w, plan.n_tile, use_ts);
   if (!L) return RT3D_ERR_UNSUPPORTED;
