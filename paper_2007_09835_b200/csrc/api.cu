@@ -257,7 +257,26 @@ rt3d_status get_sub_blob(rt3d_packed* h, DeviceBlob* blob, const SubLayout* L, D
 // ties go to the wider box along w, then h (longer contiguous runs for the TMA engine).
 // `prefer_deep`: ties go first to boxes inside one clip, then to the deeper box along t (the t-grouped CTA-pair
 // variant shares one staged input tile between the kt steps; the deeper the box, the less the extra frames weigh).
+TileBox choose_box_search(const ConvGeom& g, bool prefer_deep);
+// The search is a few thousand iterations; repeated calls on the same shape (every eager forward pass) take the
+// answer from a small per-thread table.
 TileBox choose_box(const ConvGeom& g, bool prefer_deep = false) {
+  struct Entry { int n, To, Ho, Wo, st, sh, sw, deep; TileBox box; };
+  thread_local Entry cache[16];
+  thread_local int used = 0, next = 0;
+  for (int i = 0; i < used; ++i) {
+    const Entry& e = cache[i];
+    if (e.n == g.n && e.To == g.To && e.Ho == g.Ho && e.Wo == g.Wo && e.st == g.st && e.sh == g.sh && e.sw == g.sw &&
+        e.deep == int(prefer_deep))
+      return e.box;
+  }
+  const TileBox box = choose_box_search(g, prefer_deep);
+  cache[next] = Entry{g.n, g.To, g.Ho, g.Wo, g.st, g.sh, g.sw, int(prefer_deep), box};
+  next = (next + 1) % 16;
+  if (used < 16) ++used;
+  return box;
+}
+TileBox choose_box_search(const ConvGeom& g, bool prefer_deep) {
   TileBox best{1, 1, 1, 1};
   long long best_tiles = -1;
   for (int bw = 1; bw <= g.Wo && bw <= kTileM; ++bw) {
@@ -383,7 +402,28 @@ bool encode_ymap(const rt3d_tensor* y, const int sb[4], int pw, int ph, int pt, 
 
 // Box for a call with fused pooling: fewest tiles among the boxes whose extents and whose per-warp block
 // are multiples of the pooling window (every window then lies inside one warp's 32 voxels).
+bool choose_box_pool_search(const ConvGeom& g, int pw, int ph, int pt, TileBox* out, int sb_out[4], bool prefer_deep);
 bool choose_box_pool(const ConvGeom& g, int pw, int ph, int pt, TileBox* out, int sb_out[4], bool prefer_deep = false) {
+  struct Entry { int n, To, Ho, Wo, st, sh, sw, pw, ph, pt, deep; bool ok; TileBox box; int sb[4]; };   // as in choose_box
+  thread_local Entry cache[16];
+  thread_local int used = 0, next = 0;
+  for (int i = 0; i < used; ++i) {
+    const Entry& e = cache[i];
+    if (e.n == g.n && e.To == g.To && e.Ho == g.Ho && e.Wo == g.Wo && e.st == g.st && e.sh == g.sh && e.sw == g.sw &&
+        e.pw == pw && e.ph == ph && e.pt == pt && e.deep == int(prefer_deep)) {
+      if (e.ok) { *out = e.box; for (int k = 0; k < 4; ++k) sb_out[k] = e.sb[k]; }
+      return e.ok;
+    }
+  }
+  Entry e{g.n, g.To, g.Ho, g.Wo, g.st, g.sh, g.sw, pw, ph, pt, int(prefer_deep), false, TileBox{1, 1, 1, 1}, {1, 1, 1, 1}};
+  e.ok = choose_box_pool_search(g, pw, ph, pt, &e.box, e.sb, prefer_deep);
+  cache[next] = e;
+  next = (next + 1) % 16;
+  if (used < 16) ++used;
+  if (e.ok) { *out = e.box; for (int k = 0; k < 4; ++k) sb_out[k] = e.sb[k]; }
+  return e.ok;
+}
+bool choose_box_pool_search(const ConvGeom& g, int pw, int ph, int pt, TileBox* out, int sb_out[4], bool prefer_deep) {
   long long best_tiles = -1;
   for (int bw = pw; bw <= kTileM && bw <= round_up(g.Wo, pw); bw += pw) {
     if (bw * g.sw > 256) break;
@@ -736,7 +776,7 @@ rt3d_status conv_impl(const rt3d_tensor* x, const rt3d_packed* wc, const float* 
   UmmaArgs probe = a;
   // (wide bundles: only kernels that are also wide in space; a 3x1x1 layer with 192-wide bundles lost 8 us of 43
   // inside the S3D-shaped forward with it, while 3x3x3 layers gain 1-4 %)
-  if (use_pair && g_ts_enabled.load() && g.st == 1 && (g.Kt == 2 || g.Kt == 3) && (plan.n_tile <= 128 || g.Kh * g.Kw >= 4)) {
+  if (use_pair && g_ts_enabled.load() && g.st == 1 && g.Kt >= 2 && g.Kt <= 8 && (plan.n_tile <= 128 || g.Kh * g.Kw >= 4)) {
     int sb2[4] = {1, 1, 1, 1};
     TileBox deep = a.box;
     const bool ok2 = pooled ? choose_box_pool(g, pl_w, pl_h, pl_t, &deep, sb2, true)

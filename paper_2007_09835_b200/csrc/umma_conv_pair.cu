@@ -599,7 +599,7 @@ bool umma_pair_supported(int n_tile, int n_bundles) {
 // and how much scratch that needs.  `step_ptr_host`: the layout's per-bundle step offsets (sparse path).
 bool umma_pair_ts_supported(UmmaArgs* a, int total_steps) {
   if (a->n_tile > 256 || a->n_tile % 16 || a->g.st != 1 || a->box.bn != 1 || a->box.bt < 2) return false;
-  if (a->g.Kt < 2 || a->g.Kt > 3) return false;
+  if (a->g.Kt < 2 || a->g.Kt > 8) return false;
   if (a->box.bt + a->g.Kt - 1 > 256 || total_steps > kTsTable) return false;
   UmmaArgs t = *a;
   t.ts_frame_bytes = a->box.bh * a->box.bw * 128;
