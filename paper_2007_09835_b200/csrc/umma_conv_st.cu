@@ -16,7 +16,8 @@
 //   E2    eight more epilogue warps (two per lane quadrant, alternating 32-channel pieces) drain each output
 //         frame once its last contribution has landed (+ bias, residual, ReLU, bf16, 16-byte global stores).
 // CTA pairs (tcgen05 cta_group::2): two patches per MMA, each CTA holds half of both weight tensors.
-// The MMA warp issues S(p+1) before T(p), so E1(p) overlaps S(p+1) on the tensor pipe.
+// S and T are issued by two warps (the narrow temporal MMAs are bound by the issue rate of a thread, and two issuing
+// warps overlap on the pipe); S(p+1) is issued before T(p) can start, so E1(p) overlaps S(p+1) on the tensor pipe.
 //
 // Work split: the sequence of (patch pair, output frame) steps is cut into equal contiguous ranges, one per
 // CTA pair.  A range that begins inside a clip first computes the intermediate frame before its first
@@ -42,7 +43,7 @@
 namespace rt3d {
 namespace {
 
-constexpr int kThreadsSt = 576;         // producer, MMA, 8 x E1, 8 x E2 warps
+constexpr int kThreadsSt = 608;         // producer, MMA (spatial), 8 x E1, 8 x E2 warps, MMA (temporal)
 constexpr int kStOuts = 3;              // output accumulators in flight = temporal kernel extent
 
 struct StBars {
@@ -51,6 +52,7 @@ struct StBars {
   unsigned long long mid_full;          // leader: 16 E1 warps wrote the intermediate frame back into D1
   unsigned long long out_full[kStOuts]; // both: last contribution to an output accumulator is done
   unsigned long long out_empty[kStOuts];// leader: 16 E2 warps drained it
+  unsigned long long t_done[2];         // leader: the temporal MMAs that read D1 buffer b are done (it may be overwritten)
 };
 
 // Walk over this CTA pair's frame jobs.  g counts (patch pair, output frame) steps; a segment is the part of
@@ -149,6 +151,7 @@ conv3d_umma_st_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_con
     for (int b = 0; b < 2; ++b) mbar_init(smem_u32(&bars->tmem_full[b]), 1);
     mbar_init(smem_u32(&sb->w_full), 1);
     mbar_init(smem_u32(&sb->mid_full), 16);              // leader: 8 E1 warps of each CTA
+    for (int b = 0; b < 2; ++b) mbar_init(smem_u32(&sb->t_done[b]), 1);
     for (int s = 0; s < kStOuts; ++s) {
       mbar_init(smem_u32(&sb->out_full[s]), 1);
       mbar_init(smem_u32(&sb->out_empty[s]), 16);        // leader: 8 E2 warps of each CTA
@@ -220,12 +223,12 @@ conv3d_umma_st_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_con
     if (leader) {
       uint32_t elected;
       asm volatile("{\n.reg .pred p;\nelect.sync _|p, 0xffffffff;\nselp.u32 %0, 1, 0, p;\n}\n" : "=r"(elected));
-      const uint32_t idesc1 = instr_desc_bf16_pair(a.n1), idesc2 = instr_desc_bf16_pair(a.n2);
+      const uint32_t idesc1 = instr_desc_bf16_pair(a.n1);
       // high descriptor words.  Staged input: 128-byte swizzle, 8-row groups one halo row apart.  Weights:
       // 128-byte swizzle, groups 1024 bytes apart.  (The intermediate frame is read from tensor memory.)
       const uint64_t a1_hi = uint64_t(((uint32_t(a.hw) * 128u) >> 4) | (1u << 14) | (2u << 29)) << 32;
       const uint64_t b_hi = uint64_t((1024u >> 4) | (1u << 14) | (2u << 29)) << 32;
-      const uint32_t w1_16 = w1_smem >> 4, w2_16 = w2_smem >> 4;
+      const uint32_t w1_16 = w1_smem >> 4;
       int stage = 0;
       uint32_t phase = 0;
       bool ok = mbar_wait(smem_u32(&sb->w_full), 0, bars, err, 42);
@@ -256,52 +259,15 @@ conv3d_umma_st_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_con
         if (++stage == a.stages) { stage = 0; phase ^= 1u; }
         return true;
       };
-      // Per job j: all of S(j+1), then T(j), so that E1 converts frame j while the tensor pipe works on S(j+1).
-      // (Mixing the two shapes more finely is slower: alternating single MMAs of S and T took 143 us, and
-      // alternating T's taps with thirds of S 122 us, against 93 us in this order for the R(2+1)D stage-2 block.)
+      // The spatial MMAs S(j) come from this warp and the temporal ones T(j) from warp 18: one thread issuing both
+      // needed about 4350 clocks per frame for 36 + 27 MMAs whose tensor time is 3460 (the 27 narrow ones are bound
+      // by the issue rate of a single thread), while two issuing warps overlap on the pipe.  S(j + 1) overwrites the
+      // D1 buffer that T(j - 1) read its A operand from, so it waits for that T to be done.
       if (ok && cur.live) ok = issue_s(0);
       while (ok && cur.live) {
-        if (nxt.live) { if (!issue_s(j + 1)) break; }
-        if (!mbar_wait(smem_u32(&sb->mid_full), j & 1u, bars, err, 45)) break;
-        tc_fence_after();
-        const int qb = cur.g - cur.g0 - cur.ta;            // running number of output frame o is qb + o
-        const uint32_t mid_tmem = tmem_base + (j & 1u) * uint32_t(a.n1);
-        // the taps this job issues, oldest output frame first; a frame that starts here needs its accumulator
-        // drained of the frame that used it before.  All waiting is done before the first MMA is issued.
-        bool live[3];
-        uint32_t dd[3], acc0[3];
-#pragma unroll
-        for (int dt = 0; dt < 3; ++dt) {
-          const int o = cur.p + 1 - dt;
-          live[dt] = o >= cur.ta && o < cur.tb;
-          const uint32_t q = uint32_t(qb + o), slot = q % kStOuts;
-          const bool first = cur.p == (o > 0 ? o - 1 : 0);
-          dd[dt] = out_tmem + slot * uint32_t(a.n2);
-          acc0[dt] = first ? 0u : 1u;
-          if (live[dt] && first && ok)
-            ok = mbar_wait(smem_u32(&sb->out_empty[slot]), ((q / kStOuts) & 1u) ^ 1u, bars, err, 46);
-        }
-        if (!ok) break;
-        tc_fence_after();
-#pragma unroll
-        for (int dt = 2; dt >= 0; --dt) {
-          if (!live[dt]) continue;
-          const int m0 = a.mma2_ptr[dt], m1 = a.mma2_ptr[dt + 1];
-          const uint32_t d = dd[dt];
-          uint32_t acc = acc0[dt];
-#pragma unroll 2
-          for (int m = m0; m < m1; ++m) {
-            const uint64_t bdesc = b_hi | uint64_t(w2_16 + a.tab2[2 * m + 1]);
-            if (elected) umma_bf16_pair_ta(d, mid_tmem + a.tab2[2 * m], bdesc, idesc2, acc);
-            acc = 1u;
-          }
-        }
-        if (!ok) break;
-        if (elected) {
-          const int o1 = cur.p - 1;
-          if (o1 >= cur.ta && o1 < cur.tb) umma_commit_pair(smem_u32(&sb->out_full[uint32_t(qb + o1) % kStOuts]));
-          if (cur.p == T - 1 && cur.p >= cur.ta && cur.p < cur.tb)
-            umma_commit_pair(smem_u32(&sb->out_full[uint32_t(qb + cur.p) % kStOuts]));
+        if (nxt.live) {
+          if (j >= 1 && !mbar_wait(smem_u32(&sb->t_done[(j + 1) & 1u]), ((j - 1) >> 1) & 1u, bars, err, 48)) break;
+          if (!issue_s(j + 1)) break;
         }
         cur = nxt;
         if (nxt.live) st_next(nxt);
@@ -349,6 +315,66 @@ conv3d_umma_st_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_con
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster(mid_full_leader);
+    }
+  } else if (warp == 18) {
+    // ------------------------------------------------------------------ MMA issuer of the temporal conv (leader CTA only)
+    if (leader) {
+      uint32_t elected;
+      asm volatile("{\n.reg .pred p;\nelect.sync _|p, 0xffffffff;\nselp.u32 %0, 1, 0, p;\n}\n" : "=r"(elected));
+      const uint32_t idesc2 = instr_desc_bf16_pair(a.n2);
+      const uint64_t b_hi = uint64_t((1024u >> 4) | (1u << 14) | (2u << 29)) << 32;
+      const uint32_t w2_16 = w2_smem >> 4;
+      bool ok = mbar_wait(smem_u32(&sb->w_full), 0, bars, err, 42);
+      StWalk cur;
+      st_init(cur, T, total, cluster_id, n_clusters);
+      uint32_t j = 0;
+      while (ok && cur.live) {
+        if (!mbar_wait(smem_u32(&sb->mid_full), j & 1u, bars, err, 45)) break;
+        tc_fence_after();
+        const int qb = cur.g - cur.g0 - cur.ta;            // running number of output frame o is qb + o
+        const uint32_t mid_tmem = tmem_base + (j & 1u) * uint32_t(a.n1);
+        // the taps this job issues, oldest output frame first; a frame that starts here needs its accumulator
+        // drained of the frame that used it before.  All waiting is done before the first MMA is issued.
+        bool live[3];
+        uint32_t dd[3], acc0[3];
+#pragma unroll
+        for (int dt = 0; dt < 3; ++dt) {
+          const int o = cur.p + 1 - dt;
+          live[dt] = o >= cur.ta && o < cur.tb;
+          const uint32_t q = uint32_t(qb + o), slot = q % kStOuts;
+          const bool first = cur.p == (o > 0 ? o - 1 : 0);
+          dd[dt] = out_tmem + slot * uint32_t(a.n2);
+          acc0[dt] = first ? 0u : 1u;
+          if (live[dt] && first && ok)
+            ok = mbar_wait(smem_u32(&sb->out_empty[slot]), ((q / kStOuts) & 1u) ^ 1u, bars, err, 46);
+        }
+        if (!ok) break;
+        tc_fence_after();
+#pragma unroll
+        for (int dt = 2; dt >= 0; --dt) {
+          if (!live[dt]) continue;
+          const int m0 = a.mma2_ptr[dt], m1 = a.mma2_ptr[dt + 1];
+          const uint32_t d = dd[dt];
+          uint32_t acc = acc0[dt];
+#pragma unroll 2
+          for (int m = m0; m < m1; ++m) {
+            const uint64_t bdesc = b_hi | uint64_t(w2_16 + a.tab2[2 * m + 1]);
+            if (elected) umma_bf16_pair_ta(d, mid_tmem + a.tab2[2 * m], bdesc, idesc2, acc);
+            acc = 1u;
+          }
+        }
+        if (!ok) break;
+        if (elected) {
+          const int o1 = cur.p - 1;
+          if (o1 >= cur.ta && o1 < cur.tb) umma_commit_pair(smem_u32(&sb->out_full[uint32_t(qb + o1) % kStOuts]));
+          if (cur.p == T - 1 && cur.p >= cur.ta && cur.p < cur.tb)
+            umma_commit_pair(smem_u32(&sb->out_full[uint32_t(qb + cur.p) % kStOuts]));
+        }
+        if (elected) umma_commit_pair(smem_u32(&sb->t_done[j & 1u]));
+        st_next(cur);
+        ++j;
+      }
+      __syncwarp();
     }
   } else {
     // ------------------------------------------------------------------ E2: output accumulators -> y (both CTAs, 8 warps)
