@@ -378,6 +378,11 @@ void rt3d_plan_end(void);
  * form (kernel 2) on the same handle; default 1. */
 enum { RT3D_DEBUG_WAIT_CYCLES = 1, RT3D_DEBUG_DROP_LAST_LOAD = 2, RT3D_DEBUG_T_GROUPS = 3 };
 rt3d_status rt3d_debug_set(int what, long long value);
+/* Diagnostics.  RT3D_DEBUG_WAIT_SITE: after a synchronisation of the device, the number of the wait inside a
+ * kernel that gave up since the last rt3d_last_device_status (0 = none; the numbers are the last argument of the
+ * kernels' bounded waits in the sources); -1 on error.  Does not clear the word. */
+enum { RT3D_DEBUG_WAIT_SITE = 1 };
+long long rt3d_debug_get(int what);
 
 const char* rt3d_status_string(rt3d_status s);
 const char* rt3d_version(void);

@@ -393,6 +393,15 @@ def rt3d_alloc_count() -> int:
 DEBUG_WAIT_CYCLES, DEBUG_DROP_LAST_LOAD, DEBUG_T_GROUPS = 1, 2, 3
 
 
+def rt3d_debug_get(what: int) -> int:
+    _lib.rt3d_debug_get.restype = ctypes.c_longlong
+    _lib.rt3d_debug_get.argtypes = [ctypes.c_int]
+    return int(_lib.rt3d_debug_get(int(what)))
+
+
+DEBUG_WAIT_SITE = 1
+
+
 def rt3d_debug_set(what: int, value: int):
     _check(_lib.rt3d_debug_set(int(what), int(value)), "rt3d_debug_set")
 

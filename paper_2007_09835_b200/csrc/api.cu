@@ -600,7 +600,7 @@ rt3d_status try_halo(rt3d_packed* w, DeviceBlob* blob, DeviceState* d, const rt3
   a.pool_t = a.pool_h = a.pool_w = 1;
   a.n_splits = 1; a.scratch = nullptr; a.counters = nullptr;
   a.tail_workers = 0; a.tail_scratch = nullptr; a.tail_flags = nullptr;
-  a.ts = 0; a.grp_ptr = nullptr; a.grp_first = nullptr; a.ts_a_bytes = 0; a.ts_frame_bytes = 0; a.ts_table = 0;
+  a.ts = 0; a.grp_ptr = nullptr; a.grp_first = nullptr; a.ts_a_bytes = 0; a.ts_frame_bytes = 0; a.ts_table = 0; a.ts_phases = 1;
   a.wait_cycles = 0; a.debug_drop_last_load = 0;
   ConvGeom unit = g;                       // the staged block is a plain box of input voxels
   CUtensorMap xmap, ymap;
@@ -776,7 +776,7 @@ rt3d_status conv_impl(const rt3d_tensor* x, const rt3d_packed* wc, const float* 
   UmmaArgs probe = a;
   // (wide bundles: only kernels that are also wide in space; a 3x1x1 layer with 192-wide bundles lost 8 us of 43
   // inside the S3D-shaped forward with it, while 3x3x3 layers gain 1-4 %)
-  if (use_pair && g_ts_enabled.load() && g.st == 1 && g.Kt >= 2 && g.Kt <= 8 && (plan.n_tile <= 128 || g.Kh * g.Kw >= 4)) {
+  if (use_pair && g_ts_enabled.load() && g.st <= 2 && g.Kt >= 2 && g.Kt <= 8 && (plan.n_tile <= 128 || g.Kh * g.Kw >= 4)) {
     int sb2[4] = {1, 1, 1, 1};
     TileBox deep = a.box;
     const bool ok2 = pooled ? choose_box_pool(g, pl_w, pl_h, pl_t, &deep, sb2, true)
@@ -808,7 +808,7 @@ rt3d_status conv_impl(const rt3d_tensor* x, const rt3d_packed* wc, const float* 
   a.residual = res_data; a.rcs = res_pitch;
   a.n_splits = plan.n_splits; a.scratch = nullptr; a.counters = nullptr;
   a.tail_workers = 0; a.tail_scratch = nullptr; a.tail_flags = nullptr;
-  a.ts = 0; a.grp_ptr = nullptr; a.grp_first = nullptr; a.ts_a_bytes = 0; a.ts_frame_bytes = 0; a.ts_table = 0;
+  a.ts = 0; a.grp_ptr = nullptr; a.grp_first = nullptr; a.ts_a_bytes = 0; a.ts_frame_bytes = 0; a.ts_table = 0; a.ts_phases = 1;
   a.wait_cycles = debug_wait_cycles(); a.debug_drop_last_load = g_debug_drop_last_load.load();
   if (a.n_splits > 1) {
     // split-K workspace of this handle on this device: partial tiles + per-warp arrival counters
@@ -820,9 +820,10 @@ rt3d_status conv_impl(const rt3d_tensor* x, const rt3d_packed* wc, const float* 
   if (use_ts) {
     a.ts = 1; a.grp_ptr = u->grp_ptr; a.grp_first = u->grp_first;
     a.ts_a_bytes = probe.ts_a_bytes; a.ts_frame_bytes = probe.ts_frame_bytes; a.ts_table = probe.ts_table;
+    a.ts_phases = probe.ts_phases;
   }
   CUtensorMap xmap;
-  if ((s = encode_xmap(x, g, a.box, &xmap, use_ts ? g.Kt - 1 : 0)) != RT3D_OK) return s;
+  if ((s = encode_xmap(x, g, a.box, &xmap, use_ts ? ((g.Kt - 1) / g.st) * g.st : 0)) != RT3D_OK) return s;
   CUtensorMap ymap;
   a.store_tma = (a.n_splits == 1 && rect && encode_ymap(y, sb, pl_w, pl_h, pl_t, &ymap)) ? 1 : 0;
   if (pooled && !a.store_tma) return RT3D_ERR_UNSUPPORTED;
@@ -1206,6 +1207,16 @@ rt3d_status rt3d_last_plan(rt3d_plan_info* info) {
   return RT3D_OK;
 }
 
+long long rt3d_debug_get(int what) {
+  if (what != RT3D_DEBUG_WAIT_SITE) return -1;
+  DeviceState* d = nullptr;
+  if (get_device_state(&d) != RT3D_OK) return -1;
+  if (cudaDeviceSynchronize() != cudaSuccess) return -1;
+  int32_t word = 0;
+  if (cudaMemcpy(&word, d->sched + 2, 4, cudaMemcpyDeviceToHost) != cudaSuccess) return -1;
+  return word;
+}
+
 rt3d_status rt3d_last_device_status(void* stream) {
   DeviceState* d = nullptr;
   rt3d_status s = get_device_state(&d);
@@ -1304,7 +1315,7 @@ rt3d_status rt3d_conv3d_sparse_noalloc(const rt3d_tensor* x, const rt3d_packed* 
   int sb[4];
   a.pool_t = a.pool_h = a.pool_w = 1; a.sbw = a.sbh = 1;
   a.tail_workers = 0; a.tail_scratch = nullptr; a.tail_flags = nullptr;
-  a.ts = 0; a.grp_ptr = nullptr; a.grp_first = nullptr; a.ts_a_bytes = 0; a.ts_frame_bytes = 0; a.ts_table = 0;
+  a.ts = 0; a.grp_ptr = nullptr; a.grp_first = nullptr; a.ts_a_bytes = 0; a.ts_frame_bytes = 0; a.ts_table = 0; a.ts_phases = 1;
   a.wait_cycles = 0; a.debug_drop_last_load = 0;
   a.store_tma = (a.n_splits == 1 && warp_block(a.box.bw, a.box.bh, a.box.bt, a.box.bn, sb) &&
                  encode_ymap(y, sb, 1, 1, 1, &ymap)) ? 1 : 0;

@@ -63,7 +63,8 @@ struct UmmaArgs {
   int ts;
   const int32_t* grp_ptr;                   // device, [n_bundles + 1]
   const int32_t* grp_first;                 // device, first step of each group + sentinel
-  int ts_a_bytes;                           // bytes of the deeper input tile
+  int ts_a_bytes;                           // bytes of one deeper input tile
+  int ts_phases;                            // deeper tiles per group = temporal stride: tile r holds the frames t*st + r
   int ts_frame_bytes;                       // bytes of one frame of it (bh * bw rows of 128 bytes)
   int ts_table;                             // entries reserved in shared memory for the step list (the group list follows)
   long long wait_cycles;                    // single-CTA kernel: SM clocks after which a wait gives up (0 = the default, about 1 s)

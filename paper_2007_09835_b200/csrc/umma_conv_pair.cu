@@ -73,7 +73,8 @@ conv3d_umma_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_c
   const uint32_t b_bytes = uint32_t(n_half) * 128u;             // this CTA's half of the B tile
   const uint32_t chunk_bytes = kABytes + b_bytes;
   const uint32_t ts_a_slot = (uint32_t(a.ts_a_bytes) + 1023u) & ~1023u;
-  const uint32_t stage_bytes = kTS ? ts_a_slot + uint32_t(a.g.Kt) * b_bytes : kCps * chunk_bytes;
+  const uint32_t ts_a_all = ts_a_slot * uint32_t(a.ts_phases);       // one deeper tile per phase of the temporal stride
+  const uint32_t stage_bytes = kTS ? ts_a_all + uint32_t(a.g.Kt) * b_bytes : kCps * chunk_bytes;
   const uint32_t store_smem = tiles_base + uint32_t(stages) * stage_bytes;     // 4 warps x 2 staging buffers
   Barriers* bars = reinterpret_cast<Barriers*>(smem_raw + (tiles_base - raw) + size_t(stages) * stage_bytes +
                                                4 * kStoreWarpBytes);
@@ -81,6 +82,7 @@ conv3d_umma_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_c
   float* bias_s = align16_f32(tw + 1);
   int32_t* steps_s = reinterpret_cast<int32_t*>(bias_s + a.n_bundles * a.n_tile);   // kTS only: steps, then group starts
   int32_t* grp_s = steps_s + a.ts_table;
+  uint32_t* aoff_s = reinterpret_cast<uint32_t*>(grp_s + a.ts_table + 8);   // per step: where its A operand starts in the stage
   const int ts_groups_dense = a.g.Kh * a.g.Kw * a.n_chunks;
   int32_t* err = a.sched + 2;
 
@@ -182,9 +184,16 @@ conv3d_umma_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_c
   }
   if (kTS && !kDense) {                    // the layout's tables (host uploads only, as above)
     const int total_steps = __ldg(a.step_ptr + a.n_bundles), total_groups = __ldg(a.grp_ptr + a.n_bundles);
-    for (int i = threadIdx.x; i < total_steps; i += blockDim.x) steps_s[i] = __ldg(a.steps + i);
+    for (int i = threadIdx.x; i < total_steps; i += blockDim.x) {
+      const int enc = __ldg(a.steps + i);
+      const uint32_t kt = uint32_t(enc >> 24) & 63u;
+      steps_s[i] = enc;
+      // tap kt = q * st + r reads phase tile r from frame q on
+      aoff_s[i] = (kt % uint32_t(a.ts_phases)) * ts_a_slot + (kt / uint32_t(a.ts_phases)) * uint32_t(a.ts_frame_bytes);
+    }
     for (int i = threadIdx.x; i <= total_groups; i += blockDim.x) grp_s[i] = __ldg(a.grp_first + i);
   }
+
   pdl_wait();
   for (int i = threadIdx.x; i < a.n_bundles * a.n_tile; i += blockDim.x)
     bias_s[i] = (a.bias != nullptr && i < a.g.M) ? __ldg(a.bias + i) : 0.f;
@@ -204,14 +213,21 @@ conv3d_umma_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_c
         const int gbase = kDense ? 0 : a.grp_ptr[c.bundle];
         const int ngrp = kDense ? ts_groups_dense : a.grp_ptr[c.bundle + 1] - gbase;
         const int g1 = wk.g1 < ngrp ? wk.g1 : ngrp;
-        const int wq = c.w0 * a.g.sw - a.g.pw, hq = c.h0 * a.g.sh - a.g.ph, tq = c.t0 - a.g.pt;
+        const int wq = c.w0 * a.g.sw - a.g.pw, hq = c.h0 * a.g.sh - a.g.ph, tq = c.t0 * a.g.st - a.g.pt;
+        // computed steps: (kh, kw, chunk) of the share's first group by division once, then carried (three divisions
+        // per group made this lone thread the limit of the dense path on 128-wide layers)
+        int d_ch = 0, d_kw = 0, d_kh = 0;
+        if (kDense) {
+          d_ch = wk.g0 % a.n_chunks;
+          const int hw = wk.g0 / a.n_chunks;
+          d_kw = hw % a.g.Kw; d_kh = hw / a.g.Kw;
+        }
         for (int g = wk.g0; g < g1; ++g) {
           int s0, ns, kh, kw, ch;
           if (kDense) {
             s0 = c.bundle * a.steps_dense + g * a.g.Kt; ns = a.g.Kt;
-            ch = g % a.n_chunks;
-            const int hw = g / a.n_chunks;
-            kw = hw % a.g.Kw; kh = hw / a.g.Kw;
+            ch = d_ch; kw = d_kw; kh = d_kh;
+            if (++d_ch == a.n_chunks) { d_ch = 0; if (++d_kw == a.g.Kw) { d_kw = 0; ++d_kh; } }
           } else {
             s0 = grp_s[gbase + g]; ns = grp_s[gbase + g + 1] - s0;
             const int enc = steps_s[s0];
@@ -221,11 +237,13 @@ conv3d_umma_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_c
           const uint32_t full_leader = mapa_shared(full_local, 0);
           const uint32_t s_dst = tiles_base + stage * stage_bytes;
           if (!mbar_wait(smem_u32(&bars->empty[stage]), phase ^ 1u, bars, err, 21)) { ok = false; break; }
-          if (leader) mbar_expect_tx(full_local, 2u * (uint32_t(a.ts_a_bytes) + uint32_t(ns) * b_bytes));
-          tma_load_5d_pair(s_dst, &xmap, full_leader, ch * 64, wq + kw, hq + kh, tq, c.n0);
+          if (leader) mbar_expect_tx(full_local, 2u * (uint32_t(a.ts_phases * a.ts_a_bytes) + uint32_t(ns) * b_bytes));
+          // tile r: the frames t * st + r (traversal stride st along t), so that tap kt = q * st + r is its rows from frame q on
+          for (int r = 0; r < a.ts_phases; ++r)
+            tma_load_5d_pair(s_dst + uint32_t(r) * ts_a_slot, &xmap, full_leader, ch * 64, wq + kw, hq + kh, tq + r, c.n0);
           const int wrow = s0 * a.n_tile + int(rank) * n_half;
           for (int q = 0; q < ns; ++q)
-            tma_load_2d_pair(s_dst + ts_a_slot + uint32_t(q) * b_bytes, &wmap_half, full_leader, 0, wrow + q * a.n_tile);
+            tma_load_2d_pair(s_dst + ts_a_all + uint32_t(q) * b_bytes, &wmap_half, full_leader, 0, wrow + q * a.n_tile);
           if (++stage == stages) { stage = 0; phase ^= 1u; }
         }
       }
@@ -283,6 +301,10 @@ conv3d_umma_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_c
       uint32_t j = 0, phase = 0;
       int stage = 0;
       bool ok = true, ready = false;
+      // Two issuing threads share the groups by the parity of the RUNNING group number, i.e. by stage parity (the
+      // ring has an even number of stages then): a thread that skipped one fill of a stage and came back for the
+      // next could take the older completion of that stage's barrier for the one it waits for.
+      uint32_t gg = 0;
       const int n_work = tw->n_full + tw->n_seg;
       for (int wi = 0; kTS && wi < n_work && ok; ++wi, ++j) {
         const Work wk = get_work(tw, wi, cluster_id, n_clusters);
@@ -294,22 +316,24 @@ conv3d_umma_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_c
         if (!mbar_wait(smem_u32(&bars->tmem_empty[buf]), ((j >> 1) & 1u) ^ 1u, bars, err, 22)) break;
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (buf * uint32_t(kIss) + uint32_t(me)) * uint32_t(a.n_tile);
-        int gl = 0;                                          // group inside this item (or share)
-        for (int g = wk.g0; g < g1; ++g, ++gl) {
-          if (!kDual || (gl & 1) == me) {
+        bool fresh = true;                                   // this thread's accumulator has nothing of this item yet
+        for (int g = wk.g0; g < g1; ++g, ++gg) {
+          if (!kDual || int(gg & 1u) == me) {
             int s0 = 0, ns = a.g.Kt;
             if (!kDense) { s0 = grp_s[gbase + g]; ns = grp_s[gbase + g + 1] - s0; }
             if (!mbar_wait(smem_u32(&bars->full[stage]), phase, bars, err, 23)) { ok = false; break; }
             tc_fence_after();
             const uint32_t s_base = tiles_base + stage * stage_bytes;
             for (int q = 0; q < ns; ++q) {
-              const int kt = kDense ? q : (steps_s[s0 + q] >> 24) & 63;
-              const uint64_t adesc = smem_desc_sw128(s_base + uint32_t(kt) * uint32_t(a.ts_frame_bytes));
-              const uint64_t bdesc = smem_desc_sw128(s_base + ts_a_slot + uint32_t(q) * b_bytes);
+              // computed steps (temporal stride 1 only): kt = q.  Every instruction in this loop shows in the time of
+              // a 128-wide layer (four more ALU operations per step cost 6 %).
+              const uint64_t adesc = smem_desc_sw128(s_base + (kDense ? uint32_t(q) * uint32_t(a.ts_frame_bytes) : aoff_s[s0 + q]));
+              const uint64_t bdesc = smem_desc_sw128(s_base + ts_a_all + uint32_t(q) * b_bytes);
 #pragma unroll
               for (int kk = 0; kk < 4; ++kk)
-                umma_bf16_pair(d_tmem, adesc + 2 * kk, bdesc + 2 * kk, idesc, ((gl >= kIss) | q | kk) ? 1u : 0u);
+                umma_bf16_pair(d_tmem, adesc + 2 * kk, bdesc + 2 * kk, idesc, (!fresh | q | kk) ? 1u : 0u);
             }
+            fresh = false;
             umma_commit_pair(smem_u32(&bars->empty[stage]));
           }
           if (++stage == stages) { stage = 0; phase ^= 1u; }
@@ -326,12 +350,12 @@ conv3d_umma_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_c
         if (!mbar_wait(smem_u32(&bars->tmem_empty[buf]), ((j >> 1) & 1u) ^ 1u, bars, err, 22)) break;
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (buf * uint32_t(kIss) + uint32_t(me)) * uint32_t(a.n_tile);
-        int gl = 0;                                          // step group inside this item
-        for (int i = i0; i < i1; i += kCps, ++gl) {
+        bool fresh = true;
+        for (int i = i0; i < i1; i += kCps, ++gg) {
           const int nload = i1 - i < kCps ? i1 - i : kCps;
           const int stage_n = stage + 1 == stages ? 0 : stage + 1;
           const uint32_t phase_n = stage + 1 == stages ? phase ^ 1u : phase;
-          if (!kDual || (gl & 1) == me) {
+          if (!kDual || int(gg & 1u) == me) {
             if (!ready && !mbar_wait(smem_u32(&bars->full[stage]), phase, bars, err, 23)) { ok = false; break; }
             // one issuer: poll the next stage's barrier now, its answer arrives while this stage's MMAs are issued
             ready = kDual ? false : mbar_try_wait(smem_u32(&bars->full[stage_n]), phase_n);
@@ -344,8 +368,9 @@ conv3d_umma_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_c
               const uint64_t bdesc = smem_desc_sw128(a_addr + kABytes);
 #pragma unroll
               for (int kk = 0; kk < 4; ++kk)
-                umma_bf16_pair(d_tmem, adesc + 2 * kk, bdesc + 2 * kk, idesc, ((gl >= kIss) | q | kk) ? 1u : 0u);
+                umma_bf16_pair(d_tmem, adesc + 2 * kk, bdesc + 2 * kk, idesc, (!fresh | q | kk) ? 1u : 0u);
             }
+            fresh = false;
             umma_commit_pair(smem_u32(&bars->empty[stage]));
           }
           stage = stage_n; phase = phase_n;
@@ -378,6 +403,7 @@ conv3d_umma_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_c
     const int bt_0 = r0 % a.box.bt; r0 /= a.box.bt;
     const int bn_0 = r0;
     uint32_t j = 0;
+    uint32_t gg = 0;                                       // running group number, as the issuing threads count it
     const size_t part_tile = size_t(128) * a.n_tile;       // floats per partial tile
     const int n_work = tw->n_full + tw->n_seg;
     for (int wi = 0; wi < n_work; ++wi, ++j) {
@@ -391,7 +417,7 @@ conv3d_umma_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_c
       const bool in_range = row < box_rows && nn < a.g.n && to < a.g.To && ho < a.g.Ho && wo < a.g.Wo;
       const long long vox = (((long long)nn * a.g.To + to) * a.g.Ho + ho) * a.g.Wo + wo;
       const int m_base = c.bundle * a.n_tile;
-      const uint32_t taddr = tmem_base + (uint32_t(quad * 32) << 16) + buf * uint32_t(kIss * a.n_tile);
+      uint32_t taddr = tmem_base + (uint32_t(quad * 32) << 16) + buf * uint32_t(kIss * a.n_tile);
       // the second issuer's accumulator holds something once the item (or share) has two step groups
       int units_here;                                      // step groups (of kCps steps, or t-groups) of this item or share
       if (kTS) {
@@ -400,7 +426,11 @@ conv3d_umma_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_c
       } else {
         units_here = ((wk.g1 * kCps < nsteps ? wk.g1 * kCps : nsteps) - wk.g0 * kCps + kCps - 1) / kCps;
       }
+      // two issuing threads: groups with an even running number went into the first accumulator, odd ones into the
+      // second; an item (or share) of a single group is in one of them only
       const uint32_t acc2 = (kDual && units_here >= 2) ? uint32_t(a.n_tile) : 0u;
+      if (kDual && units_here == 1 && (gg & 1u)) taddr += uint32_t(a.n_tile);
+      gg += uint32_t(units_here > 0 ? units_here : 0);
       const __nv_bfloat16* res = (rb != nullptr && in_range) ? rb + vox * a.rcs + m_base : nullptr;
       const int res_left = a.rcs - m_base;
       if (wk.nparts > 1 && wk.part != 0) {
@@ -494,8 +524,10 @@ int pick_cps(int n_tile) { return n_tile <= 128 ? 2 : 1; }
 
 int pick_stages_pair(int n_tile) {
   const size_t stage = pick_cps(n_tile) * (kABytes + size_t(n_tile / 2) * 128);
-  const int s = int(kSmemBudget / stage);
-  return s > kMaxStages ? kMaxStages : s;
+  int s = int(kSmemBudget / stage);
+  if (s > kMaxStages) s = kMaxStages;
+  if (pick_cps(n_tile) == 2) s &= ~1;           // two issuing threads take the stages by parity
+  return s;
 }
 
 size_t pair_smem_bytes(int n_tile, int n_bundles) {
@@ -506,17 +538,19 @@ size_t pair_smem_bytes(int n_tile, int n_bundles) {
 
 // t-grouped variant: a stage = one deeper input tile + Kt weight half-tiles; the tables come after the bias.
 size_t ts_stage_bytes(const UmmaArgs& a) {
-  return ((size_t(a.ts_a_bytes) + 1023) & ~size_t(1023)) + size_t(a.g.Kt) * size_t(a.n_tile / 2) * 128;
+  return size_t(a.ts_phases) * ((size_t(a.ts_a_bytes) + 1023) & ~size_t(1023)) + size_t(a.g.Kt) * size_t(a.n_tile / 2) * 128;
 }
 int pick_stages_pair_ts(const UmmaArgs& a) {
   const size_t fixed = 1024 + 4 * kStoreWarpBytes + sizeof(Barriers) + sizeof(TailWork) + 16 +
-                       size_t(a.n_tile) * a.n_bundles * 4 + (2 * size_t(a.ts_table) + 8) * 4;
-  const int s = int((size_t(227) * 1024 - fixed) / ts_stage_bytes(a));
-  return s > kMaxStages ? kMaxStages : s;
+                       size_t(a.n_tile) * a.n_bundles * 4 + (3 * size_t(a.ts_table) + 16) * 4;
+  int s = int((size_t(227) * 1024 - fixed) / ts_stage_bytes(a));
+  if (s > kMaxStages) s = kMaxStages;
+  if (pick_cps(a.n_tile) == 2) s &= ~1;         // two issuing threads take the stages by parity
+  return s;
 }
 size_t pair_smem_bytes_ts(const UmmaArgs& a) {
   return size_t(pick_stages_pair_ts(a)) * ts_stage_bytes(a) + 1024 + 4 * kStoreWarpBytes + sizeof(Barriers) + sizeof(TailWork) +
-         16 + size_t(a.n_tile) * a.n_bundles * 4 + (2 * size_t(a.ts_table) + 8) * 4;
+         16 + size_t(a.n_tile) * a.n_bundles * 4 + (3 * size_t(a.ts_table) + 16) * 4;
 }
 
 template <bool kDense, int kCps, bool kTS>
@@ -598,16 +632,22 @@ bool umma_pair_supported(int n_tile, int n_bundles) {
 // Tail split: decides how many CTA pairs share the items that do not fill a last round (0 = no split)
 // and how much scratch that needs.  `step_ptr_host`: the layout's per-bundle step offsets (sparse path).
 bool umma_pair_ts_supported(UmmaArgs* a, int total_steps) {
-  if (a->n_tile > 256 || a->n_tile % 16 || a->g.st != 1 || a->box.bn != 1 || a->box.bt < 2) return false;
-  if (a->g.Kt < 2 || a->g.Kt > 8) return false;
-  if (a->box.bt + a->g.Kt - 1 > 256 || total_steps > kTsTable) return false;
+  if (a->n_tile > 256 || a->n_tile % 16 || a->g.st < 1 || a->g.st > 2 || a->box.bn != 1 || a->box.bt < 2) return false;
+  if (a->g.Kt < 2 || a->g.Kt > 8 || a->g.Kt <= a->g.st) return false;
+  if (a->dense && a->g.st != 1) return false;               // the computed-step path has no phase tiles
   UmmaArgs t = *a;
+  t.ts_phases = a->g.st;
+  const int frames = a->box.bt + (a->g.Kt - 1) / a->g.st;          // per phase tile (the deepest phase; the others load as many)
+  if (frames * a->g.st > 256 || total_steps > kTsTable) return false;
   t.ts_frame_bytes = a->box.bh * a->box.bw * 128;
-  t.ts_a_bytes = (a->box.bt + a->g.Kt - 1) * t.ts_frame_bytes;
+  t.ts_a_bytes = frames * t.ts_frame_bytes;
   t.ts_table = a->dense ? 0 : (total_steps + 3) & ~3;
-  // at least as many steps in flight as the step-per-location form has, and it has to fit
-  if (pick_stages_pair_ts(t) < 3 || pair_smem_bytes_ts(t) > 227 * 1024) return false;
-  a->ts_frame_bytes = t.ts_frame_bytes; a->ts_a_bytes = t.ts_a_bytes; a->ts_table = t.ts_table;
+  // it has to fit with at least as many steps in flight as the step-per-location form has
+  const int stages = pick_stages_pair_ts(t);
+  if (stages < 2 || stages * a->g.Kt < 8 || pair_smem_bytes_ts(t) > 227 * 1024) return false;
+  // and to stage fewer input bytes than one tile per step does
+  if (size_t(t.ts_phases) * t.ts_a_bytes * 4 > size_t(a->g.Kt) * a->box.bt * t.ts_frame_bytes * 3) return false;
+  a->ts_frame_bytes = t.ts_frame_bytes; a->ts_a_bytes = t.ts_a_bytes; a->ts_table = t.ts_table; a->ts_phases = t.ts_phases;
   return true;
 }
 

@@ -1,7 +1,8 @@
 """GPU parity of the CTA-pair kernel's t-grouped variant (plan kernel 7) against the CPU oracle.
 
 In that variant the steps that differ only in kt share ONE staged input tile that is Kt - 1 frames deeper, each
-step reading it through a descriptor that starts kt frames in; the step order, the unit of the tail split and the
+step reading it through a descriptor that starts kt frames in (with a temporal stride of 2: one deeper tile per
+phase of the stride, tap kt reading tile kt % 2 from frame kt / 2 on); the step order, the unit of the tail split and the
 two issuing threads' halves all change with it, so it gets its own cases: 2- and 3-deep kernels, dense and sparse
 lists, lists with pruned steps (groups of one or two steps), ragged boxes and channels, spatial strides, the tail
 split in both forms, fused pooling and residual.  Tolerance as everywhere: max|err| <= 2e-2 * max|ref| (bf16).
@@ -29,6 +30,8 @@ CASES = [
     (64, 128, (3, 3, 3), (1, 1, 1), (4, 8, 28, 28), (4, 4), "bernoulli", False, True),      # 98 items on 74 pairs
     (128, 128, (3, 3, 3), (1, 1, 1), (1, 8, 28, 28), (4, 4), "bernoulli", False, True),     # 25 items: all of them split
     (64, 128, (3, 3, 3), (1, 2, 2), (2, 8, 32, 32), (4, 4), "bernoulli", False, False),     # spatial stride
+    (64, 64, (7, 1, 1), (2, 1, 1), (2, 16, 40, 40), (4, 4), "bernoulli", False, False),     # temporal stride 2: two phase tiles
+    (64, 96, (5, 3, 3), (2, 1, 1), (2, 16, 20, 20), (4, 4), "bernoulli", False, True),      # the same, five taps, every tile split
 ]
 
 
