@@ -197,6 +197,13 @@ __device__ __forceinline__ void tmem_ld_acc(uint32_t taddr, bool wide, uint32_t 
 // (>= NC: 16-byte vector stores; fewer: scalar tail, channels beyond are left untouched).
 // `res`: this voxel's residual channels starting at the same channel as v[0] (nullptr: none), of which
 // `res_avail` may be read (the channel pitch bounds the vector loads).
+// max(x, 0) and max(y, 0) rounded to nearest-even bf16, x in the low half (as __floats2bfloat162_rn packs them).
+__device__ __forceinline__ uint32_t cvt_relu_bf16x2(float x, float y) {
+  uint32_t d;
+  asm("cvt.rn.relu.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(y), "f"(x));
+  return d;
+}
+
 template <int NC>
 __device__ __forceinline__ void epilogue_cols(const uint32_t* v, const float* bias_s, int relu,
                                               __nv_bfloat16* dst, int valid, const __nv_bfloat16* res, int res_avail) {
@@ -227,23 +234,24 @@ __device__ __forceinline__ void epilogue_cols(const uint32_t* v, const float* bi
       }
     }
   }
-  if (relu) {
-#pragma unroll
-    for (int q = 0; q < NC; ++q) f[q] = fmaxf(f[q], 0.f);
-  }
   if (valid >= NC) {
 #pragma unroll
     for (int q = 0; q < NC / 8; ++q) {
       uint4 o;
-      __nv_bfloat162* po = reinterpret_cast<__nv_bfloat162*>(&o);
+      if (relu) {                                  // activation and rounding in one instruction per pair
+        o.x = cvt_relu_bf16x2(f[8 * q], f[8 * q + 1]); o.y = cvt_relu_bf16x2(f[8 * q + 2], f[8 * q + 3]);
+        o.z = cvt_relu_bf16x2(f[8 * q + 4], f[8 * q + 5]); o.w = cvt_relu_bf16x2(f[8 * q + 6], f[8 * q + 7]);
+      } else {
+        __nv_bfloat162* po = reinterpret_cast<__nv_bfloat162*>(&o);
 #pragma unroll
-      for (int e = 0; e < 4; ++e) po[e] = __floats2bfloat162_rn(f[8 * q + 2 * e], f[8 * q + 2 * e + 1]);
+        for (int e = 0; e < 4; ++e) po[e] = __floats2bfloat162_rn(f[8 * q + 2 * e], f[8 * q + 2 * e + 1]);
+      }
       reinterpret_cast<uint4*>(dst)[q] = o;
     }
   } else {
 #pragma unroll
     for (int q = 0; q < NC; ++q)                 // static indices: f stays in registers
-      if (q < valid) dst[q] = __float2bfloat16_rn(f[q]);
+      if (q < valid) dst[q] = __float2bfloat16_rn(relu ? fmaxf(f[q], 0.f) : f[q]);
   }
 }
 
@@ -397,14 +405,15 @@ __device__ __forceinline__ void epilogue_piece_tma(const uint32_t* v, const floa
   }
   uint4 o[4];
   __nv_bfloat162* po = reinterpret_cast<__nv_bfloat162*>(o);
-#pragma unroll
-  for (int q = 0; q < 16; ++q) po[q] = __floats2bfloat162_rn(f[2 * q], f[2 * q + 1]);
-  // ReLU on the packed pairs: rounding is monotonic and keeps zero, so max(round(x), 0) = round(max(x, 0)), at
-  // half the instructions
+  // ReLU and the rounding to bf16 in one instruction per pair of values (the epilogue warps of the layers with few
+  // input channels are bound by their instruction count)
   if (relu) {
-    const __nv_bfloat162 zero2 = __floats2bfloat162_rn(0.f, 0.f);
+    uint32_t* uo = reinterpret_cast<uint32_t*>(o);
 #pragma unroll
-    for (int q = 0; q < 16; ++q) po[q] = __hmax2(po[q], zero2);
+    for (int q = 0; q < 16; ++q) uo[q] = cvt_relu_bf16x2(f[2 * q], f[2 * q + 1]);
+  } else {
+#pragma unroll
+    for (int q = 0; q < 16; ++q) po[q] = __floats2bfloat162_rn(f[2 * q], f[2 * q + 1]);
   }
   // optional max-pool: after the (monotonic) activation and bf16 rounding, so it equals pooling the stored tensor
   int out_row = lane;

@@ -304,9 +304,13 @@ conv3d_umma_st_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_con
           const float4 b = (wide || q < 4) ? b4[q] : make_float4(0.f, 0.f, 0.f, 0.f);
           float f0 = __uint_as_float(v[4 * q]) + b.x, f1 = __uint_as_float(v[4 * q + 1]) + b.y;
           float f2 = __uint_as_float(v[4 * q + 2]) + b.z, f3 = __uint_as_float(v[4 * q + 3]) + b.w;
-          if (a.g.relu) { f0 = fmaxf(f0, 0.f); f1 = fmaxf(f1, 0.f); f2 = fmaxf(f2, 0.f); f3 = fmaxf(f3, 0.f); }
-          po[2 * q] = __floats2bfloat162_rn(f0, f1);
-          po[2 * q + 1] = __floats2bfloat162_rn(f2, f3);
+          if (a.g.relu) {                         // activation and rounding in one instruction per pair
+            reinterpret_cast<uint32_t*>(po)[2 * q] = cvt_relu_bf16x2(f0, f1);
+            reinterpret_cast<uint32_t*>(po)[2 * q + 1] = cvt_relu_bf16x2(f2, f3);
+          } else {
+            po[2 * q] = __floats2bfloat162_rn(f0, f1);
+            po[2 * q + 1] = __floats2bfloat162_rn(f2, f3);
+          }
         }
         if (wide) tmem_st16(taddr + uint32_t(dst_col), o);
         else tmem_st8(taddr + uint32_t(dst_col), o);
@@ -440,12 +444,13 @@ conv3d_umma_st_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_con
             float f4 = __uint_as_float(v[8 * e + 4]) + b1.x + r2.x, f5 = __uint_as_float(v[8 * e + 5]) + b1.y + r2.y;
             float f6 = __uint_as_float(v[8 * e + 6]) + b1.z + r3.x, f7 = __uint_as_float(v[8 * e + 7]) + b1.w + r3.y;
             if (a.relu2) {
-              f0 = fmaxf(f0, 0.f); f1 = fmaxf(f1, 0.f); f2 = fmaxf(f2, 0.f); f3 = fmaxf(f3, 0.f);
-              f4 = fmaxf(f4, 0.f); f5 = fmaxf(f5, 0.f); f6 = fmaxf(f6, 0.f); f7 = fmaxf(f7, 0.f);
+              ov[e].x = cvt_relu_bf16x2(f0, f1); ov[e].y = cvt_relu_bf16x2(f2, f3);
+              ov[e].z = cvt_relu_bf16x2(f4, f5); ov[e].w = cvt_relu_bf16x2(f6, f7);
+            } else {
+              __nv_bfloat162* po = reinterpret_cast<__nv_bfloat162*>(&ov[e]);
+              po[0] = __floats2bfloat162_rn(f0, f1); po[1] = __floats2bfloat162_rn(f2, f3);
+              po[2] = __floats2bfloat162_rn(f4, f5); po[3] = __floats2bfloat162_rn(f6, f7);
             }
-            __nv_bfloat162* po = reinterpret_cast<__nv_bfloat162*>(&ov[e]);
-            po[0] = __floats2bfloat162_rn(f0, f1); po[1] = __floats2bfloat162_rn(f2, f3);
-            po[2] = __floats2bfloat162_rn(f4, f5); po[3] = __floats2bfloat162_rn(f6, f7);
           }
           if (in_range) {
             const int valid = a.M2 - col;              // real output channels from here on
