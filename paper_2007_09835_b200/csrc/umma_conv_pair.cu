@@ -29,6 +29,7 @@ namespace {
 // epilogue warps add the other pairs' partial tiles to it in a fixed order and write the output.
 struct TailSeg { int item, g0, g1, part, nparts; };
 constexpr int kMaxTailSeg = 6;
+constexpr int kMaxBundles = 64;
 constexpr int kMaxTail = 128;  // left-over items are fewer than the pairs of the grid (at most 74)
 struct TailWork {
   int n_full;                 // whole items of this pair: item = cluster_id + k * n_clusters
@@ -36,6 +37,8 @@ struct TailWork {
   int t_first;                // first left-over item this pair has a share of
   TailSeg seg[kMaxTailSeg];
   int g[kMaxTail];            // step groups of each left-over item
+  int sp[kMaxBundles + 1];    // the layout's per-bundle step offsets (and group offsets, t-grouped variant): the three
+  int gp[kMaxBundles + 1];    // roles read them once per item, and two dependent global loads per item showed on short items
 };
 struct Work { int item, g0, g1, part, nparts; };
 
@@ -130,6 +133,11 @@ conv3d_umma_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_c
   // this CTA holds its TMEM columns (a successor CTA that shared the SM and allocated first could otherwise
   // starve this one while waiting for it); global memory from here on.
   pdl_launch();
+  if (!kDense)
+    for (int i = threadIdx.x; i <= a.n_bundles; i += blockDim.x) {
+      tw->sp[i] = __ldg(a.step_ptr + i);
+      if (kTS) tw->gp[i] = __ldg(a.grp_ptr + i);
+    }
   // The step counts belong to the packed layout, which only host uploads write, never a kernel: the work list
   // is built before the wait on the predecessor grid (the caller's tensors, bias included, are read after it).
   // This pair's work list.  The tail split's segment table is built by one thread per left-over item (a lone
@@ -210,8 +218,8 @@ conv3d_umma_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_c
       for (int wi = 0; kTS && wi < n_work && ok; ++wi) {
         const Work wk = get_work(tw, wi, cluster_id, n_clusters);
         const PairItem c = decode_pair_item(a, wk.item, pairs_per_bundle, n_mtiles, rank);
-        const int gbase = kDense ? 0 : a.grp_ptr[c.bundle];
-        const int ngrp = kDense ? ts_groups_dense : a.grp_ptr[c.bundle + 1] - gbase;
+        const int gbase = kDense ? 0 : tw->gp[c.bundle];
+        const int ngrp = kDense ? ts_groups_dense : tw->gp[c.bundle + 1] - gbase;
         const int g1 = wk.g1 < ngrp ? wk.g1 : ngrp;
         const int wq = c.w0 * a.g.sw - a.g.pw, hq = c.h0 * a.g.sh - a.g.ph, tq = c.t0 * a.g.st - a.g.pt;
         // computed steps: (kh, kw, chunk) of the share's first group by division once, then carried (three divisions
@@ -250,8 +258,8 @@ conv3d_umma_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_c
       for (int wi = 0; !kTS && wi < n_work && ok; ++wi) {
         const Work wk = get_work(tw, wi, cluster_id, n_clusters);
         const PairItem c = decode_pair_item(a, wk.item, pairs_per_bundle, n_mtiles, rank);
-        const int s_begin = kDense ? c.bundle * a.steps_dense : a.step_ptr[c.bundle];
-        const int nsteps = kDense ? a.steps_dense : a.step_ptr[c.bundle + 1] - s_begin;
+        const int s_begin = kDense ? c.bundle * a.steps_dense : tw->sp[c.bundle];
+        const int nsteps = kDense ? a.steps_dense : tw->sp[c.bundle + 1] - s_begin;
         const int i0 = wk.g0 * kCps, i1 = wk.g1 * kCps < nsteps ? wk.g1 * kCps : nsteps;
         const int wq = c.w0 * a.g.sw - a.g.pw, hq = c.h0 * a.g.sh - a.g.ph, tq = c.t0 * a.g.st - a.g.pt;
         int kt = 0, kh = 0, kw = 0, ch = 0;
@@ -309,8 +317,8 @@ conv3d_umma_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_c
       for (int wi = 0; kTS && wi < n_work && ok; ++wi, ++j) {
         const Work wk = get_work(tw, wi, cluster_id, n_clusters);
         const int bundle = wk.item / pairs_per_bundle;
-        const int gbase = kDense ? 0 : a.grp_ptr[bundle];
-        const int ngrp = kDense ? ts_groups_dense : a.grp_ptr[bundle + 1] - gbase;
+        const int gbase = kDense ? 0 : tw->gp[bundle];
+        const int ngrp = kDense ? ts_groups_dense : tw->gp[bundle + 1] - gbase;
         const int g1 = wk.g1 < ngrp ? wk.g1 : ngrp;
         const uint32_t buf = j & 1u;
         if (!mbar_wait(smem_u32(&bars->tmem_empty[buf]), ((j >> 1) & 1u) ^ 1u, bars, err, 22)) break;
@@ -344,7 +352,7 @@ conv3d_umma_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_c
       for (int wi = 0; !kTS && wi < n_work && ok; ++wi, ++j) {
         const Work wk = get_work(tw, wi, cluster_id, n_clusters);
         const int bundle = wk.item / pairs_per_bundle;
-        const int nsteps = kDense ? a.steps_dense : a.step_ptr[bundle + 1] - a.step_ptr[bundle];
+        const int nsteps = kDense ? a.steps_dense : tw->sp[bundle + 1] - tw->sp[bundle];
         const int i0 = wk.g0 * kCps, i1 = wk.g1 * kCps < nsteps ? wk.g1 * kCps : nsteps;
         const uint32_t buf = j & 1u;
         if (!mbar_wait(smem_u32(&bars->tmem_empty[buf]), ((j >> 1) & 1u) ^ 1u, bars, err, 22)) break;
@@ -409,7 +417,7 @@ conv3d_umma_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_c
     for (int wi = 0; wi < n_work; ++wi, ++j) {
       const Work wk = get_work(tw, wi, cluster_id, n_clusters);
       const PairItem c = decode_pair_item(a, wk.item, pairs_per_bundle, n_mtiles, rank);
-      const int nsteps = kDense ? a.steps_dense : a.step_ptr[c.bundle + 1] - a.step_ptr[c.bundle];
+      const int nsteps = kDense ? a.steps_dense : tw->sp[c.bundle + 1] - tw->sp[c.bundle];
       const uint32_t buf = j & 1u;
       if (!mbar_wait(smem_u32(&bars->tmem_full[buf]), (j >> 1) & 1u, bars, err, 24)) break;
       tc_fence_after();
@@ -421,7 +429,7 @@ conv3d_umma_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_c
       // the second issuer's accumulator holds something once the item (or share) has two step groups
       int units_here;                                      // step groups (of kCps steps, or t-groups) of this item or share
       if (kTS) {
-        const int ngrp = kDense ? ts_groups_dense : a.grp_ptr[c.bundle + 1] - a.grp_ptr[c.bundle];
+        const int ngrp = kDense ? ts_groups_dense : tw->gp[c.bundle + 1] - tw->gp[c.bundle];
         units_here = (wk.g1 < ngrp ? wk.g1 : ngrp) - wk.g0;
       } else {
         units_here = ((wk.g1 * kCps < nsteps ? wk.g1 * kCps : nsteps) - wk.g0 * kCps + kCps - 1) / kCps;
@@ -626,7 +634,8 @@ cudaError_t launch_pair_t(const UmmaArgs& a, const CUtensorMap& xm, const CUtens
 }  // namespace
 
 bool umma_pair_supported(int n_tile, int n_bundles) {
-  return n_tile % 16 == 0 && n_tile <= 256 && pick_stages_pair(n_tile) >= 2 && pair_smem_bytes(n_tile, n_bundles) <= 227 * 1024;
+  return n_tile % 16 == 0 && n_tile <= 256 && n_bundles <= kMaxBundles && pick_stages_pair(n_tile) >= 2 &&
+         pair_smem_bytes(n_tile, n_bundles) <= 227 * 1024;
 }
 
 // Tail split: decides how many CTA pairs share the items that do not fill a last round (0 = no split)
