@@ -10,9 +10,10 @@
 //
 // Synchronisation: both producers wait on their own `empty[s]` (released for both CTAs by one
 // multicast commit), both send their loads' completion bytes to the leader's `full[s]`; the
-// leader's MMA thread waits there, issues, and commits to `empty[s]` / `tmem_full[b]` of both CTAs;
-// the epilogue warps of both CTAs release the accumulator on the leader's `tmem_empty[b]`.
-// All waits are bounded as in the single-CTA kernel.
+// leader's MMA thread waits there, issues, and commits to `empty[s]` / `tmem_full[b]` of both CTAs
+// (bundles up to 128 wide: two MMA threads, which take the stages by parity and accumulate into
+// two accumulators that the epilogue adds); the epilogue warps of both CTAs release the
+// accumulator on the leader's `tmem_empty[b]`.  All waits are bounded as in the single-CTA kernel.
 #include "kernels.h"
 #include "umma_common.cuh"
 #include "umma_pair.cuh"
