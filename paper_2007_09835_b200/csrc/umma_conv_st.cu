@@ -337,43 +337,34 @@ conv3d_umma_st_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_con
         tc_fence_after();
         const int qb = cur.g - cur.g0 - cur.ta;            // running number of output frame o is qb + o
         const uint32_t mid_tmem = tmem_base + (j & 1u) * uint32_t(a.n1);
-        // the taps this job issues, oldest output frame first; a frame that starts here needs its accumulator
-        // drained of the frame that used it before.  All waiting is done before the first MMA is issued.
-        bool live[3];
-        uint32_t dd[3], acc0[3];
-#pragma unroll
-        for (int dt = 0; dt < 3; ++dt) {
-          const int o = cur.p + 1 - dt;
-          live[dt] = o >= cur.ta && o < cur.tb;
-          const uint32_t q = uint32_t(qb + o), slot = q % kStOuts;
-          const bool first = cur.p == (o > 0 ? o - 1 : 0);
-          dd[dt] = out_tmem + slot * uint32_t(a.n2);
-          acc0[dt] = first ? 0u : 1u;
-          if (live[dt] && first && ok)
-            ok = mbar_wait(smem_u32(&sb->out_empty[slot]), ((q / kStOuts) & 1u) ^ 1u, bars, err, 46);
-        }
-        if (!ok) break;
-        tc_fence_after();
+        // The taps this job issues, oldest output frame first.  The last one, out(p + 1) += mid(p) Wt[0], starts a
+        // frame and needs its accumulator drained of out(p - 2), which the tap before this job completed: the wait
+        // for that comes just before the tap, so that the output warps have the time of the other two taps (this
+        // warp issues nothing else, so waiting in the middle holds up no other MMA).
 #pragma unroll
         for (int dt = 2; dt >= 0; --dt) {
-          if (!live[dt]) continue;
+          const int o = cur.p + 1 - dt;
+          if (!(o >= cur.ta && o < cur.tb)) continue;
+          const uint32_t q = uint32_t(qb + o), slot = q % kStOuts;
+          const bool first = cur.p == (o > 0 ? o - 1 : 0);
+          if (first) {
+            if (!mbar_wait(smem_u32(&sb->out_empty[slot]), ((q / kStOuts) & 1u) ^ 1u, bars, err, 46)) { ok = false; break; }
+            tc_fence_after();
+          }
           const int m0 = a.mma2_ptr[dt], m1 = a.mma2_ptr[dt + 1];
-          const uint32_t d = dd[dt];
-          uint32_t acc = acc0[dt];
+          const uint32_t d = out_tmem + slot * uint32_t(a.n2);
+          uint32_t acc = first ? 0u : 1u;
 #pragma unroll 2
           for (int m = m0; m < m1; ++m) {
             const uint64_t bdesc = b_hi | uint64_t(w2_16 + a.tab2[2 * m + 1]);
             if (elected) umma_bf16_pair_ta(d, mid_tmem + a.tab2[2 * m], bdesc, idesc2, acc);
             acc = 1u;
           }
+          // a frame is complete with the tap of the frame after it (the last frame of a clip with its own centre tap):
+          // its output warps are told at once, not after the remaining taps of this job
+          if (elected && (dt == 2 || (dt == 1 && cur.p == T - 1))) umma_commit_pair(smem_u32(&sb->out_full[slot]));
         }
         if (!ok) break;
-        if (elected) {
-          const int o1 = cur.p - 1;
-          if (o1 >= cur.ta && o1 < cur.tb) umma_commit_pair(smem_u32(&sb->out_full[uint32_t(qb + o1) % kStOuts]));
-          if (cur.p == T - 1 && cur.p >= cur.ta && cur.p < cur.tb)
-            umma_commit_pair(smem_u32(&sb->out_full[uint32_t(qb + cur.p) % kStOuts]));
-        }
         if (elected) umma_commit_pair(smem_u32(&sb->t_done[j & 1u]));
         st_next(cur);
         ++j;
