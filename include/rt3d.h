@@ -254,7 +254,7 @@ rt3d_status rt3d_conv2plus1d_fused(const rt3d_tensor* x, const rt3d_packed* w_s,
  * memory budget, or a host thread that must never block on the allocator's device-wide
  * synchronisation.  For them this entry point runs the same tensor-core convolution, including its
  * K-split variant whose fp32 partial tiles need scratch memory, without any allocation: the scratch
- * is a fixed array inside the library (16 MiB of partial tiles plus 2 KiB of counters, resident on
+ * is a fixed array inside the library (16 MiB of partial tiles plus 4 KiB of counters, resident on
  * every GPU that loads the library until the process exits).
  *   - Same arguments, layouts and alignment rules as rt3d_conv3d_sparse (device x, y, bias); bf16 only.
  *   - Everything that does need an allocation must exist already: call rt3d_packed_prepare(w) on this

@@ -814,7 +814,7 @@ rt3d_status conv_impl(const rt3d_tensor* x, const rt3d_packed* wc, const float* 
     // split-K workspace of this handle on this device: partial tiles + per-warp arrival counters
     const long long tiles = m_tiles * L->n_bundles;
     if ((s = ensure_splitk(w, blob, size_t(tiles) * a.n_splits * kTileM * L->n_tile * sizeof(float),
-                           size_t(tiles) * 4 * sizeof(int32_t))) != RT3D_OK) return s;
+                           size_t(tiles) * 8 * sizeof(int32_t))) != RT3D_OK) return s;
     a.scratch = blob->splitk; a.counters = blob->splitk_cnt;
   }
   if (use_ts) {
@@ -926,7 +926,7 @@ rt3d_status conv2plus1d_impl(const rt3d_tensor* x, const rt3d_packed* wsc, const
 // the address is looked up per device with cudaGetSymbolAddress below.
 #define RT3D_NOALLOC_PARTIAL_TILES 128                                   /* 128 x 256 fp32 each */
 #define RT3D_NOALLOC_PARTIAL_BYTES (RT3D_NOALLOC_PARTIAL_TILES * 128 * 256 * 4)   /* 16 MiB */
-#define RT3D_NOALLOC_COUNTER_BYTES (RT3D_NOALLOC_PARTIAL_TILES * 4 * 4)  /* 4 counters per output tile */
+#define RT3D_NOALLOC_COUNTER_BYTES (RT3D_NOALLOC_PARTIAL_TILES * 8 * 4)  /* 8 counters (epilogue warps) per output tile */
 static __device__ __align__(256) unsigned char g_noalloc_ws[RT3D_NOALLOC_PARTIAL_BYTES + RT3D_NOALLOC_COUNTER_BYTES];
 
 namespace {
@@ -1302,12 +1302,12 @@ rt3d_status rt3d_conv3d_sparse_noalloc(const rt3d_tensor* x, const rt3d_packed* 
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (a.n_splits > 1) {
     const long long partial_bytes = tiles * a.n_splits * kTileM * L->n_tile * 4LL;
-    if (partial_bytes > RT3D_NOALLOC_PARTIAL_BYTES || tiles * 16 > RT3D_NOALLOC_COUNTER_BYTES)
+    if (partial_bytes > RT3D_NOALLOC_PARTIAL_BYTES || tiles * 32 > RT3D_NOALLOC_COUNTER_BYTES)
       return RT3D_ERR_WORKSPACE;
     a.scratch = reinterpret_cast<float*>(ws);
     a.counters = reinterpret_cast<int32_t*>(ws + RT3D_NOALLOC_PARTIAL_BYTES);
     // the counters must start at zero; the workspace keeps whatever the last call left behind
-    if (cudaMemsetAsync(a.counters, 0, size_t(tiles) * 16, st) != cudaSuccess) return RT3D_ERR_CUDA;
+    if (cudaMemsetAsync(a.counters, 0, size_t(tiles) * 32, st) != cudaSuccess) return RT3D_ERR_CUDA;
   }
   CUtensorMap xmap;
   if ((s = encode_xmap(x, g, a.box, &xmap)) != RT3D_OK) return s;

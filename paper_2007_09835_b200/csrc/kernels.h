@@ -54,7 +54,7 @@ struct UmmaArgs {
   int sbw, sbh;                             // extents along w, h of the block of 32 voxels an epilogue warp owns
   int n_splits;                             // K splits per output tile (1 = none)
   float* scratch;                           // device, split-K partial tiles [tile][split][128][n_tile] (n_splits > 1)
-  int32_t* counters;                        // device, [tiles * 4] arrival counters, zero between launches
+  int32_t* counters;                        // device, [tiles * 8] arrival counters (one per epilogue warp), zero between launches
   int tail_workers;                         // CTA-pair kernel: pairs sharing the left-over items of the last round (0 = off)
   float* tail_scratch;                      // device, [tail_workers][2 shares][2 CTAs][n_tile][128] fp32 partial tiles
   int32_t* tail_flags;                      // device, [tail_workers][2][2][4 warps] "partial written" flags, zero between launches

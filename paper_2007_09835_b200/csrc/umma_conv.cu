@@ -90,9 +90,10 @@ __device__ __forceinline__ void reduce_partial_cols(const float* part0, size_t s
 
 __device__ __forceinline__ void reduce_partial_row(const float* part0, size_t split_stride, int n_splits, int n_cols,
                                                    bool in_range, const float* bias_s, int relu, __nv_bfloat16* dst,
-                                                   int m_base, int M, const __nv_bfloat16* res_row, int res_left) {
+                                                   int m_base, int M, const __nv_bfloat16* res_row, int res_left,
+                                                   int col0 = 0, int col_step = 32) {
   if (!in_range) return;
-  for (int col = 0; col < n_cols; col += 32) {
+  for (int col = col0; col < n_cols; col += col_step) {
     const int m0 = m_base + col;
     if (m0 >= M) break;
     const float* p = part0 + size_t(col) * 128;
@@ -131,7 +132,8 @@ conv3d_umma_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_consta
   const int n_mtiles = a.tiles_n * a.tiles_t * a.tiles_h * a.tiles_w;
   const int n_items = n_mtiles * a.n_bundles * a.n_splits;
   const int box_rows = a.box.bn * a.box.bt * a.box.bh * a.box.bw;
-  const bool two_sets = a.n_splits == 1 && a.pool_t * a.pool_h * a.pool_w == 1;   // both epilogue warp sets work
+  const bool two_sets = a.n_splits == 1 && a.pool_t * a.pool_h * a.pool_w == 1;   // both epilogue warp sets work on a plain tile
+  const bool split_sets = a.n_splits > 1;      // and on a K split: each takes every other 32-column piece of the share and of the sum
 
   if (threadIdx.x == 32) {                     // descriptor fetches overlap the rest of the set-up
     tma_prefetch_map(&xmap);
@@ -145,7 +147,7 @@ conv3d_umma_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_consta
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(smem_u32(&bars->tmem_full[b]), 1);
-      mbar_init(smem_u32(&bars->tmem_empty[b]), two_sets ? 8 : 4);
+      mbar_init(smem_u32(&bars->tmem_empty[b]), (two_sets || split_sets) ? 8 : 4);
     }
     bars->abort_flag = 0;
     bars->wait_limit = a.wait_cycles > 0 ? a.wait_cycles : kWaitCycles;
@@ -296,7 +298,7 @@ conv3d_umma_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_consta
         else mbar_arrive(smem_u32(&bars->tmem_full[buf]));
       }
     }
-  } else if (warp < 6 || two_sets) {
+  } else if (warp < 6 || two_sets || split_sets) {
     // ------------------------------------------------------------------ epilogue (warps 2..5, and 6..9 on plain calls)
     const int quad = warp & 3;                 // TMEM lane quadrant this warp may read
     const int half = (warp - 2) >> 2;          // second set: odd pieces, direct stores
@@ -372,7 +374,7 @@ conv3d_umma_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_consta
         if (lane == 0) mbar_arrive(smem_u32(&bars->tmem_empty[buf]));
       } else {
         float* tile_part = a.scratch + size_t(c.tile_id) * a.n_splits * part_tile;
-        store_partial_row(taddr, a.n_tile, nsteps > 0, tile_part + size_t(c.split) * part_tile + row);
+        store_partial_row(taddr, a.n_tile, nsteps > 0, tile_part + size_t(c.split) * part_tile + row, half * 32, 64);
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&bars->tmem_empty[buf]));    // accumulator consumed: MMAs may go on
@@ -381,14 +383,14 @@ conv3d_umma_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_consta
         __threadfence();
         __syncwarp();
         int last = 0;
-        if (lane == 0) last = atomicAdd(a.counters + c.tile_id * 4 + quad, 1) == a.n_splits - 1;
+        if (lane == 0) last = atomicAdd(a.counters + c.tile_id * 8 + half * 4 + quad, 1) == a.n_splits - 1;
         last = __shfl_sync(0xffffffffu, last, 0);
         if (last) {
           __threadfence();
           reduce_partial_row(tile_part + row, part_tile, a.n_splits, a.n_tile, in_range, bias_s,
-                             a.g.relu, dst, m_base, a.g.M, res, res_left);
+                             a.g.relu, dst, m_base, a.g.M, res, res_left, half * 32, 64);
           __syncwarp();
-          if (lane == 0) a.counters[c.tile_id * 4 + quad] = 0;              // ready for the next launch
+          if (lane == 0) a.counters[c.tile_id * 8 + half * 4 + quad] = 0;   // ready for the next launch
         }
       }
     }
