@@ -66,7 +66,7 @@ constexpr int kTsTable = 2048;
 // tiles of the up to Kt steps (kt = 0 .. Kt-1 at one (kh, kw, chunk)) that read it, each through a descriptor that
 // starts kt frames into the tile: a third as many input bytes per step cross from L2, so more steps are in flight
 // in the same shared memory (a 64 -> 128 channel 3x3x3 layer was bound by that, at 387 clocks per step against 256).
-template <bool kDense, int kCps, bool kTS>
+template <bool kDense, int kCps, bool kTS, bool kDual>
 __global__ void __launch_bounds__(kThreadsPair, 1)
 conv3d_umma_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CUtensorMap wmap_half,
                         const __grid_constant__ CUtensorMap ymap, const UmmaArgs a, const int stages, const int tmem_cols) {
@@ -99,10 +99,9 @@ conv3d_umma_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_c
   const int cluster_id = blockIdx.x >> 1, n_clusters = gridDim.x >> 1;
   const int box_rows = a.box.bn * a.box.bt * a.box.bh * a.box.bw;
   constexpr int epi_sets = 2;
-  // Narrow bundles (kCps == 2, N <= 128): one thread cannot issue MMAs and run the barrier hand-shakes as fast as
+  // Narrow bundles (kDual, N <= 128): one thread cannot issue MMAs and run the barrier hand-shakes as fast as
   // the tensor pipe executes them, so two threads issue alternate step groups, each into its own accumulator
   // (2 buffers x 2 x N <= 512 columns); the epilogue adds the two.  Fixed order, so results stay repeatable.
-  constexpr bool kDual = kCps == 2;
   constexpr int kIss = kDual ? 2 : 1;
 
   if (threadIdx.x == 0) {
@@ -529,13 +528,15 @@ conv3d_umma_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_c
 
 // Two K steps share one barrier hand-shake when a step is short (narrow bundles: the issuing thread, not
 // the tensor pipe, is the limit there); wide bundles keep one step per stage (deeper pipeline).
-int pick_cps(int n_tile) { return n_tile <= 128 ? 2 : 1; }
+int pick_cps(int n_tile) { return n_tile <= 160 ? 2 : 1; }
+// Two issuing threads (two accumulators per buffer: 2 x 2 x N <= 512 TMEM columns).
+bool pick_dual(int n_tile) { return n_tile <= 128; }
 
 int pick_stages_pair(int n_tile) {
   const size_t stage = pick_cps(n_tile) * (kABytes + size_t(n_tile / 2) * 128);
   int s = int(kSmemBudget / stage);
   if (s > kMaxStages) s = kMaxStages;
-  if (pick_cps(n_tile) == 2) s &= ~1;           // two issuing threads take the stages by parity
+  if (pick_dual(n_tile)) s &= ~1;               // two issuing threads take the stages by parity
   return s;
 }
 
@@ -554,7 +555,7 @@ int pick_stages_pair_ts(const UmmaArgs& a) {
                        size_t(a.n_tile) * a.n_bundles * 4 + (3 * size_t(a.ts_table) + 16) * 4;
   int s = int((size_t(227) * 1024 - fixed) / ts_stage_bytes(a));
   if (s > kMaxStages) s = kMaxStages;
-  if (pick_cps(a.n_tile) == 2) s &= ~1;         // two issuing threads take the stages by parity
+  if (pick_dual(a.n_tile)) s &= ~1;             // two issuing threads take the stages by parity
   return s;
 }
 size_t pair_smem_bytes_ts(const UmmaArgs& a) {
@@ -562,13 +563,13 @@ size_t pair_smem_bytes_ts(const UmmaArgs& a) {
          16 + size_t(a.n_tile) * a.n_bundles * 4 + (3 * size_t(a.ts_table) + 16) * 4;
 }
 
-template <bool kDense, int kCps, bool kTS>
+template <bool kDense, int kCps, bool kTS, bool kDual>
 cudaError_t prepare_pair_t() {
   static bool attr_done[kMaxDevices] = {};             // the attribute is per device
   const int dev = current_device_index();
   if (dev < 0) return cudaErrorInvalidDevice;
   if (!attr_done[dev]) {
-    cudaError_t e = cudaFuncSetAttribute(conv3d_umma_pair_kernel<kDense, kCps, kTS>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    cudaError_t e = cudaFuncSetAttribute(conv3d_umma_pair_kernel<kDense, kCps, kTS, kDual>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
     if (e != cudaSuccess) return e;
     attr_done[dev] = true;
   }
@@ -588,48 +589,63 @@ void pair_launch_config(cudaLaunchConfig_t& cfg, cudaLaunchAttribute* attr, unsi
 }
 
 // CTA pairs that can be resident at once (the persistent grid), never more than SMs / 2.
-template <bool kDense, int kCps, bool kTS>
+template <bool kDense, int kCps, bool kTS, bool kDual>
 int pair_max_clusters_t(int sm_count, size_t smem) {
   static int max_clusters_dev[kMaxDevices] = {};       // the occupancy answer is per device
   const int dev = current_device_index();
   if (dev < 0) return sm_count / 2;
   int& max_clusters = max_clusters_dev[dev];
   if (max_clusters == 0) {
-    if (prepare_pair_t<kDense, kCps, kTS>() != cudaSuccess) return sm_count / 2;
+    if (prepare_pair_t<kDense, kCps, kTS, kDual>() != cudaSuccess) return sm_count / 2;
     cudaLaunchConfig_t cfg;
     cudaLaunchAttribute attr[1];
     pair_launch_config(cfg, attr, unsigned(sm_count & ~1), smem, nullptr);
     int n = 0;
-    if (cudaOccupancyMaxActiveClusters(&n, conv3d_umma_pair_kernel<kDense, kCps, kTS>, &cfg) != cudaSuccess || n <= 0) n = sm_count / 2;
+    if (cudaOccupancyMaxActiveClusters(&n, conv3d_umma_pair_kernel<kDense, kCps, kTS, kDual>, &cfg) != cudaSuccess || n <= 0) n = sm_count / 2;
     max_clusters = n;
   }
   return max_clusters < sm_count / 2 ? max_clusters : sm_count / 2;
 }
 
+// The instantiation for a bundle width: <dense path, K steps per stage, t-grouped, two issuing threads>.
+// t-grouped: a stage is a group whatever kCps says; two issuing threads up to 128 columns.  Otherwise two steps per
+// stage up to 192 columns (one issuing thread needs about 550 clocks per hand-shake and four MMAs, more than the
+// 288-384 clocks of MMAs of a 144- to 192-wide step), with two issuing threads up to 128.
+#define RT3D_PAIR_VARIANT(DENSE, TS, N_TILE, CALL)                                             \
+  do {                                                                                         \
+    if (TS) {                                                                                  \
+      if (pick_dual(N_TILE)) { if (DENSE) return CALL(true, 2, true, true); return CALL(false, 2, true, true); }       \
+      if (DENSE) return CALL(true, 1, true, false); return CALL(false, 1, true, false);         \
+    }                                                                                          \
+    if (pick_dual(N_TILE)) { if (DENSE) return CALL(true, 2, false, true); return CALL(false, 2, false, true); }       \
+    if (pick_cps(N_TILE) == 2) { if (DENSE) return CALL(true, 2, false, false); return CALL(false, 2, false, false); } \
+    if (DENSE) return CALL(true, 1, false, false); return CALL(false, 1, false, false);         \
+  } while (0)
+
 int pair_max_clusters(int n_tile, int n_bundles, bool dense, int sm_count) {
   const size_t smem = pair_smem_bytes(n_tile, n_bundles);
-  if (pick_cps(n_tile) == 2)
-    return dense ? pair_max_clusters_t<true, 2, false>(sm_count, smem) : pair_max_clusters_t<false, 2, false>(sm_count, smem);
-  return dense ? pair_max_clusters_t<true, 1, false>(sm_count, smem) : pair_max_clusters_t<false, 1, false>(sm_count, smem);
+#define RT3D_CALL(D, C, T, U) pair_max_clusters_t<D, C, T, U>(sm_count, smem)
+  RT3D_PAIR_VARIANT(dense, false, n_tile, RT3D_CALL);
+#undef RT3D_CALL
 }
 int pair_max_clusters_ts(const UmmaArgs& a, int sm_count) {
   const size_t smem = pair_smem_bytes_ts(a);
-  if (pick_cps(a.n_tile) == 2)
-    return a.dense ? pair_max_clusters_t<true, 2, true>(sm_count, smem) : pair_max_clusters_t<false, 2, true>(sm_count, smem);
-  return a.dense ? pair_max_clusters_t<true, 1, true>(sm_count, smem) : pair_max_clusters_t<false, 1, true>(sm_count, smem);
+#define RT3D_CALL(D, C, T, U) pair_max_clusters_t<D, C, T, U>(sm_count, smem)
+  RT3D_PAIR_VARIANT(a.dense != 0, true, a.n_tile, RT3D_CALL);
+#undef RT3D_CALL
 }
 
-template <bool kDense, int kCps, bool kTS>
+template <bool kDense, int kCps, bool kTS, bool kDual>
 cudaError_t launch_pair_t(const UmmaArgs& a, const CUtensorMap& xm, const CUtensorMap& wm, const CUtensorMap& ym,
                           int sm_count, int stages,
                           int cols, size_t smem, long long n_items, cudaStream_t stream) {
-  cudaError_t e = prepare_pair_t<kDense, kCps, kTS>();
+  cudaError_t e = prepare_pair_t<kDense, kCps, kTS, kDual>();
   if (e != cudaSuccess) return e;
-  long long clusters = pair_max_clusters_t<kDense, kCps, kTS>(sm_count, smem);
+  long long clusters = pair_max_clusters_t<kDense, kCps, kTS, kDual>(sm_count, smem);
   const long long want = n_items > a.tail_workers ? n_items : a.tail_workers;
   if (clusters > want) clusters = want;
   LaunchSetup ls(dim3(unsigned(2 * clusters)), dim3(kThreadsPair), smem, stream, 2);
-  return cudaLaunchKernelEx(&ls.cfg, conv3d_umma_pair_kernel<kDense, kCps, kTS>, xm, wm, ym, a, stages, cols);
+  return cudaLaunchKernelEx(&ls.cfg, conv3d_umma_pair_kernel<kDense, kCps, kTS, kDual>, xm, wm, ym, a, stages, cols);
 }
 
 }  // namespace
@@ -713,7 +729,7 @@ cudaError_t launch_conv_umma_pair(const UmmaArgs& a, const void* xmap, const voi
   const size_t smem = a.ts ? pair_smem_bytes_ts(a) : pair_smem_bytes(a.n_tile, a.n_bundles);
   if (a.ts && (smem > 227 * 1024 || stages < 2)) return cudaErrorInvalidValue;
   int cols = 32;
-  while (cols < 2 * a.n_tile * (pick_cps(a.n_tile) == 2 ? 2 : 1)) cols *= 2;     // two issuing threads: two accumulators
+  while (cols < 2 * a.n_tile * (pick_dual(a.n_tile) ? 2 : 1)) cols *= 2;     // two issuing threads: two accumulators
   if (cols > 512) return cudaErrorInvalidValue;
   const long long n_mtiles = (long long)a.tiles_n * a.tiles_t * a.tiles_h * a.tiles_w;
   const long long n_items = ((n_mtiles + 1) / 2) * a.n_bundles;
@@ -723,17 +739,9 @@ cudaError_t launch_conv_umma_pair(const UmmaArgs& a, const void* xmap, const voi
   memcpy(&xm, xmap, sizeof(CUtensorMap));
   memcpy(&wm, wmap_half, sizeof(CUtensorMap));
   memcpy(&ym, ymap ? ymap : xmap, sizeof(CUtensorMap));
-  if (a.ts && pick_cps(a.n_tile) == 2)
-    return a.dense ? launch_pair_t<true, 2, true>(a, xm, wm, ym, sm_count, stages, cols, smem, n_items, stream)
-                   : launch_pair_t<false, 2, true>(a, xm, wm, ym, sm_count, stages, cols, smem, n_items, stream);
-  if (a.ts)
-    return a.dense ? launch_pair_t<true, 1, true>(a, xm, wm, ym, sm_count, stages, cols, smem, n_items, stream)
-                   : launch_pair_t<false, 1, true>(a, xm, wm, ym, sm_count, stages, cols, smem, n_items, stream);
-  if (pick_cps(a.n_tile) == 2)
-    return a.dense ? launch_pair_t<true, 2, false>(a, xm, wm, ym, sm_count, stages, cols, smem, n_items, stream)
-                   : launch_pair_t<false, 2, false>(a, xm, wm, ym, sm_count, stages, cols, smem, n_items, stream);
-  return a.dense ? launch_pair_t<true, 1, false>(a, xm, wm, ym, sm_count, stages, cols, smem, n_items, stream)
-                 : launch_pair_t<false, 1, false>(a, xm, wm, ym, sm_count, stages, cols, smem, n_items, stream);
+#define RT3D_CALL(D, C, T, U) launch_pair_t<D, C, T, U>(a, xm, wm, ym, sm_count, stages, cols, smem, n_items, stream)
+  RT3D_PAIR_VARIANT(a.dense != 0, a.ts != 0, a.n_tile, RT3D_CALL);
+#undef RT3D_CALL
 }
 
 }  // namespace rt3d
