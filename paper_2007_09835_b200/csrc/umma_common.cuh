@@ -255,9 +255,10 @@ __device__ __forceinline__ void epilogue_cols(const uint32_t* v, const float* bi
   }
 }
 
-// Partial sums of the same tile left in scratch by other CTAs (column-major [column][128 rows] floats, pointers
-// at this thread's row), added to the 32 (or 16) accumulator columns from `col` on in a fixed order: extra_first,
+// Partial sums of the same tile left in scratch by other CTAs (layout of store_partial_row, pointers at this
+// thread's row), added to the 32 (or 16) accumulator columns from `col` on in a fixed order: extra_first,
 // then extra + p * extra_stride.  Two partial tiles' loads are in flight at a time.
+constexpr int kPartRow = 4;   // floats between consecutive rows of a partial tile (see store_partial_row)
 __device__ __forceinline__ void add_partials(uint32_t (&v)[32], bool wide, int col, const float* extra_first,
                                              const float* extra, size_t extra_stride, int n_extra) {
   const float* e0 = extra_first + size_t(col) * 128;
@@ -265,15 +266,21 @@ __device__ __forceinline__ void add_partials(uint32_t (&v)[32], bool wide, int c
     const float* ea = p < 0 ? e0 : extra + size_t(p) * extra_stride + size_t(col) * 128;
     const bool two = p + 1 < n_extra;
     const float* eb = two ? extra + size_t(p + 1) * extra_stride + size_t(col) * 128 : ea;
-    float t0[32], t1[32];
+    float4 t0[8], t1[8];
+    const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-    for (int q = 0; q < 32; ++q) {
-      const bool live = wide || q < 16;
-      t0[q] = live ? __ldcg(ea + size_t(q) * 128) : 0.f;
-      t1[q] = (live && two) ? __ldcg(eb + size_t(q) * 128) : 0.f;
+    for (int q = 0; q < 8; ++q) {
+      const bool live = wide || q < 4;
+      t0[q] = live ? __ldcg(reinterpret_cast<const float4*>(ea + size_t(q) * 512)) : zero;
+      t1[q] = (live && two) ? __ldcg(reinterpret_cast<const float4*>(eb + size_t(q) * 512)) : zero;
     }
 #pragma unroll
-    for (int q = 0; q < 32; ++q) v[q] = __float_as_uint((__uint_as_float(v[q]) + t0[q]) + t1[q]);
+    for (int q = 0; q < 8; ++q) {
+      v[4 * q] = __float_as_uint((__uint_as_float(v[4 * q]) + t0[q].x) + t1[q].x);
+      v[4 * q + 1] = __float_as_uint((__uint_as_float(v[4 * q + 1]) + t0[q].y) + t1[q].y);
+      v[4 * q + 2] = __float_as_uint((__uint_as_float(v[4 * q + 2]) + t0[q].z) + t1[q].z);
+      v[4 * q + 3] = __float_as_uint((__uint_as_float(v[4 * q + 3]) + t0[q].w) + t1[q].w);
+    }
   }
 }
 
@@ -497,9 +504,12 @@ __device__ __forceinline__ void epilogue_row_tma(uint32_t taddr, int n_cols, boo
   }
 }
 
-// Split-K partial tiles are stored column-major, [column][128 rows] floats, so that the 32 lanes of a
-// warp (32 consecutive rows) always touch 128 contiguous bytes.
-// Raw fp32 accumulator row -> scratch; `dst` already points at this thread's row of column 0.
+// Split-K partial tiles are stored as [column / 4][128 rows][4 columns] floats: a thread moves four columns of
+// its row with one 16-byte access, and the 32 lanes of a warp (32 consecutive rows) touch 512 contiguous bytes
+// (a quarter of the memory instructions of a [column][row] layout with 4-byte accesses; a row-major tile with
+// 16-byte accesses touches 32 lines per instruction and was far slower).  kPartRow floats from row to row.
+// Raw fp32 accumulator row -> scratch; `dst` already points at this thread's row (row * kPartRow) of column 0;
+// column c of that row is at dst[(c / 4) * 512 + c % 4], so a piece starting at column `col` begins at col * 128.
 __device__ __forceinline__ void store_partial_row(uint32_t taddr, int n_cols, bool has_acc, float* dst, int col0 = 0,
                                                   int col_step = 32, uint32_t acc2_off = 0) {
   for (int col = col0; col < n_cols; col += col_step) {
@@ -511,9 +521,12 @@ __device__ __forceinline__ void store_partial_row(uint32_t taddr, int n_cols, bo
 #pragma unroll
       for (int q = 0; q < 32; ++q) v[q] = 0u;
     }
+    float4* d4 = reinterpret_cast<float4*>(dst + size_t(col) * 128);
 #pragma unroll
-    for (int q = 0; q < 32; ++q)
-      if (wide || q < 16) dst[size_t(col + q) * 128] = __uint_as_float(v[q]);
+    for (int q = 0; q < 8; ++q)
+      if (wide || q < 4)
+        d4[q * 128] = make_float4(__uint_as_float(v[4 * q]), __uint_as_float(v[4 * q + 1]), __uint_as_float(v[4 * q + 2]),
+                                  __uint_as_float(v[4 * q + 3]));
   }
 }
 

@@ -69,18 +69,29 @@ __device__ __forceinline__ void reduce_partial_cols(const float* part0, size_t s
   for (int q = 0; q < NC; ++q) acc[q] = 0.f;
   int s = 0;
   for (; s + 1 < n_splits; s += 2) {
-    float t0[NC], t1[NC];
+    float4 t0[NC / 4], t1[NC / 4];
     const float* p0 = part0 + size_t(s) * split_stride;
     const float* p1 = p0 + split_stride;
 #pragma unroll
-    for (int q = 0; q < NC; ++q) { t0[q] = __ldcg(p0 + size_t(q) * 128); t1[q] = __ldcg(p1 + size_t(q) * 128); }
+    for (int q = 0; q < NC / 4; ++q) {
+      t0[q] = __ldcg(reinterpret_cast<const float4*>(p0 + size_t(q) * 512));
+      t1[q] = __ldcg(reinterpret_cast<const float4*>(p1 + size_t(q) * 512));
+    }
 #pragma unroll
-    for (int q = 0; q < NC; ++q) acc[q] = (acc[q] + t0[q]) + t1[q];
+    for (int q = 0; q < NC / 4; ++q) {
+      acc[4 * q] = (acc[4 * q] + t0[q].x) + t1[q].x;
+      acc[4 * q + 1] = (acc[4 * q + 1] + t0[q].y) + t1[q].y;
+      acc[4 * q + 2] = (acc[4 * q + 2] + t0[q].z) + t1[q].z;
+      acc[4 * q + 3] = (acc[4 * q + 3] + t0[q].w) + t1[q].w;
+    }
   }
   if (s < n_splits) {
     const float* p0 = part0 + size_t(s) * split_stride;
 #pragma unroll
-    for (int q = 0; q < NC; ++q) acc[q] += __ldcg(p0 + size_t(q) * 128);
+    for (int q = 0; q < NC / 4; ++q) {
+      const float4 t = __ldcg(reinterpret_cast<const float4*>(p0 + size_t(q) * 512));
+      acc[4 * q] += t.x; acc[4 * q + 1] += t.y; acc[4 * q + 2] += t.z; acc[4 * q + 3] += t.w;
+    }
   }
   uint32_t v[NC];
 #pragma unroll
@@ -374,7 +385,7 @@ conv3d_umma_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_consta
         if (lane == 0) mbar_arrive(smem_u32(&bars->tmem_empty[buf]));
       } else {
         float* tile_part = a.scratch + size_t(c.tile_id) * a.n_splits * part_tile;
-        store_partial_row(taddr, a.n_tile, nsteps > 0, tile_part + size_t(c.split) * part_tile + row, half * 32, 64);
+        store_partial_row(taddr, a.n_tile, nsteps > 0, tile_part + size_t(c.split) * part_tile + row * kPartRow, half * 32, 64);
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&bars->tmem_empty[buf]));    // accumulator consumed: MMAs may go on
@@ -387,7 +398,7 @@ conv3d_umma_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_consta
         last = __shfl_sync(0xffffffffu, last, 0);
         if (last) {
           __threadfence();
-          reduce_partial_row(tile_part + row, part_tile, a.n_splits, a.n_tile, in_range, bias_s,
+          reduce_partial_row(tile_part + row * kPartRow, part_tile, a.n_splits, a.n_tile, in_range, bias_s,
                              a.g.relu, dst, m_base, a.g.M, res, res_left, half * 32, 64);
           __syncwarp();
           if (lane == 0) a.counters[c.tile_id * 8 + half * 4 + quad] = 0;   // ready for the next launch

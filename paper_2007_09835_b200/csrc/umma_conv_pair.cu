@@ -445,7 +445,7 @@ conv3d_umma_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_c
         // A share of a tile another pair owns: leave the raw partial sums in scratch and raise this warp's flag.
         // It is the first segment of this pair's range.
         const int slot = cluster_id * 2 + int(rank);
-        store_partial_row(taddr, a.n_tile, true, a.tail_scratch + size_t(slot) * part_tile + row, col0, col_step, acc2);
+        store_partial_row(taddr, a.n_tile, true, a.tail_scratch + size_t(slot) * part_tile + row * kPartRow, col0, col_step, acc2);
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive_cluster(mapa_shared(smem_u32(&bars->tmem_empty[buf]), 0));
@@ -476,8 +476,8 @@ conv3d_umma_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_c
         ok = __shfl_sync(0xffffffffu, ok, 0);
         if (!ok) break;
         __threadfence();
-        const float* e_first = a.tail_scratch + size_t((cluster_id + 1) * 2 + int(rank)) * part_tile + row;
-        const float* e_more = a.tail_scratch + size_t((cluster_id + 2) * 2 + int(rank)) * part_tile + row;
+        const float* e_first = a.tail_scratch + size_t((cluster_id + 1) * 2 + int(rank)) * part_tile + row * kPartRow;
+        const float* e_more = a.tail_scratch + size_t((cluster_id + 2) * 2 + int(rank)) * part_tile + row * kPartRow;
         if (a.store_tma) {
           ts.c1 = (c.w0 + bw_0) / a.pool_w; ts.c2 = (c.h0 + bh_0) / a.pool_h; ts.c3 = (c.t0 + bt_0) / a.pool_t; ts.c4 = c.n0 + bn_0;
           epilogue_row_tma(taddr, a.n_tile, true, quad * 32 < box_rows, in_range, bias_s, a.g.relu,
