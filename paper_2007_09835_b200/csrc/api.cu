@@ -470,6 +470,9 @@ bool smallc_eligible(const DeviceState* d, rt3d_packed* w, const rt3d_tensor* x,
 rt3d_status launch_smallc(rt3d_packed* w, DeviceBlob* blob, const DeviceState* d, const SmallCLayout* L,
                           const rt3d_tensor* x, const ConvGeom& g, const float* bias, rt3d_tensor* y, cudaStream_t st,
                           const void* residual, int rcs, int pool_h, int pool_w, bool x_pad_zero) {
+  // pooled rows leave as whole 32-channel pieces through the bulk-store epilogue; a trailing 16-channel piece is
+  // written by plain per-voxel stores, which know nothing of pooling
+  if (pool_h * pool_w > 1 && L->n_pad % 32) return RT3D_ERR_UNSUPPORTED;
   DeviceBlob::SmallC* sc = nullptr;
   {
     std::lock_guard<std::mutex> lock(w->mu);

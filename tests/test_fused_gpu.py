@@ -64,6 +64,7 @@ POOL_CASES = [
     (64, 64, (3, 3, 3), (3, 5, 13, 9), (2, 2, 2)),        # odd extents: last windows are dropped
     (64, 256, (1, 3, 3), (2, 3, 16, 16), (1, 2, 2)),
     (64, 64, (3, 3, 3), (2, 6, 10, 12), (2, 1, 2)),
+    (8, 96, (3, 3, 3), (1, 5, 23, 21), (1, 2, 2)),        # small-C_in kernel, odd extents, three whole pieces
 ]
 
 
@@ -120,6 +121,15 @@ def test_fused_pool_refusals():
     y = torch.zeros((1, 2, 4, 4, 48), dtype=torch.bfloat16, device="cuda")
     with pytest.raises(rt3d.Rt3dError) as e:
         lay.fused(xd, y, pool=(2, 2, 2), algo=rt3d.ALGO_UMMA)
+    assert e.value.status == rt3d.ERR_UNSUPPORTED
+    # the same on the small-C_in kernel: 112 channels = three pieces and a half (the call used to write the half
+    # piece unpooled, at the unpooled voxel's offset: beyond the pooled tensor)
+    spec1 = synth.ConvSpec("p", 8, 112, (3, 3, 5), (1, 2, 1), (0, 1, 0), True)
+    L1 = synth.make_layer(spec1, 12, 5, 4, 4, "bernoulli", 0.3)
+    lay1 = nets.ConvLayer(spec1, L1["w"], L1["bias"], L1["mask"], 4, 4, torch.bfloat16)
+    xd1 = nets.to_device(synth.make_input(4, (1, 15, 22, 56, 8)))
+    with pytest.raises(rt3d.Rt3dError) as e:
+        lay1.fused(xd1, torch.zeros((1, 13, 5, 26, 112), dtype=torch.bfloat16, device="cuda"), pool=(1, 2, 2))
     assert e.value.status == rt3d.ERR_UNSUPPORTED
     spec2 = synth.ConvSpec("p", 64, 64, (3, 3, 3), (1, 1, 1), (1, 1, 1), True)
     L2 = synth.make_layer(spec2, 12, 4, 4, 4, "bernoulli", 0.4)
