@@ -691,6 +691,61 @@ mixed_issue_kernel(long long* out, int n0, int count0, int n1, int count1, int32
   }
 }
 
+// ------------------------------------------------------------------------------------------ M12
+// The A operand of the small-C_in kernel: no-swizzle core matrices (8 voxels x 16 bytes) that are windows of a
+// staged image whose rows are `sbo` bytes apart, the two K halves of an MMA `lbo` bytes apart (two kernel
+// locations), successive MMAs shifted by `shift` bytes (the next kernel column).  M = 128, N = 64, K = 16; B is
+// the kernel's weight image (no swizzle, K halves 1 KB apart).  Same timing scheme as M1.
+__global__ void __launch_bounds__(128, 1)
+ns_window_kernel(long long* out, int count, int issuers, uint32_t sbo, uint32_t lbo, uint32_t shift, int32_t* err) {
+  extern __shared__ unsigned char smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  const uint32_t a_smem = base, b_smem = base + kARegion;
+  Barriers* bars = reinterpret_cast<Barriers*>(smem_raw + (base - raw) + kARegion + kBRegion);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  for (uint32_t i = threadIdx.x; i < (kARegion + kBRegion) / 4; i += blockDim.x)
+    reinterpret_cast<uint32_t*>(smem_raw + (base - raw))[i] = 0x3c003c00u;
+  if (threadIdx.x == 0) {
+    for (int q = 0; q < kMaxStages; ++q) { mbar_init(smem_u32(&bars->full[q]), 1); mbar_init(smem_u32(&bars->empty[q]), 1); }
+    bars->abort_flag = 0;
+    bars->wait_limit = kWaitCycles;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 0) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&bars->tmem_base)), "r"(256u) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = bars->tmem_base;
+  if (lane == 0 && warp < issuers) {
+    const uint32_t idesc = idesc_any(0, 128, 64);
+    const uint32_t d = tmem_base + uint32_t(warp) * 64u;
+    const int mine = count / issuers;
+    const long long t0 = clock64();
+    for (int i = 0; i < mine; ++i) {
+      const uint64_t adesc = smem_desc_noswizzle(a_smem + uint32_t(warp) * 8192u + uint32_t(i & 3) * shift, lbo, sbo);
+      const uint64_t bdesc = smem_desc_noswizzle(b_smem + uint32_t(i & 3) * 2048u, 1024u, 128u);
+      mma_any<0, false, 1>(d, adesc, 0u, bdesc, idesc, i ? 1u : 0u);
+    }
+    const long long t1 = clock64();
+    umma_commit(smem_u32(&bars->full[warp]));
+    mbar_wait(smem_u32(&bars->full[warp]), 0, bars, err, 12);
+    const long long t2 = clock64();
+    out[warp * 2] = t1 - t0;
+    out[warp * 2 + 1] = t2 - t0;
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(256u) : "memory");
+  }
+}
+
 // ------------------------------------------------------------------------------------------ M3
 // kShape: 0 m16n8k16 bf16, 1 m16n8k8 bf16, 2 m16n8k8 tf32, 3 m16n8k4 tf32.  Eight independent accumulator
 // tiles per warp, operands in registers.
@@ -1076,6 +1131,28 @@ int main(int argc, char** argv) {
       cudaMemcpy(h, d_out, 16, cudaMemcpyDeviceToHost);
       printf("| %d | %d | %lld | %lld | %.0f |\n", cb[0], cb[1], h[0], h[1], cb[0] * 72.0 + cb[1] * 32.0);
     }
+  }
+
+  printf("\n## M12: the small-C_in kernel's A operand: no-swizzle windows of a staged image (M = 128, N = 64, K = 16), one CTA\n\n");
+  printf("| row pitch (SBO) | K halves apart (LBO) | shift between MMAs | issuers | done clk/MMA |\n|---|---|---|---|---|\n");
+  {
+    const size_t smem = 1024 + kARegion + kBRegion + sizeof(Barriers) + 64;
+    cudaFuncSetAttribute(ns_window_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
+    const uint32_t cases[][3] = {{128, 2048, 128}, {128, 16, 16}, {160, 16, 16}, {160, 160, 16}, {160, 2720, 16}, {160, 16, 0},
+                                 {256, 16, 16}, {256, 256, 32}, {176, 16, 16}};
+    for (const auto& c : cases)
+      for (int issuers = 1; issuers <= 3; ++issuers) {
+        long long h[6] = {0, 0, 0, 0, 0, 0};
+        const int cnt = 240;
+        for (int rep = 0; rep < 2; ++rep) {
+          ns_window_kernel<<<1, 128, smem>>>(d_out, cnt, issuers, c[0], c[1], c[2], d_err);
+          if (!sync_ok("ns_window")) return 1;
+        }
+        cudaMemcpy(h, d_out, 48, cudaMemcpyDeviceToHost);
+        long long md = 0;
+        for (int w = 0; w < issuers; ++w) md = h[2 * w + 1] > md ? h[2 * w + 1] : md;
+        printf("| %u | %u | %u | %d | %.1f |\n", c[0], c[1], c[2], issuers, double(md) / cnt);
+      }
   }
 
   printf("\n## M2: tcgen05.mma cta_group::1 kind::tf32 (K = 8)\n\n");
