@@ -56,6 +56,37 @@ def test_no_allocation_after_planning():
     assert torch.equal(net2.forward(x1), y1)
 
 
+def test_no_allocation_after_planning_other_networks():
+    """The same for the R(2+1)D-shaped network with its fused pairs and side-stream projections, and for the
+    S3D-shaped network with its parallel branches writing into channel slices."""
+    def dev(layers, specs):
+        return {sp.name: nets.ConvLayer(sp, layers[sp.name]["w"], layers[sp.name]["bias"], layers[sp.name]["mask"], 4, 4,
+                                        torch.bfloat16) for sp in specs}
+    stem, blocks, layers = netref.make_r2plus1d_layers(3, 0.4)
+    specs = list(stem)
+    for blk in blocks:
+        specs += list(blk.convs) + ([blk.shortcut] if blk.shortcut is not None else [])
+    plan_s, layers_s = netref.make_s3d_layers(5, 1 / 2.1)
+    specs_s = synth.s3d_convs(plan_s)
+    cases = [
+        (lambda: nets.R2Plus1DNet(stem, blocks, dev(layers, specs), fuse_residual=True, fuse_pairs=True),
+         oracle.bf16_round(synth.make_input(3, (4, 16, 112, 112, 3)))),
+        (lambda: nets.S3DNet(plan_s, dev(layers_s, specs_s)), oracle.bf16_round(synth.make_input(5, (2, 16, 224, 224, 3)))),
+    ]
+    for make, x in cases:
+        net = make()
+        xd = nets.to_device(x)
+        with rt3d.planning():
+            net.forward(xd)
+        torch.cuda.synchronize()
+        allocs = rt3d.rt3d_alloc_count()
+        y = net.forward(xd).clone()
+        torch.cuda.synchronize()
+        assert rt3d.rt3d_alloc_count() == allocs, "a compute call allocated after planning"
+        assert rt3d.rt3d_last_device_status() == rt3d.OK
+        assert torch.equal(make().forward(xd), y)                 # same bits as an unplanned network
+
+
 def test_bounded_wait_times_out_and_the_library_recovers():
     spec = synth.ConvSpec("to", 64, 64, (3, 3, 3), (1, 1, 1), (1, 1, 1), True)
     L = synth.make_layer(spec, 9, 4, 4, 4, "bernoulli", 0.5)
