@@ -332,3 +332,30 @@ def test_sparsity_sweep_full_batch_one_variant_per_group_size(sweep_input, g_m, 
     y = nets.to_numpy(lay(xd), 256)
     ref = oracle.conv3d(x, L["w"], L["mask"], L["bias"], sp.stride, sp.pad, True, round_bf16=True)
     assert rel_err(y, ref) <= TOL
+
+
+# ------------------------------------------------------------------------------ CUDA-graph replay
+@pytest.mark.parametrize("which", ["c3d", "r2plus1d", "s3d"])
+def test_graph_replay_matches_eager(which, request):
+    """The forward passes are timed as captured CUDA graphs (dependent launches, side streams as parallel branches):
+    a replay must give the bits of the eager pass, also after new clips were copied into the captured input buffer."""
+    if which == "c3d":
+        plan, layers, specs, x2, rec, final = request.getfixturevalue("c3d")
+        make = lambda: nets.C3DNet(plan, device_layers(layers, specs), fuse_pool=True)
+    elif which == "r2plus1d":
+        stem, blocks, layers, specs, x2, rec, final = request.getfixturevalue("r21d")
+        make = lambda: nets.R2Plus1DNet(stem, blocks, device_layers(layers, specs), fuse_residual=True, fuse_pairs=True)
+    else:
+        plan, layers, x2, rec, final = request.getfixturevalue("s3d")
+        make = lambda: nets.S3DNet(plan, device_layers(layers, synth.s3d_convs(plan)))
+    xa = nets.to_device(x2)
+    xb = nets.to_device(oracle.bf16_round(synth.make_input(77, x2.shape)))
+    eager = make()
+    ya, yb = eager.forward(xa).clone(), eager.forward(xb).clone()
+    g = nets.GraphedForward(make(), xa.clone())
+    assert torch.equal(g().clone(), ya)
+    g.x.copy_(xb)
+    assert torch.equal(g().clone(), yb)
+    g.x.copy_(xa)
+    assert torch.equal(g().clone(), ya)
+    assert rt3d.rt3d_last_device_status() == rt3d.OK
