@@ -247,7 +247,11 @@ const SmallCLayout* get_smallc_layout(rt3d_packed* p, int sh, int sw) {
     L.pair_off[i] = pos[i].first;
     slot[size_t(pos[i].second)] = int(i);
   }
-  if (pos.size() % 2) L.pair_off[pos.size()] = L.pair_off[pos.size() - 1] + 16;   // unused half: zero weights
+  // An odd count leaves the last pair's second K half without a location: zero weights, read through the SAME window
+  // as the first half.  (A window 16 bytes further on runs, for the tile's last voxel, past the end of the staged
+  // image into shared memory that no load ever wrote; a NaN or infinity there times zero is a NaN in that voxel's
+  // accumulators, which a following max-pool silently drops: rare, run-to-run different outputs.)
+  if (pos.size() % 2) L.pair_off[pos.size()] = L.pair_off[pos.size() - 1];
   const uint16_t* tiles = reinterpret_cast<const uint16_t*>(p->tiles.data());
   for (int pr = 0; pr < p->P; ++pr)
     for (int q = 0; q < p->Q; ++q)
