@@ -390,7 +390,7 @@ def rt3d_alloc_count() -> int:
     return int(_lib.rt3d_alloc_count())
 
 
-DEBUG_WAIT_CYCLES, DEBUG_DROP_LAST_LOAD, DEBUG_T_GROUPS = 1, 2, 3
+DEBUG_WAIT_CYCLES, DEBUG_DROP_LAST_LOAD, DEBUG_T_GROUPS, DEBUG_POISON = 1, 2, 3, 4
 
 
 def rt3d_debug_get(what: int) -> int:

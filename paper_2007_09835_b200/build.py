@@ -13,7 +13,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "librt3d.so")
-SOURCES = ["api.cu", "pack.cpp", "simt_kernels.cu", "umma_conv.cu", "umma_conv_pair.cu", "umma_conv_halo.cu", "umma_conv_st.cu", "umma_conv_sub.cu", "umma_smallc.cu", "reweight.cu"]
+SOURCES = ["api.cu", "pack.cpp", "simt_kernels.cu", "umma_conv.cu", "umma_conv_pair.cu", "umma_conv_halo.cu", "umma_conv_st.cu", "umma_conv_sub.cu", "umma_smallc.cu", "reweight.cu", "debug_poison.cu"]
 HEADERS = ["kernels.h", "rt3d_internal.h", "umma_common.cuh", "umma_pair.cuh", "pdl.cuh", "tile_consts.h"]
 MICROBENCH = os.path.join(HERE, "rt3d_microbench")       # stand-alone instruction-rate microbenchmarks
 

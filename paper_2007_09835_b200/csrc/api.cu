@@ -1339,6 +1339,14 @@ rt3d_status rt3d_debug_set(int what, long long value) {
   if (what == RT3D_DEBUG_WAIT_CYCLES) { if (value < 0) return RT3D_ERR_INVALID_ARG; g_debug_wait_cycles.store(value); return RT3D_OK; }
   if (what == RT3D_DEBUG_DROP_LAST_LOAD) { g_debug_drop_last_load.store(value != 0); return RT3D_OK; }
   if (what == RT3D_DEBUG_T_GROUPS) { g_ts_enabled.store(value != 0); return RT3D_OK; }
+  if (what == RT3D_DEBUG_POISON) {
+    DeviceState* d = nullptr;
+    rt3d_status s = get_device_state(&d);
+    if (s != RT3D_OK) return s;
+    if (d->cc_major != 10) return RT3D_ERR_UNSUPPORTED;
+    if (launch_debug_poison(uint32_t(value), d->sm_count, d->sched + 8, nullptr) != cudaSuccess) return RT3D_ERR_CUDA;
+    return cudaDeviceSynchronize() == cudaSuccess ? RT3D_OK : RT3D_ERR_CUDA;
+  }
   return RT3D_ERR_INVALID_ARG;
 }
 

@@ -187,6 +187,9 @@ cudaError_t launch_conv_umma_smallc(const SmallCArgs& a, const void* xmap, const
                                     cudaStream_t stream);
 size_t smallc_smem_bytes(int n_pairs, int n_pad, int stage_bytes);
 
+// Test hook (debug_poison.cu): every SM's shared memory and tensor memory filled with `pattern`; `sink`: a device int.
+cudaError_t launch_debug_poison(uint32_t pattern, int sm_count, int* sink, cudaStream_t stream);
+
 // Shared memory the tcgen05 kernel needs for a bundle width (for the host-side eligibility check).
 size_t umma_smem_bytes(int n_tile, int n_bundles);
 

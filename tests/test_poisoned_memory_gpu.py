@@ -1,0 +1,114 @@
+"""GPU parity with every SM's shared memory and tensor memory poisoned before each call.
+
+The kernels multiply padding (unused K halves, channels and rows beyond the real extents) by zeros, which is exact
+only while the padding is finite.  A read of shared memory that no load of the kernel itself wrote sees what an
+earlier kernel left there: almost always finite, so the result is right and the fault invisible.  The test hook
+RT3D_DEBUG_POISON fills shared and tensor memory with NaN (or infinity) patterns first; after it, such a read gives
+NaNs in the output, or, behind a max-pool that drops NaNs, a wrong maximum.  (This is how the small-C_in kernel's
+window past the staged image would have been caught; it showed only as 2 % of C3D batch-1 replays differing.)
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import rt3d_synth as synth
+import paper_2007_09835_b200 as rt3d
+from paper_2007_09835_b200 import nets
+
+from test_random_shapes_gpu import draw_conv_case
+
+pytestmark = pytest.mark.gpu
+
+NAN2, INF2 = 0x7FC07FC0, 0x7F807F80          # two bf16 NaNs / two bf16 infinities per 32-bit word (fp32: NaN too)
+
+
+def poison(pattern):
+    torch.cuda.synchronize()
+    rt3d.rt3d_debug_set(rt3d.DEBUG_POISON, pattern)
+
+
+FIRST_LAYERS = [
+    # cin, cout, k, stride, pad, (n,t,h,w), pool
+    (3, 64, (3, 3, 3), (1, 1, 1), (1, 1, 1), (1, 4, 32, 24), (1, 2, 2)),     # 27 locations: odd, one unused K half
+    (3, 64, (3, 3, 3), (1, 1, 1), (1, 1, 1), (1, 4, 32, 24), (1, 1, 1)),
+    (3, 45, (1, 7, 7), (1, 2, 2), (0, 3, 3), (2, 3, 56, 40), (1, 1, 1)),     # 49 locations, four stride phases
+    (8, 32, (3, 5, 3), (1, 3, 1), (1, 2, 1), (1, 3, 50, 12), (1, 1, 1)),
+    (1, 16, (3, 1, 1), (1, 1, 1), (1, 0, 0), (1, 6, 9, 9), (1, 1, 1)),
+]
+
+
+@pytest.mark.parametrize("pattern", [NAN2, INF2])
+@pytest.mark.parametrize("case", FIRST_LAYERS)
+def test_first_layer_kernel_after_poison(case, pattern):
+    cin, cout, k, stride, pad, (n, t, h, w), pool = case
+    spec = synth.ConvSpec("p", cin, cout, k, stride, pad, True)
+    L = synth.make_layer(spec, 15, cin + cout, 4, 4, "bernoulli", 1.0 if k == (3, 3, 3) else 0.5)
+    x = synth.make_input(1500 + cin, (n, t, h, w, cin))
+    conv = oracle.bf16_round(oracle.conv3d(x, L["w"], L["mask"], L["bias"], stride, pad, True, round_bf16=True))
+    ref = oracle.maxpool3d(conv, pool, pool) if pool != (1, 1, 1) else conv
+    lay = nets.ConvLayer(spec, L["w"], L["bias"], L["mask"], 4, 4, torch.bfloat16)
+    xd = nets.to_device(x)
+    y = torch.zeros(ref.shape[:4] + (nets.pitch_for(cout, torch.bfloat16),), dtype=torch.bfloat16, device="cuda")
+    lay.fused(xd, y, pool=pool)                   # first use: uploads
+    for _ in range(3):
+        poison(pattern)
+        lay.fused(xd, y, pool=pool, x_pad_zero=True)
+        torch.cuda.synchronize()
+        assert rt3d.rt3d_last_plan()["kernel"] == 3
+        got = nets.to_numpy(y, cout)
+        assert np.isfinite(got).all()
+        assert np.abs(got - ref).max() <= 2e-2 * np.abs(ref).max()
+
+
+@pytest.mark.parametrize("case", range(32))
+def test_random_conv_layers_after_poison(case):
+    rng = np.random.default_rng(81000 + case)
+    cin, cout, k, stride, pad, (n, t, h, w), (g_m, g_n), kind, dens, dense, relu, algo, use_res, pool = draw_conv_case(rng)
+    spec = synth.ConvSpec("r", cin, cout, k, stride, pad, relu)
+    L = synth.make_layer(spec, 33, case, g_m, g_n, kind, None if kind == "none" else dens)
+    x = synth.make_input(3300 + case, (n, t, h, w, cin))
+    lin = oracle.conv3d(x, L["w"], None if dense else L["mask"], L["bias"], stride, pad, False, round_bf16=False)
+    act = oracle.bf16_round((np.maximum(lin, 0) if relu else lin).astype(np.float32))
+    pool = tuple(p if d >= p else 1 for p, d in zip(pool, act.shape[1:4]))
+    ref = oracle.maxpool3d(act, pool, pool) if pool != (1, 1, 1) else act
+    lay = nets.ConvLayer(spec, L["w"], L["bias"], L["mask"], g_m, g_n, torch.bfloat16, dense=dense)
+    xd = nets.to_device(x)
+    y = torch.zeros(ref.shape[:4] + (nets.pitch_for(cout, torch.bfloat16),), dtype=torch.bfloat16, device="cuda")
+    try:
+        lay.fused(xd, y, pool=pool, algo=algo)
+    except rt3d.Rt3dError as e:
+        assert e.status == rt3d.ERR_UNSUPPORTED, e
+        pytest.skip(f"declined: {e}")
+    for pattern in (NAN2, INF2):
+        poison(pattern)
+        lay.fused(xd, y, pool=pool, algo=algo)
+        torch.cuda.synchronize()
+        assert rt3d.rt3d_last_device_status() == rt3d.OK
+        got = nets.to_numpy(y, cout)
+        assert np.isfinite(got).all(), rt3d.rt3d_last_plan()
+        assert np.abs(got - ref).max() <= 2e-2 * np.abs(ref).max(), rt3d.rt3d_last_plan()
+
+
+def test_factorised_pair_after_poison():
+    sp_s = synth.ConvSpec("s", 64, 144, (1, 3, 3), (1, 1, 1), (0, 1, 1), True)
+    sp_t = synth.ConvSpec("t", 144, 64, (3, 1, 1), (1, 1, 1), (1, 0, 0), True)
+    Ls = synth.make_layer(sp_s, 43, 1, 4, 4, "bernoulli", 0.4)
+    Lt = synth.make_layer(sp_t, 44, 2, 4, 4, "bernoulli", 0.4)
+    x = synth.make_input(4400, (2, 6, 20, 12, 64))
+    mid = oracle.bf16_round(oracle.conv3d(x, Ls["w"], Ls["mask"], Ls["bias"], (1, 1, 1), (0, 1, 1), True, round_bf16=True))
+    ref = oracle.conv3d(mid, Lt["w"], Lt["mask"], Lt["bias"], (1, 1, 1), (1, 0, 0), True, round_bf16=True)
+    ls = nets.ConvLayer(sp_s, Ls["w"], Ls["bias"], Ls["mask"], 4, 4, torch.bfloat16)
+    lt = nets.ConvLayer(sp_t, Lt["w"], Lt["bias"], Lt["mask"], 4, 4, torch.bfloat16)
+    xd = nets.to_device(x)
+    y = torch.zeros((2, 6, 20, 12, 64), dtype=torch.bfloat16, device="cuda")
+    for pattern in (0, NAN2, INF2):
+        if pattern:
+            poison(pattern)
+        rt3d.rt3d_conv2plus1d_fused(rt3d.tensor_desc(xd, 64), ls.packed, ls.bias, (0, 1, 1), True, lt.packed, lt.bias,
+                                    (1, 0, 0), True, rt3d.tensor_desc(y, 64))
+        torch.cuda.synchronize()
+        assert rt3d.rt3d_last_device_status() == rt3d.OK
+        got = nets.to_numpy(y, 64)
+        assert np.isfinite(got).all()
+        assert np.abs(got - ref).max() <= 2e-2 * np.abs(ref).max()
