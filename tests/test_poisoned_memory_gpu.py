@@ -112,3 +112,52 @@ def test_factorised_pair_after_poison():
         got = nets.to_numpy(y, 64)
         assert np.isfinite(got).all()
         assert np.abs(got - ref).max() <= 2e-2 * np.abs(ref).max()
+
+
+@pytest.mark.parametrize("which,batch", [("c3d", 1), ("c3d", 16), ("r2plus1d", 2), ("s3d", 1)])
+def test_forward_passes_with_poison_before_every_launch(which, batch, monkeypatch):
+    """Every kernel of a forward pass launched right after a poisoning: the output must have the bits of an
+    ordinary pass (no kernel depends on what its predecessors left in shared or tensor memory)."""
+    import netref
+    from paper_2007_09835_b200 import binding as B
+
+    def dev(layers, specs):
+        return {sp.name: nets.ConvLayer(sp, layers[sp.name]["w"], layers[sp.name]["bias"], layers[sp.name]["mask"], 4, 4,
+                                        torch.bfloat16) for sp in specs}
+    if which == "c3d":
+        plan, layers = netref.make_c3d_layers(2, 1 / 3.6)
+        net = nets.C3DNet(plan, dev(layers, [op for op in plan if isinstance(op, synth.ConvSpec)]), fuse_pool=True)
+        shape = (batch, 16, 112, 112, 3)
+    elif which == "r2plus1d":
+        stem, blocks, layers = netref.make_r2plus1d_layers(3, 0.4)
+        specs = list(stem)
+        for blk in blocks:
+            specs += list(blk.convs) + ([blk.shortcut] if blk.shortcut is not None else [])
+        net = nets.R2Plus1DNet(stem, blocks, dev(layers, specs), fuse_residual=True, fuse_pairs=True)
+        shape = (batch, 16, 112, 112, 3)
+    else:
+        plan, layers = netref.make_s3d_layers(5, 1 / 2.1)
+        net = nets.S3DNet(plan, dev(layers, synth.s3d_convs(plan)), parallel_branches=False)
+        shape = (batch, 16, 224, 224, 3)
+    x = nets.to_device(oracle.bf16_round(synth.make_input(9, shape)))
+    y0 = net.forward(x).clone()
+    torch.cuda.synchronize()
+    state = {"pattern": NAN2, "launches": 0}
+
+    def poisoned(orig):
+        def call(*a, **k):
+            poison(state["pattern"])
+            state["launches"] += 1
+            return orig(*a, **k)
+        return call
+    for name in ("rt3d_conv3d_sparse", "rt3d_conv3d_dense", "rt3d_conv3d_sparse_fused", "rt3d_conv2plus1d_fused",
+                 "rt3d_maxpool3d", "rt3d_add_relu"):
+        monkeypatch.setattr(B, name, poisoned(getattr(B, name)))
+    for pattern in (NAN2, INF2):
+        state["pattern"] = pattern
+        y = net.forward(x).clone()
+        torch.cuda.synchronize()
+        assert torch.isfinite(y.float()).all()
+        assert torch.equal(y, y0)
+    assert state["launches"] >= 18
+    assert rt3d.rt3d_last_device_status() == rt3d.OK
