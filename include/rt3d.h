@@ -379,7 +379,8 @@ void rt3d_plan_end(void);
  * RT3D_DEBUG_POISON: runs, on the default stream, a kernel that fills the shared memory and the tensor memory of
  * every SM with the 32-bit pattern `value` (e.g. 0x7FC07FC0: two bf16 NaNs) and waits for it: a kernel launched next
  * that reads shared or tensor memory it did not write itself (padding multiplied by zero weights, say) then
- * produces NaNs instead of depending silently on what ran before it.  Device work only; nothing else changes. */
+ * produces NaNs instead of depending silently on what ran before it.  The partial-tile scratch of every handle's
+ * K splits on the device is set to all ones (NaNs) as well.  Device work only; nothing else changes. */
 enum { RT3D_DEBUG_WAIT_CYCLES = 1, RT3D_DEBUG_DROP_LAST_LOAD = 2, RT3D_DEBUG_T_GROUPS = 3, RT3D_DEBUG_POISON = 4 };
 rt3d_status rt3d_debug_set(int what, long long value);
 /* Diagnostics.  RT3D_DEBUG_WAIT_SITE: after a synchronisation of the device, the number of the wait inside a

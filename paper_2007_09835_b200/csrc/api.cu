@@ -1345,7 +1345,14 @@ rt3d_status rt3d_debug_set(int what, long long value) {
     if (s != RT3D_OK) return s;
     if (d->cc_major != 10) return RT3D_ERR_UNSUPPORTED;
     if (launch_debug_poison(uint32_t(value), d->sm_count, d->sched + 8, nullptr) != cudaSuccess) return RT3D_ERR_CUDA;
-    return cudaDeviceSynchronize() == cudaSuccess ? RT3D_OK : RT3D_ERR_CUDA;
+    if (cudaDeviceSynchronize() != cudaSuccess) return RT3D_ERR_CUDA;
+    // the K splits' partial tiles in global memory too (all ones: NaNs as fp32); their counters and flags stay zero
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return RT3D_ERR_CUDA;
+    std::lock_guard<std::mutex> reg(g_blobs_mu);
+    for (DeviceBlob* b : g_blobs)
+      if (b->device == dev && b->splitk && cudaMemset(b->splitk, 0xFF, b->splitk_bytes) != cudaSuccess) return RT3D_ERR_CUDA;
+    return RT3D_OK;
   }
   return RT3D_ERR_INVALID_ARG;
 }
