@@ -1,7 +1,8 @@
 """Tensors beyond 2^31 elements (outputs of 4.9 GB): index arithmetic, tensor-map extents and work-item counts at
 sizes the oracle cannot follow.  The batch is two seeded clips repeated, so every clip has a reference: the same
 layer run on the two clips alone (itself covered by the oracle tests); the first, middle and last clips of the
-large run must match it bit for bit (same tile shapes and summation order per clip).  Needs about 10 GB."""
+large run must match it (to 1e-2 of the largest value for the convolutions, whose grid may cut K differently at the
+larger size; bit for bit for pools and adds).  Needs about 10 GB."""
 import pytest
 import torch
 
@@ -46,8 +47,9 @@ def test_conv_outputs_beyond_2_31_elements(case):
     if pool == (1, 1, 1):
         assert y.numel() > 2**31
     assert float(y2.float().abs().max()) > 0
-    for i in picks(batch):
-        assert torch.equal(y[i], y2[i % 2]), i
+    scale = float(y2.float().abs().max())
+    for i in picks(batch):          # equal up to the summation order of a K split the larger grid may choose
+        assert float((y[i].float() - y2[i % 2].float()).abs().max()) <= 1e-2 * scale, i
     del x, y
     torch.cuda.empty_cache()
 
