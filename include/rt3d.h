@@ -22,7 +22,11 @@
  *     after that kernel has completed (environment RT3D_PDL=0 turns the attribute off).
  *   - Argument errors are detected on the host before anything is launched.
  *   - Activation layout: NDHWC = [n][t][h][w][c] with a channel pitch c_stride >= c
- *     (elements between consecutive voxels).  Weight layout handed to the packers:
+ *     (elements between consecutive voxels).  An output tensor's padding channels c .. c_stride-1 are left as
+ *     they are, except those that share the last 16-byte unit of a voxel row with real channels (bf16:
+ *     channels c .. 8*ceil(c/8)-1): the tensor-core kernels' bulk stores move whole 16-byte units and write
+ *     zeros there.  (A channel slice of a wider tensor that is followed by another slice starts that slice
+ *     on a 16-byte boundary anyway, so only a row's last slice can have such channels.)  Weight layout handed to the packers:
  *     [M][N][Kt][Kh][Kw], M filters, N input channels (Section 3; the paper's kernel depth
  *     K_d is the temporal extent Kt).  Kernel location index kpos = (kt*Kh + kh)*Kw + kw.
  *   - Convolution is cross-correlation with zero padding, no dilation; output extent

@@ -478,3 +478,25 @@ def test_cost_model_counts_kept_macs():
     assert dense == spec.dense_macs(1, 8, 28, 28)
     assert kept * 27 == dense * 14
     assert nbytes == (6272 * 16 + 6272 * 32) * 4 + 448 * 16 * 4 + 448 * 2 + 33 * 4 + 32 * 4
+
+
+@pytest.mark.parametrize("algo", ["auto", "pair", "simt"])
+def test_padding_channels_of_the_output(algo):
+    """300 output channels at a pitch of 320: the padding channels 304..319 must be left alone by every kernel; the four
+    padding channels that share the last 16-byte unit of a row with channels 296..299 are either left alone (CUDA-core
+    kernel, per-element stores) or written as zeros (bulk stores of the tensor-core kernels move whole units)."""
+    spec = synth.ConvSpec("pad", 16, 300, (1, 3, 2), (1, 2, 1), (0, 1, 1), True)
+    L = synth.make_layer(spec, 51, 58, 8, 8, "bernoulli", 0.2)
+    x = synth.make_input(6158, (8, 4, 32, 9, 16))
+    ref = oracle.conv3d(x, L["w"], L["mask"], L["bias"], spec.stride, spec.pad, True, round_bf16=True)
+    lay = nets.ConvLayer(spec, L["w"], L["bias"], L["mask"], 8, 8, torch.bfloat16)
+    xd = nets.to_device(x)
+    y = torch.full(tuple(lay.out_shape(xd)[:4]) + (320,), 9.0, dtype=torch.bfloat16, device="cuda")
+    lay(xd, y, algo={"auto": rt3d.ALGO_AUTO, "pair": rt3d.ALGO_UMMA_PAIR, "simt": rt3d.ALGO_SIMT}[algo])
+    assert rt3d.rt3d_last_device_status() == rt3d.OK
+    check(nets.to_numpy(y, 300), ref, torch.bfloat16, f"padding {algo}")
+    assert (y[..., 304:] == 9.0).all()
+    unit = y[..., 300:304]
+    assert ((unit == 9.0) | (unit == 0.0)).all()
+    if algo == "simt":
+        assert (unit == 9.0).all()
