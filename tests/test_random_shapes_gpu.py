@@ -151,3 +151,42 @@ def test_random_max_pools_bit_exact(case):
     torch.cuda.synchronize()
     got = nets.to_numpy(y, c)
     assert got.shape == ref.shape and np.array_equal(got, ref)
+
+
+@pytest.mark.parametrize("case", range(24))
+def test_random_channel_slices_against_oracle(case):
+    """Input and output as channel slices of wider tensors (the way an Inception block's branches read a shared input
+    and write into their part of the concatenation): the result matches the oracle and the neighbouring channels of
+    the output tensor keep their contents."""
+    from paper_2007_09835_b200 import binding as B
+    rng = np.random.default_rng(80000 + case)
+    cin = int(rng.choice([8, 16, 24, 64, 96, 128, 192, 256]))
+    cout = int(rng.choice([16, 32, 48, 64, 96, 128, 160, 192, 256, 384]))
+    k = tuple(int(rng.choice([1, 1, 3, 3])) for _ in range(3))
+    stride = tuple(int(rng.choice([1, 1, 2])) for _ in range(3))
+    pad = tuple(q // 2 for q in k)
+    n, t = int(rng.integers(1, 5)), int(rng.integers(1, 9))
+    h, w = int(rng.integers(4, 40)), int(rng.integers(4, 40))
+    xl, xr = 8 * int(rng.integers(0, 4)), 8 * int(rng.integers(0, 4))
+    yl, yr = 8 * int(rng.integers(0, 5)), 8 * int(rng.integers(0, 5))
+    relu = bool(rng.random() < 0.7)
+    algo = [rt3d.ALGO_AUTO, rt3d.ALGO_AUTO, rt3d.ALGO_UMMA, rt3d.ALGO_UMMA_PAIR, rt3d.ALGO_SIMT][int(rng.integers(0, 5))]
+    spec = synth.ConvSpec("s", cin, cout, k, stride, pad, relu)
+    L = synth.make_layer(spec, 95, case, 4, 4, "bernoulli", float(rng.choice([0.2, 0.5])))
+    x = synth.make_input(9500 + case, (n, t, h, w, cin))
+    ref = oracle.conv3d(x, L["w"], L["mask"], L["bias"], stride, pad, relu, round_bf16=True)
+    lay = nets.ConvLayer(spec, L["w"], L["bias"], L["mask"], 4, 4, torch.bfloat16)
+    xw = torch.full((n, t, h, w, xl + cin + xr), 77.0, dtype=torch.bfloat16, device="cuda")    # junk beside the input slice
+    xw[..., xl:xl + cin] = torch.from_numpy(x).to(torch.bfloat16).cuda()
+    yw = torch.full(tuple(ref.shape[:4]) + (yl + cout + yr,), 9.0, dtype=torch.bfloat16, device="cuda")
+    try:
+        lay.run_desc(B.channel_slice_desc(xw, xl, cin), B.channel_slice_desc(yw, yl, cout), algo=algo)
+    except rt3d.Rt3dError as e:
+        assert e.status == rt3d.ERR_UNSUPPORTED, e
+        lay.run_desc(B.channel_slice_desc(xw, xl, cin), B.channel_slice_desc(yw, yl, cout))
+    torch.cuda.synchronize()
+    assert rt3d.rt3d_last_device_status() == rt3d.OK
+    got = yw[..., yl:yl + cout].float().cpu().numpy()
+    assert np.isfinite(got).all()
+    assert np.abs(got - ref).max() <= TOL * np.abs(ref).max(), rt3d.rt3d_last_plan()
+    assert (yw[..., :yl] == 9.0).all() and (yw[..., yl + cout:] == 9.0).all()
